@@ -1,0 +1,229 @@
+/*
+ * tsr.h -- C ABI of libtsr: the per-step optimizer hot path of TSR-Adam
+ * (two-sided low-rank Adam) on one NVIDIA B200 (sm_100a).
+ *
+ * For every m x n weight block W with local gradient G the method keeps two
+ * orthonormal bases U (m x r) and V (n x r) and Adam moments M, Vm of the
+ * r x r core (Algorithm 1 of the paper; Sections 3.3-3.5):
+ *
+ *     C  = U^T G V                                   core projection
+ *     M  = b1 M + (1-b1) C ;  Vm = b2 Vm + (1-b2) C o C
+ *     D  = (M / (1-b1^t)) / (sqrt(Vm / (1-b2^t)) + eps)
+ *     W  = W - lr (scale * U D V^T + weight_decay * W)
+ *
+ * and, every K steps, refreshes (U, V) from the current gradient by a
+ * randomized SVD with k = r + p sketch columns and q power iterations.
+ *
+ * General rules
+ *   - Every pointer in tsr_mat_ptrs and every `workspace` pointer is a DEVICE
+ *     pointer owned by the caller; the library never frees or reallocates it.
+ *     Descriptor / index / hyper-parameter arguments are HOST pointers.  The
+ *     only calls that take HOST data buffers are the *_host entry points.
+ *   - All matrices are row-major.  G and W carry explicit leading dimensions
+ *     (in elements); U is m x r, V is n x r, M / Vm / C are r x r, all dense
+ *     FP32.  Buffers of different roles must not alias.
+ *   - G is read-only.  W, U, V, M, Vm, C are updated in place.
+ *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*,
+ *     NULL = the legacy default stream) unless stated otherwise, and calls on
+ *     one context must be issued from one host thread at a time.
+ *   - Every call returns a tsr_status.  Argument errors are detected on the
+ *     host before anything is launched and leave all buffers untouched.
+ *     Conditions detected on the device (a rank-deficient sketch, an
+ *     eigen-solver that ran out of sweeps, a non-finite value) are recorded per
+ *     block and read back with tsr_poll_status; no kernel traps or spins
+ *     without a bound.
+ *   - There is no CPU fallback: without a CUDA device every compute call
+ *     returns TSR_ERR_CUDA.
+ *   - Gradients in BF16 with 16-byte aligned pointers and row pitches take the
+ *     tensor-core path (tcgen05 MMAs fed by TMA, FP32 accumulation; U, V, the
+ *     intermediate products and D are rounded to BF16 as MMA operands).
+ *     FP32 gradients, or buffers that miss the alignment rule, take an
+ *     all-FP32 CUDA-core path.
+ */
+#ifndef TSR_H_
+#define TSR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(_WIN32)
+#define TSR_API
+#else
+#define TSR_API __attribute__((visibility("default")))
+#endif
+
+typedef struct tsr_ctx tsr_ctx; /* opaque plan: shapes, bound pointers, device tables */
+
+typedef enum {
+    TSR_OK = 0,
+    TSR_ERR_INVALID_ARG = 1,    /* null pointer, bad index, bad enum                      */
+    TSR_ERR_SHAPE = 2,          /* non-positive size, ld < cols, r + p > min(m, n)        */
+    TSR_ERR_ALIGNMENT = 3,      /* a pointer that must be 16-byte aligned is not          */
+    TSR_ERR_WORKSPACE = 4,      /* workspace missing or too small                         */
+    TSR_ERR_CUDA = 5,           /* a CUDA runtime / driver call failed, or no device      */
+    TSR_ERR_UNSUPPORTED = 6,    /* dtype or option not implemented                        */
+    TSR_ERR_NOT_CONVERGED = 7,  /* device: eigen-solver hit its sweep limit               */
+    TSR_ERR_RANK_DEFICIENT = 8, /* device: a sketch lost rank; bases are still orthonormal only approximately */
+    TSR_ERR_NONFINITE = 9,      /* device: NaN / Inf met in a refresh                     */
+    TSR_ERR_TIMEOUT = 10,       /* device: a bounded wait ran out                         */
+    TSR_ERR_NOT_BOUND = 11      /* compute call before tsr_bind                           */
+} tsr_status;
+
+typedef enum { TSR_F32 = 0, TSR_BF16 = 1 } tsr_dtype;
+
+/* Update rule in core space: Algorithm 1 (Adam) or Algorithm 2 (momentum SGD, D = M,
+ * no second moment, no weight decay, no bias correction; beta1 is its momentum). */
+typedef enum { TSR_RULE_ADAM = 0, TSR_RULE_SGD = 1 } tsr_rule;
+
+/* One matrix block.  Embedding blocks are ordinary blocks with their own (r, K)
+ * (Section 3.6); is_embedding only labels them for tsr_embed_step. */
+typedef struct {
+    int64_t m, n;         /* rows, columns of G and W                                   */
+    int64_t ldg, ldw;     /* leading dimensions of G and W in elements (>= n)           */
+    int32_t r;            /* rank of the bases                                          */
+    int32_t p;            /* oversampling: sketches have k = r + p columns, k <= min(m,n) */
+    int32_t q;            /* power iterations in the refresh (>= 0)                     */
+    int32_t K;            /* refresh when step % K == 0; K <= 0 disables in-loop refresh */
+    int32_t g_dtype;      /* tsr_dtype of G                                             */
+    int32_t w_dtype;      /* tsr_dtype of W; only TSR_F32 is implemented                */
+    int32_t is_embedding; /* 0 / 1                                                      */
+    int32_t reserved;     /* must be 0                                                  */
+} tsr_mat_desc;
+
+typedef struct {
+    const void *G; /* m x n (ldg), g_dtype                                              */
+    void *W;       /* m x n (ldw), FP32, updated in place                               */
+    float *U;      /* m x r                                                             */
+    float *V;      /* n x r                                                             */
+    float *M;      /* r x r first moment                                                */
+    float *Vm;     /* r x r second moment (unused by TSR_RULE_SGD, may then be NULL)    */
+    float *C;      /* r x r core, written by every projection: the tensor a data-parallel
+                      job would all-reduce (Algorithm 1, "C_bar <- AR(C)")              */
+} tsr_mat_ptrs;
+
+typedef struct {
+    float lr, beta1, beta2, eps, weight_decay;
+    float scale;   /* multiplies the lifted update U D V^T only; 1 = Algorithm 1 as printed */
+    int64_t step;  /* t >= 1: global step counter used for bias correction and refresh schedule */
+    int32_t rule;  /* tsr_rule                                                          */
+    int32_t reserved;
+} tsr_hyper;
+
+/* ---- library / context management (host only) ------------------------------------------- */
+
+TSR_API int tsr_version(void);
+TSR_API const char *tsr_status_string(tsr_status s);
+/* Text of the last error recorded on ctx (empty string if none); valid until the next call. */
+TSR_API const char *tsr_last_error(const tsr_ctx *ctx);
+
+/* Validates `count` descriptors and builds the plan.  descs is copied.  Returns
+ * TSR_ERR_SHAPE / TSR_ERR_UNSUPPORTED / TSR_ERR_INVALID_ARG and sets *ctx = NULL on failure. */
+TSR_API tsr_status tsr_create(tsr_ctx **ctx, const tsr_mat_desc *descs, int32_t count);
+TSR_API tsr_status tsr_destroy(tsr_ctx *ctx);
+
+/* Bytes of device scratch the context needs.  step_bytes covers projection, core update and
+ * back-projection (BF16 operand copies of U and V, the m x r intermediates, device tables);
+ * refresh_bytes covers one refresh of all blocks at once.  tsr_bind wants a single buffer of
+ * step_bytes + refresh_bytes. */
+TSR_API tsr_status tsr_workspace_bytes(const tsr_ctx *ctx, size_t *step_bytes, size_t *refresh_bytes);
+
+/* Attaches the caller's device buffers and the scratch buffer (256-byte aligned), encodes the
+ * TMA descriptors and uploads the device tables.  Synchronous; may be called again to re-point
+ * the context.  The contents of U, V are not read here: call tsr_init_subspace[_grouped] or,
+ * after writing U and V yourself, tsr_bases_changed. */
+TSR_API tsr_status tsr_bind(tsr_ctx *ctx, const tsr_mat_ptrs *ptrs, int32_t count, void *workspace,
+                            size_t workspace_bytes);
+
+/* Tells the library that the caller overwrote U and/or V of the listed blocks (idx = NULL: all):
+ * rebuilds the BF16 operand copies the tensor-core path keeps in the workspace. */
+TSR_API tsr_status tsr_bases_changed(tsr_ctx *ctx, const int32_t *idx, int32_t count, void *stream);
+
+/* ---- single-block calls (block index i of the plan) ------------------------------------- */
+
+/* Algorithm 1, initialisation: M <- 0, Vm <- 0 and (U, V) <- one refresh on the bound G.
+ * omega: device pointer to an n x (r+p) FP32 Gaussian test matrix, or NULL to draw it from
+ * `seed` with the library's counter-based generator (see tsr_generate_omega). */
+TSR_API tsr_status tsr_init_subspace(tsr_ctx *ctx, int32_t i, uint64_t seed, const float *omega, void *stream);
+
+/* Section 3.3: C <- U^T G V. */
+TSR_API tsr_status tsr_project_core(tsr_ctx *ctx, int32_t i, void *stream);
+
+/* Section 3.4: moments and normalised core D from the (possibly all-reduced) C in place in
+ * the C buffer's companion scratch; uses hyper->step for bias correction. */
+TSR_API tsr_status tsr_adam_core_step(tsr_ctx *ctx, int32_t i, const tsr_hyper *hyper, void *stream);
+
+/* Section 3.4: W <- W - lr (scale * U D V^T + weight_decay * W) with the D left by the last
+ * tsr_adam_core_step of this block.  The lifted update is never written to memory. */
+TSR_API tsr_status tsr_backproject_apply(tsr_ctx *ctx, int32_t i, const tsr_hyper *hyper, void *stream);
+
+/* Section 3.5: randomized-SVD refresh of (U, V) from the bound G; moments are left untouched. */
+TSR_API tsr_status tsr_rsvd_refresh(tsr_ctx *ctx, int32_t i, uint64_t seed, const float *omega, void *stream);
+
+/* Section 3.6: one full step of an embedding block on its own (r_emb, K_emb): refresh if
+ * hyper->step % K == 0, then project, core update, back-project and apply. */
+TSR_API tsr_status tsr_embed_step(tsr_ctx *ctx, int32_t i, const tsr_hyper *hyper, uint64_t seed, void *stream);
+
+/* ---- grouped calls: the same operations over a list of blocks in a few launches ---------- */
+/* idx: host array of `count` block indices, or NULL for all blocks of the plan (count ignored).
+ * omegas: host array with one device pointer per listed block, or NULL (library-drawn). */
+
+TSR_API tsr_status tsr_init_subspace_grouped(tsr_ctx *ctx, const int32_t *idx, int32_t count, uint64_t seed,
+                                             const float *const *omegas, void *stream);
+TSR_API tsr_status tsr_project_core_grouped(tsr_ctx *ctx, const int32_t *idx, int32_t count, void *stream);
+TSR_API tsr_status tsr_adam_core_step_grouped(tsr_ctx *ctx, const int32_t *idx, int32_t count,
+                                              const tsr_hyper *hyper, void *stream);
+TSR_API tsr_status tsr_backproject_apply_grouped(tsr_ctx *ctx, const int32_t *idx, int32_t count,
+                                                 const tsr_hyper *hyper, void *stream);
+TSR_API tsr_status tsr_rsvd_refresh_grouped(tsr_ctx *ctx, const int32_t *idx, int32_t count, uint64_t seed,
+                                            const float *const *omegas, void *stream);
+TSR_API tsr_status tsr_embed_step_grouped(tsr_ctx *ctx, const int32_t *idx, int32_t count,
+                                          const tsr_hyper *hyper, uint64_t seed, void *stream);
+
+/* One optimizer step of Algorithm 1 for every block: refresh the blocks whose K divides
+ * hyper->step (each block, embeddings included, on its own K), then project, update the core
+ * moments and apply.  fuse_adam != 0 runs the core update inside the projection kernel's
+ * epilogue (valid when no all-reduce of C is needed between the two); 0 runs the three stages
+ * as separate launches.  Both orders give the same result. */
+TSR_API tsr_status tsr_step_grouped(tsr_ctx *ctx, const tsr_hyper *hyper, uint64_t seed, int32_t fuse_adam,
+                                    void *stream);
+
+/* The same step driven from HOST memory: G_host[i] is a host pointer to block i's gradient,
+ * dense m x n in the block's g_dtype; each is copied into the bound device G buffer, the step
+ * runs, and the cores of all blocks are copied back, packed block after block (r*r floats
+ * each), into C_host (may be NULL).  Returns after the stream has been synchronised. */
+TSR_API tsr_status tsr_step_grouped_host(tsr_ctx *ctx, const void *const *G_host, float *C_host,
+                                         const tsr_hyper *hyper, uint64_t seed, int32_t fuse_adam, void *stream);
+
+/* ---- reporting -------------------------------------------------------------------------- */
+
+/* Section 3.2: bytes one worker would hand to the all-reduce in one step, summed over blocks:
+ * *core = sum r^2 * bytes_per_elem (every step); *sketch = sum (r+p)(m+n) * bytes_per_elem for
+ * the blocks that refresh at `step` (0 if none; step <= 0 counts a refresh of every block). */
+TSR_API tsr_status tsr_comm_bytes(const tsr_ctx *ctx, int64_t step, int32_t bytes_per_elem, uint64_t *core,
+                                  uint64_t *sketch);
+
+/* Optimizer-state elements (U, V, M, Vm) summed over blocks: sum (m+n) r + 2 r^2 (Table 2). */
+TSR_API tsr_status tsr_state_elems(const tsr_ctx *ctx, uint64_t *elems);
+
+/* Copies the per-block device status words (a tsr_status each; TSR_OK if nothing was detected
+ * since the last poll) into the HOST array per_block_status[count] and clears them.
+ * Synchronises `stream`. */
+TSR_API tsr_status tsr_poll_status(tsr_ctx *ctx, int32_t *per_block_status, int32_t count, void *stream);
+
+/* Fills the DEVICE buffer out (n x k FP32, row-major) with the N(0,1) matrix the library
+ * would draw for (seed, block i): entry e = row * k + col comes from a counter-based hash of
+ * (seed, i, e) followed by a Box-Muller transform, so the draw does not depend on the launch
+ * shape. */
+TSR_API tsr_status tsr_generate_omega(tsr_ctx *ctx, int32_t i, uint64_t seed, float *out, void *stream);
+
+/* 1 if block i takes the tensor-core path, 0 if the FP32 CUDA-core path, < 0 on a bad index. */
+TSR_API int32_t tsr_block_uses_tensor_cores(const tsr_ctx *ctx, int32_t i);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TSR_H_ */

@@ -1,0 +1,985 @@
+// Host side of libtsr: the C ABI declared in tsr.h, plan construction, workspace layout,
+// TMA descriptor encoding and the launch sequences of Algorithm 1 (project -> core update ->
+// lift and apply, with the randomized-SVD refresh of Section 3.5 when due).
+#include <math.h>
+#include <stdarg.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <algorithm>
+#include <new>
+
+#include "tsr_internal.h"
+
+using namespace tsr;
+
+namespace {
+
+enum Kind : int { KT = 0, KC, KCS, KP, KA, KY, KZ, NKIND };
+
+struct Block {
+    tsr_mat_desc d;
+    tsr_mat_ptrs p;
+    bool fast = false;        // tensor-core path
+    int k = 0;                // r + p
+    int64_t rl = 0, ml = 0, nl = 0;  // padded leading dimensions of BF16 operand copies
+    // step scratch
+    bf16 *Ub = nullptr, *Ubt = nullptr, *Vb = nullptr, *Vbt = nullptr, *Tt = nullptr, *Pb = nullptr;
+    bf16 *Db = nullptr, *Dbt = nullptr;
+    float *partial = nullptr;
+    int nsplit = 1, kb_per_split = 0;
+    float *T32 = nullptr, *P32 = nullptr, *D32 = nullptr;
+    // refresh scratch
+    bf16 *Gt = nullptr, *Xt = nullptr;
+    float *Om = nullptr;
+    float *buf[3] = {nullptr, nullptr, nullptr};
+    double *S = nullptr, *Xw = nullptr, *Wj = nullptr, *gpart = nullptr, *lam = nullptr;
+    float *Rinv = nullptr, *Wu = nullptr, *Wv = nullptr;
+    int tile_begin[NKIND], tile_end[NKIND];
+};
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct Arena {  // bump allocator over the caller's workspace; base == nullptr only measures
+    char *base;
+    size_t off;
+    void *take(size_t bytes)
+    {
+        off = (off + 255) & ~(size_t)255;
+        void *p = base ? (void *)(base + off) : nullptr;
+        off += bytes;
+        return p;
+    }
+};
+
+}  // namespace
+
+struct tsr_ctx {
+    std::vector<Block> blocks;
+    std::vector<int> order;                    // table order: blocks by descending m*n
+    std::vector<UmmaTile> tiles[NKIND];        // host copies
+    bool bound = false;
+    bool any_fast = false;
+    size_t step_bytes = 0, refresh_bytes = 0;
+    std::string err;
+    // device tables (inside the workspace)
+    UmmaProblem *d_probs[NKIND] = {};
+    UmmaTile *d_tiles[NKIND] = {};
+    CoreUpdateArgs *d_cu_all = nullptr, *d_cu_split = nullptr;
+    RefreshDev *d_refresh = nullptr;
+    int32_t *d_status = nullptr;
+    int32_t *d_list = nullptr;                 // scratch: block list of the running call
+    int32_t *d_list2 = nullptr;                // scratch: second list (split-K blocks, ...)
+    RowItem *d_items[4] = {};                  // [side*2 + 0]: 64-row slabs, [side*2 + 1]: Gram slabs
+    size_t items_cap[4] = {};
+    EncodeTiledFn encode = nullptr;
+    int max_r = 0, max_k = 0;
+};
+
+namespace {
+
+tsr_status fail(tsr_ctx *ctx, tsr_status s, const char *fmt, ...)
+{
+    if (ctx) {
+        char buf[512];
+        va_list ap;
+        va_start(ap, fmt);
+        vsnprintf(buf, sizeof buf, fmt, ap);
+        va_end(ap);
+        ctx->err = buf;
+    }
+    return s;
+}
+
+#define TSR_CUDA(ctx, call)                                                                            \
+    do {                                                                                               \
+        cudaError_t e__ = (call);                                                                      \
+        if (e__ != cudaSuccess)                                                                        \
+            return fail(ctx, TSR_ERR_CUDA, "%s failed: %s", #call, cudaGetErrorString(e__));           \
+    } while (0)
+
+bool aligned16(const void *p) { return ((uintptr_t)p & 15) == 0; }
+
+int elem_size(int dtype) { return dtype == TSR_BF16 ? 2 : 4; }
+
+// Walks the workspace layout; with a.base == nullptr it only measures.
+void layout(tsr_ctx *ctx, Arena &a, bool assign, size_t *step_end)
+{
+    const int nb = (int)ctx->blocks.size();
+    // ---- step area: device tables
+    for (int kd = 0; kd < NKIND; ++kd) {
+        void *p = a.take(sizeof(UmmaProblem) * (size_t)nb);
+        void *t = a.take(sizeof(UmmaTile) * std::max<size_t>(1, ctx->tiles[kd].size()));
+        if (assign) { ctx->d_probs[kd] = (UmmaProblem *)p; ctx->d_tiles[kd] = (UmmaTile *)t; }
+    }
+    void *p1 = a.take(sizeof(CoreUpdateArgs) * (size_t)nb);
+    void *p2 = a.take(sizeof(CoreUpdateArgs) * (size_t)nb);
+    void *p3 = a.take(sizeof(RefreshDev) * (size_t)nb);
+    void *p4 = a.take(sizeof(int32_t) * (size_t)nb);
+    void *p5 = a.take(sizeof(int32_t) * (size_t)nb);
+    void *p6 = a.take(sizeof(int32_t) * (size_t)nb);
+    if (assign) {
+        ctx->d_cu_all = (CoreUpdateArgs *)p1; ctx->d_cu_split = (CoreUpdateArgs *)p2;
+        ctx->d_refresh = (RefreshDev *)p3; ctx->d_status = (int32_t *)p4;
+        ctx->d_list = (int32_t *)p5; ctx->d_list2 = (int32_t *)p6;
+    }
+    size_t cap[4] = {0, 0, 0, 0};
+    for (const Block &b : ctx->blocks) {
+        cap[0] += (size_t)((b.d.m + RG_ROWS - 1) / RG_ROWS);
+        cap[1] += (size_t)gram_chunks(b.d.m);
+        cap[2] += (size_t)((b.d.n + RG_ROWS - 1) / RG_ROWS);
+        cap[3] += (size_t)gram_chunks(b.d.n);
+    }
+    for (int i = 0; i < 4; ++i) {
+        void *q = a.take(sizeof(RowItem) * cap[i]);
+        if (assign) { ctx->d_items[i] = (RowItem *)q; ctx->items_cap[i] = cap[i]; }
+    }
+    // ---- step area: per-block operands
+    for (Block &b : ctx->blocks) {
+        const int64_t m = b.d.m, n = b.d.n, r = b.d.r;
+        if (b.fast) {
+            void *ub = a.take((size_t)(m * b.rl) * 2), *ubt = a.take((size_t)(r * b.ml) * 2);
+            void *vb = a.take((size_t)(n * b.rl) * 2), *vbt = a.take((size_t)(r * b.nl) * 2);
+            void *tt = a.take((size_t)(r * b.ml) * 2), *pb = a.take((size_t)(m * b.rl) * 2);
+            void *db = a.take((size_t)(r * b.rl) * 2), *dbt = a.take((size_t)(r * b.rl) * 2);
+            void *part = b.nsplit > 1 ? a.take((size_t)b.nsplit * r * r * 4) : nullptr;
+            if (assign) {
+                b.Ub = (bf16 *)ub; b.Ubt = (bf16 *)ubt; b.Vb = (bf16 *)vb; b.Vbt = (bf16 *)vbt;
+                b.Tt = (bf16 *)tt; b.Pb = (bf16 *)pb; b.Db = (bf16 *)db; b.Dbt = (bf16 *)dbt;
+                b.partial = (float *)part;
+            }
+        } else {
+            void *t = a.take((size_t)(m * r) * 4), *pp = a.take((size_t)(m * r) * 4);
+            if (assign) { b.T32 = (float *)t; b.P32 = (float *)pp; }
+        }
+        void *d32 = a.take((size_t)(r * r) * 4);
+        if (assign) b.D32 = (float *)d32;
+    }
+    a.off = (a.off + 255) & ~(size_t)255;
+    *step_end = a.off;
+    // ---- refresh area
+    for (Block &b : ctx->blocks) {
+        const int64_t m = b.d.m, n = b.d.n, r = b.d.r, k = b.k;
+        const int64_t mx = std::max(m, n);
+        if (b.fast) {
+            void *gt = a.take((size_t)(n * b.ml) * 2);
+            void *xt = a.take((size_t)(2 * k * std::max(b.ml, b.nl)) * 2);
+            if (assign) { b.Gt = (bf16 *)gt; b.Xt = (bf16 *)xt; }
+        }
+        void *om = a.take((size_t)(n * k) * 4);
+        void *b0 = a.take((size_t)(mx * k) * 4), *b1 = a.take((size_t)(mx * k) * 4), *b2 = a.take((size_t)(mx * k) * 4);
+        void *S = a.take((size_t)(k * k) * 8), *Xw = a.take((size_t)(k * k) * 8), *Wj = a.take((size_t)(k * k) * 8);
+        void *gp = a.take((size_t)gram_chunks(mx) * k * k * 8);
+        void *lam = a.take((size_t)k * 8);
+        void *ri = a.take((size_t)(k * k) * 4), *wu = a.take((size_t)(k * r) * 4), *wv = a.take((size_t)(k * r) * 4);
+        if (assign) {
+            b.Om = (float *)om; b.buf[0] = (float *)b0; b.buf[1] = (float *)b1; b.buf[2] = (float *)b2;
+            b.S = (double *)S; b.Xw = (double *)Xw; b.Wj = (double *)Wj; b.gpart = (double *)gp; b.lam = (double *)lam;
+            b.Rinv = (float *)ri; b.Wu = (float *)wu; b.Wv = (float *)wv;
+        }
+    }
+    a.off = (a.off + 255) & ~(size_t)255;
+}
+
+void add_tiles(tsr_ctx *ctx, int kind, int bi, int M, int N, int K, int kb_per_split)
+{
+    Block &b = ctx->blocks[bi];
+    std::vector<UmmaTile> &v = ctx->tiles[kind];
+    b.tile_begin[kind] = (int)v.size();
+    const int nkb = (K + 63) / 64;
+    const int nsp = kb_per_split > 0 ? (nkb + kb_per_split - 1) / kb_per_split : 1;
+    for (int m0 = 0; m0 < M; m0 += 128)
+        for (int n0 = 0; n0 < N; n0 += 128)
+            for (int s = 0; s < nsp; ++s) {
+                UmmaTile t;
+                t.prob = bi; t.m0 = m0; t.n0 = n0;
+                t.kb0 = kb_per_split > 0 ? s * kb_per_split : 0;
+                t.kb1 = kb_per_split > 0 ? std::min(nkb, (s + 1) * kb_per_split) : nkb;
+                t.split = s;
+                v.push_back(t);
+            }
+    b.tile_end[kind] = (int)v.size();
+}
+
+void build_tiles(tsr_ctx *ctx)
+{
+    for (int kd = 0; kd < NKIND; ++kd) ctx->tiles[kd].clear();
+    for (int bi : ctx->order) {
+        Block &b = ctx->blocks[bi];
+        for (int kd = 0; kd < NKIND; ++kd) b.tile_begin[kd] = b.tile_end[kd] = (int)ctx->tiles[kd].size();
+        if (!b.fast) continue;
+        const int m = (int)b.d.m, n = (int)b.d.n, r = b.d.r, k = b.k;
+        add_tiles(ctx, KT, bi, m, r, n, 0);
+        if (b.nsplit > 1) add_tiles(ctx, KCS, bi, r, r, m, b.kb_per_split);
+        else add_tiles(ctx, KC, bi, r, r, m, 0);
+        add_tiles(ctx, KP, bi, m, r, r, 0);
+        add_tiles(ctx, KA, bi, m, n, r, 0);
+        add_tiles(ctx, KY, bi, m, k, n, 0);
+        add_tiles(ctx, KZ, bi, n, k, m, 0);
+    }
+}
+
+// BF16 row-major [rows x cols] (ld elements) -> tensor map with a 64 x box_rows box, 128B swizzle.
+tsr_status encode_map(tsr_ctx *ctx, CUtensorMap *out, const void *base, int64_t rows, int64_t cols, int64_t ld,
+                      int box_rows)
+{
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+    cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult rc = ctx->encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box,
+                              estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (rc != CUDA_SUCCESS)
+        return fail(ctx, TSR_ERR_CUDA, "cuTensorMapEncodeTiled failed (%d) rows=%lld cols=%lld ld=%lld", (int)rc,
+                    (long long)rows, (long long)cols, (long long)ld);
+    return TSR_OK;
+}
+
+StepScalars make_scalars(const tsr_hyper *h)
+{
+    StepScalars sc;
+    sc.beta1 = h->beta1; sc.beta2 = h->beta2; sc.eps = h->eps;
+    const double t = (double)h->step;
+    sc.inv_bc1 = (float)(1.0 / (1.0 - pow((double)h->beta1, t)));
+    sc.inv_bc2 = (float)(1.0 / (1.0 - pow((double)h->beta2, t)));
+    sc.rule = h->rule;
+    if (h->rule == TSR_RULE_SGD) {
+        sc.decay = 1.0f;
+        sc.step_scale = h->lr;
+    } else {
+        sc.decay = 1.0f - h->lr * h->weight_decay;
+        sc.step_scale = h->lr * h->scale;
+    }
+    return sc;
+}
+
+tsr_status check_hyper(tsr_ctx *ctx, const tsr_hyper *h)
+{
+    if (!h) return fail(ctx, TSR_ERR_INVALID_ARG, "hyper is NULL");
+    if (h->step < 1) return fail(ctx, TSR_ERR_INVALID_ARG, "hyper.step must be >= 1");
+    if (h->rule != TSR_RULE_ADAM && h->rule != TSR_RULE_SGD) return fail(ctx, TSR_ERR_INVALID_ARG, "unknown rule");
+    if (!(h->beta1 >= 0.f && h->beta1 < 1.f) || !(h->beta2 >= 0.f && h->beta2 < 1.f))
+        return fail(ctx, TSR_ERR_INVALID_ARG, "betas must lie in [0, 1)");
+    return TSR_OK;
+}
+
+// Resolves (idx, count) into a validated list of block indices.
+tsr_status resolve_list(tsr_ctx *ctx, const int32_t *idx, int32_t count, std::vector<int> &out)
+{
+    out.clear();
+    const int nb = (int)ctx->blocks.size();
+    if (!idx) {
+        for (int i = 0; i < nb; ++i) out.push_back(i);
+        return TSR_OK;
+    }
+    if (count < 0) return fail(ctx, TSR_ERR_INVALID_ARG, "negative count");
+    std::vector<char> seen(nb, 0);
+    for (int j = 0; j < count; ++j) {
+        if (idx[j] < 0 || idx[j] >= nb) return fail(ctx, TSR_ERR_INVALID_ARG, "block index %d out of range", idx[j]);
+        if (seen[idx[j]]) return fail(ctx, TSR_ERR_INVALID_ARG, "block index %d listed twice", idx[j]);
+        seen[idx[j]] = 1;
+        out.push_back(idx[j]);
+    }
+    return TSR_OK;
+}
+
+tsr_status check_ready(tsr_ctx *ctx)
+{
+    if (!ctx) return TSR_ERR_INVALID_ARG;
+    if (!ctx->bound) return fail(ctx, TSR_ERR_NOT_BOUND, "tsr_bind has not been called");
+    return TSR_OK;
+}
+
+// Launches one tensor-core GEMM kind over the listed blocks (adjacent table ranges are merged).
+tsr_status launch_kind(tsr_ctx *ctx, int kind, const std::vector<int> &list, int epilogue, int planes,
+                       const StepScalars &sc, cudaStream_t st)
+{
+    std::vector<std::pair<int, int>> ranges;
+    for (int bi : list) {
+        const Block &b = ctx->blocks[bi];
+        if (b.tile_end[kind] > b.tile_begin[kind]) ranges.push_back({b.tile_begin[kind], b.tile_end[kind]});
+    }
+    std::sort(ranges.begin(), ranges.end());
+    size_t i = 0;
+    while (i < ranges.size()) {
+        int lo = ranges[i].first, hi = ranges[i].second;
+        size_t j = i + 1;
+        while (j < ranges.size() && ranges[j].first == hi) { hi = ranges[j].second; ++j; }
+        TSR_CUDA(ctx, umma_gemm_launch(ctx->d_probs[kind], ctx->d_tiles[kind] + lo, hi - lo, 128, epilogue, planes, sc,
+                                       ctx->d_status, st));
+        i = j;
+    }
+    return TSR_OK;
+}
+
+tsr_status upload_list(tsr_ctx *ctx, int32_t *dst, const std::vector<int> &v, cudaStream_t st)
+{
+    if (v.empty()) return TSR_OK;
+    TSR_CUDA(ctx, cudaMemcpyAsync(dst, v.data(), v.size() * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    return TSR_OK;
+}
+
+// ---- Section 3.3: C = U^T G V (optionally with the fused core update) -------------------
+tsr_status do_project(tsr_ctx *ctx, const std::vector<int> &list, bool fuse, const StepScalars &sc, cudaStream_t st)
+{
+    tsr_status s;
+    if (ctx->any_fast) {
+        if ((s = launch_kind(ctx, KT, list, EPI_STORE_BF16_T, 1, sc, st)) != TSR_OK) return s;
+        if ((s = launch_kind(ctx, KC, list, fuse ? EPI_CORE_UPDATE : EPI_STORE_F32, 1, sc, st)) != TSR_OK) return s;
+        if ((s = launch_kind(ctx, KCS, list, EPI_STORE_F32, 1, sc, st)) != TSR_OK) return s;
+    }
+    std::vector<int> split, later;
+    int max_r = 1;
+    for (int bi : list) {
+        Block &b = ctx->blocks[bi];
+        const int m = (int)b.d.m, n = (int)b.d.n, r = b.d.r;
+        if (!b.fast) {
+            // T = G V, C = U^T T on CUDA cores
+            TSR_CUDA(ctx, simt_gemm(m, r, n, b.p.G, b.d.g_dtype, b.d.ldg, 1, b.p.V, r, 1, b.T32, r, SIMT_STORE, 0, 0, st));
+            TSR_CUDA(ctx, simt_gemm(r, r, m, b.p.U, TSR_F32, 1, r, b.T32, r, 1, b.p.C, r, SIMT_STORE, 0, 0, st));
+            if (fuse) { later.push_back(bi); max_r = std::max(max_r, r); }
+        } else if (b.nsplit > 1) {
+            split.push_back(bi);
+            max_r = std::max(max_r, r);
+        }
+    }
+    if (!split.empty()) {   // sum the split-K slabs (and, when fused, run the core update on the sum)
+        if ((s = upload_list(ctx, ctx->d_list2, split, st)) != TSR_OK) return s;
+        TSR_CUDA(ctx, core_update_launch(ctx->d_cu_split, ctx->d_list2, (int)split.size(), max_r, sc, fuse ? 0 : 1, st));
+    }
+    if (!later.empty()) {
+        if ((s = upload_list(ctx, ctx->d_list2, later, st)) != TSR_OK) return s;
+        TSR_CUDA(ctx, core_update_launch(ctx->d_cu_all, ctx->d_list2, (int)later.size(), max_r, sc, 0, st));
+    }
+    return TSR_OK;
+}
+
+// ---- Section 3.4: moments and D from C ----------------------------------------------------
+tsr_status do_core_update(tsr_ctx *ctx, const std::vector<int> &list, const StepScalars &sc, cudaStream_t st)
+{
+    tsr_status s;
+    int max_r = 1;
+    for (int bi : list) max_r = std::max(max_r, (int)ctx->blocks[bi].d.r);
+    if ((s = upload_list(ctx, ctx->d_list, list, st)) != TSR_OK) return s;
+    TSR_CUDA(ctx, core_update_launch(ctx->d_cu_all, ctx->d_list, (int)list.size(), max_r, sc, 0, st));
+    return TSR_OK;
+}
+
+// ---- Section 3.4: W <- decay W - step_scale U D V^T ---------------------------------------
+tsr_status do_apply(tsr_ctx *ctx, const std::vector<int> &list, const StepScalars &sc, cudaStream_t st)
+{
+    tsr_status s;
+    if (ctx->any_fast) {
+        if ((s = launch_kind(ctx, KP, list, EPI_STORE_BF16, 1, sc, st)) != TSR_OK) return s;
+        if ((s = launch_kind(ctx, KA, list, EPI_APPLY, 1, sc, st)) != TSR_OK) return s;
+    }
+    for (int bi : list) {
+        Block &b = ctx->blocks[bi];
+        if (b.fast) continue;
+        const int m = (int)b.d.m, n = (int)b.d.n, r = b.d.r;
+        TSR_CUDA(ctx, simt_gemm(m, r, r, b.p.U, TSR_F32, r, 1, b.D32, r, 1, b.P32, r, SIMT_STORE, 0, 0, st));
+        TSR_CUDA(ctx, simt_gemm(m, n, r, b.P32, TSR_F32, r, 1, b.p.V, 1, r, (float *)b.p.W, b.d.ldw, SIMT_APPLY, sc.decay,
+                                sc.step_scale, st));
+    }
+    return TSR_OK;
+}
+
+tsr_status do_shadows(tsr_ctx *ctx, const std::vector<int> &list, cudaStream_t st)
+{
+    for (int bi : list) {
+        Block &b = ctx->blocks[bi];
+        if (!b.fast) continue;
+        TSR_CUDA(ctx, make_shadows(b.p.U, (int)b.d.m, b.d.r, b.Ub, b.rl, b.Ubt, b.ml, st));
+        TSR_CUDA(ctx, make_shadows(b.p.V, (int)b.d.n, b.d.r, b.Vb, b.rl, b.Vbt, b.nl, st));
+    }
+    return TSR_OK;
+}
+
+// ---- Section 3.5: randomized-SVD refresh ---------------------------------------------------
+struct RefreshLists {
+    std::vector<int> list;
+    int nitems[4];
+    int kmax, rmax;
+};
+
+tsr_status orth_pass(tsr_ctx *ctx, const RefreshLists &L, int side, int src, int dst, cudaStream_t st)
+{
+    const int nl = (int)L.list.size();
+    TSR_CUDA(ctx, gram_batched(ctx->d_refresh, ctx->d_items[side * 2 + 1], L.nitems[side * 2 + 1], ctx->d_list, nl, side,
+                               src, L.kmax, st));
+    TSR_CUDA(ctx, chol_inverse_batched(ctx->d_refresh, ctx->d_list, nl, st));
+    TSR_CUDA(ctx, rows_gemm_batched(ctx->d_refresh, ctx->d_items[side * 2], L.nitems[side * 2], side, src, 0, dst, L.kmax, st));
+    return TSR_OK;
+}
+
+// orth(buf[0]) -> buf[2] by Cholesky-QR applied twice (buf[1] holds the first pass).
+tsr_status orth(tsr_ctx *ctx, const RefreshLists &L, int side, cudaStream_t st)
+{
+    tsr_status s;
+    if ((s = orth_pass(ctx, L, side, 0, 1, st)) != TSR_OK) return s;
+    return orth_pass(ctx, L, side, 1, 2, st);
+}
+
+// buf[0] (rows_out x k) = G X  (transposed = false, X = buf[2] or Omega, n x k)
+//                      or G^T X (transposed = true,  X = buf[2], m x k)
+tsr_status sketch(tsr_ctx *ctx, const RefreshLists &L, bool transposed, bool from_omega,
+                  const float *const *omegas, cudaStream_t st)
+{
+    StepScalars sc = {};
+    tsr_status s;
+    for (size_t j = 0; j < L.list.size(); ++j) {
+        Block &b = ctx->blocks[L.list[j]];
+        const int m = (int)b.d.m, n = (int)b.d.n, k = b.k;
+        const float *X = from_omega ? ((omegas && omegas[j]) ? omegas[j] : b.Om) : b.buf[2];
+        if (b.fast) {
+            const int rows = transposed ? m : n;                 // rows of X
+            const int64_t ld = transposed ? b.ml : b.nl;
+            TSR_CUDA(ctx, split_transpose(X, rows, k, b.Xt, ld, k, 2, st));
+        } else if (!transposed) {
+            TSR_CUDA(ctx, simt_gemm(m, k, n, b.p.G, b.d.g_dtype, b.d.ldg, 1, X, k, 1, b.buf[0], k, SIMT_STORE, 0, 0, st));
+        } else {
+            TSR_CUDA(ctx, simt_gemm(n, k, m, b.p.G, b.d.g_dtype, 1, b.d.ldg, X, k, 1, b.buf[0], k, SIMT_STORE, 0, 0, st));
+        }
+    }
+    if (ctx->any_fast)
+        if ((s = launch_kind(ctx, transposed ? KZ : KY, L.list, EPI_STORE_F32, 2, sc, st)) != TSR_OK) return s;
+    return TSR_OK;
+}
+
+tsr_status do_refresh(tsr_ctx *ctx, const std::vector<int> &list, uint64_t seed, const float *const *omegas,
+                      cudaStream_t st)
+{
+    if (list.empty()) return TSR_OK;
+    tsr_status s;
+    RefreshLists L;
+    L.list = list;
+    L.kmax = 1; L.rmax = 1;
+    std::vector<RowItem> items[4];
+    int qmax = 0;
+    for (int bi : list) {
+        const Block &b = ctx->blocks[bi];
+        L.kmax = std::max(L.kmax, b.k);
+        L.rmax = std::max(L.rmax, (int)b.d.r);
+        qmax = std::max(qmax, (int)b.d.q);
+        for (int side = 0; side < 2; ++side) {
+            const int rows = (int)(side ? b.d.n : b.d.m);
+            for (int r0 = 0; r0 < rows; r0 += RG_ROWS) items[side * 2].push_back({bi, r0});
+            for (int r0 = 0; r0 < rows; r0 += GRAM_ROWS) items[side * 2 + 1].push_back({bi, r0});
+        }
+    }
+    for (int bi : list)
+        if (ctx->blocks[bi].d.q != qmax)
+            return fail(ctx, TSR_ERR_UNSUPPORTED, "blocks refreshed in one grouped call must share q");
+    if ((s = upload_list(ctx, ctx->d_list, list, st)) != TSR_OK) return s;
+    for (int i = 0; i < 4; ++i) {
+        L.nitems[i] = (int)items[i].size();
+        TSR_CUDA(ctx, cudaMemcpyAsync(ctx->d_items[i], items[i].data(), items[i].size() * sizeof(RowItem),
+                                      cudaMemcpyHostToDevice, st));
+    }
+    // Omega and the transposed gradient copies
+    for (size_t j = 0; j < list.size(); ++j) {
+        Block &b = ctx->blocks[list[j]];
+        if (!(omegas && omegas[j]))
+            TSR_CUDA(ctx, fill_gaussian(b.Om, (int64_t)b.d.n * b.k, seed, (uint64_t)list[j], st));
+        if (b.fast)
+            TSR_CUDA(ctx, transpose_bf16((const bf16 *)b.p.G, (int)b.d.m, (int)b.d.n, b.d.ldg, b.Gt, b.ml, st));
+    }
+    // Y = G Omega; Q = orth(Y)
+    if ((s = sketch(ctx, L, false, true, omegas, st)) != TSR_OK) return s;
+    if ((s = orth(ctx, L, 0, st)) != TSR_OK) return s;
+    for (int it = 0; it < qmax; ++it) {
+        // Yrow = G^T Q; Qrow = orth(Yrow); Y = G Qrow; Q = orth(Y)
+        if ((s = sketch(ctx, L, true, false, nullptr, st)) != TSR_OK) return s;
+        if ((s = orth(ctx, L, 1, st)) != TSR_OK) return s;
+        if ((s = sketch(ctx, L, false, false, nullptr, st)) != TSR_OK) return s;
+        if ((s = orth(ctx, L, 0, st)) != TSR_OK) return s;
+    }
+    // B^T = G^T Q (n x k) in buf[0]; small SVD through the k x k Gram matrix B B^T
+    if ((s = sketch(ctx, L, true, false, nullptr, st)) != TSR_OK) return s;
+    const int nl = (int)list.size();
+    TSR_CUDA(ctx, gram_batched(ctx->d_refresh, ctx->d_items[3], L.nitems[3], ctx->d_list, nl, 1, 0, L.kmax, st));
+    TSR_CUDA(ctx, jacobi_batched(ctx->d_refresh, ctx->d_list, nl, 40, st));
+    // V = B^T Wt / sigma ; U = Q Wt
+    TSR_CUDA(ctx, rows_gemm_batched(ctx->d_refresh, ctx->d_items[2], L.nitems[2], 1, 0, 2, 4, L.rmax, st));
+    TSR_CUDA(ctx, rows_gemm_batched(ctx->d_refresh, ctx->d_items[0], L.nitems[0], 0, 2, 1, 3, L.rmax, st));
+    return do_shadows(ctx, list, st);
+}
+
+tsr_status zero_moments(tsr_ctx *ctx, const std::vector<int> &list, cudaStream_t st)
+{
+    for (int bi : list) {
+        Block &b = ctx->blocks[bi];
+        const int64_t rr = (int64_t)b.d.r * b.d.r;
+        TSR_CUDA(ctx, fill_zero_f32(b.p.M, rr, st));
+        if (b.p.Vm) TSR_CUDA(ctx, fill_zero_f32(b.p.Vm, rr, st));
+    }
+    return TSR_OK;
+}
+
+tsr_status do_step(tsr_ctx *ctx, const std::vector<int> &list, const tsr_hyper *h, uint64_t seed, bool fuse,
+                   cudaStream_t st)
+{
+    tsr_status s;
+    std::vector<int> due;
+    for (int bi : list) {
+        const Block &b = ctx->blocks[bi];
+        if (b.d.K > 0 && h->step % b.d.K == 0) due.push_back(bi);
+    }
+    if (!due.empty()) {
+        // blocks with different q refresh in separate groups
+        std::vector<int> qs;
+        for (int bi : due) if (std::find(qs.begin(), qs.end(), (int)ctx->blocks[bi].d.q) == qs.end()) qs.push_back(ctx->blocks[bi].d.q);
+        for (int q : qs) {
+            std::vector<int> grp;
+            for (int bi : due) if (ctx->blocks[bi].d.q == q) grp.push_back(bi);
+            if ((s = do_refresh(ctx, grp, seed ^ ((uint64_t)h->step * 0x9E3779B97F4A7C15ull), nullptr, st)) != TSR_OK) return s;
+        }
+    }
+    const StepScalars sc = make_scalars(h);
+    if ((s = do_project(ctx, list, fuse, sc, st)) != TSR_OK) return s;
+    if (!fuse && (s = do_core_update(ctx, list, sc, st)) != TSR_OK) return s;
+    return do_apply(ctx, list, sc, st);
+}
+
+}  // namespace
+
+// =============================================================================================
+// C ABI
+// =============================================================================================
+extern "C" {
+
+int tsr_version(void) { return 100; }
+
+const char *tsr_status_string(tsr_status s)
+{
+    switch (s) {
+    case TSR_OK: return "ok";
+    case TSR_ERR_INVALID_ARG: return "invalid argument";
+    case TSR_ERR_SHAPE: return "bad shape";
+    case TSR_ERR_ALIGNMENT: return "bad alignment";
+    case TSR_ERR_WORKSPACE: return "workspace missing or too small";
+    case TSR_ERR_CUDA: return "CUDA error";
+    case TSR_ERR_UNSUPPORTED: return "unsupported";
+    case TSR_ERR_NOT_CONVERGED: return "eigen-solver did not converge";
+    case TSR_ERR_RANK_DEFICIENT: return "rank-deficient sketch";
+    case TSR_ERR_NONFINITE: return "non-finite value";
+    case TSR_ERR_TIMEOUT: return "bounded device wait ran out";
+    case TSR_ERR_NOT_BOUND: return "context not bound";
+    }
+    return "unknown status";
+}
+
+const char *tsr_last_error(const tsr_ctx *ctx) { return ctx ? ctx->err.c_str() : ""; }
+
+tsr_status tsr_create(tsr_ctx **out, const tsr_mat_desc *descs, int32_t count)
+{
+    if (!out) return TSR_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!descs || count <= 0) return TSR_ERR_INVALID_ARG;
+    for (int i = 0; i < count; ++i) {
+        const tsr_mat_desc &d = descs[i];
+        if (d.m <= 0 || d.n <= 0 || d.r <= 0 || d.p < 0 || d.q < 0) return TSR_ERR_SHAPE;
+        if (d.ldg < d.n || d.ldw < d.n) return TSR_ERR_SHAPE;
+        if ((int64_t)d.r + d.p > std::min(d.m, d.n)) return TSR_ERR_SHAPE;
+        if (d.m > 0x3fffffff || d.n > 0x3fffffff || d.r + d.p > 1056) return TSR_ERR_SHAPE;
+        if (d.g_dtype != TSR_F32 && d.g_dtype != TSR_BF16) return TSR_ERR_UNSUPPORTED;
+        if (d.w_dtype != TSR_F32) return TSR_ERR_UNSUPPORTED;
+        if (d.reserved != 0 || (d.is_embedding != 0 && d.is_embedding != 1)) return TSR_ERR_INVALID_ARG;
+    }
+    tsr_ctx *ctx = new (std::nothrow) tsr_ctx;
+    if (!ctx) return TSR_ERR_INVALID_ARG;
+    ctx->blocks.resize(count);
+    for (int i = 0; i < count; ++i) {
+        Block &b = ctx->blocks[i];
+        b.d = descs[i];
+        memset(&b.p, 0, sizeof b.p);
+        b.k = b.d.r + b.d.p;
+        b.rl = round_up(b.d.r, 8); b.ml = round_up(b.d.m, 8); b.nl = round_up(b.d.n, 8);
+        // Candidate for the tensor-core path: BF16 gradient with 16-byte row pitches.  Pointer
+        // alignment is checked at bind time.
+        b.fast = (b.d.g_dtype == TSR_BF16) && ((b.d.ldg * 2) % 16 == 0) && ((b.d.ldw * 4) % 16 == 0);
+        const int nkb = (int)((b.d.m + 63) / 64);
+        if (nkb > 128) { b.kb_per_split = 32; b.nsplit = (nkb + 31) / 32; }
+        ctx->max_r = std::max(ctx->max_r, (int)b.d.r);
+        ctx->max_k = std::max(ctx->max_k, b.k);
+        ctx->order.push_back(i);
+    }
+    std::stable_sort(ctx->order.begin(), ctx->order.end(), [&](int a, int b) {
+        return ctx->blocks[a].d.m * ctx->blocks[a].d.n > ctx->blocks[b].d.m * ctx->blocks[b].d.n;
+    });
+    build_tiles(ctx);
+    Arena a{nullptr, 0};
+    size_t step_end = 0;
+    layout(ctx, a, false, &step_end);
+    ctx->step_bytes = step_end;
+    ctx->refresh_bytes = a.off - step_end;
+    *out = ctx;
+    return TSR_OK;
+}
+
+tsr_status tsr_destroy(tsr_ctx *ctx)
+{
+    if (!ctx) return TSR_ERR_INVALID_ARG;
+    delete ctx;
+    return TSR_OK;
+}
+
+tsr_status tsr_workspace_bytes(const tsr_ctx *ctx, size_t *step_bytes, size_t *refresh_bytes)
+{
+    if (!ctx || !step_bytes || !refresh_bytes) return TSR_ERR_INVALID_ARG;
+    *step_bytes = ctx->step_bytes;
+    *refresh_bytes = ctx->refresh_bytes;
+    return TSR_OK;
+}
+
+tsr_status tsr_bind(tsr_ctx *ctx, const tsr_mat_ptrs *ptrs, int32_t count, void *workspace, size_t workspace_bytes)
+{
+    if (!ctx) return TSR_ERR_INVALID_ARG;
+    if (!ptrs || count != (int32_t)ctx->blocks.size()) return fail(ctx, TSR_ERR_INVALID_ARG, "ptrs/count mismatch");
+    if (!workspace || workspace_bytes < ctx->step_bytes + ctx->refresh_bytes)
+        return fail(ctx, TSR_ERR_WORKSPACE, "workspace needs %zu bytes", ctx->step_bytes + ctx->refresh_bytes);
+    if (((uintptr_t)workspace & 255) != 0) return fail(ctx, TSR_ERR_ALIGNMENT, "workspace must be 256-byte aligned");
+    for (int i = 0; i < count; ++i) {
+        const tsr_mat_ptrs &p = ptrs[i];
+        if (!p.G || !p.W || !p.U || !p.V || !p.M || !p.C) return fail(ctx, TSR_ERR_INVALID_ARG, "block %d: NULL pointer", i);
+        if (((uintptr_t)p.U | (uintptr_t)p.V | (uintptr_t)p.M | (uintptr_t)p.C | (uintptr_t)p.W) & 3)
+            return fail(ctx, TSR_ERR_ALIGNMENT, "block %d: FP32 buffer not 4-byte aligned", i);
+    }
+    int dev_count = 0;
+    if (cudaGetDeviceCount(&dev_count) != cudaSuccess || dev_count <= 0)
+        return fail(ctx, TSR_ERR_CUDA, "no CUDA device available");
+    ctx->bound = false;
+    bool layout_changed = false;
+    for (int i = 0; i < count; ++i) {
+        Block &b = ctx->blocks[i];
+        b.p = ptrs[i];
+        const bool cand = (b.d.g_dtype == TSR_BF16) && ((b.d.ldg * 2) % 16 == 0) && ((b.d.ldw * 4) % 16 == 0);
+        const bool fast = cand && aligned16(b.p.G) && aligned16(b.p.W);
+        if (fast != b.fast) { b.fast = fast; layout_changed = true; }
+    }
+    if (layout_changed) {   // a misaligned pointer moved a block to the CUDA-core path
+        build_tiles(ctx);
+        Arena m{nullptr, 0};
+        size_t se = 0;
+        layout(ctx, m, false, &se);
+        ctx->step_bytes = se;
+        ctx->refresh_bytes = m.off - se;
+        if (workspace_bytes < m.off) return fail(ctx, TSR_ERR_WORKSPACE, "workspace needs %zu bytes", m.off);
+    }
+    ctx->any_fast = false;
+    for (const Block &b : ctx->blocks) ctx->any_fast = ctx->any_fast || b.fast;
+    Arena a{(char *)workspace, 0};
+    size_t step_end = 0;
+    layout(ctx, a, true, &step_end);
+
+    if (ctx->any_fast) {
+        if (!ctx->encode) {
+            void *fn = nullptr;
+            cudaDriverEntryPointQueryResult qres;
+            TSR_CUDA(ctx, cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
+            if (!fn || qres != cudaDriverEntryPointSuccess) return fail(ctx, TSR_ERR_CUDA, "cuTensorMapEncodeTiled unavailable");
+            ctx->encode = (EncodeTiledFn)fn;
+        }
+        TSR_CUDA(ctx, umma_configure());
+    }
+
+    const int nb = count;
+    std::vector<UmmaProblem> probs[NKIND];
+    for (int kd = 0; kd < NKIND; ++kd) { probs[kd].resize(nb); memset((void *)probs[kd].data(), 0, sizeof(UmmaProblem) * nb); }
+    std::vector<CoreUpdateArgs> cu_all(nb), cu_split(nb);
+    std::vector<RefreshDev> rdev(nb);
+    tsr_status s;
+    for (int i = 0; i < nb; ++i) {
+        Block &b = ctx->blocks[i];
+        const int64_t m = b.d.m, n = b.d.n, r = b.d.r, k = b.k;
+        CoreUpdateArgs &ca = cu_all[i];
+        memset(&ca, 0, sizeof ca);
+        ca.C = b.p.C; ca.Cout = b.p.C; ca.mom1 = b.p.M; ca.mom2 = b.p.Vm; ca.d_f32 = b.D32;
+        ca.d_bf16 = b.fast ? b.Db : nullptr; ca.dt_bf16 = b.fast ? b.Dbt : nullptr; ca.ldd = b.rl;
+        ca.split_stride = 0; ca.r = (int)r; ca.nsplit = 1;
+        cu_split[i] = ca;
+        cu_split[i].C = b.partial; cu_split[i].nsplit = b.nsplit; cu_split[i].split_stride = r * r;
+        RefreshDev &rd = rdev[i];
+        memset(&rd, 0, sizeof rd);
+        rd.m = (int)m; rd.n = (int)n; rd.k = (int)k; rd.r = (int)r;
+        for (int j = 0; j < 3; ++j) rd.buf[j] = b.buf[j];
+        rd.S = b.S; rd.Xw = b.Xw; rd.Wj = b.Wj; rd.gpart = b.gpart; rd.lam = b.lam;
+        rd.Rinv = b.Rinv; rd.Wu = b.Wu; rd.Wv = b.Wv; rd.U = b.p.U; rd.V = b.p.V; rd.status = ctx->d_status + i;
+        if (!b.fast) continue;
+        auto base = [&](UmmaProblem &P, int M, int N, int K, int epi) {
+            P.M = M; P.N = N; P.K = K; P.planes = 1; P.plane_rows = 0; P.block = i; P.epilogue = epi;
+        };
+        {   // T~ = (G V)^T : A = G [m x n], B = V^T copy [r x n]
+            UmmaProblem &P = probs[KT][i];
+            base(P, (int)m, (int)r, (int)n, EPI_STORE_BF16_T);
+            if ((s = encode_map(ctx, &P.tmA, b.p.G, m, n, b.d.ldg, 128)) != TSR_OK) return s;
+            if ((s = encode_map(ctx, &P.tmB, b.Vbt, r, n, b.nl, 128)) != TSR_OK) return s;
+            P.out = b.Tt; P.ld_out = b.ml;
+        }
+        for (int kd : {KC, KCS}) {   // C = U^T T : A = U^T copy [r x m], B = T~ [r x m]
+            UmmaProblem &P = probs[kd][i];
+            base(P, (int)r, (int)r, (int)m, EPI_CORE_UPDATE);
+            if ((s = encode_map(ctx, &P.tmA, b.Ubt, r, m, b.ml, 128)) != TSR_OK) return s;
+            if ((s = encode_map(ctx, &P.tmB, b.Tt, r, m, b.ml, 128)) != TSR_OK) return s;
+            P.out = (kd == KC) ? (void *)b.p.C : (void *)b.partial;
+            P.ld_out = r; P.split_stride = r * r;
+            P.mom1 = b.p.M; P.mom2 = b.p.Vm; P.d_bf16 = b.Db; P.dt_bf16 = b.Dbt; P.ldd = b.rl;
+        }
+        {   // P = U D : A = U copy [m x r], B = D^T copy [r x r]
+            UmmaProblem &P = probs[KP][i];
+            base(P, (int)m, (int)r, (int)r, EPI_STORE_BF16);
+            if ((s = encode_map(ctx, &P.tmA, b.Ub, m, r, b.rl, 128)) != TSR_OK) return s;
+            if ((s = encode_map(ctx, &P.tmB, b.Dbt, r, r, b.rl, 128)) != TSR_OK) return s;
+            P.out = b.Pb; P.ld_out = b.rl;
+        }
+        {   // W update : A = P [m x r], B = V copy [n x r]
+            UmmaProblem &P = probs[KA][i];
+            base(P, (int)m, (int)n, (int)r, EPI_APPLY);
+            if ((s = encode_map(ctx, &P.tmA, b.Pb, m, r, b.rl, 128)) != TSR_OK) return s;
+            if ((s = encode_map(ctx, &P.tmB, b.Vb, n, r, b.rl, 128)) != TSR_OK) return s;
+            P.out = b.p.W; P.ld_out = b.d.ldw;
+        }
+        {   // Y = G X : A = G, B = X^T planes [2k x n]
+            UmmaProblem &P = probs[KY][i];
+            base(P, (int)m, (int)k, (int)n, EPI_STORE_F32);
+            P.planes = 2; P.plane_rows = (int)k;
+            if ((s = encode_map(ctx, &P.tmA, b.p.G, m, n, b.d.ldg, 128)) != TSR_OK) return s;
+            if ((s = encode_map(ctx, &P.tmB, b.Xt, 2 * k, n, b.nl, 128)) != TSR_OK) return s;
+            P.out = b.buf[0]; P.ld_out = k;
+        }
+        {   // Z = G^T X : A = G^T copy [n x m], B = X^T planes [2k x m]
+            UmmaProblem &P = probs[KZ][i];
+            base(P, (int)n, (int)k, (int)m, EPI_STORE_F32);
+            P.planes = 2; P.plane_rows = (int)k;
+            if ((s = encode_map(ctx, &P.tmA, b.Gt, n, m, b.ml, 128)) != TSR_OK) return s;
+            if ((s = encode_map(ctx, &P.tmB, b.Xt, 2 * k, m, b.ml, 128)) != TSR_OK) return s;
+            P.out = b.buf[0]; P.ld_out = k;
+        }
+    }
+    for (int kd = 0; kd < NKIND; ++kd) {
+        TSR_CUDA(ctx, cudaMemcpy(ctx->d_probs[kd], probs[kd].data(), sizeof(UmmaProblem) * nb, cudaMemcpyHostToDevice));
+        if (!ctx->tiles[kd].empty())
+            TSR_CUDA(ctx, cudaMemcpy(ctx->d_tiles[kd], ctx->tiles[kd].data(), sizeof(UmmaTile) * ctx->tiles[kd].size(),
+                                     cudaMemcpyHostToDevice));
+    }
+    TSR_CUDA(ctx, cudaMemcpy(ctx->d_cu_all, cu_all.data(), sizeof(CoreUpdateArgs) * nb, cudaMemcpyHostToDevice));
+    TSR_CUDA(ctx, cudaMemcpy(ctx->d_cu_split, cu_split.data(), sizeof(CoreUpdateArgs) * nb, cudaMemcpyHostToDevice));
+    TSR_CUDA(ctx, cudaMemcpy(ctx->d_refresh, rdev.data(), sizeof(RefreshDev) * nb, cudaMemcpyHostToDevice));
+    TSR_CUDA(ctx, cudaMemset(ctx->d_status, 0, sizeof(int32_t) * nb));
+    ctx->bound = true;
+    ctx->err.clear();
+    return TSR_OK;
+}
+
+tsr_status tsr_bases_changed(tsr_ctx *ctx, const int32_t *idx, int32_t count, void *stream)
+{
+    tsr_status s = check_ready(ctx);
+    if (s != TSR_OK) return s;
+    std::vector<int> list;
+    if ((s = resolve_list(ctx, idx, count, list)) != TSR_OK) return s;
+    return do_shadows(ctx, list, (cudaStream_t)stream);
+}
+
+// ---- grouped calls ------------------------------------------------------------------------
+tsr_status tsr_init_subspace_grouped(tsr_ctx *ctx, const int32_t *idx, int32_t count, uint64_t seed,
+                                     const float *const *omegas, void *stream)
+{
+    tsr_status s = check_ready(ctx);
+    if (s != TSR_OK) return s;
+    std::vector<int> list;
+    if ((s = resolve_list(ctx, idx, count, list)) != TSR_OK) return s;
+    if ((s = zero_moments(ctx, list, (cudaStream_t)stream)) != TSR_OK) return s;
+    return tsr_rsvd_refresh_grouped(ctx, idx, count, seed, omegas, stream);
+}
+
+tsr_status tsr_rsvd_refresh_grouped(tsr_ctx *ctx, const int32_t *idx, int32_t count, uint64_t seed,
+                                    const float *const *omegas, void *stream)
+{
+    tsr_status s = check_ready(ctx);
+    if (s != TSR_OK) return s;
+    std::vector<int> list;
+    if ((s = resolve_list(ctx, idx, count, list)) != TSR_OK) return s;
+    // group by q, keeping each block's omega with it
+    std::vector<int> qs;
+    for (int bi : list) if (std::find(qs.begin(), qs.end(), (int)ctx->blocks[bi].d.q) == qs.end()) qs.push_back(ctx->blocks[bi].d.q);
+    for (int q : qs) {
+        std::vector<int> grp;
+        std::vector<const float *> om;
+        for (size_t j = 0; j < list.size(); ++j)
+            if (ctx->blocks[list[j]].d.q == q) { grp.push_back(list[j]); om.push_back(omegas ? omegas[j] : nullptr); }
+        if ((s = do_refresh(ctx, grp, seed, omegas ? om.data() : nullptr, (cudaStream_t)stream)) != TSR_OK) return s;
+    }
+    return TSR_OK;
+}
+
+tsr_status tsr_project_core_grouped(tsr_ctx *ctx, const int32_t *idx, int32_t count, void *stream)
+{
+    tsr_status s = check_ready(ctx);
+    if (s != TSR_OK) return s;
+    std::vector<int> list;
+    if ((s = resolve_list(ctx, idx, count, list)) != TSR_OK) return s;
+    StepScalars sc = {};
+    return do_project(ctx, list, false, sc, (cudaStream_t)stream);
+}
+
+tsr_status tsr_adam_core_step_grouped(tsr_ctx *ctx, const int32_t *idx, int32_t count, const tsr_hyper *hyper,
+                                      void *stream)
+{
+    tsr_status s = check_ready(ctx);
+    if (s != TSR_OK) return s;
+    if ((s = check_hyper(ctx, hyper)) != TSR_OK) return s;
+    std::vector<int> list;
+    if ((s = resolve_list(ctx, idx, count, list)) != TSR_OK) return s;
+    return do_core_update(ctx, list, make_scalars(hyper), (cudaStream_t)stream);
+}
+
+tsr_status tsr_backproject_apply_grouped(tsr_ctx *ctx, const int32_t *idx, int32_t count, const tsr_hyper *hyper,
+                                         void *stream)
+{
+    tsr_status s = check_ready(ctx);
+    if (s != TSR_OK) return s;
+    if ((s = check_hyper(ctx, hyper)) != TSR_OK) return s;
+    std::vector<int> list;
+    if ((s = resolve_list(ctx, idx, count, list)) != TSR_OK) return s;
+    return do_apply(ctx, list, make_scalars(hyper), (cudaStream_t)stream);
+}
+
+tsr_status tsr_embed_step_grouped(tsr_ctx *ctx, const int32_t *idx, int32_t count, const tsr_hyper *hyper,
+                                  uint64_t seed, void *stream)
+{
+    tsr_status s = check_ready(ctx);
+    if (s != TSR_OK) return s;
+    if ((s = check_hyper(ctx, hyper)) != TSR_OK) return s;
+    std::vector<int> list;
+    if (!idx) {
+        for (int i = 0; i < (int)ctx->blocks.size(); ++i) if (ctx->blocks[i].d.is_embedding) list.push_back(i);
+    } else if ((s = resolve_list(ctx, idx, count, list)) != TSR_OK) {
+        return s;
+    }
+    for (int bi : list)
+        if (!ctx->blocks[bi].d.is_embedding) return fail(ctx, TSR_ERR_INVALID_ARG, "block %d is not an embedding", bi);
+    return do_step(ctx, list, hyper, seed, true, (cudaStream_t)stream);
+}
+
+tsr_status tsr_step_grouped(tsr_ctx *ctx, const tsr_hyper *hyper, uint64_t seed, int32_t fuse_adam, void *stream)
+{
+    tsr_status s = check_ready(ctx);
+    if (s != TSR_OK) return s;
+    if ((s = check_hyper(ctx, hyper)) != TSR_OK) return s;
+    std::vector<int> list;
+    resolve_list(ctx, nullptr, 0, list);
+    return do_step(ctx, list, hyper, seed, fuse_adam != 0, (cudaStream_t)stream);
+}
+
+tsr_status tsr_step_grouped_host(tsr_ctx *ctx, const void *const *G_host, float *C_host, const tsr_hyper *hyper,
+                                 uint64_t seed, int32_t fuse_adam, void *stream)
+{
+    tsr_status s = check_ready(ctx);
+    if (s != TSR_OK) return s;
+    if (!G_host) return fail(ctx, TSR_ERR_INVALID_ARG, "G_host is NULL");
+    if ((s = check_hyper(ctx, hyper)) != TSR_OK) return s;
+    cudaStream_t st = (cudaStream_t)stream;
+    const int nb = (int)ctx->blocks.size();
+    for (int i = 0; i < nb; ++i) {
+        const Block &b = ctx->blocks[i];
+        if (!G_host[i]) return fail(ctx, TSR_ERR_INVALID_ARG, "G_host[%d] is NULL", i);
+        const size_t es = (size_t)elem_size(b.d.g_dtype);
+        TSR_CUDA(ctx, cudaMemcpy2DAsync(const_cast<void *>(b.p.G), (size_t)b.d.ldg * es, G_host[i], (size_t)b.d.n * es,
+                                        (size_t)b.d.n * es, (size_t)b.d.m, cudaMemcpyHostToDevice, st));
+    }
+    if ((s = tsr_step_grouped(ctx, hyper, seed, fuse_adam, stream)) != TSR_OK) return s;
+    if (C_host) {
+        size_t off = 0;
+        for (int i = 0; i < nb; ++i) {
+            const Block &b = ctx->blocks[i];
+            const size_t cnt = (size_t)b.d.r * b.d.r;
+            TSR_CUDA(ctx, cudaMemcpyAsync(C_host + off, b.p.C, cnt * sizeof(float), cudaMemcpyDeviceToHost, st));
+            off += cnt;
+        }
+    }
+    TSR_CUDA(ctx, cudaStreamSynchronize(st));
+    return TSR_OK;
+}
+
+// ---- single-block calls ---------------------------------------------------------------------
+tsr_status tsr_init_subspace(tsr_ctx *ctx, int32_t i, uint64_t seed, const float *omega, void *stream)
+{
+    const float *om[1] = {omega};
+    return tsr_init_subspace_grouped(ctx, &i, 1, seed, omega ? om : nullptr, stream);
+}
+tsr_status tsr_rsvd_refresh(tsr_ctx *ctx, int32_t i, uint64_t seed, const float *omega, void *stream)
+{
+    const float *om[1] = {omega};
+    return tsr_rsvd_refresh_grouped(ctx, &i, 1, seed, omega ? om : nullptr, stream);
+}
+tsr_status tsr_project_core(tsr_ctx *ctx, int32_t i, void *stream) { return tsr_project_core_grouped(ctx, &i, 1, stream); }
+tsr_status tsr_adam_core_step(tsr_ctx *ctx, int32_t i, const tsr_hyper *hyper, void *stream)
+{
+    return tsr_adam_core_step_grouped(ctx, &i, 1, hyper, stream);
+}
+tsr_status tsr_backproject_apply(tsr_ctx *ctx, int32_t i, const tsr_hyper *hyper, void *stream)
+{
+    return tsr_backproject_apply_grouped(ctx, &i, 1, hyper, stream);
+}
+tsr_status tsr_embed_step(tsr_ctx *ctx, int32_t i, const tsr_hyper *hyper, uint64_t seed, void *stream)
+{
+    return tsr_embed_step_grouped(ctx, &i, 1, hyper, seed, stream);
+}
+
+// ---- reporting --------------------------------------------------------------------------------
+tsr_status tsr_comm_bytes(const tsr_ctx *ctx, int64_t step, int32_t bytes_per_elem, uint64_t *core, uint64_t *sketch)
+{
+    if (!ctx || !core || !sketch || bytes_per_elem <= 0) return TSR_ERR_INVALID_ARG;
+    uint64_t c = 0, sk = 0;
+    for (const Block &b : ctx->blocks) {
+        c += (uint64_t)b.d.r * (uint64_t)b.d.r * (uint64_t)bytes_per_elem;
+        const bool refresh = step <= 0 || (b.d.K > 0 && step % b.d.K == 0);
+        if (refresh) sk += (uint64_t)b.k * (uint64_t)(b.d.m + b.d.n) * (uint64_t)bytes_per_elem;
+    }
+    *core = c;
+    *sketch = sk;
+    return TSR_OK;
+}
+
+tsr_status tsr_state_elems(const tsr_ctx *ctx, uint64_t *elems)
+{
+    if (!ctx || !elems) return TSR_ERR_INVALID_ARG;
+    uint64_t e = 0;
+    for (const Block &b : ctx->blocks) e += (uint64_t)(b.d.m + b.d.n) * b.d.r + 2ull * b.d.r * b.d.r;
+    *elems = e;
+    return TSR_OK;
+}
+
+tsr_status tsr_poll_status(tsr_ctx *ctx, int32_t *per_block_status, int32_t count, void *stream)
+{
+    tsr_status s = check_ready(ctx);
+    if (s != TSR_OK) return s;
+    if (!per_block_status || count != (int32_t)ctx->blocks.size()) return fail(ctx, TSR_ERR_INVALID_ARG, "bad status array");
+    cudaStream_t st = (cudaStream_t)stream;
+    TSR_CUDA(ctx, cudaMemcpyAsync(per_block_status, ctx->d_status, sizeof(int32_t) * count, cudaMemcpyDeviceToHost, st));
+    TSR_CUDA(ctx, cudaMemsetAsync(ctx->d_status, 0, sizeof(int32_t) * count, st));
+    TSR_CUDA(ctx, cudaStreamSynchronize(st));
+    return TSR_OK;
+}
+
+tsr_status tsr_generate_omega(tsr_ctx *ctx, int32_t i, uint64_t seed, float *out, void *stream)
+{
+    if (!ctx) return TSR_ERR_INVALID_ARG;
+    if (i < 0 || i >= (int32_t)ctx->blocks.size() || !out) return fail(ctx, TSR_ERR_INVALID_ARG, "bad block index or NULL out");
+    int dev_count = 0;
+    if (cudaGetDeviceCount(&dev_count) != cudaSuccess || dev_count <= 0) return fail(ctx, TSR_ERR_CUDA, "no CUDA device available");
+    const Block &b = ctx->blocks[i];
+    TSR_CUDA(ctx, fill_gaussian(out, (int64_t)b.d.n * b.k, seed, (uint64_t)i, (cudaStream_t)stream));
+    return TSR_OK;
+}
+
+int32_t tsr_block_uses_tensor_cores(const tsr_ctx *ctx, int32_t i)
+{
+    if (!ctx || i < 0 || i >= (int32_t)ctx->blocks.size()) return -1;
+    return ctx->blocks[i].fast ? 1 : 0;
+}
+
+}  // extern "C"

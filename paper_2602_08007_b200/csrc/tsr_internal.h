@@ -1,0 +1,145 @@
+// Internal declarations shared by the translation units of libtsr (not part of the C ABI).
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <string>
+#include <vector>
+
+#include "tsr.h"
+
+namespace tsr {
+
+typedef __nv_bfloat16 bf16;
+
+inline int64_t round_up(int64_t x, int64_t a) { return (x + a - 1) / a * a; }
+
+// ---------------------------------------------------------------------------------------
+// Tensor-core grouped GEMM:  D[M x N] = A[M x K] * B[N x K]^T, both operands BF16 with K
+// contiguous ("K-major"), FP32 accumulation in tensor memory.  B may come as two planes
+// (hi + lo) that are accumulated into the same D.
+// ---------------------------------------------------------------------------------------
+enum UmmaEpilogue : int {
+    EPI_STORE_F32 = 0,     // out_f32[row * ld + col] = acc
+    EPI_STORE_BF16 = 1,    // out_bf16[row * ld + col] = bf16(acc)
+    EPI_STORE_BF16_T = 2,  // out_bf16[col * ld + row] = bf16(acc)          (transposed)
+    EPI_CORE_UPDATE = 3,   // acc is a tile of the core C: write C, update M / Vm, write D, D^T as BF16
+    EPI_APPLY = 4          // W[row * ld + col] = decay * W - step_scale * acc
+};
+
+struct alignas(64) UmmaProblem {
+    CUtensorMap tmA;       // box 64 (K) x 128 (M rows), 128-byte swizzle
+    CUtensorMap tmB;       // box 64 (K) x BN (N rows); plane 1 lives plane_rows rows below plane 0
+    int32_t M, N, K;
+    int32_t planes;        // 1 or 2
+    int32_t plane_rows;    // row offset of the second plane inside the B tensor map
+    int32_t block;         // plan index of the matrix block (for status words)
+    int32_t epilogue;      // UmmaEpilogue
+    int32_t pad0;
+    void *out;             // EPI_STORE_*: destination; EPI_APPLY: W; EPI_CORE_UPDATE: C (split-K: partial buffer)
+    int64_t ld_out;
+    int64_t split_stride;  // elements between split-K partial slabs (EPI_STORE_F32 with split tiles)
+    float *mom1;           // EPI_CORE_UPDATE
+    float *mom2;
+    bf16 *d_bf16;          // D   [r x ldd]
+    bf16 *dt_bf16;         // D^T [r x ldd]
+    int64_t ldd;
+};
+
+struct UmmaTile {
+    int32_t prob;
+    int32_t m0, n0;        // element offsets of the tile
+    int32_t kb0, kb1;      // range of 64-wide K blocks [kb0, kb1)
+    int32_t split;         // split-K slab index (0 when not split)
+};
+
+struct StepScalars {       // per-step scalars shared by all blocks
+    float beta1, beta2, eps;
+    float inv_bc1, inv_bc2; // 1 / (1 - beta^t)
+    float decay;            // 1 - lr * weight_decay
+    float step_scale;       // lr * scale
+    int32_t rule;           // tsr_rule
+};
+
+// Launchers (tsr_umma.cu).  tiles / probs are device pointers.  bn = 64, 128 or 256.
+cudaError_t umma_gemm_launch(const UmmaProblem *probs, const UmmaTile *tiles, int num_tiles, int bn, int epilogue,
+                             int planes, const StepScalars &sc, int32_t *status, cudaStream_t stream);
+cudaError_t umma_configure();  // sets the dynamic shared-memory attributes once per process
+
+// ---------------------------------------------------------------------------------------
+// CUDA-core helpers (tsr_simt.cu)
+// ---------------------------------------------------------------------------------------
+enum SimtEpilogue : int { SIMT_STORE = 0, SIMT_APPLY = 1 };
+
+// D[M x N] (ldd) = sum_k A(i,k) B(k,j),  A(i,k) = A[i*sa_i + k*sa_k],  B(k,j) = B[k*sb_k + j*sb_j].
+// a_dtype: TSR_F32 or TSR_BF16; B and D are FP32.  SIMT_APPLY: D = decay * D - step_scale * acc.
+cudaError_t simt_gemm(int M, int N, int K, const void *A, int a_dtype, int64_t sa_i, int64_t sa_k, const float *B,
+                      int64_t sb_k, int64_t sb_j, float *D, int64_t ldd, int epilogue, float decay, float step_scale,
+                      cudaStream_t stream);
+
+struct CoreUpdateArgs {     // one entry per block for the stand-alone core update
+    const float *C;         // r x r, or split-K partial slabs
+    float *Cout;            // where the summed core goes when nsplit > 1 (else unused)
+    float *mom1, *mom2;
+    float *d_f32;           // may be NULL
+    bf16 *d_bf16, *dt_bf16; // may be NULL
+    int64_t ldd;
+    int64_t split_stride;
+    int32_t r, nsplit;
+};
+// Runs the core update for the blocks args_dev[list_dev[0..nblocks)].  mode 0: full update;
+// mode 1: only sum split-K slabs into Cout.
+cudaError_t core_update_launch(const CoreUpdateArgs *args_dev, const int32_t *list_dev, int nblocks, int max_r,
+                               const StepScalars &sc, int mode, cudaStream_t stream);
+
+// BF16 operand copies of a basis X (rows x r, FP32): Xb[rows x ldb] and Xbt[r x ldt].
+cudaError_t make_shadows(const float *X, int rows, int r, bf16 *Xb, int64_t ldb, bf16 *Xbt, int64_t ldt,
+                         cudaStream_t stream);
+// out[cols x ldo] = in[rows x ldi]^T (BF16)
+cudaError_t transpose_bf16(const bf16 *in, int rows, int cols, int64_t ldi, bf16 *out, int64_t ldo, cudaStream_t stream);
+// X (rows x k FP32) -> planes hi / lo of X^T: out[plane][k x ldo]; plane stride = plane_rows * ldo elements.
+cudaError_t split_transpose(const float *X, int rows, int k, bf16 *out, int64_t ldo, int plane_rows, int planes,
+                            cudaStream_t stream);
+cudaError_t fill_gaussian(float *out, int64_t count, uint64_t seed, uint64_t stream_id, cudaStream_t stream);
+cudaError_t fill_zero_f32(float *p, int64_t count, cudaStream_t stream);
+
+// ---------------------------------------------------------------------------------------
+// Small dense linear algebra for the refresh (tsr_linalg.cu).  All launchers are batched over
+// a list of blocks; the per-block pointers live in a device-resident RefreshDev table.
+// ---------------------------------------------------------------------------------------
+struct RefreshDev {
+    int32_t m, n, k, r;
+    float *buf[3];      // three scratch matrices, each max(m, n) x k FP32
+    double *S;          // k x k Gram matrix / Cholesky factor
+    double *Xw;         // k x k work (inverse factor)
+    double *Wj;         // k x k eigenvectors
+    double *gpart;      // Gram partial sums, gram_chunks(max(m, n)) * k * k
+    double *lam;        // k eigenvalues, descending
+    float *Rinv;        // k x k
+    float *Wu, *Wv;     // k x r
+    float *U, *V;       // the block's bases (FP32 masters)
+    int32_t *status;    // the block's status word
+};
+struct RowItem { int32_t block; int32_t row0; };   // a slab of rows of one block
+
+constexpr int GRAM_ROWS = 2048;   // rows per Gram work item
+constexpr int RG_ROWS = 64;       // rows per rows_gemm work item
+__host__ __device__ inline int gram_chunks(int64_t rows) { return (int)((rows + GRAM_ROWS - 1) / GRAM_ROWS); }
+
+// side: 0 = matrices with m rows, 1 = matrices with n rows.
+// S = X^T X with X = buf[src_sel] (FP32), FP64 accumulation, deterministic.
+cudaError_t gram_batched(const RefreshDev *rd, const RowItem *items, int nitems, const int32_t *list, int nlist,
+                         int side, int src_sel, int kmax, cudaStream_t stream);
+// Cholesky S = R^T R in place and Rinv = float(R^{-1}).
+cudaError_t chol_inverse_batched(const RefreshDev *rd, const int32_t *list, int nlist, cudaStream_t stream);
+// dst = buf[src_sel] * Mat;  mat_sel: 0 Rinv (k x k), 1 Wu (k x r), 2 Wv (k x r);
+// dst_sel: 0..2 buf[], 3 = U, 4 = V.
+cudaError_t rows_gemm_batched(const RefreshDev *rd, const RowItem *items, int nitems, int side, int src_sel,
+                              int mat_sel, int dst_sel, int nmax, cudaStream_t stream);
+// Eigen-decomposition of S by cyclic Jacobi, descending sort, Wu = W[:, :r], Wv = W[:, :r] / sqrt(lambda).
+cudaError_t jacobi_batched(const RefreshDev *rd, const int32_t *list, int nlist, int max_sweeps, cudaStream_t stream);
+
+}  // namespace tsr

@@ -1,0 +1,372 @@
+// Small dense linear algebra of the subspace refresh (Section 3.5), batched over blocks:
+// Gram matrices in FP64, Cholesky factor and its inverse (orth = Cholesky-QR applied twice),
+// tall-times-small products, and a cyclic Jacobi eigen-solver on the k x k Gram matrix of B^T
+// that yields the small SVD.
+//
+// All kernels are bounded loops; anything that goes wrong numerically (a non-positive pivot,
+// a non-finite entry, the sweep limit) is written to the block's status word.
+#include "tsr_internal.h"
+
+namespace tsr {
+
+// ---------------------------------------------------------------------------------------
+// S = X^T X, X rows x k FP32, accumulation in FP64.  Rows are cut into slabs of GRAM_ROWS;
+// each slab writes its own partial (upper-triangular tiles only), a second kernel adds the
+// partials in slab order and mirrors the result, so the sum is deterministic.
+// ---------------------------------------------------------------------------------------
+constexpr int GR_T = 32;  // output tile edge
+
+__global__ void __launch_bounds__(256)
+gram_partial_kernel(const RefreshDev *__restrict__ rd, const RowItem *__restrict__ items, int side, int src_sel)
+{
+    const RowItem it = items[blockIdx.z];
+    const RefreshDev d = rd[it.block];
+    const int k = d.k;
+    const int ti = blockIdx.y, tj = blockIdx.x;
+    if (tj < ti || ti * GR_T >= k || tj * GR_T >= k) return;
+    const int rows = side ? d.n : d.m;
+    const float *__restrict__ X = d.buf[src_sel];
+    __shared__ float Xi[16][GR_T + 1];
+    __shared__ float Xj[16][GR_T + 1];
+    const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;  // 16 x 16 threads, 2 x 2 outputs each
+    const int row_begin = it.row0;
+    const int row_end = min(rows, row_begin + GRAM_ROWS);
+    double acc[2][2] = {{0.0, 0.0}, {0.0, 0.0}};
+    for (int r0 = row_begin; r0 < row_end; r0 += 16) {
+        for (int e = threadIdx.x; e < 16 * GR_T; e += 256) {
+            const int rr = e / GR_T, cc = e % GR_T;
+            const int row = r0 + rr;
+            const int ci = ti * GR_T + cc, cj = tj * GR_T + cc;
+            Xi[rr][cc] = (row < row_end && ci < k) ? X[(int64_t)row * k + ci] : 0.f;
+            Xj[rr][cc] = (row < row_end && cj < k) ? X[(int64_t)row * k + cj] : 0.f;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int rr = 0; rr < 16; ++rr) {
+            const double a0 = Xi[rr][ty * 2], a1 = Xi[rr][ty * 2 + 1];
+            const double b0 = Xj[rr][tx * 2], b1 = Xj[rr][tx * 2 + 1];
+            acc[0][0] += a0 * b0; acc[0][1] += a0 * b1;
+            acc[1][0] += a1 * b0; acc[1][1] += a1 * b1;
+        }
+        __syncthreads();
+    }
+    double *P = d.gpart + (int64_t)(it.row0 / GRAM_ROWS) * k * k;
+#pragma unroll
+    for (int a = 0; a < 2; ++a)
+#pragma unroll
+        for (int b = 0; b < 2; ++b) {
+            const int i = ti * GR_T + ty * 2 + a, j = tj * GR_T + tx * 2 + b;
+            if (i < k && j < k) P[(int64_t)i * k + j] = acc[a][b];
+        }
+}
+
+__global__ void gram_reduce_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ list, int side)
+{
+    const RefreshDev d = rd[list[blockIdx.y]];
+    const int k = d.k;
+    const int chunks = gram_chunks(side ? d.n : d.m);
+    const int64_t total = (int64_t)k * k;
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
+        const int i = (int)(e / k), j = (int)(e % k);
+        const bool upper = (j / GR_T) >= (i / GR_T);  // only tiles with tj >= ti were written
+        const int64_t src = upper ? e : (int64_t)j * k + i;
+        double s = 0.0;
+        for (int c = 0; c < chunks; ++c) s += d.gpart[(int64_t)c * total + src];
+        d.S[e] = s;
+    }
+}
+
+cudaError_t gram_batched(const RefreshDev *rd, const RowItem *items, int nitems, const int32_t *list, int nlist,
+                         int side, int src_sel, int kmax, cudaStream_t stream)
+{
+    if (nitems <= 0 || nlist <= 0) return cudaSuccess;
+    const int t = (kmax + GR_T - 1) / GR_T;
+    gram_partial_kernel<<<dim3(t, t, nitems), 256, 0, stream>>>(rd, items, side, src_sel);
+    int gx = (int)(((int64_t)kmax * kmax + 255) / 256);
+    if (gx > 128) gx = 128;
+    gram_reduce_kernel<<<dim3(gx, nlist), 256, 0, stream>>>(rd, list, side);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------
+// Cholesky S = R^T R with R upper triangular (one CTA per matrix, FP64, in place), followed by
+// Rinv = R^{-1} written as FP32.  A pivot that is not safely positive is replaced by a floor
+// relative to the largest diagonal entry and the block is flagged TSR_ERR_RANK_DEFICIENT.
+// ---------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(1024)
+chol_inverse_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ list)
+{
+    const RefreshDev d = rd[list[blockIdx.x]];
+    const int k = d.k;
+    double *__restrict__ S = d.S;
+    double *__restrict__ X = d.Xw;
+    __shared__ double s_piv;
+    __shared__ double s_floor;
+    __shared__ int s_flag;
+    const int tid = threadIdx.x, nt = blockDim.x;
+    if (tid == 0) {
+        double mx = 0.0;
+        int bad = 0;
+        for (int i = 0; i < k; ++i) {
+            const double v = S[(int64_t)i * k + i];
+            if (!(v == v) || v > 1e300 || v < -1e300) bad = 1;
+            if (v > mx) mx = v;
+        }
+        s_floor = mx * 1e-13;
+        if (!(s_floor > 0.0)) s_floor = 1e-300;
+        s_flag = bad ? TSR_ERR_NONFINITE : 0;
+    }
+    __syncthreads();
+    for (int j = 0; j < k; ++j) {
+        if (tid == 0) {
+            double v = S[(int64_t)j * k + j];
+            if (!(v > s_floor)) {
+                if (s_flag == 0) s_flag = TSR_ERR_RANK_DEFICIENT;
+                v = s_floor;
+            }
+            s_piv = sqrt(v);
+        }
+        __syncthreads();
+        const double piv = s_piv;
+        for (int l = j + tid; l < k; l += nt) S[(int64_t)j * k + l] = (l == j) ? piv : S[(int64_t)j * k + l] / piv;
+        __syncthreads();
+        // trailing update of the upper triangle: S[i][l] -= R[j][i] R[j][l], j < i <= l
+        const int rem = k - j - 1;
+        for (int64_t e = tid; e < (int64_t)rem * rem; e += nt) {
+            const int i = j + 1 + (int)(e / rem), l = j + 1 + (int)(e % rem);
+            if (l >= i) S[(int64_t)i * k + l] -= S[(int64_t)j * k + i] * S[(int64_t)j * k + l];
+        }
+        __syncthreads();
+    }
+    // X = R^{-1} (upper): column c by back substitution, one thread per column
+    for (int c = tid; c < k; c += nt) {
+        for (int i = c; i >= 0; --i) {
+            double s = (i == c) ? 1.0 : 0.0;
+            for (int l = i + 1; l <= c; ++l) s -= S[(int64_t)i * k + l] * X[(int64_t)l * k + c];
+            X[(int64_t)i * k + c] = s / S[(int64_t)i * k + i];
+        }
+        for (int i = c + 1; i < k; ++i) X[(int64_t)i * k + c] = 0.0;
+    }
+    __syncthreads();
+    for (int64_t e = tid; e < (int64_t)k * k; e += nt) d.Rinv[e] = (float)X[e];
+    if (tid == 0 && s_flag != 0) atomicMax(d.status, s_flag);
+}
+
+cudaError_t chol_inverse_batched(const RefreshDev *rd, const int32_t *list, int nlist, cudaStream_t stream)
+{
+    if (nlist <= 0) return cudaSuccess;
+    chol_inverse_kernel<<<nlist, 1024, 0, stream>>>(rd, list);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------
+// dst[rows x N] = src[rows x k] * Mat[k x N]   (FP32, 64 x 64 tiles, one slab of 64 rows per item)
+// ---------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+rows_gemm_kernel(const RefreshDev *__restrict__ rd, const RowItem *__restrict__ items, int side, int src_sel,
+                 int mat_sel, int dst_sel)
+{
+    const RowItem it = items[blockIdx.y];
+    const RefreshDev d = rd[it.block];
+    const int K = d.k;
+    const int N = (mat_sel == 0) ? d.k : d.r;
+    const int n0 = blockIdx.x * 64;
+    if (n0 >= N) return;
+    const int rows = side ? d.n : d.m;
+    const float *__restrict__ A = d.buf[src_sel];
+    const float *__restrict__ B = (mat_sel == 0) ? d.Rinv : (mat_sel == 1 ? d.Wu : d.Wv);
+    float *__restrict__ D = (dst_sel < 3) ? d.buf[dst_sel] : (dst_sel == 3 ? d.U : d.V);
+    const int m0 = it.row0;
+
+    __shared__ float As[16][64 + 4];
+    __shared__ float Bs[16][64 + 4];
+    const int tid = threadIdx.x, tx = tid % 16, ty = tid / 16;
+    float acc[4][4];
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+        for (int b = 0; b < 4; ++b) acc[a][b] = 0.f;
+    for (int k0 = 0; k0 < K; k0 += 16) {
+#pragma unroll
+        for (int l = 0; l < 4; ++l) {
+            const int e = tid + l * 256;
+            const int ak = e % 16, ai = e / 16;
+            const int gi = m0 + ai, gk = k0 + ak;
+            As[ak][ai] = (gi < rows && gk < K) ? A[(int64_t)gi * K + gk] : 0.f;
+            const int bj = e % 64, bk = e / 64;
+            const int gj = n0 + bj, gk2 = k0 + bk;
+            Bs[bk][bj] = (gj < N && gk2 < K) ? B[(int64_t)gk2 * N + gj] : 0.f;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int kk = 0; kk < 16; ++kk) {
+            float av[4], bv[4];
+#pragma unroll
+            for (int a = 0; a < 4; ++a) av[a] = As[kk][ty * 4 + a];
+#pragma unroll
+            for (int b = 0; b < 4; ++b) bv[b] = Bs[kk][tx * 4 + b];
+#pragma unroll
+            for (int a = 0; a < 4; ++a)
+#pragma unroll
+                for (int b = 0; b < 4; ++b) acc[a][b] = fmaf(av[a], bv[b], acc[a][b]);
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int a = 0; a < 4; ++a) {
+        const int gi = m0 + ty * 4 + a;
+        if (gi >= rows) continue;
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+            const int gj = n0 + tx * 4 + b;
+            if (gj < N) D[(int64_t)gi * N + gj] = acc[a][b];
+        }
+    }
+}
+
+cudaError_t rows_gemm_batched(const RefreshDev *rd, const RowItem *items, int nitems, int side, int src_sel,
+                              int mat_sel, int dst_sel, int nmax, cudaStream_t stream)
+{
+    if (nitems <= 0) return cudaSuccess;
+    rows_gemm_kernel<<<dim3((nmax + 63) / 64, nitems), 256, 0, stream>>>(rd, items, side, src_sel, mat_sel, dst_sel);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------
+// Cyclic Jacobi eigen-solver for a symmetric k x k matrix (FP64), one CTA per matrix.
+// Round-robin ordering: every round rotates k/2 disjoint index pairs at once; the two-sided
+// update S <- J^T S J is done on 2 x 2 blocks (pair A rows x pair B columns), the eigenvector
+// accumulation W <- W J on rows of W.  Stops after a sweep without any rotation, or after
+// max_sweeps (then flags TSR_ERR_NOT_CONVERGED).
+// Afterwards eigenvalues are ranked in descending order and the leading r eigenvectors are
+// written out: Wu = W[:, :r]; Wv = W[:, :r] / sqrt(lambda)  (B^T W / sigma = right vectors).
+// ---------------------------------------------------------------------------------------
+constexpr int JAC_MAX_K = 1056;
+
+__global__ void __launch_bounds__(1024)
+jacobi_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ list, int max_sweeps)
+{
+    const RefreshDev d = rd[list[blockIdx.x]];
+    const int k = d.k, r = d.r;
+    double *__restrict__ S = d.S;
+    double *__restrict__ W = d.Wj;
+    __shared__ double s_c[JAC_MAX_K / 2], s_s[JAC_MAX_K / 2];
+    __shared__ short s_p[JAC_MAX_K / 2], s_q[JAC_MAX_K / 2];
+    __shared__ int s_rot;
+    __shared__ int s_flag;
+    const int tid = threadIdx.x, nt = blockDim.x;
+    const int ke = (k + 1) & ~1;  // even number of slots; slot k (if any) is a bye
+    const int np = ke / 2;
+
+    for (int64_t e = tid; e < (int64_t)k * k; e += nt) W[e] = ((e / k) == (e % k)) ? 1.0 : 0.0;
+    if (tid == 0) s_flag = 0;
+    __syncthreads();
+
+    bool converged = false;
+    for (int sweep = 0; sweep < max_sweeps && !converged; ++sweep) {
+        if (tid == 0) s_rot = 0;
+        __syncthreads();
+        for (int round = 0; round < ke - 1; ++round) {
+            for (int i = tid; i < np; i += nt) {
+                int a, b;
+                if (i == 0) { a = ke - 1; b = round % (ke - 1); }
+                else { a = (round + i) % (ke - 1); b = (round + ke - 1 - i) % (ke - 1); }
+                int p = min(a, b), q = max(a, b);
+                double c = 1.0, s = 0.0;
+                if (q < k) {
+                    const double spp = S[(int64_t)p * k + p], sqq = S[(int64_t)q * k + q], spq = S[(int64_t)p * k + q];
+                    if (spq != 0.0 && fabs(spq) > 1e-15 * sqrt(fabs(spp * sqq))) {
+                        const double zeta = (sqq - spp) / (2.0 * spq);
+                        const double t = ((zeta >= 0.0) ? 1.0 : -1.0) / (fabs(zeta) + sqrt(1.0 + zeta * zeta));
+                        c = 1.0 / sqrt(1.0 + t * t);
+                        s = c * t;
+                        atomicAdd(&s_rot, 1);
+                    }
+                } else {
+                    q = -1;  // bye: p has no partner this round
+                }
+                s_c[i] = c; s_s[i] = s; s_p[i] = (short)p; s_q[i] = (short)q;
+            }
+            __syncthreads();
+            // S <- J^T S J on 2 x 2 blocks; every entry belongs to exactly one (A, B) block
+            for (int e = tid; e < np * np; e += nt) {
+                const int A = e / np, B = e % np;
+                const int pA = s_p[A], qA = s_q[A], pB = s_p[B], qB = s_q[B];
+                const double cA = s_c[A], sA = s_s[A], cB = s_c[B], sB = s_s[B];
+                if (sA == 0.0 && sB == 0.0) continue;
+                if (qA < 0 && qB < 0) continue;
+                if (qA < 0) {  // single row pA, column pair B
+                    const double x = S[(int64_t)pA * k + pB], y = S[(int64_t)pA * k + qB];
+                    S[(int64_t)pA * k + pB] = cB * x - sB * y;
+                    S[(int64_t)pA * k + qB] = sB * x + cB * y;
+                    continue;
+                }
+                if (qB < 0) {  // row pair A, single column pB
+                    const double x = S[(int64_t)pA * k + pB], y = S[(int64_t)qA * k + pB];
+                    S[(int64_t)pA * k + pB] = cA * x - sA * y;
+                    S[(int64_t)qA * k + pB] = sA * x + cA * y;
+                    continue;
+                }
+                double x00 = S[(int64_t)pA * k + pB], x01 = S[(int64_t)pA * k + qB];
+                double x10 = S[(int64_t)qA * k + pB], x11 = S[(int64_t)qA * k + qB];
+                const double r00 = cA * x00 - sA * x10, r01 = cA * x01 - sA * x11;  // rows: J_A^T
+                const double r10 = sA * x00 + cA * x10, r11 = sA * x01 + cA * x11;
+                x00 = cB * r00 - sB * r01; x01 = sB * r00 + cB * r01;                // columns: J_B
+                x10 = cB * r10 - sB * r11; x11 = sB * r10 + cB * r11;
+                if (A == B) { x01 = 0.0; x10 = 0.0; }
+                S[(int64_t)pA * k + pB] = x00; S[(int64_t)pA * k + qB] = x01;
+                S[(int64_t)qA * k + pB] = x10; S[(int64_t)qA * k + qB] = x11;
+            }
+            // W <- W J
+            for (int e = tid; e < k * np; e += nt) {
+                const int i = e / np, B = e % np;
+                const int qB = s_q[B];
+                const double sB = s_s[B];
+                if (qB < 0 || sB == 0.0) continue;
+                const int pB = s_p[B];
+                const double cB = s_c[B];
+                const double x = W[(int64_t)i * k + pB], y = W[(int64_t)i * k + qB];
+                W[(int64_t)i * k + pB] = cB * x - sB * y;
+                W[(int64_t)i * k + qB] = sB * x + cB * y;
+            }
+            __syncthreads();
+        }
+        converged = (s_rot == 0);
+        __syncthreads();
+    }
+    if (tid == 0 && !converged) s_flag = TSR_ERR_NOT_CONVERGED;
+    __syncthreads();
+
+    // rank eigenvalues (descending; ties by index) and emit the leading r columns
+    for (int j = tid; j < k; j += nt) {
+        const double lj = S[(int64_t)j * k + j];
+        if (!(lj == lj)) s_flag = TSR_ERR_NONFINITE;
+        int rank = 0;
+        for (int l = 0; l < k; ++l) {
+            const double ll = S[(int64_t)l * k + l];
+            rank += (ll > lj || (ll == lj && l < j)) ? 1 : 0;
+        }
+        d.lam[rank] = lj;
+        if (rank < r) {
+            double inv = 0.0;
+            if (lj > 1e-300) inv = 1.0 / sqrt(lj);
+            else s_flag = TSR_ERR_RANK_DEFICIENT;
+            for (int i = 0; i < k; ++i) {
+                const double w = W[(int64_t)i * k + j];
+                d.Wu[(int64_t)i * r + rank] = (float)w;
+                d.Wv[(int64_t)i * r + rank] = (float)(w * inv);
+            }
+        }
+    }
+    __syncthreads();
+    if (tid == 0 && s_flag != 0) atomicMax(d.status, s_flag);
+}
+
+cudaError_t jacobi_batched(const RefreshDev *rd, const int32_t *list, int nlist, int max_sweeps, cudaStream_t stream)
+{
+    if (nlist <= 0) return cudaSuccess;
+    jacobi_kernel<<<nlist, 1024, 0, stream>>>(rd, list, max_sweeps);
+    return cudaGetLastError();
+}
+
+}  // namespace tsr

@@ -1,0 +1,279 @@
+// CUDA-core kernels of libtsr: the all-FP32 path (FP32 gradients, or buffers that miss the
+// 16-byte alignment the tensor-core path needs), the stand-alone core update (Section 3.4),
+// operand conversion for the tensor-core path, and the Gaussian generator for Omega.
+#include "tsr_internal.h"
+#include "tsr_device.cuh"
+
+namespace tsr {
+
+// ---------------------------------------------------------------------------------------
+// Generic strided FP32 GEMM, 64 x 64 output tile, 16-deep K slices, 4 x 4 outputs per thread.
+// ---------------------------------------------------------------------------------------
+template <typename TA>
+__device__ __forceinline__ float load_as_float(const TA *p);
+template <>
+__device__ __forceinline__ float load_as_float<float>(const float *p) { return *p; }
+template <>
+__device__ __forceinline__ float load_as_float<bf16>(const bf16 *p) { return __bfloat162float(*p); }
+
+constexpr int SG_BM = 64, SG_BN = 64, SG_BK = 16;
+
+template <typename TA, int EPI>
+__global__ void __launch_bounds__(256)
+simt_gemm_kernel(int M, int N, int K, const TA *__restrict__ A, int64_t sa_i, int64_t sa_k,
+                 const float *__restrict__ B, int64_t sb_k, int64_t sb_j, float *__restrict__ D, int64_t ldd,
+                 float decay, float step_scale)
+{
+    __shared__ float As[SG_BK][SG_BM + 4];
+    __shared__ float Bs[SG_BK][SG_BN + 4];
+    const int tid = threadIdx.x;
+    const int tx = tid % 16, ty = tid / 16;
+    const int m0 = blockIdx.y * SG_BM, n0 = blockIdx.x * SG_BN;
+
+    float acc[4][4];
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+        for (int b = 0; b < 4; ++b) acc[a][b] = 0.f;
+
+    // Loader index maps: put the unit-stride index on consecutive threads.
+    const bool a_k_fast = (sa_k == 1);
+    const bool b_j_fast = (sb_j == 1);
+
+    for (int k0 = 0; k0 < K; k0 += SG_BK) {
+#pragma unroll
+        for (int l = 0; l < 4; ++l) {
+            const int e = tid + l * 256;  // 0..1023
+            int ai, ak;
+            if (a_k_fast) { ak = e % SG_BK; ai = e / SG_BK; } else { ai = e % SG_BM; ak = e / SG_BM; }
+            const int gi = m0 + ai, gk = k0 + ak;
+            As[ak][ai] = (gi < M && gk < K) ? load_as_float<TA>(A + (int64_t)gi * sa_i + (int64_t)gk * sa_k) : 0.f;
+            int bj, bk;
+            if (b_j_fast) { bj = e % SG_BN; bk = e / SG_BN; } else { bk = e % SG_BK; bj = e / SG_BK; }
+            const int gj = n0 + bj, gk2 = k0 + bk;
+            Bs[bk][bj] = (gj < N && gk2 < K) ? B[(int64_t)gk2 * sb_k + (int64_t)gj * sb_j] : 0.f;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int kk = 0; kk < SG_BK; ++kk) {
+            float av[4], bv[4];
+#pragma unroll
+            for (int a = 0; a < 4; ++a) av[a] = As[kk][ty * 4 + a];
+#pragma unroll
+            for (int b = 0; b < 4; ++b) bv[b] = Bs[kk][tx * 4 + b];
+#pragma unroll
+            for (int a = 0; a < 4; ++a)
+#pragma unroll
+                for (int b = 0; b < 4; ++b) acc[a][b] = fmaf(av[a], bv[b], acc[a][b]);
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int a = 0; a < 4; ++a) {
+        const int gi = m0 + ty * 4 + a;
+        if (gi >= M) continue;
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+            const int gj = n0 + tx * 4 + b;
+            if (gj >= N) continue;
+            float *d = D + (int64_t)gi * ldd + gj;
+            if (EPI == SIMT_APPLY) {
+                *d = __fmaf_rn(-step_scale, acc[a][b], __fmul_rn(decay, *d));
+            } else {
+                *d = acc[a][b];
+            }
+        }
+    }
+}
+
+cudaError_t simt_gemm(int M, int N, int K, const void *A, int a_dtype, int64_t sa_i, int64_t sa_k, const float *B,
+                      int64_t sb_k, int64_t sb_j, float *D, int64_t ldd, int epilogue, float decay, float step_scale,
+                      cudaStream_t stream)
+{
+    if (M <= 0 || N <= 0) return cudaSuccess;
+    dim3 grid((N + SG_BN - 1) / SG_BN, (M + SG_BM - 1) / SG_BM);
+    if (a_dtype == TSR_BF16) {
+        if (epilogue == SIMT_APPLY)
+            simt_gemm_kernel<bf16, SIMT_APPLY><<<grid, 256, 0, stream>>>(M, N, K, (const bf16 *)A, sa_i, sa_k, B, sb_k, sb_j, D, ldd, decay, step_scale);
+        else
+            simt_gemm_kernel<bf16, SIMT_STORE><<<grid, 256, 0, stream>>>(M, N, K, (const bf16 *)A, sa_i, sa_k, B, sb_k, sb_j, D, ldd, decay, step_scale);
+    } else {
+        if (epilogue == SIMT_APPLY)
+            simt_gemm_kernel<float, SIMT_APPLY><<<grid, 256, 0, stream>>>(M, N, K, (const float *)A, sa_i, sa_k, B, sb_k, sb_j, D, ldd, decay, step_scale);
+        else
+            simt_gemm_kernel<float, SIMT_STORE><<<grid, 256, 0, stream>>>(M, N, K, (const float *)A, sa_i, sa_k, B, sb_k, sb_j, D, ldd, decay, step_scale);
+    }
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------
+// Core-space update (Section 3.4; Algorithm 2 for the SGD rule).  The same arithmetic, with
+// the same explicit rounding steps, is used by the tensor-core projection epilogue so that
+// the fused and the unfused orders agree bit for bit.
+// ---------------------------------------------------------------------------------------
+// mode 0: full update; mode 1: only sum the split-K slabs into Cout.
+__global__ void core_update_kernel(const CoreUpdateArgs *__restrict__ args, const int32_t *__restrict__ list,
+                                   StepScalars sc, int mode)
+{
+    const CoreUpdateArgs a = args[list[blockIdx.y]];
+    const int r = a.r;
+    const int64_t total = (int64_t)r * r;
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
+        float c = a.C[e];
+        if (a.nsplit > 1) {
+            for (int s = 1; s < a.nsplit; ++s) c = __fadd_rn(c, a.C[e + (int64_t)s * a.split_stride]);
+            a.Cout[e] = c;
+        }
+        if (mode == 1) continue;
+        float m1 = a.mom1[e];
+        float m2 = (sc.rule == TSR_RULE_SGD) ? 0.f : a.mom2[e];
+        const float d = core_update_elem(c, m1, m2, sc);
+        a.mom1[e] = m1;
+        if (sc.rule != TSR_RULE_SGD) a.mom2[e] = m2;
+        if (a.d_f32) a.d_f32[e] = d;
+        const int row = (int)(e / r), col = (int)(e % r);
+        if (a.d_bf16) a.d_bf16[(int64_t)row * a.ldd + col] = __float2bfloat16_rn(d);
+        if (a.dt_bf16) a.dt_bf16[(int64_t)col * a.ldd + row] = __float2bfloat16_rn(d);
+    }
+}
+
+cudaError_t core_update_launch(const CoreUpdateArgs *args_dev, const int32_t *list_dev, int nblocks, int max_r,
+                               const StepScalars &sc, int mode, cudaStream_t stream)
+{
+    if (nblocks <= 0) return cudaSuccess;
+    int gx = (int)(((int64_t)max_r * max_r + 255) / 256);
+    if (gx > 64) gx = 64;
+    if (gx < 1) gx = 1;
+    core_update_kernel<<<dim3(gx, nblocks), 256, 0, stream>>>(args_dev, list_dev, sc, mode);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------
+// Operand conversion
+// ---------------------------------------------------------------------------------------
+__global__ void shadows_kernel(const float *__restrict__ X, int rows, int r, bf16 *__restrict__ Xb, int64_t ldb,
+                               bf16 *__restrict__ Xbt, int64_t ldt)
+{
+    __shared__ float tile[32][33];
+    const int r0 = blockIdx.y * 32, c0 = blockIdx.x * 32;
+    for (int i = threadIdx.y; i < 32; i += blockDim.y) {
+        const int row = r0 + i, col = c0 + threadIdx.x;
+        float v = 0.f;
+        if (row < rows && col < r) {
+            v = X[(int64_t)row * r + col];
+            if (Xb) Xb[(int64_t)row * ldb + col] = __float2bfloat16_rn(v);
+        }
+        tile[i][threadIdx.x] = v;
+    }
+    __syncthreads();
+    if (Xbt) {
+        for (int i = threadIdx.y; i < 32; i += blockDim.y) {
+            const int col = c0 + i, row = r0 + threadIdx.x;
+            if (row < rows && col < r) Xbt[(int64_t)col * ldt + row] = __float2bfloat16_rn(tile[threadIdx.x][i]);
+        }
+    }
+}
+
+cudaError_t make_shadows(const float *X, int rows, int r, bf16 *Xb, int64_t ldb, bf16 *Xbt, int64_t ldt,
+                         cudaStream_t stream)
+{
+    dim3 grid((r + 31) / 32, (rows + 31) / 32);
+    shadows_kernel<<<grid, dim3(32, 8), 0, stream>>>(X, rows, r, Xb, ldb, Xbt, ldt);
+    return cudaGetLastError();
+}
+
+__global__ void transpose_bf16_kernel(const bf16 *__restrict__ in, int rows, int cols, int64_t ldi,
+                                      bf16 *__restrict__ out, int64_t ldo)
+{
+    __shared__ bf16 tile[64][66];
+    const int r0 = blockIdx.y * 64, c0 = blockIdx.x * 64;
+    for (int i = threadIdx.y; i < 64; i += blockDim.y)
+        for (int j = threadIdx.x; j < 64; j += blockDim.x) {
+            const int row = r0 + i, col = c0 + j;
+            tile[i][j] = (row < rows && col < cols) ? in[(int64_t)row * ldi + col] : __float2bfloat16_rn(0.f);
+        }
+    __syncthreads();
+    for (int i = threadIdx.y; i < 64; i += blockDim.y)
+        for (int j = threadIdx.x; j < 64; j += blockDim.x) {
+            const int col = c0 + i, row = r0 + j;
+            if (row < rows && col < cols) out[(int64_t)col * ldo + row] = tile[j][i];
+        }
+}
+
+cudaError_t transpose_bf16(const bf16 *in, int rows, int cols, int64_t ldi, bf16 *out, int64_t ldo, cudaStream_t stream)
+{
+    dim3 grid((cols + 63) / 64, (rows + 63) / 64);
+    transpose_bf16_kernel<<<grid, dim3(32, 8), 0, stream>>>(in, rows, cols, ldi, out, ldo);
+    return cudaGetLastError();
+}
+
+// X (rows x k) FP32 -> X^T as BF16 planes: hi = bf16(x), lo = bf16(x - hi).
+__global__ void split_transpose_kernel(const float *__restrict__ X, int rows, int k, bf16 *__restrict__ out,
+                                       int64_t ldo, int plane_rows, int planes)
+{
+    __shared__ float tile[32][33];
+    const int r0 = blockIdx.y * 32, c0 = blockIdx.x * 32;
+    for (int i = threadIdx.y; i < 32; i += blockDim.y) {
+        const int row = r0 + i, col = c0 + threadIdx.x;
+        tile[i][threadIdx.x] = (row < rows && col < k) ? X[(int64_t)row * k + col] : 0.f;
+    }
+    __syncthreads();
+    for (int i = threadIdx.y; i < 32; i += blockDim.y) {
+        const int col = c0 + i, row = r0 + threadIdx.x;
+        if (row < rows && col < k) {
+            const float v = tile[threadIdx.x][i];
+            const bf16 hi = __float2bfloat16_rn(v);
+            out[(int64_t)col * ldo + row] = hi;
+            if (planes > 1)
+                out[((int64_t)plane_rows + col) * ldo + row] = __float2bfloat16_rn(v - __bfloat162float(hi));
+        }
+    }
+}
+
+cudaError_t split_transpose(const float *X, int rows, int k, bf16 *out, int64_t ldo, int plane_rows, int planes,
+                            cudaStream_t stream)
+{
+    dim3 grid((k + 31) / 32, (rows + 31) / 32);
+    split_transpose_kernel<<<grid, dim3(32, 8), 0, stream>>>(X, rows, k, out, ldo, plane_rows, planes);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------
+// Counter-based N(0,1) generator for Omega (Algorithm 1, "Sample shared Omega (shared RNG
+// seed)"): element e of stream `stream_id` hashes (seed, stream_id, e) with two rounds of a
+// 64-bit mixer, then Box-Muller on the two 32-bit halves.  Independent of the launch shape.
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ uint64_t mix64(uint64_t z)
+{
+    z += 0x9E3779B97F4A7C15ull;
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    return z ^ (z >> 31);
+}
+
+__global__ void gaussian_kernel(float *__restrict__ out, int64_t count, uint64_t seed, uint64_t stream_id)
+{
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < count; e += (int64_t)gridDim.x * blockDim.x) {
+        const uint64_t h = mix64(mix64(seed ^ (stream_id * 0xD1342543DE82EF95ull)) + (uint64_t)e);
+        const uint32_t a = (uint32_t)h, b = (uint32_t)(h >> 32);
+        const float u1 = ((float)(a >> 8) + 0.5f) * (1.0f / 16777216.0f);  // (0,1)
+        const float u2 = ((float)(b >> 8) + 0.5f) * (1.0f / 16777216.0f);
+        out[e] = sqrtf(-2.0f * logf(u1)) * cospif(2.0f * u2);
+    }
+}
+
+cudaError_t fill_gaussian(float *out, int64_t count, uint64_t seed, uint64_t stream_id, cudaStream_t stream)
+{
+    if (count <= 0) return cudaSuccess;
+    int64_t blocks = (count + 255) / 256;
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    gaussian_kernel<<<(int)blocks, 256, 0, stream>>>(out, count, seed, stream_id);
+    return cudaGetLastError();
+}
+
+cudaError_t fill_zero_f32(float *p, int64_t count, cudaStream_t stream)
+{
+    return cudaMemsetAsync(p, 0, (size_t)count * sizeof(float), stream);
+}
+
+}  // namespace tsr

@@ -1,0 +1,297 @@
+"""GPU parity: the CUDA library (through its C ABI) against the FP64 CPU oracle, element by
+element on the same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import tsr_inputs as ti
+from helpers import (TOL_BF16, TOL_F32, check_refresh, fill_gradient, fill_weights, rel_fro, set_bases, to64)
+
+pytestmark = pytest.mark.gpu
+
+
+def _plan(blocks, dtype):
+    import paper_2602_08007_b200 as tsr
+    return tsr, tsr.Plan(blocks, g_dtype=dtype)
+
+
+def _run_steps(tsr, plan, shapes, dtype, steps, fuse, tol, wd=0.0, scale=1.0, rule=0, cfg=90):
+    """Given bases already in the plan: lock-step `steps` optimizer steps against the oracle."""
+    nb = len(shapes)
+    blks = []
+    for i, s in enumerate(shapes):
+        W0 = fill_weights(plan, i, ti.seed_for(cfg, i, 0, ti.ROLE_WEIGHT))
+        ob = oracle.OracleBlock(W0, s["r"], s.get("p", 0), s.get("q", 0), 0, sgd=(rule == 1))
+        ob.set_bases(to64(plan.U[i]), to64(plan.V[i]))
+        plan.M[i].zero_(); plan.Vm[i].zero_()
+        blks.append(ob)
+    worst = {"C": 0.0, "M": 0.0, "Vm": 0.0, "W": 0.0}
+    for t in range(1, steps + 1):
+        G64 = [fill_gradient(plan, i, ti.seed_for(cfg, i, t, ti.ROLE_GRAD)) for i in range(nb)]
+        h = tsr.make_hyper(t, lr=1e-3, weight_decay=wd, scale=scale, rule=rule)
+        if fuse:
+            plan.step(h, fuse_adam=True)
+        else:
+            plan.project_core()
+            plan.adam_core_step(h)
+            plan.backproject_apply(h)
+        torch.cuda.synchronize()
+        for i, ob in enumerate(blks):
+            ob.step(G64[i], lr=1e-3, weight_decay=wd, scale=scale)
+            worst["C"] = max(worst["C"], rel_fro(to64(plan.C[i]), ob.C))
+            worst["M"] = max(worst["M"], rel_fro(to64(plan.M[i]), ob.M))
+            if rule == 0:
+                worst["Vm"] = max(worst["Vm"], rel_fro(to64(plan.Vm[i]), ob.Vm))
+            worst["W"] = max(worst["W"], rel_fro(to64(plan.W[i]), ob.W))
+    assert plan.poll_status() == [0] * nb
+    for key, val in worst.items():
+        assert val < tol, (key, val, worst)
+    return worst
+
+
+def _given_bases(plan, shapes, seed0=500):
+    for i, s in enumerate(shapes):
+        set_bases(plan, i, ti.orthonormal(s["m"], s["r"], seed0 + 2 * i), ti.orthonormal(s["n"], s["r"], seed0 + 2 * i + 1))
+    plan.bases_changed()
+
+
+F32_SHAPES = [dict(m=512, n=1376, r=128), dict(m=200, n=330, r=24), dict(m=70, n=65, r=8)]
+BF16_SHAPES = [dict(m=256, n=384, r=64), dict(m=200, n=328, r=40), dict(m=1000, n=136, r=16),
+               dict(m=384, n=256, r=128)]
+
+
+@pytest.mark.parametrize("fuse", [False, True])
+def test_fp32_path_steps_match_oracle(fuse):
+    tsr, plan = _plan(F32_SHAPES, torch.float32)
+    assert not any(plan.uses_tensor_cores(i) for i in range(len(F32_SHAPES)))
+    _given_bases(plan, F32_SHAPES)
+    _run_steps(tsr, plan, F32_SHAPES, torch.float32, 10, fuse, TOL_F32)
+
+
+def test_fp32_path_decay_and_scale():
+    tsr, plan = _plan(F32_SHAPES[1:], torch.float32)
+    _given_bases(plan, F32_SHAPES[1:])
+    _run_steps(tsr, plan, F32_SHAPES[1:], torch.float32, 4, True, TOL_F32, wd=0.1, scale=0.25)
+
+
+@pytest.mark.parametrize("fuse", [False, True])
+def test_bf16_path_steps_match_oracle(fuse):
+    tsr, plan = _plan(BF16_SHAPES, torch.bfloat16)
+    assert all(plan.uses_tensor_cores(i) for i in range(len(BF16_SHAPES)))
+    _given_bases(plan, BF16_SHAPES)
+    _run_steps(tsr, plan, BF16_SHAPES, torch.bfloat16, 10, fuse, TOL_BF16)
+
+
+def test_bf16_path_decay_scale_and_sgd_rule():
+    tsr, plan = _plan(BF16_SHAPES[:2], torch.bfloat16)
+    _given_bases(plan, BF16_SHAPES[:2])
+    _run_steps(tsr, plan, BF16_SHAPES[:2], torch.bfloat16, 4, True, TOL_BF16, wd=0.1, scale=0.25)
+
+
+def test_fused_and_unfused_orders_agree_bitwise():
+    import paper_2602_08007_b200 as tsr
+    res = []
+    for fuse in (False, True):
+        plan = tsr.Plan(BF16_SHAPES, g_dtype=torch.bfloat16)
+        _given_bases(plan, BF16_SHAPES)
+        for i in range(len(BF16_SHAPES)):
+            fill_weights(plan, i, 7 + i)
+        for t in (1, 2, 3):
+            for i in range(len(BF16_SHAPES)):
+                fill_gradient(plan, i, 100 * t + i)
+            h = tsr.make_hyper(t)
+            if fuse:
+                plan.step(h, fuse_adam=True)
+            else:
+                plan.step(h, fuse_adam=False)
+        torch.cuda.synchronize()
+        res.append([(plan.W[i].clone(), plan.M[i].clone(), plan.Vm[i].clone(), plan.C[i].clone())
+                    for i in range(len(BF16_SHAPES))])
+    for a, b in zip(*res):
+        for x, y in zip(a, b):
+            assert torch.equal(x, y)
+
+
+def test_split_k_core_matches_oracle():
+    # m large enough that the core GEMM is split along K (tall embedding-like block)
+    shapes = [dict(m=9000, n=128, r=32)]
+    tsr, plan = _plan(shapes, torch.bfloat16)
+    _given_bases(plan, shapes)
+    _run_steps(tsr, plan, shapes, torch.bfloat16, 3, True, TOL_BF16)
+    _run_steps(tsr, plan, shapes, torch.bfloat16, 3, False, TOL_BF16)
+
+
+@pytest.mark.parametrize("dtype,shape,gap", [
+    (torch.float32, dict(m=512, n=1376, r=128, p=8, q=1), 64),
+    (torch.float32, dict(m=90, n=150, r=20, p=4, q=2), 10),
+    (torch.bfloat16, dict(m=512, n=1376, r=128, p=8, q=1), 64),
+    (torch.bfloat16, dict(m=1376, n=512, r=128, p=8, q=1), 64),
+    (torch.bfloat16, dict(m=200, n=328, r=40, p=8, q=2), 20),
+    (torch.bfloat16, dict(m=2000, n=256, r=64, p=8, q=1), 32),
+])
+def test_refresh_matches_oracle_at_gap(dtype, shape, gap):
+    tsr, plan = _plan([shape], dtype)
+    m, n, r, p, q = shape["m"], shape["n"], shape["r"], shape["p"], shape["q"]
+    G64 = fill_gradient(plan, 0, ti.seed_for(91, 0, 0, ti.ROLE_INIT_GRAD), signal_rank=gap)
+    Om = ti.omega(n, r + p, ti.seed_for(91, 0, 0, ti.ROLE_INIT_OMEGA)).cuda()
+    plan.M[0].fill_(3.0)
+    plan.init_subspace(omegas=[Om])
+    torch.cuda.synchronize()
+    assert plan.poll_status() == [0]
+    assert float(plan.M[0].abs().max()) == 0.0 and float(plan.Vm[0].abs().max()) == 0.0
+    check_refresh(plan, 0, G64, to64(Om), r, q, gap)
+    # refresh alone leaves the moments untouched
+    plan.M[0].fill_(2.0)
+    plan.rsvd_refresh(omegas=[Om])
+    torch.cuda.synchronize()
+    assert float(plan.M[0].min()) == 2.0
+
+
+def test_refresh_with_signal_rank_equal_r():
+    shape = dict(m=384, n=512, r=64, p=8, q=1)
+    tsr, plan = _plan([shape], torch.bfloat16)
+    G64 = fill_gradient(plan, 0, 77, signal_rank=64)
+    Om = ti.omega(512, 72, 78).cuda()
+    plan.init_subspace(omegas=[Om])
+    torch.cuda.synchronize()
+    check_refresh(plan, 0, G64, to64(Om), 64, 1, 64)
+
+
+def test_library_drawn_omega_is_standard_normal_and_used():
+    shape = dict(m=256, n=640, r=32, p=8, q=1)
+    tsr, plan = _plan([shape, shape], torch.bfloat16)
+    a = plan.generate_omega(0, 1234)
+    b = plan.generate_omega(1, 1234)
+    c = plan.generate_omega(0, 1235)
+    a2 = plan.generate_omega(0, 1234)
+    torch.cuda.synchronize()
+    assert torch.equal(a, a2) and not torch.equal(a, b) and not torch.equal(a, c)
+    x = to64(a).ravel()
+    assert abs(x.mean()) < 0.02 and abs(x.std() - 1.0) < 0.02
+    assert abs(((x - x.mean()) ** 3).mean()) < 0.05 and abs((x ** 4).mean() - 3.0) < 0.15
+    assert abs(np.corrcoef(x, to64(b).ravel())[0, 1]) < 0.02
+    # a refresh with the library's own Omega gives orthonormal bases aligned with the signal
+    for i in range(2):
+        G64 = fill_gradient(plan, i, 300 + i, signal_rank=16)
+    plan.init_subspace(seed=99)
+    torch.cuda.synchronize()
+    assert plan.poll_status() == [0, 0]
+    U = to64(plan.U[1])
+    assert np.linalg.norm(U.T @ U - np.eye(32)) < 1e-4
+    Un = np.linalg.svd(G64)[0]
+    assert np.linalg.norm(U[:, :16] @ U[:, :16].T - Un[:, :16] @ Un[:, :16].T) < 1e-3
+
+
+def test_mini_llama_grouped_lockstep_with_refresh():
+    """A small LLaMA-shaped set (attention, gate/up, down, embedding with its own rank and
+    schedule), BF16 gradients: init by refresh, then steps with an in-loop refresh at t = 3; after
+    every refresh the GPU's bases are handed to the oracle and the two continue in lock-step."""
+    import paper_2602_08007_b200 as tsr
+    hidden, ffn, vocab, r, re_ = 128, 344, 1000, 32, 16
+    shapes = []
+    for _ in range(2):
+        shapes += [dict(m=hidden, n=hidden, r=r, p=8, q=1, K=3)] * 4
+        shapes += [dict(m=ffn, n=hidden, r=r, p=8, q=1, K=3)] * 2 + [dict(m=hidden, n=ffn, r=r, p=8, q=1, K=3)]
+    shapes.append(dict(m=vocab, n=hidden, r=re_, p=8, q=1, K=6, is_embedding=True))
+    nb = len(shapes)
+    # K = 0 in the plan: the test drives the refresh itself so that both sides see the same Omega
+    plan = tsr.Plan([dict(s, K=0) for s in shapes], g_dtype=torch.bfloat16)
+    cfg = 92
+    G0 = [fill_gradient(plan, i, ti.seed_for(cfg, i, 0, ti.ROLE_INIT_GRAD), signal_rank=8) for i in range(nb)]
+    Om0 = [ti.omega(s["n"], s["r"] + s["p"], ti.seed_for(cfg, i, 0, ti.ROLE_INIT_OMEGA)).cuda() for i, s in enumerate(shapes)]
+    plan.init_subspace(omegas=Om0)
+    torch.cuda.synchronize()
+    blks = []
+    for i, s in enumerate(shapes):
+        check_refresh(plan, i, G0[i], to64(Om0[i]), s["r"], 1, 8)
+        W0 = fill_weights(plan, i, ti.seed_for(cfg, i, 0, ti.ROLE_WEIGHT))
+        ob = oracle.OracleBlock(W0, s["r"], s["p"], s["q"], s["K"])
+        ob.set_bases(to64(plan.U[i]), to64(plan.V[i]))
+        blks.append(ob)
+    worst = 0.0
+    for t in range(1, 8):
+        G64 = [fill_gradient(plan, i, ti.seed_for(cfg, i, t, ti.ROLE_GRAD), signal_rank=8) for i in range(nb)]
+        due = [i for i, s in enumerate(shapes) if t % s["K"] == 0]
+        if due:
+            oms = [ti.omega(shapes[i]["n"], shapes[i]["r"] + 8, ti.seed_for(cfg, i, t, ti.ROLE_OMEGA)).cuda() for i in due]
+            plan.rsvd_refresh(idx=due, omegas=oms)
+            torch.cuda.synchronize()
+            for j, i in enumerate(due):
+                assert blks[i].refresh_due()
+                check_refresh(plan, i, G64[i], to64(oms[j]), shapes[i]["r"], 1, 8)
+                blks[i].set_bases(to64(plan.U[i]), to64(plan.V[i]))
+        h = tsr.make_hyper(t)
+        plan.step(h, fuse_adam=(t % 2 == 0))
+        torch.cuda.synchronize()
+        for i, ob in enumerate(blks):
+            ob.step(G64[i], lr=1e-3, skip_refresh=True)
+            for a, b in ((plan.C[i], ob.C), (plan.M[i], ob.M), (plan.Vm[i], ob.Vm), (plan.W[i], ob.W)):
+                worst = max(worst, rel_fro(to64(a), b))
+    assert plan.poll_status() == [0] * nb
+    assert worst < TOL_BF16, worst
+
+
+def test_step_grouped_refreshes_on_schedule_and_embed_step():
+    import paper_2602_08007_b200 as tsr
+    shapes = [dict(m=256, n=320, r=32, p=8, q=1, K=2), dict(m=1200, n=256, r=16, p=8, q=1, K=3, is_embedding=True)]
+    plan = tsr.Plan(shapes, g_dtype=torch.bfloat16)
+    for i in range(2):
+        fill_gradient(plan, i, 40 + i, signal_rank=8)
+        fill_weights(plan, i, 50 + i)
+    plan.init_subspace(seed=5)
+    torch.cuda.synchronize()
+    prev = [plan.U[i].clone() for i in range(2)]
+    changed = []
+    for t in range(1, 7):
+        for i in range(2):
+            fill_gradient(plan, i, 1000 * t + i, signal_rank=8)
+        plan.step(tsr.make_hyper(t), seed=5)
+        torch.cuda.synchronize()
+        changed.append([not torch.equal(prev[i], plan.U[i]) for i in range(2)])
+        prev = [plan.U[i].clone() for i in range(2)]
+    assert [c[0] for c in changed] == [False, True, False, True, False, True]
+    assert [c[1] for c in changed] == [False, False, True, False, False, True]
+    for i in range(2):
+        U = to64(plan.U[i])
+        assert np.linalg.norm(U.T @ U - np.eye(U.shape[1])) < 1e-4
+    # embed_step touches only the embedding block
+    w0 = plan.W[0].clone()
+    w1 = plan.W[1].clone()
+    plan.embed_step(tsr.make_hyper(7), seed=5)
+    torch.cuda.synchronize()
+    assert torch.equal(w0, plan.W[0]) and not torch.equal(w1, plan.W[1])
+    with pytest.raises(tsr.TsrError):
+        plan.embed_step(tsr.make_hyper(7), idx=[0])
+
+
+def test_unaligned_leading_dimension_takes_cuda_core_path():
+    import paper_2602_08007_b200 as tsr
+    shapes = [dict(m=130, n=77, r=16)]            # 77 * 2 bytes is not a multiple of 16
+    plan = tsr.Plan(shapes, g_dtype=torch.bfloat16, pad=False)
+    assert not plan.uses_tensor_cores(0)
+    _given_bases(plan, shapes)
+    _run_steps(tsr, plan, shapes, torch.bfloat16, 3, True, TOL_F32)
+
+
+def test_step_from_host_buffers():
+    import paper_2602_08007_b200 as tsr
+    shapes = BF16_SHAPES[:2]
+    plan = tsr.Plan(shapes, g_dtype=torch.bfloat16)
+    ref = tsr.Plan(shapes, g_dtype=torch.bfloat16)
+    for pl in (plan, ref):
+        _given_bases(pl, shapes)
+        for i in range(2):
+            fill_weights(pl, i, 60 + i)
+    gh = [ti.gradient(s["m"], s["n"], 70 + i, dtype=torch.bfloat16).contiguous().pin_memory() for i, s in enumerate(shapes)]
+    c_host = torch.empty(sum(s["r"] ** 2 for s in shapes), dtype=torch.float32).pin_memory()
+    plan.step_host(gh, c_host, tsr.make_hyper(1))
+    for i in range(2):
+        ref.G[i].copy_(gh[i].cuda())
+    ref.step(tsr.make_hyper(1))
+    torch.cuda.synchronize()
+    off = 0
+    for i, s in enumerate(shapes):
+        assert torch.equal(plan.W[i], ref.W[i])
+        assert torch.equal(c_host[off:off + s["r"] ** 2].view(s["r"], s["r"]), ref.C[i].cpu())
+        off += s["r"] ** 2
