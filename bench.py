@@ -1,0 +1,398 @@
+#!/usr/bin/env python
+"""Benchmark of the TSR-Adam optimizer hot path (libtsr) on synthetic LLaMA-shaped gradient sets.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 4] [--impl ours|reference]
+
+A "step" is one full optimizer step over every matrix block of the model: core projection
+C = U^T G V, core-space Adam, lift and in-place weight update, plus the randomized-SVD refresh
+on the steps where the schedule asks for one (t mod K == 0).  The default workload is the
+LLaMA-1B-shaped set (169 blocks, r = 512, embedding rank 256, BF16 gradients, FP32 weights);
+its gradients (2.5 GB) and weights (5.1 GB) are far larger than the 126 MB L2, so no explicit
+flush is needed between steps.  Prints ONE JSON line (rank 0).
+
+The path does not shard across GPUs (no collective on the data path): with N > 1 every rank
+runs an independent replica on its own GPU and the line reports the slowest rank.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+import tsr_inputs as ti  # noqa: E402
+
+METRIC = "tsr_adam_step_ms"
+UNIT = "ms/step"
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            d = json.load(fh)
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"]),
+                "bf16_tflops_sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def step_work(w: ti.Workload):
+    """Algorithmic flops and bytes of one non-refresh step, per stage."""
+    ges = 2 if w.g_dtype == "bf16" else 4
+    out = {"proj_flops": 0.0, "proj_bytes": 0.0, "apply_flops": 0.0, "apply_bytes": 0.0,
+           "apply_kernel_flops": 0.0, "apply_kernel_bytes": 0.0}
+    for b in w.blocks:
+        m, n, r = b.m, b.n, b.r
+        small = 2.0 * min(m, n) * r * r
+        out["proj_flops"] += 2.0 * m * n * r + small
+        out["proj_bytes"] += ges * m * n + 2.0 * (m + n) * r + 24.0 * r * r
+        out["apply_flops"] += 2.0 * m * n * r + small
+        out["apply_bytes"] += 8.0 * m * n + 2.0 * (m + n) * r
+        # the apply kernel proper: W <- decay W - step_scale P V^T with P = U D (m x r) given
+        out["apply_kernel_flops"] += 2.0 * m * n * r
+        out["apply_kernel_bytes"] += 8.0 * m * n + 2.0 * (m + n) * r
+    out["step_flops"] = out["proj_flops"] + out["apply_flops"]
+    out["step_bytes"] = out["proj_bytes"] + out["apply_bytes"]
+    return out
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
+
+    def __init__(self, index: int):
+        super().__init__(daemon=True)
+        self.index = index
+        self.stop_flag = threading.Event()
+        self.sm, self.reasons, self.max_sm = [], set(), None
+        self.ok = False
+
+    def run(self):
+        try:
+            import pynvml as nv
+            nv.nvmlInit()
+            h = nv.nvmlDeviceGetHandleByIndex(self.index)
+            self.max_sm = nv.nvmlDeviceGetMaxClockInfo(h, nv.NVML_CLOCK_SM)
+            names = {
+                getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8): "hw_slowdown",
+                getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+                getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+                getattr(nv, "nvmlClocksThrottleReasonSwPowerCap", 0x4): "sw_power_cap",
+            }
+            self.ok = True
+            while not self.stop_flag.is_set():
+                self.sm.append(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM))
+                mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(h)
+                for bit, name in names.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+                time.sleep(0.05)
+        except Exception:
+            self.ok = False
+
+    def summary(self):
+        if not self.ok or not self.sm:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_sm, "reasons": ["nvml_unavailable"]}
+        return {"sm_mhz": statistics.median(self.sm), "sm_max_mhz": self.max_sm, "reasons": sorted(self.reasons)}
+
+
+def physical_gpu_index(local_rank: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except Exception:
+            return local_rank
+    return local_rank
+
+
+# --------------------------------------------------------------------------------------------
+# reference arm / cpu baseline: the FP64 oracle on the host cores, on a bounded sample
+# --------------------------------------------------------------------------------------------
+def oracle_sample(w: ti.Workload, seconds_hint: float = 2.0):
+    """Picks the sample the oracle is timed on: one square attention-shaped block of the workload
+    (the most frequent shape), or the single block of config 0."""
+    blk = w.blocks[0]
+    return blk
+
+
+def oracle_step_time(w: ti.Workload, blk, reps: int = 1):
+    """Seconds the oracle needs for one optimizer step (project, core Adam, lift+apply) of `blk`."""
+    import numpy as np
+
+    import oracle
+    dt = torch.bfloat16 if w.g_dtype == "bf16" else torch.float32
+    G = ti.gradient(blk.m, blk.n, 1, dtype=dt).double().numpy()
+    ob = oracle.OracleBlock(ti.weights(blk.m, blk.n, 2).double().numpy(), blk.r, blk.p, blk.q, 0)
+    ob.set_bases(ti.orthonormal(blk.m, blk.r, 3).double().numpy(), ti.orthonormal(blk.n, blk.r, 4).double().numpy())
+    times = []
+    for rep in range(reps):
+        t0 = time.perf_counter()
+        ob.step(G, lr=1e-3)
+        times.append(time.perf_counter() - t0)
+    assert np.isfinite(ob.W).all()
+    return min(times)
+
+
+def cpu_baseline(w: ti.Workload):
+    import oracle
+    blk = oracle_sample(w)
+    work = step_work(w)
+    sample = step_work(ti.Workload("sample", w.config_id, w.g_dtype, 1, (blk,)))
+    sec = oracle_step_time(w, blk)
+    scale = work["step_flops"] / sample["step_flops"]
+    return {"value": sec * scale * 1e3, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": "one %dx%d r=%d block timed for one step (%.2f s), scaled by algorithmic flops x%.1f to the "
+                      "whole %s set" % (blk.m, blk.n, blk.r, sec, scale, w.name)}
+
+
+def run_reference(args, w: ti.Workload):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    blk = oracle_sample(w)
+    work = step_work(w)
+    sample = step_work(ti.Workload("sample", w.config_id, w.g_dtype, 1, (blk,)))
+    scale = work["step_flops"] / sample["step_flops"]
+    # size the per-step sample so the whole run stays within a few minutes
+    for _ in range(args.warmup):
+        oracle_step_time(w, blk)
+    t = [oracle_step_time(w, blk) for _ in range(args.steps)]
+    ms = statistics.mean(t) * scale * 1e3
+    line = {
+        "impl": "reference", "metric": METRIC, "value": ms, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "blocks": len(w.blocks)},
+        "cpu_baseline": {"value": ms, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                         "sample": "each step = one %dx%d r=%d block through the FP64 oracle, scaled by algorithmic "
+                                   "flops x%.1f to the whole set" % (blk.m, blk.n, blk.r, scale)},
+        "e2e": {"value": ms, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# --------------------------------------------------------------------------------------------
+# our arm
+# --------------------------------------------------------------------------------------------
+def build_plan(w: ti.Workload, device):
+    import paper_2602_08007_b200 as tsr
+    dt = torch.bfloat16 if w.g_dtype == "bf16" else torch.float32
+    plan = tsr.Plan(list(w.blocks), g_dtype=dt, device=device)
+    for i, b in enumerate(w.blocks):
+        plan.G[i].copy_(ti.gradient(b.m, b.n, ti.seed_for(w.config_id, i, 0, ti.ROLE_INIT_GRAD), dtype=dt, device=device))
+        plan.W[i].copy_(ti.weights(b.m, b.n, ti.seed_for(w.config_id, i, 0, ti.ROLE_WEIGHT), device=device))
+    return tsr, plan
+
+
+def fresh_gradients(plan, w, t, device):
+    dt = plan.g_dtype
+    for i, b in enumerate(w.blocks):
+        plan.G[i].copy_(ti.gradient(b.m, b.n, ti.seed_for(w.config_id, i, t, ti.ROLE_GRAD), dtype=dt, device=device))
+
+
+def run_ours(args, w: ti.Workload):
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist_mod.init_process_group("nccl", device_id=device)
+        dist = dist_mod
+
+    tsr, plan = build_plan(w, device)
+    peaks = measured_peaks()
+    work = step_work(w)
+    nb = len(w.blocks)
+    seed = ti.BASE_SEED
+
+    plan.init_subspace(seed=seed)            # Algorithm 1 initialisation: one refresh on G_0
+    torch.cuda.synchronize()
+    fresh_gradients(plan, w, 1, device)
+    flush = None
+    if args.flush_l2:
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)
+
+    def one_step(t):
+        if flush is not None:
+            flush.fill_(t & 0xFF)
+        plan.step(tsr.make_hyper(t), seed=seed, fuse_adam=True)
+
+    # warm-up on steps that are not refresh steps
+    for wstep in range(args.warmup):
+        one_step(1)
+    torch.cuda.synchronize()
+    status = plan.poll_status()
+
+    plan.set_profiling(True)
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    stage = []
+    sampler = ClockSampler(physical_gpu_index(local_rank))
+    launches0 = plan.launch_count()
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    wall0 = time.perf_counter()
+    for j in range(args.steps):
+        t = j + 1
+        if flush is not None:
+            flush.fill_(t & 0xFF)
+        ev[j][0].record()
+        plan.step(tsr.make_hyper(t), seed=seed, fuse_adam=True)
+        ev[j][1].record()
+        if args.stage_times:
+            stage.append(plan.stage_ms())     # waits for this step; only with --stage-times
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    wall = time.perf_counter() - wall0
+    sampler.stop_flag.set()
+    sampler.join(timeout=2)
+    launches = plan.launch_count() - launches0
+    step_ms = [a.elapsed_time(b) for a, b in ev]
+    refresh_steps = [j for j in range(args.steps) if any(b.K > 0 and (j + 1) % b.K == 0 for b in w.blocks)]
+    plain = [step_ms[j] for j in range(args.steps) if j not in refresh_steps] or step_ms
+    total_ms = sum(step_ms)
+    ms_per_step = total_ms / args.steps
+    status2 = plan.poll_status()
+
+    # stage breakdown and the dominant kernel (apply), measured with CUDA events on plain steps
+    plan.set_profiling(True)
+    st_rows = []
+    for rep in range(max(5, min(20, args.steps))):
+        if flush is not None:
+            flush.fill_(rep)
+        plan.step(tsr.make_hyper(1), seed=seed, fuse_adam=True)
+        st_rows.append(plan.stage_ms())
+    st_med = [statistics.median(r[i] for r in st_rows) for i in range(6)]
+    apply_ms = st_med[5]
+    proj_ms = st_med[1] + st_med[2]
+
+    # refresh alone
+    refresh_ms = None
+    if args.refresh_reps > 0:
+        rts = []
+        for rep in range(args.refresh_reps):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            plan.rsvd_refresh(seed=seed + 1 + rep)
+            b.record()
+            torch.cuda.synchronize()
+            rts.append(a.elapsed_time(b))
+        refresh_ms = min(rts)
+    status3 = plan.poll_status()
+
+    # end to end from host buffers: H2D of every gradient, the step, D2H of the packed cores
+    e2e = None
+    if args.e2e_steps > 0:
+        dt = plan.g_dtype
+        g_host = [torch.empty(b.m, b.n, dtype=dt).pin_memory() for b in w.blocks]
+        for i in range(nb):
+            g_host[i].copy_(plan.G[i])
+        c_host = torch.empty(sum(b.r * b.r for b in w.blocks), dtype=torch.float32).pin_memory()
+        plan.step_host(g_host, c_host, tsr.make_hyper(1), seed=seed)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for j in range(args.e2e_steps):
+            plan.step_host(g_host, c_host, tsr.make_hyper(1), seed=seed)
+        torch.cuda.synchronize()
+        e2e_ms = (time.perf_counter() - t0) * 1e3 / args.e2e_steps
+        e2e = {"value": e2e_ms, "unit": UNIT, "h2d_bytes_per_step": sum(g.numel() * g.element_size() for g in g_host),
+               "d2h_bytes_per_step": c_host.numel() * 4}
+
+    # max over ranks
+    if dist is not None:
+        tens = torch.tensor([ms_per_step, wall * 1e3 / args.steps, apply_ms, proj_ms], device=device, dtype=torch.float64)
+        dist.all_reduce(tens, op=dist.ReduceOp.MAX)
+        ms_per_step, wall_ms_per_step, apply_ms, proj_ms = [float(x) for x in tens]
+    else:
+        wall_ms_per_step = wall * 1e3 / args.steps
+
+    if rank == 0:
+        hbm = peaks["hbm_gbs"]
+        tc = peaks["bf16_tflops_sustained"]
+        apply_gbs = work["apply_kernel_bytes"] / (apply_ms * 1e-3) / 1e9
+        proj_tflops = work["proj_flops"] / (proj_ms * 1e-3) / 1e12
+        proj_roof_ms = max(work["proj_flops"] / (tc * 1e12), work["proj_bytes"] / (hbm * 1e9)) * 1e3
+        apply_roof_ms = max(work["apply_kernel_flops"] / (tc * 1e12), work["apply_kernel_bytes"] / (hbm * 1e9)) * 1e3
+        plain_ms = statistics.median(plain)
+        core_b, sketch_b = plan.comm_bytes(0, 4)
+        line = {
+            "metric": METRIC, "value": ms_per_step, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16" if w.g_dtype == "bf16" else "f32", "data": "synthetic",
+            "config": {"workload": w.name, "blocks": nb, "rank": w.blocks[0].r, "embedding_rank": w.blocks[-1].r,
+                       "refresh_interval": w.blocks[0].K, "refresh_steps_in_timed_region": len(refresh_steps),
+                       "l2": "flushed between steps" if flush is not None else "inputs (G %.2f GB + W %.2f GB) exceed L2"
+                       % (sum(b.m * b.n for b in w.blocks) * (2 if w.g_dtype == "bf16" else 4) / 1e9,
+                          sum(b.m * b.n for b in w.blocks) * 4 / 1e9),
+                       "parallelism": "replicas only" if world > 1 else "single gpu"},
+            "step_ms_no_refresh": plain_ms,
+            "wall_ms_per_step": wall_ms_per_step,
+            "refresh_ms": refresh_ms,
+            "step_tflops": work["step_flops"] / (plain_ms * 1e-3) / 1e12,
+            "stage_ms": {"refresh": st_med[0], "gemm_GV": st_med[1], "gemm_core": st_med[2], "core_update": st_med[3],
+                         "gemm_UD": st_med[4], "apply": st_med[5]},
+            "roofline": {"kernel": "umma_gemm_kernel<EPI_APPLY> (W <- decay W - lr P V^T)", "bound": "hbm",
+                         "achieved": apply_gbs, "peak": hbm, "unit": "GB/s", "frac": apply_gbs / hbm, "traffic": None,
+                         "peak_source": peaks["source"] + " copy bandwidth", "ms": apply_ms, "roof_ms": apply_roof_ms},
+            "roofline_projection": {"kernels": "umma_gemm_kernel<EPI_STORE_BF16_T> + <EPI_CORE_UPDATE>",
+                                    "bound": "tensor" if work["proj_flops"] / (tc * 1e12) > work["proj_bytes"] / (hbm * 1e9) else "hbm",
+                                    "achieved_tflops": proj_tflops, "ms": proj_ms, "roof_ms": proj_roof_ms,
+                                    "frac": proj_roof_ms / proj_ms},
+            "comm_bytes": {"core_per_step": core_b, "sketch_per_refresh": sketch_b,
+                           "dense_fp32_per_step": 4 * sum(b.m * b.n for b in w.blocks)},
+            "device_status": sorted(set(status + status2 + status3)),
+            "clocks": sampler.summary(),
+            "e2e": e2e,
+            "gpu_launches": launches,
+        }
+        if not args.no_cpu_baseline and world == 1:
+            line["cpu_baseline"] = cpu_baseline(w)
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", type=int, default=4, help="0..4: the five benchmark configurations")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--flush-l2", action="store_true", help="write a 256 MB buffer before every step")
+    ap.add_argument("--stage-times", action="store_true", help="also read stage timings inside the timed loop")
+    ap.add_argument("--refresh-reps", type=int, default=1)
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+    w = ti.workload(args.config)
+    if args.config < 3:
+        args.flush_l2 = True
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()

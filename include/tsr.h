@@ -220,6 +220,19 @@ TSR_API tsr_status tsr_poll_status(tsr_ctx *ctx, int32_t *per_block_status, int3
  * shape. */
 TSR_API tsr_status tsr_generate_omega(tsr_ctx *ctx, int32_t i, uint64_t seed, float *out, void *stream);
 
+/* Stage timing of tsr_step_grouped for profiling (off by default).  When enabled, every
+ * tsr_step_grouped / tsr_embed_step records CUDA events at its stage boundaries on the step's
+ * stream; tsr_get_stage_ms waits for the last recorded step and returns, in milliseconds,
+ * ms[0] refresh (0 when none was due), ms[1] T = G V, ms[2] core GEMM C = U^T T (with the
+ * fused core update and the split-K reduction), ms[3] stand-alone core update (unfused order
+ * only), ms[4] P = U D, ms[5] the apply kernel W <- decay W - step_scale P V^T.  count must be 6.
+ * Enabling creates the events (a small driver allocation); disabling destroys them. */
+TSR_API tsr_status tsr_set_profiling(tsr_ctx *ctx, int32_t enable);
+TSR_API tsr_status tsr_get_stage_ms(tsr_ctx *ctx, float *ms, int32_t count);
+
+/* Number of CUDA kernels this context has launched since tsr_create. */
+TSR_API tsr_status tsr_launch_count(const tsr_ctx *ctx, uint64_t *count);
+
 /* 1 if block i takes the tensor-core path, 0 if the FP32 CUDA-core path, < 0 on a bad index. */
 TSR_API int32_t tsr_block_uses_tensor_cores(const tsr_ctx *ctx, int32_t i);
 

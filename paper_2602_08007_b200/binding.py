@@ -53,6 +53,7 @@ EXPORTS = [
     "tsr_project_core_grouped", "tsr_adam_core_step_grouped", "tsr_backproject_apply_grouped",
     "tsr_rsvd_refresh_grouped", "tsr_embed_step_grouped", "tsr_step_grouped", "tsr_step_grouped_host",
     "tsr_comm_bytes", "tsr_state_elems", "tsr_poll_status", "tsr_generate_omega", "tsr_block_uses_tensor_cores",
+    "tsr_set_profiling", "tsr_get_stage_ms", "tsr_launch_count",
 ]
 
 
@@ -106,6 +107,9 @@ def lib():
         L.tsr_generate_omega.argtypes = [vp, i32, u64, vp, vp]
         L.tsr_block_uses_tensor_cores.argtypes = [vp, i32]
         L.tsr_block_uses_tensor_cores.restype = i32
+        L.tsr_set_profiling.argtypes = [vp, i32]
+        L.tsr_get_stage_ms.argtypes = [vp, P(ctypes.c_float), i32]
+        L.tsr_launch_count.argtypes = [vp, P(u64)]
         _lib = L
     return _lib
 
@@ -279,6 +283,19 @@ class Plan:
         arr = (ctypes.c_int32 * nb)()
         self._check(lib().tsr_poll_status(self.ctx, arr, nb, _stream_ptr(stream)))
         return list(arr)
+
+    def set_profiling(self, enable: bool):
+        self._check(lib().tsr_set_profiling(self.ctx, 1 if enable else 0))
+
+    def stage_ms(self) -> List[float]:
+        arr = (ctypes.c_float * 6)()
+        self._check(lib().tsr_get_stage_ms(self.ctx, arr, 6))
+        return list(arr)
+
+    def launch_count(self) -> int:
+        c = ctypes.c_uint64()
+        self._check(lib().tsr_launch_count(self.ctx, ctypes.byref(c)))
+        return c.value
 
     def generate_omega(self, i: int, seed: int, stream=None) -> torch.Tensor:
         d = self.descs[i]

@@ -16,6 +16,7 @@ using namespace tsr;
 namespace {
 
 enum Kind : int { KT = 0, KC, KCS, KP, KA, KY, KZ, NKIND };
+constexpr int TSR_NUM_STAGES = 6;  // refresh, G*V, core GEMM, core update, U*D, apply
 
 struct Block {
     tsr_mat_desc d;
@@ -76,6 +77,12 @@ struct tsr_ctx {
     size_t items_cap[4] = {};
     EncodeTiledFn encode = nullptr;
     int max_r = 0, max_k = 0;
+    uint64_t launches = 0;                     // kernels launched through this context
+    bool profiling = false;
+    cudaEvent_t ev[TSR_NUM_STAGES + 1] = {};   // stage boundaries of the last step (profiling only)
+    bool ev_valid = false;
+    cudaStream_t stage_stream = nullptr;
+    int stage_next = 0;
 };
 
 namespace {
@@ -98,6 +105,12 @@ tsr_status fail(tsr_ctx *ctx, tsr_status s, const char *fmt, ...)
         cudaError_t e__ = (call);                                                                      \
         if (e__ != cudaSuccess)                                                                        \
             return fail(ctx, TSR_ERR_CUDA, "%s failed: %s", #call, cudaGetErrorString(e__));           \
+    } while (0)
+
+#define TSR_KERNEL(ctx, n, call)                                                                       \
+    do {                                                                                               \
+        TSR_CUDA(ctx, call);                                                                           \
+        (ctx)->launches += (n);                                                                        \
     } while (0)
 
 bool aligned16(const void *p) { return ((uintptr_t)p & 15) == 0; }
@@ -266,6 +279,13 @@ tsr_status check_hyper(tsr_ctx *ctx, const tsr_hyper *h)
     return TSR_OK;
 }
 
+// Profiling: records the stage-boundary events ev[stage_next .. upto] on the step's stream.
+void mark_stage(tsr_ctx *ctx, int upto)
+{
+    if (!ctx->profiling) return;
+    for (; ctx->stage_next <= upto; ++ctx->stage_next) cudaEventRecord(ctx->ev[ctx->stage_next], ctx->stage_stream);
+}
+
 // Resolves (idx, count) into a validated list of block indices.
 tsr_status resolve_list(tsr_ctx *ctx, const int32_t *idx, int32_t count, std::vector<int> &out)
 {
@@ -310,6 +330,7 @@ tsr_status launch_kind(tsr_ctx *ctx, int kind, const std::vector<int> &list, int
         while (j < ranges.size() && ranges[j].first == hi) { hi = ranges[j].second; ++j; }
         TSR_CUDA(ctx, umma_gemm_launch(ctx->d_probs[kind], ctx->d_tiles[kind] + lo, hi - lo, 128, epilogue, planes, sc,
                                        ctx->d_status, st));
+        ctx->launches++;
         i = j;
     }
     return TSR_OK;
@@ -328,6 +349,7 @@ tsr_status do_project(tsr_ctx *ctx, const std::vector<int> &list, bool fuse, con
     tsr_status s;
     if (ctx->any_fast) {
         if ((s = launch_kind(ctx, KT, list, EPI_STORE_BF16_T, 1, sc, st)) != TSR_OK) return s;
+        mark_stage(ctx, 2);
         if ((s = launch_kind(ctx, KC, list, fuse ? EPI_CORE_UPDATE : EPI_STORE_F32, 1, sc, st)) != TSR_OK) return s;
         if ((s = launch_kind(ctx, KCS, list, EPI_STORE_F32, 1, sc, st)) != TSR_OK) return s;
     }
@@ -338,8 +360,8 @@ tsr_status do_project(tsr_ctx *ctx, const std::vector<int> &list, bool fuse, con
         const int m = (int)b.d.m, n = (int)b.d.n, r = b.d.r;
         if (!b.fast) {
             // T = G V, C = U^T T on CUDA cores
-            TSR_CUDA(ctx, simt_gemm(m, r, n, b.p.G, b.d.g_dtype, b.d.ldg, 1, b.p.V, r, 1, b.T32, r, SIMT_STORE, 0, 0, st));
-            TSR_CUDA(ctx, simt_gemm(r, r, m, b.p.U, TSR_F32, 1, r, b.T32, r, 1, b.p.C, r, SIMT_STORE, 0, 0, st));
+            TSR_KERNEL(ctx, 1, simt_gemm(m, r, n, b.p.G, b.d.g_dtype, b.d.ldg, 1, b.p.V, r, 1, b.T32, r, SIMT_STORE, 0, 0, st));
+            TSR_KERNEL(ctx, 1, simt_gemm(r, r, m, b.p.U, TSR_F32, 1, r, b.T32, r, 1, b.p.C, r, SIMT_STORE, 0, 0, st));
             if (fuse) { later.push_back(bi); max_r = std::max(max_r, r); }
         } else if (b.nsplit > 1) {
             split.push_back(bi);
@@ -348,12 +370,13 @@ tsr_status do_project(tsr_ctx *ctx, const std::vector<int> &list, bool fuse, con
     }
     if (!split.empty()) {   // sum the split-K slabs (and, when fused, run the core update on the sum)
         if ((s = upload_list(ctx, ctx->d_list2, split, st)) != TSR_OK) return s;
-        TSR_CUDA(ctx, core_update_launch(ctx->d_cu_split, ctx->d_list2, (int)split.size(), max_r, sc, fuse ? 0 : 1, st));
+        TSR_KERNEL(ctx, 1, core_update_launch(ctx->d_cu_split, ctx->d_list2, (int)split.size(), max_r, sc, fuse ? 0 : 1, st));
     }
     if (!later.empty()) {
         if ((s = upload_list(ctx, ctx->d_list2, later, st)) != TSR_OK) return s;
-        TSR_CUDA(ctx, core_update_launch(ctx->d_cu_all, ctx->d_list2, (int)later.size(), max_r, sc, 0, st));
+        TSR_KERNEL(ctx, 1, core_update_launch(ctx->d_cu_all, ctx->d_list2, (int)later.size(), max_r, sc, 0, st));
     }
+    mark_stage(ctx, 3);
     return TSR_OK;
 }
 
@@ -364,7 +387,7 @@ tsr_status do_core_update(tsr_ctx *ctx, const std::vector<int> &list, const Step
     int max_r = 1;
     for (int bi : list) max_r = std::max(max_r, (int)ctx->blocks[bi].d.r);
     if ((s = upload_list(ctx, ctx->d_list, list, st)) != TSR_OK) return s;
-    TSR_CUDA(ctx, core_update_launch(ctx->d_cu_all, ctx->d_list, (int)list.size(), max_r, sc, 0, st));
+    TSR_KERNEL(ctx, 1, core_update_launch(ctx->d_cu_all, ctx->d_list, (int)list.size(), max_r, sc, 0, st));
     return TSR_OK;
 }
 
@@ -374,14 +397,15 @@ tsr_status do_apply(tsr_ctx *ctx, const std::vector<int> &list, const StepScalar
     tsr_status s;
     if (ctx->any_fast) {
         if ((s = launch_kind(ctx, KP, list, EPI_STORE_BF16, 1, sc, st)) != TSR_OK) return s;
+        mark_stage(ctx, 5);
         if ((s = launch_kind(ctx, KA, list, EPI_APPLY, 1, sc, st)) != TSR_OK) return s;
     }
     for (int bi : list) {
         Block &b = ctx->blocks[bi];
         if (b.fast) continue;
         const int m = (int)b.d.m, n = (int)b.d.n, r = b.d.r;
-        TSR_CUDA(ctx, simt_gemm(m, r, r, b.p.U, TSR_F32, r, 1, b.D32, r, 1, b.P32, r, SIMT_STORE, 0, 0, st));
-        TSR_CUDA(ctx, simt_gemm(m, n, r, b.P32, TSR_F32, r, 1, b.p.V, 1, r, (float *)b.p.W, b.d.ldw, SIMT_APPLY, sc.decay,
+        TSR_KERNEL(ctx, 1, simt_gemm(m, r, r, b.p.U, TSR_F32, r, 1, b.D32, r, 1, b.P32, r, SIMT_STORE, 0, 0, st));
+        TSR_KERNEL(ctx, 1, simt_gemm(m, n, r, b.P32, TSR_F32, r, 1, b.p.V, 1, r, (float *)b.p.W, b.d.ldw, SIMT_APPLY, sc.decay,
                                 sc.step_scale, st));
     }
     return TSR_OK;
@@ -392,8 +416,8 @@ tsr_status do_shadows(tsr_ctx *ctx, const std::vector<int> &list, cudaStream_t s
     for (int bi : list) {
         Block &b = ctx->blocks[bi];
         if (!b.fast) continue;
-        TSR_CUDA(ctx, make_shadows(b.p.U, (int)b.d.m, b.d.r, b.Ub, b.rl, b.Ubt, b.ml, st));
-        TSR_CUDA(ctx, make_shadows(b.p.V, (int)b.d.n, b.d.r, b.Vb, b.rl, b.Vbt, b.nl, st));
+        TSR_KERNEL(ctx, 1, make_shadows(b.p.U, (int)b.d.m, b.d.r, b.Ub, b.rl, b.Ubt, b.ml, st));
+        TSR_KERNEL(ctx, 1, make_shadows(b.p.V, (int)b.d.n, b.d.r, b.Vb, b.rl, b.Vbt, b.nl, st));
     }
     return TSR_OK;
 }
@@ -408,10 +432,10 @@ struct RefreshLists {
 tsr_status orth_pass(tsr_ctx *ctx, const RefreshLists &L, int side, int src, int dst, cudaStream_t st)
 {
     const int nl = (int)L.list.size();
-    TSR_CUDA(ctx, gram_batched(ctx->d_refresh, ctx->d_items[side * 2 + 1], L.nitems[side * 2 + 1], ctx->d_list, nl, side,
+    TSR_KERNEL(ctx, 2, gram_batched(ctx->d_refresh, ctx->d_items[side * 2 + 1], L.nitems[side * 2 + 1], ctx->d_list, nl, side,
                                src, L.kmax, st));
-    TSR_CUDA(ctx, chol_inverse_batched(ctx->d_refresh, ctx->d_list, nl, st));
-    TSR_CUDA(ctx, rows_gemm_batched(ctx->d_refresh, ctx->d_items[side * 2], L.nitems[side * 2], side, src, 0, dst, L.kmax, st));
+    TSR_KERNEL(ctx, 1, chol_inverse_batched(ctx->d_refresh, ctx->d_list, nl, st));
+    TSR_KERNEL(ctx, 1, rows_gemm_batched(ctx->d_refresh, ctx->d_items[side * 2], L.nitems[side * 2], side, src, 0, dst, L.kmax, st));
     return TSR_OK;
 }
 
@@ -437,11 +461,11 @@ tsr_status sketch(tsr_ctx *ctx, const RefreshLists &L, bool transposed, bool fro
         if (b.fast) {
             const int rows = transposed ? m : n;                 // rows of X
             const int64_t ld = transposed ? b.ml : b.nl;
-            TSR_CUDA(ctx, split_transpose(X, rows, k, b.Xt, ld, k, 2, st));
+            TSR_KERNEL(ctx, 1, split_transpose(X, rows, k, b.Xt, ld, k, 2, st));
         } else if (!transposed) {
-            TSR_CUDA(ctx, simt_gemm(m, k, n, b.p.G, b.d.g_dtype, b.d.ldg, 1, X, k, 1, b.buf[0], k, SIMT_STORE, 0, 0, st));
+            TSR_KERNEL(ctx, 1, simt_gemm(m, k, n, b.p.G, b.d.g_dtype, b.d.ldg, 1, X, k, 1, b.buf[0], k, SIMT_STORE, 0, 0, st));
         } else {
-            TSR_CUDA(ctx, simt_gemm(n, k, m, b.p.G, b.d.g_dtype, 1, b.d.ldg, X, k, 1, b.buf[0], k, SIMT_STORE, 0, 0, st));
+            TSR_KERNEL(ctx, 1, simt_gemm(n, k, m, b.p.G, b.d.g_dtype, 1, b.d.ldg, X, k, 1, b.buf[0], k, SIMT_STORE, 0, 0, st));
         }
     }
     if (ctx->any_fast)
@@ -483,9 +507,9 @@ tsr_status do_refresh(tsr_ctx *ctx, const std::vector<int> &list, uint64_t seed,
     for (size_t j = 0; j < list.size(); ++j) {
         Block &b = ctx->blocks[list[j]];
         if (!(omegas && omegas[j]))
-            TSR_CUDA(ctx, fill_gaussian(b.Om, (int64_t)b.d.n * b.k, seed, (uint64_t)list[j], st));
+            TSR_KERNEL(ctx, 1, fill_gaussian(b.Om, (int64_t)b.d.n * b.k, seed, (uint64_t)list[j], st));
         if (b.fast)
-            TSR_CUDA(ctx, transpose_bf16((const bf16 *)b.p.G, (int)b.d.m, (int)b.d.n, b.d.ldg, b.Gt, b.ml, st));
+            TSR_KERNEL(ctx, 1, transpose_bf16((const bf16 *)b.p.G, (int)b.d.m, (int)b.d.n, b.d.ldg, b.Gt, b.ml, st));
     }
     // Y = G Omega; Q = orth(Y)
     if ((s = sketch(ctx, L, false, true, omegas, st)) != TSR_OK) return s;
@@ -500,11 +524,11 @@ tsr_status do_refresh(tsr_ctx *ctx, const std::vector<int> &list, uint64_t seed,
     // B^T = G^T Q (n x k) in buf[0]; small SVD through the k x k Gram matrix B B^T
     if ((s = sketch(ctx, L, true, false, nullptr, st)) != TSR_OK) return s;
     const int nl = (int)list.size();
-    TSR_CUDA(ctx, gram_batched(ctx->d_refresh, ctx->d_items[3], L.nitems[3], ctx->d_list, nl, 1, 0, L.kmax, st));
-    TSR_CUDA(ctx, jacobi_batched(ctx->d_refresh, ctx->d_list, nl, 40, st));
+    TSR_KERNEL(ctx, 2, gram_batched(ctx->d_refresh, ctx->d_items[3], L.nitems[3], ctx->d_list, nl, 1, 0, L.kmax, st));
+    TSR_KERNEL(ctx, 1, jacobi_batched(ctx->d_refresh, ctx->d_list, nl, 40, st));
     // V = B^T Wt / sigma ; U = Q Wt
-    TSR_CUDA(ctx, rows_gemm_batched(ctx->d_refresh, ctx->d_items[2], L.nitems[2], 1, 0, 2, 4, L.rmax, st));
-    TSR_CUDA(ctx, rows_gemm_batched(ctx->d_refresh, ctx->d_items[0], L.nitems[0], 0, 2, 1, 3, L.rmax, st));
+    TSR_KERNEL(ctx, 1, rows_gemm_batched(ctx->d_refresh, ctx->d_items[2], L.nitems[2], 1, 0, 2, 4, L.rmax, st));
+    TSR_KERNEL(ctx, 1, rows_gemm_batched(ctx->d_refresh, ctx->d_items[0], L.nitems[0], 0, 2, 1, 3, L.rmax, st));
     return do_shadows(ctx, list, st);
 }
 
@@ -523,6 +547,7 @@ tsr_status do_step(tsr_ctx *ctx, const std::vector<int> &list, const tsr_hyper *
                    cudaStream_t st)
 {
     tsr_status s;
+    if (ctx->profiling) TSR_CUDA(ctx, cudaEventRecord(ctx->ev[0], st));
     std::vector<int> due;
     for (int bi : list) {
         const Block &b = ctx->blocks[bi];
@@ -539,9 +564,20 @@ tsr_status do_step(tsr_ctx *ctx, const std::vector<int> &list, const tsr_hyper *
         }
     }
     const StepScalars sc = make_scalars(h);
+    ctx->stage_stream = st;
+    ctx->stage_next = 1;
+    if (ctx->profiling) {
+        ctx->ev_valid = false;
+        TSR_CUDA(ctx, cudaEventRecord(ctx->ev[1], st));
+        ctx->stage_next = 2;
+    }
     if ((s = do_project(ctx, list, fuse, sc, st)) != TSR_OK) return s;
     if (!fuse && (s = do_core_update(ctx, list, sc, st)) != TSR_OK) return s;
-    return do_apply(ctx, list, sc, st);
+    mark_stage(ctx, 4);
+    if ((s = do_apply(ctx, list, sc, st)) != TSR_OK) return s;
+    mark_stage(ctx, 6);
+    if (ctx->profiling) ctx->ev_valid = true;
+    return TSR_OK;
 }
 
 }  // namespace
@@ -623,6 +659,8 @@ tsr_status tsr_create(tsr_ctx **out, const tsr_mat_desc *descs, int32_t count)
 tsr_status tsr_destroy(tsr_ctx *ctx)
 {
     if (!ctx) return TSR_ERR_INVALID_ARG;
+    if (ctx->profiling)
+        for (cudaEvent_t e : ctx->ev) if (e) cudaEventDestroy(e);
     delete ctx;
     return TSR_OK;
 }
@@ -972,7 +1010,38 @@ tsr_status tsr_generate_omega(tsr_ctx *ctx, int32_t i, uint64_t seed, float *out
     int dev_count = 0;
     if (cudaGetDeviceCount(&dev_count) != cudaSuccess || dev_count <= 0) return fail(ctx, TSR_ERR_CUDA, "no CUDA device available");
     const Block &b = ctx->blocks[i];
-    TSR_CUDA(ctx, fill_gaussian(out, (int64_t)b.d.n * b.k, seed, (uint64_t)i, (cudaStream_t)stream));
+    TSR_KERNEL(ctx, 1, fill_gaussian(out, (int64_t)b.d.n * b.k, seed, (uint64_t)i, (cudaStream_t)stream));
+    return TSR_OK;
+}
+
+tsr_status tsr_set_profiling(tsr_ctx *ctx, int32_t enable)
+{
+    if (!ctx) return TSR_ERR_INVALID_ARG;
+    if (enable && !ctx->profiling) {
+        for (cudaEvent_t &e : ctx->ev) TSR_CUDA(ctx, cudaEventCreate(&e));
+        ctx->profiling = true;
+        ctx->ev_valid = false;
+    } else if (!enable && ctx->profiling) {
+        for (cudaEvent_t &e : ctx->ev) { if (e) cudaEventDestroy(e); e = nullptr; }
+        ctx->profiling = false;
+        ctx->ev_valid = false;
+    }
+    return TSR_OK;
+}
+
+tsr_status tsr_get_stage_ms(tsr_ctx *ctx, float *ms, int32_t count)
+{
+    if (!ctx || !ms || count != TSR_NUM_STAGES) return TSR_ERR_INVALID_ARG;
+    if (!ctx->profiling || !ctx->ev_valid) return fail(ctx, TSR_ERR_INVALID_ARG, "no profiled step recorded");
+    TSR_CUDA(ctx, cudaEventSynchronize(ctx->ev[TSR_NUM_STAGES]));
+    for (int i = 0; i < TSR_NUM_STAGES; ++i) TSR_CUDA(ctx, cudaEventElapsedTime(&ms[i], ctx->ev[i], ctx->ev[i + 1]));
+    return TSR_OK;
+}
+
+tsr_status tsr_launch_count(const tsr_ctx *ctx, uint64_t *count)
+{
+    if (!ctx || !count) return TSR_ERR_INVALID_ARG;
+    *count = ctx->launches;
     return TSR_OK;
 }
 
