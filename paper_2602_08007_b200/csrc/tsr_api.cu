@@ -78,6 +78,7 @@ struct tsr_ctx {
     EncodeTiledFn encode = nullptr;
     int max_r = 0, max_k = 0;
     uint64_t launches = 0;                     // kernels launched through this context
+    int num_sms = 148;
     bool profiling = false;
     cudaEvent_t ev[TSR_NUM_STAGES + 1] = {};   // stage boundaries of the last step (profiling only)
     bool ev_valid = false;
@@ -251,6 +252,20 @@ tsr_status encode_map(tsr_ctx *ctx, CUtensorMap *out, const void *base, int64_t 
     return TSR_OK;
 }
 
+// FP32 row-major [rows x cols] (ld elements) -> tensor map with a 32 x 32 box, 128B swizzle.
+tsr_status encode_map_w(tsr_ctx *ctx, CUtensorMap *out, const void *base, int64_t rows, int64_t cols, int64_t ld)
+{
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)ld * 4};
+    cuuint32_t box[2] = {32, 32};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult rc = ctx->encode(out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void *>(base), dims, strides, box, estr,
+                              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (rc != CUDA_SUCCESS) return fail(ctx, TSR_ERR_CUDA, "cuTensorMapEncodeTiled (W) failed (%d)", (int)rc);
+    return TSR_OK;
+}
+
 StepScalars make_scalars(const tsr_hyper *h)
 {
     StepScalars sc;
@@ -328,8 +343,12 @@ tsr_status launch_kind(tsr_ctx *ctx, int kind, const std::vector<int> &list, int
         int lo = ranges[i].first, hi = ranges[i].second;
         size_t j = i + 1;
         while (j < ranges.size() && ranges[j].first == hi) { hi = ranges[j].second; ++j; }
-        TSR_CUDA(ctx, umma_gemm_launch(ctx->d_probs[kind], ctx->d_tiles[kind] + lo, hi - lo, 128, epilogue, planes, sc,
-                                       ctx->d_status, st));
+        if (kind == KA)
+            TSR_CUDA(ctx, umma_apply_launch(ctx->d_probs[kind], ctx->d_tiles[kind] + lo, hi - lo, ctx->num_sms, sc,
+                                            ctx->d_status, st));
+        else
+            TSR_CUDA(ctx, umma_gemm_launch(ctx->d_probs[kind], ctx->d_tiles[kind] + lo, hi - lo, 128, epilogue, planes, sc,
+                                           ctx->d_status, st));
         ctx->launches++;
         i = j;
     }
@@ -722,6 +741,10 @@ tsr_status tsr_bind(tsr_ctx *ctx, const tsr_mat_ptrs *ptrs, int32_t count, void 
             ctx->encode = (EncodeTiledFn)fn;
         }
         TSR_CUDA(ctx, umma_configure());
+        TSR_CUDA(ctx, umma_apply_configure());
+        int dev = 0;
+        TSR_CUDA(ctx, cudaGetDevice(&dev));
+        TSR_CUDA(ctx, cudaDeviceGetAttribute(&ctx->num_sms, cudaDevAttrMultiProcessorCount, dev));
     }
 
     const int nb = count;
@@ -778,6 +801,7 @@ tsr_status tsr_bind(tsr_ctx *ctx, const tsr_mat_ptrs *ptrs, int32_t count, void 
             base(P, (int)m, (int)n, (int)r, EPI_APPLY);
             if ((s = encode_map(ctx, &P.tmA, b.Pb, m, r, b.rl, 128)) != TSR_OK) return s;
             if ((s = encode_map(ctx, &P.tmB, b.Vb, n, r, b.rl, 128)) != TSR_OK) return s;
+            if ((s = encode_map_w(ctx, &P.tmW, b.p.W, m, n, b.d.ldw)) != TSR_OK) return s;
             P.out = b.p.W; P.ld_out = b.d.ldw;
         }
         {   // Y = G X : A = G, B = X^T planes [2k x n]

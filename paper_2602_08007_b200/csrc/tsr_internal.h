@@ -33,6 +33,7 @@ enum UmmaEpilogue : int {
 struct alignas(64) UmmaProblem {
     CUtensorMap tmA;       // box 64 (K) x 128 (M rows), 128-byte swizzle
     CUtensorMap tmB;       // box 64 (K) x BN (N rows); plane 1 lives plane_rows rows below plane 0
+    CUtensorMap tmW;       // apply only: FP32 W, box 32 columns x 32 rows, 128-byte swizzle
     int32_t M, N, K;
     int32_t planes;        // 1 or 2
     int32_t plane_rows;    // row offset of the second plane inside the B tensor map
@@ -68,6 +69,10 @@ struct StepScalars {       // per-step scalars shared by all blocks
 cudaError_t umma_gemm_launch(const UmmaProblem *probs, const UmmaTile *tiles, int num_tiles, int bn, int epilogue,
                              int planes, const StepScalars &sc, int32_t *status, cudaStream_t stream);
 cudaError_t umma_configure();  // sets the dynamic shared-memory attributes once per process
+// Persistent apply kernel (tsr_umma_apply.cu): W <- decay W - step_scale P V^T over a tile table.
+cudaError_t umma_apply_configure();
+cudaError_t umma_apply_launch(const UmmaProblem *probs, const UmmaTile *tiles, int num_tiles, int num_sms,
+                              const StepScalars &sc, int32_t *status, cudaStream_t stream);
 
 // ---------------------------------------------------------------------------------------
 // CUDA-core helpers (tsr_simt.cu)

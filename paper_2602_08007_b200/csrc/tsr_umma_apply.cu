@@ -1,0 +1,251 @@
+// Persistent back-projection + weight update (Section 3.4) on tcgen05 tensor cores:
+//
+//   W[m x n] <- decay * W - step_scale * (P V^T),   P = U D (m x r, BF16),  V (n x r, BF16)
+//
+// The lifted update never reaches memory: each 128 x 128 tile of P V^T is accumulated in tensor
+// memory and consumed by the epilogue, which streams the matching W tile through shared memory
+// with TMA (read-modify-write of 8 bytes per weight is what bounds this kernel).
+//
+// One CTA per SM loops over the tiles of all blocks (static round-robin over a device-resident
+// tile table).  Roles:
+//   warp 0      TMA producer for the P / V operand stages (128-byte swizzle, ring of stages)
+//   warp 1      tensor-memory allocation; one lane issues the MMAs into one of two 128-column
+//               accumulators, so the MMAs of tile i+1 overlap the epilogue of tile i
+//   warps 4-7   epilogue; warp q owns accumulator rows 32q..32q+31 and a private ring of
+//               32 x 32 FP32 W boxes (4 KB, 128-byte swizzle): it prefetches its W boxes
+//               several boxes (more than a tile) ahead, combines them with the accumulator
+//               (tcgen05.ld, lane = row), writes the result back into the same box and issues
+//               the TMA store.  TMA zero-fills loads and clips stores at ragged edges, so no
+//               predicate is needed.
+// All waits are bounded (see mbar_wait); on expiry the CTA flags TSR_ERR_TIMEOUT and drains.
+#include "tsr_internal.h"
+#include "tsr_umma.cuh"
+
+namespace tsr {
+
+constexpr int AP_THREADS = 256;
+constexpr int AP_BN = 128;
+constexpr int AP_STAGES = 4;                 // operand stages: 16 KB (P) + 16 KB (V)
+constexpr int AP_STAGE_BYTES = 32768;
+constexpr int AP_NBOX = 6;                   // W boxes per epilogue warp
+constexpr int AP_LAG = 2;                    // a box is refilled AP_LAG stores after its own store
+constexpr int AP_BOX_BYTES = 4096;
+constexpr int AP_WBOX_OFFSET = AP_STAGES * AP_STAGE_BYTES;
+constexpr int AP_BAR_OFFSET = AP_WBOX_OFFSET + 4 * AP_NBOX * AP_BOX_BYTES;
+constexpr int AP_NBARS = 2 * AP_STAGES + 4 + 4 * AP_NBOX;
+constexpr int AP_SMEM = AP_BAR_OFFSET + AP_NBARS * 8 + 64 + 1024;
+
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, uint32_t src, int x, int y)
+{
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"((uint64_t)map), "r"(src), "r"(x), "r"(y)
+                 : "memory");
+}
+
+struct ChunkCursor {   // walks the (tile, 32-column chunk) sequence of this CTA
+    int tile_idx;      // index into the tile table; >= num_tiles: exhausted
+    int c;             // chunk inside the tile
+    int m0, n0, prob, N, M;
+};
+
+__device__ __forceinline__ void cursor_load(ChunkCursor &cur, const UmmaTile *tiles, const UmmaProblem *probs,
+                                            int num_tiles)
+{
+    if (cur.tile_idx < num_tiles) {
+        const UmmaTile t = tiles[cur.tile_idx];
+        cur.m0 = t.m0; cur.n0 = t.n0; cur.prob = t.prob;
+        cur.N = probs[t.prob].N;
+        cur.M = probs[t.prob].M;
+    }
+}
+__device__ __forceinline__ void cursor_next(ChunkCursor &cur, const UmmaTile *tiles, const UmmaProblem *probs,
+                                            int num_tiles, int stride)
+{
+    cur.c++;
+    if (cur.c >= 4 || cur.n0 + cur.c * 32 >= cur.N) {
+        cur.c = 0;
+        cur.tile_idx += stride;
+        cursor_load(cur, tiles, probs, num_tiles);
+    }
+}
+
+__global__ void __launch_bounds__(AP_THREADS, 1)
+umma_apply_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restrict__ tiles, int num_tiles,
+                  StepScalars sc, int32_t *__restrict__ status)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint64_t *bars = (uint64_t *)(smem + AP_BAR_OFFSET);
+    uint64_t *bar_full = bars;                       // [AP_STAGES]
+    uint64_t *bar_empty = bars + AP_STAGES;          // [AP_STAGES]
+    uint64_t *bar_acc_full = bars + 2 * AP_STAGES;   // [2]
+    uint64_t *bar_acc_empty = bar_acc_full + 2;      // [2]
+    uint64_t *bar_w = bar_acc_empty + 2;             // [4][AP_NBOX]
+    uint32_t *tmem_slot = (uint32_t *)(bars + AP_NBARS);
+    __shared__ int s_timeout;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int stride = gridDim.x;
+
+    if (threadIdx.x == 0) {
+        s_timeout = 0;
+        for (int s = 0; s < AP_STAGES; ++s) { mbar_init(smem_u32(bar_full + s), 1); mbar_init(smem_u32(bar_empty + s), 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(bar_acc_full + b), 1); mbar_init(smem_u32(bar_acc_empty + b), 4); }
+        for (int i = 0; i < 4 * AP_NBOX; ++i) mbar_init(smem_u32(bar_w + i), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(256u)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int t = blockIdx.x; t < num_tiles && ok; t += stride) {
+                const UmmaTile tile = tiles[t];
+                const UmmaProblem *P = probs + tile.prob;
+                const int nkb = (P->K + UM_BK - 1) / UM_BK;
+                for (int kb = 0; kb < nkb; ++kb, ++it) {
+                    const int s = it % AP_STAGES;
+                    const uint32_t ph = (it / AP_STAGES) & 1u;
+                    if (!mbar_wait(smem_u32(bar_empty + s), ph ^ 1u)) { s_timeout = 1; ok = false; break; }
+                    const uint32_t full = smem_u32(bar_full + s);
+                    mbar_expect_tx(full, (uint32_t)AP_STAGE_BYTES);
+                    uint8_t *st = smem + s * AP_STAGE_BYTES;
+                    tma_load_2d(smem_u32(st), &P->tmA, full, kb * UM_BK, tile.m0);
+                    tma_load_2d(smem_u32(st + 16384), &P->tmB, full, kb * UM_BK, tile.n0);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = umma_idesc(AP_BN);
+            uint32_t it = 0, tc = 0;
+            bool ok = true;
+            for (int t = blockIdx.x; t < num_tiles && ok; t += stride, ++tc) {
+                const UmmaTile tile = tiles[t];
+                const int nkb = (probs[tile.prob].K + UM_BK - 1) / UM_BK;
+                const uint32_t buf = tc & 1u;
+                if (!mbar_wait(smem_u32(bar_acc_empty + buf), ((tc >> 1) & 1u) ^ 1u)) { s_timeout = 1; ok = false; break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + buf * AP_BN;
+                for (int kb = 0; kb < nkb; ++kb, ++it) {
+                    const int s = it % AP_STAGES;
+                    const uint32_t ph = (it / AP_STAGES) & 1u;
+                    if (!mbar_wait(smem_u32(bar_full + s), ph)) { s_timeout = 1; ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t a_base = smem_u32(smem + s * AP_STAGE_BYTES);
+                    const uint32_t b_base = a_base + 16384;
+#pragma unroll
+                    for (int k4 = 0; k4 < UM_BK / 16; ++k4)
+                        tc_mma_bf16(d_tmem, umma_desc_sw128(a_base + k4 * 32), umma_desc_sw128(b_base + k4 * 32), idesc,
+                                    (kb | k4) ? 1u : 0u);
+                    tc_commit(smem_u32(bar_empty + s));
+                }
+                tc_commit(smem_u32(bar_acc_full + buf));
+            }
+        }
+    } else if (warp >= 4) {
+        const int q = warp & 3;
+        uint8_t *boxes = smem + AP_WBOX_OFFSET + q * AP_NBOX * AP_BOX_BYTES;
+        uint64_t *wbar = bar_w + q * AP_NBOX;
+        ChunkCursor pre, cur;
+        pre.tile_idx = blockIdx.x; pre.c = 0; pre.m0 = pre.n0 = pre.prob = 0; pre.N = 0; pre.M = 0;
+        cursor_load(pre, tiles, probs, num_tiles);
+        cur = pre;
+        uint32_t issued = 0, cons = 0, tc = 0;
+        bool ok = true;
+        // initial prefetch: AP_NBOX - AP_LAG boxes
+        for (int i = 0; i < AP_NBOX - AP_LAG && pre.tile_idx < num_tiles; ++i) {
+            if (lane == 0) {
+                const uint32_t slot = issued % AP_NBOX;
+                mbar_expect_tx(smem_u32(wbar + slot), AP_BOX_BYTES);
+                tma_load_2d(smem_u32(boxes + slot * AP_BOX_BYTES), &probs[pre.prob].tmW, smem_u32(wbar + slot),
+                            pre.n0 + pre.c * 32, pre.m0 + q * 32);
+            }
+            ++issued;
+            cursor_next(pre, tiles, probs, num_tiles, stride);
+        }
+        while (cur.tile_idx < num_tiles && ok) {
+            const uint32_t buf = tc & 1u;
+            if (cur.c == 0) {
+                if (!mbar_wait(smem_u32(bar_acc_full + buf), (tc >> 1) & 1u)) { s_timeout = 1; ok = false; break; }
+                tc_fence_after();
+            }
+            const uint32_t slot = cons % AP_NBOX;
+            uint32_t v[32];
+            tc_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + buf * AP_BN + (uint32_t)(cur.c * 32), v);
+            const bool last_chunk = (cur.c == 3) || (cur.n0 + (cur.c + 1) * 32 >= cur.N);
+            if (last_chunk) {   // accumulator fully read by this warp: hand it back to the MMA warp
+                tc_fence_before();
+                if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar_acc_empty + buf)) : "memory");
+            }
+            if (!mbar_wait(smem_u32(wbar + slot), (cons / AP_NBOX) & 1u)) { s_timeout = 1; ok = false; break; }
+            uint8_t *box = boxes + slot * AP_BOX_BYTES + lane * 128;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                float4 *p = (float4 *)(box + ((j ^ (lane & 7)) << 4));
+                float4 x = *p;
+                x.x = __fmaf_rn(-sc.step_scale, __uint_as_float(v[4 * j + 0]), __fmul_rn(sc.decay, x.x));
+                x.y = __fmaf_rn(-sc.step_scale, __uint_as_float(v[4 * j + 1]), __fmul_rn(sc.decay, x.y));
+                x.z = __fmaf_rn(-sc.step_scale, __uint_as_float(v[4 * j + 2]), __fmul_rn(sc.decay, x.z));
+                x.w = __fmaf_rn(-sc.step_scale, __uint_as_float(v[4 * j + 3]), __fmul_rn(sc.decay, x.w));
+                *p = x;
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) {
+                if (cur.m0 + q * 32 < cur.M)   // rows past the end were zero-filled on load; nothing to store
+                    tma_store_2d(&probs[cur.prob].tmW, smem_u32(boxes + slot * AP_BOX_BYTES), cur.n0 + cur.c * 32, cur.m0 + q * 32);
+                asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+            }
+            ++cons;
+            // refill the box whose store was issued AP_LAG stores ago
+            if (pre.tile_idx < num_tiles) {
+                if (lane == 0) {
+                    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(AP_LAG - 1) : "memory");
+                    const uint32_t pslot = issued % AP_NBOX;
+                    mbar_expect_tx(smem_u32(wbar + pslot), AP_BOX_BYTES);
+                    tma_load_2d(smem_u32(boxes + pslot * AP_BOX_BYTES), &probs[pre.prob].tmW, smem_u32(wbar + pslot),
+                                pre.n0 + pre.c * 32, pre.m0 + q * 32);
+                }
+                ++issued;
+                cursor_next(pre, tiles, probs, num_tiles, stride);
+            }
+            if (last_chunk) ++tc;
+            cursor_next(cur, tiles, probs, num_tiles, stride);
+        }
+        if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+    }
+    if (s_timeout) __nanosleep(2000000);   // let copies in flight land before the CTA goes away
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(256u) : "memory");
+    }
+    if (threadIdx.x == 0 && s_timeout && status) atomicMax(status, (int)TSR_ERR_TIMEOUT);
+}
+
+cudaError_t umma_apply_configure()
+{
+    return cudaFuncSetAttribute(umma_apply_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, AP_SMEM);
+}
+
+cudaError_t umma_apply_launch(const UmmaProblem *probs, const UmmaTile *tiles, int num_tiles, int num_sms,
+                              const StepScalars &sc, int32_t *status, cudaStream_t stream)
+{
+    if (num_tiles <= 0) return cudaSuccess;
+    const int grid = num_tiles < num_sms ? num_tiles : num_sms;
+    umma_apply_kernel<<<grid, AP_THREADS, AP_SMEM, stream>>>(probs, tiles, num_tiles, sc, status);
+    return cudaGetLastError();
+}
+
+}  // namespace tsr
