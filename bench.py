@@ -221,7 +221,15 @@ def run_ours(args, w: ti.Workload):
     nb = len(w.blocks)
     seed = ti.BASE_SEED
 
-    plan.init_subspace(seed=seed)            # Algorithm 1 initialisation: one refresh on G_0
+    if args.random_bases:
+        # profiling aid: skip the initial refresh, use random (not orthonormal) bases; timings of the
+        # step kernels do not depend on the values
+        for i, b in enumerate(w.blocks):
+            plan.U[i].normal_(0.0, b.m ** -0.5)
+            plan.V[i].normal_(0.0, b.n ** -0.5)
+        plan.bases_changed()
+    else:
+        plan.init_subspace(seed=seed)        # Algorithm 1 initialisation: one refresh on G_0
     torch.cuda.synchronize()
     fresh_gradients(plan, w, 1, device)
     flush = None
@@ -382,6 +390,8 @@ def main():
     ap.add_argument("--refresh-reps", type=int, default=1)
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--random-bases", action="store_true",
+                    help="profiling aid: random bases instead of the initial refresh (numbers not for reporting)")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3

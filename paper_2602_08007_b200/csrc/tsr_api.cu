@@ -79,6 +79,7 @@ struct tsr_ctx {
     int max_r = 0, max_k = 0;
     uint64_t launches = 0;                     // kernels launched through this context
     int num_sms = 148;
+    int bn[NKIND] = {128, 128, 128, 128, 128, 128, 128};   // tile width of each GEMM kind
     bool profiling = false;
     cudaEvent_t ev[TSR_NUM_STAGES + 1] = {};   // stage boundaries of the last step (profiling only)
     bool ev_valid = false;
@@ -199,13 +200,14 @@ void layout(tsr_ctx *ctx, Arena &a, bool assign, size_t *step_end)
 
 void add_tiles(tsr_ctx *ctx, int kind, int bi, int M, int N, int K, int kb_per_split)
 {
+    const int bn = ctx->bn[kind];
     Block &b = ctx->blocks[bi];
     std::vector<UmmaTile> &v = ctx->tiles[kind];
     b.tile_begin[kind] = (int)v.size();
     const int nkb = (K + 63) / 64;
     const int nsp = kb_per_split > 0 ? (nkb + kb_per_split - 1) / kb_per_split : 1;
     for (int m0 = 0; m0 < M; m0 += 128)
-        for (int n0 = 0; n0 < N; n0 += 128)
+        for (int n0 = 0; n0 < N; n0 += bn)
             for (int s = 0; s < nsp; ++s) {
                 UmmaTile t;
                 t.prob = bi; t.m0 = m0; t.n0 = n0;
@@ -220,6 +222,9 @@ void add_tiles(tsr_ctx *ctx, int kind, int bi, int M, int N, int K, int kb_per_s
 void build_tiles(tsr_ctx *ctx)
 {
     for (int kd = 0; kd < NKIND; ++kd) ctx->tiles[kd].clear();
+    int rmax = 0;
+    for (const Block &b : ctx->blocks) if (b.fast) rmax = std::max(rmax, (int)b.d.r);
+    for (int kd : {KT, KC, KCS, KP}) ctx->bn[kd] = rmax >= 256 ? 256 : 128;
     for (int bi : ctx->order) {
         Block &b = ctx->blocks[bi];
         for (int kd = 0; kd < NKIND; ++kd) b.tile_begin[kd] = b.tile_end[kd] = (int)ctx->tiles[kd].size();
@@ -347,8 +352,8 @@ tsr_status launch_kind(tsr_ctx *ctx, int kind, const std::vector<int> &list, int
             TSR_CUDA(ctx, umma_apply_launch(ctx->d_probs[kind], ctx->d_tiles[kind] + lo, hi - lo, ctx->num_sms, sc,
                                             ctx->d_status, st));
         else
-            TSR_CUDA(ctx, umma_gemm_launch(ctx->d_probs[kind], ctx->d_tiles[kind] + lo, hi - lo, 128, epilogue, planes, sc,
-                                           ctx->d_status, st));
+            TSR_CUDA(ctx, umma_gemm_launch(ctx->d_probs[kind], ctx->d_tiles[kind] + lo, hi - lo, ctx->num_sms, ctx->bn[kind],
+                                           epilogue, planes, sc, ctx->d_status, st));
         ctx->launches++;
         i = j;
     }
@@ -777,14 +782,14 @@ tsr_status tsr_bind(tsr_ctx *ctx, const tsr_mat_ptrs *ptrs, int32_t count, void 
             UmmaProblem &P = probs[KT][i];
             base(P, (int)m, (int)r, (int)n, EPI_STORE_BF16_T);
             if ((s = encode_map(ctx, &P.tmA, b.p.G, m, n, b.d.ldg, 128)) != TSR_OK) return s;
-            if ((s = encode_map(ctx, &P.tmB, b.Vbt, r, n, b.nl, 128)) != TSR_OK) return s;
+            if ((s = encode_map(ctx, &P.tmB, b.Vbt, r, n, b.nl, ctx->bn[KT])) != TSR_OK) return s;
             P.out = b.Tt; P.ld_out = b.ml;
         }
         for (int kd : {KC, KCS}) {   // C = U^T T : A = U^T copy [r x m], B = T~ [r x m]
             UmmaProblem &P = probs[kd][i];
             base(P, (int)r, (int)r, (int)m, EPI_CORE_UPDATE);
             if ((s = encode_map(ctx, &P.tmA, b.Ubt, r, m, b.ml, 128)) != TSR_OK) return s;
-            if ((s = encode_map(ctx, &P.tmB, b.Tt, r, m, b.ml, 128)) != TSR_OK) return s;
+            if ((s = encode_map(ctx, &P.tmB, b.Tt, r, m, b.ml, ctx->bn[kd])) != TSR_OK) return s;
             P.out = (kd == KC) ? (void *)b.p.C : (void *)b.partial;
             P.ld_out = r; P.split_stride = r * r;
             P.mom1 = b.p.M; P.mom2 = b.p.Vm; P.d_bf16 = b.Db; P.dt_bf16 = b.Dbt; P.ldd = b.rl;
@@ -793,7 +798,7 @@ tsr_status tsr_bind(tsr_ctx *ctx, const tsr_mat_ptrs *ptrs, int32_t count, void 
             UmmaProblem &P = probs[KP][i];
             base(P, (int)m, (int)r, (int)r, EPI_STORE_BF16);
             if ((s = encode_map(ctx, &P.tmA, b.Ub, m, r, b.rl, 128)) != TSR_OK) return s;
-            if ((s = encode_map(ctx, &P.tmB, b.Dbt, r, r, b.rl, 128)) != TSR_OK) return s;
+            if ((s = encode_map(ctx, &P.tmB, b.Dbt, r, r, b.rl, ctx->bn[KP])) != TSR_OK) return s;
             P.out = b.Pb; P.ld_out = b.rl;
         }
         {   // W update : A = P [m x r], B = V copy [n x r]

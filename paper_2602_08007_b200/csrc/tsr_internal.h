@@ -65,9 +65,9 @@ struct StepScalars {       // per-step scalars shared by all blocks
     int32_t rule;           // tsr_rule
 };
 
-// Launchers (tsr_umma.cu).  tiles / probs are device pointers.  bn = 64, 128 or 256.
-cudaError_t umma_gemm_launch(const UmmaProblem *probs, const UmmaTile *tiles, int num_tiles, int bn, int epilogue,
-                             int planes, const StepScalars &sc, int32_t *status, cudaStream_t stream);
+// Launchers (tsr_umma.cu).  tiles / probs are device pointers.  bn = 128 or 256 (tile width).
+cudaError_t umma_gemm_launch(const UmmaProblem *probs, const UmmaTile *tiles, int num_tiles, int num_sms, int bn,
+                             int epilogue, int planes, const StepScalars &sc, int32_t *status, cudaStream_t stream);
 cudaError_t umma_configure();  // sets the dynamic shared-memory attributes once per process
 // Persistent apply kernel (tsr_umma_apply.cu): W <- decay W - step_scale P V^T over a tile table.
 cudaError_t umma_apply_configure();

@@ -1,71 +1,70 @@
-// Grouped BF16 GEMM on the 5th-generation tensor cores (tcgen05) for sm_100a.
+// Grouped, persistent BF16 GEMM on the 5th-generation tensor cores (tcgen05) for sm_100a.
 //
 //   D[M x N] = A[M x K] * B[N x K]^T     A, B BF16 with K contiguous, FP32 accumulation
 //
-// One CTA computes one 128 x BN output tile listed in a device-resident tile table (tiles of
-// all matrix blocks of a model share one launch).  Roles inside the CTA:
+// One CTA per SM walks a device-resident tile table (tiles of all matrix blocks of a model
+// share one launch; static round-robin).  A tile is 128 x BN outputs over a range of 64-wide
+// K blocks.  Roles inside the CTA:
 //   warp 0    one lane issues the TMA loads (128-byte swizzled 64-wide K slices) into a ring of
 //             shared-memory stages and signals "full" mbarriers with the byte count;
-//   warp 1    allocates tensor memory; one lane issues tcgen05.mma (128 x BN x 16 per
-//             instruction) from shared-memory descriptors into the TMEM accumulator and
-//             commits to the "empty" mbarrier of the stage, finally to the "accumulator ready"
-//             mbarrier;
-//   warps 2-5 read the accumulator with tcgen05.ld (lane = output row) and run the epilogue:
-//             plain / transposed stores, the fused core update of Section 3.4, or the fused
-//             weight update W <- decay * W - step_scale * acc (the lifted update never reaches
-//             memory).
+//   warp 1    allocates tensor memory (two accumulators of BN columns); one lane issues
+//             tcgen05.mma (128 x N x 16 per instruction, N = the tile's width rounded up to 16)
+//             from shared-memory descriptors and commits to the stage's "empty" mbarrier and,
+//             per tile, to the accumulator's "full" mbarrier.  The MMAs of tile i+1 overlap the
+//             epilogue of tile i;
+//   warps 4-7 read the accumulator with tcgen05.ld (lane = output row, 32 columns at a time).
+//             Row-major outputs are transposed through a warp-private shared-memory patch so
+//             that every global access is a full 128-byte (FP32) or 64-byte (BF16) row
+//             segment.  Epilogues: plain FP32 / BF16 stores, the transposed BF16 store, and the
+//             fused core update of Section 3.4.
 // Ragged edges rely on TMA zero fill for loads and on predicated stores.
 // Every mbarrier wait is bounded by a clock budget; on expiry the CTA records
-// TSR_ERR_TIMEOUT in the block's status word, skips its stores and still releases its tensor
-// memory before it exits.
+// TSR_ERR_TIMEOUT, stops storing and still releases its tensor memory before it exits.
 #include "tsr_device.cuh"
 #include "tsr_internal.h"
 #include "tsr_umma.cuh"
 
 namespace tsr {
 
-template <int EPI>
-struct UmmaCfg {
-    static constexpr int STAGES = (EPI == EPI_APPLY || EPI == EPI_STORE_BF16) ? 2 : 4;
-};
+constexpr int UG_THREADS = 256;
 
-template <int BN, int PLANES, int STAGES>
+template <int BN, int PLANES>
 struct UmmaSmem {
     static constexpr int A_BYTES = UM_BM * UM_BK * 2;
     static constexpr int B_BYTES = BN * UM_BK * 2;
     static constexpr int STAGE_BYTES = A_BYTES + PLANES * B_BYTES;
-    static constexpr int BAR_OFFSET = STAGES * STAGE_BYTES;
-    static constexpr int TOTAL = BAR_OFFSET + 256 + 1024;  // barriers + slack for 1024-byte alignment
+    static constexpr int STAGES = (192 * 1024) / STAGE_BYTES > 6 ? 6 : (192 * 1024) / STAGE_BYTES;
+    static constexpr int PATCH_OFFSET = STAGES * STAGE_BYTES;
+    static constexpr int PATCH_BYTES = 32 * 33 * 4;                  // per epilogue warp
+    static constexpr int BAR_OFFSET = PATCH_OFFSET + 4 * PATCH_BYTES;
+    static constexpr int NBARS = 2 * STAGES + 4;
+    static constexpr int TOTAL = BAR_OFFSET + NBARS * 8 + 64 + 1024;  // + slack for 1024-byte alignment
 };
 
 template <int BN, int EPI, int PLANES>
-__global__ void __launch_bounds__(UM_THREADS)
-umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restrict__ tiles, StepScalars sc,
-                 int32_t *__restrict__ status)
+__global__ void __launch_bounds__(UG_THREADS, 1)
+umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restrict__ tiles, int num_tiles,
+                 StepScalars sc, int32_t *__restrict__ status)
 {
-    constexpr int STAGES = UmmaCfg<EPI>::STAGES;
-    using SM = UmmaSmem<BN, PLANES, STAGES>;
-    constexpr uint32_t TMEM_COLS = (BN <= 32) ? 32 : (BN <= 64 ? 64 : (BN <= 128 ? 128 : 256));
+    using SM = UmmaSmem<BN, PLANES>;
+    constexpr int STAGES = SM::STAGES;
+    constexpr uint32_t TMEM_COLS = 2 * BN;   // 256 or 512
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint64_t *bars = (uint64_t *)(smem + SM::BAR_OFFSET);
-    // bars[0..STAGES) full, [STAGES..2*STAGES) empty, [2*STAGES] accumulator ready
-    uint32_t *tmem_slot = (uint32_t *)(bars + 2 * STAGES + 1);
+    uint64_t *bar_full = bars, *bar_empty = bars + STAGES;
+    uint64_t *bar_acc_full = bars + 2 * STAGES, *bar_acc_empty = bar_acc_full + 2;
+    uint32_t *tmem_slot = (uint32_t *)(bars + SM::NBARS);
     __shared__ int s_timeout;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const UmmaTile tile = tiles[blockIdx.x];
-    const UmmaProblem *__restrict__ P = probs + tile.prob;
-    const int nkb = tile.kb1 - tile.kb0;
+    const int stride = gridDim.x;
 
     if (threadIdx.x == 0) {
         s_timeout = 0;
-        for (int s = 0; s < STAGES; ++s) {
-            mbar_init(smem_u32(bars + s), 1);
-            mbar_init(smem_u32(bars + STAGES + s), 1);
-        }
-        mbar_init(smem_u32(bars + 2 * STAGES), 1);
+        for (int s = 0; s < STAGES; ++s) { mbar_init(smem_u32(bar_full + s), 1); mbar_init(smem_u32(bar_empty + s), 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(bar_acc_full + b), 1); mbar_init(smem_u32(bar_acc_empty + b), 4); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
@@ -81,154 +80,243 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
 
     if (warp == 0) {
         if (lane == 0) {
-            for (int i = 0; i < nkb; ++i) {
-                const int s = i % STAGES;
-                const uint32_t ph = (uint32_t)(i / STAGES) & 1u;
-                if (!mbar_wait(smem_u32(bars + STAGES + s), ph ^ 1u)) { s_timeout = 1; break; }
-                const uint32_t full = smem_u32(bars + s);
-                mbar_expect_tx(full, (uint32_t)SM::STAGE_BYTES);
-                uint8_t *st = smem + s * SM::STAGE_BYTES;
-                const int kx = (tile.kb0 + i) * UM_BK;
-                tma_load_2d(smem_u32(st), &P->tmA, full, kx, tile.m0);
+            uint32_t it = 0;
+            bool ok = true;
+            for (int t = blockIdx.x; t < num_tiles && ok; t += stride) {
+                const UmmaTile tile = tiles[t];
+                const UmmaProblem *P = probs + tile.prob;
+                for (int kb = tile.kb0; kb < tile.kb1; ++kb, ++it) {
+                    const int s = it % STAGES;
+                    const uint32_t ph = (it / STAGES) & 1u;
+                    if (!mbar_wait(smem_u32(bar_empty + s), ph ^ 1u)) { s_timeout = 1; ok = false; break; }
+                    const uint32_t full = smem_u32(bar_full + s);
+                    mbar_expect_tx(full, (uint32_t)SM::STAGE_BYTES);
+                    uint8_t *st = smem + s * SM::STAGE_BYTES;
+                    tma_load_2d(smem_u32(st), &P->tmA, full, kb * UM_BK, tile.m0);
 #pragma unroll
-                for (int pl = 0; pl < PLANES; ++pl)
-                    tma_load_2d(smem_u32(st + SM::A_BYTES + pl * SM::B_BYTES), &P->tmB, full, kx,
-                                tile.n0 + pl * P->plane_rows);
+                    for (int pl = 0; pl < PLANES; ++pl)
+                        tma_load_2d(smem_u32(st + SM::A_BYTES + pl * SM::B_BYTES), &P->tmB, full, kb * UM_BK,
+                                    tile.n0 + pl * P->plane_rows);
+                }
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            constexpr uint32_t idesc = umma_idesc(BN);
+            uint32_t it = 0, tc = 0;
             bool ok = true;
-            for (int i = 0; i < nkb && ok; ++i) {
-                const int s = i % STAGES;
-                const uint32_t ph = (uint32_t)(i / STAGES) & 1u;
-                if (!mbar_wait(smem_u32(bars + s), ph)) { s_timeout = 1; ok = false; break; }
+            for (int t = blockIdx.x; t < num_tiles && ok; t += stride, ++tc) {
+                const UmmaTile tile = tiles[t];
+                int n_eff = probs[tile.prob].N - tile.n0;
+                n_eff = n_eff >= BN ? BN : ((n_eff + 15) & ~15);
+                const uint32_t idesc = umma_idesc(n_eff);
+                const uint32_t buf = tc & 1u;
+                if (!mbar_wait(smem_u32(bar_acc_empty + buf), ((tc >> 1) & 1u) ^ 1u)) { s_timeout = 1; ok = false; break; }
                 tc_fence_after();
-                const uint32_t a_base = smem_u32(smem + s * SM::STAGE_BYTES);
+                const uint32_t d_tmem = tmem_base + buf * BN;
+                for (int kb = tile.kb0; kb < tile.kb1; ++kb, ++it) {
+                    const int s = it % STAGES;
+                    const uint32_t ph = (it / STAGES) & 1u;
+                    if (!mbar_wait(smem_u32(bar_full + s), ph)) { s_timeout = 1; ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t a_base = smem_u32(smem + s * SM::STAGE_BYTES);
 #pragma unroll
-                for (int pl = 0; pl < PLANES; ++pl) {
-                    const uint32_t b_base = a_base + SM::A_BYTES + pl * SM::B_BYTES;
+                    for (int pl = 0; pl < PLANES; ++pl) {
+                        const uint32_t b_base = a_base + SM::A_BYTES + pl * SM::B_BYTES;
 #pragma unroll
-                    for (int k4 = 0; k4 < UM_BK / 16; ++k4) {
-                        const uint64_t adesc = umma_desc_sw128(a_base + k4 * 32);
-                        const uint64_t bdesc = umma_desc_sw128(b_base + k4 * 32);
-                        tc_mma_bf16(tmem_base, adesc, bdesc, idesc, (i | pl | k4) ? 1u : 0u);
+                        for (int k4 = 0; k4 < UM_BK / 16; ++k4)
+                            tc_mma_bf16(d_tmem, umma_desc_sw128(a_base + k4 * 32), umma_desc_sw128(b_base + k4 * 32),
+                                        idesc, ((kb - tile.kb0) | pl | k4) ? 1u : 0u);
                     }
+                    tc_commit(smem_u32(bar_empty + s));
                 }
-                tc_commit(smem_u32(bars + STAGES + s));
+                tc_commit(smem_u32(bar_acc_full + buf));
             }
-            tc_commit(smem_u32(bars + 2 * STAGES));
         }
-    } else {
-        // epilogue: warps 2..5 own TMEM lane quarters (warp % 4)
-        const int quarter = warp & 3;
-        bool ok = mbar_wait(smem_u32(bars + 2 * STAGES), 0);
-        if (!ok) s_timeout = 1;
-        ok = ok && (s_timeout == 0);
-        tc_fence_after();
-        const int row = tile.m0 + quarter * 32 + lane;
-        const bool row_ok = ok && row < P->M;
-        const int N = P->N;
+    } else if (warp >= 4) {
+        const int q = warp & 3;
+        float *patch = (float *)(smem + SM::PATCH_OFFSET + q * SM::PATCH_BYTES);   // [32][33]
+        uint32_t tc = 0;
+        bool ok = true;
+        for (int t = blockIdx.x; t < num_tiles && ok; t += stride, ++tc) {
+            const UmmaTile tile = tiles[t];
+            const UmmaProblem *__restrict__ P = probs + tile.prob;
+            const uint32_t buf = tc & 1u;
+            if (!mbar_wait(smem_u32(bar_acc_full + buf), (tc >> 1) & 1u)) { s_timeout = 1; ok = false; break; }
+            tc_fence_after();
+            const int N = P->N, M = P->M;
+            const int row0 = tile.m0 + q * 32;
+            const int nrows = min(32, M - row0);        // may be <= 0
 #pragma unroll 1
-        for (int c0 = 0; c0 < BN; c0 += 32) {
-            if (tile.n0 + c0 >= N) break;
-            uint32_t v[32];
-            tc_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c0, v);
-            if (!row_ok) continue;
-            const int col0 = tile.n0 + c0;
-            const bool full_chunk = (col0 + 32 <= N);
-            if (EPI == EPI_STORE_F32) {
-                float *out = (float *)P->out + (int64_t)tile.split * P->split_stride + (int64_t)row * P->ld_out + col0;
-                if (full_chunk && (P->ld_out & 3) == 0 && (col0 & 3) == 0) {
-#pragma unroll
-                    for (int j = 0; j < 32; j += 4)
-                        *(float4 *)(out + j) = make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]),
-                                                           __uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
-                } else {
-                    for (int j = 0; j < 32 && col0 + j < N; ++j) out[j] = __uint_as_float(v[j]);
+            for (int c0 = 0; c0 < BN; c0 += 32) {
+                const int col0 = tile.n0 + c0;
+                if (col0 >= N) break;
+                uint32_t v[32];
+                tc_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + buf * BN + (uint32_t)c0, v);
+                if (c0 + 32 >= BN || col0 + 32 >= N) {   // last chunk of the tile: release the accumulator
+                    tc_fence_before();
+                    if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar_acc_empty + buf)) : "memory");
                 }
-            } else if (EPI == EPI_STORE_BF16) {
-                bf16 *out = (bf16 *)P->out + (int64_t)row * P->ld_out + col0;
-                if (full_chunk && (P->ld_out & 7) == 0) {
+                if (nrows <= 0) continue;
+                const int ncols = min(32, N - col0);
+                if (EPI == EPI_STORE_BF16_T) {
+                    // out[col][row]: for a fixed column the 32 lanes hold 32 consecutive rows
+                    bf16 *out = (bf16 *)P->out + (int64_t)col0 * P->ld_out + row0 + lane;
+                    if (lane < nrows) {
 #pragma unroll
-                    for (int j = 0; j < 32; j += 8) {
-                        uint4 pk;
-                        __nv_bfloat162 h0 = __floats2bfloat162_rn(__uint_as_float(v[j]), __uint_as_float(v[j + 1]));
-                        __nv_bfloat162 h1 = __floats2bfloat162_rn(__uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
-                        __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(v[j + 4]), __uint_as_float(v[j + 5]));
-                        __nv_bfloat162 h3 = __floats2bfloat162_rn(__uint_as_float(v[j + 6]), __uint_as_float(v[j + 7]));
-                        pk.x = *(uint32_t *)&h0; pk.y = *(uint32_t *)&h1; pk.z = *(uint32_t *)&h2; pk.w = *(uint32_t *)&h3;
-                        *(uint4 *)(out + j) = pk;
+                        for (int j = 0; j < 32; ++j)
+                            if (j < ncols) out[(int64_t)j * P->ld_out] = __float2bfloat16_rn(__uint_as_float(v[j]));
                     }
-                } else {
-                    for (int j = 0; j < 32 && col0 + j < N; ++j) out[j] = __float2bfloat16_rn(__uint_as_float(v[j]));
+                    continue;
                 }
-            } else if (EPI == EPI_STORE_BF16_T) {
-                bf16 *out = (bf16 *)P->out + (int64_t)col0 * P->ld_out + row;
+                // Fast paths (full 32-column chunk, aligned rows): lane = row, each lane moves whole
+                // 32-byte sectors of its own row.
+                const bool full_chunk = (ncols == 32);
+                if (EPI == EPI_STORE_F32 && full_chunk && (P->ld_out & 3) == 0 && (col0 & 3) == 0 &&
+                    (((uintptr_t)P->out) & 15) == 0 && (P->split_stride & 3) == 0) {
+                    if (lane < nrows) {
+                        float *out = (float *)P->out + (int64_t)tile.split * P->split_stride + (int64_t)(row0 + lane) * P->ld_out + col0;
 #pragma unroll
-                for (int j = 0; j < 32; ++j)
-                    if (col0 + j < N) out[(int64_t)j * P->ld_out] = __float2bfloat16_rn(__uint_as_float(v[j]));
-            } else if (EPI == EPI_CORE_UPDATE) {
-                const int64_t base = (int64_t)row * N + col0;  // C, M, Vm are dense r x r (N = r)
-                float *Cc = (float *)P->out + base;
-                float *m1p = P->mom1 + base;
-                float *m2p = P->mom2 + base;
-                bf16 *dp = P->d_bf16 + (int64_t)row * P->ldd + col0;
-                bf16 *dtp = P->dt_bf16 + (int64_t)col0 * P->ldd + row;
-                for (int j = 0; j < 32 && col0 + j < N; ++j) {
-                    const float c = __uint_as_float(v[j]);
-                    float m1 = m1p[j];
-                    float m2 = (sc.rule == TSR_RULE_SGD) ? 0.f : m2p[j];
-                    const float dd = core_update_elem(c, m1, m2, sc);
-                    Cc[j] = c;
-                    m1p[j] = m1;
-                    if (sc.rule != TSR_RULE_SGD) m2p[j] = m2;
-                    const bf16 db = __float2bfloat16_rn(dd);
-                    dp[j] = db;
-                    dtp[(int64_t)j * P->ldd] = db;
-                }
-            } else if (EPI == EPI_APPLY) {
-                float *w = (float *)P->out + (int64_t)row * P->ld_out + col0;
-                if (full_chunk && (P->ld_out & 3) == 0 && (col0 & 3) == 0) {
-#pragma unroll
-                    for (int j = 0; j < 32; j += 4) {
-                        float4 x = *(float4 *)(w + j);
-                        x.x = __fmaf_rn(-sc.step_scale, __uint_as_float(v[j]), __fmul_rn(sc.decay, x.x));
-                        x.y = __fmaf_rn(-sc.step_scale, __uint_as_float(v[j + 1]), __fmul_rn(sc.decay, x.y));
-                        x.z = __fmaf_rn(-sc.step_scale, __uint_as_float(v[j + 2]), __fmul_rn(sc.decay, x.z));
-                        x.w = __fmaf_rn(-sc.step_scale, __uint_as_float(v[j + 3]), __fmul_rn(sc.decay, x.w));
-                        *(float4 *)(w + j) = x;
+                        for (int j = 0; j < 32; j += 4)
+                            *(float4 *)(out + j) = make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]),
+                                                               __uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
                     }
-                } else {
-                    for (int j = 0; j < 32 && col0 + j < N; ++j)
-                        w[j] = __fmaf_rn(-sc.step_scale, __uint_as_float(v[j]), __fmul_rn(sc.decay, w[j]));
+                    continue;
                 }
+                if (EPI == EPI_STORE_BF16 && full_chunk && (P->ld_out & 7) == 0 && (col0 & 7) == 0 &&
+                    (((uintptr_t)P->out) & 15) == 0) {
+                    if (lane < nrows) {
+                        bf16 *out = (bf16 *)P->out + (int64_t)(row0 + lane) * P->ld_out + col0;
+#pragma unroll
+                        for (int j = 0; j < 32; j += 8) {
+                            uint4 pk;
+                            __nv_bfloat162 h0 = __floats2bfloat162_rn(__uint_as_float(v[j]), __uint_as_float(v[j + 1]));
+                            __nv_bfloat162 h1 = __floats2bfloat162_rn(__uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
+                            __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(v[j + 4]), __uint_as_float(v[j + 5]));
+                            __nv_bfloat162 h3 = __floats2bfloat162_rn(__uint_as_float(v[j + 6]), __uint_as_float(v[j + 7]));
+                            pk.x = *(uint32_t *)&h0; pk.y = *(uint32_t *)&h1; pk.z = *(uint32_t *)&h2; pk.w = *(uint32_t *)&h3;
+                            *(uint4 *)(out + j) = pk;
+                        }
+                    }
+                    continue;
+                }
+                if (EPI == EPI_CORE_UPDATE && full_chunk && (N & 7) == 0 && (P->ldd & 7) == 0 &&
+                    ((((uintptr_t)P->out) | ((uintptr_t)P->mom1) | ((uintptr_t)P->mom2) | ((uintptr_t)P->d_bf16)) & 15) == 0) {
+                    if (lane < nrows) {
+                        const int64_t e0 = (int64_t)(row0 + lane) * N + col0;   // C, M, Vm are dense r x r (N = r)
+                        float *cp = (float *)P->out + e0;
+                        float *m1p = P->mom1 + e0;
+                        float *m2p = P->mom2 + e0;
+                        bf16 *dp = P->d_bf16 + (int64_t)(row0 + lane) * P->ldd + col0;
+                        bf16 *dtp = P->dt_bf16 + (int64_t)col0 * P->ldd + row0 + lane;
+                        const int64_t ldd = P->ldd;
+                        const bool sgd = (sc.rule == TSR_RULE_SGD);
+                        float m1[32], m2[32];
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4) {
+                            const float4 a = *(const float4 *)(m1p + j);
+                            m1[j] = a.x; m1[j + 1] = a.y; m1[j + 2] = a.z; m1[j + 3] = a.w;
+                        }
+                        if (!sgd) {
+#pragma unroll
+                            for (int j = 0; j < 32; j += 4) {
+                                const float4 a = *(const float4 *)(m2p + j);
+                                m2[j] = a.x; m2[j + 1] = a.y; m2[j + 2] = a.z; m2[j + 3] = a.w;
+                            }
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) m2[j] = 0.f;
+                        }
+                        float dd[32];
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) dd[j] = core_update_elem(__uint_as_float(v[j]), m1[j], m2[j], sc);
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4) {
+                            *(float4 *)(cp + j) = make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]),
+                                                              __uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
+                            *(float4 *)(m1p + j) = make_float4(m1[j], m1[j + 1], m1[j + 2], m1[j + 3]);
+                            if (!sgd) *(float4 *)(m2p + j) = make_float4(m2[j], m2[j + 1], m2[j + 2], m2[j + 3]);
+                        }
+#pragma unroll
+                        for (int j = 0; j < 32; j += 8) {
+                            uint4 pk;
+                            __nv_bfloat162 h0 = __floats2bfloat162_rn(dd[j], dd[j + 1]);
+                            __nv_bfloat162 h1 = __floats2bfloat162_rn(dd[j + 2], dd[j + 3]);
+                            __nv_bfloat162 h2 = __floats2bfloat162_rn(dd[j + 4], dd[j + 5]);
+                            __nv_bfloat162 h3 = __floats2bfloat162_rn(dd[j + 6], dd[j + 7]);
+                            pk.x = *(uint32_t *)&h0; pk.y = *(uint32_t *)&h1; pk.z = *(uint32_t *)&h2; pk.w = *(uint32_t *)&h3;
+                            *(uint4 *)(dp + j) = pk;
+                        }
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) dtp[(int64_t)j * ldd] = __float2bfloat16_rn(dd[j]);
+                    }
+                    continue;
+                }
+                // Ragged or unaligned chunk: transpose through the patch so that lane = column and
+                // the loop index = row; accesses stay row-contiguous.
+#pragma unroll
+                for (int j = 0; j < 32; ++j) patch[lane * 33 + j] = __uint_as_float(v[j]);
+                __syncwarp();
+                const int col = col0 + lane;
+                const bool col_ok = lane < ncols;
+                if (EPI == EPI_STORE_F32) {
+                    float *out = (float *)P->out + (int64_t)tile.split * P->split_stride + (int64_t)row0 * P->ld_out + col;
+                    if (col_ok)
+                        for (int i = 0; i < nrows; ++i) out[(int64_t)i * P->ld_out] = patch[i * 33 + lane];
+                } else if (EPI == EPI_STORE_BF16) {
+                    bf16 *out = (bf16 *)P->out + (int64_t)row0 * P->ld_out + col;
+                    if (col_ok)
+                        for (int i = 0; i < nrows; ++i) out[(int64_t)i * P->ld_out] = __float2bfloat16_rn(patch[i * 33 + lane]);
+                } else if (EPI == EPI_CORE_UPDATE) {
+                    // C, M, Vm are dense r x r (N = r)
+                    if (col_ok) {
+                        for (int i = 0; i < nrows; ++i) {
+                            const int64_t e = (int64_t)(row0 + i) * N + col;
+                            const float c = patch[i * 33 + lane];
+                            float m1 = P->mom1[e];
+                            float m2 = (sc.rule == TSR_RULE_SGD) ? 0.f : P->mom2[e];
+                            const float dd = core_update_elem(c, m1, m2, sc);
+                            ((float *)P->out)[e] = c;
+                            P->mom1[e] = m1;
+                            if (sc.rule != TSR_RULE_SGD) P->mom2[e] = m2;
+                            P->d_bf16[(int64_t)(row0 + i) * P->ldd + col] = __float2bfloat16_rn(dd);
+                            patch[i * 33 + lane] = dd;
+                        }
+                    }
+                    __syncwarp();
+                    // D^T: back to lane = row
+                    if (lane < nrows) {
+                        bf16 *dt = P->dt_bf16 + (int64_t)col0 * P->ldd + row0 + lane;
+                        for (int j = 0; j < ncols; ++j) dt[(int64_t)j * P->ldd] = __float2bfloat16_rn(patch[lane * 33 + j]);
+                    }
+                }
+                __syncwarp();
             }
         }
     }
+    if (s_timeout) __nanosleep(2000000);   // let copies in flight land before the CTA goes away
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
     }
-    if (threadIdx.x == 0 && s_timeout && status) atomicMax(status + P->block, (int)TSR_ERR_TIMEOUT);
+    if (threadIdx.x == 0 && s_timeout && status) atomicMax(status, (int)TSR_ERR_TIMEOUT);
 }
 
 template <int BN, int EPI, int PLANES>
-static cudaError_t launch_one(const UmmaProblem *probs, const UmmaTile *tiles, int num_tiles, const StepScalars &sc,
-                              int32_t *status, cudaStream_t stream)
+static cudaError_t launch_one(const UmmaProblem *probs, const UmmaTile *tiles, int num_tiles, int num_sms,
+                              const StepScalars &sc, int32_t *status, cudaStream_t stream)
 {
-    using SM = UmmaSmem<BN, PLANES, UmmaCfg<EPI>::STAGES>;
-    umma_gemm_kernel<BN, EPI, PLANES><<<num_tiles, UM_THREADS, SM::TOTAL, stream>>>(probs, tiles, sc, status);
+    using SM = UmmaSmem<BN, PLANES>;
+    const int grid = num_tiles < num_sms ? num_tiles : num_sms;
+    umma_gemm_kernel<BN, EPI, PLANES><<<grid, UG_THREADS, SM::TOTAL, stream>>>(probs, tiles, num_tiles, sc, status);
     return cudaGetLastError();
 }
 
 template <int BN, int EPI, int PLANES>
 static cudaError_t configure_one()
 {
-    using SM = UmmaSmem<BN, PLANES, UmmaCfg<EPI>::STAGES>;
+    using SM = UmmaSmem<BN, PLANES>;
     return cudaFuncSetAttribute(umma_gemm_kernel<BN, EPI, PLANES>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 SM::TOTAL);
 }
@@ -237,29 +325,46 @@ cudaError_t umma_configure()
 {
     cudaError_t e;
     if ((e = configure_one<128, EPI_STORE_F32, 1>()) != cudaSuccess) return e;
+    if ((e = configure_one<256, EPI_STORE_F32, 1>()) != cudaSuccess) return e;
     if ((e = configure_one<128, EPI_STORE_F32, 2>()) != cudaSuccess) return e;
     if ((e = configure_one<128, EPI_STORE_BF16, 1>()) != cudaSuccess) return e;
+    if ((e = configure_one<256, EPI_STORE_BF16, 1>()) != cudaSuccess) return e;
     if ((e = configure_one<128, EPI_STORE_BF16_T, 1>()) != cudaSuccess) return e;
+    if ((e = configure_one<256, EPI_STORE_BF16_T, 1>()) != cudaSuccess) return e;
     if ((e = configure_one<128, EPI_CORE_UPDATE, 1>()) != cudaSuccess) return e;
-    if ((e = configure_one<128, EPI_APPLY, 1>()) != cudaSuccess) return e;
+    if ((e = configure_one<256, EPI_CORE_UPDATE, 1>()) != cudaSuccess) return e;
     return cudaSuccess;
 }
 
-cudaError_t umma_gemm_launch(const UmmaProblem *probs, const UmmaTile *tiles, int num_tiles, int bn, int epilogue,
-                             int planes, const StepScalars &sc, int32_t *status, cudaStream_t stream)
+cudaError_t umma_gemm_launch(const UmmaProblem *probs, const UmmaTile *tiles, int num_tiles, int num_sms, int bn,
+                             int epilogue, int planes, const StepScalars &sc, int32_t *status, cudaStream_t stream)
 {
     if (num_tiles <= 0) return cudaSuccess;
-    if (bn != 128) return cudaErrorInvalidValue;
-    switch (epilogue) {
-    case EPI_STORE_F32:
-        return planes == 2 ? launch_one<128, EPI_STORE_F32, 2>(probs, tiles, num_tiles, sc, status, stream)
-                           : launch_one<128, EPI_STORE_F32, 1>(probs, tiles, num_tiles, sc, status, stream);
-    case EPI_STORE_BF16: return launch_one<128, EPI_STORE_BF16, 1>(probs, tiles, num_tiles, sc, status, stream);
-    case EPI_STORE_BF16_T: return launch_one<128, EPI_STORE_BF16_T, 1>(probs, tiles, num_tiles, sc, status, stream);
-    case EPI_CORE_UPDATE: return launch_one<128, EPI_CORE_UPDATE, 1>(probs, tiles, num_tiles, sc, status, stream);
-    case EPI_APPLY: return launch_one<128, EPI_APPLY, 1>(probs, tiles, num_tiles, sc, status, stream);
-    default: return cudaErrorInvalidValue;
+#define TSR_UG(BN_, EPI_, PL_) return launch_one<BN_, EPI_, PL_>(probs, tiles, num_tiles, num_sms, sc, status, stream)
+    if (planes == 2) {
+        if (bn == 128 && epilogue == EPI_STORE_F32) TSR_UG(128, EPI_STORE_F32, 2);
+        return cudaErrorInvalidValue;
     }
+    if (bn == 128) {
+        switch (epilogue) {
+        case EPI_STORE_F32: TSR_UG(128, EPI_STORE_F32, 1);
+        case EPI_STORE_BF16: TSR_UG(128, EPI_STORE_BF16, 1);
+        case EPI_STORE_BF16_T: TSR_UG(128, EPI_STORE_BF16_T, 1);
+        case EPI_CORE_UPDATE: TSR_UG(128, EPI_CORE_UPDATE, 1);
+        default: return cudaErrorInvalidValue;
+        }
+    }
+    if (bn == 256) {
+        switch (epilogue) {
+        case EPI_STORE_F32: TSR_UG(256, EPI_STORE_F32, 1);
+        case EPI_STORE_BF16: TSR_UG(256, EPI_STORE_BF16, 1);
+        case EPI_STORE_BF16_T: TSR_UG(256, EPI_STORE_BF16_T, 1);
+        case EPI_CORE_UPDATE: TSR_UG(256, EPI_CORE_UPDATE, 1);
+        default: return cudaErrorInvalidValue;
+        }
+    }
+#undef TSR_UG
+    return cudaErrorInvalidValue;
 }
 
 }  // namespace tsr
