@@ -38,7 +38,7 @@ def _run_steps(tsr, plan, shapes, dtype, steps, fuse, tol, wd=0.0, scale=1.0, ru
             plan.backproject_apply(h)
         torch.cuda.synchronize()
         for i, ob in enumerate(blks):
-            ob.step(G64[i], lr=1e-3, weight_decay=wd, scale=scale)
+            ob.step(G64[i], lr=1e-3, weight_decay=wd, scale=scale)   # the SGD rule ignores wd / scale
             worst["C"] = max(worst["C"], rel_fro(to64(plan.C[i]), ob.C))
             worst["M"] = max(worst["M"], rel_fro(to64(plan.M[i]), ob.M))
             if rule == 0:
@@ -83,10 +83,30 @@ def test_bf16_path_steps_match_oracle(fuse):
     _run_steps(tsr, plan, BF16_SHAPES, torch.bfloat16, 10, fuse, TOL_BF16)
 
 
-def test_bf16_path_decay_scale_and_sgd_rule():
+def test_bf16_path_decay_and_scale():
     tsr, plan = _plan(BF16_SHAPES[:2], torch.bfloat16)
     _given_bases(plan, BF16_SHAPES[:2])
     _run_steps(tsr, plan, BF16_SHAPES[:2], torch.bfloat16, 4, True, TOL_BF16, wd=0.1, scale=0.25)
+
+
+# ranks >= 256 switch the grouped GEMMs to 256-wide tiles (two accumulators of 256 columns)
+WIDE_SHAPES = [dict(m=640, n=768, r=256), dict(m=1100, n=1024, r=512), dict(m=600, n=520, r=264)]
+
+
+@pytest.mark.parametrize("fuse", [False, True])
+def test_bf16_path_wide_tiles_match_oracle(fuse):
+    tsr, plan = _plan(WIDE_SHAPES, torch.bfloat16)
+    _given_bases(plan, WIDE_SHAPES)
+    _run_steps(tsr, plan, WIDE_SHAPES, torch.bfloat16, 3, fuse, TOL_BF16)
+
+
+@pytest.mark.parametrize("dtype,shapes,tol", [(torch.float32, F32_SHAPES[1:], TOL_F32),
+                                              (torch.bfloat16, BF16_SHAPES[:2], TOL_BF16)])
+def test_sgd_rule_matches_algorithm_2(dtype, shapes, tol):
+    tsr, plan = _plan(shapes, dtype)
+    _given_bases(plan, shapes)
+    _run_steps(tsr, plan, shapes, dtype, 5, True, tol, rule=1)
+    _run_steps(tsr, plan, shapes, dtype, 3, False, tol, rule=1)
 
 
 def test_fused_and_unfused_orders_agree_bitwise():
