@@ -233,6 +233,34 @@ TSR_API tsr_status tsr_get_stage_ms(tsr_ctx *ctx, float *ms, int32_t count);
 /* Number of CUDA kernels this context has launched since tsr_create. */
 TSR_API tsr_status tsr_launch_count(const tsr_ctx *ctx, uint64_t *count);
 
+/* Core projection C = U^T G V of ONE block without any allocation.  (The paper has no
+ * counterpart of this call; it exists for callers that cannot allocate device memory.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside a host callback or a
+ * region that must not synchronise the device, in a process whose memory is owned by another
+ * framework's pool with nothing left to hand out, or under an allocator that forbids foreign
+ * allocations -- and that cannot provide the scratch buffer tsr_bind asks for either.  Here the
+ * only scratch the computation needs, the m x r intermediate T = G V, sits in a fixed
+ * TSR_STATIC_SCRATCH_FLOATS-element FP32 array inside the library image (4 MiB of device
+ * memory per GPU that loads the library, held until the process exits).
+ *
+ * All pointers are DEVICE pointers: G is m x n (leading dimension ldg, g_dtype TSR_F32 or
+ * TSR_BF16), U is m x r, V is n x r, C is r x r (output), all row-major, U / V / C FP32 dense.
+ * The call takes no context, calls no cudaMalloc / cudaFree or any allocating routine, and runs
+ * on the CUDA-core FP32 path (same kernels and therefore the same bits as tsr_project_core on
+ * that path).  Limits and errors: m * r must not exceed TSR_STATIC_SCRATCH_FLOATS, otherwise
+ * TSR_ERR_WORKSPACE is returned and nothing is launched; bad pointers / shapes / dtypes give
+ * TSR_ERR_INVALID_ARG / TSR_ERR_SHAPE / TSR_ERR_UNSUPPORTED.
+ * The first call on each device looks up the array's device address (cudaGetSymbolAddress,
+ * with that device current); make that first call outside any stream capture.
+ * Every call on a device shares the one array and finds the previous call's contents in it;
+ * nothing needs clearing because T is fully overwritten before it is read.  Two calls whose
+ * kernels may overlap on the GPU (different streams, or different host threads without
+ * ordering) race on the array: serialise them on one stream. */
+#define TSR_STATIC_SCRATCH_FLOATS (1 << 20)
+TSR_API tsr_status tsr_project_core_static(const void *G, int32_t g_dtype, int64_t m, int64_t n, int64_t ldg,
+                                           const float *U, const float *V, int32_t r, float *C, void *stream);
+
 /* 1 if block i takes the tensor-core path, 0 if the FP32 CUDA-core path, < 0 on a bad index. */
 TSR_API int32_t tsr_block_uses_tensor_cores(const tsr_ctx *ctx, int32_t i);
 

@@ -53,7 +53,7 @@ EXPORTS = [
     "tsr_project_core_grouped", "tsr_adam_core_step_grouped", "tsr_backproject_apply_grouped",
     "tsr_rsvd_refresh_grouped", "tsr_embed_step_grouped", "tsr_step_grouped", "tsr_step_grouped_host",
     "tsr_comm_bytes", "tsr_state_elems", "tsr_poll_status", "tsr_generate_omega", "tsr_block_uses_tensor_cores",
-    "tsr_set_profiling", "tsr_get_stage_ms", "tsr_launch_count",
+    "tsr_set_profiling", "tsr_get_stage_ms", "tsr_launch_count", "tsr_project_core_static",
 ]
 
 
@@ -110,6 +110,7 @@ def lib():
         L.tsr_set_profiling.argtypes = [vp, i32]
         L.tsr_get_stage_ms.argtypes = [vp, P(ctypes.c_float), i32]
         L.tsr_launch_count.argtypes = [vp, P(u64)]
+        L.tsr_project_core_static.argtypes = [vp, i32, i64, i64, i64, vp, vp, i32, vp, vp]
         _lib = L
     return _lib
 
@@ -136,6 +137,23 @@ def _stream_ptr(stream) -> Optional[int]:
     if stream is None:
         stream = torch.cuda.current_stream()
     return ctypes.c_void_p(stream.cuda_stream)
+
+
+STATIC_SCRATCH_FLOATS = 1 << 20
+
+
+def project_core_static(G: torch.Tensor, U: torch.Tensor, V: torch.Tensor, C: torch.Tensor, stream=None) -> None:
+    """C = U^T G V through tsr_project_core_static: no context, no workspace, no allocation --
+    for callers that are not allowed to allocate device memory.  G is a 2-D (possibly row-padded)
+    FP32 or BF16 tensor, U (m x r), V (n x r) and C (r x r) dense FP32, all on the current device."""
+    m, n = G.shape
+    r = U.shape[1]
+    dt = TSR_BF16 if G.dtype == torch.bfloat16 else TSR_F32
+    rc = lib().tsr_project_core_static(ctypes.c_void_p(G.data_ptr()), dt, m, n, G.stride(0),
+                                       ctypes.c_void_p(U.data_ptr()), ctypes.c_void_p(V.data_ptr()), r,
+                                       ctypes.c_void_p(C.data_ptr()), _stream_ptr(stream))
+    if rc != TSR_OK:
+        raise TsrError(rc, "tsr_project_core_static")
 
 
 class Plan:
