@@ -36,6 +36,11 @@ struct Block {
     float *buf[3] = {nullptr, nullptr, nullptr};
     double *S = nullptr, *Xw = nullptr, *Wj = nullptr, *gpart = nullptr, *lam = nullptr;
     float *Rinv = nullptr, *Wu = nullptr, *Wv = nullptr;
+    double *tau = nullptr, *dvec = nullptr, *evec = nullptr;
+    double2 *rot = nullptr;
+    int2 *sweeps = nullptr;
+    int32_t *nsweeps = nullptr, *rank = nullptr;
+    int rot_cap = 0, sweep_cap = 0;
     int tile_begin[NKIND], tile_end[NKIND];
 };
 
@@ -73,8 +78,8 @@ struct tsr_ctx {
     int32_t *d_status = nullptr;
     int32_t *d_list = nullptr;                 // scratch: block list of the running call
     int32_t *d_list2 = nullptr;                // scratch: second list (split-K blocks, ...)
-    RowItem *d_items[4] = {};                  // [side*2 + 0]: 64-row slabs, [side*2 + 1]: Gram slabs
-    size_t items_cap[4] = {};
+    RowItem *d_items[5] = {};                  // [side*2 + 0]: 64-row slabs, [side*2 + 1]: Gram slabs, [4]: eigenvector panels
+    size_t items_cap[5] = {};
     EncodeTiledFn encode = nullptr;
     int max_r = 0, max_k = 0;
     uint64_t launches = 0;                     // kernels launched through this context
@@ -140,14 +145,15 @@ void layout(tsr_ctx *ctx, Arena &a, bool assign, size_t *step_end)
         ctx->d_refresh = (RefreshDev *)p3; ctx->d_status = (int32_t *)p4;
         ctx->d_list = (int32_t *)p5; ctx->d_list2 = (int32_t *)p6;
     }
-    size_t cap[4] = {0, 0, 0, 0};
+    size_t cap[5] = {0, 0, 0, 0, 0};
     for (const Block &b : ctx->blocks) {
         cap[0] += (size_t)((b.d.m + RG_ROWS - 1) / RG_ROWS);
         cap[1] += (size_t)gram_chunks(b.d.m);
         cap[2] += (size_t)((b.d.n + RG_ROWS - 1) / RG_ROWS);
         cap[3] += (size_t)gram_chunks(b.d.n);
+        cap[4] += (size_t)((b.k + 7) / 8);
     }
-    for (int i = 0; i < 4; ++i) {
+    for (int i = 0; i < 5; ++i) {
         void *q = a.take(sizeof(RowItem) * cap[i]);
         if (assign) { ctx->d_items[i] = (RowItem *)q; ctx->items_cap[i] = cap[i]; }
     }
@@ -189,7 +195,14 @@ void layout(tsr_ctx *ctx, Arena &a, bool assign, size_t *step_end)
         void *gp = a.take((size_t)gram_chunks(mx) * k * k * 8);
         void *lam = a.take((size_t)k * 8);
         void *ri = a.take((size_t)(k * k) * 4), *wu = a.take((size_t)(k * r) * 4), *wv = a.take((size_t)(k * r) * 4);
+        const int rot_cap = (int)std::min<int64_t>(3 * k * k + 64, 0x7fffffff), sweep_cap = (int)(64 * k);
+        void *tau = a.take((size_t)k * 8), *dv = a.take((size_t)k * 8), *ev = a.take((size_t)k * 8);
+        void *rot = a.take((size_t)rot_cap * 16), *sw = a.take((size_t)sweep_cap * 8);
+        void *nsw = a.take(4), *rk = a.take((size_t)k * 4);
         if (assign) {
+            b.tau = (double *)tau; b.dvec = (double *)dv; b.evec = (double *)ev; b.rot = (double2 *)rot;
+            b.sweeps = (int2 *)sw; b.nsweeps = (int32_t *)nsw; b.rank = (int32_t *)rk;
+            b.rot_cap = rot_cap; b.sweep_cap = sweep_cap;
             b.Om = (float *)om; b.buf[0] = (float *)b0; b.buf[1] = (float *)b1; b.buf[2] = (float *)b2;
             b.S = (double *)S; b.Xw = (double *)Xw; b.Wj = (double *)Wj; b.gpart = (double *)gp; b.lam = (double *)lam;
             b.Rinv = (float *)ri; b.Wu = (float *)wu; b.Wv = (float *)wv;
@@ -458,7 +471,7 @@ tsr_status orth_pass(tsr_ctx *ctx, const RefreshLists &L, int side, int src, int
     const int nl = (int)L.list.size();
     TSR_KERNEL(ctx, 2, gram_batched(ctx->d_refresh, ctx->d_items[side * 2 + 1], L.nitems[side * 2 + 1], ctx->d_list, nl, side,
                                src, L.kmax, st));
-    TSR_KERNEL(ctx, 1, chol_inverse_batched(ctx->d_refresh, ctx->d_list, nl, st));
+    TSR_KERNEL(ctx, 1, chol_inverse_batched(ctx->d_refresh, ctx->d_list, nl, L.kmax, st));
     TSR_KERNEL(ctx, 1, rows_gemm_batched(ctx->d_refresh, ctx->d_items[side * 2], L.nitems[side * 2], side, src, 0, dst, L.kmax, st));
     return TSR_OK;
 }
@@ -549,7 +562,16 @@ tsr_status do_refresh(tsr_ctx *ctx, const std::vector<int> &list, uint64_t seed,
     if ((s = sketch(ctx, L, true, false, nullptr, st)) != TSR_OK) return s;
     const int nl = (int)list.size();
     TSR_KERNEL(ctx, 2, gram_batched(ctx->d_refresh, ctx->d_items[3], L.nitems[3], ctx->d_list, nl, 1, 0, L.kmax, st));
-    TSR_KERNEL(ctx, 1, jacobi_batched(ctx->d_refresh, ctx->d_list, nl, 40, st));
+    if (L.kmax >= 200) {   // too large for the Jacobi solver: tridiagonal route
+        const int pr = eig_panel_rows(L.kmax);
+        std::vector<RowItem> panels;
+        for (int bi : list)
+            for (int r0 = 0; r0 < ctx->blocks[bi].k; r0 += pr) panels.push_back({bi, r0});
+        TSR_CUDA(ctx, cudaMemcpyAsync(ctx->d_items[4], panels.data(), panels.size() * sizeof(RowItem), cudaMemcpyHostToDevice, st));
+        TSR_KERNEL(ctx, 4, eig_tridiag_batched(ctx->d_refresh, ctx->d_list, nl, ctx->d_items[4], (int)panels.size(), L.kmax, st));
+    } else {
+        TSR_KERNEL(ctx, 1, jacobi_batched(ctx->d_refresh, ctx->d_list, nl, 40, st));
+    }
     // V = B^T Wt / sigma ; U = Q Wt
     TSR_KERNEL(ctx, 1, rows_gemm_batched(ctx->d_refresh, ctx->d_items[2], L.nitems[2], 1, 0, 2, 4, L.rmax, st));
     TSR_KERNEL(ctx, 1, rows_gemm_batched(ctx->d_refresh, ctx->d_items[0], L.nitems[0], 0, 2, 1, 3, L.rmax, st));
@@ -774,6 +796,8 @@ tsr_status tsr_bind(tsr_ctx *ctx, const tsr_mat_ptrs *ptrs, int32_t count, void 
         for (int j = 0; j < 3; ++j) rd.buf[j] = b.buf[j];
         rd.S = b.S; rd.Xw = b.Xw; rd.Wj = b.Wj; rd.gpart = b.gpart; rd.lam = b.lam;
         rd.Rinv = b.Rinv; rd.Wu = b.Wu; rd.Wv = b.Wv; rd.U = b.p.U; rd.V = b.p.V; rd.status = ctx->d_status + i;
+        rd.tau = b.tau; rd.dvec = b.dvec; rd.evec = b.evec; rd.rot = b.rot; rd.sweeps = b.sweeps; rd.nsweeps = b.nsweeps;
+        rd.rank = b.rank; rd.rot_cap = b.rot_cap; rd.sweep_cap = b.sweep_cap;
         if (!b.fast) continue;
         auto base = [&](UmmaProblem &P, int M, int N, int K, int epi) {
             P.M = M; P.N = N; P.K = K; P.planes = 1; P.plane_rows = 0; P.block = i; P.epilogue = epi;

@@ -1,0 +1,278 @@
+// Symmetric eigen-decomposition of the k x k Gram matrix S = B B^T of the refresh (Section 3.5:
+// "compute a small SVD") for ranks too large for a shared-memory Jacobi solver.
+//
+// Classical three-stage scheme, batched over blocks, FP64 throughout:
+//   1. Householder reduction to tridiagonal form T = Q^T S Q (one CTA per matrix; the
+//      reflectors are kept in the rows of S above the first superdiagonal);
+//   2. implicit-shift QL iteration on (d, e) alone, one thread per matrix, which LOGS every
+//      plane rotation instead of applying it;
+//   3. the eigenvectors W = Q Z: every warp takes a panel of rows of the identity into shared
+//      memory (lane = row), runs them through the reflectors (giving rows of Q) and then through
+//      the logged rotations, and writes the leading r columns in descending eigenvalue order:
+//      Wu = W[:, :r] and Wv = W[:, :r] / sqrt(lambda).
+// Rows are independent under right-multiplication, so stage 3 needs no synchronisation and
+// the rotations never touch global memory.
+// Failure to converge within the iteration or log budget flags TSR_ERR_NOT_CONVERGED.
+#include "tsr_internal.h"
+
+namespace tsr {
+
+constexpr int TR_THREADS = 1024;
+
+// ---- stage 1: tridiagonalisation -----------------------------------------------------------
+__global__ void __launch_bounds__(TR_THREADS)
+tridiag_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ list, int kpad)
+{
+    extern __shared__ double tr_smem[];          // v, p, w : 3 x kpad
+    double *vs = tr_smem, *ps = tr_smem + kpad, *ws = tr_smem + 2 * kpad;
+    __shared__ double red[32];
+    __shared__ double s_scalar[4];
+    const RefreshDev d = rd[list[blockIdx.x]];
+    const int k = d.k;
+    double *__restrict__ A = d.S;
+    const int tid = threadIdx.x, nt = blockDim.x, warp = tid >> 5, lane = tid & 31, nwarps = nt >> 5;
+
+    auto block_sum = [&](double x) -> double {
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) x += __shfl_xor_sync(0xffffffffu, x, off);
+        __syncthreads();
+        if (lane == 0) red[warp] = x;
+        __syncthreads();
+        double t = (lane < nwarps) ? red[lane] : 0.0;
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) t += __shfl_xor_sync(0xffffffffu, t, off);
+        return t;   // every thread of every warp holds the total
+    };
+
+    for (int j = 0; j + 2 < k; ++j) {
+        const int len = k - j - 1;               // x = A[j][j+1 .. k-1]
+        double *xrow = A + (int64_t)j * k + j + 1;
+        double part = 0.0;
+        for (int i = tid; i < len; i += nt) { const double x = xrow[i]; vs[i] = x; part += x * x; }
+        const double nrm2 = block_sum(part);
+        const double x0 = vs[0];
+        const double nrm = sqrt(nrm2);
+        const double tail2 = nrm2 - x0 * x0;
+        if (!(tail2 > 0.0) || nrm == 0.0) {      // nothing to annihilate: H_j = I
+            if (tid == 0) { d.tau[j] = 0.0; d.dvec[j] = A[(int64_t)j * k + j]; d.evec[j] = x0; }
+            __syncthreads();
+            continue;
+        }
+        const double alpha = (x0 >= 0.0) ? -nrm : nrm;
+        const double v0 = x0 - alpha;
+        const double tau = -v0 / alpha;
+        __syncthreads();
+        for (int i = tid; i < len; i += nt) {
+            const double v = (i == 0) ? 1.0 : vs[i] / v0;
+            vs[i] = v;
+            if (i > 0) xrow[i] = v;              // keep the reflector for stage 3
+        }
+        if (tid == 0) { d.tau[j] = tau; d.dvec[j] = A[(int64_t)j * k + j]; d.evec[j] = alpha; }
+        __syncthreads();
+        // p = tau * A22 v      (A22 = A[j+1.., j+1..], row-wise dot products, one warp per row)
+        for (int a = warp; a < len; a += nwarps) {
+            const double *row = A + (int64_t)(j + 1 + a) * k + j + 1;
+            double acc = 0.0;
+            for (int b = lane; b < len; b += 32) acc += row[b] * vs[b];
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+            if (lane == 0) ps[a] = tau * acc;
+        }
+        __syncthreads();
+        part = 0.0;
+        for (int i = tid; i < len; i += nt) part += ps[i] * vs[i];
+        const double pv = block_sum(part);
+        const double kk = 0.5 * tau * pv;
+        for (int i = tid; i < len; i += nt) ws[i] = ps[i] - kk * vs[i];
+        __syncthreads();
+        // A22 -= v w^T + w v^T
+        for (int a = warp; a < len; a += nwarps) {
+            double *row = A + (int64_t)(j + 1 + a) * k + j + 1;
+            const double va = vs[a], wa = ws[a];
+            for (int b = lane; b < len; b += 32) row[b] -= va * ws[b] + wa * vs[b];
+        }
+        __syncthreads();
+    }
+    if (tid == 0) {
+        if (k >= 2) {
+            d.dvec[k - 2] = A[(int64_t)(k - 2) * k + (k - 2)];
+            d.evec[k - 2] = A[(int64_t)(k - 2) * k + (k - 1)];
+            d.tau[k - 2] = 0.0;
+        }
+        d.dvec[k - 1] = A[(int64_t)(k - 1) * k + (k - 1)];
+        d.evec[k - 1] = 0.0;
+        d.tau[k - 1] = 0.0;
+    }
+}
+
+// ---- stage 2: implicit QL on the tridiagonal matrix, logging the rotations ------------------
+// e[i] couples d[i] and d[i+1].  Sweep header: x = index of the first rotation (m - 1), y = count;
+// rotation t of a sweep acts on columns (x - t, x - t + 1).
+__global__ void ql_log_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ list)
+{
+    if (threadIdx.x != 0) return;
+    const RefreshDev D = rd[list[blockIdx.x]];
+    const int n = D.k;
+    double *__restrict__ d = D.dvec;
+    double *__restrict__ e = D.evec;
+    double2 *__restrict__ rot = D.rot;
+    int2 *__restrict__ sweeps = D.sweeps;
+    int nrot = 0, nsw = 0;
+    bool failed = false;
+    for (int l = 0; l < n && !failed; ++l) {
+        int iter = 0;
+        while (true) {
+            int m = l;
+            for (; m < n - 1; ++m) {
+                const double dd = fabs(d[m]) + fabs(d[m + 1]);
+                if (fabs(e[m]) <= 2.3e-16 * dd) break;
+            }
+            if (m == l) break;
+            if (++iter > 60 || nsw >= D.sweep_cap || nrot + (m - l) > D.rot_cap) { failed = true; break; }
+            double g = (d[l + 1] - d[l]) / (2.0 * e[l]);
+            double r = hypot(g, 1.0);
+            g = d[m] - d[l] + e[l] / (g + (g >= 0.0 ? fabs(r) : -fabs(r)));
+            double s = 1.0, c = 1.0, p = 0.0;
+            const int first = nrot;
+            int i = m - 1;
+            bool early = false;
+            for (; i >= l; --i) {
+                const double f = s * e[i], b = c * e[i];
+                r = hypot(f, g);
+                e[i + 1] = r;
+                if (r == 0.0) { d[i + 1] -= p; e[m] = 0.0; early = true; break; }
+                s = f / r;
+                c = g / r;
+                g = d[i + 1] - p;
+                r = (d[i] - g) * s + 2.0 * c * b;
+                p = s * r;
+                d[i + 1] = g + p;
+                g = c * r - b;
+                rot[nrot++] = make_double2(c, s);
+            }
+            if (nrot > first) sweeps[nsw++] = make_int2(m - 1, nrot - first);
+            if (early) continue;
+            d[l] -= p;
+            e[l] = g;
+            e[m] = 0.0;
+        }
+    }
+    *D.nsweeps = nsw;
+    if (failed) atomicMax(D.status, (int)TSR_ERR_NOT_CONVERGED);
+}
+
+// ---- stage 3: rows of W = Q Z in shared memory, then select and scale -----------------------
+__global__ void __launch_bounds__(32)
+eigvec_panel_kernel(const RefreshDev *__restrict__ rd, const RowItem *__restrict__ items, int pr)
+{
+    extern __shared__ double z[];                 // z[col * pr + lane]
+    const RowItem it = items[blockIdx.x];
+    const RefreshDev D = rd[it.block];
+    const int k = D.k, r = D.r;
+    const int lane = threadIdx.x;
+    const int row = it.row0 + lane;
+    const bool active = lane < pr && row < k;
+    if (lane < pr)
+        for (int c = 0; c < k; ++c) z[c * pr + lane] = (c == row) ? 1.0 : 0.0;
+    __syncwarp();
+    if (active) {
+        // x <- x H_0 H_1 ... : x[j+1:] -= tau_j (x[j+1:] . v_j) v_j,  v_j = (1, S[j][j+2:])
+        const double *__restrict__ A = D.S;
+        for (int j = 0; j + 2 < k; ++j) {
+            const double tau = D.tau[j];
+            if (tau == 0.0) continue;
+            const double *v = A + (int64_t)j * k;   // v[c] for c >= j+2
+            double dot = z[(j + 1) * pr + lane];
+            for (int c = j + 2; c < k; ++c) dot += z[c * pr + lane] * v[c];
+            dot *= tau;
+            z[(j + 1) * pr + lane] -= dot;
+            for (int c = j + 2; c < k; ++c) z[c * pr + lane] -= dot * v[c];
+        }
+        // logged rotations
+        const int nsw = *D.nsweeps;
+        const double2 *__restrict__ rot = D.rot;
+        const int2 *__restrict__ sweeps = D.sweeps;
+        int off = 0;
+        for (int sidx = 0; sidx < nsw; ++sidx) {
+            const int2 sw = sweeps[sidx];
+            int i = sw.x;
+            double f = z[(i + 1) * pr + lane];
+            for (int t = 0; t < sw.y; ++t, --i) {
+                const double2 cs = rot[off + t];
+                const double zi = z[i * pr + lane];
+                z[(i + 1) * pr + lane] = cs.y * zi + cs.x * f;
+                f = cs.x * zi - cs.y * f;
+            }
+            z[(i + 1) * pr + lane] = f;
+            off += sw.y;
+        }
+        // rank the eigenvalues (descending, ties by index) and emit the leading r columns
+        const double *__restrict__ lam = D.dvec;
+        for (int j = 0; j < k; ++j) {
+            const int rank = D.rank[j];
+            if (rank < r) {
+                const double lj = lam[j];
+                const double inv = (lj > 1e-300) ? 1.0 / sqrt(lj) : 0.0;
+                const double w = z[j * pr + lane];
+                D.Wu[(int64_t)row * r + rank] = (float)w;
+                D.Wv[(int64_t)row * r + rank] = (float)(w * inv);
+            }
+        }
+    }
+}
+
+__global__ void eig_rank_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ list)
+{
+    const RefreshDev D = rd[list[blockIdx.x]];
+    const int k = D.k, r = D.r;
+    int flag = 0;
+    for (int j = threadIdx.x; j < k; j += blockDim.x) {
+        const double lj = D.dvec[j];
+        if (!(lj == lj)) flag = TSR_ERR_NONFINITE;
+        int rank = 0;
+        for (int l = 0; l < k; ++l) {
+            const double ll = D.dvec[l];
+            rank += (ll > lj || (ll == lj && l < j)) ? 1 : 0;
+        }
+        D.rank[j] = rank;
+        D.lam[rank] = lj;
+        if (rank < r && !(lj > 1e-300) && flag == 0) flag = TSR_ERR_RANK_DEFICIENT;
+    }
+    if (flag) atomicMax(D.status, flag);
+}
+
+int eig_panel_rows(int kmax)
+{
+    int pr = (110 * 1024) / (8 * kmax);
+    if (pr > 32) pr = 32;
+    pr &= ~7;
+    if (pr < 8) pr = 8;
+    return pr;
+}
+
+cudaError_t eig_tridiag_batched(const RefreshDev *rd, const int32_t *list, int nlist, const RowItem *panel_items,
+                                int npanels, int kmax, cudaStream_t stream)
+{
+    if (nlist <= 0) return cudaSuccess;
+    const int kpad = kmax + 8;
+    const size_t tr_bytes = (size_t)3 * kpad * sizeof(double);
+    const int pr = eig_panel_rows(kmax);
+    const size_t pn_bytes = (size_t)pr * kmax * sizeof(double);
+    static size_t tr_cfg = 0, pn_cfg = 0;
+    cudaError_t e;
+    if (tr_bytes > tr_cfg) {
+        if ((e = cudaFuncSetAttribute(tridiag_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tr_bytes)) != cudaSuccess) return e;
+        tr_cfg = tr_bytes;
+    }
+    if (pn_bytes > pn_cfg) {
+        if ((e = cudaFuncSetAttribute(eigvec_panel_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pn_bytes)) != cudaSuccess) return e;
+        pn_cfg = pn_bytes;
+    }
+    tridiag_kernel<<<nlist, TR_THREADS, tr_bytes, stream>>>(rd, list, kpad);
+    ql_log_kernel<<<nlist, 32, 0, stream>>>(rd, list);
+    eig_rank_kernel<<<nlist, 256, 0, stream>>>(rd, list);
+    eigvec_panel_kernel<<<npanels, 32, pn_bytes, stream>>>(rd, panel_items, pr);
+    return cudaGetLastError();
+}
+
+}  // namespace tsr

@@ -127,6 +127,13 @@ struct RefreshDev {
     float *Wu, *Wv;     // k x r
     float *U, *V;       // the block's bases (FP32 masters)
     int32_t *status;    // the block's status word
+    // tridiagonal eigen-solver (tsr_eig.cu)
+    double *tau, *dvec, *evec;   // k each: reflector scales, diagonal / eigenvalues, off-diagonal
+    double2 *rot;                // logged plane rotations (c, s)
+    int2 *sweeps;                // per QL sweep: first rotation index, count
+    int32_t *nsweeps;            // number of logged sweeps
+    int32_t *rank;               // k: descending rank of each eigenvalue
+    int32_t rot_cap, sweep_cap;
 };
 struct RowItem { int32_t block; int32_t row0; };   // a slab of rows of one block
 
@@ -139,12 +146,18 @@ __host__ __device__ inline int gram_chunks(int64_t rows) { return (int)((rows + 
 cudaError_t gram_batched(const RefreshDev *rd, const RowItem *items, int nitems, const int32_t *list, int nlist,
                          int side, int src_sel, int kmax, cudaStream_t stream);
 // Cholesky S = R^T R in place and Rinv = float(R^{-1}).
-cudaError_t chol_inverse_batched(const RefreshDev *rd, const int32_t *list, int nlist, cudaStream_t stream);
+cudaError_t chol_inverse_batched(const RefreshDev *rd, const int32_t *list, int nlist, int kmax, cudaStream_t stream);
 // dst = buf[src_sel] * Mat;  mat_sel: 0 Rinv (k x k), 1 Wu (k x r), 2 Wv (k x r);
 // dst_sel: 0..2 buf[], 3 = U, 4 = V.
 cudaError_t rows_gemm_batched(const RefreshDev *rd, const RowItem *items, int nitems, int side, int src_sel,
                               int mat_sel, int dst_sel, int nmax, cudaStream_t stream);
 // Eigen-decomposition of S by cyclic Jacobi, descending sort, Wu = W[:, :r], Wv = W[:, :r] / sqrt(lambda).
+// The same result through Householder tridiagonalisation + implicit QL with logged rotations
+// (for k too large for the Jacobi solver).  panel_items: (block, row0) slabs of eig_panel_rows(kmax)
+// rows of the k x k eigenvector matrix.
+int eig_panel_rows(int kmax);
+cudaError_t eig_tridiag_batched(const RefreshDev *rd, const int32_t *list, int nlist, const RowItem *panel_items,
+                                int npanels, int kmax, cudaStream_t stream);
 cudaError_t jacobi_batched(const RefreshDev *rd, const int32_t *list, int nlist, int max_sweeps, cudaStream_t stream);
 
 }  // namespace tsr

@@ -90,20 +90,28 @@ cudaError_t gram_batched(const RefreshDev *rd, const RowItem *items, int nitems,
 
 // ---------------------------------------------------------------------------------------
 // Cholesky S = R^T R with R upper triangular (one CTA per matrix, FP64, in place), followed by
-// Rinv = R^{-1} written as FP32.  A pivot that is not safely positive is replaced by a floor
-// relative to the largest diagonal entry and the block is flagged TSR_ERR_RANK_DEFICIENT.
+// Rinv = R^{-1} written as FP32.  Blocked: 16 rows of R at a time are factored in shared memory,
+// then the trailing upper triangle gets one rank-16 update, so the matrix in global memory is
+// read and written once per panel instead of once per row.  The inverse is computed 16 columns
+// at a time by back substitution, one warp per column with the column held in shared memory.
+// A pivot that is not safely positive is replaced by a floor relative to the largest diagonal
+// entry and the block is flagged TSR_ERR_RANK_DEFICIENT.
 // ---------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(1024)
-chol_inverse_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ list)
+constexpr int CH_NB = 16;
+constexpr int CH_THREADS = 1024;
+
+__global__ void __launch_bounds__(CH_THREADS)
+chol_inverse_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ list, int kpad)
 {
+    extern __shared__ double ch_smem[];   // [CH_NB][kpad] panel of R rows, reused as 2 x [kpad][CH_NB] inverse panels
     const RefreshDev d = rd[list[blockIdx.x]];
     const int k = d.k;
     double *__restrict__ S = d.S;
-    double *__restrict__ X = d.Xw;
     __shared__ double s_piv;
     __shared__ double s_floor;
     __shared__ int s_flag;
     const int tid = threadIdx.x, nt = blockDim.x;
+    const int warp = tid >> 5, lane = tid & 31, nwarps = nt >> 5;
     if (tid == 0) {
         double mx = 0.0;
         int bad = 0;
@@ -117,45 +125,93 @@ chol_inverse_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict
         s_flag = bad ? TSR_ERR_NONFINITE : 0;
     }
     __syncthreads();
-    for (int j = 0; j < k; ++j) {
-        if (tid == 0) {
-            double v = S[(int64_t)j * k + j];
-            if (!(v > s_floor)) {
-                if (s_flag == 0) s_flag = TSR_ERR_RANK_DEFICIENT;
-                v = s_floor;
+    for (int jb = 0; jb < k; jb += CH_NB) {
+        const int nb = min(CH_NB, k - jb);
+        const int w = k - jb;                       // panel width: columns jb..k-1
+        double *P = ch_smem;                        // P[j][c] = S[jb + j][jb + c]
+        for (int e = tid; e < nb * w; e += nt) {
+            const int j = e / w, c = e % w;
+            P[j * kpad + c] = (c >= j) ? S[(int64_t)(jb + j) * k + jb + c] : 0.0;
+        }
+        __syncthreads();
+        for (int j = 0; j < nb; ++j) {
+            if (tid == 0) {
+                double v = P[j * kpad + j];
+                if (!(v > s_floor)) {
+                    if (s_flag == 0) s_flag = TSR_ERR_RANK_DEFICIENT;
+                    v = s_floor;
+                }
+                s_piv = sqrt(v);
             }
-            s_piv = sqrt(v);
+            __syncthreads();
+            const double piv = s_piv;
+            for (int c = j + tid; c < w; c += nt) P[j * kpad + c] = (c == j) ? piv : P[j * kpad + c] / piv;
+            __syncthreads();
+            // rows j+1..nb-1 of the panel: P[i][c] -= R[j][i] R[j][c], c >= i
+            const int rows_left = nb - j - 1;
+            for (int e = tid; e < rows_left * w; e += nt) {
+                const int i = j + 1 + e / w, c = e % w;
+                if (c >= i) P[i * kpad + c] -= P[j * kpad + i] * P[j * kpad + c];
+            }
+            __syncthreads();
         }
-        __syncthreads();
-        const double piv = s_piv;
-        for (int l = j + tid; l < k; l += nt) S[(int64_t)j * k + l] = (l == j) ? piv : S[(int64_t)j * k + l] / piv;
-        __syncthreads();
-        // trailing update of the upper triangle: S[i][l] -= R[j][i] R[j][l], j < i <= l
-        const int rem = k - j - 1;
-        for (int64_t e = tid; e < (int64_t)rem * rem; e += nt) {
-            const int i = j + 1 + (int)(e / rem), l = j + 1 + (int)(e % rem);
-            if (l >= i) S[(int64_t)i * k + l] -= S[(int64_t)j * k + i] * S[(int64_t)j * k + l];
+        // final rows of R go back to global memory
+        for (int e = tid; e < nb * w; e += nt) {
+            const int j = e / w, c = e % w;
+            if (c >= j) S[(int64_t)(jb + j) * k + jb + c] = P[j * kpad + c];
+        }
+        // rank-nb update of the trailing upper triangle
+        for (int i = jb + nb + warp; i < k; i += nwarps) {
+            const int ci = i - jb;
+            double ri[CH_NB];
+#pragma unroll
+            for (int j = 0; j < CH_NB; ++j) ri[j] = (j < nb) ? P[j * kpad + ci] : 0.0;
+            for (int l = i + lane; l < k; l += 32) {
+                const int cl = l - jb;
+                double acc = 0.0;
+#pragma unroll
+                for (int j = 0; j < CH_NB; ++j) acc += ri[j] * ((j < nb) ? P[j * kpad + cl] : 0.0);
+                S[(int64_t)i * k + l] -= acc;
+            }
         }
         __syncthreads();
     }
-    // X = R^{-1} (upper): column c by back substitution, one thread per column
-    for (int c = tid; c < k; c += nt) {
-        for (int i = c; i >= 0; --i) {
-            double s = (i == c) ? 1.0 : 0.0;
-            for (int l = i + 1; l <= c; ++l) s -= S[(int64_t)i * k + l] * X[(int64_t)l * k + c];
-            X[(int64_t)i * k + c] = s / S[(int64_t)i * k + i];
+    // X = R^{-1} (upper triangular).  Column c: X[i][c] = (delta_ic - sum_{l=i+1..c} R[i][l] X[l][c]) / R[i][i],
+    // i = c .. 0.  One warp per column; the column lives in shared memory ([row][column-in-panel]).
+    double *Xs = ch_smem;
+    const int cols_per_round = min(nwarps, 2 * CH_NB);          // 32 columns: 2 x CH_NB x kpad doubles
+    for (int c0 = 0; c0 < k; c0 += cols_per_round) {
+        const int c = c0 + warp;
+        if (warp < cols_per_round && c < k) {
+            double *xc = Xs + (int64_t)warp * kpad;              // this warp's column, contiguous
+            for (int i = c; i >= 0; --i) {
+                double part = 0.0;
+                const double *Ri = S + (int64_t)i * k;
+                for (int l = i + 1 + lane; l <= c; l += 32) part += Ri[l] * xc[l];
+#pragma unroll
+                for (int off = 16; off > 0; off >>= 1) part += __shfl_xor_sync(0xffffffffu, part, off);
+                if (lane == 0) xc[i] = (((i == c) ? 1.0 : 0.0) - part) / Ri[i];
+                __syncwarp();
+            }
+            for (int i = lane; i < k; i += 32) d.Rinv[(int64_t)i * k + c] = (i <= c) ? (float)xc[i] : 0.f;
         }
-        for (int i = c + 1; i < k; ++i) X[(int64_t)i * k + c] = 0.0;
+        __syncthreads();
     }
-    __syncthreads();
-    for (int64_t e = tid; e < (int64_t)k * k; e += nt) d.Rinv[e] = (float)X[e];
     if (tid == 0 && s_flag != 0) atomicMax(d.status, s_flag);
 }
 
-cudaError_t chol_inverse_batched(const RefreshDev *rd, const int32_t *list, int nlist, cudaStream_t stream)
+cudaError_t chol_inverse_batched(const RefreshDev *rd, const int32_t *list, int nlist, int kmax, cudaStream_t stream)
 {
     if (nlist <= 0) return cudaSuccess;
-    chol_inverse_kernel<<<nlist, 1024, 0, stream>>>(rd, list);
+    const int kpad = (kmax + 1) | 1;   // odd row pitch (in doubles) keeps shared-memory columns conflict-free
+    const size_t bytes = (size_t)2 * CH_NB * kpad * sizeof(double);
+    static size_t configured = 0;
+    if (bytes > configured) {
+        cudaError_t e = cudaFuncSetAttribute(chol_inverse_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+        if (e != cudaSuccess) return e;
+        configured = bytes;
+    }
+    chol_inverse_kernel<<<nlist, CH_THREADS, bytes, stream>>>(rd, list, kpad);
     return cudaGetLastError();
 }
 

@@ -149,6 +149,8 @@ def test_split_k_core_matches_oracle():
     (torch.bfloat16, dict(m=1376, n=512, r=128, p=8, q=1), 64),
     (torch.bfloat16, dict(m=200, n=328, r=40, p=8, q=2), 20),
     (torch.bfloat16, dict(m=2000, n=256, r=64, p=8, q=1), 32),
+    (torch.bfloat16, dict(m=600, n=704, r=256, p=8, q=1), 64),      # k = 264: tridiagonal eigen-solver
+    (torch.float32, dict(m=300, n=420, r=200, p=9, q=1), 48),       # k = 209 (odd), FP32 path
 ])
 def test_refresh_matches_oracle_at_gap(dtype, shape, gap):
     tsr, plan = _plan([shape], dtype)
