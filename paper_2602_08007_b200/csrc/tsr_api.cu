@@ -476,10 +476,15 @@ tsr_status orth_pass(tsr_ctx *ctx, const RefreshLists &L, int side, int src, int
     return TSR_OK;
 }
 
-// orth(buf[0]) -> buf[2] by Cholesky-QR applied twice (buf[1] holds the first pass).
-tsr_status orth(tsr_ctx *ctx, const RefreshLists &L, int side, cudaStream_t st)
+// orth(buf[0]) -> buf[2] by Cholesky-QR with the Gram matrix accumulated in FP64.
+// The basis that enters B = Q^T G and U = Q U~ (final = true) gets a second pass (buf[1] holds the
+// first one), which brings Q^T Q to the identity at FP32 rounding level.  The bases inside the
+// power iteration only have to span the right subspace and stay well conditioned: one pass
+// leaves Q^T Q = I + O(kappa(Y)^2 u) with exactly the same range, so a single pass is used there.
+tsr_status orth(tsr_ctx *ctx, const RefreshLists &L, int side, bool final, cudaStream_t st)
 {
     tsr_status s;
+    if (!final) return orth_pass(ctx, L, side, 0, 2, st);
     if ((s = orth_pass(ctx, L, side, 0, 1, st)) != TSR_OK) return s;
     return orth_pass(ctx, L, side, 1, 2, st);
 }
@@ -550,13 +555,13 @@ tsr_status do_refresh(tsr_ctx *ctx, const std::vector<int> &list, uint64_t seed,
     }
     // Y = G Omega; Q = orth(Y)
     if ((s = sketch(ctx, L, false, true, omegas, st)) != TSR_OK) return s;
-    if ((s = orth(ctx, L, 0, st)) != TSR_OK) return s;
+    if ((s = orth(ctx, L, 0, qmax == 0, st)) != TSR_OK) return s;
     for (int it = 0; it < qmax; ++it) {
         // Yrow = G^T Q; Qrow = orth(Yrow); Y = G Qrow; Q = orth(Y)
         if ((s = sketch(ctx, L, true, false, nullptr, st)) != TSR_OK) return s;
-        if ((s = orth(ctx, L, 1, st)) != TSR_OK) return s;
+        if ((s = orth(ctx, L, 1, false, st)) != TSR_OK) return s;
         if ((s = sketch(ctx, L, false, false, nullptr, st)) != TSR_OK) return s;
-        if ((s = orth(ctx, L, 0, st)) != TSR_OK) return s;
+        if ((s = orth(ctx, L, 0, it == qmax - 1, st)) != TSR_OK) return s;
     }
     // B^T = G^T Q (n x k) in buf[0]; small SVD through the k x k Gram matrix B B^T
     if ((s = sketch(ctx, L, true, false, nullptr, st)) != TSR_OK) return s;

@@ -108,57 +108,68 @@ tridiag_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ li
 // ---- stage 2: implicit QL on the tridiagonal matrix, logging the rotations ------------------
 // e[i] couples d[i] and d[i+1].  Sweep header: x = index of the first rotation (m - 1), y = count;
 // rotation t of a sweep acts on columns (x - t, x - t + 1).
-__global__ void ql_log_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ list)
+__global__ void __launch_bounds__(32)
+ql_log_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ list)
 {
-    if (threadIdx.x != 0) return;
+    extern __shared__ double ql_smem[];           // d[n], e[n]
     const RefreshDev D = rd[list[blockIdx.x]];
     const int n = D.k;
-    double *__restrict__ d = D.dvec;
-    double *__restrict__ e = D.evec;
-    double2 *__restrict__ rot = D.rot;
-    int2 *__restrict__ sweeps = D.sweeps;
-    int nrot = 0, nsw = 0;
-    bool failed = false;
-    for (int l = 0; l < n && !failed; ++l) {
-        int iter = 0;
-        while (true) {
-            int m = l;
-            for (; m < n - 1; ++m) {
-                const double dd = fabs(d[m]) + fabs(d[m + 1]);
-                if (fabs(e[m]) <= 2.3e-16 * dd) break;
+    double *d = ql_smem, *e = ql_smem + n;
+    for (int i = threadIdx.x; i < n; i += 32) { d[i] = D.dvec[i]; e[i] = D.evec[i]; }
+    __syncwarp();
+    if (threadIdx.x == 0) {
+        double2 *__restrict__ rot = D.rot;
+        int2 *__restrict__ sweeps = D.sweeps;
+        int nrot = 0, nsw = 0;
+        bool failed = false;
+        for (int l = 0; l < n && !failed; ++l) {
+            int iter = 0;
+            while (true) {
+                int m = l;
+                for (; m < n - 1; ++m) {
+                    const double dd = fabs(d[m]) + fabs(d[m + 1]);
+                    if (fabs(e[m]) <= 2.3e-16 * dd) break;
+                }
+                if (m == l) break;
+                if (++iter > 60 || nsw >= D.sweep_cap || nrot + (m - l) > D.rot_cap) { failed = true; break; }
+                double g = (d[l + 1] - d[l]) / (2.0 * e[l]);
+                double r = sqrt(g * g + 1.0);
+                g = d[m] - d[l] + e[l] / (g + (g >= 0.0 ? r : -r));
+                double s = 1.0, c = 1.0, p = 0.0;
+                const int first = nrot;
+                int i = m - 1;
+                bool early = false;
+                for (; i >= l; --i) {
+                    const double ei = e[i];
+                    const double f = s * ei, b = c * ei;
+                    // r = hypot(f, g).  The entries are bounded by the eigenvalues of a Gram matrix of FP32
+                    // data, so the squares stay far inside the FP64 range and no rescaling is needed.
+                    const double r2 = f * f + g * g;
+                    if (r2 == 0.0) { e[i + 1] = 0.0; d[i + 1] -= p; e[m] = 0.0; early = true; break; }
+                    const double rinv = rsqrt(r2);
+                    r = r2 * rinv;
+                    e[i + 1] = r;
+                    s = f * rinv;
+                    c = g * rinv;
+                    g = d[i + 1] - p;
+                    r = (d[i] - g) * s + 2.0 * c * b;
+                    p = s * r;
+                    d[i + 1] = g + p;
+                    g = c * r - b;
+                    rot[nrot++] = make_double2(c, s);
+                }
+                if (nrot > first) sweeps[nsw++] = make_int2(m - 1, nrot - first);
+                if (early) continue;
+                d[l] -= p;
+                e[l] = g;
+                e[m] = 0.0;
             }
-            if (m == l) break;
-            if (++iter > 60 || nsw >= D.sweep_cap || nrot + (m - l) > D.rot_cap) { failed = true; break; }
-            double g = (d[l + 1] - d[l]) / (2.0 * e[l]);
-            double r = hypot(g, 1.0);
-            g = d[m] - d[l] + e[l] / (g + (g >= 0.0 ? fabs(r) : -fabs(r)));
-            double s = 1.0, c = 1.0, p = 0.0;
-            const int first = nrot;
-            int i = m - 1;
-            bool early = false;
-            for (; i >= l; --i) {
-                const double f = s * e[i], b = c * e[i];
-                r = hypot(f, g);
-                e[i + 1] = r;
-                if (r == 0.0) { d[i + 1] -= p; e[m] = 0.0; early = true; break; }
-                s = f / r;
-                c = g / r;
-                g = d[i + 1] - p;
-                r = (d[i] - g) * s + 2.0 * c * b;
-                p = s * r;
-                d[i + 1] = g + p;
-                g = c * r - b;
-                rot[nrot++] = make_double2(c, s);
-            }
-            if (nrot > first) sweeps[nsw++] = make_int2(m - 1, nrot - first);
-            if (early) continue;
-            d[l] -= p;
-            e[l] = g;
-            e[m] = 0.0;
         }
+        *D.nsweeps = nsw;
+        if (failed) atomicMax(D.status, (int)TSR_ERR_NOT_CONVERGED);
     }
-    *D.nsweeps = nsw;
-    if (failed) atomicMax(D.status, (int)TSR_ERR_NOT_CONVERGED);
+    __syncwarp();
+    for (int i = threadIdx.x; i < n; i += 32) D.dvec[i] = d[i];
 }
 
 // ---- stage 3: rows of W = Q Z in shared memory, then select and scale -----------------------
@@ -175,20 +186,40 @@ eigvec_panel_kernel(const RefreshDev *__restrict__ rd, const RowItem *__restrict
     if (lane < pr)
         for (int c = 0; c < k; ++c) z[c * pr + lane] = (c == row) ? 1.0 : 0.0;
     __syncwarp();
-    if (active) {
-        // x <- x H_0 H_1 ... : x[j+1:] -= tau_j (x[j+1:] . v_j) v_j,  v_j = (1, S[j][j+2:])
+    // Every lane takes part in the loads and shuffles below; lanes without a row carry zeros.
+    {
+        // x <- x H_0 H_1 ... : x[j+1:] -= tau_j (x[j+1:] . v_j) v_j,  v_j = (1, S[j][j+2:]).
+        // The reflector is fetched 32 entries at a time (one per lane) and broadcast by shuffle.
         const double *__restrict__ A = D.S;
+        const int zl = (lane < pr) ? lane : 0;
         for (int j = 0; j + 2 < k; ++j) {
             const double tau = D.tau[j];
             if (tau == 0.0) continue;
             const double *v = A + (int64_t)j * k;   // v[c] for c >= j+2
-            double dot = z[(j + 1) * pr + lane];
-            for (int c = j + 2; c < k; ++c) dot += z[c * pr + lane] * v[c];
-            dot *= tau;
-            z[(j + 1) * pr + lane] -= dot;
-            for (int c = j + 2; c < k; ++c) z[c * pr + lane] -= dot * v[c];
+            double dot0 = z[(j + 1) * pr + zl], dot1 = 0.0;
+            for (int c0 = j + 2; c0 < k; c0 += 32) {
+                const int cn = min(32, k - c0);
+                const double vl = (lane < cn) ? v[c0 + lane] : 0.0;
+                int u = 0;
+                for (; u + 1 < cn; u += 2) {
+                    dot0 += z[(c0 + u) * pr + zl] * __shfl_sync(0xffffffffu, vl, u);
+                    dot1 += z[(c0 + u + 1) * pr + zl] * __shfl_sync(0xffffffffu, vl, u + 1);
+                }
+                if (u < cn) dot0 += z[(c0 + u) * pr + zl] * __shfl_sync(0xffffffffu, vl, u);
+            }
+            const double dot = (dot0 + dot1) * tau;
+            if (active) z[(j + 1) * pr + zl] -= dot;
+            for (int c0 = j + 2; c0 < k; c0 += 32) {
+                const int cn = min(32, k - c0);
+                const double vl = (lane < cn) ? v[c0 + lane] : 0.0;
+                for (int u = 0; u < cn; ++u) {
+                    const double vu = __shfl_sync(0xffffffffu, vl, u);
+                    if (active) z[(c0 + u) * pr + zl] -= dot * vu;
+                }
+            }
         }
-        // logged rotations
+        __syncwarp();
+        // logged rotations, fetched 32 at a time (one per lane) and broadcast by shuffle
         const int nsw = *D.nsweeps;
         const double2 *__restrict__ rot = D.rot;
         const int2 *__restrict__ sweeps = D.sweeps;
@@ -196,16 +227,26 @@ eigvec_panel_kernel(const RefreshDev *__restrict__ rd, const RowItem *__restrict
         for (int sidx = 0; sidx < nsw; ++sidx) {
             const int2 sw = sweeps[sidx];
             int i = sw.x;
-            double f = z[(i + 1) * pr + lane];
-            for (int t = 0; t < sw.y; ++t, --i) {
-                const double2 cs = rot[off + t];
-                const double zi = z[i * pr + lane];
-                z[(i + 1) * pr + lane] = cs.y * zi + cs.x * f;
-                f = cs.x * zi - cs.y * f;
+            double f = z[(i + 1) * pr + zl];
+            for (int t0 = 0; t0 < sw.y; t0 += 32) {
+                const int cn = min(32, sw.y - t0);
+                double2 mine = make_double2(1.0, 0.0);
+                if (lane < cn) mine = rot[off + t0 + lane];
+#pragma unroll 4
+                for (int u = 0; u < cn; ++u, --i) {
+                    const double c = __shfl_sync(0xffffffffu, mine.x, u);
+                    const double sn = __shfl_sync(0xffffffffu, mine.y, u);
+                    const double zi = z[i * pr + zl];
+                    if (active) z[(i + 1) * pr + zl] = sn * zi + c * f;
+                    f = c * zi - sn * f;
+                }
             }
-            z[(i + 1) * pr + lane] = f;
+            if (active) z[(i + 1) * pr + zl] = f;
             off += sw.y;
         }
+    }
+    __syncwarp();
+    if (active) {
         // rank the eigenvalues (descending, ties by index) and emit the leading r columns
         const double *__restrict__ lam = D.dvec;
         for (int j = 0; j < k; ++j) {
@@ -269,7 +310,7 @@ cudaError_t eig_tridiag_batched(const RefreshDev *rd, const int32_t *list, int n
         pn_cfg = pn_bytes;
     }
     tridiag_kernel<<<nlist, TR_THREADS, tr_bytes, stream>>>(rd, list, kpad);
-    ql_log_kernel<<<nlist, 32, 0, stream>>>(rd, list);
+    ql_log_kernel<<<nlist, 32, (size_t)2 * kmax * sizeof(double), stream>>>(rd, list);
     eig_rank_kernel<<<nlist, 256, 0, stream>>>(rd, list);
     eigvec_panel_kernel<<<npanels, 32, pn_bytes, stream>>>(rd, panel_items, pr);
     return cudaGetLastError();
