@@ -286,7 +286,7 @@ def run_ours(args, w: ti.Workload):
     for rep in range(max(5, min(20, args.steps))):
         if flush is not None:
             flush.fill_(rep)
-        plan.step(tsr.make_hyper(1), seed=seed, fuse_adam=True)
+        plan.step(tsr.make_hyper(1), seed=seed, fuse_adam=not args.unfused)
         st_rows.append(plan.stage_ms())
     st_med = [statistics.median(r[i] for r in st_rows) for i in range(6)]
     apply_ms = st_med[5]
@@ -390,6 +390,7 @@ def main():
     ap.add_argument("--refresh-reps", type=int, default=1)
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--unfused", action="store_true", help="diagnostic: run the core update as its own launch")
     ap.add_argument("--random-bases", action="store_true",
                     help="profiling aid: random bases instead of the initial refresh (numbers not for reporting)")
     args = ap.parse_args()

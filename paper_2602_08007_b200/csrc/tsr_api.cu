@@ -288,6 +288,8 @@ StepScalars make_scalars(const tsr_hyper *h)
 {
     StepScalars sc;
     sc.beta1 = h->beta1; sc.beta2 = h->beta2; sc.eps = h->eps;
+    sc.omb1 = (float)(1.0 - (double)h->beta1);
+    sc.omb2 = (float)(1.0 - (double)h->beta2);
     const double t = (double)h->step;
     sc.inv_bc1 = (float)(1.0 / (1.0 - pow((double)h->beta1, t)));
     sc.inv_bc2 = (float)(1.0 / (1.0 - pow((double)h->beta2, t)));
@@ -791,7 +793,7 @@ tsr_status tsr_bind(tsr_ctx *ctx, const tsr_mat_ptrs *ptrs, int32_t count, void 
         CoreUpdateArgs &ca = cu_all[i];
         memset(&ca, 0, sizeof ca);
         ca.C = b.p.C; ca.Cout = b.p.C; ca.mom1 = b.p.M; ca.mom2 = b.p.Vm; ca.d_f32 = b.D32;
-        ca.d_bf16 = b.fast ? b.Db : nullptr; ca.dt_bf16 = b.fast ? b.Dbt : nullptr; ca.ldd = b.rl;
+        ca.d_bf16 = nullptr; ca.dt_bf16 = b.fast ? b.Dbt : nullptr; ca.ldd = b.rl;
         ca.split_stride = 0; ca.r = (int)r; ca.nsplit = 1;
         cu_split[i] = ca;
         cu_split[i].C = b.partial; cu_split[i].nsplit = b.nsplit; cu_split[i].split_stride = r * r;
@@ -821,7 +823,7 @@ tsr_status tsr_bind(tsr_ctx *ctx, const tsr_mat_ptrs *ptrs, int32_t count, void 
             if ((s = encode_map(ctx, &P.tmB, b.Tt, r, m, b.ml, ctx->bn[kd])) != TSR_OK) return s;
             P.out = (kd == KC) ? (void *)b.p.C : (void *)b.partial;
             P.ld_out = r; P.split_stride = r * r;
-            P.mom1 = b.p.M; P.mom2 = b.p.Vm; P.d_bf16 = b.Db; P.dt_bf16 = b.Dbt; P.ldd = b.rl;
+            P.mom1 = b.p.M; P.mom2 = b.p.Vm; P.d_bf16 = nullptr; P.dt_bf16 = b.Dbt; P.ldd = b.rl;
         }
         {   // P = U D : A = U copy [m x r], B = D^T copy [r x r]
             UmmaProblem &P = probs[KP][i];

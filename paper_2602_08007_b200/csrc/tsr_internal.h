@@ -59,6 +59,7 @@ struct UmmaTile {
 
 struct StepScalars {       // per-step scalars shared by all blocks
     float beta1, beta2, eps;
+    float omb1, omb2;       // 1 - beta, formed in FP64 from the FP32 betas the caller passed
     float inv_bc1, inv_bc2; // 1 / (1 - beta^t)
     float decay;            // 1 - lr * weight_decay
     float step_scale;       // lr * scale

@@ -26,7 +26,8 @@
 
 namespace tsr {
 
-constexpr int UG_THREADS = 256;
+constexpr int UG_THREADS = 384;   // warps 0-1: TMA / MMA, warps 2-3 idle, warps 4-11: epilogue
+constexpr int UG_EPI_WARPS = 8;
 
 template <int BN, int PLANES>
 struct UmmaSmem {
@@ -36,7 +37,7 @@ struct UmmaSmem {
     static constexpr int STAGES = (192 * 1024) / STAGE_BYTES > 6 ? 6 : (192 * 1024) / STAGE_BYTES;
     static constexpr int PATCH_OFFSET = STAGES * STAGE_BYTES;
     static constexpr int PATCH_BYTES = 32 * 33 * 4;                  // per epilogue warp
-    static constexpr int BAR_OFFSET = PATCH_OFFSET + 4 * PATCH_BYTES;
+    static constexpr int BAR_OFFSET = PATCH_OFFSET + UG_EPI_WARPS * PATCH_BYTES;
     static constexpr int NBARS = 2 * STAGES + 4;
     static constexpr int TOTAL = BAR_OFFSET + NBARS * 8 + 64 + 1024;  // + slack for 1024-byte alignment
 };
@@ -64,7 +65,7 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
     if (threadIdx.x == 0) {
         s_timeout = 0;
         for (int s = 0; s < STAGES; ++s) { mbar_init(smem_u32(bar_full + s), 1); mbar_init(smem_u32(bar_empty + s), 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(bar_acc_full + b), 1); mbar_init(smem_u32(bar_acc_empty + b), 4); }
+        for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(bar_acc_full + b), 1); mbar_init(smem_u32(bar_acc_empty + b), UG_EPI_WARPS); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
@@ -133,26 +134,48 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
             }
         }
     } else if (warp >= 4) {
+        // eight epilogue warps: warp e reads TMEM lanes 32 (e % 4) .. + 31 (the quarter a warp may
+        // access is fixed by its index modulo 4) and the column half e / 4 of the tile
         const int q = warp & 3;
-        float *patch = (float *)(smem + SM::PATCH_OFFSET + q * SM::PATCH_BYTES);   // [32][33]
+        const int half = (warp - 4) >> 2;
+        float *patch = (float *)(smem + SM::PATCH_OFFSET + (warp - 4) * SM::PATCH_BYTES);   // [32][33]
         uint32_t tc = 0;
         bool ok = true;
         for (int t = blockIdx.x; t < num_tiles && ok; t += stride, ++tc) {
             const UmmaTile tile = tiles[t];
             const UmmaProblem *__restrict__ P = probs + tile.prob;
             const uint32_t buf = tc & 1u;
-            if (!mbar_wait(smem_u32(bar_acc_full + buf), (tc >> 1) & 1u)) { s_timeout = 1; ok = false; break; }
-            tc_fence_after();
             const int N = P->N, M = P->M;
             const int row0 = tile.m0 + q * 32;
+            if (EPI == EPI_CORE_UPDATE) {
+                // pull this warp's slice of the moments towards L2 while the MMAs of the tile run
+                const int prow = row0 + lane;
+                if (prow < M) {
+                    const int w = min(BN / 2, N - tile.n0 - half * (BN / 2));
+                    const char *a1 = (const char *)(P->mom1 + (int64_t)prow * N + tile.n0 + half * (BN / 2));
+                    const char *a2 = (const char *)(P->mom2 + (int64_t)prow * N + tile.n0 + half * (BN / 2));
+                    for (int o = 0; o < w * 4; o += 128) {
+                        asm volatile("prefetch.global.L2 [%0];" ::"l"(a1 + o));
+                        if (sc.rule != TSR_RULE_SGD) asm volatile("prefetch.global.L2 [%0];" ::"l"(a2 + o));
+                    }
+                }
+            }
+            if (!mbar_wait(smem_u32(bar_acc_full + buf), (tc >> 1) & 1u)) { s_timeout = 1; ok = false; break; }
+            tc_fence_after();
             const int nrows = min(32, M - row0);        // may be <= 0
+            const int c_begin = half * (BN / 2), c_end = c_begin + BN / 2;
+            if (tile.n0 + c_begin >= N) {   // this warp's column half lies outside the matrix
+                tc_fence_before();
+                if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar_acc_empty + buf)) : "memory");
+                continue;
+            }
 #pragma unroll 1
-            for (int c0 = 0; c0 < BN; c0 += 32) {
+            for (int c0 = c_begin; c0 < c_end; c0 += 32) {
                 const int col0 = tile.n0 + c0;
                 if (col0 >= N) break;
                 uint32_t v[32];
                 tc_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + buf * BN + (uint32_t)c0, v);
-                if (c0 + 32 >= BN || col0 + 32 >= N) {   // last chunk of the tile: release the accumulator
+                if (c0 + 32 >= c_end || col0 + 32 >= N) {   // this warp's last chunk of the tile: release the accumulator
                     tc_fence_before();
                     if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar_acc_empty + buf)) : "memory");
                 }
@@ -168,11 +191,12 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
                     }
                     continue;
                 }
-                // Fast paths (full 32-column chunk, aligned rows): lane = row, each lane moves whole
-                // 32-byte sectors of its own row.
-                const bool full_chunk = (ncols == 32);
-                if (EPI == EPI_STORE_F32 && full_chunk && (P->ld_out & 3) == 0 && (col0 & 3) == 0 &&
+                // Fast paths (full 32 x 32 chunk): transpose through the warp's patch so that lane = column;
+                // every global access is then one full row segment (128 bytes of FP32, 64 of BF16).
+                const bool full_chunk = (ncols == 32) && (nrows == 32);
+                if (EPI == EPI_STORE_F32 && ncols == 32 && (P->ld_out & 3) == 0 && (col0 & 3) == 0 &&
                     (((uintptr_t)P->out) & 15) == 0 && (P->split_stride & 3) == 0) {
+                    // lane = row: each lane writes 128 contiguous bytes of its own row
                     if (lane < nrows) {
                         float *out = (float *)P->out + (int64_t)tile.split * P->split_stride + (int64_t)(row0 + lane) * P->ld_out + col0;
 #pragma unroll
@@ -182,7 +206,7 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
                     }
                     continue;
                 }
-                if (EPI == EPI_STORE_BF16 && full_chunk && (P->ld_out & 7) == 0 && (col0 & 7) == 0 &&
+                if (EPI == EPI_STORE_BF16 && ncols == 32 && (P->ld_out & 7) == 0 && (col0 & 7) == 0 &&
                     (((uintptr_t)P->out) & 15) == 0) {
                     if (lane < nrows) {
                         bf16 *out = (bf16 *)P->out + (int64_t)(row0 + lane) * P->ld_out + col0;
@@ -199,56 +223,44 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
                     }
                     continue;
                 }
-                if (EPI == EPI_CORE_UPDATE && full_chunk && (N & 7) == 0 && (P->ldd & 7) == 0 &&
-                    ((((uintptr_t)P->out) | ((uintptr_t)P->mom1) | ((uintptr_t)P->mom2) | ((uintptr_t)P->d_bf16)) & 15) == 0) {
-                    if (lane < nrows) {
-                        const int64_t e0 = (int64_t)(row0 + lane) * N + col0;   // C, M, Vm are dense r x r (N = r)
+                if (full_chunk && EPI == EPI_CORE_UPDATE) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) patch[lane * 33 + j] = __uint_as_float(v[j]);
+                    __syncwarp();
+                    if (false) {
+                    } else if (EPI == EPI_CORE_UPDATE) {
+                        const int64_t e0 = (int64_t)row0 * N + col0 + lane;   // C, M, Vm are dense r x r (N = r)
                         float *cp = (float *)P->out + e0;
                         float *m1p = P->mom1 + e0;
                         float *m2p = P->mom2 + e0;
-                        bf16 *dp = P->d_bf16 + (int64_t)(row0 + lane) * P->ldd + col0;
-                        bf16 *dtp = P->dt_bf16 + (int64_t)col0 * P->ldd + row0 + lane;
+                        bf16 *dp = P->d_bf16 ? P->d_bf16 + (int64_t)row0 * P->ldd + col0 + lane : nullptr;
                         const int64_t ldd = P->ldd;
                         const bool sgd = (sc.rule == TSR_RULE_SGD);
-                        float m1[32], m2[32];
 #pragma unroll
-                        for (int j = 0; j < 32; j += 4) {
-                            const float4 a = *(const float4 *)(m1p + j);
-                            m1[j] = a.x; m1[j + 1] = a.y; m1[j + 2] = a.z; m1[j + 3] = a.w;
-                        }
-                        if (!sgd) {
+                        for (int i0 = 0; i0 < 32; i0 += 16) {
+                            float m1[16], m2[16];
 #pragma unroll
-                            for (int j = 0; j < 32; j += 4) {
-                                const float4 a = *(const float4 *)(m2p + j);
-                                m2[j] = a.x; m2[j + 1] = a.y; m2[j + 2] = a.z; m2[j + 3] = a.w;
+                            for (int i = 0; i < 16; ++i) m1[i] = m1p[(int64_t)(i0 + i) * N];
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) m2[i] = sgd ? 0.f : m2p[(int64_t)(i0 + i) * N];
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) {
+                                const float c = patch[(i0 + i) * 33 + lane];
+                                const float dd = core_update_elem(c, m1[i], m2[i], sc);
+                                cp[(int64_t)(i0 + i) * N] = c;
+                                m1p[(int64_t)(i0 + i) * N] = m1[i];
+                                if (!sgd) m2p[(int64_t)(i0 + i) * N] = m2[i];
+                                if (dp) dp[(int64_t)(i0 + i) * ldd] = __float2bfloat16_rn(dd);
+                                patch[(i0 + i) * 33 + lane] = dd;
                             }
-                        } else {
-#pragma unroll
-                            for (int j = 0; j < 32; ++j) m2[j] = 0.f;
                         }
-                        float dd[32];
+                        __syncwarp();
+                        // D^T: back to lane = row
+                        bf16 *dtp = P->dt_bf16 + (int64_t)col0 * ldd + row0 + lane;
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) dd[j] = core_update_elem(__uint_as_float(v[j]), m1[j], m2[j], sc);
-#pragma unroll
-                        for (int j = 0; j < 32; j += 4) {
-                            *(float4 *)(cp + j) = make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]),
-                                                              __uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
-                            *(float4 *)(m1p + j) = make_float4(m1[j], m1[j + 1], m1[j + 2], m1[j + 3]);
-                            if (!sgd) *(float4 *)(m2p + j) = make_float4(m2[j], m2[j + 1], m2[j + 2], m2[j + 3]);
-                        }
-#pragma unroll
-                        for (int j = 0; j < 32; j += 8) {
-                            uint4 pk;
-                            __nv_bfloat162 h0 = __floats2bfloat162_rn(dd[j], dd[j + 1]);
-                            __nv_bfloat162 h1 = __floats2bfloat162_rn(dd[j + 2], dd[j + 3]);
-                            __nv_bfloat162 h2 = __floats2bfloat162_rn(dd[j + 4], dd[j + 5]);
-                            __nv_bfloat162 h3 = __floats2bfloat162_rn(dd[j + 6], dd[j + 7]);
-                            pk.x = *(uint32_t *)&h0; pk.y = *(uint32_t *)&h1; pk.z = *(uint32_t *)&h2; pk.w = *(uint32_t *)&h3;
-                            *(uint4 *)(dp + j) = pk;
-                        }
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) dtp[(int64_t)j * ldd] = __float2bfloat16_rn(dd[j]);
+                        for (int j = 0; j < 32; ++j) dtp[(int64_t)j * ldd] = __float2bfloat16_rn(patch[lane * 33 + j]);
                     }
+                    __syncwarp();
                     continue;
                 }
                 // Ragged or unaligned chunk: transpose through the patch so that lane = column and
@@ -278,7 +290,7 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
                             ((float *)P->out)[e] = c;
                             P->mom1[e] = m1;
                             if (sc.rule != TSR_RULE_SGD) P->mom2[e] = m2;
-                            P->d_bf16[(int64_t)(row0 + i) * P->ldd + col] = __float2bfloat16_rn(dd);
+                            if (P->d_bf16) P->d_bf16[(int64_t)(row0 + i) * P->ldd + col] = __float2bfloat16_rn(dd);
                             patch[i * 33 + lane] = dd;
                         }
                     }

@@ -66,3 +66,12 @@ def check_refresh(plan, i, G64, Om64, r, q, gap, tol_sub=TOL_SUBSPACE):
     assert np.linalg.norm(proj(U[:, :gap]) - proj(Uo[:, :gap])) < tol_sub
     assert np.linalg.norm(proj(V[:, :gap]) - proj(Vo[:, :gap])) < tol_sub
     return Uo, Vo, sig
+
+
+def f32(x: float) -> float:
+    """The value an FP32 field of tsr_hyper holds for x, widened exactly to FP64 (the oracle is
+    given the same bits the library receives)."""
+    return float(np.float32(x))
+
+
+HYPER = dict(lr=f32(1e-3), beta1=f32(0.9), beta2=f32(0.999), eps=f32(1e-8))

@@ -6,7 +6,7 @@ import torch
 
 import oracle
 import tsr_inputs as ti
-from helpers import (TOL_BF16, TOL_F32, check_refresh, fill_gradient, fill_weights, rel_fro, set_bases, to64)
+from helpers import (HYPER, TOL_BF16, TOL_F32, check_refresh, f32, fill_gradient, fill_weights, rel_fro, set_bases, to64)
 
 pytestmark = pytest.mark.gpu
 
@@ -38,7 +38,7 @@ def _run_steps(tsr, plan, shapes, dtype, steps, fuse, tol, wd=0.0, scale=1.0, ru
             plan.backproject_apply(h)
         torch.cuda.synchronize()
         for i, ob in enumerate(blks):
-            ob.step(G64[i], lr=1e-3, weight_decay=wd, scale=scale)   # the SGD rule ignores wd / scale
+            ob.step(G64[i], weight_decay=f32(wd), scale=f32(scale), **HYPER)   # the SGD rule ignores wd / scale
             worst["C"] = max(worst["C"], rel_fro(to64(plan.C[i]), ob.C))
             worst["M"] = max(worst["M"], rel_fro(to64(plan.M[i]), ob.M))
             if rule == 0:
@@ -247,7 +247,7 @@ def test_mini_llama_grouped_lockstep_with_refresh():
         plan.step(h, fuse_adam=(t % 2 == 0))
         torch.cuda.synchronize()
         for i, ob in enumerate(blks):
-            ob.step(G64[i], lr=1e-3, skip_refresh=True)
+            ob.step(G64[i], skip_refresh=True, **HYPER)
             for a, b in ((plan.C[i], ob.C), (plan.M[i], ob.M), (plan.Vm[i], ob.Vm), (plan.W[i], ob.W)):
                 worst = max(worst, rel_fro(to64(a), b))
     assert plan.poll_status() == [0] * nb
