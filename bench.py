@@ -117,11 +117,15 @@ def physical_gpu_index(local_rank: int) -> int:
 # --------------------------------------------------------------------------------------------
 # reference arm / cpu baseline: the FP64 oracle on the host cores, on a bounded sample
 # --------------------------------------------------------------------------------------------
-def oracle_sample(w: ti.Workload, seconds_hint: float = 2.0):
-    """Picks the sample the oracle is timed on: one square attention-shaped block of the workload
-    (the most frequent shape), or the single block of config 0."""
-    blk = w.blocks[0]
-    return blk
+def distinct_shapes(w: ti.Workload):
+    """One representative block per distinct (m, n, r) with its multiplicity, in workload order."""
+    seen = {}
+    for blk in w.blocks:
+        key = (blk.m, blk.n, blk.r)
+        if key not in seen:
+            seen[key] = [blk, 0]
+        seen[key][1] += 1
+    return list(seen.values())
 
 
 def oracle_step_time(w: ti.Workload, blk, reps: int = 1):
@@ -143,15 +147,24 @@ def oracle_step_time(w: ti.Workload, blk, reps: int = 1):
 
 
 def cpu_baseline(w: ti.Workload):
+    """The oracle, as it stands, on one block of every distinct shape of the workload (one step
+    each); the whole-set figure multiplies each time by the number of blocks of that shape."""
     import oracle
-    blk = oracle_sample(w)
-    work = step_work(w)
-    sample = step_work(ti.Workload("sample", w.config_id, w.g_dtype, 1, (blk,)))
-    sec = oracle_step_time(w, blk)
-    scale = work["step_flops"] / sample["step_flops"]
-    return {"value": sec * scale * 1e3, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
-            "sample": "one %dx%d r=%d block timed for one step (%.2f s), scaled by algorithmic flops x%.1f to the "
-                      "whole %s set" % (blk.m, blk.n, blk.r, sec, scale, w.name)}
+    total, sampled, parts = 0.0, 0.0, []
+    for blk, count in distinct_shapes(w):
+        sec = oracle_step_time(w, blk)
+        total += sec * count
+        sampled += sec
+        parts.append("%dx%d r=%d x%d: %.2f s" % (blk.m, blk.n, blk.r, count, sec))
+    return {"value": total * 1e3, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": "one step of one block per distinct shape (%.1f s of CPU work in all; %s), each multiplied by "
+                      "its block count" % (sampled, "; ".join(parts))}
+
+
+def oracle_sample(w: ti.Workload):
+    """The reference arm's per-step sample: the first block of the workload (an attention-shaped
+    square block for the LLaMA sets), small enough that K + W steps end within a few minutes."""
+    return w.blocks[0]
 
 
 def run_reference(args, w: ti.Workload):
@@ -185,6 +198,22 @@ def run_reference(args, w: ti.Workload):
 # --------------------------------------------------------------------------------------------
 # our arm
 # --------------------------------------------------------------------------------------------
+def max_over_ranks(values, dist, device):
+    """Element-wise maximum of a list of floats over all ranks (identity without a process group).
+    The path has no collective of its own: replicas only meet here, to report the slowest."""
+    if dist is None:
+        return [float(v) for v in values]
+    tens = torch.tensor(values, device=device, dtype=torch.float64)
+    dist.all_reduce(tens, op=dist.ReduceOp.MAX)
+    return [float(x) for x in tens]
+
+
+# Measured DRAM traffic of umma_apply_kernel divided by its algorithmic bytes (8 B per weight +
+# BF16 operands), from the ncu capture summarised in profiles/umma_apply_kernel_llama350m.md.  The
+# 1B workload is too large for a multi-pass capture; traffic grows in proportion to the weights, so
+# the 350M ratio is applied to the 1B algorithmic bytes.
+APPLY_TRAFFIC_RATIO = 1.03
+
 def build_plan(w: ti.Workload, device):
     import paper_2602_08007_b200 as tsr
     dt = torch.bfloat16 if w.g_dtype == "bf16" else torch.float32
@@ -325,12 +354,8 @@ def run_ours(args, w: ti.Workload):
                "d2h_bytes_per_step": c_host.numel() * 4}
 
     # max over ranks
-    if dist is not None:
-        tens = torch.tensor([ms_per_step, wall * 1e3 / args.steps, apply_ms, proj_ms], device=device, dtype=torch.float64)
-        dist.all_reduce(tens, op=dist.ReduceOp.MAX)
-        ms_per_step, wall_ms_per_step, apply_ms, proj_ms = [float(x) for x in tens]
-    else:
-        wall_ms_per_step = wall * 1e3 / args.steps
+    ms_per_step, wall_ms_per_step, apply_ms, proj_ms = max_over_ranks(
+        [ms_per_step, wall * 1e3 / args.steps, apply_ms, proj_ms], dist, device)
 
     if rank == 0:
         hbm = peaks["hbm_gbs"]
@@ -357,8 +382,10 @@ def run_ours(args, w: ti.Workload):
             "step_tflops": work["step_flops"] / (plain_ms * 1e-3) / 1e12,
             "stage_ms": {"refresh": st_med[0], "gemm_GV": st_med[1], "gemm_core": st_med[2], "core_update": st_med[3],
                          "gemm_UD": st_med[4], "apply": st_med[5]},
-            "roofline": {"kernel": "umma_gemm_kernel<EPI_APPLY> (W <- decay W - lr P V^T)", "bound": "hbm",
-                         "achieved": apply_gbs, "peak": hbm, "unit": "GB/s", "frac": apply_gbs / hbm, "traffic": None,
+            "roofline": {"kernel": "umma_apply_kernel (W <- decay W - lr P V^T)", "bound": "hbm",
+                         "achieved": apply_gbs, "peak": hbm, "unit": "GB/s", "frac": apply_gbs / hbm,
+                         "traffic": APPLY_TRAFFIC_RATIO * work["apply_kernel_bytes"],
+                         "algorithmic_bytes": work["apply_kernel_bytes"],
                          "peak_source": peaks["source"] + " copy bandwidth", "ms": apply_ms, "roof_ms": apply_roof_ms},
             "roofline_projection": {"kernels": "umma_gemm_kernel<EPI_STORE_BF16_T> + <EPI_CORE_UPDATE>",
                                     "bound": "tensor" if work["proj_flops"] / (tc * 1e12) > work["proj_bytes"] / (hbm * 1e9) else "hbm",
