@@ -212,7 +212,7 @@ def max_over_ranks(values, dist, device):
 # BF16 operands), from the ncu capture summarised in profiles/umma_apply_kernel_llama350m.md.  The
 # 1B workload is too large for a multi-pass capture; traffic grows in proportion to the weights, so
 # the 350M ratio is applied to the 1B algorithmic bytes.
-APPLY_TRAFFIC_RATIO = 1.03
+APPLY_TRAFFIC_RATIO = 0.98
 
 def build_plan(w: ti.Workload, device):
     import paper_2602_08007_b200 as tsr
