@@ -1,0 +1,160 @@
+"""Edge and degenerate cases of the CUDA path: tiny and extreme shapes, q = 0 / p = 0, exactly
+rank-deficient and non-finite gradients (flagged per block, never a fault), run-to-run
+determinism and checkpoint / resume."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import tsr_inputs as ti
+from helpers import HYPER, TOL_BF16, TOL_F32, check_refresh, fill_gradient, fill_weights, proj, rel_fro, set_bases, to64
+
+pytestmark = pytest.mark.gpu
+
+
+def _tsr():
+    import paper_2602_08007_b200 as tsr
+    return tsr
+
+
+@pytest.mark.parametrize("dtype,shape,gap", [
+    (torch.float32, dict(m=24, n=17, r=5, p=2, q=1), 3),        # tiny, nothing a multiple of any tile
+    (torch.bfloat16, dict(m=64, n=48, r=8, p=0, q=0), 4),       # no oversampling, no power iteration
+    (torch.bfloat16, dict(m=40, n=136, r=32, p=8, q=1), 8),     # k = min(m, n): the sketch spans everything
+    (torch.float32, dict(m=150, n=90, r=30, p=6, q=3), 12),     # three power iterations
+])
+def test_refresh_small_and_extreme_shapes(dtype, shape, gap):
+    tsr = _tsr()
+    plan = tsr.Plan([shape], g_dtype=dtype)
+    G64 = fill_gradient(plan, 0, 31, signal_rank=gap)
+    Om = ti.omega(shape["n"], shape["r"] + shape["p"], 32).cuda()
+    plan.init_subspace(omegas=[Om])
+    torch.cuda.synchronize()
+    assert plan.poll_status() == [0]
+    tol_sub = 1e-3 if shape["q"] > 0 else 2e-2     # without a power iteration the sketch itself is less accurate
+    check_refresh(plan, 0, G64, to64(Om), shape["r"], shape["q"], gap, tol_sub=tol_sub)
+
+
+def test_tiny_step_matches_oracle():
+    tsr = _tsr()
+    shapes = [dict(m=9, n=7, r=3), dict(m=33, n=65, r=8)]
+    plan = tsr.Plan(shapes, g_dtype=torch.float32)
+    blks = []
+    for i, s in enumerate(shapes):
+        set_bases(plan, i, ti.orthonormal(s["m"], s["r"], 40 + i), ti.orthonormal(s["n"], s["r"], 50 + i))
+        W0 = fill_weights(plan, i, 60 + i)
+        ob = oracle.OracleBlock(W0, s["r"], 0, 0, 0)
+        ob.set_bases(to64(plan.U[i]), to64(plan.V[i]))
+        blks.append(ob)
+    plan.bases_changed()
+    for t in (1, 2, 3):
+        G64 = [fill_gradient(plan, i, 70 + 10 * t + i, signal_rank=2) for i in range(2)]
+        plan.step(tsr.make_hyper(t))
+        torch.cuda.synchronize()
+        for i, ob in enumerate(blks):
+            ob.step(G64[i], **HYPER)
+            assert rel_fro(to64(plan.W[i]), ob.W) < TOL_F32 and rel_fro(to64(plan.C[i]), ob.C) < TOL_F32
+
+
+def test_exactly_rank_deficient_gradient_is_flagged_not_fatal():
+    tsr = _tsr()
+    shape = dict(m=256, n=320, r=32, p=8, q=1)
+    plan = tsr.Plan([shape, shape], g_dtype=torch.float32)
+    # block 0: exact rank 12 < k = 40 (no noise); block 1: an ordinary full-rank gradient
+    G0 = fill_gradient(plan, 0, 81, signal_rank=12, noise_std=0.0)
+    G1 = fill_gradient(plan, 1, 82, signal_rank=12)
+    oms = [ti.omega(320, 40, 83).cuda(), ti.omega(320, 40, 84).cuda()]
+    plan.init_subspace(omegas=oms)
+    torch.cuda.synchronize()
+    st = plan.poll_status()
+    assert st[0] == 8 and st[1] == 0                      # TSR_ERR_RANK_DEFICIENT on block 0 only
+    U0, V0 = to64(plan.U[0]), to64(plan.V[0])
+    assert np.isfinite(U0).all() and np.isfinite(V0).all()
+    # the rank-12 range of G is still captured by the leading directions
+    Un, sn, Vnt = np.linalg.svd(G0)
+    assert np.linalg.norm(proj(U0[:, :12]) - proj(Un[:, :12])) < 1e-3
+    assert np.linalg.norm(proj(V0[:, :12]) - proj(Vnt.T[:, :12])) < 1e-3
+    check_refresh(plan, 1, G1, to64(oms[1]), 32, 1, 12)   # the healthy block is untouched by its neighbour
+    assert plan.poll_status() == [0, 0]                   # polling clears the words
+
+
+def test_nonfinite_gradient_flags_its_block_only():
+    tsr = _tsr()
+    shape = dict(m=192, n=256, r=16, p=8, q=1)
+    res = []
+    for poison in (False, True):
+        plan = tsr.Plan([shape, shape], g_dtype=torch.bfloat16)
+        for i in range(2):
+            fill_gradient(plan, i, 90 + i, signal_rank=8)
+            fill_weights(plan, i, 92 + i)
+        if poison:
+            plan.G[0][5, 7] = float("nan")
+        oms = [ti.omega(256, 24, 94).cuda(), ti.omega(256, 24, 95).cuda()]
+        plan.init_subspace(omegas=oms)
+        plan.step(tsr.make_hyper(1))
+        torch.cuda.synchronize()
+        st = plan.poll_status()
+        res.append((st, plan.W[1].clone(), plan.U[1].clone()))
+    assert res[0][0] == [0, 0]
+    assert res[1][0][0] == 9 and res[1][0][1] == 0        # TSR_ERR_NONFINITE on the poisoned block only
+    assert torch.equal(res[0][1], res[1][1]) and torch.equal(res[0][2], res[1][2])
+
+
+def test_runs_are_bitwise_reproducible_and_resumable():
+    tsr = _tsr()
+    w = ti.workload(1)
+    shapes = [dict(m=b.m, n=b.n, r=b.r, p=b.p, q=b.q, K=3, is_embedding=b.is_embedding) for b in (w.blocks[0], w.blocks[4], w.blocks[6])]
+    shapes.append(dict(m=9000, n=512, r=64, p=8, q=1, K=3, is_embedding=True))     # split-K core GEMM
+
+    def run(steps_a, steps_b):
+        plan = tsr.Plan(shapes, g_dtype=torch.bfloat16)
+        for i, s in enumerate(shapes):
+            fill_gradient(plan, i, 200 + i)
+            fill_weights(plan, i, 210 + i)
+        plan.init_subspace(seed=11)
+        for t in range(1, steps_a + 1):
+            for i in range(len(shapes)):
+                fill_gradient(plan, i, 1000 * t + i)
+            plan.step(tsr.make_hyper(t), seed=11)
+        if steps_b:
+            # checkpoint: the state is the caller's tensors plus the step counter; resume in a new plan
+            torch.cuda.synchronize()
+            plan2 = tsr.Plan(shapes, g_dtype=torch.bfloat16)
+            for i in range(len(shapes)):
+                for a, b in ((plan2.W, plan.W), (plan2.U, plan.U), (plan2.V, plan.V), (plan2.M, plan.M), (plan2.Vm, plan.Vm)):
+                    a[i].copy_(b[i])
+            plan2.bases_changed()
+            plan = plan2
+            for t in range(steps_a + 1, steps_a + steps_b + 1):
+                for i in range(len(shapes)):
+                    fill_gradient(plan, i, 1000 * t + i)
+                plan.step(tsr.make_hyper(t), seed=11)
+        torch.cuda.synchronize()
+        assert plan.poll_status() == [0] * len(shapes)
+        return [(plan.W[i].clone(), plan.U[i].clone(), plan.M[i].clone(), plan.Vm[i].clone()) for i in range(len(shapes))]
+
+    a = run(7, 0)
+    b = run(7, 0)
+    c = run(4, 3)          # refreshes at t = 3 and t = 6 fall on either side of the checkpoint
+    for x, y, z in zip(a, b, c):
+        for p_, q_, r_ in zip(x, y, z):
+            assert torch.equal(p_, q_) and torch.equal(p_, r_)
+
+
+def test_bind_rejects_bad_arguments_without_touching_buffers():
+    tsr = _tsr()
+    import ctypes
+    plan = tsr.Plan([dict(m=64, n=64, r=8)], g_dtype=torch.bfloat16)
+    w_before = plan.W[0].clone()
+    L = tsr.lib()
+    h = tsr.make_hyper(0)                                  # step must be >= 1
+    assert L.tsr_step_grouped(plan.ctx, ctypes.byref(h), 0, 1, None) == 1
+    h = tsr.make_hyper(1, beta1=1.5)
+    assert L.tsr_step_grouped(plan.ctx, ctypes.byref(h), 0, 1, None) == 1
+    idx = (ctypes.c_int32 * 2)(0, 0)                       # duplicate index
+    assert L.tsr_project_core_grouped(plan.ctx, idx, 2, None) == 1
+    idx = (ctypes.c_int32 * 1)(3)                          # out of range
+    assert L.tsr_project_core_grouped(plan.ctx, idx, 1, None) == 1
+    assert b"out of range" in L.tsr_last_error(plan.ctx)
+    torch.cuda.synchronize()
+    assert torch.equal(w_before, plan.W[0])
