@@ -186,43 +186,57 @@ eigvec_panel_kernel(const RefreshDev *__restrict__ rd, const RowItem *__restrict
     if (lane < pr)
         for (int c = 0; c < k; ++c) z[c * pr + lane] = (c == row) ? 1.0 : 0.0;
     __syncwarp();
-    // Every lane takes part in the loads and shuffles below; lanes without a row carry zeros.
+    // Lanes without a row (lane >= pr, or a row past the end) shadow lane 0's reads and never write.
     {
         // x <- x H_0 H_1 ... : x[j+1:] -= tau_j (x[j+1:] . v_j) v_j,  v_j = (1, S[j][j+2:]).
-        // The reflector is fetched 32 entries at a time (one per lane) and broadcast by shuffle.
+        // The reflector is staged 64 entries at a time in a small shared buffer that every lane reads.
         const double *__restrict__ A = D.S;
         const int zl = (lane < pr) ? lane : 0;
+        double *vbuf = z + (size_t)k * pr;       // 64 doubles behind the panel
         for (int j = 0; j + 2 < k; ++j) {
             const double tau = D.tau[j];
             if (tau == 0.0) continue;
             const double *v = A + (int64_t)j * k;   // v[c] for c >= j+2
-            double dot0 = z[(j + 1) * pr + zl], dot1 = 0.0;
-            for (int c0 = j + 2; c0 < k; c0 += 32) {
-                const int cn = min(32, k - c0);
-                const double vl = (lane < cn) ? v[c0 + lane] : 0.0;
+            double d0 = z[(j + 1) * pr + zl], d1 = 0.0, d2 = 0.0, d3 = 0.0;
+            for (int c0 = j + 2; c0 < k; c0 += 64) {
+                const int cn = min(64, k - c0);
+                __syncwarp();
+                vbuf[lane] = (lane < cn) ? v[c0 + lane] : 0.0;
+                vbuf[lane + 32] = (lane + 32 < cn) ? v[c0 + lane + 32] : 0.0;
+                __syncwarp();
+                const double *zc = z + (size_t)c0 * pr + zl;
                 int u = 0;
-                for (; u + 1 < cn; u += 2) {
-                    dot0 += z[(c0 + u) * pr + zl] * __shfl_sync(0xffffffffu, vl, u);
-                    dot1 += z[(c0 + u + 1) * pr + zl] * __shfl_sync(0xffffffffu, vl, u + 1);
+                for (; u + 3 < cn; u += 4) {
+                    d0 += zc[(u + 0) * pr] * vbuf[u + 0];
+                    d1 += zc[(u + 1) * pr] * vbuf[u + 1];
+                    d2 += zc[(u + 2) * pr] * vbuf[u + 2];
+                    d3 += zc[(u + 3) * pr] * vbuf[u + 3];
                 }
-                if (u < cn) dot0 += z[(c0 + u) * pr + zl] * __shfl_sync(0xffffffffu, vl, u);
+                for (; u < cn; ++u) d0 += zc[u * pr] * vbuf[u];
             }
-            const double dot = (dot0 + dot1) * tau;
+            const double dot = ((d0 + d1) + (d2 + d3)) * tau;
             if (active) z[(j + 1) * pr + zl] -= dot;
-            for (int c0 = j + 2; c0 < k; c0 += 32) {
-                const int cn = min(32, k - c0);
-                const double vl = (lane < cn) ? v[c0 + lane] : 0.0;
-                for (int u = 0; u < cn; ++u) {
-                    const double vu = __shfl_sync(0xffffffffu, vl, u);
-                    if (active) z[(c0 + u) * pr + zl] -= dot * vu;
+            for (int c0 = j + 2; c0 < k; c0 += 64) {
+                const int cn = min(64, k - c0);
+                __syncwarp();
+                vbuf[lane] = (lane < cn) ? v[c0 + lane] : 0.0;
+                vbuf[lane + 32] = (lane + 32 < cn) ? v[c0 + lane + 32] : 0.0;
+                __syncwarp();
+                if (active) {
+                    double *zc = z + (size_t)c0 * pr + zl;
+#pragma unroll 4
+                    for (int u = 0; u < cn; ++u) zc[u * pr] -= dot * vbuf[u];
                 }
             }
         }
         __syncwarp();
-        // logged rotations, fetched 32 at a time (one per lane) and broadcast by shuffle
+        // logged rotations, staged 32 at a time in the shared buffer; four rotations are applied per
+        // trip with their inputs loaded up front, so that no shared-memory load sits on the
+        // dependent chain f -> f
         const int nsw = *D.nsweeps;
         const double2 *__restrict__ rot = D.rot;
         const int2 *__restrict__ sweeps = D.sweeps;
+        double2 *rbuf = (double2 *)vbuf;
         int off = 0;
         for (int sidx = 0; sidx < nsw; ++sidx) {
             const int2 sw = sweeps[sidx];
@@ -230,15 +244,28 @@ eigvec_panel_kernel(const RefreshDev *__restrict__ rd, const RowItem *__restrict
             double f = z[(i + 1) * pr + zl];
             for (int t0 = 0; t0 < sw.y; t0 += 32) {
                 const int cn = min(32, sw.y - t0);
-                double2 mine = make_double2(1.0, 0.0);
-                if (lane < cn) mine = rot[off + t0 + lane];
-#pragma unroll 4
-                for (int u = 0; u < cn; ++u, --i) {
-                    const double c = __shfl_sync(0xffffffffu, mine.x, u);
-                    const double sn = __shfl_sync(0xffffffffu, mine.y, u);
+                __syncwarp();
+                if (lane < cn) rbuf[lane] = rot[off + t0 + lane];
+                __syncwarp();
+                int u = 0;
+                for (; u + 3 < cn; u += 4, i -= 4) {
+                    const double z0 = z[(i - 0) * pr + zl], z1 = z[(i - 1) * pr + zl];
+                    const double z2 = z[(i - 2) * pr + zl], z3 = z[(i - 3) * pr + zl];
+                    const double2 r0 = rbuf[u], r1 = rbuf[u + 1], r2 = rbuf[u + 2], r3 = rbuf[u + 3];
+                    const double o0 = r0.y * z0 + r0.x * f;  f = r0.x * z0 - r0.y * f;
+                    const double o1 = r1.y * z1 + r1.x * f;  f = r1.x * z1 - r1.y * f;
+                    const double o2 = r2.y * z2 + r2.x * f;  f = r2.x * z2 - r2.y * f;
+                    const double o3 = r3.y * z3 + r3.x * f;  f = r3.x * z3 - r3.y * f;
+                    if (active) {
+                        z[(i + 1) * pr + zl] = o0; z[(i - 0) * pr + zl] = o1;
+                        z[(i - 1) * pr + zl] = o2; z[(i - 2) * pr + zl] = o3;
+                    }
+                }
+                for (; u < cn; ++u, --i) {
+                    const double2 r0 = rbuf[u];
                     const double zi = z[i * pr + zl];
-                    if (active) z[(i + 1) * pr + zl] = sn * zi + c * f;
-                    f = c * zi - sn * f;
+                    if (active) z[(i + 1) * pr + zl] = r0.y * zi + r0.x * f;
+                    f = r0.x * zi - r0.y * f;
                 }
             }
             if (active) z[(i + 1) * pr + zl] = f;
@@ -298,7 +325,7 @@ cudaError_t eig_tridiag_batched(const RefreshDev *rd, const int32_t *list, int n
     const int kpad = kmax + 8;
     const size_t tr_bytes = (size_t)3 * kpad * sizeof(double);
     const int pr = eig_panel_rows(kmax);
-    const size_t pn_bytes = (size_t)pr * kmax * sizeof(double);
+    const size_t pn_bytes = (size_t)pr * kmax * sizeof(double) + 64 * sizeof(double);   // panel + staging buffer
     static size_t tr_cfg = 0, pn_cfg = 0;
     cudaError_t e;
     if (tr_bytes > tr_cfg) {
@@ -307,6 +334,8 @@ cudaError_t eig_tridiag_batched(const RefreshDev *rd, const int32_t *list, int n
     }
     if (pn_bytes > pn_cfg) {
         if ((e = cudaFuncSetAttribute(eigvec_panel_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pn_bytes)) != cudaSuccess) return e;
+        // ask for the largest shared-memory carve-out so that two panels fit on one SM
+        if ((e = cudaFuncSetAttribute(eigvec_panel_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 100)) != cudaSuccess) return e;
         pn_cfg = pn_bytes;
     }
     tridiag_kernel<<<nlist, TR_THREADS, tr_bytes, stream>>>(rd, list, kpad);

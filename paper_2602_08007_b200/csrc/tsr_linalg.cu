@@ -14,7 +14,7 @@ namespace tsr {
 // each slab writes its own partial (upper-triangular tiles only), a second kernel adds the
 // partials in slab order and mirrors the result, so the sum is deterministic.
 // ---------------------------------------------------------------------------------------
-constexpr int GR_T = 32;  // output tile edge
+constexpr int GR_T = 64;  // output tile edge
 
 __global__ void __launch_bounds__(256)
 gram_partial_kernel(const RefreshDev *__restrict__ rd, const RowItem *__restrict__ items, int side, int src_sel)
@@ -26,36 +26,57 @@ gram_partial_kernel(const RefreshDev *__restrict__ rd, const RowItem *__restrict
     if (tj < ti || ti * GR_T >= k || tj * GR_T >= k) return;
     const int rows = side ? d.n : d.m;
     const float *__restrict__ X = d.buf[src_sel];
-    __shared__ float Xi[16][GR_T + 1];
-    __shared__ float Xj[16][GR_T + 1];
-    const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;  // 16 x 16 threads, 2 x 2 outputs each
+    __shared__ __align__(16) float Xi[16][GR_T + 4];
+    __shared__ __align__(16) float Xj[16][GR_T + 4];
+    const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;  // 16 x 16 threads, 4 x 4 outputs each
     const int row_begin = it.row0;
     const int row_end = min(rows, row_begin + GRAM_ROWS);
-    double acc[2][2] = {{0.0, 0.0}, {0.0, 0.0}};
-    for (int r0 = row_begin; r0 < row_end; r0 += 16) {
-        for (int e = threadIdx.x; e < 16 * GR_T; e += 256) {
+    double acc[4][4];
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+        for (int b = 0; b < 4; ++b) acc[a][b] = 0.0;
+    float ri[4], rj[4];
+    auto fetch = [&](int r0) {
+#pragma unroll
+        for (int l = 0; l < 4; ++l) {
+            const int e = threadIdx.x + l * 256;
             const int rr = e / GR_T, cc = e % GR_T;
             const int row = r0 + rr;
             const int ci = ti * GR_T + cc, cj = tj * GR_T + cc;
-            Xi[rr][cc] = (row < row_end && ci < k) ? X[(int64_t)row * k + ci] : 0.f;
-            Xj[rr][cc] = (row < row_end && cj < k) ? X[(int64_t)row * k + cj] : 0.f;
+            ri[l] = (row < row_end && ci < k) ? X[(int64_t)row * k + ci] : 0.f;
+            rj[l] = (row < row_end && cj < k) ? X[(int64_t)row * k + cj] : 0.f;
+        }
+    };
+    fetch(row_begin);
+    for (int r0 = row_begin; r0 < row_end; r0 += 16) {
+#pragma unroll
+        for (int l = 0; l < 4; ++l) {
+            const int e = threadIdx.x + l * 256;
+            Xi[e / GR_T][e % GR_T] = ri[l];
+            Xj[e / GR_T][e % GR_T] = rj[l];
         }
         __syncthreads();
+        if (r0 + 16 < row_end) fetch(r0 + 16);
 #pragma unroll
         for (int rr = 0; rr < 16; ++rr) {
-            const double a0 = Xi[rr][ty * 2], a1 = Xi[rr][ty * 2 + 1];
-            const double b0 = Xj[rr][tx * 2], b1 = Xj[rr][tx * 2 + 1];
-            acc[0][0] += a0 * b0; acc[0][1] += a0 * b1;
-            acc[1][0] += a1 * b0; acc[1][1] += a1 * b1;
+            const float4 af = *(const float4 *)&Xi[rr][ty * 4];
+            const float4 bf = *(const float4 *)&Xj[rr][tx * 4];
+            const double av[4] = {af.x, af.y, af.z, af.w};
+            const double bv[4] = {bf.x, bf.y, bf.z, bf.w};
+#pragma unroll
+            for (int a = 0; a < 4; ++a)
+#pragma unroll
+                for (int b = 0; b < 4; ++b) acc[a][b] += av[a] * bv[b];
         }
         __syncthreads();
     }
     double *P = d.gpart + (int64_t)(it.row0 / GRAM_ROWS) * k * k;
 #pragma unroll
-    for (int a = 0; a < 2; ++a)
+    for (int a = 0; a < 4; ++a)
 #pragma unroll
-        for (int b = 0; b < 2; ++b) {
-            const int i = ti * GR_T + ty * 2 + a, j = tj * GR_T + tx * 2 + b;
+        for (int b = 0; b < 4; ++b) {
+            const int i = ti * GR_T + ty * 4 + a, j = tj * GR_T + tx * 4 + b;
             if (i < k && j < k) P[(int64_t)i * k + j] = acc[a][b];
         }
 }
@@ -103,7 +124,7 @@ constexpr int CH_THREADS = 1024;
 __global__ void __launch_bounds__(CH_THREADS)
 chol_inverse_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ list, int kpad)
 {
-    extern __shared__ double ch_smem[];   // [CH_NB][kpad] panel of R rows, reused as 2 x [kpad][CH_NB] inverse panels
+    extern __shared__ double ch_smem[];   // [CH_NB][kpad] panel of R rows, reused as [2 * CH_NB][kpad] columns of the inverse
     const RefreshDev d = rd[list[blockIdx.x]];
     const int k = d.k;
     double *__restrict__ S = d.S;
@@ -209,6 +230,8 @@ cudaError_t chol_inverse_batched(const RefreshDev *rd, const int32_t *list, int 
     if (bytes > configured) {
         cudaError_t e = cudaFuncSetAttribute(chol_inverse_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
         if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(chol_inverse_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
+        if (e != cudaSuccess) return e;
         configured = bytes;
     }
     chol_inverse_kernel<<<nlist, CH_THREADS, bytes, stream>>>(rd, list, kpad);
@@ -234,33 +257,44 @@ rows_gemm_kernel(const RefreshDev *__restrict__ rd, const RowItem *__restrict__ 
     float *__restrict__ D = (dst_sel < 3) ? d.buf[dst_sel] : (dst_sel == 3 ? d.U : d.V);
     const int m0 = it.row0;
 
-    __shared__ float As[16][64 + 4];
-    __shared__ float Bs[16][64 + 4];
+    __shared__ __align__(16) float As[16][64 + 4];
+    __shared__ __align__(16) float Bs[16][64 + 4];
     const int tid = threadIdx.x, tx = tid % 16, ty = tid / 16;
     float acc[4][4];
 #pragma unroll
     for (int a = 0; a < 4; ++a)
 #pragma unroll
         for (int b = 0; b < 4; ++b) acc[a][b] = 0.f;
-    for (int k0 = 0; k0 < K; k0 += 16) {
+    // global -> registers -> shared, with the next K slice in flight while the current one is used
+    float ra[4], rb[4];
+    auto fetch = [&](int k0) {
 #pragma unroll
         for (int l = 0; l < 4; ++l) {
             const int e = tid + l * 256;
             const int ak = e % 16, ai = e / 16;
             const int gi = m0 + ai, gk = k0 + ak;
-            As[ak][ai] = (gi < rows && gk < K) ? A[(int64_t)gi * K + gk] : 0.f;
+            ra[l] = (gi < rows && gk < K) ? A[(int64_t)gi * K + gk] : 0.f;
             const int bj = e % 64, bk = e / 64;
             const int gj = n0 + bj, gk2 = k0 + bk;
-            Bs[bk][bj] = (gj < N && gk2 < K) ? B[(int64_t)gk2 * N + gj] : 0.f;
+            rb[l] = (gj < N && gk2 < K) ? B[(int64_t)gk2 * N + gj] : 0.f;
+        }
+    };
+    fetch(0);
+    for (int k0 = 0; k0 < K; k0 += 16) {
+#pragma unroll
+        for (int l = 0; l < 4; ++l) {
+            const int e = tid + l * 256;
+            As[e % 16][e / 16] = ra[l];
+            Bs[e / 64][e % 64] = rb[l];
         }
         __syncthreads();
+        if (k0 + 16 < K) fetch(k0 + 16);
 #pragma unroll
         for (int kk = 0; kk < 16; ++kk) {
-            float av[4], bv[4];
-#pragma unroll
-            for (int a = 0; a < 4; ++a) av[a] = As[kk][ty * 4 + a];
-#pragma unroll
-            for (int b = 0; b < 4; ++b) bv[b] = Bs[kk][tx * 4 + b];
+            const float4 af = *(const float4 *)&As[kk][ty * 4];
+            const float4 bf = *(const float4 *)&Bs[kk][tx * 4];
+            const float av[4] = {af.x, af.y, af.z, af.w};
+            const float bv[4] = {bf.x, bf.y, bf.z, bf.w};
 #pragma unroll
             for (int a = 0; a < 4; ++a)
 #pragma unroll
