@@ -353,6 +353,27 @@ def run_ours(args, w: ti.Workload):
         e2e = {"value": e2e_ms, "unit": UNIT, "h2d_bytes_per_step": sum(g.numel() * g.element_size() for g in g_host),
                "d2h_bytes_per_step": c_host.numel() * 4}
 
+    # dense AdamW for non-matrix parameters (Section 3.4): HBM-bound, 28 bytes per FP32 parameter
+    dense = None
+    if args.dense_params > 0:
+        n = args.dense_params
+        dp = [torch.randn(n, device=device) for _ in range(1)]
+        dg = [torch.randn(n, device=device) for _ in range(1)]
+        dm = [torch.zeros(n, device=device) for _ in range(1)]
+        dv = [torch.zeros(n, device=device) for _ in range(1)]
+        for t in range(1, 4):
+            tsr.dense_adamw(dp, dg, dm, dv, tsr.make_hyper(t))
+        a, bb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for t in range(4, 9):
+            tsr.dense_adamw(dp, dg, dm, dv, tsr.make_hyper(t))
+        bb.record()
+        torch.cuda.synchronize()
+        dms = a.elapsed_time(bb) / 5
+        dense = {"params": n, "ms": dms, "achieved_gbs": 28.0 * n / (dms * 1e-3) / 1e9,
+                 "frac_of_hbm": 28.0 * n / (dms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+        del dp, dg, dm, dv
+
     # max over ranks
     ms_per_step, wall_ms_per_step, apply_ms, proj_ms = max_over_ranks(
         [ms_per_step, wall * 1e3 / args.steps, apply_ms, proj_ms], dist, device)
@@ -393,6 +414,7 @@ def run_ours(args, w: ti.Workload):
                                     "frac": proj_roof_ms / proj_ms},
             "comm_bytes": {"core_per_step": core_b, "sketch_per_refresh": sketch_b,
                            "dense_fp32_per_step": 4 * sum(b.m * b.n for b in w.blocks)},
+            "dense_adamw": dense,
             "device_status": sorted(set(status + status2 + status3)),
             "clocks": sampler.summary(),
             "e2e": e2e,
@@ -417,6 +439,8 @@ def main():
     ap.add_argument("--refresh-reps", type=int, default=1)
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--dense-params", type=int, default=1 << 26,
+                    help="size of the dense-AdamW micro-measurement (0 = skip)")
     ap.add_argument("--unfused", action="store_true", help="diagnostic: run the core update as its own launch")
     ap.add_argument("--random-bases", action="store_true",
                     help="profiling aid: random bases instead of the initial refresh (numbers not for reporting)")

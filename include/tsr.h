@@ -198,6 +198,26 @@ TSR_API tsr_status tsr_step_grouped(tsr_ctx *ctx, const tsr_hyper *hyper, uint64
 TSR_API tsr_status tsr_step_grouped_host(tsr_ctx *ctx, const void *const *G_host, float *C_host,
                                          const tsr_hyper *hyper, uint64_t seed, int32_t fuse_adam, void *stream);
 
+/* ---- dense parameters ------------------------------------------------------------------------ */
+
+/* One dense (non-matrix) parameter tensor: biases, normalisation weights.  All DEVICE pointers;
+ * param, m, v are FP32 arrays of `count` elements updated in place, grad is FP32 or BF16. */
+typedef struct {
+    float *param;
+    const void *grad;
+    float *m, *v;
+    int64_t count;
+    int32_t g_dtype; /* tsr_dtype of grad */
+    int32_t reserved;
+} tsr_dense_tensor;
+
+/* Sections 3.1 / 3.4: parameters that are not matrix blocks are updated by dense AdamW,
+ *   m <- b1 m + (1-b1) g;  v <- b2 v + (1-b2) g o g;  p <- p - lr (m_hat / (sqrt(v_hat) + eps) + wd p),
+ * for all listed tensors in one multi-tensor launch per 48 tensors.  `tensors` is a HOST array;
+ * hyper->scale is ignored; hyper->rule must be TSR_RULE_ADAM.  Needs no context and no
+ * workspace.  Errors (null pointers, negative counts, bad dtype) are found before any launch. */
+TSR_API tsr_status tsr_dense_adamw(const tsr_dense_tensor *tensors, int32_t count, const tsr_hyper *hyper, void *stream);
+
 /* ---- reporting -------------------------------------------------------------------------- */
 
 /* Section 3.2: bytes one worker would hand to the all-reduce in one step, summed over blocks:

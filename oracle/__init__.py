@@ -10,6 +10,7 @@ from .tsr_oracle import (  # noqa: F401
     backproject_apply,
     build,
     core_bytes,
+    dense_adamw,
     exact_svd_refresh,
     num_threads,
     orth,

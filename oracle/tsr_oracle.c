@@ -103,6 +103,26 @@ int tsro_sgd_core(int64_t count, const double *Cbar, double *M, double *D, doubl
 }
 
 /* ------------------------------------------------------------------------- */
+/* Dense AdamW for parameters that are not matrix blocks (Section 3.1, the    */
+/* dense update; Section 3.4 "all non-matrix parameters ... are updated in    */
+/* dense form"): moments, bias correction, decoupled weight decay.            */
+/* ------------------------------------------------------------------------- */
+int tsro_dense_adamw(int64_t count, double *P, const double *G, double *M, double *Vm, double lr,
+                     double beta1, double beta2, double eps, double weight_decay, int64_t t)
+{
+    const double bc1 = 1.0 - pow(beta1, (double)t);
+    const double bc2 = 1.0 - pow(beta2, (double)t);
+    for (int64_t e = 0; e < count; ++e) {
+        const double g = G[e];
+        M[e] = beta1 * M[e] + (1.0 - beta1) * g;
+        Vm[e] = beta2 * Vm[e] + (1.0 - beta2) * (g * g);
+        const double upd = (M[e] / bc1) / (sqrt(Vm[e] / bc2) + eps);
+        P[e] = P[e] - lr * (upd + weight_decay * P[e]);
+    }
+    return 0;
+}
+
+/* ------------------------------------------------------------------------- */
 /* Lift and AdamW apply, Algorithm 1: dW = U D V^T; W <- W - eta(dW + lam W). */
 /* `scale` multiplies the lifted update only (the experiments' "scaling       */
 /* factor"; 1 reproduces Algorithm 1 as printed).                             */

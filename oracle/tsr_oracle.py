@@ -45,6 +45,7 @@ def _load():
             lib.tsro_project_one_sided.argtypes = [_i64, _i64, _i64, _ptr, _i64, _ptr, _ptr]
             lib.tsro_adam_core.argtypes = [_i64, _ptr, _ptr, _ptr, _ptr, _dbl, _dbl, _dbl, _i64]
             lib.tsro_sgd_core.argtypes = [_i64, _ptr, _ptr, _ptr, _dbl]
+            lib.tsro_dense_adamw.argtypes = [_i64, _ptr, _ptr, _ptr, _ptr, _dbl, _dbl, _dbl, _dbl, _dbl, _i64]
             lib.tsro_backproject_apply.argtypes = [_i64, _i64, _i64, _ptr, _ptr, _ptr, _ptr, _i64, _dbl, _dbl, _dbl]
             lib.tsro_orth.argtypes = [_i64, _i64, _ptr, _ptr, _ptr]
             lib.tsro_svd_jacobi.argtypes = [_i64, _i64, _ptr, _ptr, _ptr, _ptr, ctypes.c_int]
@@ -120,6 +121,14 @@ def sgd_core(C, M, beta) -> np.ndarray:
     D = np.empty_like(C)
     _load().tsro_sgd_core(C.size, _p(C), _p(M), _p(D), beta)
     return D
+
+
+def dense_adamw(P, G, M, Vm, lr, beta1, beta2, eps, weight_decay, t) -> None:
+    """Textbook AdamW on a dense parameter array; P, M, Vm (float64, contiguous) updated in place."""
+    G = _f64(G)
+    P, M, Vm = _f64(P, True), _f64(M, True), _f64(Vm, True)
+    assert P.size == G.size == M.size == Vm.size
+    _load().tsro_dense_adamw(P.size, _p(P), _p(G), _p(M), _p(Vm), lr, beta1, beta2, eps, weight_decay, int(t))
 
 
 def backproject_apply(U, D, V, W, lr, weight_decay=0.0, scale=1.0) -> None:

@@ -40,6 +40,11 @@ class MatPtrs(ctypes.Structure):
                 ("M", ctypes.c_void_p), ("Vm", ctypes.c_void_p), ("C", ctypes.c_void_p)]
 
 
+class DenseTensor(ctypes.Structure):
+    _fields_ = [("param", ctypes.c_void_p), ("grad", ctypes.c_void_p), ("m", ctypes.c_void_p), ("v", ctypes.c_void_p),
+                ("count", ctypes.c_int64), ("g_dtype", ctypes.c_int32), ("reserved", ctypes.c_int32)]
+
+
 class Hyper(ctypes.Structure):
     _fields_ = [("lr", ctypes.c_float), ("beta1", ctypes.c_float), ("beta2", ctypes.c_float), ("eps", ctypes.c_float),
                 ("weight_decay", ctypes.c_float), ("scale", ctypes.c_float), ("step", ctypes.c_int64),
@@ -53,7 +58,7 @@ EXPORTS = [
     "tsr_project_core_grouped", "tsr_adam_core_step_grouped", "tsr_backproject_apply_grouped",
     "tsr_rsvd_refresh_grouped", "tsr_embed_step_grouped", "tsr_step_grouped", "tsr_step_grouped_host",
     "tsr_comm_bytes", "tsr_state_elems", "tsr_poll_status", "tsr_generate_omega", "tsr_block_uses_tensor_cores",
-    "tsr_set_profiling", "tsr_get_stage_ms", "tsr_launch_count", "tsr_project_core_static",
+    "tsr_set_profiling", "tsr_get_stage_ms", "tsr_launch_count", "tsr_project_core_static", "tsr_dense_adamw",
 ]
 
 
@@ -111,6 +116,7 @@ def lib():
         L.tsr_get_stage_ms.argtypes = [vp, P(ctypes.c_float), i32]
         L.tsr_launch_count.argtypes = [vp, P(u64)]
         L.tsr_project_core_static.argtypes = [vp, i32, i64, i64, i64, vp, vp, i32, vp, vp]
+        L.tsr_dense_adamw.argtypes = [P(DenseTensor), i32, P(Hyper), vp]
         _lib = L
     return _lib
 
@@ -154,6 +160,20 @@ def project_core_static(G: torch.Tensor, U: torch.Tensor, V: torch.Tensor, C: to
                                        ctypes.c_void_p(C.data_ptr()), _stream_ptr(stream))
     if rc != TSR_OK:
         raise TsrError(rc, "tsr_project_core_static")
+
+
+def dense_adamw(params, grads, ms, vs, hyper: Hyper, stream=None) -> None:
+    """tsr_dense_adamw over lists of torch tensors (params / ms / vs FP32, grads FP32 or BF16,
+    all contiguous and on the current device), updated in place."""
+    n = len(params)
+    arr = (DenseTensor * max(n, 1))()
+    for i in range(n):
+        assert params[i].is_contiguous() and grads[i].is_contiguous() and params[i].dtype == torch.float32
+        arr[i] = DenseTensor(params[i].data_ptr(), grads[i].data_ptr(), ms[i].data_ptr(), vs[i].data_ptr(),
+                             params[i].numel(), TSR_BF16 if grads[i].dtype == torch.bfloat16 else TSR_F32, 0)
+    rc = lib().tsr_dense_adamw(arr, n, ctypes.byref(hyper), _stream_ptr(stream))
+    if rc != TSR_OK:
+        raise TsrError(rc, "tsr_dense_adamw")
 
 
 class Plan:

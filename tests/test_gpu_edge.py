@@ -158,3 +158,27 @@ def test_bind_rejects_bad_arguments_without_touching_buffers():
     assert b"out of range" in L.tsr_last_error(plan.ctx)
     torch.cuda.synchronize()
     assert torch.equal(w_before, plan.W[0])
+
+
+def test_dense_adamw_matches_oracle():
+    """Parameters that are not matrix blocks: multi-tensor dense AdamW against the oracle's."""
+    tsr = _tsr()
+    sizes = [1, 257, 70000, 0, 2048] + [33] * 60            # more than one batch of 48 tensors, one empty
+    gens = torch.Generator().manual_seed(5)
+    P = [torch.randn(n, generator=gens).cuda() for n in sizes]
+    M = [torch.zeros(n).cuda() for n in sizes]
+    V = [torch.zeros(n).cuda() for n in sizes]
+    Po = [to64(p).copy() for p in P]
+    Mo = [np.zeros(n) for n in sizes]
+    Vo = [np.zeros(n) for n in sizes]
+    from helpers import f32
+    for t in range(1, 6):
+        G = [(torch.randn(n, generator=gens).to(torch.bfloat16 if i % 2 else torch.float32)).cuda() for i, n in enumerate(sizes)]
+        tsr.dense_adamw(P, G, M, V, tsr.make_hyper(t, lr=3e-3, beta2=0.95, weight_decay=0.1))
+        torch.cuda.synchronize()
+        for i in range(len(sizes)):
+            oracle.dense_adamw(Po[i], to64(G[i]), Mo[i], Vo[i], f32(3e-3), f32(0.9), f32(0.95), f32(1e-8), f32(0.1), t)
+            if sizes[i]:
+                assert rel_fro(to64(P[i]), Po[i]) < 1e-6 and rel_fro(to64(M[i]), Mo[i]) < 1e-6 and rel_fro(to64(V[i]), Vo[i]) < 1e-6
+    with pytest.raises(tsr.TsrError):
+        tsr.dense_adamw(P[:1], G[:1], M[:1], V[:1], tsr.make_hyper(1, rule=1))

@@ -65,6 +65,20 @@ def test_scale_multiplies_lifted_update_only():
     assert np.abs(blk.W - expect).max() < 1e-14
 
 
+def test_dense_adamw_matches_torch_adamw():
+    rng = np.random.default_rng(12)
+    p0 = rng.standard_normal(257)
+    P, M, Vm = p0.copy(), np.zeros(257), np.zeros(257)
+    w = torch.tensor(p0, dtype=torch.float64, requires_grad=True)
+    opt = torch.optim.AdamW([w], lr=3e-3, betas=(0.9, 0.95), eps=1e-8, weight_decay=0.1)
+    for t in range(1, 9):
+        g = rng.standard_normal(257)
+        oracle.dense_adamw(P, g, M, Vm, 3e-3, 0.9, 0.95, 1e-8, 0.1, t)
+        w.grad = torch.tensor(g, dtype=torch.float64)
+        opt.step()
+        assert np.abs(P - w.detach().numpy()).max() < 1e-14
+
+
 # ---- core Adam: closed forms ------------------------------------------------------------
 def test_adam_constant_core_closed_form():
     # constant core c: m_t = (1-b1^t)c, v_t = (1-b2^t)c^2  =>  D = c / (|c| + eps) at every t
