@@ -90,6 +90,12 @@ struct tsr_ctx {
     bool ev_valid = false;
     cudaStream_t stage_stream = nullptr;
     int stage_next = 0;
+    // refresh runs as up to NGROUP independent groups of blocks on side streams, so that the
+    // latency-bound small-matrix kernels of one group overlap the GEMM-like kernels of another
+    static constexpr int NGROUP = 4;
+    cudaStream_t aux[NGROUP] = {};
+    cudaEvent_t ev_fork = nullptr, ev_join[NGROUP] = {};
+    bool aux_ready = false;
 };
 
 namespace {
@@ -466,15 +472,17 @@ struct RefreshLists {
     std::vector<int> list;
     int nitems[4];
     int kmax, rmax;
+    int32_t *dlist;        // this group's slice of the device list / item tables
+    RowItem *ditems[5];
 };
 
 tsr_status orth_pass(tsr_ctx *ctx, const RefreshLists &L, int side, int src, int dst, cudaStream_t st)
 {
     const int nl = (int)L.list.size();
-    TSR_KERNEL(ctx, 2, gram_batched(ctx->d_refresh, ctx->d_items[side * 2 + 1], L.nitems[side * 2 + 1], ctx->d_list, nl, side,
+    TSR_KERNEL(ctx, 2, gram_batched(ctx->d_refresh, L.ditems[side * 2 + 1], L.nitems[side * 2 + 1], L.dlist, nl, side,
                                src, L.kmax, st));
-    TSR_KERNEL(ctx, 1, chol_inverse_batched(ctx->d_refresh, ctx->d_list, nl, L.kmax, st));
-    TSR_KERNEL(ctx, 1, rows_gemm_batched(ctx->d_refresh, ctx->d_items[side * 2], L.nitems[side * 2], side, src, 0, dst, L.kmax, st));
+    TSR_KERNEL(ctx, 1, chol_inverse_batched(ctx->d_refresh, L.dlist, nl, L.kmax, st));
+    TSR_KERNEL(ctx, 1, rows_gemm_batched(ctx->d_refresh, L.ditems[side * 2], L.nitems[side * 2], side, src, 0, dst, L.kmax, st));
     return TSR_OK;
 }
 
@@ -517,13 +525,17 @@ tsr_status sketch(tsr_ctx *ctx, const RefreshLists &L, bool transposed, bool fro
     return TSR_OK;
 }
 
-tsr_status do_refresh(tsr_ctx *ctx, const std::vector<int> &list, uint64_t seed, const float *const *omegas,
-                      cudaStream_t st)
+// One group of blocks through the whole refresh on stream st.  list_off / item_off: where this
+// group's slices start inside the context's device list / item tables.
+tsr_status do_refresh_group(tsr_ctx *ctx, const std::vector<int> &list, uint64_t seed, const float *const *omegas,
+                            cudaStream_t st, size_t list_off, const size_t *item_off)
 {
     if (list.empty()) return TSR_OK;
     tsr_status s;
     RefreshLists L;
     L.list = list;
+    L.dlist = ctx->d_list + list_off;
+    for (int i = 0; i < 5; ++i) L.ditems[i] = ctx->d_items[i] + item_off[i];
     L.kmax = 1; L.rmax = 1;
     std::vector<RowItem> items[4];
     int qmax = 0;
@@ -541,10 +553,10 @@ tsr_status do_refresh(tsr_ctx *ctx, const std::vector<int> &list, uint64_t seed,
     for (int bi : list)
         if (ctx->blocks[bi].d.q != qmax)
             return fail(ctx, TSR_ERR_UNSUPPORTED, "blocks refreshed in one grouped call must share q");
-    if ((s = upload_list(ctx, ctx->d_list, list, st)) != TSR_OK) return s;
+    if ((s = upload_list(ctx, L.dlist, list, st)) != TSR_OK) return s;
     for (int i = 0; i < 4; ++i) {
         L.nitems[i] = (int)items[i].size();
-        TSR_CUDA(ctx, cudaMemcpyAsync(ctx->d_items[i], items[i].data(), items[i].size() * sizeof(RowItem),
+        TSR_CUDA(ctx, cudaMemcpyAsync(L.ditems[i], items[i].data(), items[i].size() * sizeof(RowItem),
                                       cudaMemcpyHostToDevice, st));
     }
     // Omega and the transposed gradient copies
@@ -568,21 +580,63 @@ tsr_status do_refresh(tsr_ctx *ctx, const std::vector<int> &list, uint64_t seed,
     // B^T = G^T Q (n x k) in buf[0]; small SVD through the k x k Gram matrix B B^T
     if ((s = sketch(ctx, L, true, false, nullptr, st)) != TSR_OK) return s;
     const int nl = (int)list.size();
-    TSR_KERNEL(ctx, 2, gram_batched(ctx->d_refresh, ctx->d_items[3], L.nitems[3], ctx->d_list, nl, 1, 0, L.kmax, st));
+    TSR_KERNEL(ctx, 2, gram_batched(ctx->d_refresh, L.ditems[3], L.nitems[3], L.dlist, nl, 1, 0, L.kmax, st));
     if (L.kmax >= 200) {   // too large for the Jacobi solver: tridiagonal route
         const int pr = eig_panel_rows(L.kmax);
         std::vector<RowItem> panels;
         for (int bi : list)
             for (int r0 = 0; r0 < ctx->blocks[bi].k; r0 += pr) panels.push_back({bi, r0});
-        TSR_CUDA(ctx, cudaMemcpyAsync(ctx->d_items[4], panels.data(), panels.size() * sizeof(RowItem), cudaMemcpyHostToDevice, st));
-        TSR_KERNEL(ctx, 4, eig_tridiag_batched(ctx->d_refresh, ctx->d_list, nl, ctx->d_items[4], (int)panels.size(), L.kmax, st));
+        TSR_CUDA(ctx, cudaMemcpyAsync(L.ditems[4], panels.data(), panels.size() * sizeof(RowItem), cudaMemcpyHostToDevice, st));
+        TSR_KERNEL(ctx, 4, eig_tridiag_batched(ctx->d_refresh, L.dlist, nl, L.ditems[4], (int)panels.size(), L.kmax, st));
     } else {
-        TSR_KERNEL(ctx, 1, jacobi_batched(ctx->d_refresh, ctx->d_list, nl, 40, st));
+        TSR_KERNEL(ctx, 1, jacobi_batched(ctx->d_refresh, L.dlist, nl, 40, st));
     }
     // V = B^T Wt / sigma ; U = Q Wt
-    TSR_KERNEL(ctx, 1, rows_gemm_batched(ctx->d_refresh, ctx->d_items[2], L.nitems[2], 1, 0, 2, 4, L.rmax, st));
-    TSR_KERNEL(ctx, 1, rows_gemm_batched(ctx->d_refresh, ctx->d_items[0], L.nitems[0], 0, 2, 1, 3, L.rmax, st));
+    TSR_KERNEL(ctx, 1, rows_gemm_batched(ctx->d_refresh, L.ditems[2], L.nitems[2], 1, 0, 2, 4, L.rmax, st));
+    TSR_KERNEL(ctx, 1, rows_gemm_batched(ctx->d_refresh, L.ditems[0], L.nitems[0], 0, 2, 1, 3, L.rmax, st));
     return do_shadows(ctx, list, st);
+}
+
+// Refresh of a list of blocks (all with the same q).  Large lists are cut into up to NGROUP groups
+// of consecutive blocks (in tile-table order) that run concurrently on the context's side streams;
+// the caller's stream forks into them and joins afterwards, so the call keeps stream semantics.
+tsr_status do_refresh(tsr_ctx *ctx, const std::vector<int> &list, uint64_t seed, const float *const *omegas,
+                      cudaStream_t st)
+{
+    if (list.empty()) return TSR_OK;
+    const size_t zero[5] = {0, 0, 0, 0, 0};
+    int ngroup = std::min<int>(tsr_ctx::NGROUP, (int)list.size() / 8);
+    if (!ctx->aux_ready || ngroup < 2) return do_refresh_group(ctx, list, seed, omegas, st, 0, zero);
+    // order the listed blocks as the tile tables do, remembering each one's omega
+    std::vector<int> pos(ctx->blocks.size(), 0);
+    for (size_t i = 0; i < ctx->order.size(); ++i) pos[ctx->order[i]] = (int)i;
+    std::vector<size_t> perm(list.size());
+    for (size_t i = 0; i < perm.size(); ++i) perm[i] = i;
+    std::sort(perm.begin(), perm.end(), [&](size_t x, size_t y) { return pos[list[x]] < pos[list[y]]; });
+    TSR_CUDA(ctx, cudaEventRecord(ctx->ev_fork, st));
+    size_t list_off = 0, item_off[5] = {0, 0, 0, 0, 0};
+    tsr_status result = TSR_OK;
+    for (int g = 0; g < ngroup; ++g) {
+        const size_t lo = perm.size() * g / ngroup, hi = perm.size() * (g + 1) / ngroup;
+        std::vector<int> grp;
+        std::vector<const float *> om;
+        for (size_t i = lo; i < hi; ++i) { grp.push_back(list[perm[i]]); om.push_back(omegas ? omegas[perm[i]] : nullptr); }
+        TSR_CUDA(ctx, cudaStreamWaitEvent(ctx->aux[g], ctx->ev_fork, 0));
+        tsr_status s = do_refresh_group(ctx, grp, seed, omegas ? om.data() : nullptr, ctx->aux[g], list_off, item_off);
+        if (s != TSR_OK && result == TSR_OK) result = s;
+        TSR_CUDA(ctx, cudaEventRecord(ctx->ev_join[g], ctx->aux[g]));
+        TSR_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_join[g], 0));
+        list_off += grp.size();
+        for (int bi : grp) {
+            const Block &b = ctx->blocks[bi];
+            item_off[0] += (size_t)((b.d.m + RG_ROWS - 1) / RG_ROWS);
+            item_off[1] += (size_t)gram_chunks(b.d.m);
+            item_off[2] += (size_t)((b.d.n + RG_ROWS - 1) / RG_ROWS);
+            item_off[3] += (size_t)gram_chunks(b.d.n);
+            item_off[4] += (size_t)((b.k + 7) / 8);
+        }
+    }
+    return result;
 }
 
 tsr_status zero_moments(tsr_ctx *ctx, const std::vector<int> &list, cudaStream_t st)
@@ -714,6 +768,10 @@ tsr_status tsr_destroy(tsr_ctx *ctx)
     if (!ctx) return TSR_ERR_INVALID_ARG;
     if (ctx->profiling)
         for (cudaEvent_t e : ctx->ev) if (e) cudaEventDestroy(e);
+    if (ctx->aux_ready) {
+        for (int g = 0; g < tsr_ctx::NGROUP; ++g) { cudaStreamDestroy(ctx->aux[g]); cudaEventDestroy(ctx->ev_join[g]); }
+        cudaEventDestroy(ctx->ev_fork);
+    }
     delete ctx;
     return TSR_OK;
 }
@@ -867,6 +925,14 @@ tsr_status tsr_bind(tsr_ctx *ctx, const tsr_mat_ptrs *ptrs, int32_t count, void 
     TSR_CUDA(ctx, cudaMemcpy(ctx->d_cu_split, cu_split.data(), sizeof(CoreUpdateArgs) * nb, cudaMemcpyHostToDevice));
     TSR_CUDA(ctx, cudaMemcpy(ctx->d_refresh, rdev.data(), sizeof(RefreshDev) * nb, cudaMemcpyHostToDevice));
     TSR_CUDA(ctx, cudaMemset(ctx->d_status, 0, sizeof(int32_t) * nb));
+    if (!ctx->aux_ready) {
+        for (int g = 0; g < tsr_ctx::NGROUP; ++g) {
+            TSR_CUDA(ctx, cudaStreamCreateWithFlags(&ctx->aux[g], cudaStreamNonBlocking));
+            TSR_CUDA(ctx, cudaEventCreateWithFlags(&ctx->ev_join[g], cudaEventDisableTiming));
+        }
+        TSR_CUDA(ctx, cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming));
+        ctx->aux_ready = true;
+    }
     ctx->bound = true;
     ctx->err.clear();
     return TSR_OK;

@@ -12,11 +12,13 @@
 //             from shared-memory descriptors and commits to the stage's "empty" mbarrier and,
 //             per tile, to the accumulator's "full" mbarrier.  The MMAs of tile i+1 overlap the
 //             epilogue of tile i;
-//   warps 4-7 read the accumulator with tcgen05.ld (lane = output row, 32 columns at a time).
-//             Row-major outputs are transposed through a warp-private shared-memory patch so
-//             that every global access is a full 128-byte (FP32) or 64-byte (BF16) row
-//             segment.  Epilogues: plain FP32 / BF16 stores, the transposed BF16 store, and the
-//             fused core update of Section 3.4.
+//   warps 4-11 read the accumulator with tcgen05.ld (lane = output row, 32 columns at a time;
+//             warp e owns TMEM lanes 32 (e % 4).. and the column half e / 4 of the tile).
+//             Epilogues: plain FP32 / BF16 stores (each lane writes whole 32-byte sectors of its
+//             own row), the transposed BF16 store, and the fused core update of Section 3.4,
+//             which goes through a warp-private shared-memory transpose so that its moment
+//             read-modify-write touches full 128-byte row segments, with the moment tiles
+//             prefetched to L2 while the tile's MMAs run.
 // Ragged edges rely on TMA zero fill for loads and on predicated stores.
 // Every mbarrier wait is bounded by a clock budget; on expiry the CTA records
 // TSR_ERR_TIMEOUT, stops storing and still releases its tensor memory before it exits.
@@ -227,8 +229,7 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
 #pragma unroll
                     for (int j = 0; j < 32; ++j) patch[lane * 33 + j] = __uint_as_float(v[j]);
                     __syncwarp();
-                    if (false) {
-                    } else if (EPI == EPI_CORE_UPDATE) {
+                    {
                         const int64_t e0 = (int64_t)row0 * N + col0 + lane;   // C, M, Vm are dense r x r (N = r)
                         float *cp = (float *)P->out + e0;
                         float *m1p = P->mom1 + e0;
