@@ -441,6 +441,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--dense-params", type=int, default=1 << 26,
                     help="size of the dense-AdamW micro-measurement (0 = skip)")
+    ap.add_argument("--layers", type=int, default=0, help="profiling aid: truncate the model to this many layers")
     ap.add_argument("--unfused", action="store_true", help="diagnostic: run the core update as its own launch")
     ap.add_argument("--random-bases", action="store_true",
                     help="profiling aid: random bases instead of the initial refresh (numbers not for reporting)")
@@ -448,6 +449,10 @@ def main():
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
     w = ti.workload(args.config)
+    if args.layers > 0 and args.config > 0:
+        # profiling aid: keep the first `layers` transformer layers (7 blocks each) and the embedding
+        keep = tuple(w.blocks[:7 * args.layers]) + (w.blocks[-1],)
+        w = ti.Workload(w.name + "-first%dlayers" % args.layers, w.config_id, w.g_dtype, w.steps, keep)
     if args.config < 3:
         args.flush_l2 = True
     if args.impl == "reference":

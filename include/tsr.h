@@ -79,6 +79,13 @@ typedef enum { TSR_F32 = 0, TSR_BF16 = 1 } tsr_dtype;
  * no second moment, no weight decay, no bias correction; beta1 is its momentum). */
 typedef enum { TSR_RULE_ADAM = 0, TSR_RULE_SGD = 1 } tsr_rule;
 
+/* Per-block options.  TSR_BLOCK_REEXPRESS_MOMENT: at every refresh (not at tsr_init_subspace,
+ * whose moments are zero) replace the first moment by M' = Unew^T (Uold M Vold^T) Vnew, i.e. keep
+ * the lifted moment, projected onto the refreshed subspaces -- the "refresh alignment" the
+ * paper's convergence analysis assumes.  Algorithm 1 as printed leaves M untouched (flag clear).
+ * The second moment is never re-expressed.  Costs (m + n) r + 3 r^2 floats of extra scratch. */
+typedef enum { TSR_BLOCK_REEXPRESS_MOMENT = 1 } tsr_block_flags;
+
 /* One matrix block.  Embedding blocks are ordinary blocks with their own (r, K)
  * (Section 3.6); is_embedding only labels them for tsr_embed_step. */
 typedef struct {
@@ -91,7 +98,7 @@ typedef struct {
     int32_t g_dtype;      /* tsr_dtype of G                                             */
     int32_t w_dtype;      /* tsr_dtype of W; only TSR_F32 is implemented                */
     int32_t is_embedding; /* 0 / 1                                                      */
-    int32_t reserved;     /* must be 0                                                  */
+    int32_t flags;        /* bit set of tsr_block_flags; 0 = Algorithm 1 as printed     */
 } tsr_mat_desc;
 
 typedef struct {

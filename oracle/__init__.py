@@ -16,6 +16,7 @@ from .tsr_oracle import (  # noqa: F401
     orth,
     project_core,
     project_one_sided,
+    reexpress_moment,
     rsvd_refresh,
     sgd_core,
     sketch_bytes,

@@ -392,6 +392,33 @@ done:
     return rc;
 }
 
+/* ------------------------------------------------------------------------- */
+/* Moment re-expression at a refresh (the "refresh alignment" assumption of   */
+/* the convergence analysis, Appendix): the core moment is replaced by the    */
+/* one whose lifted matrix is the old lifted moment projected onto the new    */
+/* subspaces,  M' = Unew^T (Uold M Vold^T) Vnew.  Algorithm 1 itself leaves   */
+/* M untouched; this is an option.                                            */
+/* ------------------------------------------------------------------------- */
+int tsro_reexpress_moment(int64_t m, int64_t n, int64_t r, const double *Uold, const double *Vold,
+                          const double *Unew, const double *Vnew, double *M)
+{
+    double *L = (double *)calloc((size_t)m * (size_t)n, sizeof(double));   /* lifted old moment */
+    double *UM = (double *)calloc((size_t)m * (size_t)r, sizeof(double));
+    if (!L || !UM) { free(L); free(UM); return -1; }
+    for (int64_t i = 0; i < m; ++i)
+        for (int64_t a = 0; a < r; ++a)
+            for (int64_t b = 0; b < r; ++b) UM[IDX(i, b, r)] += Uold[IDX(i, a, r)] * M[IDX(a, b, r)];
+    for (int64_t i = 0; i < m; ++i)
+        for (int64_t j = 0; j < n; ++j) {
+            double s = 0.0;
+            for (int64_t b = 0; b < r; ++b) s += UM[IDX(i, b, r)] * Vold[IDX(j, b, r)];
+            L[IDX(i, j, n)] = s;
+        }
+    int rc = tsro_project_core(m, n, r, L, n, Unew, Vnew, M);
+    free(L); free(UM);
+    return rc;
+}
+
 /* Exact-SVD refresh (the "naive" arm of Section 3.5): top-r singular vectors of G itself. */
 int tsro_exact_svd_refresh(int64_t m, int64_t n, int64_t r, const double *G, int64_t ldg, double *U,
                            double *V, double *sigma)

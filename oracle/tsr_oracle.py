@@ -50,6 +50,7 @@ def _load():
             lib.tsro_orth.argtypes = [_i64, _i64, _ptr, _ptr, _ptr]
             lib.tsro_svd_jacobi.argtypes = [_i64, _i64, _ptr, _ptr, _ptr, _ptr, ctypes.c_int]
             lib.tsro_rsvd_refresh.argtypes = [_i64, _i64, _i64, _i64, _i64, _ptr, _i64, _ptr, _ptr, _ptr, _ptr]
+            lib.tsro_reexpress_moment.argtypes = [_i64, _i64, _i64, _ptr, _ptr, _ptr, _ptr, _ptr]
             lib.tsro_exact_svd_refresh.argtypes = [_i64, _i64, _i64, _ptr, _i64, _ptr, _ptr, _ptr]
             for name in ("tsro_core_bytes", "tsro_sketch_bytes", "tsro_state_elems"):
                 getattr(lib, name).restype = ctypes.c_uint64
@@ -171,6 +172,15 @@ def rsvd_refresh(G, Omega, r, q):
     _check(_load().tsro_rsvd_refresh(m, n, r, k - r, q, _p(G), n, _p(Omega), _p(U), _p(V), _p(S)),
            "rsvd_refresh")
     return U, V, S
+
+
+def reexpress_moment(M, Uold, Vold, Unew, Vnew) -> None:
+    """M <- Unew^T (Uold M Vold^T) Vnew, in place (optional moment re-expression at a refresh)."""
+    M = _f64(M, True)
+    Uold, Vold, Unew, Vnew = _f64(Uold), _f64(Vold), _f64(Unew), _f64(Vnew)
+    m, r = Uold.shape
+    n = Vold.shape[0]
+    _check(_load().tsro_reexpress_moment(m, n, r, _p(Uold), _p(Vold), _p(Unew), _p(Vnew), _p(M)), "reexpress_moment")
 
 
 def exact_svd_refresh(G, r):

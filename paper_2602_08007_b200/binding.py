@@ -20,6 +20,7 @@ _lib = None
 TSR_OK = 0
 TSR_F32, TSR_BF16 = 0, 1
 TSR_RULE_ADAM, TSR_RULE_SGD = 0, 1
+TSR_BLOCK_REEXPRESS_MOMENT = 1
 
 STATUS_NAMES = {
     0: "TSR_OK", 1: "TSR_ERR_INVALID_ARG", 2: "TSR_ERR_SHAPE", 3: "TSR_ERR_ALIGNMENT", 4: "TSR_ERR_WORKSPACE",
@@ -32,7 +33,7 @@ class MatDesc(ctypes.Structure):
     _fields_ = [("m", ctypes.c_int64), ("n", ctypes.c_int64), ("ldg", ctypes.c_int64), ("ldw", ctypes.c_int64),
                 ("r", ctypes.c_int32), ("p", ctypes.c_int32), ("q", ctypes.c_int32), ("K", ctypes.c_int32),
                 ("g_dtype", ctypes.c_int32), ("w_dtype", ctypes.c_int32), ("is_embedding", ctypes.c_int32),
-                ("reserved", ctypes.c_int32)]
+                ("flags", ctypes.c_int32)]
 
 
 class MatPtrs(ctypes.Structure):
@@ -220,7 +221,7 @@ class Plan:
             self.C.append(torch.zeros(r, r, dtype=torch.float32, device=self.device))
             self.descs[i] = MatDesc(m, n, ldg, ldw, r, int(g("p", 0)), int(g("q", 0)), int(g("K", 0)),
                                     TSR_BF16 if g_dtype == torch.bfloat16 else TSR_F32, TSR_F32,
-                                    1 if g("is_embedding", False) else 0, 0)
+                                    1 if g("is_embedding", False) else 0, int(g("flags", 0)))
         self.ctx = ctypes.c_void_p()
         self._check(L.tsr_create(ctypes.byref(self.ctx), self.descs, nb), create=True)
         sb, rb = ctypes.c_size_t(), ctypes.c_size_t()

@@ -41,6 +41,7 @@ struct Block {
     int2 *sweeps = nullptr;
     int32_t *nsweeps = nullptr, *rank = nullptr;
     int rot_cap = 0, sweep_cap = 0;
+    float *Uold = nullptr, *Vold = nullptr, *Ra = nullptr, *Rb = nullptr, *Rt = nullptr;   // moment re-expression
     int tile_begin[NKIND], tile_end[NKIND];
 };
 
@@ -209,6 +210,13 @@ void layout(tsr_ctx *ctx, Arena &a, bool assign, size_t *step_end)
             b.tau = (double *)tau; b.dvec = (double *)dv; b.evec = (double *)ev; b.rot = (double2 *)rot;
             b.sweeps = (int2 *)sw; b.nsweeps = (int32_t *)nsw; b.rank = (int32_t *)rk;
             b.rot_cap = rot_cap; b.sweep_cap = sweep_cap;
+        }
+        if (b.d.flags & TSR_BLOCK_REEXPRESS_MOMENT) {
+            void *uo = a.take((size_t)(m * r) * 4), *vo = a.take((size_t)(n * r) * 4);
+            void *ra = a.take((size_t)(r * r) * 4), *rb = a.take((size_t)(r * r) * 4), *rt = a.take((size_t)(r * r) * 4);
+            if (assign) { b.Uold = (float *)uo; b.Vold = (float *)vo; b.Ra = (float *)ra; b.Rb = (float *)rb; b.Rt = (float *)rt; }
+        }
+        if (assign) {
             b.Om = (float *)om; b.buf[0] = (float *)b0; b.buf[1] = (float *)b1; b.buf[2] = (float *)b2;
             b.S = (double *)S; b.Xw = (double *)Xw; b.Wj = (double *)Wj; b.gpart = (double *)gp; b.lam = (double *)lam;
             b.Rinv = (float *)ri; b.Wu = (float *)wu; b.Wv = (float *)wv;
@@ -528,7 +536,7 @@ tsr_status sketch(tsr_ctx *ctx, const RefreshLists &L, bool transposed, bool fro
 // One group of blocks through the whole refresh on stream st.  list_off / item_off: where this
 // group's slices start inside the context's device list / item tables.
 tsr_status do_refresh_group(tsr_ctx *ctx, const std::vector<int> &list, uint64_t seed, const float *const *omegas,
-                            cudaStream_t st, size_t list_off, const size_t *item_off)
+                            cudaStream_t st, size_t list_off, const size_t *item_off, bool reexpress)
 {
     if (list.empty()) return TSR_OK;
     tsr_status s;
@@ -592,8 +600,25 @@ tsr_status do_refresh_group(tsr_ctx *ctx, const std::vector<int> &list, uint64_t
         TSR_KERNEL(ctx, 1, jacobi_batched(ctx->d_refresh, L.dlist, nl, 40, st));
     }
     // V = B^T Wt / sigma ; U = Q Wt
+    if (reexpress)   // keep the outgoing bases of the blocks that asked for moment re-expression
+        for (int bi : list) {
+            Block &b = ctx->blocks[bi];
+            if (!(b.d.flags & TSR_BLOCK_REEXPRESS_MOMENT)) continue;
+            TSR_CUDA(ctx, cudaMemcpyAsync(b.Uold, b.p.U, (size_t)b.d.m * b.d.r * 4, cudaMemcpyDeviceToDevice, st));
+            TSR_CUDA(ctx, cudaMemcpyAsync(b.Vold, b.p.V, (size_t)b.d.n * b.d.r * 4, cudaMemcpyDeviceToDevice, st));
+        }
     TSR_KERNEL(ctx, 1, rows_gemm_batched(ctx->d_refresh, L.ditems[2], L.nitems[2], 1, 0, 2, 4, L.rmax, st));
     TSR_KERNEL(ctx, 1, rows_gemm_batched(ctx->d_refresh, L.ditems[0], L.nitems[0], 0, 2, 1, 3, L.rmax, st));
+    if (reexpress)   // M <- (Unew^T Uold) M (Vold^T Vnew)
+        for (int bi : list) {
+            Block &b = ctx->blocks[bi];
+            if (!(b.d.flags & TSR_BLOCK_REEXPRESS_MOMENT)) continue;
+            const int m = (int)b.d.m, n = (int)b.d.n, r = b.d.r;
+            TSR_KERNEL(ctx, 1, simt_gemm(r, r, m, b.p.U, TSR_F32, 1, r, b.Uold, r, 1, b.Ra, r, SIMT_STORE, 0, 0, st));
+            TSR_KERNEL(ctx, 1, simt_gemm(r, r, n, b.Vold, TSR_F32, 1, r, b.p.V, r, 1, b.Rb, r, SIMT_STORE, 0, 0, st));
+            TSR_KERNEL(ctx, 1, simt_gemm(r, r, r, b.Ra, TSR_F32, r, 1, b.p.M, r, 1, b.Rt, r, SIMT_STORE, 0, 0, st));
+            TSR_KERNEL(ctx, 1, simt_gemm(r, r, r, b.Rt, TSR_F32, r, 1, b.Rb, r, 1, b.p.M, r, SIMT_STORE, 0, 0, st));
+        }
     return do_shadows(ctx, list, st);
 }
 
@@ -601,12 +626,12 @@ tsr_status do_refresh_group(tsr_ctx *ctx, const std::vector<int> &list, uint64_t
 // of consecutive blocks (in tile-table order) that run concurrently on the context's side streams;
 // the caller's stream forks into them and joins afterwards, so the call keeps stream semantics.
 tsr_status do_refresh(tsr_ctx *ctx, const std::vector<int> &list, uint64_t seed, const float *const *omegas,
-                      cudaStream_t st)
+                      cudaStream_t st, bool reexpress)
 {
     if (list.empty()) return TSR_OK;
     const size_t zero[5] = {0, 0, 0, 0, 0};
     int ngroup = std::min<int>(tsr_ctx::NGROUP, (int)list.size() / 8);
-    if (!ctx->aux_ready || ngroup < 2) return do_refresh_group(ctx, list, seed, omegas, st, 0, zero);
+    if (!ctx->aux_ready || ngroup < 2) return do_refresh_group(ctx, list, seed, omegas, st, 0, zero, reexpress);
     // order the listed blocks as the tile tables do, remembering each one's omega
     std::vector<int> pos(ctx->blocks.size(), 0);
     for (size_t i = 0; i < ctx->order.size(); ++i) pos[ctx->order[i]] = (int)i;
@@ -622,7 +647,7 @@ tsr_status do_refresh(tsr_ctx *ctx, const std::vector<int> &list, uint64_t seed,
         std::vector<const float *> om;
         for (size_t i = lo; i < hi; ++i) { grp.push_back(list[perm[i]]); om.push_back(omegas ? omegas[perm[i]] : nullptr); }
         TSR_CUDA(ctx, cudaStreamWaitEvent(ctx->aux[g], ctx->ev_fork, 0));
-        tsr_status s = do_refresh_group(ctx, grp, seed, omegas ? om.data() : nullptr, ctx->aux[g], list_off, item_off);
+        tsr_status s = do_refresh_group(ctx, grp, seed, omegas ? om.data() : nullptr, ctx->aux[g], list_off, item_off, reexpress);
         if (s != TSR_OK && result == TSR_OK) result = s;
         TSR_CUDA(ctx, cudaEventRecord(ctx->ev_join[g], ctx->aux[g]));
         TSR_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_join[g], 0));
@@ -667,7 +692,7 @@ tsr_status do_step(tsr_ctx *ctx, const std::vector<int> &list, const tsr_hyper *
         for (int q : qs) {
             std::vector<int> grp;
             for (int bi : due) if (ctx->blocks[bi].d.q == q) grp.push_back(bi);
-            if ((s = do_refresh(ctx, grp, seed ^ ((uint64_t)h->step * 0x9E3779B97F4A7C15ull), nullptr, st)) != TSR_OK) return s;
+            if ((s = do_refresh(ctx, grp, seed ^ ((uint64_t)h->step * 0x9E3779B97F4A7C15ull), nullptr, st, true)) != TSR_OK) return s;
         }
     }
     const StepScalars sc = make_scalars(h);
@@ -730,7 +755,7 @@ tsr_status tsr_create(tsr_ctx **out, const tsr_mat_desc *descs, int32_t count)
         if (d.m > 0x3fffffff || d.n > 0x3fffffff || d.r + d.p > 1056) return TSR_ERR_SHAPE;
         if (d.g_dtype != TSR_F32 && d.g_dtype != TSR_BF16) return TSR_ERR_UNSUPPORTED;
         if (d.w_dtype != TSR_F32) return TSR_ERR_UNSUPPORTED;
-        if (d.reserved != 0 || (d.is_embedding != 0 && d.is_embedding != 1)) return TSR_ERR_INVALID_ARG;
+        if ((d.flags & ~(int32_t)TSR_BLOCK_REEXPRESS_MOMENT) != 0 || (d.is_embedding != 0 && d.is_embedding != 1)) return TSR_ERR_INVALID_ARG;
     }
     tsr_ctx *ctx = new (std::nothrow) tsr_ctx;
     if (!ctx) return TSR_ERR_INVALID_ARG;
@@ -947,6 +972,9 @@ tsr_status tsr_bases_changed(tsr_ctx *ctx, const int32_t *idx, int32_t count, vo
     return do_shadows(ctx, list, (cudaStream_t)stream);
 }
 
+static tsr_status refresh_listed(tsr_ctx *ctx, const int32_t *idx, int32_t count, uint64_t seed,
+                                 const float *const *omegas, void *stream, bool reexpress);
+
 // ---- grouped calls ------------------------------------------------------------------------
 tsr_status tsr_init_subspace_grouped(tsr_ctx *ctx, const int32_t *idx, int32_t count, uint64_t seed,
                                      const float *const *omegas, void *stream)
@@ -956,11 +984,11 @@ tsr_status tsr_init_subspace_grouped(tsr_ctx *ctx, const int32_t *idx, int32_t c
     std::vector<int> list;
     if ((s = resolve_list(ctx, idx, count, list)) != TSR_OK) return s;
     if ((s = zero_moments(ctx, list, (cudaStream_t)stream)) != TSR_OK) return s;
-    return tsr_rsvd_refresh_grouped(ctx, idx, count, seed, omegas, stream);
+    return refresh_listed(ctx, idx, count, seed, omegas, stream, false);   // moments are zero: nothing to re-express
 }
 
-tsr_status tsr_rsvd_refresh_grouped(tsr_ctx *ctx, const int32_t *idx, int32_t count, uint64_t seed,
-                                    const float *const *omegas, void *stream)
+static tsr_status refresh_listed(tsr_ctx *ctx, const int32_t *idx, int32_t count, uint64_t seed,
+                                 const float *const *omegas, void *stream, bool reexpress)
 {
     tsr_status s = check_ready(ctx);
     if (s != TSR_OK) return s;
@@ -974,9 +1002,15 @@ tsr_status tsr_rsvd_refresh_grouped(tsr_ctx *ctx, const int32_t *idx, int32_t co
         std::vector<const float *> om;
         for (size_t j = 0; j < list.size(); ++j)
             if (ctx->blocks[list[j]].d.q == q) { grp.push_back(list[j]); om.push_back(omegas ? omegas[j] : nullptr); }
-        if ((s = do_refresh(ctx, grp, seed, omegas ? om.data() : nullptr, (cudaStream_t)stream)) != TSR_OK) return s;
+        if ((s = do_refresh(ctx, grp, seed, omegas ? om.data() : nullptr, (cudaStream_t)stream, reexpress)) != TSR_OK) return s;
     }
     return TSR_OK;
+}
+
+tsr_status tsr_rsvd_refresh_grouped(tsr_ctx *ctx, const int32_t *idx, int32_t count, uint64_t seed,
+                                    const float *const *omegas, void *stream)
+{
+    return refresh_listed(ctx, idx, count, seed, omegas, stream, true);
 }
 
 tsr_status tsr_project_core_grouped(tsr_ctx *ctx, const int32_t *idx, int32_t count, void *stream)

@@ -182,3 +182,34 @@ def test_dense_adamw_matches_oracle():
                 assert rel_fro(to64(P[i]), Po[i]) < 1e-6 and rel_fro(to64(M[i]), Mo[i]) < 1e-6 and rel_fro(to64(V[i]), Vo[i]) < 1e-6
     with pytest.raises(tsr.TsrError):
         tsr.dense_adamw(P[:1], G[:1], M[:1], V[:1], tsr.make_hyper(1, rule=1))
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_optional_moment_reexpression_at_refresh(dtype):
+    """TSR_BLOCK_REEXPRESS_MOMENT: M' = Unew^T (Uold M Vold^T) Vnew at an explicit refresh; the
+    unflagged neighbour keeps Algorithm 1's behaviour (M untouched)."""
+    tsr = _tsr()
+    base = dict(m=192, n=256, r=24, p=8, q=1)
+    plan = tsr.Plan([dict(base, flags=tsr.TSR_BLOCK_REEXPRESS_MOMENT), dict(base)], g_dtype=dtype)
+    for i in range(2):
+        fill_gradient(plan, i, 300 + i, signal_rank=12)
+        fill_weights(plan, i, 310 + i)
+    plan.init_subspace(seed=3)
+    for t in (1, 2):
+        for i in range(2):
+            fill_gradient(plan, i, 320 + 10 * t + i, signal_rank=12)
+        plan.step(tsr.make_hyper(t))
+    torch.cuda.synchronize()
+    Uo, Vo, Mo = [to64(plan.U[i]) for i in range(2)], [to64(plan.V[i]) for i in range(2)], [to64(plan.M[i]) for i in range(2)]
+    Vm_before = plan.Vm[0].clone()
+    for i in range(2):
+        fill_gradient(plan, i, 390 + i, signal_rank=12)
+    plan.rsvd_refresh(seed=4)
+    torch.cuda.synchronize()
+    assert plan.poll_status() == [0, 0]
+    M_expect = Mo[0].copy()
+    oracle.reexpress_moment(M_expect, Uo[0], Vo[0], to64(plan.U[0]), to64(plan.V[0]))
+    assert rel_fro(to64(plan.M[0]), M_expect) < 1e-5
+    assert rel_fro(to64(plan.M[0]), Mo[0]) > 1e-2            # it did change
+    assert torch.equal(plan.Vm[0], Vm_before)                # the second moment is never re-expressed
+    assert np.array_equal(to64(plan.M[1]), Mo[1])            # unflagged block: Algorithm 1 as printed

@@ -61,6 +61,21 @@ def test_create_validates_shapes(tsr):
     assert tsr.lib().tsr_create(None, None, 0) == 1
 
 
+def test_block_flags_are_validated_and_sized(tsr):
+    D = tsr.MatDesc
+    rc, ctx = _create(tsr, [D(64, 64, 64, 64, 8, 0, 0, 0, 0, 0, 0, 2)])          # unknown flag bit
+    assert rc == 1
+    sizes = []
+    for flags in (0, tsr.TSR_BLOCK_REEXPRESS_MOMENT):
+        rc, ctx = _create(tsr, [D(256, 320, 320, 320, 32, 8, 1, 0, 0, 0, 0, flags)])
+        assert rc == 0
+        sb, rb = ctypes.c_size_t(), ctypes.c_size_t()
+        tsr.lib().tsr_workspace_bytes(ctx, ctypes.byref(sb), ctypes.byref(rb))
+        sizes.append(rb.value)
+        tsr.lib().tsr_destroy(ctx)
+    assert sizes[1] - sizes[0] >= 4 * ((256 + 320) * 32 + 3 * 32 * 32)             # old bases + three r x r scratch
+
+
 def test_compute_before_bind_is_refused(tsr):
     rc, ctx = _create(tsr, [tsr.MatDesc(64, 64, 64, 64, 8, 0, 0, 0, 0, 0, 0, 0)])
     assert rc == 0

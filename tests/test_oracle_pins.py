@@ -331,6 +331,26 @@ def test_step_refreshes_before_projecting_and_keeps_moments():
     assert np.allclose(blk.M, 0.9 * M_before + 0.1 * blk.C, atol=1e-14)
 
 
+def test_moment_reexpression_is_the_double_projection():
+    m, n, r = 18, 25, 4
+    rng = np.random.default_rng(70)
+    Uo, Vo, Un, Vn = _rand_orth(m, r, 71), _rand_orth(n, r, 72), _rand_orth(m, r, 73), _rand_orth(n, r, 74)
+    M0 = rng.standard_normal((r, r))
+    M = M0.copy()
+    oracle.reexpress_moment(M, Uo, Vo, Un, Vn)
+    lifted_old = Uo @ M0 @ Vo.T
+    # the new lifted moment is the old one projected onto the new subspaces from both sides
+    assert np.abs(Un @ M @ Vn.T - _proj(Un) @ lifted_old @ _proj(Vn)).max() < 1e-13
+    # unchanged subspaces, rotated bases: M' = Ru^T M Rv; identical bases: M' = M
+    Ru, Rv = _rand_orth(r, r, 75), _rand_orth(r, r, 76)
+    M = M0.copy()
+    oracle.reexpress_moment(M, Uo, Vo, Uo @ Ru, Vo @ Rv)
+    assert np.abs(M - Ru.T @ M0 @ Rv).max() < 1e-13
+    M = M0.copy()
+    oracle.reexpress_moment(M, Uo, Vo, Uo, Vo)
+    assert np.abs(M - M0).max() < 1e-13
+
+
 # ---- byte and state accounting against the numbers the paper prints ---------------------
 def _golden_rows():
     rows = []
