@@ -251,7 +251,9 @@ void build_tiles(tsr_ctx *ctx)
     for (int kd = 0; kd < NKIND; ++kd) ctx->tiles[kd].clear();
     int rmax = 0;
     for (const Block &b : ctx->blocks) if (b.fast) rmax = std::max(rmax, (int)b.d.r);
-    for (int kd : {KT, KC, KCS, KP}) ctx->bn[kd] = rmax >= 256 ? 256 : 128;
+    for (int kd : {KT, KP}) ctx->bn[kd] = rmax >= 256 ? 256 : 128;
+    // the core GEMM has few, long tiles: 256-wide tiles only pay once r reaches 512 (measured)
+    for (int kd : {KC, KCS}) ctx->bn[kd] = rmax >= 512 ? 256 : 128;
     for (int bi : ctx->order) {
         Block &b = ctx->blocks[bi];
         for (int kd = 0; kd < NKIND; ++kd) b.tile_begin[kd] = b.tile_end[kd] = (int)ctx->tiles[kd].size();
