@@ -228,12 +228,13 @@ void layout(tsr_ctx *ctx, Arena &a, bool assign, size_t *step_end)
 void add_tiles(tsr_ctx *ctx, int kind, int bi, int M, int N, int K, int kb_per_split)
 {
     const int bn = ctx->bn[kind];
+    const int bm = (kind == KA) ? 128 : 256;   // the grouped GEMM runs on CTA pairs: 256-row tiles
     Block &b = ctx->blocks[bi];
     std::vector<UmmaTile> &v = ctx->tiles[kind];
     b.tile_begin[kind] = (int)v.size();
     const int nkb = (K + 63) / 64;
     const int nsp = kb_per_split > 0 ? (nkb + kb_per_split - 1) / kb_per_split : 1;
-    for (int m0 = 0; m0 < M; m0 += 128)
+    for (int m0 = 0; m0 < M; m0 += bm)
         for (int n0 = 0; n0 < N; n0 += bn)
             for (int s = 0; s < nsp; ++s) {
                 UmmaTile t;
@@ -898,14 +899,14 @@ tsr_status tsr_bind(tsr_ctx *ctx, const tsr_mat_ptrs *ptrs, int32_t count, void 
             UmmaProblem &P = probs[KT][i];
             base(P, (int)m, (int)r, (int)n, EPI_STORE_BF16_T);
             if ((s = encode_map(ctx, &P.tmA, b.p.G, m, n, b.d.ldg, 128)) != TSR_OK) return s;
-            if ((s = encode_map(ctx, &P.tmB, b.Vbt, r, n, b.nl, ctx->bn[KT])) != TSR_OK) return s;
+            if ((s = encode_map(ctx, &P.tmB, b.Vbt, r, n, b.nl, ctx->bn[KT] / 2)) != TSR_OK) return s;
             P.out = b.Tt; P.ld_out = b.ml;
         }
         for (int kd : {KC, KCS}) {   // C = U^T T : A = U^T copy [r x m], B = T~ [r x m]
             UmmaProblem &P = probs[kd][i];
             base(P, (int)r, (int)r, (int)m, EPI_CORE_UPDATE);
             if ((s = encode_map(ctx, &P.tmA, b.Ubt, r, m, b.ml, 128)) != TSR_OK) return s;
-            if ((s = encode_map(ctx, &P.tmB, b.Tt, r, m, b.ml, ctx->bn[kd])) != TSR_OK) return s;
+            if ((s = encode_map(ctx, &P.tmB, b.Tt, r, m, b.ml, ctx->bn[kd] / 2)) != TSR_OK) return s;
             P.out = (kd == KC) ? (void *)b.p.C : (void *)b.partial;
             P.ld_out = r; P.split_stride = r * r;
             P.mom1 = b.p.M; P.mom2 = b.p.Vm; P.d_bf16 = nullptr; P.dt_bf16 = b.Dbt; P.ldd = b.rl;
@@ -914,7 +915,7 @@ tsr_status tsr_bind(tsr_ctx *ctx, const tsr_mat_ptrs *ptrs, int32_t count, void 
             UmmaProblem &P = probs[KP][i];
             base(P, (int)m, (int)r, (int)r, EPI_STORE_BF16);
             if ((s = encode_map(ctx, &P.tmA, b.Ub, m, r, b.rl, 128)) != TSR_OK) return s;
-            if ((s = encode_map(ctx, &P.tmB, b.Dbt, r, r, b.rl, ctx->bn[KP])) != TSR_OK) return s;
+            if ((s = encode_map(ctx, &P.tmB, b.Dbt, r, r, b.rl, ctx->bn[KP] / 2)) != TSR_OK) return s;
             P.out = b.Pb; P.ld_out = b.rl;
         }
         {   // W update : A = P [m x r], B = V copy [n x r]
@@ -930,7 +931,7 @@ tsr_status tsr_bind(tsr_ctx *ctx, const tsr_mat_ptrs *ptrs, int32_t count, void 
             base(P, (int)m, (int)k, (int)n, EPI_STORE_F32);
             P.planes = 2; P.plane_rows = (int)k;
             if ((s = encode_map(ctx, &P.tmA, b.p.G, m, n, b.d.ldg, 128)) != TSR_OK) return s;
-            if ((s = encode_map(ctx, &P.tmB, b.Xt, 2 * k, n, b.nl, 128)) != TSR_OK) return s;
+            if ((s = encode_map(ctx, &P.tmB, b.Xt, 2 * k, n, b.nl, 64)) != TSR_OK) return s;
             P.out = b.buf[0]; P.ld_out = k;
         }
         {   // Z = G^T X : A = G^T copy [n x m], B = X^T planes [2k x m]
@@ -938,7 +939,7 @@ tsr_status tsr_bind(tsr_ctx *ctx, const tsr_mat_ptrs *ptrs, int32_t count, void 
             base(P, (int)n, (int)k, (int)m, EPI_STORE_F32);
             P.planes = 2; P.plane_rows = (int)k;
             if ((s = encode_map(ctx, &P.tmA, b.Gt, n, m, b.ml, 128)) != TSR_OK) return s;
-            if ((s = encode_map(ctx, &P.tmB, b.Xt, 2 * k, m, b.ml, 128)) != TSR_OK) return s;
+            if ((s = encode_map(ctx, &P.tmB, b.Xt, 2 * k, m, b.ml, 64)) != TSR_OK) return s;
             P.out = b.buf[0]; P.ld_out = k;
         }
     }

@@ -34,7 +34,7 @@ constexpr int UG_EPI_WARPS = 8;
 template <int BN, int PLANES>
 struct UmmaSmem {
     static constexpr int A_BYTES = UM_BM * UM_BK * 2;
-    static constexpr int B_BYTES = BN * UM_BK * 2;
+    static constexpr int B_BYTES = (BN / 2) * UM_BK * 2;   // each CTA of the pair stages half of the B rows
     static constexpr int STAGE_BYTES = A_BYTES + PLANES * B_BYTES;
     static constexpr int STAGES = (192 * 1024) / STAGE_BYTES > 6 ? 6 : (192 * 1024) / STAGE_BYTES;
     static constexpr int PATCH_OFFSET = STAGES * STAGE_BYTES;
@@ -45,7 +45,7 @@ struct UmmaSmem {
 };
 
 template <int BN, int EPI, int PLANES>
-__global__ void __launch_bounds__(UG_THREADS, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(UG_THREADS, 1)
 umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restrict__ tiles, int num_tiles,
                  StepScalars sc, int32_t *__restrict__ status)
 {
@@ -62,22 +62,25 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
     __shared__ int s_timeout;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int stride = gridDim.x;
+    const uint32_t rank = cluster_ctarank();          // 0 = leader of the CTA pair
+    const int pair = blockIdx.x >> 1;
+    const int stride = gridDim.x >> 1;
 
     if (threadIdx.x == 0) {
         s_timeout = 0;
         for (int s = 0; s < STAGES; ++s) { mbar_init(smem_u32(bar_full + s), 1); mbar_init(smem_u32(bar_empty + s), 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(bar_acc_full + b), 1); mbar_init(smem_u32(bar_acc_empty + b), UG_EPI_WARPS); }
+        for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(bar_acc_full + b), 1); mbar_init(smem_u32(bar_acc_empty + b), 2 * UG_EPI_WARPS); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+    if (warp == 1) {   // the same warp of both CTAs allocates the pair's tensor memory
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
                      "r"(TMEM_COLS)
                      : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
     __syncthreads();
+    cluster_sync();      // the peer's barriers are initialised before anything signals them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
@@ -85,33 +88,37 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
         if (lane == 0) {
             uint32_t it = 0;
             bool ok = true;
-            for (int t = blockIdx.x; t < num_tiles && ok; t += stride) {
+            for (int t = pair; t < num_tiles && ok; t += stride) {
                 const UmmaTile tile = tiles[t];
                 const UmmaProblem *P = probs + tile.prob;
+                int n_eff = P->N - tile.n0;
+                n_eff = n_eff >= BN ? BN : ((n_eff + 15) & ~15);
+                const int b_row = tile.n0 + (int)rank * (n_eff / 2);   // this CTA's half of the B rows
                 for (int kb = tile.kb0; kb < tile.kb1; ++kb, ++it) {
                     const int s = it % STAGES;
                     const uint32_t ph = (it / STAGES) & 1u;
                     if (!mbar_wait(smem_u32(bar_empty + s), ph ^ 1u)) { s_timeout = 1; ok = false; break; }
-                    const uint32_t full = smem_u32(bar_full + s);
-                    mbar_expect_tx(full, (uint32_t)SM::STAGE_BYTES);
+                    // both CTAs' copies report their bytes to the leader's "full" barrier
+                    const uint32_t full = leader_addr(smem_u32(bar_full + s));
+                    if (rank == 0) mbar_expect_tx(smem_u32(bar_full + s), 2u * (uint32_t)SM::STAGE_BYTES);
                     uint8_t *st = smem + s * SM::STAGE_BYTES;
-                    tma_load_2d(smem_u32(st), &P->tmA, full, kb * UM_BK, tile.m0);
+                    tma_load_2d_pair(smem_u32(st), &P->tmA, full, kb * UM_BK, tile.m0 + (int)rank * UM_BM);
 #pragma unroll
                     for (int pl = 0; pl < PLANES; ++pl)
-                        tma_load_2d(smem_u32(st + SM::A_BYTES + pl * SM::B_BYTES), &P->tmB, full, kb * UM_BK,
-                                    tile.n0 + pl * P->plane_rows);
+                        tma_load_2d_pair(smem_u32(st + SM::A_BYTES + pl * SM::B_BYTES), &P->tmB, full, kb * UM_BK,
+                                         b_row + pl * P->plane_rows);
                 }
             }
         }
     } else if (warp == 1) {
-        if (lane == 0) {
+        if (lane == 0 && rank == 0) {   // the leader issues the pair's MMAs (256 x N x 16 each)
             uint32_t it = 0, tc = 0;
             bool ok = true;
-            for (int t = blockIdx.x; t < num_tiles && ok; t += stride, ++tc) {
+            for (int t = pair; t < num_tiles && ok; t += stride, ++tc) {
                 const UmmaTile tile = tiles[t];
                 int n_eff = probs[tile.prob].N - tile.n0;
                 n_eff = n_eff >= BN ? BN : ((n_eff + 15) & ~15);
-                const uint32_t idesc = umma_idesc(n_eff);
+                const uint32_t idesc = umma_idesc_pair(n_eff);
                 const uint32_t buf = tc & 1u;
                 if (!mbar_wait(smem_u32(bar_acc_empty + buf), ((tc >> 1) & 1u) ^ 1u)) { s_timeout = 1; ok = false; break; }
                 tc_fence_after();
@@ -127,12 +134,12 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
                         const uint32_t b_base = a_base + SM::A_BYTES + pl * SM::B_BYTES;
 #pragma unroll
                         for (int k4 = 0; k4 < UM_BK / 16; ++k4)
-                            tc_mma_bf16(d_tmem, umma_desc_sw128(a_base + k4 * 32), umma_desc_sw128(b_base + k4 * 32),
-                                        idesc, ((kb - tile.kb0) | pl | k4) ? 1u : 0u);
+                            tc_mma_bf16_pair(d_tmem, umma_desc_sw128(a_base + k4 * 32), umma_desc_sw128(b_base + k4 * 32),
+                                             idesc, ((kb - tile.kb0) | pl | k4) ? 1u : 0u);
                     }
-                    tc_commit(smem_u32(bar_empty + s));
+                    tc_commit_pair(smem_u32(bar_empty + s));       // frees the stage in both CTAs
                 }
-                tc_commit(smem_u32(bar_acc_full + buf));
+                tc_commit_pair(smem_u32(bar_acc_full + buf));      // accumulator ready, in both CTAs
             }
         }
     } else if (warp >= 4) {
@@ -143,12 +150,12 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
         float *patch = (float *)(smem + SM::PATCH_OFFSET + (warp - 4) * SM::PATCH_BYTES);   // [32][33]
         uint32_t tc = 0;
         bool ok = true;
-        for (int t = blockIdx.x; t < num_tiles && ok; t += stride, ++tc) {
+        for (int t = pair; t < num_tiles && ok; t += stride, ++tc) {
             const UmmaTile tile = tiles[t];
             const UmmaProblem *__restrict__ P = probs + tile.prob;
             const uint32_t buf = tc & 1u;
             const int N = P->N, M = P->M;
-            const int row0 = tile.m0 + q * 32;
+            const int row0 = tile.m0 + (int)rank * UM_BM + q * 32;   // this CTA holds rows 128 rank .. of the tile
             if (EPI == EPI_CORE_UPDATE) {
                 // pull this warp's slice of the moments towards L2 while the MMAs of the tile run
                 const int prow = row0 + lane;
@@ -168,7 +175,7 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
             const int c_begin = half * (BN / 2), c_end = c_begin + BN / 2;
             if (tile.n0 + c_begin >= N) {   // this warp's column half lies outside the matrix
                 tc_fence_before();
-                if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar_acc_empty + buf)) : "memory");
+                if (lane == 0) mbar_arrive_leader(smem_u32(bar_acc_empty + buf));
                 continue;
             }
 #pragma unroll 1
@@ -179,7 +186,7 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
                 tc_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + buf * BN + (uint32_t)c0, v);
                 if (c0 + 32 >= c_end || col0 + 32 >= N) {   // this warp's last chunk of the tile: release the accumulator
                     tc_fence_before();
-                    if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar_acc_empty + buf)) : "memory");
+                    if (lane == 0) mbar_arrive_leader(smem_u32(bar_acc_empty + buf));
                 }
                 if (nrows <= 0) continue;
                 const int ncols = min(32, N - col0);
@@ -309,9 +316,10 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
     if (s_timeout) __nanosleep(2000000);   // let copies in flight land before the CTA goes away
     tc_fence_before();
     __syncthreads();
+    cluster_sync();      // neither CTA may leave while the peer still uses its shared or tensor memory
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
     }
     if (threadIdx.x == 0 && s_timeout && status) atomicMax(status, (int)TSR_ERR_TIMEOUT);
 }
@@ -321,8 +329,8 @@ static cudaError_t launch_one(const UmmaProblem *probs, const UmmaTile *tiles, i
                               const StepScalars &sc, int32_t *status, cudaStream_t stream)
 {
     using SM = UmmaSmem<BN, PLANES>;
-    const int grid = num_tiles < num_sms ? num_tiles : num_sms;
-    umma_gemm_kernel<BN, EPI, PLANES><<<grid, UG_THREADS, SM::TOTAL, stream>>>(probs, tiles, num_tiles, sc, status);
+    const int pairs = num_tiles < num_sms / 2 ? num_tiles : num_sms / 2;
+    umma_gemm_kernel<BN, EPI, PLANES><<<2 * pairs, UG_THREADS, SM::TOTAL, stream>>>(probs, tiles, num_tiles, sc, status);
     return cudaGetLastError();
 }
 
