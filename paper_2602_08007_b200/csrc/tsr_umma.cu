@@ -2,23 +2,32 @@
 //
 //   D[M x N] = A[M x K] * B[N x K]^T     A, B BF16 with K contiguous, FP32 accumulation
 //
-// One CTA per SM walks a device-resident tile table (tiles of all matrix blocks of a model
-// share one launch; static round-robin).  A tile is 128 x BN outputs over a range of 64-wide
-// K blocks.  Roles inside the CTA:
-//   warp 0    one lane issues the TMA loads (128-byte swizzled 64-wide K slices) into a ring of
-//             shared-memory stages and signals "full" mbarriers with the byte count;
-//   warp 1    allocates tensor memory (two accumulators of BN columns); one lane issues
-//             tcgen05.mma (128 x N x 16 per instruction, N = the tile's width rounded up to 16)
-//             from shared-memory descriptors and commits to the stage's "empty" mbarrier and,
-//             per tile, to the accumulator's "full" mbarrier.  The MMAs of tile i+1 overlap the
-//             epilogue of tile i;
+// The grid is one CTA per SM, grouped into clusters of two (a CTA pair).  Every pair walks a
+// device-resident tile table (tiles of all matrix blocks of a model share one launch; static
+// round-robin over pairs).  A tile is 256 x BN outputs over a range of 64-wide K blocks: CTA c of
+// the pair owns output rows 128 c .. 128 c + 127 and holds that half of the accumulator in its
+// own tensor memory.  Roles inside each CTA:
+//   warp 0    one lane issues the TMA loads (128-byte swizzled 64-wide K slices) of this CTA's
+//             128 rows of A and of HALF of the tile's B rows into a ring of shared-memory stages;
+//             the bytes of both CTAs complete on the LEADER's "full" mbarrier (its address is
+//             mapped into the peer with mapa), so each SM ingests only half of B per K block.
+//             No load uses cluster multicast;
+//   warp 1    allocates tensor memory (two accumulators of BN columns).  In the leader CTA one
+//             lane issues tcgen05.mma.cta_group::2 (256 x N x 16 per instruction, N = the tile's
+//             width rounded up to 16; it reads A and B halves from both CTAs' shared memory) and
+//             commits, multicast to both CTAs, to the stage's "empty" mbarrier and, per tile, to
+//             the accumulator's "full" mbarrier.  The MMAs of tile i+1 overlap the epilogue of
+//             tile i;
 //   warps 4-11 read the accumulator with tcgen05.ld (lane = output row, 32 columns at a time;
-//             warp e owns TMEM lanes 32 (e % 4).. and the column half e / 4 of the tile).
+//             warp e owns TMEM lanes 32 (e % 4).. and the column half (e - 4) / 4 of the tile) and
+//             release it by arriving on the leader's "accumulator empty" mbarrier.
 //             Epilogues: plain FP32 / BF16 stores (each lane writes whole 32-byte sectors of its
 //             own row), the transposed BF16 store, and the fused core update of Section 3.4,
 //             which goes through a warp-private shared-memory transpose so that its moment
 //             read-modify-write touches full 128-byte row segments, with the moment tiles
 //             prefetched to L2 while the tile's MMAs run.
+// A cluster barrier at entry orders barrier initialisation before remote arrivals, and one at
+// exit keeps either CTA from leaving while its peer still reads its shared or tensor memory.
 // Ragged edges rely on TMA zero fill for loads and on predicated stores.
 // Every mbarrier wait is bounded by a clock budget; on expiry the CTA records
 // TSR_ERR_TIMEOUT, stops storing and still releases its tensor memory before it exits.
