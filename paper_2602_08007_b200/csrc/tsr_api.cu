@@ -38,7 +38,7 @@ struct Block {
     float *Rinv = nullptr, *Wu = nullptr, *Wv = nullptr;
     double *tau = nullptr, *dvec = nullptr, *evec = nullptr;
     double2 *rot = nullptr;
-    int2 *sweeps = nullptr;
+    int2 *sweeps = nullptr, *groups = nullptr;
     int32_t *nsweeps = nullptr, *rank = nullptr;
     int rot_cap = 0, sweep_cap = 0;
     float *Uold = nullptr, *Vold = nullptr, *Ra = nullptr, *Rb = nullptr, *Rt = nullptr;   // moment re-expression
@@ -93,9 +93,9 @@ struct tsr_ctx {
     int stage_next = 0;
     // refresh runs as up to NGROUP independent groups of blocks on side streams, so that the
     // latency-bound small-matrix kernels of one group overlap the GEMM-like kernels of another
-    static constexpr int NGROUP = 4;
+    static constexpr int NGROUP = 8;
     cudaStream_t aux[NGROUP] = {};
-    cudaEvent_t ev_fork = nullptr, ev_join[NGROUP] = {};
+    cudaEvent_t ev_fork = nullptr, ev_join[NGROUP] = {}, ev_stagger[NGROUP] = {};
     bool aux_ready = false;
 };
 
@@ -202,13 +202,14 @@ void layout(tsr_ctx *ctx, Arena &a, bool assign, size_t *step_end)
         void *gp = a.take((size_t)gram_chunks(mx) * k * k * 8);
         void *lam = a.take((size_t)k * 8);
         void *ri = a.take((size_t)(k * k) * 4), *wu = a.take((size_t)(k * r) * 4), *wv = a.take((size_t)(k * r) * 4);
-        const int rot_cap = (int)std::min<int64_t>(3 * k * k + 64, 0x7fffffff), sweep_cap = (int)(64 * k);
+        const int rot_cap = (int)std::min<int64_t>(eig_rot_capacity((int)k), 0x7fffffff), sweep_cap = (int)(64 * k);
         void *tau = a.take((size_t)k * 8), *dv = a.take((size_t)k * 8), *ev = a.take((size_t)k * 8);
         void *rot = a.take((size_t)rot_cap * 16), *sw = a.take((size_t)sweep_cap * 8);
+        void *grp = a.take((size_t)(sweep_cap / 32 + 1) * 8);
         void *nsw = a.take(4), *rk = a.take((size_t)k * 4);
         if (assign) {
             b.tau = (double *)tau; b.dvec = (double *)dv; b.evec = (double *)ev; b.rot = (double2 *)rot;
-            b.sweeps = (int2 *)sw; b.nsweeps = (int32_t *)nsw; b.rank = (int32_t *)rk;
+            b.sweeps = (int2 *)sw; b.groups = (int2 *)grp; b.nsweeps = (int32_t *)nsw; b.rank = (int32_t *)rk;
             b.rot_cap = rot_cap; b.sweep_cap = sweep_cap;
         }
         if (b.d.flags & TSR_BLOCK_REEXPRESS_MOMENT) {
@@ -539,7 +540,8 @@ tsr_status sketch(tsr_ctx *ctx, const RefreshLists &L, bool transposed, bool fro
 // One group of blocks through the whole refresh on stream st.  list_off / item_off: where this
 // group's slices start inside the context's device list / item tables.
 tsr_status do_refresh_group(tsr_ctx *ctx, const std::vector<int> &list, uint64_t seed, const float *const *omegas,
-                            cudaStream_t st, size_t list_off, const size_t *item_off, bool reexpress)
+                            cudaStream_t st, size_t list_off, const size_t *item_off, bool reexpress,
+                            cudaEvent_t started = nullptr)
 {
     if (list.empty()) return TSR_OK;
     tsr_status s;
@@ -581,6 +583,7 @@ tsr_status do_refresh_group(tsr_ctx *ctx, const std::vector<int> &list, uint64_t
     // Y = G Omega; Q = orth(Y)
     if ((s = sketch(ctx, L, false, true, omegas, st)) != TSR_OK) return s;
     if ((s = orth(ctx, L, 0, qmax == 0, st)) != TSR_OK) return s;
+    if (started) TSR_CUDA(ctx, cudaEventRecord(started, st));   // the next group may start now (see do_refresh)
     for (int it = 0; it < qmax; ++it) {
         // Yrow = G^T Q; Qrow = orth(Yrow); Y = G Qrow; Q = orth(Y)
         if ((s = sketch(ctx, L, true, false, nullptr, st)) != TSR_OK) return s;
@@ -633,7 +636,8 @@ tsr_status do_refresh(tsr_ctx *ctx, const std::vector<int> &list, uint64_t seed,
 {
     if (list.empty()) return TSR_OK;
     const size_t zero[5] = {0, 0, 0, 0, 0};
-    int ngroup = std::min<int>(tsr_ctx::NGROUP, (int)list.size() / 8);
+    static const int ng_env = getenv("TSR_NGROUP") ? atoi(getenv("TSR_NGROUP")) : 4;   // EXPERIMENT
+    int ngroup = std::min<int>(std::min<int>(ng_env, tsr_ctx::NGROUP), (int)list.size() / 8);
     if (!ctx->aux_ready || ngroup < 2) return do_refresh_group(ctx, list, seed, omegas, st, 0, zero, reexpress);
     // order the listed blocks as the tile tables do, remembering each one's omega
     std::vector<int> pos(ctx->blocks.size(), 0);
@@ -650,7 +654,13 @@ tsr_status do_refresh(tsr_ctx *ctx, const std::vector<int> &list, uint64_t seed,
         std::vector<const float *> om;
         for (size_t i = lo; i < hi; ++i) { grp.push_back(list[perm[i]]); om.push_back(omegas ? omegas[perm[i]] : nullptr); }
         TSR_CUDA(ctx, cudaStreamWaitEvent(ctx->aux[g], ctx->ev_fork, 0));
-        tsr_status s = do_refresh_group(ctx, grp, seed, omegas ? om.data() : nullptr, ctx->aux[g], list_off, item_off, reexpress);
+        // Groups start one orthonormalisation apart: in lock-step all groups would sit in the same
+        // one-CTA-per-matrix kernel at the same time (more CTAs than SMs, two waves) and leave the
+        // SMs idle that the throughput-bound kernels of another group could use.
+        static const int stag_env = getenv("TSR_STAGGER") ? atoi(getenv("TSR_STAGGER")) : 1;   // EXPERIMENT
+        if (g > 0 && stag_env) TSR_CUDA(ctx, cudaStreamWaitEvent(ctx->aux[g], ctx->ev_stagger[g - 1], 0));
+        tsr_status s = do_refresh_group(ctx, grp, seed, omegas ? om.data() : nullptr, ctx->aux[g], list_off, item_off,
+                                        reexpress, ctx->ev_stagger[g]);
         if (s != TSR_OK && result == TSR_OK) result = s;
         TSR_CUDA(ctx, cudaEventRecord(ctx->ev_join[g], ctx->aux[g]));
         TSR_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_join[g], 0));
@@ -797,7 +807,7 @@ tsr_status tsr_destroy(tsr_ctx *ctx)
     if (ctx->profiling)
         for (cudaEvent_t e : ctx->ev) if (e) cudaEventDestroy(e);
     if (ctx->aux_ready) {
-        for (int g = 0; g < tsr_ctx::NGROUP; ++g) { cudaStreamDestroy(ctx->aux[g]); cudaEventDestroy(ctx->ev_join[g]); }
+        for (int g = 0; g < tsr_ctx::NGROUP; ++g) { cudaStreamDestroy(ctx->aux[g]); cudaEventDestroy(ctx->ev_join[g]); cudaEventDestroy(ctx->ev_stagger[g]); }
         cudaEventDestroy(ctx->ev_fork);
     }
     delete ctx;
@@ -889,7 +899,7 @@ tsr_status tsr_bind(tsr_ctx *ctx, const tsr_mat_ptrs *ptrs, int32_t count, void 
         for (int j = 0; j < 3; ++j) rd.buf[j] = b.buf[j];
         rd.S = b.S; rd.Xw = b.Xw; rd.Wj = b.Wj; rd.gpart = b.gpart; rd.lam = b.lam;
         rd.Rinv = b.Rinv; rd.Wu = b.Wu; rd.Wv = b.Wv; rd.U = b.p.U; rd.V = b.p.V; rd.status = ctx->d_status + i;
-        rd.tau = b.tau; rd.dvec = b.dvec; rd.evec = b.evec; rd.rot = b.rot; rd.sweeps = b.sweeps; rd.nsweeps = b.nsweeps;
+        rd.tau = b.tau; rd.dvec = b.dvec; rd.evec = b.evec; rd.rot = b.rot; rd.sweeps = b.sweeps; rd.groups = b.groups; rd.nsweeps = b.nsweeps;
         rd.rank = b.rank; rd.rot_cap = b.rot_cap; rd.sweep_cap = b.sweep_cap;
         if (!b.fast) continue;
         auto base = [&](UmmaProblem &P, int M, int N, int K, int epi) {
@@ -957,6 +967,7 @@ tsr_status tsr_bind(tsr_ctx *ctx, const tsr_mat_ptrs *ptrs, int32_t count, void 
         for (int g = 0; g < tsr_ctx::NGROUP; ++g) {
             TSR_CUDA(ctx, cudaStreamCreateWithFlags(&ctx->aux[g], cudaStreamNonBlocking));
             TSR_CUDA(ctx, cudaEventCreateWithFlags(&ctx->ev_join[g], cudaEventDisableTiming));
+            TSR_CUDA(ctx, cudaEventCreateWithFlags(&ctx->ev_stagger[g], cudaEventDisableTiming));
         }
         TSR_CUDA(ctx, cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming));
         ctx->aux_ready = true;

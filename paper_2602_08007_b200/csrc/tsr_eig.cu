@@ -108,6 +108,20 @@ tridiag_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ li
 // ---- stage 2: implicit QL on the tridiagonal matrix, logging the rotations ------------------
 // e[i] couples d[i] and d[i+1].  Sweep header: x = index of the first rotation (m - 1), y = count;
 // rotation t of a sweep acts on columns (x - t, x - t + 1).
+//
+// Two log layouts.  SKEW = false: rotations in the order they are generated.  SKEW = true: the
+// layout the systolic eigenvector kernel reads.  Sweeps are taken in groups of 32 (sweep s is lane
+// s % 32 of group s / 32).  A group streams the columns k-1, k-2, ..., lg of a row through the 32
+// lanes, lane t two steps behind lane t-1, so lane t meets column j at step (k-1-j) + 2t; the
+// rotation of sweep t on columns (j, j+1) is stored at rot[(base + (k-1-j) + 2t) * 32 + t], i.e. the
+// 32 rotations a warp needs at one step are contiguous.  lg is the l of the group's first sweep
+// (l never decreases).  groups[g] = (base row, E = k - lg + 1 stream elements); entries that no
+// sweep writes are never used (the reader tests each lane's column against its sweep's range).
+constexpr int SYS_LAG = 2;                        // steps between neighbouring lanes
+constexpr int SYS_FILL = SYS_LAG * 31;            // steps until the last lane sees the first column
+constexpr int SYS_PF = 8;                         // steps of rotations the reader fetches ahead
+
+template <bool SKEW>
 __global__ void __launch_bounds__(32)
 ql_log_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ list)
 {
@@ -120,7 +134,10 @@ ql_log_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ lis
     if (threadIdx.x == 0) {
         double2 *__restrict__ rot = D.rot;
         int2 *__restrict__ sweeps = D.sweeps;
+        int2 *__restrict__ groups = D.groups;
         int nrot = 0, nsw = 0;
+        int64_t next_row = 0;                     // SKEW: first free row of the skewed log
+        double2 *lane_rot = rot;                  // SKEW: rot + (base * 32 + t) + 32 * SYS_LAG * t
         bool failed = false;
         for (int l = 0; l < n && !failed; ++l) {
             int iter = 0;
@@ -131,7 +148,18 @@ ql_log_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ lis
                     if (fabs(e[m]) <= 2.3e-16 * dd) break;
                 }
                 if (m == l) break;
-                if (++iter > 60 || nsw >= D.sweep_cap || nrot + (m - l) > D.rot_cap) { failed = true; break; }
+                if (++iter > 60 || nsw >= D.sweep_cap) { failed = true; break; }
+                if (SKEW) {
+                    const int t = nsw & 31;
+                    if (t == 0) {                 // a new group starts with this sweep
+                        const int E = n - l + 1;
+                        if ((next_row + E + SYS_FILL + 2 * SYS_PF) * 32 > (int64_t)D.rot_cap) { failed = true; break; }
+                        groups[nsw >> 5] = make_int2((int)next_row, E);
+                        next_row += E + SYS_FILL;
+                    }
+                    const int2 gr = groups[nsw >> 5];
+                    lane_rot = rot + ((int64_t)gr.x + SYS_LAG * t) * 32 + t;
+                } else if (nrot + (m - l) > D.rot_cap) { failed = true; break; }
                 double g = (d[l + 1] - d[l]) / (2.0 * e[l]);
                 double r = sqrt(g * g + 1.0);
                 g = d[m] - d[l] + e[l] / (g + (g >= 0.0 ? r : -r));
@@ -156,7 +184,8 @@ ql_log_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ lis
                     p = s * r;
                     d[i + 1] = g + p;
                     g = c * r - b;
-                    rot[nrot++] = make_double2(c, s);
+                    if (SKEW) { lane_rot[(int64_t)(n - 1 - i) * 32] = make_double2(c, s); ++nrot; }
+                    else rot[nrot++] = make_double2(c, s);
                 }
                 if (nrot > first) sweeps[nsw++] = make_int2(m - 1, nrot - first);
                 if (early) continue;
@@ -309,13 +338,205 @@ __global__ void eig_rank_kernel(const RefreshDev *__restrict__ rd, const int32_t
     if (flag) atomicMax(D.status, flag);
 }
 
+// ---- stage 3, systolic form (k <= SYS_KMAX) ---------------------------------------------------
+// 3a: rows of Q = H_0 H_1 ... in registers.  A warp owns RQ rows; lane holds columns lane + 32 i.
+// The reflectors are staged for the whole CTA, a few at a time, in shared memory.
+constexpr int SYS_KMAX = 1056;
+constexpr int SYS_WARPS = 8;
+
+template <int NCH, int RQ>
+__global__ void __launch_bounds__(SYS_WARPS * 32)
+eig_qrows_kernel(const RefreshDev *__restrict__ rd, const RowItem *__restrict__ items)
+{
+    constexpr int LD = NCH * 32;
+    constexpr int QV_BATCH = NCH > 17 ? 4 : 8;    // reflectors staged per round (static shared memory <= 48 KB)
+    __shared__ double vs[QV_BATCH][LD];
+    __shared__ double taus[QV_BATCH];
+    const RowItem it = items[blockIdx.x];
+    const RefreshDev D = rd[it.block];
+    const int k = D.k;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int row0 = it.row0 + warp * RQ;
+    const double *__restrict__ A = D.S;
+    double x[RQ][NCH];
+#pragma unroll
+    for (int q = 0; q < RQ; ++q)
+#pragma unroll
+        for (int i = 0; i < NCH; ++i) x[q][i] = (lane + 32 * i == row0 + q) ? 1.0 : 0.0;
+
+    for (int j0 = 0; j0 + 2 < k; j0 += QV_BATCH) {
+        __syncthreads();
+        for (int idx = threadIdx.x; idx < QV_BATCH * LD; idx += SYS_WARPS * 32) {
+            const int b = idx / LD, c = idx - b * LD, j = j0 + b;
+            double v = 0.0;
+            if (j + 2 < k && c < k) v = (c == j + 1) ? 1.0 : (c >= j + 2 ? A[(int64_t)j * k + c] : 0.0);
+            vs[b][c] = v;
+        }
+        if (threadIdx.x < QV_BATCH) taus[threadIdx.x] = (j0 + threadIdx.x + 2 < k) ? D.tau[j0 + threadIdx.x] : 0.0;
+        __syncthreads();
+#pragma unroll 1
+        for (int b = 0; b < QV_BATCH; ++b) {
+            const double tau = taus[b];
+            if (tau == 0.0) continue;
+            const int i0 = (j0 + b + 1) >> 5;     // chunks below hold only zeros of v
+            double dot[RQ];
+#pragma unroll
+            for (int q = 0; q < RQ; ++q) dot[q] = 0.0;
+#pragma unroll
+            for (int i = 0; i < NCH; ++i)
+                if (i >= i0) {
+                    const double v = vs[b][lane + 32 * i];
+#pragma unroll
+                    for (int q = 0; q < RQ; ++q) dot[q] += x[q][i] * v;
+                }
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1)
+#pragma unroll
+                for (int q = 0; q < RQ; ++q) dot[q] += __shfl_xor_sync(0xffffffffu, dot[q], off);
+#pragma unroll
+            for (int q = 0; q < RQ; ++q) dot[q] *= tau;
+#pragma unroll
+            for (int i = 0; i < NCH; ++i)
+                if (i >= i0) {
+                    const double v = vs[b][lane + 32 * i];
+#pragma unroll
+                    for (int q = 0; q < RQ; ++q) x[q][i] -= dot[q] * v;
+                }
+        }
+    }
+#pragma unroll
+    for (int q = 0; q < RQ; ++q) {
+        const int row = row0 + q;
+        if (row < k) {
+#pragma unroll
+            for (int i = 0; i < NCH; ++i) {
+                const int c = lane + 32 * i;
+                if (c < k) D.Wj[(int64_t)row * k + c] = x[q][i];
+            }
+        }
+    }
+}
+
+// 3b: the logged rotations as a systolic pipeline.  A warp owns R rows of Q in shared memory.
+// Per group of 32 sweeps the columns k-1 ... lg of each row enter at lane 0, one per step; lane t
+// applies its sweep's rotation to the incoming column and the value it holds, passes the finished
+// column on to lane t+1 (one shuffle) and keeps the other; lane 31 writes the finished columns
+// back.  All 32 sweeps of a group advance in every step and the R rows are independent chains.
+template <int R>
+__global__ void __launch_bounds__(SYS_WARPS * 32)
+eig_rot_systolic_kernel(const RefreshDev *__restrict__ rd, const RowItem *__restrict__ items)
+{
+    extern __shared__ double zs[];                // [SYS_WARPS][R][k]
+    const RowItem it = items[blockIdx.x];
+    const RefreshDev D = rd[it.block];
+    const int k = D.k, r = D.r;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int row0 = it.row0 + warp * R;
+    if (row0 >= k) return;                        // warps never synchronise with one another
+    double *z = zs + (size_t)warp * R * k;
+#pragma unroll
+    for (int q = 0; q < R; ++q) {
+        const int row = min(row0 + q, k - 1);     // rows past the end shadow the last row, never stored
+        for (int c = lane; c < k; c += 32) z[q * k + c] = D.Wj[(int64_t)row * k + c];
+    }
+    __syncwarp();
+    const int nsw = *D.nsweeps;
+    const int ngroups = (nsw + 31) >> 5;
+    for (int g = 0; g < ngroups; ++g) {
+        const int2 gr = D.groups[g];
+        const int E = gr.y, T = E + SYS_FILL;
+        const int sidx = 32 * g + lane;
+        int hi = -1, lo = 0;                      // this lane's sweep acts on columns lo .. hi
+        if (sidx < nsw) { const int2 sw = D.sweeps[sidx]; hi = sw.x; lo = sw.x - sw.y + 1; }
+        const double2 *__restrict__ rp = D.rot + (int64_t)gr.x * 32 + lane;
+        double held[R], out[R];
+#pragma unroll
+        for (int q = 0; q < R; ++q) { held[q] = 0.0; out[q] = 0.0; }
+        int j = k - 1 + SYS_LAG * lane;           // column this lane consumes at step tau
+        // the rotations of the next SYS_PF steps are fetched while the current ones are applied
+        double2 nxt[SYS_PF];
+#pragma unroll
+        for (int u = 0; u < SYS_PF; ++u) nxt[u] = __ldg(rp + (int64_t)u * 32);
+        for (int tau0 = 0; tau0 < T; tau0 += SYS_PF) {
+            double2 cur[SYS_PF];
+#pragma unroll
+            for (int u = 0; u < SYS_PF; ++u) cur[u] = nxt[u];
+#pragma unroll
+            for (int u = 0; u < SYS_PF; ++u) nxt[u] = __ldg(rp + (int64_t)(tau0 + SYS_PF + u) * 32);
+#pragma unroll
+            for (int u = 0; u < SYS_PF; ++u, --j) {
+                const int tau = tau0 + u;
+                if (tau >= T) break;
+                const bool act = (j <= hi) && (j >= lo);
+                const double c = act ? cur[u].x : 1.0, s = act ? cur[u].y : 0.0;
+                const int cin = max(k - 1 - tau, 0);      // column entering lane 0 (all lanes read it: a broadcast)
+                const int cout = k - (tau - SYS_FILL);    // column leaving lane 31
+                const bool feed = (lane == 0), real = (tau < E - 1);
+                const bool emit = (lane == 31) && (tau > SYS_FILL);
+                double zin[R];
+#pragma unroll
+                for (int q = 0; q < R; ++q) zin[q] = z[q * k + cin];
+#pragma unroll
+                for (int q = 0; q < R; ++q) {
+                    const double up = __shfl_up_sync(0xffffffffu, out[q], 1);
+                    const double in = feed ? (real ? zin[q] : 0.0) : up;
+                    const double ch = c * held[q], sh = s * held[q];
+                    const double o = fma(s, in, ch);
+                    held[q] = fma(c, in, -sh);
+                    out[q] = o;
+                    if (emit) z[q * k + cout] = o;
+                }
+            }
+        }
+        __syncwarp();
+    }
+    // rank the eigenvalues (descending, ties by index) and emit the leading r columns
+    const double *__restrict__ lam = D.dvec;
+    for (int jj = lane; jj < k; jj += 32) {
+        const int rank = D.rank[jj];
+        if (rank >= r) continue;
+        const double lj = lam[jj];
+        const double inv = (lj > 1e-300) ? 1.0 / sqrt(lj) : 0.0;
+#pragma unroll
+        for (int q = 0; q < R; ++q) {
+            const int row = row0 + q;
+            if (row < k) {
+                const double w = z[q * k + jj];
+                D.Wu[(int64_t)row * r + rank] = (float)w;
+                D.Wv[(int64_t)row * r + rank] = (float)(w * inv);
+            }
+        }
+    }
+}
+
+static int sys_rows_per_warp(int kmax) { return kmax <= 544 ? 4 : 2; }
+
 int eig_panel_rows(int kmax)
 {
+    if (kmax <= SYS_KMAX) return SYS_WARPS * sys_rows_per_warp(kmax);
     int pr = (110 * 1024) / (8 * kmax);
     if (pr > 32) pr = 32;
     pr &= ~7;
     if (pr < 8) pr = 8;
     return pr;
+}
+
+int64_t eig_rot_capacity(int k)
+{
+    if (k <= SYS_KMAX) {   // rows of the skewed log (typical need: 0.03 k^2 + 4 k), 32 entries each
+        const int64_t rows = (int64_t)k * k / 10 + 12 * (int64_t)k + 512;
+        return rows * 32;
+    }
+    return 3 * (int64_t)k * k + 64;
+}
+
+template <typename F>
+static cudaError_t raise_smem(F *fn, size_t bytes, size_t *configured)
+{
+    if (bytes <= *configured) return cudaSuccess;
+    cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+    if (e == cudaSuccess) *configured = bytes;
+    return e;
 }
 
 cudaError_t eig_tridiag_batched(const RefreshDev *rd, const int32_t *list, int nlist, const RowItem *panel_items,
@@ -324,22 +545,38 @@ cudaError_t eig_tridiag_batched(const RefreshDev *rd, const int32_t *list, int n
     if (nlist <= 0) return cudaSuccess;
     const int kpad = kmax + 8;
     const size_t tr_bytes = (size_t)3 * kpad * sizeof(double);
+    static size_t tr_cfg = 0, pn_cfg = 0, sys4_cfg = 0, sys2_cfg = 0;
+    cudaError_t e;
+    if ((e = raise_smem(tridiag_kernel, tr_bytes, &tr_cfg)) != cudaSuccess) return e;
+    tridiag_kernel<<<nlist, TR_THREADS, tr_bytes, stream>>>(rd, list, kpad);
+    const size_t ql_bytes = (size_t)2 * kmax * sizeof(double);
+    if (kmax <= SYS_KMAX) {
+        const int threads = SYS_WARPS * 32;
+        if (kmax <= 288) eig_qrows_kernel<9, 4><<<npanels, threads, 0, stream>>>(rd, panel_items);
+        else if (kmax <= 544) eig_qrows_kernel<17, 4><<<npanels, threads, 0, stream>>>(rd, panel_items);
+        else eig_qrows_kernel<33, 2><<<npanels, threads, 0, stream>>>(rd, panel_items);
+        ql_log_kernel<true><<<nlist, 32, ql_bytes, stream>>>(rd, list);
+        eig_rank_kernel<<<nlist, 256, 0, stream>>>(rd, list);
+        const int R = sys_rows_per_warp(kmax);
+        const size_t sys_bytes = (size_t)SYS_WARPS * R * kmax * sizeof(double);
+        if (R == 4) {
+            if ((e = raise_smem(eig_rot_systolic_kernel<4>, sys_bytes, &sys4_cfg)) != cudaSuccess) return e;
+            eig_rot_systolic_kernel<4><<<npanels, threads, sys_bytes, stream>>>(rd, panel_items);
+        } else {
+            if ((e = raise_smem(eig_rot_systolic_kernel<2>, sys_bytes, &sys2_cfg)) != cudaSuccess) return e;
+            eig_rot_systolic_kernel<2><<<npanels, threads, sys_bytes, stream>>>(rd, panel_items);
+        }
+        return cudaGetLastError();
+    }
     const int pr = eig_panel_rows(kmax);
     const size_t pn_bytes = (size_t)pr * kmax * sizeof(double) + 64 * sizeof(double);   // panel + staging buffer
-    static size_t tr_cfg = 0, pn_cfg = 0;
-    cudaError_t e;
-    if (tr_bytes > tr_cfg) {
-        if ((e = cudaFuncSetAttribute(tridiag_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tr_bytes)) != cudaSuccess) return e;
-        tr_cfg = tr_bytes;
-    }
     if (pn_bytes > pn_cfg) {
         if ((e = cudaFuncSetAttribute(eigvec_panel_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pn_bytes)) != cudaSuccess) return e;
         // ask for the largest shared-memory carve-out so that two panels fit on one SM
         if ((e = cudaFuncSetAttribute(eigvec_panel_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 100)) != cudaSuccess) return e;
         pn_cfg = pn_bytes;
     }
-    tridiag_kernel<<<nlist, TR_THREADS, tr_bytes, stream>>>(rd, list, kpad);
-    ql_log_kernel<<<nlist, 32, (size_t)2 * kmax * sizeof(double), stream>>>(rd, list);
+    ql_log_kernel<false><<<nlist, 32, ql_bytes, stream>>>(rd, list);
     eig_rank_kernel<<<nlist, 256, 0, stream>>>(rd, list);
     eigvec_panel_kernel<<<npanels, 32, pn_bytes, stream>>>(rd, panel_items, pr);
     return cudaGetLastError();

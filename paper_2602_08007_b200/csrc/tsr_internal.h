@@ -131,7 +131,8 @@ struct RefreshDev {
     // tridiagonal eigen-solver (tsr_eig.cu)
     double *tau, *dvec, *evec;   // k each: reflector scales, diagonal / eigenvalues, off-diagonal
     double2 *rot;                // logged plane rotations (c, s)
-    int2 *sweeps;                // per QL sweep: first rotation index, count
+    int2 *sweeps;                // per QL sweep: column of the first rotation, count
+    int2 *groups;                // skewed log: per group of 32 sweeps (first row, stream elements)
     int32_t *nsweeps;            // number of logged sweeps
     int32_t *rank;               // k: descending rank of each eigenvalue
     int32_t rot_cap, sweep_cap;
@@ -155,8 +156,9 @@ cudaError_t rows_gemm_batched(const RefreshDev *rd, const RowItem *items, int ni
 // Eigen-decomposition of S by cyclic Jacobi, descending sort, Wu = W[:, :r], Wv = W[:, :r] / sqrt(lambda).
 // The same result through Householder tridiagonalisation + implicit QL with logged rotations
 // (for k too large for the Jacobi solver).  panel_items: (block, row0) slabs of eig_panel_rows(kmax)
-// rows of the k x k eigenvector matrix.
+// rows of the k x k eigenvector matrix.  eig_rot_capacity(k): entries of the rotation log to provide.
 int eig_panel_rows(int kmax);
+int64_t eig_rot_capacity(int k);
 cudaError_t eig_tridiag_batched(const RefreshDev *rd, const int32_t *list, int nlist, const RowItem *panel_items,
                                 int npanels, int kmax, cudaStream_t stream);
 cudaError_t jacobi_batched(const RefreshDev *rd, const int32_t *list, int nlist, int max_sweeps, cudaStream_t stream);

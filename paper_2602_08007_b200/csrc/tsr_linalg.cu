@@ -111,10 +111,15 @@ cudaError_t gram_batched(const RefreshDev *rd, const RowItem *items, int nitems,
 
 // ---------------------------------------------------------------------------------------
 // Cholesky S = R^T R with R upper triangular (one CTA per matrix, FP64, in place), followed by
-// Rinv = R^{-1} written as FP32.  Blocked: 16 rows of R at a time are factored in shared memory,
-// then the trailing upper triangle gets one rank-16 update, so the matrix in global memory is
-// read and written once per panel instead of once per row.  The inverse is computed 16 columns
-// at a time by back substitution, one warp per column with the column held in shared memory.
+// Rinv = R^{-1} written as FP32.  Both halves are blocked by 16 and synchronise the CTA a few
+// times per block instead of once per row:
+//   factorisation (right-looking): a 16-row panel of S sits in shared memory; one warp factors
+//   its 16 x 16 diagonal block, every other column of the panel is then one thread's forward
+//   substitution, and the trailing upper triangle gets one rank-16 update (two rows per warp);
+//   inverse (X = R^{-1}, block rows from the bottom up): with the 16 rows of R staged in shared
+//   memory, thread c accumulates sum_l R[i][l] X[l][c] over the rows l of X that are already
+//   known (FP64 copy in Xw, coalesced over c), then solves the 16 x 16 triangular system of its
+//   column in registers.  The sum over l is split between the two halves of the CTA.
 // A pivot that is not safely positive is replaced by a floor relative to the largest diagonal
 // entry and the block is flagged TSR_ERR_RANK_DEFICIENT.
 // ---------------------------------------------------------------------------------------
@@ -124,97 +129,185 @@ constexpr int CH_THREADS = 1024;
 __global__ void __launch_bounds__(CH_THREADS)
 chol_inverse_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ list, int kpad)
 {
-    extern __shared__ double ch_smem[];   // [CH_NB][kpad] panel of R rows, reused as [2 * CH_NB][kpad] columns of the inverse
+    extern __shared__ __align__(16) double ch_smem[];   // P[CH_NB][kpad]; red[CH_NB][kpad]
     const RefreshDev d = rd[list[blockIdx.x]];
     const int k = d.k;
     double *__restrict__ S = d.S;
-    __shared__ double s_piv;
+    double *__restrict__ X = d.Xw;
+    double *P = ch_smem;
+    double *red = ch_smem + (size_t)CH_NB * kpad;
     __shared__ double s_floor;
     __shared__ int s_flag;
     const int tid = threadIdx.x, nt = blockDim.x;
     const int warp = tid >> 5, lane = tid & 31, nwarps = nt >> 5;
-    if (tid == 0) {
+    if (warp == 0) {
         double mx = 0.0;
         int bad = 0;
-        for (int i = 0; i < k; ++i) {
+        for (int i = lane; i < k; i += 32) {
             const double v = S[(int64_t)i * k + i];
             if (!(v == v) || v > 1e300 || v < -1e300) bad = 1;
             if (v > mx) mx = v;
         }
-        s_floor = mx * 1e-13;
-        if (!(s_floor > 0.0)) s_floor = 1e-300;
-        s_flag = bad ? TSR_ERR_NONFINITE : 0;
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            mx = fmax(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+            bad |= __shfl_xor_sync(0xffffffffu, bad, off);
+        }
+        if (lane == 0) {
+            s_floor = mx * 1e-13;
+            if (!(s_floor > 0.0)) s_floor = 1e-300;
+            s_flag = bad ? TSR_ERR_NONFINITE : 0;
+        }
     }
     __syncthreads();
+    // ---- factorisation
     for (int jb = 0; jb < k; jb += CH_NB) {
         const int nb = min(CH_NB, k - jb);
         const int w = k - jb;                       // panel width: columns jb..k-1
-        double *P = ch_smem;                        // P[j][c] = S[jb + j][jb + c]
-        for (int e = tid; e < nb * w; e += nt) {
-            const int j = e / w, c = e % w;
+        for (int e = tid; e < nb * w; e += nt) {    // P[j][c] = S[jb + j][jb + c]
+            const int j = e / w, c = e - j * w;
             P[j * kpad + c] = (c >= j) ? S[(int64_t)(jb + j) * k + jb + c] : 0.0;
         }
         __syncthreads();
-        for (int j = 0; j < nb; ++j) {
-            if (tid == 0) {
+        if (warp == 0) {                            // the nb x nb diagonal block
+            const double floor_v = s_floor;
+            for (int j = 0; j < nb; ++j) {
                 double v = P[j * kpad + j];
-                if (!(v > s_floor)) {
-                    if (s_flag == 0) s_flag = TSR_ERR_RANK_DEFICIENT;
-                    v = s_floor;
+                if (!(v > floor_v)) {
+                    if (lane == 0 && s_flag == 0) s_flag = TSR_ERR_RANK_DEFICIENT;
+                    v = floor_v;
                 }
-                s_piv = sqrt(v);
+                const double piv = sqrt(v);
+                __syncwarp();
+                if (lane < nb && lane >= j) P[j * kpad + lane] = (lane == j) ? piv : P[j * kpad + lane] / piv;
+                __syncwarp();
+                for (int e = lane; e < nb * nb; e += 32) {
+                    const int i = e / nb, c = e - i * nb;
+                    if (i > j && c >= i) P[i * kpad + c] -= P[j * kpad + i] * P[j * kpad + c];
+                }
+                __syncwarp();
             }
-            __syncthreads();
-            const double piv = s_piv;
-            for (int c = j + tid; c < w; c += nt) P[j * kpad + c] = (c == j) ? piv : P[j * kpad + c] / piv;
-            __syncthreads();
-            // rows j+1..nb-1 of the panel: P[i][c] -= R[j][i] R[j][c], c >= i
-            const int rows_left = nb - j - 1;
-            for (int e = tid; e < rows_left * w; e += nt) {
-                const int i = j + 1 + e / w, c = e % w;
-                if (c >= i) P[i * kpad + c] -= P[j * kpad + i] * P[j * kpad + c];
-            }
-            __syncthreads();
         }
-        // final rows of R go back to global memory
-        for (int e = tid; e < nb * w; e += nt) {
-            const int j = e / w, c = e % w;
+        __syncthreads();
+        for (int c = nb + tid; c < w; c += nt) {    // R12 = R11^{-T} S12, one column per thread
+            double x[CH_NB];
+#pragma unroll
+            for (int j = 0; j < CH_NB; ++j) {
+                if (j < nb) {
+                    double acc = P[j * kpad + c];
+#pragma unroll
+                    for (int l = 0; l < j; ++l) acc -= P[l * kpad + j] * x[l];
+                    x[j] = acc / P[j * kpad + j];
+                } else {
+                    x[j] = 0.0;
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < CH_NB; ++j)
+                if (j < nb) P[j * kpad + c] = x[j];
+        }
+        __syncthreads();
+        for (int e = tid; e < nb * w; e += nt) {    // the finished rows of R
+            const int j = e / w, c = e - j * w;
             if (c >= j) S[(int64_t)(jb + j) * k + jb + c] = P[j * kpad + c];
         }
-        // rank-nb update of the trailing upper triangle
-        for (int i = jb + nb + warp; i < k; i += nwarps) {
+        // rank-nb update of the trailing upper triangle, rows i and i + 1 per warp
+        for (int i = jb + nb + 2 * warp; i < k; i += 2 * nwarps) {
             const int ci = i - jb;
-            double ri[CH_NB];
+            const bool two = (i + 1 < k);
+            double r0[CH_NB], r1[CH_NB];
 #pragma unroll
-            for (int j = 0; j < CH_NB; ++j) ri[j] = (j < nb) ? P[j * kpad + ci] : 0.0;
+            for (int j = 0; j < CH_NB; ++j) {
+                r0[j] = (j < nb) ? P[j * kpad + ci] : 0.0;
+                r1[j] = (j < nb && two) ? P[j * kpad + ci + 1] : 0.0;
+            }
             for (int l = i + lane; l < k; l += 32) {
                 const int cl = l - jb;
-                double acc = 0.0;
+                double a0 = 0.0, a1 = 0.0;
 #pragma unroll
-                for (int j = 0; j < CH_NB; ++j) acc += ri[j] * ((j < nb) ? P[j * kpad + cl] : 0.0);
-                S[(int64_t)i * k + l] -= acc;
+                for (int j = 0; j < CH_NB; ++j) {
+                    const double pj = (j < nb) ? P[j * kpad + cl] : 0.0;
+                    a0 += r0[j] * pj;
+                    a1 += r1[j] * pj;
+                }
+                S[(int64_t)i * k + l] -= a0;
+                if (two && l > i) S[(int64_t)(i + 1) * k + l] -= a1;
             }
         }
         __syncthreads();
     }
-    // X = R^{-1} (upper triangular).  Column c: X[i][c] = (delta_ic - sum_{l=i+1..c} R[i][l] X[l][c]) / R[i][i],
-    // i = c .. 0.  One warp per column; the column lives in shared memory ([row][column-in-panel]).
-    double *Xs = ch_smem;
-    const int cols_per_round = min(nwarps, 2 * CH_NB);          // 32 columns: 2 x CH_NB x kpad doubles
-    for (int c0 = 0; c0 < k; c0 += cols_per_round) {
-        const int c = c0 + warp;
-        if (warp < cols_per_round && c < k) {
-            double *xc = Xs + (int64_t)warp * kpad;              // this warp's column, contiguous
-            for (int i = c; i >= 0; --i) {
-                double part = 0.0;
-                const double *Ri = S + (int64_t)i * k;
-                for (int l = i + 1 + lane; l <= c; l += 32) part += Ri[l] * xc[l];
+    // ---- X = R^{-1}, block rows from the bottom up
+    const int half = tid / (CH_THREADS / 2), th = tid % (CH_THREADS / 2);
+    const int nblk = (k + CH_NB - 1) / CH_NB;
+    for (int I = nblk - 1; I >= 0; --I) {
+        const int i0 = I * CH_NB, nb = min(CH_NB, k - i0);
+        for (int e = tid; e < nb * (k - i0); e += nt) {   // P[j][c] = R[i0 + j][c], c >= i0
+            const int j = e / (k - i0), c = i0 + (e - j * (k - i0));
+            P[j * kpad + c] = S[(int64_t)(i0 + j) * k + c];
+        }
+        if (tid < 2 * CH_NB) P[(tid >> 1) * kpad + k + (tid & 1)] = 0.0;   // a pair may reach one column past k - 1
+        __syncthreads();
+        const int l0 = i0 + nb;                      // first row of X that is already known (a multiple of 16)
+        for (int c = i0 + th; c < k; c += CH_THREADS / 2) {
+            double acc[CH_NB];
 #pragma unroll
-                for (int off = 16; off > 0; off >>= 1) part += __shfl_xor_sync(0xffffffffu, part, off);
-                if (lane == 0) xc[i] = (((i == c) ? 1.0 : 0.0) - part) / Ri[i];
-                __syncwarp();
+            for (int j = 0; j < CH_NB; ++j) acc[j] = 0.0;
+            // rows l0 .. c of X in pairs; X is zero below its diagonal, so a pair may reach one row past c
+            for (int l = l0 + 2 * half; l <= c; l += 4) {
+                const double x0 = X[(int64_t)l * k + c];
+                const double x1 = (l + 1 < k) ? X[(int64_t)(l + 1) * k + c] : 0.0;
+#pragma unroll
+                for (int j = 0; j < CH_NB; ++j) {
+                    const double2 rr = *(const double2 *)&P[j * kpad + l];
+                    acc[j] += rr.x * x0 + rr.y * x1;
+                }
             }
-            for (int i = lane; i < k; i += 32) d.Rinv[(int64_t)i * k + c] = (i <= c) ? (float)xc[i] : 0.f;
+            if (half == 1) {
+#pragma unroll
+                for (int j = 0; j < CH_NB; ++j) red[j * kpad + c] = acc[j];
+            }
+        }
+        __syncthreads();
+        if (half == 0) {
+            for (int c = i0 + th; c < k; c += CH_THREADS / 2) {
+                double acc[CH_NB];
+#pragma unroll
+                for (int j = 0; j < CH_NB; ++j) acc[j] = 0.0;
+                for (int l = l0; l <= c; l += 4) {
+                    const double x0 = X[(int64_t)l * k + c];
+                    const double x1 = (l + 1 < k) ? X[(int64_t)(l + 1) * k + c] : 0.0;
+#pragma unroll
+                    for (int j = 0; j < CH_NB; ++j) {
+                        const double2 rr = *(const double2 *)&P[j * kpad + l];
+                        acc[j] += rr.x * x0 + rr.y * x1;
+                    }
+                }
+                double y[CH_NB];
+#pragma unroll
+                for (int j = CH_NB - 1; j >= 0; --j) {
+                    if (j < nb) {
+                        double sj = ((i0 + j == c) ? 1.0 : 0.0) - (acc[j] + red[j * kpad + c]);
+#pragma unroll
+                        for (int l = j + 1; l < CH_NB; ++l)
+                            if (l < nb) sj -= P[j * kpad + i0 + l] * y[l];
+                        y[j] = sj / P[j * kpad + i0 + j];
+                    } else {
+                        y[j] = 0.0;
+                    }
+                }
+#pragma unroll
+                for (int j = 0; j < CH_NB; ++j)
+                    if (j < nb) {
+                        X[(int64_t)(i0 + j) * k + c] = y[j];
+                        d.Rinv[(int64_t)(i0 + j) * k + c] = (float)y[j];
+                    }
+            }
+        } else {                                     // the other half clears the part left of the diagonal block
+            for (int e = th; e < nb * i0; e += CH_THREADS / 2) {
+                const int j = e / i0, c = e - j * i0;
+                X[(int64_t)(i0 + j) * k + c] = 0.0;
+                d.Rinv[(int64_t)(i0 + j) * k + c] = 0.f;
+            }
         }
         __syncthreads();
     }
@@ -224,13 +317,11 @@ chol_inverse_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict
 cudaError_t chol_inverse_batched(const RefreshDev *rd, const int32_t *list, int nlist, int kmax, cudaStream_t stream)
 {
     if (nlist <= 0) return cudaSuccess;
-    const int kpad = (kmax + 1) | 1;   // odd row pitch (in doubles) keeps shared-memory columns conflict-free
+    const int kpad = (kmax + 3) & ~1;   // even row pitch (in doubles): pairs of a row are read as one 16-byte word
     const size_t bytes = (size_t)2 * CH_NB * kpad * sizeof(double);
     static size_t configured = 0;
     if (bytes > configured) {
         cudaError_t e = cudaFuncSetAttribute(chol_inverse_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
-        if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(chol_inverse_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
         if (e != cudaSuccess) return e;
         configured = bytes;
     }
