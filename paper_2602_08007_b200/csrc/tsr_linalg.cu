@@ -114,28 +114,35 @@ cudaError_t gram_batched(const RefreshDev *rd, const RowItem *items, int nitems,
 // Rinv = R^{-1} written as FP32.  Both halves are blocked by 16 and synchronise the CTA a few
 // times per block instead of once per row:
 //   factorisation (right-looking): a 16-row panel of S sits in shared memory; one warp factors
-//   its 16 x 16 diagonal block, every other column of the panel is then one thread's forward
-//   substitution, and the trailing upper triangle gets one rank-16 update (two rows per warp);
+//   its 16 x 16 diagonal block R11 and inverts it (which is also the diagonal block of R^{-1});
+//   every other column of the panel is then one thread's product with R11^{-T}, and the trailing
+//   upper triangle gets one rank-16 update (two rows per warp, four loads in flight per lane);
 //   inverse (X = R^{-1}, block rows from the bottom up): with the 16 rows of R staged in shared
 //   memory, thread c accumulates sum_l R[i][l] X[l][c] over the rows l of X that are already
-//   known (FP64 copy in Xw, coalesced over c), then solves the 16 x 16 triangular system of its
-//   column in registers.  The sum over l is split between the two halves of the CTA.
+//   known (FP64 copy in Xw, coalesced over c) and multiplies by -R11^{-1}.
 // A pivot that is not safely positive is replaced by a floor relative to the largest diagonal
 // entry and the block is flagged TSR_ERR_RANK_DEFICIENT.
 // ---------------------------------------------------------------------------------------
 constexpr int CH_NB = 16;
-constexpr int CH_THREADS = 1024;
+constexpr int CH_THREADS = 512;
+constexpr int CH_U = 2;      // columns per lane and trip in the trailing update
+#ifdef CH_PROFILE
+#define CH_TICK(slot) do { if (threadIdx.x == 0 && blockIdx.x == 0) { const long long t_ = clock64(); ch_prof[slot] += t_ - ch_t0; ch_t0 = t_; } } while (0)
+#else
+#define CH_TICK(slot) do { } while (0)
+#endif
 
 __global__ void __launch_bounds__(CH_THREADS)
 chol_inverse_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ list, int kpad)
 {
-    extern __shared__ __align__(16) double ch_smem[];   // P[CH_NB][kpad]; red[CH_NB][kpad]
+    extern __shared__ __align__(16) double ch_smem[];   // P[CH_NB][kpad]
     const RefreshDev d = rd[list[blockIdx.x]];
     const int k = d.k;
     double *__restrict__ S = d.S;
     double *__restrict__ X = d.Xw;
     double *P = ch_smem;
-    double *red = ch_smem + (size_t)CH_NB * kpad;
+    __shared__ double dinv[CH_NB][CH_NB + 1];    // inverse of the current diagonal block (upper triangular)
+    __shared__ double rdiag[CH_NB];              // 1 / R[j][j] of the current diagonal block
     __shared__ double s_floor;
     __shared__ int s_flag;
     const int tid = threadIdx.x, nt = blockDim.x;
@@ -160,6 +167,9 @@ chol_inverse_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict
         }
     }
     __syncthreads();
+#ifdef CH_PROFILE
+    long long ch_t0 = clock64();
+#endif
     // ---- factorisation
     for (int jb = 0; jb < k; jb += CH_NB) {
         const int nb = min(CH_NB, k - jb);
@@ -169,7 +179,8 @@ chol_inverse_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict
             P[j * kpad + c] = (c >= j) ? S[(int64_t)(jb + j) * k + jb + c] : 0.0;
         }
         __syncthreads();
-        if (warp == 0) {                            // the nb x nb diagonal block
+        CH_TICK(0);
+        if (warp == 0) {                            // the nb x nb diagonal block and its inverse
             const double floor_v = s_floor;
             for (int j = 0; j < nb; ++j) {
                 double v = P[j * kpad + j];
@@ -177,41 +188,53 @@ chol_inverse_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict
                     if (lane == 0 && s_flag == 0) s_flag = TSR_ERR_RANK_DEFICIENT;
                     v = floor_v;
                 }
-                const double piv = sqrt(v);
+                const double piv = sqrt(v), rpiv = 1.0 / piv;
                 __syncwarp();
-                if (lane < nb && lane >= j) P[j * kpad + lane] = (lane == j) ? piv : P[j * kpad + lane] / piv;
+                if (lane == 0) rdiag[j] = rpiv;
+                if (lane < nb && lane >= j) P[j * kpad + lane] = (lane == j) ? piv : P[j * kpad + lane] * rpiv;
                 __syncwarp();
-                for (int e = lane; e < nb * nb; e += 32) {
-                    const int i = e / nb, c = e - i * nb;
-                    if (i > j && c >= i) P[i * kpad + c] -= P[j * kpad + i] * P[j * kpad + c];
+                for (int e = lane; e < CH_NB * CH_NB; e += 32) {
+                    const int i = e / CH_NB, c = e % CH_NB;
+                    if (i > j && c >= i && c < nb) P[i * kpad + c] -= P[j * kpad + i] * P[j * kpad + c];
                 }
                 __syncwarp();
             }
+            if (lane < CH_NB) {                     // column `lane` of R11^{-1} by back substitution
+                const int c = lane;
+                for (int i = CH_NB - 1; i >= 0; --i) {
+                    double acc = (i == c) ? 1.0 : 0.0;
+                    for (int l = i + 1; l <= c && l < nb; ++l) acc -= P[i * kpad + l] * dinv[l][c];
+                    const double xi = (i <= c && c < nb) ? acc * rdiag[i] : 0.0;
+                    dinv[i][c] = xi;
+                    if (i < nb && c < nb) {
+                        X[(int64_t)(jb + i) * k + jb + c] = xi;
+                        d.Rinv[(int64_t)(jb + i) * k + jb + c] = (float)xi;
+                    }
+                }
+            }
         }
         __syncthreads();
+        CH_TICK(1);
         for (int c = nb + tid; c < w; c += nt) {    // R12 = R11^{-T} S12, one column per thread
-            double x[CH_NB];
+            double sv[CH_NB];
+#pragma unroll
+            for (int l = 0; l < CH_NB; ++l) sv[l] = (l < nb) ? P[l * kpad + c] : 0.0;
 #pragma unroll
             for (int j = 0; j < CH_NB; ++j) {
-                if (j < nb) {
-                    double acc = P[j * kpad + c];
+                double acc = 0.0;
 #pragma unroll
-                    for (int l = 0; l < j; ++l) acc -= P[l * kpad + j] * x[l];
-                    x[j] = acc / P[j * kpad + j];
-                } else {
-                    x[j] = 0.0;
-                }
+                for (int l = 0; l <= j; ++l) acc += dinv[l][j] * sv[l];
+                if (j < nb) P[j * kpad + c] = acc;
             }
-#pragma unroll
-            for (int j = 0; j < CH_NB; ++j)
-                if (j < nb) P[j * kpad + c] = x[j];
         }
         __syncthreads();
+        CH_TICK(2);
         for (int e = tid; e < nb * w; e += nt) {    // the finished rows of R
             const int j = e / w, c = e - j * w;
             if (c >= j) S[(int64_t)(jb + j) * k + jb + c] = P[j * kpad + c];
         }
-        // rank-nb update of the trailing upper triangle, rows i and i + 1 per warp
+        // rank-nb update of the trailing upper triangle: rows i and i + 1 per warp, CH_U columns per
+        // lane and trip with their loads issued before the arithmetic
         for (int i = jb + nb + 2 * warp; i < k; i += 2 * nwarps) {
             const int ci = i - jb;
             const bool two = (i + 1 < k);
@@ -221,95 +244,97 @@ chol_inverse_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict
                 r0[j] = (j < nb) ? P[j * kpad + ci] : 0.0;
                 r1[j] = (j < nb && two) ? P[j * kpad + ci + 1] : 0.0;
             }
-            for (int l = i + lane; l < k; l += 32) {
-                const int cl = l - jb;
-                double a0 = 0.0, a1 = 0.0;
+            double *row0 = S + (int64_t)i * k, *row1 = S + (int64_t)(i + 1) * k;
+            for (int lb = i + lane; lb < k; lb += 32 * CH_U) {
+                double s0[CH_U], s1[CH_U], a0[CH_U], a1[CH_U];
+#pragma unroll
+                for (int u = 0; u < CH_U; ++u) {
+                    const int l = lb + 32 * u;
+                    s0[u] = (l < k) ? row0[l] : 0.0;
+                    s1[u] = (two && l < k && l > i) ? row1[l] : 0.0;
+                    a0[u] = 0.0; a1[u] = 0.0;
+                }
 #pragma unroll
                 for (int j = 0; j < CH_NB; ++j) {
-                    const double pj = (j < nb) ? P[j * kpad + cl] : 0.0;
-                    a0 += r0[j] * pj;
-                    a1 += r1[j] * pj;
+#pragma unroll
+                    for (int u = 0; u < CH_U; ++u) {
+                        const int cl = min(lb + 32 * u, k - 1) - jb;
+                        const double pj = P[j * kpad + cl];
+                        a0[u] += r0[j] * pj;
+                        a1[u] += r1[j] * pj;
+                    }
                 }
-                S[(int64_t)i * k + l] -= a0;
-                if (two && l > i) S[(int64_t)(i + 1) * k + l] -= a1;
+#pragma unroll
+                for (int u = 0; u < CH_U; ++u) {
+                    const int l = lb + 32 * u;
+                    if (l < k) {
+                        row0[l] = s0[u] - a0[u];
+                        if (two && l > i) row1[l] = s1[u] - a1[u];
+                    }
+                }
             }
         }
         __syncthreads();
+        CH_TICK(3);
     }
-    // ---- X = R^{-1}, block rows from the bottom up
-    const int half = tid / (CH_THREADS / 2), th = tid % (CH_THREADS / 2);
+    // ---- X = R^{-1}, block rows from the bottom up (the diagonal blocks are already in place)
     const int nblk = (k + CH_NB - 1) / CH_NB;
     for (int I = nblk - 1; I >= 0; --I) {
         const int i0 = I * CH_NB, nb = min(CH_NB, k - i0);
-        for (int e = tid; e < nb * (k - i0); e += nt) {   // P[j][c] = R[i0 + j][c], c >= i0
-            const int j = e / (k - i0), c = i0 + (e - j * (k - i0));
+        const int l0 = i0 + nb;                      // first row of X that is already known (a multiple of 16)
+        for (int e = tid; e < nb * (k - l0); e += nt) {   // P[j][c] = R[i0 + j][c], c >= l0
+            const int j = e / (k - l0), c = l0 + (e - j * (k - l0));
             P[j * kpad + c] = S[(int64_t)(i0 + j) * k + c];
         }
-        if (tid < 2 * CH_NB) P[(tid >> 1) * kpad + k + (tid & 1)] = 0.0;   // a pair may reach one column past k - 1
+        if (tid < 4 * CH_NB) P[(tid >> 2) * kpad + k + (tid & 3)] = 0.0;   // a group may reach three columns past k - 1
+        if (tid < CH_NB * CH_NB) {
+            const int i = tid / CH_NB, c = tid % CH_NB;
+            dinv[i][c] = (i < nb && c < nb && c >= i) ? X[(int64_t)(i0 + i) * k + i0 + c] : 0.0;
+        }
         __syncthreads();
-        const int l0 = i0 + nb;                      // first row of X that is already known (a multiple of 16)
-        for (int c = i0 + th; c < k; c += CH_THREADS / 2) {
+        CH_TICK(4);
+        for (int c = l0 + tid; c < k; c += nt) {
             double acc[CH_NB];
 #pragma unroll
             for (int j = 0; j < CH_NB; ++j) acc[j] = 0.0;
-            // rows l0 .. c of X in pairs; X is zero below its diagonal, so a pair may reach one row past c
-            for (int l = l0 + 2 * half; l <= c; l += 4) {
-                const double x0 = X[(int64_t)l * k + c];
-                const double x1 = (l + 1 < k) ? X[(int64_t)(l + 1) * k + c] : 0.0;
+            // rows l0 .. c of X four at a time (X is zero below its diagonal, so a group may reach past
+            // row c); the next group is fetched while the current one is used
+            auto xload = [&](int l) -> double { return (l < k) ? X[(int64_t)l * k + c] : 0.0; };
+            int l = l0;
+            double x0 = xload(l), x1 = xload(l + 1), x2 = xload(l + 2), x3 = xload(l + 3);
+            for (; l <= c; l += 4) {
+                const int ln = l + 4;
+                double n0 = 0.0, n1 = 0.0, n2 = 0.0, n3 = 0.0;
+                if (ln <= c) { n0 = xload(ln); n1 = xload(ln + 1); n2 = xload(ln + 2); n3 = xload(ln + 3); }
 #pragma unroll
                 for (int j = 0; j < CH_NB; ++j) {
-                    const double2 rr = *(const double2 *)&P[j * kpad + l];
-                    acc[j] += rr.x * x0 + rr.y * x1;
+                    const double2 ra = *(const double2 *)&P[j * kpad + l];
+                    const double2 rb = *(const double2 *)&P[j * kpad + l + 2];
+                    acc[j] += (ra.x * x0 + ra.y * x1) + (rb.x * x2 + rb.y * x3);
+                }
+                x0 = n0; x1 = n1; x2 = n2; x3 = n3;
+            }
+            CH_TICK(5);
+            // X[I][c] = -R11^{-1} acc
+#pragma unroll
+            for (int j = 0; j < CH_NB; ++j) {
+                double y = 0.0;
+#pragma unroll
+                for (int l2 = j; l2 < CH_NB; ++l2) y -= dinv[j][l2] * acc[l2];
+                if (j < nb) {
+                    X[(int64_t)(i0 + j) * k + c] = y;
+                    d.Rinv[(int64_t)(i0 + j) * k + c] = (float)y;
                 }
             }
-            if (half == 1) {
-#pragma unroll
-                for (int j = 0; j < CH_NB; ++j) red[j * kpad + c] = acc[j];
-            }
+            CH_TICK(6);
+        }
+        for (int e = tid; e < nb * i0; e += nt) {    // zeros left of the diagonal block
+            const int j = e / i0, c = e - j * i0;
+            X[(int64_t)(i0 + j) * k + c] = 0.0;
+            d.Rinv[(int64_t)(i0 + j) * k + c] = 0.f;
         }
         __syncthreads();
-        if (half == 0) {
-            for (int c = i0 + th; c < k; c += CH_THREADS / 2) {
-                double acc[CH_NB];
-#pragma unroll
-                for (int j = 0; j < CH_NB; ++j) acc[j] = 0.0;
-                for (int l = l0; l <= c; l += 4) {
-                    const double x0 = X[(int64_t)l * k + c];
-                    const double x1 = (l + 1 < k) ? X[(int64_t)(l + 1) * k + c] : 0.0;
-#pragma unroll
-                    for (int j = 0; j < CH_NB; ++j) {
-                        const double2 rr = *(const double2 *)&P[j * kpad + l];
-                        acc[j] += rr.x * x0 + rr.y * x1;
-                    }
-                }
-                double y[CH_NB];
-#pragma unroll
-                for (int j = CH_NB - 1; j >= 0; --j) {
-                    if (j < nb) {
-                        double sj = ((i0 + j == c) ? 1.0 : 0.0) - (acc[j] + red[j * kpad + c]);
-#pragma unroll
-                        for (int l = j + 1; l < CH_NB; ++l)
-                            if (l < nb) sj -= P[j * kpad + i0 + l] * y[l];
-                        y[j] = sj / P[j * kpad + i0 + j];
-                    } else {
-                        y[j] = 0.0;
-                    }
-                }
-#pragma unroll
-                for (int j = 0; j < CH_NB; ++j)
-                    if (j < nb) {
-                        X[(int64_t)(i0 + j) * k + c] = y[j];
-                        d.Rinv[(int64_t)(i0 + j) * k + c] = (float)y[j];
-                    }
-            }
-        } else {                                     // the other half clears the part left of the diagonal block
-            for (int e = th; e < nb * i0; e += CH_THREADS / 2) {
-                const int j = e / i0, c = e - j * i0;
-                X[(int64_t)(i0 + j) * k + c] = 0.0;
-                d.Rinv[(int64_t)(i0 + j) * k + c] = 0.f;
-            }
-        }
-        __syncthreads();
+        CH_TICK(7);
     }
     if (tid == 0 && s_flag != 0) atomicMax(d.status, s_flag);
 }
@@ -317,8 +342,8 @@ chol_inverse_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict
 cudaError_t chol_inverse_batched(const RefreshDev *rd, const int32_t *list, int nlist, int kmax, cudaStream_t stream)
 {
     if (nlist <= 0) return cudaSuccess;
-    const int kpad = (kmax + 3) & ~1;   // even row pitch (in doubles): pairs of a row are read as one 16-byte word
-    const size_t bytes = (size_t)2 * CH_NB * kpad * sizeof(double);
+    const int kpad = (kmax + 5) & ~1;   // even row pitch (in doubles): pairs of a row are read as one 16-byte word
+    const size_t bytes = (size_t)CH_NB * kpad * sizeof(double);
     static size_t configured = 0;
     if (bytes > configured) {
         cudaError_t e = cudaFuncSetAttribute(chol_inverse_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
@@ -370,8 +395,10 @@ rows_gemm_kernel(const RefreshDev *__restrict__ rd, const RowItem *__restrict__ 
             rb[l] = (gj < N && gk2 < K) ? B[(int64_t)gk2 * N + gj] : 0.f;
         }
     };
+    // Rinv is upper triangular: columns n0 .. n0 + 63 of the product only need rows 0 .. n0 + 63 of it
+    const int Kend = (mat_sel == 0) ? min(K, n0 + 64) : K;
     fetch(0);
-    for (int k0 = 0; k0 < K; k0 += 16) {
+    for (int k0 = 0; k0 < Kend; k0 += 16) {
 #pragma unroll
         for (int l = 0; l < 4; ++l) {
             const int e = tid + l * 256;
@@ -379,7 +406,7 @@ rows_gemm_kernel(const RefreshDev *__restrict__ rd, const RowItem *__restrict__ 
             Bs[e / 64][e % 64] = rb[l];
         }
         __syncthreads();
-        if (k0 + 16 < K) fetch(k0 + 16);
+        if (k0 + 16 < Kend) fetch(k0 + 16);
 #pragma unroll
         for (int kk = 0; kk < 16; ++kk) {
             const float4 af = *(const float4 *)&As[kk][ty * 4];
