@@ -69,14 +69,23 @@ tridiag_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ li
         }
         if (tid == 0) { d.tau[j] = tau; d.dvec[j] = A[(int64_t)j * k + j]; d.evec[j] = alpha; }
         __syncthreads();
-        // p = tau * A22 v      (A22 = A[j+1.., j+1..], row-wise dot products, one warp per row)
-        for (int a = warp; a < len; a += nwarps) {
-            const double *row = A + (int64_t)(j + 1 + a) * k + j + 1;
-            double acc = 0.0;
-            for (int b = lane; b < len; b += 32) acc += row[b] * vs[b];
+        // p = tau * A22 v      (A22 = A[j+1.., j+1..], row-wise dot products; a warp takes four rows at a
+        // time so that four loads are in flight per lane)
+        for (int a0 = 4 * warp; a0 < len; a0 += 4 * nwarps) {
+            const double *row0 = A + (int64_t)(j + 1 + a0) * k + j + 1;
+            const int na = min(4, len - a0);
+            double acc[4] = {0.0, 0.0, 0.0, 0.0};
+            for (int b = lane; b < len; b += 32) {
+                const double vb = vs[b];
 #pragma unroll
-            for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
-            if (lane == 0) ps[a] = tau * acc;
+                for (int u = 0; u < 4; ++u)
+                    if (u < na) acc[u] += row0[(int64_t)u * k + b] * vb;
+            }
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1)
+#pragma unroll
+                for (int u = 0; u < 4; ++u) acc[u] += __shfl_xor_sync(0xffffffffu, acc[u], off);
+            if (lane < na) ps[a0 + lane] = tau * (lane == 0 ? acc[0] : lane == 1 ? acc[1] : lane == 2 ? acc[2] : acc[3]);
         }
         __syncthreads();
         part = 0.0;
@@ -85,11 +94,22 @@ tridiag_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ li
         const double kk = 0.5 * tau * pv;
         for (int i = tid; i < len; i += nt) ws[i] = ps[i] - kk * vs[i];
         __syncthreads();
-        // A22 -= v w^T + w v^T
-        for (int a = warp; a < len; a += nwarps) {
-            double *row = A + (int64_t)(j + 1 + a) * k + j + 1;
-            const double va = vs[a], wa = ws[a];
-            for (int b = lane; b < len; b += 32) row[b] -= va * ws[b] + wa * vs[b];
+        // A22 -= v w^T + w v^T   (four rows per warp and trip)
+        for (int a0 = 4 * warp; a0 < len; a0 += 4 * nwarps) {
+            double *row0 = A + (int64_t)(j + 1 + a0) * k + j + 1;
+            const int na = min(4, len - a0);
+            double va[4], wa[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) { va[u] = (u < na) ? vs[a0 + u] : 0.0; wa[u] = (u < na) ? ws[a0 + u] : 0.0; }
+            for (int b = lane; b < len; b += 32) {
+                const double vb = vs[b], wb = ws[b];
+                double x[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) x[u] = (u < na) ? row0[(int64_t)u * k + b] : 0.0;
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    if (u < na) row0[(int64_t)u * k + b] = x[u] - (va[u] * wb + wa[u] * vb);
+            }
         }
         __syncthreads();
     }
@@ -167,8 +187,10 @@ ql_log_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ lis
                 const int first = nrot;
                 int i = m - 1;
                 bool early = false;
+                double e_nx = e[i], d_nx = d[i];      // fetched one rotation ahead of the stores below
                 for (; i >= l; --i) {
-                    const double ei = e[i];
+                    const double ei = e_nx, di = d_nx;
+                    if (i > l) { e_nx = e[i - 1]; d_nx = d[i - 1]; }
                     const double f = s * ei, b = c * ei;
                     // r = hypot(f, g).  The entries are bounded by the eigenvalues of a Gram matrix of FP32
                     // data, so the squares stay far inside the FP64 range and no rescaling is needed.
@@ -180,7 +202,7 @@ ql_log_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ lis
                     s = f * rinv;
                     c = g * rinv;
                     g = d[i + 1] - p;
-                    r = (d[i] - g) * s + 2.0 * c * b;
+                    r = (di - g) * s + 2.0 * c * b;
                     p = s * r;
                     d[i + 1] = g + p;
                     g = c * r - b;
@@ -339,13 +361,13 @@ __global__ void eig_rank_kernel(const RefreshDev *__restrict__ rd, const int32_t
 }
 
 // ---- stage 3, systolic form (k <= SYS_KMAX) ---------------------------------------------------
-// 3a: rows of Q = H_0 H_1 ... in registers.  A warp owns RQ rows; lane holds columns lane + 32 i.
+// 3a: rows of Q = H_0 H_1 ... in registers.  A warp owns RQ rows (NW warps per CTA); lane holds columns lane + 32 i.
 // The reflectors are staged for the whole CTA, a few at a time, in shared memory.
 constexpr int SYS_KMAX = 1056;
 constexpr int SYS_WARPS = 8;
 
-template <int NCH, int RQ>
-__global__ void __launch_bounds__(SYS_WARPS * 32)
+template <int NCH, int RQ, int NW>
+__global__ void __launch_bounds__(NW * 32)
 eig_qrows_kernel(const RefreshDev *__restrict__ rd, const RowItem *__restrict__ items)
 {
     constexpr int LD = NCH * 32;
@@ -366,7 +388,7 @@ eig_qrows_kernel(const RefreshDev *__restrict__ rd, const RowItem *__restrict__ 
 
     for (int j0 = 0; j0 + 2 < k; j0 += QV_BATCH) {
         __syncthreads();
-        for (int idx = threadIdx.x; idx < QV_BATCH * LD; idx += SYS_WARPS * 32) {
+        for (int idx = threadIdx.x; idx < QV_BATCH * LD; idx += NW * 32) {
             const int b = idx / LD, c = idx - b * LD, j = j0 + b;
             double v = 0.0;
             if (j + 2 < k && c < k) v = (c == j + 1) ? 1.0 : (c >= j + 2 ? A[(int64_t)j * k + c] : 0.0);
@@ -552,9 +574,10 @@ cudaError_t eig_tridiag_batched(const RefreshDev *rd, const int32_t *list, int n
     const size_t ql_bytes = (size_t)2 * kmax * sizeof(double);
     if (kmax <= SYS_KMAX) {
         const int threads = SYS_WARPS * 32;
-        if (kmax <= 288) eig_qrows_kernel<9, 4><<<npanels, threads, 0, stream>>>(rd, panel_items);
-        else if (kmax <= 544) eig_qrows_kernel<17, 4><<<npanels, threads, 0, stream>>>(rd, panel_items);
-        else eig_qrows_kernel<33, 2><<<npanels, threads, 0, stream>>>(rd, panel_items);
+        // same row slabs as the rotation kernel (32 or 16 rows), spread over 16 warps
+        if (kmax <= 288) eig_qrows_kernel<9, 2, 16><<<npanels, 512, 0, stream>>>(rd, panel_items);
+        else if (kmax <= 544) eig_qrows_kernel<17, 2, 16><<<npanels, 512, 0, stream>>>(rd, panel_items);
+        else eig_qrows_kernel<33, 1, 16><<<npanels, 512, 0, stream>>>(rd, panel_items);
         ql_log_kernel<true><<<nlist, 32, ql_bytes, stream>>>(rd, list);
         eig_rank_kernel<<<nlist, 256, 0, stream>>>(rd, list);
         const int R = sys_rows_per_warp(kmax);

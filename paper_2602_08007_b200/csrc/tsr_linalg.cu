@@ -11,10 +11,23 @@ namespace tsr {
 
 // ---------------------------------------------------------------------------------------
 // S = X^T X, X rows x k FP32, accumulation in FP64.  Rows are cut into slabs of GRAM_ROWS;
-// each slab writes its own partial (upper-triangular tiles only), a second kernel adds the
+// each slab writes its own partial (upper-triangular part only), a second kernel adds the
 // partials in slab order and mirrors the result, so the sum is deterministic.
+// The products run on the FP64 tensor-core path (mma.sync m8n8k4: FP32 inputs convert to FP64
+// exactly, FP64 fused accumulation): a CTA owns a 64 x 64 tile of S, its eight warps 32 x 16
+// regions of it as 4 x 2 sub-tiles of 8 x 8.  Sub-tiles below the diagonal or past column k are
+// skipped, so the work follows the upper triangle to a granularity of 8.
 // ---------------------------------------------------------------------------------------
-constexpr int GR_T = 64;  // output tile edge
+constexpr int GR_T = 64;   // output tile edge
+constexpr int GR_S = 8;    // sub-tile edge (the MMA shape)
+constexpr int GR_PITCH = 72;   // floats per staged row: 72 = 8 mod 32 keeps the fragment loads conflict-free
+
+__device__ __forceinline__ void dmma_8x8x4(double &c0, double &c1, double a, double b)
+{
+    asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
+                 : "+d"(c0), "+d"(c1)
+                 : "d"(a), "d"(b));
+}
 
 __global__ void __launch_bounds__(256)
 gram_partial_kernel(const RefreshDev *__restrict__ rd, const RowItem *__restrict__ items, int side, int src_sel)
@@ -26,16 +39,29 @@ gram_partial_kernel(const RefreshDev *__restrict__ rd, const RowItem *__restrict
     if (tj < ti || ti * GR_T >= k || tj * GR_T >= k) return;
     const int rows = side ? d.n : d.m;
     const float *__restrict__ X = d.buf[src_sel];
-    __shared__ __align__(16) float Xi[16][GR_T + 4];
-    __shared__ __align__(16) float Xj[16][GR_T + 4];
-    const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;  // 16 x 16 threads, 4 x 4 outputs each
+    __shared__ __align__(16) float Xi[16][GR_PITCH];
+    __shared__ __align__(16) float Xj[16][GR_PITCH];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int wi = warp >> 2, wj = warp & 3;         // warp grid 2 x 4: rows 32 wi .., columns 16 wj ..
+    const int g = lane >> 2, q = lane & 3;           // fragment coordinates
     const int row_begin = it.row0;
     const int row_end = min(rows, row_begin + GRAM_ROWS);
-    double acc[4][4];
+    // which of the warp's 4 x 2 sub-tiles hold anything to compute
+    bool need[4][2];
+    bool any = false;
 #pragma unroll
     for (int a = 0; a < 4; ++a)
 #pragma unroll
-        for (int b = 0; b < 4; ++b) acc[a][b] = 0.0;
+        for (int b = 0; b < 2; ++b) {
+            const int si = ti * (GR_T / GR_S) + wi * 4 + a, sj = tj * (GR_T / GR_S) + wj * 2 + b;
+            need[a][b] = (sj >= si) && (si * GR_S < k) && (sj * GR_S < k);
+            any = any || need[a][b];
+        }
+    double acc[4][2][2];
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+        for (int b = 0; b < 2; ++b) acc[a][b][0] = acc[a][b][1] = 0.0;
     float ri[4], rj[4];
     auto fetch = [&](int r0) {
 #pragma unroll
@@ -58,16 +84,20 @@ gram_partial_kernel(const RefreshDev *__restrict__ rd, const RowItem *__restrict
         }
         __syncthreads();
         if (r0 + 16 < row_end) fetch(r0 + 16);
+        if (any) {
 #pragma unroll
-        for (int rr = 0; rr < 16; ++rr) {
-            const float4 af = *(const float4 *)&Xi[rr][ty * 4];
-            const float4 bf = *(const float4 *)&Xj[rr][tx * 4];
-            const double av[4] = {af.x, af.y, af.z, af.w};
-            const double bv[4] = {bf.x, bf.y, bf.z, bf.w};
+            for (int kk = 0; kk < 4; ++kk) {             // four rows of X per MMA
+                double af[4], bf[2];
 #pragma unroll
-            for (int a = 0; a < 4; ++a)
+                for (int a = 0; a < 4; ++a) af[a] = (double)Xi[kk * 4 + q][wi * 32 + a * GR_S + g];
 #pragma unroll
-                for (int b = 0; b < 4; ++b) acc[a][b] += av[a] * bv[b];
+                for (int b = 0; b < 2; ++b) bf[b] = (double)Xj[kk * 4 + q][wj * 16 + b * GR_S + g];
+#pragma unroll
+                for (int a = 0; a < 4; ++a)
+#pragma unroll
+                    for (int b = 0; b < 2; ++b)
+                        if (need[a][b]) dmma_8x8x4(acc[a][b][0], acc[a][b][1], af[a], bf[b]);
+            }
         }
         __syncthreads();
     }
@@ -75,9 +105,12 @@ gram_partial_kernel(const RefreshDev *__restrict__ rd, const RowItem *__restrict
 #pragma unroll
     for (int a = 0; a < 4; ++a)
 #pragma unroll
-        for (int b = 0; b < 4; ++b) {
-            const int i = ti * GR_T + ty * 4 + a, j = tj * GR_T + tx * 4 + b;
-            if (i < k && j < k) P[(int64_t)i * k + j] = acc[a][b];
+        for (int b = 0; b < 2; ++b) {
+            if (!need[a][b]) continue;
+            const int i = ti * GR_T + wi * 32 + a * GR_S + g;
+            const int j = tj * GR_T + wj * 16 + b * GR_S + 2 * q;
+            if (i < k && j < k) P[(int64_t)i * k + j] = acc[a][b][0];
+            if (i < k && j + 1 < k) P[(int64_t)i * k + j + 1] = acc[a][b][1];
         }
 }
 
@@ -89,7 +122,7 @@ __global__ void gram_reduce_kernel(const RefreshDev *__restrict__ rd, const int3
     const int64_t total = (int64_t)k * k;
     for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
         const int i = (int)(e / k), j = (int)(e % k);
-        const bool upper = (j / GR_T) >= (i / GR_T);  // only tiles with tj >= ti were written
+        const bool upper = (j / GR_S) >= (i / GR_S);  // only sub-tiles on or above the diagonal were written
         const int64_t src = upper ? e : (int64_t)j * k + i;
         double s = 0.0;
         for (int c = 0; c < chunks; ++c) s += d.gpart[(int64_t)c * total + src];
