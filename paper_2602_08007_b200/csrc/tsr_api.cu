@@ -15,7 +15,9 @@ using namespace tsr;
 
 namespace {
 
-enum Kind : int { KT = 0, KC, KCS, KP, KA, KY, KZ, NKIND };
+// KR*: tall-times-small products of the refresh on tensor cores (three TF32 products): rows of side
+// 0 (m) or 1 (n) times R^{-1} into buf[1] / buf[2], and the final U = Q Wu, V = B^T Wv.
+enum Kind : int { KT = 0, KC, KCS, KP, KA, KY, KZ, KR01, KR02, KR12, KRU, KRV, NKIND };
 constexpr int TSR_NUM_STAGES = 6;  // refresh, G*V, core GEMM, core update, U*D, apply
 
 struct Block {
@@ -39,6 +41,8 @@ struct Block {
     double *tau = nullptr, *dvec = nullptr, *evec = nullptr;
     double2 *rot = nullptr;
     int2 *sweeps = nullptr, *groups = nullptr;
+    float *Xs = nullptr, *Bts = nullptr;   // TF32 operand planes (value truncated to TF32, remainder): rows, small matrix^T
+    bool tc_rows = false;                  // tall-times-small products of the refresh run on tensor cores
     int32_t *nsweeps = nullptr, *rank = nullptr;
     int rot_cap = 0, sweep_cap = 0;
     float *Uold = nullptr, *Vold = nullptr, *Ra = nullptr, *Rb = nullptr, *Rt = nullptr;   // moment re-expression
@@ -85,7 +89,7 @@ struct tsr_ctx {
     int max_r = 0, max_k = 0;
     uint64_t launches = 0;                     // kernels launched through this context
     int num_sms = 148;
-    int bn[NKIND] = {128, 128, 128, 128, 128, 128, 128};   // tile width of each GEMM kind
+    int bn[NKIND] = {128, 128, 128, 128, 128, 128, 128, 256, 256, 256, 256, 256};   // tile width of each GEMM kind
     bool profiling = false;
     cudaEvent_t ev[TSR_NUM_STAGES + 1] = {};   // stage boundaries of the last step (profiling only)
     bool ev_valid = false;
@@ -196,6 +200,10 @@ void layout(tsr_ctx *ctx, Arena &a, bool assign, size_t *step_end)
             void *xt = a.take((size_t)(2 * k * std::max(b.ml, b.nl)) * 2);
             if (assign) { b.Gt = (bf16 *)gt; b.Xt = (bf16 *)xt; }
         }
+        if (b.tc_rows) {
+            void *xs = a.take((size_t)(2 * mx * k) * 4), *bts = a.take((size_t)(2 * k * k) * 4);
+            if (assign) { b.Xs = (float *)xs; b.Bts = (float *)bts; }
+        }
         void *om = a.take((size_t)(n * k) * 4);
         void *b0 = a.take((size_t)(mx * k) * 4), *b1 = a.take((size_t)(mx * k) * 4), *b2 = a.take((size_t)(mx * k) * 4);
         void *S = a.take((size_t)(k * k) * 8), *Xw = a.take((size_t)(k * k) * 8), *Wj = a.take((size_t)(k * k) * 8);
@@ -226,7 +234,9 @@ void layout(tsr_ctx *ctx, Arena &a, bool assign, size_t *step_end)
     a.off = (a.off + 255) & ~(size_t)255;
 }
 
-void add_tiles(tsr_ctx *ctx, int kind, int bi, int M, int N, int K, int kb_per_split)
+// tri > 0: B is the transpose of an upper-triangular matrix, so the columns n0 .. of the product only
+// need the first n0 + bn entries of the contraction (tri = elements per K block).
+void add_tiles(tsr_ctx *ctx, int kind, int bi, int M, int N, int K, int kb_per_split, int tri = 0)
 {
     const int bn = ctx->bn[kind];
     const int bm = (kind == KA) ? 128 : 256;   // the grouped GEMM runs on CTA pairs: 256-row tiles
@@ -242,6 +252,7 @@ void add_tiles(tsr_ctx *ctx, int kind, int bi, int M, int N, int K, int kb_per_s
                 t.prob = bi; t.m0 = m0; t.n0 = n0;
                 t.kb0 = kb_per_split > 0 ? s * kb_per_split : 0;
                 t.kb1 = kb_per_split > 0 ? std::min(nkb, (s + 1) * kb_per_split) : nkb;
+                if (tri > 0) t.kb1 = std::min(nkb, (n0 + bn + tri - 1) / tri);
                 t.split = s;
                 v.push_back(t);
             }
@@ -268,6 +279,13 @@ void build_tiles(tsr_ctx *ctx)
         add_tiles(ctx, KA, bi, m, n, r, 0);
         add_tiles(ctx, KY, bi, m, k, n, 0);
         add_tiles(ctx, KZ, bi, n, k, m, 0);
+        if (b.tc_rows) {   // K blocks of 32 FP32 elements: pass 2 k so that the count comes out as ceil(k / 32)
+            add_tiles(ctx, KR01, bi, m, k, 2 * k, 0, 32);
+            add_tiles(ctx, KR02, bi, m, k, 2 * k, 0, 32);
+            add_tiles(ctx, KR12, bi, n, k, 2 * k, 0, 32);
+            add_tiles(ctx, KRU, bi, m, r, 2 * k, 0);
+            add_tiles(ctx, KRV, bi, n, r, 2 * k, 0);
+        }
     }
 }
 
@@ -285,6 +303,23 @@ tsr_status encode_map(tsr_ctx *ctx, CUtensorMap *out, const void *base, int64_t 
     if (rc != CUDA_SUCCESS)
         return fail(ctx, TSR_ERR_CUDA, "cuTensorMapEncodeTiled failed (%d) rows=%lld cols=%lld ld=%lld", (int)rc,
                     (long long)rows, (long long)cols, (long long)ld);
+    return TSR_OK;
+}
+
+// FP32 row-major [rows x cols] (ld elements) -> tensor map with a 32 x box_rows box (128 bytes of K), 128B swizzle.
+tsr_status encode_map_f32(tsr_ctx *ctx, CUtensorMap *out, const void *base, int64_t rows, int64_t cols, int64_t ld,
+                          int box_rows)
+{
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)ld * 4};
+    cuuint32_t box[2] = {32, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult rc = ctx->encode(out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void *>(base), dims, strides, box, estr,
+                              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (rc != CUDA_SUCCESS)
+        return fail(ctx, TSR_ERR_CUDA, "cuTensorMapEncodeTiled (FP32 operand) failed (%d) rows=%lld cols=%lld", (int)rc,
+                    (long long)rows, (long long)cols);
     return TSR_OK;
 }
 
@@ -488,14 +523,39 @@ struct RefreshLists {
     RowItem *ditems[5];
 };
 
-tsr_status orth_pass(tsr_ctx *ctx, const RefreshLists &L, int side, int src, int dst, cudaStream_t st)
+// dst = buf[src] * Mat for every block of the list (see rows_gemm_batched for the selectors).  Lists
+// whose blocks all qualify run on tensor cores: the rows and the transposed small matrix are split
+// into a TF32 plane and a remainder plane, and the product is three TF32 MMAs per K step.
+tsr_status rows_product(tsr_ctx *ctx, const RefreshLists &L, int side, int src, int mat, int dst, bool exact_not_needed,
+                        cudaStream_t st)
+{
+    const int nl = (int)L.list.size();
+    // The tensor cores accumulate with less than FP32 rounding accuracy (measured: bases came out
+    // orthonormal to 2e-4 instead of 1e-6), so the three products whose result is final -- the second
+    // Cholesky-QR pass and U, V -- stay on the FP32 CUDA-core kernel.
+    bool tc = exact_not_needed;
+    for (int bi : L.list) tc = tc && ctx->blocks[bi].tc_rows;
+    if (!tc) {
+        TSR_KERNEL(ctx, 1, rows_gemm_batched(ctx->d_refresh, L.ditems[side * 2], L.nitems[side * 2], side, src, mat, dst,
+                                             mat == 0 ? L.kmax : L.rmax, st));
+        return TSR_OK;
+    }
+    const int kind = (dst == 3) ? KRU : (dst == 4) ? KRV : (side == 1) ? KR12 : (dst == 1 ? KR01 : KR02);
+    if (side == 1 && dst != 2 && dst != 4) return fail(ctx, TSR_ERR_INVALID_ARG, "unexpected destination of a row product");
+    TSR_KERNEL(ctx, 2, split_operands_batched(ctx->d_refresh, L.ditems[side * 2], L.nitems[side * 2], L.dlist, nl, side, src,
+                                              mat, L.kmax, st));
+    StepScalars sc;
+    memset(&sc, 0, sizeof sc);
+    return launch_kind(ctx, kind, L.list, EPI_STORE_F32, 3, sc, st);
+}
+
+tsr_status orth_pass(tsr_ctx *ctx, const RefreshLists &L, int side, int src, int dst, bool refined_later, cudaStream_t st)
 {
     const int nl = (int)L.list.size();
     TSR_KERNEL(ctx, 2, gram_batched(ctx->d_refresh, L.ditems[side * 2 + 1], L.nitems[side * 2 + 1], L.dlist, nl, side,
                                src, L.kmax, st));
     TSR_KERNEL(ctx, 1, chol_inverse_batched(ctx->d_refresh, L.dlist, nl, L.kmax, st));
-    TSR_KERNEL(ctx, 1, rows_gemm_batched(ctx->d_refresh, L.ditems[side * 2], L.nitems[side * 2], side, src, 0, dst, L.kmax, st));
-    return TSR_OK;
+    return rows_product(ctx, L, side, src, 0, dst, refined_later, st);
 }
 
 // orth(buf[0]) -> buf[2] by Cholesky-QR with the Gram matrix accumulated in FP64.
@@ -506,9 +566,9 @@ tsr_status orth_pass(tsr_ctx *ctx, const RefreshLists &L, int side, int src, int
 tsr_status orth(tsr_ctx *ctx, const RefreshLists &L, int side, bool final, cudaStream_t st)
 {
     tsr_status s;
-    if (!final) return orth_pass(ctx, L, side, 0, 2, st);
-    if ((s = orth_pass(ctx, L, side, 0, 1, st)) != TSR_OK) return s;
-    return orth_pass(ctx, L, side, 1, 2, st);
+    if (!final) return orth_pass(ctx, L, side, 0, 2, true, st);
+    if ((s = orth_pass(ctx, L, side, 0, 1, true, st)) != TSR_OK) return s;
+    return orth_pass(ctx, L, side, 1, 2, false, st);
 }
 
 // buf[0] (rows_out x k) = G X  (transposed = false, X = buf[2] or Omega, n x k)
@@ -596,12 +656,17 @@ tsr_status do_refresh_group(tsr_ctx *ctx, const std::vector<int> &list, uint64_t
     const int nl = (int)list.size();
     TSR_KERNEL(ctx, 2, gram_batched(ctx->d_refresh, L.ditems[3], L.nitems[3], L.dlist, nl, 1, 0, L.kmax, st));
     if (L.kmax >= 200) {   // too large for the Jacobi solver: tridiagonal route
-        const int pr = eig_panel_rows(L.kmax);
+        const int pr = eig_panel_rows(L.kmax), qr = eig_qrows_rows(L.kmax);
         std::vector<RowItem> panels;
         for (int bi : list)
             for (int r0 = 0; r0 < ctx->blocks[bi].k; r0 += pr) panels.push_back({bi, r0});
+        const size_t npan = panels.size();
+        if (qr > 0)
+            for (int bi : list)
+                for (int r0 = 0; r0 < ctx->blocks[bi].k; r0 += qr) panels.push_back({bi, r0});
         TSR_CUDA(ctx, cudaMemcpyAsync(L.ditems[4], panels.data(), panels.size() * sizeof(RowItem), cudaMemcpyHostToDevice, st));
-        TSR_KERNEL(ctx, 4, eig_tridiag_batched(ctx->d_refresh, L.dlist, nl, L.ditems[4], (int)panels.size(), L.kmax, st));
+        TSR_KERNEL(ctx, 5, eig_tridiag_batched(ctx->d_refresh, L.dlist, nl, L.ditems[4], (int)npan, L.ditems[4] + npan,
+                                               (int)(panels.size() - npan), L.kmax, st));
     } else {
         TSR_KERNEL(ctx, 1, jacobi_batched(ctx->d_refresh, L.dlist, nl, 40, st));
     }
@@ -613,8 +678,8 @@ tsr_status do_refresh_group(tsr_ctx *ctx, const std::vector<int> &list, uint64_t
             TSR_CUDA(ctx, cudaMemcpyAsync(b.Uold, b.p.U, (size_t)b.d.m * b.d.r * 4, cudaMemcpyDeviceToDevice, st));
             TSR_CUDA(ctx, cudaMemcpyAsync(b.Vold, b.p.V, (size_t)b.d.n * b.d.r * 4, cudaMemcpyDeviceToDevice, st));
         }
-    TSR_KERNEL(ctx, 1, rows_gemm_batched(ctx->d_refresh, L.ditems[2], L.nitems[2], 1, 0, 2, 4, L.rmax, st));
-    TSR_KERNEL(ctx, 1, rows_gemm_batched(ctx->d_refresh, L.ditems[0], L.nitems[0], 0, 2, 1, 3, L.rmax, st));
+    if ((s = rows_product(ctx, L, 1, 0, 2, 4, false, st)) != TSR_OK) return s;
+    if ((s = rows_product(ctx, L, 0, 2, 1, 3, false, st)) != TSR_OK) return s;
     if (reexpress)   // M <- (Unew^T Uold) M (Vold^T Vnew)
         for (int bi : list) {
             Block &b = ctx->blocks[bi];
@@ -782,6 +847,7 @@ tsr_status tsr_create(tsr_ctx **out, const tsr_mat_desc *descs, int32_t count)
         // Candidate for the tensor-core path: BF16 gradient with 16-byte row pitches.  Pointer
         // alignment is checked at bind time.
         b.fast = (b.d.g_dtype == TSR_BF16) && ((b.d.ldg * 2) % 16 == 0) && ((b.d.ldw * 4) % 16 == 0);
+        b.tc_rows = b.fast && (b.k % 4 == 0);   // FP32 rows of k elements as a TMA operand: 16-byte row pitch
         const int nkb = (int)((b.d.m + 63) / 64);
         if (nkb > 128) { b.kb_per_split = 32; b.nsplit = (nkb + 31) / 32; }
         ctx->max_r = std::max(ctx->max_r, (int)b.d.r);
@@ -845,7 +911,7 @@ tsr_status tsr_bind(tsr_ctx *ctx, const tsr_mat_ptrs *ptrs, int32_t count, void 
         b.p = ptrs[i];
         const bool cand = (b.d.g_dtype == TSR_BF16) && ((b.d.ldg * 2) % 16 == 0) && ((b.d.ldw * 4) % 16 == 0);
         const bool fast = cand && aligned16(b.p.G) && aligned16(b.p.W);
-        if (fast != b.fast) { b.fast = fast; layout_changed = true; }
+        if (fast != b.fast) { b.fast = fast; b.tc_rows = fast && (b.k % 4 == 0); layout_changed = true; }
     }
     if (layout_changed) {   // a misaligned pointer moved a block to the CUDA-core path
         build_tiles(ctx);
@@ -898,6 +964,7 @@ tsr_status tsr_bind(tsr_ctx *ctx, const tsr_mat_ptrs *ptrs, int32_t count, void 
         rd.m = (int)m; rd.n = (int)n; rd.k = (int)k; rd.r = (int)r;
         for (int j = 0; j < 3; ++j) rd.buf[j] = b.buf[j];
         rd.S = b.S; rd.Xw = b.Xw; rd.Wj = b.Wj; rd.gpart = b.gpart; rd.lam = b.lam;
+        rd.Xs = b.Xs; rd.Bts = b.Bts;
         rd.Rinv = b.Rinv; rd.Wu = b.Wu; rd.Wv = b.Wv; rd.U = b.p.U; rd.V = b.p.V; rd.status = ctx->d_status + i;
         rd.tau = b.tau; rd.dvec = b.dvec; rd.evec = b.evec; rd.rot = b.rot; rd.sweeps = b.sweeps; rd.groups = b.groups; rd.nsweeps = b.nsweeps;
         rd.rank = b.rank; rd.rot_cap = b.rot_cap; rd.sweep_cap = b.sweep_cap;
@@ -951,6 +1018,19 @@ tsr_status tsr_bind(tsr_ctx *ctx, const tsr_mat_ptrs *ptrs, int32_t count, void 
             if ((s = encode_map(ctx, &P.tmA, b.Gt, n, m, b.ml, 128)) != TSR_OK) return s;
             if ((s = encode_map(ctx, &P.tmB, b.Xt, 2 * k, m, b.ml, 64)) != TSR_OK) return s;
             P.out = b.buf[0]; P.ld_out = k;
+        }
+        if (b.tc_rows) {   // rows [M x k] (planes Xs) times small matrix^T planes Bts [N x k]
+            const int64_t mx = std::max(m, n);
+            struct { int kd; int64_t M, N; float *out; } rk[5] = {
+                {KR01, m, k, b.buf[1]}, {KR02, m, k, b.buf[2]}, {KR12, n, k, b.buf[2]}, {KRU, m, r, b.p.U}, {KRV, n, r, b.p.V}};
+            for (const auto &e : rk) {
+                UmmaProblem &P = probs[e.kd][i];
+                base(P, (int)e.M, (int)e.N, (int)k, EPI_STORE_F32);
+                P.planes = 3; P.plane_rows = (int)k; P.a_plane_rows = (int)mx;
+                if ((s = encode_map_f32(ctx, &P.tmA, b.Xs, 2 * mx, k, k, 128)) != TSR_OK) return s;
+                if ((s = encode_map_f32(ctx, &P.tmB, b.Bts, 2 * k, k, k, ctx->bn[e.kd] / 2)) != TSR_OK) return s;
+                P.out = e.out; P.ld_out = e.N;
+            }
         }
     }
     for (int kd = 0; kd < NKIND; ++kd) {

@@ -364,7 +364,8 @@ __global__ void eig_rank_kernel(const RefreshDev *__restrict__ rd, const int32_t
 // 3a: rows of Q = H_0 H_1 ... in registers.  A warp owns RQ rows (NW warps per CTA); lane holds columns lane + 32 i.
 // The reflectors are staged for the whole CTA, a few at a time, in shared memory.
 constexpr int SYS_KMAX = 1056;
-constexpr int SYS_WARPS = 8;
+constexpr int SYS_WARPS = 12;    // warps of the rotation kernel (three per scheduler)
+constexpr int QR_WARPS = 16;     // warps of the Q-rows kernel
 
 template <int NCH, int RQ, int NW>
 __global__ void __launch_bounds__(NW * 32)
@@ -533,6 +534,8 @@ eig_rot_systolic_kernel(const RefreshDev *__restrict__ rd, const RowItem *__rest
 
 static int sys_rows_per_warp(int kmax) { return kmax <= 544 ? 4 : 2; }
 
+int eig_qrows_rows(int kmax) { return kmax <= SYS_KMAX ? QR_WARPS * (kmax <= 544 ? 2 : 1) : 0; }
+
 int eig_panel_rows(int kmax)
 {
     if (kmax <= SYS_KMAX) return SYS_WARPS * sys_rows_per_warp(kmax);
@@ -562,7 +565,7 @@ static cudaError_t raise_smem(F *fn, size_t bytes, size_t *configured)
 }
 
 cudaError_t eig_tridiag_batched(const RefreshDev *rd, const int32_t *list, int nlist, const RowItem *panel_items,
-                                int npanels, int kmax, cudaStream_t stream)
+                                int npanels, const RowItem *qrows_items, int nqrows, int kmax, cudaStream_t stream)
 {
     if (nlist <= 0) return cudaSuccess;
     const int kpad = kmax + 8;
@@ -574,10 +577,9 @@ cudaError_t eig_tridiag_batched(const RefreshDev *rd, const int32_t *list, int n
     const size_t ql_bytes = (size_t)2 * kmax * sizeof(double);
     if (kmax <= SYS_KMAX) {
         const int threads = SYS_WARPS * 32;
-        // same row slabs as the rotation kernel (32 or 16 rows), spread over 16 warps
-        if (kmax <= 288) eig_qrows_kernel<9, 2, 16><<<npanels, 512, 0, stream>>>(rd, panel_items);
-        else if (kmax <= 544) eig_qrows_kernel<17, 2, 16><<<npanels, 512, 0, stream>>>(rd, panel_items);
-        else eig_qrows_kernel<33, 1, 16><<<npanels, 512, 0, stream>>>(rd, panel_items);
+        if (kmax <= 288) eig_qrows_kernel<9, 2, QR_WARPS><<<nqrows, QR_WARPS * 32, 0, stream>>>(rd, qrows_items);
+        else if (kmax <= 544) eig_qrows_kernel<17, 2, QR_WARPS><<<nqrows, QR_WARPS * 32, 0, stream>>>(rd, qrows_items);
+        else eig_qrows_kernel<33, 1, QR_WARPS><<<nqrows, QR_WARPS * 32, 0, stream>>>(rd, qrows_items);
         ql_log_kernel<true><<<nlist, 32, ql_bytes, stream>>>(rd, list);
         eig_rank_kernel<<<nlist, 256, 0, stream>>>(rd, list);
         const int R = sys_rows_per_warp(kmax);

@@ -20,7 +20,8 @@ inline int64_t round_up(int64_t x, int64_t a) { return (x + a - 1) / a * a; }
 // ---------------------------------------------------------------------------------------
 // Tensor-core grouped GEMM:  D[M x N] = A[M x K] * B[N x K]^T, both operands BF16 with K
 // contiguous ("K-major"), FP32 accumulation in tensor memory.  B may come as two planes
-// (hi + lo) that are accumulated into the same D.
+// (hi + lo) that are accumulated into the same D.  planes = 3 selects FP32 data as three TF32
+// products (both operands in a truncated and a remainder plane, K blocks of 32 elements).
 // ---------------------------------------------------------------------------------------
 enum UmmaEpilogue : int {
     EPI_STORE_F32 = 0,     // out_f32[row * ld + col] = acc
@@ -39,7 +40,7 @@ struct alignas(64) UmmaProblem {
     int32_t plane_rows;    // row offset of the second plane inside the B tensor map
     int32_t block;         // plan index of the matrix block (for status words)
     int32_t epilogue;      // UmmaEpilogue
-    int32_t pad0;
+    int32_t a_plane_rows;  // three-product mode: row offset of the remainder plane inside the A tensor map
     void *out;             // EPI_STORE_*: destination; EPI_APPLY: W; EPI_CORE_UPDATE: C (split-K: partial buffer)
     int64_t ld_out;
     int64_t split_stride;  // elements between split-K partial slabs (EPI_STORE_F32 with split tiles)
@@ -126,6 +127,7 @@ struct RefreshDev {
     double *lam;        // k eigenvalues, descending
     float *Rinv;        // k x k
     float *Wu, *Wv;     // k x r
+    float *Xs, *Bts;    // TF32 operand planes of the tensor-core row products (may be NULL)
     float *U, *V;       // the block's bases (FP32 masters)
     int32_t *status;    // the block's status word
     // tridiagonal eigen-solver (tsr_eig.cu)
@@ -153,14 +155,20 @@ cudaError_t chol_inverse_batched(const RefreshDev *rd, const int32_t *list, int 
 // dst_sel: 0..2 buf[], 3 = U, 4 = V.
 cudaError_t rows_gemm_batched(const RefreshDev *rd, const RowItem *items, int nitems, int side, int src_sel,
                               int mat_sel, int dst_sel, int nmax, cudaStream_t stream);
+// Operand planes for the tensor-core form of the product above: every value as a TF32 part and a
+// remainder; rows of buf[src_sel] into Xs, the transposed small matrix into Bts.
+cudaError_t split_operands_batched(const RefreshDev *rd, const RowItem *items, int nitems, const int32_t *list, int nlist,
+                                   int side, int src_sel, int mat_sel, int kmax, cudaStream_t stream);
 // Eigen-decomposition of S by cyclic Jacobi, descending sort, Wu = W[:, :r], Wv = W[:, :r] / sqrt(lambda).
 // The same result through Householder tridiagonalisation + implicit QL with logged rotations
 // (for k too large for the Jacobi solver).  panel_items: (block, row0) slabs of eig_panel_rows(kmax)
 // rows of the k x k eigenvector matrix.  eig_rot_capacity(k): entries of the rotation log to provide.
+// qrows_items: slabs of eig_qrows_rows(kmax) rows for the kernel that forms the rows of Q (0: not used).
 int eig_panel_rows(int kmax);
+int eig_qrows_rows(int kmax);
 int64_t eig_rot_capacity(int k);
 cudaError_t eig_tridiag_batched(const RefreshDev *rd, const int32_t *list, int nlist, const RowItem *panel_items,
-                                int npanels, int kmax, cudaStream_t stream);
+                                int npanels, const RowItem *qrows_items, int nqrows, int kmax, cudaStream_t stream);
 cudaError_t jacobi_batched(const RefreshDev *rd, const int32_t *list, int nlist, int max_sweeps, cudaStream_t stream);
 
 }  // namespace tsr

@@ -474,6 +474,74 @@ cudaError_t rows_gemm_batched(const RefreshDev *rd, const RowItem *items, int ni
 }
 
 // ---------------------------------------------------------------------------------------
+// Operand planes for the tensor-core form of dst = buf[src] * Mat (three TF32 products).
+// Every FP32 value x is written as hi = x with the low 13 mantissa bits cleared (a TF32 number) and
+// lo = x - hi (exact).  Rows: Xs[row][c] = hi, Xs[mx + row][c] = lo with mx = max(m, n).
+// Small matrix, transposed so that the contraction index is contiguous: Bts[j][l] = hi(Mat[l][j]),
+// Bts[k + j][l] = lo(Mat[l][j]).
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ float tf32_hi(float x) { return __uint_as_float(__float_as_uint(x) & 0xffffe000u); }
+
+__global__ void __launch_bounds__(256)
+split_rows_kernel(const RefreshDev *__restrict__ rd, const RowItem *__restrict__ items, int side, int src_sel)
+{
+    const RowItem it = items[blockIdx.x];
+    const RefreshDev d = rd[it.block];
+    const int k = d.k;
+    const int rows = side ? d.n : d.m;
+    const int64_t mx = max(d.m, d.n);
+    const int nrow = min(RG_ROWS, rows - it.row0);
+    const float4 *__restrict__ X = (const float4 *)(d.buf[src_sel] + (int64_t)it.row0 * k);
+    float4 *__restrict__ H = (float4 *)(d.Xs + (int64_t)it.row0 * k);
+    float4 *__restrict__ Lo = (float4 *)(d.Xs + (mx + it.row0) * k);
+    const int n4 = nrow * k / 4;                  // k is a multiple of 4 on this path
+    for (int e = threadIdx.x; e < n4; e += 256) {
+        const float4 x = X[e];
+        float4 h, l;
+        h.x = tf32_hi(x.x); h.y = tf32_hi(x.y); h.z = tf32_hi(x.z); h.w = tf32_hi(x.w);
+        l.x = x.x - h.x; l.y = x.y - h.y; l.z = x.z - h.z; l.w = x.w - h.w;
+        H[e] = h;
+        Lo[e] = l;
+    }
+}
+
+__global__ void __launch_bounds__(256)
+split_mat_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ list, int mat_sel)
+{
+    const RefreshDev d = rd[list[blockIdx.z]];
+    const int k = d.k;
+    const int N = (mat_sel == 0) ? d.k : d.r;
+    const int l0 = blockIdx.y * 32, j0 = blockIdx.x * 32;   // Mat[l][j], l < k, j < N
+    if (l0 >= k || j0 >= N) return;
+    const float *__restrict__ M = (mat_sel == 0) ? d.Rinv : (mat_sel == 1 ? d.Wu : d.Wv);
+    __shared__ float t[32][33];
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    for (int a = ty; a < 32; a += 8) {
+        const int l = l0 + a, j = j0 + tx;
+        t[a][tx] = (l < k && j < N) ? M[(int64_t)l * N + j] : 0.f;
+    }
+    __syncthreads();
+    for (int a = ty; a < 32; a += 8) {
+        const int j = j0 + a, l = l0 + tx;
+        if (j < N && l < k) {
+            const float x = t[tx][a], h = tf32_hi(x);
+            d.Bts[(int64_t)j * k + l] = h;
+            d.Bts[(int64_t)(k + j) * k + l] = x - h;
+        }
+    }
+}
+
+cudaError_t split_operands_batched(const RefreshDev *rd, const RowItem *items, int nitems, const int32_t *list, int nlist,
+                                   int side, int src_sel, int mat_sel, int kmax, cudaStream_t stream)
+{
+    if (nitems <= 0 || nlist <= 0) return cudaSuccess;
+    split_rows_kernel<<<nitems, 256, 0, stream>>>(rd, items, side, src_sel);
+    const int t = (kmax + 31) / 32;
+    split_mat_kernel<<<dim3(t, t, nlist), 256, 0, stream>>>(rd, list, mat_sel);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------
 // Cyclic Jacobi eigen-solver for a symmetric k x k matrix (FP64), one CTA per matrix.
 // Round-robin ordering: every round rotates k/2 disjoint index pairs at once; the two-sided
 // update S <- J^T S J is done on 2 x 2 blocks (pair A rows x pair B columns), the eigenvector

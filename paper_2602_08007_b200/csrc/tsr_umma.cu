@@ -40,11 +40,18 @@ namespace tsr {
 constexpr int UG_THREADS = 384;   // warps 0-1: TMA / MMA, warps 2-3 idle, warps 4-11: epilogue
 constexpr int UG_EPI_WARPS = 8;
 
+// PLANES = 1, 2: BF16 operands, B in one or two planes (hi + lo) accumulated into the same D.
+// PLANES = 3: FP32 data as three TF32 products.  A and B each come as a plane of values truncated
+// to TF32 and a plane of remainders (both FP32 containers, K blocks of 32 elements); D accumulates
+// A_hi B_hi + A_hi B_lo + A_lo B_hi, which carries about 21 mantissa bits of each operand.
 template <int BN, int PLANES>
 struct UmmaSmem {
-    static constexpr int A_BYTES = UM_BM * UM_BK * 2;
-    static constexpr int B_BYTES = (BN / 2) * UM_BK * 2;   // each CTA of the pair stages half of the B rows
-    static constexpr int STAGE_BYTES = A_BYTES + PLANES * B_BYTES;
+    static constexpr int A_PLANES = PLANES == 3 ? 2 : 1;
+    static constexpr int B_PLANES = PLANES == 3 ? 2 : PLANES;
+    static constexpr int BK_ELEMS = PLANES == 3 ? 32 : UM_BK;        // elements per 128-byte K block
+    static constexpr int A_BYTES = UM_BM * 128;                       // one plane of this CTA's A rows
+    static constexpr int B_BYTES = (BN / 2) * 128;                    // each CTA of the pair stages half of the B rows
+    static constexpr int STAGE_BYTES = A_PLANES * A_BYTES + B_PLANES * B_BYTES;
     static constexpr int STAGES = (192 * 1024) / STAGE_BYTES > 6 ? 6 : (192 * 1024) / STAGE_BYTES;
     static constexpr int PATCH_OFFSET = STAGES * STAGE_BYTES;
     static constexpr int PATCH_BYTES = 32 * 33 * 4;                  // per epilogue warp
@@ -111,11 +118,14 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
                     const uint32_t full = leader_addr(smem_u32(bar_full + s));
                     if (rank == 0) mbar_expect_tx(smem_u32(bar_full + s), 2u * (uint32_t)SM::STAGE_BYTES);
                     uint8_t *st = smem + s * SM::STAGE_BYTES;
-                    tma_load_2d_pair(smem_u32(st), &P->tmA, full, kb * UM_BK, tile.m0 + (int)rank * UM_BM);
 #pragma unroll
-                    for (int pl = 0; pl < PLANES; ++pl)
-                        tma_load_2d_pair(smem_u32(st + SM::A_BYTES + pl * SM::B_BYTES), &P->tmB, full, kb * UM_BK,
-                                         b_row + pl * P->plane_rows);
+                    for (int pl = 0; pl < SM::A_PLANES; ++pl)
+                        tma_load_2d_pair(smem_u32(st + pl * SM::A_BYTES), &P->tmA, full, kb * SM::BK_ELEMS,
+                                         tile.m0 + (int)rank * UM_BM + pl * P->a_plane_rows);
+#pragma unroll
+                    for (int pl = 0; pl < SM::B_PLANES; ++pl)
+                        tma_load_2d_pair(smem_u32(st + SM::A_PLANES * SM::A_BYTES + pl * SM::B_BYTES), &P->tmB, full,
+                                         kb * SM::BK_ELEMS, b_row + pl * P->plane_rows);
                 }
             }
         }
@@ -127,7 +137,7 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
                 const UmmaTile tile = tiles[t];
                 int n_eff = probs[tile.prob].N - tile.n0;
                 n_eff = n_eff >= BN ? BN : ((n_eff + 15) & ~15);
-                const uint32_t idesc = umma_idesc_pair(n_eff);
+                const uint32_t idesc = PLANES == 3 ? umma_idesc_pair_tf32(n_eff) : umma_idesc_pair(n_eff);
                 const uint32_t buf = tc & 1u;
                 if (!mbar_wait(smem_u32(bar_acc_empty + buf), ((tc >> 1) & 1u) ^ 1u)) { s_timeout = 1; ok = false; break; }
                 tc_fence_after();
@@ -138,13 +148,26 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
                     if (!mbar_wait(smem_u32(bar_full + s), ph)) { s_timeout = 1; ok = false; break; }
                     tc_fence_after();
                     const uint32_t a_base = smem_u32(smem + s * SM::STAGE_BYTES);
+                    if (PLANES == 3) {
+                        // (A plane, B plane) = (hi, hi), (hi, lo), (lo, hi); 32 bytes of K per instruction
 #pragma unroll
-                    for (int pl = 0; pl < PLANES; ++pl) {
-                        const uint32_t b_base = a_base + SM::A_BYTES + pl * SM::B_BYTES;
+                        for (int pr = 0; pr < 3; ++pr) {
+                            const uint32_t a_pl = a_base + (pr == 2 ? SM::A_BYTES : 0);
+                            const uint32_t b_pl = a_base + 2 * SM::A_BYTES + (pr == 1 ? SM::B_BYTES : 0);
 #pragma unroll
-                        for (int k4 = 0; k4 < UM_BK / 16; ++k4)
-                            tc_mma_bf16_pair(d_tmem, umma_desc_sw128(a_base + k4 * 32), umma_desc_sw128(b_base + k4 * 32),
-                                             idesc, ((kb - tile.kb0) | pl | k4) ? 1u : 0u);
+                            for (int k4 = 0; k4 < 4; ++k4)
+                                tc_mma_tf32_pair(d_tmem, umma_desc_sw128(a_pl + k4 * 32), umma_desc_sw128(b_pl + k4 * 32),
+                                                 idesc, ((kb - tile.kb0) | pr | k4) ? 1u : 0u);
+                        }
+                    } else {
+#pragma unroll
+                        for (int pl = 0; pl < SM::B_PLANES; ++pl) {
+                            const uint32_t b_base = a_base + SM::A_BYTES + pl * SM::B_BYTES;
+#pragma unroll
+                            for (int k4 = 0; k4 < UM_BK / 16; ++k4)
+                                tc_mma_bf16_pair(d_tmem, umma_desc_sw128(a_base + k4 * 32), umma_desc_sw128(b_base + k4 * 32),
+                                                 idesc, ((kb - tile.kb0) | pl | k4) ? 1u : 0u);
+                        }
                     }
                     tc_commit_pair(smem_u32(bar_empty + s));       // frees the stage in both CTAs
                 }
@@ -357,6 +380,7 @@ cudaError_t umma_configure()
     if ((e = configure_one<128, EPI_STORE_F32, 1>()) != cudaSuccess) return e;
     if ((e = configure_one<256, EPI_STORE_F32, 1>()) != cudaSuccess) return e;
     if ((e = configure_one<128, EPI_STORE_F32, 2>()) != cudaSuccess) return e;
+    if ((e = configure_one<256, EPI_STORE_F32, 3>()) != cudaSuccess) return e;
     if ((e = configure_one<128, EPI_STORE_BF16, 1>()) != cudaSuccess) return e;
     if ((e = configure_one<256, EPI_STORE_BF16, 1>()) != cudaSuccess) return e;
     if ((e = configure_one<128, EPI_STORE_BF16_T, 1>()) != cudaSuccess) return e;
@@ -373,6 +397,10 @@ cudaError_t umma_gemm_launch(const UmmaProblem *probs, const UmmaTile *tiles, in
 #define TSR_UG(BN_, EPI_, PL_) return launch_one<BN_, EPI_, PL_>(probs, tiles, num_tiles, num_sms, sc, status, stream)
     if (planes == 2) {
         if (bn == 128 && epilogue == EPI_STORE_F32) TSR_UG(128, EPI_STORE_F32, 2);
+        return cudaErrorInvalidValue;
+    }
+    if (planes == 3) {
+        if (bn == 256 && epilogue == EPI_STORE_F32) TSR_UG(256, EPI_STORE_F32, 3);
         return cudaErrorInvalidValue;
     }
     if (bn == 128) {

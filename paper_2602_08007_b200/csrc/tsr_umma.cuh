@@ -88,6 +88,17 @@ __device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint64_t adesc
         ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
+// The same on TF32 operands (32-bit containers, K = 8 per instruction).
+__device__ __forceinline__ void tc_mma_tf32_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                                 uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
 // Arrives, once all MMAs issued so far have completed, on the barrier at the same address in BOTH CTAs.
 __device__ __forceinline__ void tc_commit_pair(uint32_t bar)
 {
@@ -104,6 +115,11 @@ __device__ __forceinline__ void mbar_arrive_leader(uint32_t bar)
 __host__ __device__ constexpr uint32_t umma_idesc_pair(int bn)
 {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+}
+// TF32 operands (format code 2), FP32 accumulator.
+__host__ __device__ constexpr uint32_t umma_idesc_pair_tf32(int bn)
+{
+    return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
 }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
