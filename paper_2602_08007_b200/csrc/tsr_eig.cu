@@ -141,6 +141,16 @@ constexpr int SYS_LAG = 2;                        // steps between neighbouring 
 constexpr int SYS_FILL = SYS_LAG * 31;            // steps until the last lane sees the first column
 constexpr int SYS_PF = 8;                         // steps of rotations the reader fetches ahead
 
+// 1 / sqrt(x) for a positive, normal x: hardware estimate (about 22 bits) and one third-order
+// correction, which leaves an error of a few units of 2^-53; no special-case branches.
+__device__ __forceinline__ double rsqrt_nocheck(double x)
+{
+    double y;
+    asm("rsqrt.approx.ftz.f64 %0, %1;" : "=d"(y) : "d"(x));
+    const double e = fma(-x * y, y, 1.0);
+    return fma(y * e, fma(0.375, e, 0.5), y);
+}
+
 template <bool SKEW>
 __global__ void __launch_bounds__(32)
 ql_log_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ list)
@@ -187,27 +197,37 @@ ql_log_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ lis
                 const int first = nrot;
                 int i = m - 1;
                 bool early = false;
-                double e_nx = e[i], d_nx = d[i];      // fetched one rotation ahead of the stores below
+                // The loop is one dependent chain g -> r2 -> 1/sqrt(r2) -> g.  Everything that does not need
+                // the reciprocal square root is formed before it: with rinv = 1/sqrt(f^2 + g^2),
+                // s = f rinv, c = g rinv, (d[i] - g1) s + 2 c b = u rinv with u = (d[i] - g1) f + 2 g b,
+                // so p = s (u rinv) = f u rinv^2 and the next g = c (u rinv) - b = g u rinv^2 - b.
+                // d[i+1] and the next d[i], e[i] travel in registers (fetched ahead of the stores).
+                double e_nx = e[i], d_nx = d[i], dprev = d[m];
+                double2 *lr = SKEW ? lane_rot + (int64_t)(n - 1 - i) * 32 : rot + nrot;
                 for (; i >= l; --i) {
                     const double ei = e_nx, di = d_nx;
                     if (i > l) { e_nx = e[i - 1]; d_nx = d[i - 1]; }
                     const double f = s * ei, b = c * ei;
                     // r = hypot(f, g).  The entries are bounded by the eigenvalues of a Gram matrix of FP32
                     // data, so the squares stay far inside the FP64 range and no rescaling is needed.
-                    const double r2 = f * f + g * g;
-                    if (r2 == 0.0) { e[i + 1] = 0.0; d[i + 1] -= p; e[m] = 0.0; early = true; break; }
-                    const double rinv = rsqrt(r2);
-                    r = r2 * rinv;
-                    e[i + 1] = r;
+                    const double r2 = fma(f, f, g * g);
+                    if (r2 == 0.0) { e[i + 1] = 0.0; d[i + 1] = dprev - p; e[m] = 0.0; early = true; break; }
+                    const double g1 = dprev - p;
+                    const double u = fma(di - g1, f, 2.0 * g * b);
+                    const double gu = g * u, fu = f * u;
+                    const double rinv = rsqrt_nocheck(r2);
+                    const double rinv2 = rinv * rinv;
+                    const double gn = fma(gu, rinv2, -b);     // the chain continues here
+                    p = fu * rinv2;
                     s = f * rinv;
                     c = g * rinv;
-                    g = d[i + 1] - p;
-                    r = (di - g) * s + 2.0 * c * b;
-                    p = s * r;
-                    d[i + 1] = g + p;
-                    g = c * r - b;
-                    if (SKEW) { lane_rot[(int64_t)(n - 1 - i) * 32] = make_double2(c, s); ++nrot; }
-                    else rot[nrot++] = make_double2(c, s);
+                    g = gn;
+                    e[i + 1] = r2 * rinv;
+                    d[i + 1] = g1 + p;
+                    *lr = make_double2(c, s);
+                    lr += SKEW ? 32 : 1;
+                    ++nrot;
+                    dprev = di;
                 }
                 if (nrot > first) sweeps[nsw++] = make_int2(m - 1, nrot - first);
                 if (early) continue;
