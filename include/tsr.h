@@ -61,7 +61,7 @@ typedef struct tsr_ctx tsr_ctx; /* opaque plan: shapes, bound pointers, device t
 typedef enum {
     TSR_OK = 0,
     TSR_ERR_INVALID_ARG = 1,    /* null pointer, bad index, bad enum                      */
-    TSR_ERR_SHAPE = 2,          /* non-positive size, ld < cols, r + p > min(m, n)        */
+    TSR_ERR_SHAPE = 2,          /* non-positive size, ld < cols, r + p > min(m, n) or > 1056 */
     TSR_ERR_ALIGNMENT = 3,      /* a pointer that must be 16-byte aligned is not          */
     TSR_ERR_WORKSPACE = 4,      /* workspace missing or too small                         */
     TSR_ERR_CUDA = 5,           /* a CUDA runtime / driver call failed, or no device      */
@@ -92,7 +92,7 @@ typedef struct {
     int64_t m, n;         /* rows, columns of G and W                                   */
     int64_t ldg, ldw;     /* leading dimensions of G and W in elements (>= n)           */
     int32_t r;            /* rank of the bases                                          */
-    int32_t p;            /* oversampling: sketches have k = r + p columns, k <= min(m,n) */
+    int32_t p;            /* oversampling: sketches have k = r + p columns, k <= min(m,n), k <= 1056 */
     int32_t q;            /* power iterations in the refresh (>= 0)                     */
     int32_t K;            /* refresh when step % K == 0; K <= 0 disables in-loop refresh */
     int32_t g_dtype;      /* tsr_dtype of G                                             */

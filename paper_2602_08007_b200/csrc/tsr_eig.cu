@@ -6,12 +6,11 @@
 //      reflectors are kept in the rows of S above the first superdiagonal);
 //   2. implicit-shift QL iteration on (d, e) alone, one thread per matrix, which LOGS every
 //      plane rotation instead of applying it;
-//   3. the eigenvectors W = Q Z: every warp takes a panel of rows of the identity into shared
-//      memory (lane = row), runs them through the reflectors (giving rows of Q) and then through
-//      the logged rotations, and writes the leading r columns in descending eigenvalue order:
-//      Wu = W[:, :r] and Wv = W[:, :r] / sqrt(lambda).
-// Rows are independent under right-multiplication, so stage 3 needs no synchronisation and
-// the rotations never touch global memory.
+//   3. the eigenvectors W = Q Z, row slab by row slab (rows are independent under
+//      right-multiplication): a first kernel forms the rows of Q from the reflectors with the
+//      rows held in registers; a second one streams every row through the logged rotations as
+//      a systolic pipeline over the lanes of a warp (32 sweeps advance per step) and writes the
+//      leading r columns in descending eigenvalue order: Wu = W[:, :r], Wv = W[:, :r] / sqrt(lambda).
 // Failure to converge within the iteration or log budget flags TSR_ERR_NOT_CONVERGED.
 #include "tsr_internal.h"
 
@@ -129,8 +128,7 @@ tridiag_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ li
 // e[i] couples d[i] and d[i+1].  Sweep header: x = index of the first rotation (m - 1), y = count;
 // rotation t of a sweep acts on columns (x - t, x - t + 1).
 //
-// Two log layouts.  SKEW = false: rotations in the order they are generated.  SKEW = true: the
-// layout the systolic eigenvector kernel reads.  Sweeps are taken in groups of 32 (sweep s is lane
+// The log is written in the layout the systolic eigenvector kernel reads.  Sweeps are taken in groups of 32 (sweep s is lane
 // s % 32 of group s / 32).  A group streams the columns k-1, k-2, ..., lg of a row through the 32
 // lanes, lane t two steps behind lane t-1, so lane t meets column j at step (k-1-j) + 2t; the
 // rotation of sweep t on columns (j, j+1) is stored at rot[(base + (k-1-j) + 2t) * 32 + t], i.e. the
@@ -151,7 +149,6 @@ __device__ __forceinline__ double rsqrt_nocheck(double x)
     return fma(y * e, fma(0.375, e, 0.5), y);
 }
 
-template <bool SKEW>
 __global__ void __launch_bounds__(32)
 ql_log_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ list)
 {
@@ -166,8 +163,8 @@ ql_log_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ lis
         int2 *__restrict__ sweeps = D.sweeps;
         int2 *__restrict__ groups = D.groups;
         int nrot = 0, nsw = 0;
-        int64_t next_row = 0;                     // SKEW: first free row of the skewed log
-        double2 *lane_rot = rot;                  // SKEW: rot + (base * 32 + t) + 32 * SYS_LAG * t
+        int64_t next_row = 0;                     // first free row of the skewed log
+        double2 *lane_rot = rot;                  // rot + (base * 32 + t) + 32 * SYS_LAG * t
         bool failed = false;
         for (int l = 0; l < n && !failed; ++l) {
             int iter = 0;
@@ -179,7 +176,7 @@ ql_log_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ lis
                 }
                 if (m == l) break;
                 if (++iter > 60 || nsw >= D.sweep_cap) { failed = true; break; }
-                if (SKEW) {
+                {
                     const int t = nsw & 31;
                     if (t == 0) {                 // a new group starts with this sweep
                         const int E = n - l + 1;
@@ -189,7 +186,7 @@ ql_log_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ lis
                     }
                     const int2 gr = groups[nsw >> 5];
                     lane_rot = rot + ((int64_t)gr.x + SYS_LAG * t) * 32 + t;
-                } else if (nrot + (m - l) > D.rot_cap) { failed = true; break; }
+                }
                 double g = (d[l + 1] - d[l]) / (2.0 * e[l]);
                 double r = sqrt(g * g + 1.0);
                 g = d[m] - d[l] + e[l] / (g + (g >= 0.0 ? r : -r));
@@ -203,7 +200,7 @@ ql_log_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ lis
                 // so p = s (u rinv) = f u rinv^2 and the next g = c (u rinv) - b = g u rinv^2 - b.
                 // d[i+1] and the next d[i], e[i] travel in registers (fetched ahead of the stores).
                 double e_nx = e[i], d_nx = d[i], dprev = d[m];
-                double2 *lr = SKEW ? lane_rot + (int64_t)(n - 1 - i) * 32 : rot + nrot;
+                double2 *lr = lane_rot + (int64_t)(n - 1 - i) * 32;
                 for (; i >= l; --i) {
                     const double ei = e_nx, di = d_nx;
                     if (i > l) { e_nx = e[i - 1]; d_nx = d[i - 1]; }
@@ -225,7 +222,7 @@ ql_log_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ lis
                     e[i + 1] = r2 * rinv;
                     d[i + 1] = g1 + p;
                     *lr = make_double2(c, s);
-                    lr += SKEW ? 32 : 1;
+                    lr += 32;
                     ++nrot;
                     dprev = di;
                 }
@@ -241,123 +238,6 @@ ql_log_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ lis
     }
     __syncwarp();
     for (int i = threadIdx.x; i < n; i += 32) D.dvec[i] = d[i];
-}
-
-// ---- stage 3: rows of W = Q Z in shared memory, then select and scale -----------------------
-__global__ void __launch_bounds__(32)
-eigvec_panel_kernel(const RefreshDev *__restrict__ rd, const RowItem *__restrict__ items, int pr)
-{
-    extern __shared__ double z[];                 // z[col * pr + lane]
-    const RowItem it = items[blockIdx.x];
-    const RefreshDev D = rd[it.block];
-    const int k = D.k, r = D.r;
-    const int lane = threadIdx.x;
-    const int row = it.row0 + lane;
-    const bool active = lane < pr && row < k;
-    if (lane < pr)
-        for (int c = 0; c < k; ++c) z[c * pr + lane] = (c == row) ? 1.0 : 0.0;
-    __syncwarp();
-    // Lanes without a row (lane >= pr, or a row past the end) shadow lane 0's reads and never write.
-    {
-        // x <- x H_0 H_1 ... : x[j+1:] -= tau_j (x[j+1:] . v_j) v_j,  v_j = (1, S[j][j+2:]).
-        // The reflector is staged 64 entries at a time in a small shared buffer that every lane reads.
-        const double *__restrict__ A = D.S;
-        const int zl = (lane < pr) ? lane : 0;
-        double *vbuf = z + (size_t)k * pr;       // 64 doubles behind the panel
-        for (int j = 0; j + 2 < k; ++j) {
-            const double tau = D.tau[j];
-            if (tau == 0.0) continue;
-            const double *v = A + (int64_t)j * k;   // v[c] for c >= j+2
-            double d0 = z[(j + 1) * pr + zl], d1 = 0.0, d2 = 0.0, d3 = 0.0;
-            for (int c0 = j + 2; c0 < k; c0 += 64) {
-                const int cn = min(64, k - c0);
-                __syncwarp();
-                vbuf[lane] = (lane < cn) ? v[c0 + lane] : 0.0;
-                vbuf[lane + 32] = (lane + 32 < cn) ? v[c0 + lane + 32] : 0.0;
-                __syncwarp();
-                const double *zc = z + (size_t)c0 * pr + zl;
-                int u = 0;
-                for (; u + 3 < cn; u += 4) {
-                    d0 += zc[(u + 0) * pr] * vbuf[u + 0];
-                    d1 += zc[(u + 1) * pr] * vbuf[u + 1];
-                    d2 += zc[(u + 2) * pr] * vbuf[u + 2];
-                    d3 += zc[(u + 3) * pr] * vbuf[u + 3];
-                }
-                for (; u < cn; ++u) d0 += zc[u * pr] * vbuf[u];
-            }
-            const double dot = ((d0 + d1) + (d2 + d3)) * tau;
-            if (active) z[(j + 1) * pr + zl] -= dot;
-            for (int c0 = j + 2; c0 < k; c0 += 64) {
-                const int cn = min(64, k - c0);
-                __syncwarp();
-                vbuf[lane] = (lane < cn) ? v[c0 + lane] : 0.0;
-                vbuf[lane + 32] = (lane + 32 < cn) ? v[c0 + lane + 32] : 0.0;
-                __syncwarp();
-                if (active) {
-                    double *zc = z + (size_t)c0 * pr + zl;
-#pragma unroll 4
-                    for (int u = 0; u < cn; ++u) zc[u * pr] -= dot * vbuf[u];
-                }
-            }
-        }
-        __syncwarp();
-        // logged rotations, staged 32 at a time in the shared buffer; four rotations are applied per
-        // trip with their inputs loaded up front, so that no shared-memory load sits on the
-        // dependent chain f -> f
-        const int nsw = *D.nsweeps;
-        const double2 *__restrict__ rot = D.rot;
-        const int2 *__restrict__ sweeps = D.sweeps;
-        double2 *rbuf = (double2 *)vbuf;
-        int off = 0;
-        for (int sidx = 0; sidx < nsw; ++sidx) {
-            const int2 sw = sweeps[sidx];
-            int i = sw.x;
-            double f = z[(i + 1) * pr + zl];
-            for (int t0 = 0; t0 < sw.y; t0 += 32) {
-                const int cn = min(32, sw.y - t0);
-                __syncwarp();
-                if (lane < cn) rbuf[lane] = rot[off + t0 + lane];
-                __syncwarp();
-                int u = 0;
-                for (; u + 3 < cn; u += 4, i -= 4) {
-                    const double z0 = z[(i - 0) * pr + zl], z1 = z[(i - 1) * pr + zl];
-                    const double z2 = z[(i - 2) * pr + zl], z3 = z[(i - 3) * pr + zl];
-                    const double2 r0 = rbuf[u], r1 = rbuf[u + 1], r2 = rbuf[u + 2], r3 = rbuf[u + 3];
-                    const double o0 = r0.y * z0 + r0.x * f;  f = r0.x * z0 - r0.y * f;
-                    const double o1 = r1.y * z1 + r1.x * f;  f = r1.x * z1 - r1.y * f;
-                    const double o2 = r2.y * z2 + r2.x * f;  f = r2.x * z2 - r2.y * f;
-                    const double o3 = r3.y * z3 + r3.x * f;  f = r3.x * z3 - r3.y * f;
-                    if (active) {
-                        z[(i + 1) * pr + zl] = o0; z[(i - 0) * pr + zl] = o1;
-                        z[(i - 1) * pr + zl] = o2; z[(i - 2) * pr + zl] = o3;
-                    }
-                }
-                for (; u < cn; ++u, --i) {
-                    const double2 r0 = rbuf[u];
-                    const double zi = z[i * pr + zl];
-                    if (active) z[(i + 1) * pr + zl] = r0.y * zi + r0.x * f;
-                    f = r0.x * zi - r0.y * f;
-                }
-            }
-            if (active) z[(i + 1) * pr + zl] = f;
-            off += sw.y;
-        }
-    }
-    __syncwarp();
-    if (active) {
-        // rank the eigenvalues (descending, ties by index) and emit the leading r columns
-        const double *__restrict__ lam = D.dvec;
-        for (int j = 0; j < k; ++j) {
-            const int rank = D.rank[j];
-            if (rank < r) {
-                const double lj = lam[j];
-                const double inv = (lj > 1e-300) ? 1.0 / sqrt(lj) : 0.0;
-                const double w = z[j * pr + lane];
-                D.Wu[(int64_t)row * r + rank] = (float)w;
-                D.Wv[(int64_t)row * r + rank] = (float)(w * inv);
-            }
-        }
-    }
 }
 
 __global__ void eig_rank_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ list)
@@ -554,25 +434,18 @@ eig_rot_systolic_kernel(const RefreshDev *__restrict__ rd, const RowItem *__rest
 
 static int sys_rows_per_warp(int kmax) { return kmax <= 544 ? 4 : 2; }
 
-int eig_qrows_rows(int kmax) { return kmax <= SYS_KMAX ? QR_WARPS * (kmax <= 544 ? 2 : 1) : 0; }
+int eig_qrows_rows(int kmax) { return QR_WARPS * (kmax <= 544 ? 2 : 1); }
 
 int eig_panel_rows(int kmax)
 {
-    if (kmax <= SYS_KMAX) return SYS_WARPS * sys_rows_per_warp(kmax);
-    int pr = (110 * 1024) / (8 * kmax);
-    if (pr > 32) pr = 32;
-    pr &= ~7;
-    if (pr < 8) pr = 8;
-    return pr;
+    return SYS_WARPS * sys_rows_per_warp(kmax);
 }
 
 int64_t eig_rot_capacity(int k)
 {
-    if (k <= SYS_KMAX) {   // rows of the skewed log (typical need: 0.03 k^2 + 4 k), 32 entries each
-        const int64_t rows = (int64_t)k * k / 10 + 12 * (int64_t)k + 512;
-        return rows * 32;
-    }
-    return 3 * (int64_t)k * k + 64;
+    // rows of the skewed log (typical need: 0.03 k^2 + 4 k), 32 entries each
+    const int64_t rows = (int64_t)k * k / 10 + 12 * (int64_t)k + 512;
+    return rows * 32;
 }
 
 template <typename F>
@@ -590,7 +463,7 @@ cudaError_t eig_tridiag_batched(const RefreshDev *rd, const int32_t *list, int n
     if (nlist <= 0) return cudaSuccess;
     const int kpad = kmax + 8;
     const size_t tr_bytes = (size_t)3 * kpad * sizeof(double);
-    static size_t tr_cfg = 0, pn_cfg = 0, sys4_cfg = 0, sys2_cfg = 0;
+    static size_t tr_cfg = 0, sys4_cfg = 0, sys2_cfg = 0;
     cudaError_t e;
     if ((e = raise_smem(tridiag_kernel, tr_bytes, &tr_cfg)) != cudaSuccess) return e;
     tridiag_kernel<<<nlist, TR_THREADS, tr_bytes, stream>>>(rd, list, kpad);
@@ -600,7 +473,7 @@ cudaError_t eig_tridiag_batched(const RefreshDev *rd, const int32_t *list, int n
         if (kmax <= 288) eig_qrows_kernel<9, 2, QR_WARPS><<<nqrows, QR_WARPS * 32, 0, stream>>>(rd, qrows_items);
         else if (kmax <= 544) eig_qrows_kernel<17, 2, QR_WARPS><<<nqrows, QR_WARPS * 32, 0, stream>>>(rd, qrows_items);
         else eig_qrows_kernel<33, 1, QR_WARPS><<<nqrows, QR_WARPS * 32, 0, stream>>>(rd, qrows_items);
-        ql_log_kernel<true><<<nlist, 32, ql_bytes, stream>>>(rd, list);
+        ql_log_kernel<<<nlist, 32, ql_bytes, stream>>>(rd, list);
         eig_rank_kernel<<<nlist, 256, 0, stream>>>(rd, list);
         const int R = sys_rows_per_warp(kmax);
         const size_t sys_bytes = (size_t)SYS_WARPS * R * kmax * sizeof(double);
@@ -613,18 +486,7 @@ cudaError_t eig_tridiag_batched(const RefreshDev *rd, const int32_t *list, int n
         }
         return cudaGetLastError();
     }
-    const int pr = eig_panel_rows(kmax);
-    const size_t pn_bytes = (size_t)pr * kmax * sizeof(double) + 64 * sizeof(double);   // panel + staging buffer
-    if (pn_bytes > pn_cfg) {
-        if ((e = cudaFuncSetAttribute(eigvec_panel_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pn_bytes)) != cudaSuccess) return e;
-        // ask for the largest shared-memory carve-out so that two panels fit on one SM
-        if ((e = cudaFuncSetAttribute(eigvec_panel_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 100)) != cudaSuccess) return e;
-        pn_cfg = pn_bytes;
-    }
-    ql_log_kernel<false><<<nlist, 32, ql_bytes, stream>>>(rd, list);
-    eig_rank_kernel<<<nlist, 256, 0, stream>>>(rd, list);
-    eigvec_panel_kernel<<<npanels, 32, pn_bytes, stream>>>(rd, panel_items, pr);
-    return cudaGetLastError();
+    return cudaErrorInvalidValue;   // k is limited to SYS_KMAX when a context is created
 }
 
 }  // namespace tsr

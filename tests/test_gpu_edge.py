@@ -22,6 +22,8 @@ def _tsr():
     (torch.bfloat16, dict(m=64, n=48, r=8, p=0, q=0), 4),       # no oversampling, no power iteration
     (torch.bfloat16, dict(m=40, n=136, r=32, p=8, q=1), 8),     # k = min(m, n): the sketch spans everything
     (torch.float32, dict(m=150, n=90, r=30, p=6, q=3), 12),     # three power iterations
+    (torch.bfloat16, dict(m=320, n=304, r=250, p=5, q=1), 16),  # odd k = 255: tridiagonal eigen-solver, no TMA row products
+    (torch.bfloat16, dict(m=640, n=704, r=560, p=8, q=1), 16),  # k = 568: the wide variants of the eigenvector kernels
 ])
 def test_refresh_small_and_extreme_shapes(dtype, shape, gap):
     tsr = _tsr()

@@ -50,6 +50,7 @@ def test_create_validates_shapes(tsr):
         D(16, 16, 8, 16, 4, 0, 0, 0, 0, 0, 0, 0),                    # ldg < n
         D(16, 16, 16, 16, 12, 8, 0, 0, 0, 0, 0, 0),                  # r + p > min(m, n)
         D(16, 16, 16, 16, 4, 0, -1, 0, 0, 0, 0, 0),                  # q < 0
+        D(2048, 2048, 2048, 2048, 1050, 8, 1, 0, 0, 0, 0, 0),        # r + p beyond the eigen-solver's limit of 1056
     ]
     for d in bad:
         rc, ctx = _create(tsr, [d])
