@@ -97,7 +97,7 @@ struct tsr_ctx {
     int stage_next = 0;
     // refresh runs as up to NGROUP independent groups of blocks on side streams, so that the
     // latency-bound small-matrix kernels of one group overlap the GEMM-like kernels of another
-    static constexpr int NGROUP = 8;
+    static constexpr int NGROUP = 4;
     cudaStream_t aux[NGROUP] = {};
     cudaEvent_t ev_fork = nullptr, ev_join[NGROUP] = {}, ev_stagger[NGROUP] = {};
     bool aux_ready = false;
@@ -267,6 +267,9 @@ void build_tiles(tsr_ctx *ctx)
     for (int kd : {KT, KP}) ctx->bn[kd] = rmax >= 256 ? 256 : 128;
     // the core GEMM has few, long tiles: 256-wide tiles only pay once r reaches 512 (measured)
     for (int kd : {KC, KCS}) ctx->bn[kd] = rmax >= 512 ? 256 : 128;
+    // apply: 256-wide tiles halve the P traffic per byte of W, which pays once the operands are as wide
+    // as r = 512 (measured 2.28 -> 2.05 ms on the 1B set; at r = 256 the narrow tile is faster)
+    ctx->bn[KA] = rmax >= 512 ? 256 : 128;
     for (int bi : ctx->order) {
         Block &b = ctx->blocks[bi];
         for (int kd = 0; kd < NKIND; ++kd) b.tile_begin[kd] = b.tile_end[kd] = (int)ctx->tiles[kd].size();
@@ -417,8 +420,8 @@ tsr_status launch_kind(tsr_ctx *ctx, int kind, const std::vector<int> &list, int
         size_t j = i + 1;
         while (j < ranges.size() && ranges[j].first == hi) { hi = ranges[j].second; ++j; }
         if (kind == KA)
-            TSR_CUDA(ctx, umma_apply_launch(ctx->d_probs[kind], ctx->d_tiles[kind] + lo, hi - lo, ctx->num_sms, sc,
-                                            ctx->d_status, st));
+            TSR_CUDA(ctx, umma_apply_launch(ctx->d_probs[kind], ctx->d_tiles[kind] + lo, hi - lo, ctx->num_sms, ctx->bn[kind],
+                                            sc, ctx->d_status, st));
         else
             TSR_CUDA(ctx, umma_gemm_launch(ctx->d_probs[kind], ctx->d_tiles[kind] + lo, hi - lo, ctx->num_sms, ctx->bn[kind],
                                            epilogue, planes, sc, ctx->d_status, st));
@@ -701,8 +704,7 @@ tsr_status do_refresh(tsr_ctx *ctx, const std::vector<int> &list, uint64_t seed,
 {
     if (list.empty()) return TSR_OK;
     const size_t zero[5] = {0, 0, 0, 0, 0};
-    static const int ng_env = getenv("TSR_NGROUP") ? atoi(getenv("TSR_NGROUP")) : 4;   // EXPERIMENT
-    int ngroup = std::min<int>(std::min<int>(ng_env, tsr_ctx::NGROUP), (int)list.size() / 8);
+    int ngroup = std::min<int>(tsr_ctx::NGROUP, (int)list.size() / 8);
     if (!ctx->aux_ready || ngroup < 2) return do_refresh_group(ctx, list, seed, omegas, st, 0, zero, reexpress);
     // order the listed blocks as the tile tables do, remembering each one's omega
     std::vector<int> pos(ctx->blocks.size(), 0);
@@ -722,8 +724,7 @@ tsr_status do_refresh(tsr_ctx *ctx, const std::vector<int> &list, uint64_t seed,
         // Groups start one orthonormalisation apart: in lock-step all groups would sit in the same
         // one-CTA-per-matrix kernel at the same time (more CTAs than SMs, two waves) and leave the
         // SMs idle that the throughput-bound kernels of another group could use.
-        static const int stag_env = getenv("TSR_STAGGER") ? atoi(getenv("TSR_STAGGER")) : 1;   // EXPERIMENT
-        if (g > 0 && stag_env) TSR_CUDA(ctx, cudaStreamWaitEvent(ctx->aux[g], ctx->ev_stagger[g - 1], 0));
+        if (g > 0) TSR_CUDA(ctx, cudaStreamWaitEvent(ctx->aux[g], ctx->ev_stagger[g - 1], 0));
         tsr_status s = do_refresh_group(ctx, grp, seed, omegas ? om.data() : nullptr, ctx->aux[g], list_off, item_off,
                                         reexpress, ctx->ev_stagger[g]);
         if (s != TSR_OK && result == TSR_OK) result = s;

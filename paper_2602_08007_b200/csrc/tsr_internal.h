@@ -73,7 +73,7 @@ cudaError_t umma_gemm_launch(const UmmaProblem *probs, const UmmaTile *tiles, in
 cudaError_t umma_configure();  // sets the dynamic shared-memory attributes once per process
 // Persistent apply kernel (tsr_umma_apply.cu): W <- decay W - step_scale P V^T over a tile table.
 cudaError_t umma_apply_configure();
-cudaError_t umma_apply_launch(const UmmaProblem *probs, const UmmaTile *tiles, int num_tiles, int num_sms,
+cudaError_t umma_apply_launch(const UmmaProblem *probs, const UmmaTile *tiles, int num_tiles, int num_sms, int bn,
                               const StepScalars &sc, int32_t *status, cudaStream_t stream);
 
 // ---------------------------------------------------------------------------------------

@@ -2,14 +2,14 @@
 //
 //   W[m x n] <- decay * W - step_scale * (P V^T),   P = U D (m x r, BF16),  V (n x r, BF16)
 //
-// The lifted update never reaches memory: each 128 x 128 tile of P V^T is accumulated in tensor
-// memory and consumed by the epilogue, which streams the matching W tile through shared memory
-// with TMA (read-modify-write of 8 bytes per weight is what bounds this kernel).
+// The lifted update never reaches memory: each 128 x BN tile of P V^T (BN = 128, or 256 for r >= 512)
+// is accumulated in tensor memory and consumed by the epilogue, which streams the matching W tile
+// through shared memory with TMA (read-modify-write of 8 bytes per weight is what bounds this kernel).
 //
 // One CTA per SM loops over the tiles of all blocks (static round-robin over a device-resident
 // tile table).  Roles:
 //   warp 0      TMA producer for the P / V operand stages (128-byte swizzle, ring of stages)
-//   warp 1      tensor-memory allocation; one lane issues the MMAs into one of two 128-column
+//   warp 1      tensor-memory allocation; one lane issues the MMAs into one of two BN-column
 //               accumulators, so the MMAs of tile i+1 overlap the epilogue of tile i
 //   warps 4-7   epilogue; warp q owns accumulator rows 32q..32q+31 and a private ring of
 //               32 x 32 FP32 W boxes (4 KB, 128-byte swizzle): it prefetches its W boxes
@@ -24,16 +24,25 @@
 namespace tsr {
 
 constexpr int AP_THREADS = 256;
-constexpr int AP_BN = 128;
-constexpr int AP_STAGES = 4;                 // operand stages: 16 KB (P) + 16 KB (V)
-constexpr int AP_STAGE_BYTES = 32768;
-constexpr int AP_NBOX = 6;                   // W boxes per epilogue warp
 constexpr int AP_LAG = 2;                    // a box is refilled AP_LAG stores after its own store
 constexpr int AP_BOX_BYTES = 4096;
-constexpr int AP_WBOX_OFFSET = AP_STAGES * AP_STAGE_BYTES;
-constexpr int AP_BAR_OFFSET = AP_WBOX_OFFSET + 4 * AP_NBOX * AP_BOX_BYTES;
-constexpr int AP_NBARS = 2 * AP_STAGES + 4 + 4 * AP_NBOX;
-constexpr int AP_SMEM = AP_BAR_OFFSET + AP_NBARS * 8 + 64 + 1024;
+
+// Tile width 128: four operand stages and six W boxes per epilogue warp.  Tile width 256 (the P tile
+// is then used for twice as many outputs, which lowers the operand bytes an SM has to pull in per
+// byte of W): three stages of 16 KB (P) + 32 KB (V), five W boxes per warp, both accumulators fill
+// the 512 columns of tensor memory.
+template <int BN>
+struct ApplyCfg {
+    static constexpr int STAGES = BN == 256 ? 3 : 4;
+    static constexpr int STAGE_BYTES = 16384 + BN * 128;
+    static constexpr int NBOX = BN == 256 ? 5 : 6;
+    static constexpr int CHUNKS = BN / 32;
+    static constexpr int WBOX_OFFSET = STAGES * STAGE_BYTES;
+    static constexpr int BAR_OFFSET = WBOX_OFFSET + 4 * NBOX * AP_BOX_BYTES;
+    static constexpr int NBARS = 2 * STAGES + 4 + 4 * NBOX;
+    static constexpr int SMEM = BAR_OFFSET + NBARS * 8 + 64 + 1024;
+    static constexpr uint32_t TMEM_COLS = 2 * BN;
+};
 
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, uint32_t src, int x, int y)
 {
@@ -58,21 +67,27 @@ __device__ __forceinline__ void cursor_load(ChunkCursor &cur, const UmmaTile *ti
         cur.M = probs[t.prob].M;
     }
 }
+template <int CHUNKS>
 __device__ __forceinline__ void cursor_next(ChunkCursor &cur, const UmmaTile *tiles, const UmmaProblem *probs,
                                             int num_tiles, int stride)
 {
     cur.c++;
-    if (cur.c >= 4 || cur.n0 + cur.c * 32 >= cur.N) {
+    if (cur.c >= CHUNKS || cur.n0 + cur.c * 32 >= cur.N) {
         cur.c = 0;
         cur.tile_idx += stride;
         cursor_load(cur, tiles, probs, num_tiles);
     }
 }
 
+template <int BN>
 __global__ void __launch_bounds__(AP_THREADS, 1)
 umma_apply_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restrict__ tiles, int num_tiles,
                   StepScalars sc, int32_t *__restrict__ status)
 {
+    using CF = ApplyCfg<BN>;
+    constexpr int AP_STAGES = CF::STAGES, AP_STAGE_BYTES = CF::STAGE_BYTES, AP_NBOX = CF::NBOX;
+    constexpr int AP_WBOX_OFFSET = CF::WBOX_OFFSET, AP_BAR_OFFSET = CF::BAR_OFFSET, AP_NBARS = CF::NBARS;
+    constexpr int AP_BN = BN;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint64_t *bars = (uint64_t *)(smem + AP_BAR_OFFSET);
@@ -95,7 +110,7 @@ umma_apply_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restr
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(256u)
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(CF::TMEM_COLS)
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
@@ -121,6 +136,7 @@ umma_apply_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restr
                     uint8_t *st = smem + s * AP_STAGE_BYTES;
                     tma_load_2d(smem_u32(st), &P->tmA, full, kb * UM_BK, tile.m0);
                     tma_load_2d(smem_u32(st + 16384), &P->tmB, full, kb * UM_BK, tile.n0);
+                    if (BN == 256) tma_load_2d(smem_u32(st + 32768), &P->tmB, full, kb * UM_BK, tile.n0 + 128);
                 }
             }
         }
@@ -171,7 +187,7 @@ umma_apply_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restr
                             pre.n0 + pre.c * 32, pre.m0 + q * 32);
             }
             ++issued;
-            cursor_next(pre, tiles, probs, num_tiles, stride);
+            cursor_next<CF::CHUNKS>(pre, tiles, probs, num_tiles, stride);
         }
         while (cur.tile_idx < num_tiles && ok) {
             const uint32_t buf = tc & 1u;
@@ -182,7 +198,7 @@ umma_apply_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restr
             const uint32_t slot = cons % AP_NBOX;
             uint32_t v[32];
             tc_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + buf * AP_BN + (uint32_t)(cur.c * 32), v);
-            const bool last_chunk = (cur.c == 3) || (cur.n0 + (cur.c + 1) * 32 >= cur.N);
+            const bool last_chunk = (cur.c == CF::CHUNKS - 1) || (cur.n0 + (cur.c + 1) * 32 >= cur.N);
             if (last_chunk) {   // accumulator fully read by this warp: hand it back to the MMA warp
                 tc_fence_before();
                 if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar_acc_empty + buf)) : "memory");
@@ -217,10 +233,10 @@ umma_apply_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restr
                                 pre.n0 + pre.c * 32, pre.m0 + q * 32);
                 }
                 ++issued;
-                cursor_next(pre, tiles, probs, num_tiles, stride);
+                cursor_next<CF::CHUNKS>(pre, tiles, probs, num_tiles, stride);
             }
             if (last_chunk) ++tc;
-            cursor_next(cur, tiles, probs, num_tiles, stride);
+            cursor_next<CF::CHUNKS>(cur, tiles, probs, num_tiles, stride);
         }
         if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     }
@@ -229,22 +245,27 @@ umma_apply_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restr
     __syncthreads();
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(256u) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(CF::TMEM_COLS) : "memory");
     }
     if (threadIdx.x == 0 && s_timeout && status) atomicMax(status, (int)TSR_ERR_TIMEOUT);
 }
 
 cudaError_t umma_apply_configure()
 {
-    return cudaFuncSetAttribute(umma_apply_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, AP_SMEM);
+    cudaError_t e = cudaFuncSetAttribute(umma_apply_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, ApplyCfg<128>::SMEM);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(umma_apply_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, ApplyCfg<256>::SMEM);
 }
 
-cudaError_t umma_apply_launch(const UmmaProblem *probs, const UmmaTile *tiles, int num_tiles, int num_sms,
+cudaError_t umma_apply_launch(const UmmaProblem *probs, const UmmaTile *tiles, int num_tiles, int num_sms, int bn,
                               const StepScalars &sc, int32_t *status, cudaStream_t stream)
 {
     if (num_tiles <= 0) return cudaSuccess;
     const int grid = num_tiles < num_sms ? num_tiles : num_sms;
-    umma_apply_kernel<<<grid, AP_THREADS, AP_SMEM, stream>>>(probs, tiles, num_tiles, sc, status);
+    if (bn == 256)
+        umma_apply_kernel<256><<<grid, AP_THREADS, ApplyCfg<256>::SMEM, stream>>>(probs, tiles, num_tiles, sc, status);
+    else
+        umma_apply_kernel<128><<<grid, AP_THREADS, ApplyCfg<128>::SMEM, stream>>>(probs, tiles, num_tiles, sc, status);
     return cudaGetLastError();
 }
 
