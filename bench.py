@@ -209,9 +209,10 @@ def max_over_ranks(values, dist, device):
 
 
 # Measured DRAM traffic of umma_apply_kernel divided by its algorithmic bytes (8 B per weight +
-# BF16 operands), from the ncu capture summarised in profiles/umma_apply_kernel_llama350m.md.  The
+# BF16 operands), from the ncu capture summarised in profiles/umma_apply_kernel.md.  The
 # 1B workload is too large for a multi-pass capture; traffic grows in proportion to the weights, so
-# the 350M ratio is applied to the 1B algorithmic bytes.
+# the ratio measured on smaller sets (0.98 on the 350M set and on a six-layer slice of the 1B set)
+# is applied to the 1B algorithmic bytes.
 APPLY_TRAFFIC_RATIO = 0.98
 
 def build_plan(w: ti.Workload, device):
