@@ -133,6 +133,53 @@ def test_fused_and_unfused_orders_agree_bitwise():
             assert torch.equal(x, y)
 
 
+def test_two_workers_averaging_the_core_match_the_oracle():
+    """The synchronisation point of Section 3.2 emulated on one GPU: two workers with the same
+    state and different local gradients each project, the caller averages the r x r cores
+    (what the all-reduce would do) and writes the average into every worker's C, and the core
+    update and the lift run from it.  Both workers must stay identical and follow the oracle
+    taken through the same three steps with the averaged core."""
+    import paper_2602_08007_b200 as tsr
+    shapes = [dict(m=256, n=384, r=64), dict(m=200, n=328, r=40)]
+    nw = 2
+    plans = [tsr.Plan(shapes, g_dtype=torch.bfloat16) for _ in range(nw)]
+    Wo, Mo, Vo, Uo, Vbo = [], [], [], [], []
+    for i, sh in enumerate(shapes):
+        U = ti.orthonormal(sh["m"], sh["r"], 900 + 2 * i)
+        V = ti.orthonormal(sh["n"], sh["r"], 901 + 2 * i)
+        for pl in plans:
+            set_bases(pl, i, U, V)
+            W0 = fill_weights(pl, i, 50 + i)
+            pl.M[i].zero_(); pl.Vm[i].zero_()
+        Wo.append(W0.copy()); Uo.append(to64(U)); Vbo.append(to64(V))
+        Mo.append(np.zeros((sh["r"], sh["r"]))); Vo.append(np.zeros((sh["r"], sh["r"])))
+    for pl in plans:
+        pl.bases_changed()
+    worst = 0.0
+    for t in (1, 2, 3):
+        h = tsr.make_hyper(t, lr=1e-3)
+        G64 = [[fill_gradient(pl, i, 1000 * t + 10 * w + i) for i in range(len(shapes))] for w, pl in enumerate(plans)]
+        for pl in plans:
+            pl.project_core()
+        torch.cuda.synchronize()
+        for i in range(len(shapes)):
+            avg = sum(pl.C[i] for pl in plans) / nw
+            for pl in plans:
+                pl.C[i].copy_(avg)
+        for pl in plans:
+            pl.adam_core_step(h)
+            pl.backproject_apply(h)
+        torch.cuda.synchronize()
+        for i in range(len(shapes)):
+            Cbar = sum(oracle.project_core(G64[w][i], Uo[i], Vbo[i]) for w in range(nw)) / nw
+            D = oracle.adam_core(Cbar, Mo[i], Vo[i], HYPER["beta1"], HYPER["beta2"], HYPER["eps"], t)
+            oracle.backproject_apply(Uo[i], D, Vbo[i], Wo[i], HYPER["lr"])
+            assert torch.equal(plans[0].W[i], plans[1].W[i]) and torch.equal(plans[0].M[i], plans[1].M[i])
+            worst = max(worst, rel_fro(to64(plans[0].C[i]), Cbar), rel_fro(to64(plans[0].M[i]), Mo[i]),
+                        rel_fro(to64(plans[0].Vm[i]), Vo[i]), rel_fro(to64(plans[0].W[i]), Wo[i]))
+    assert worst < TOL_BF16, worst
+
+
 def test_split_k_core_matches_oracle():
     # m large enough that the core GEMM is split along K (tall embedding-like block)
     shapes = [dict(m=9000, n=128, r=32)]
