@@ -16,16 +16,26 @@
 
 namespace tsr {
 
-constexpr int TR_THREADS = 1024;
+constexpr int TR_THREADS = 512;
+constexpr int TR_NB = 8;          // columns per panel
 
 // ---- stage 1: tridiagonalisation -----------------------------------------------------------
+// Panels of TR_NB columns with the rank-2 updates deferred (the scheme of LAPACK's blocked
+// reduction): inside a panel the trailing matrix T0 is left as it was at the start of the panel
+// and the reflector pairs (v_i, w_i) found so far are kept in shared memory; the current matrix
+// is T0 - sum_i (v_i w_i^T + w_i v_i^T).  A column step reads T0 once (the matrix-vector
+// product); the trailing matrix is rewritten once per panel instead of once per column, which
+// cuts the traffic per column from three passes to 1 + 2 / TR_NB.  The matrix is symmetric and
+// stored in full; row j is used where the textbook takes column j.  Indices s, t below are
+// relative to the first row / column j0 of the panel.
 __global__ void __launch_bounds__(TR_THREADS)
 tridiag_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ list, int kpad)
 {
-    extern __shared__ double tr_smem[];          // v, p, w : 3 x kpad
-    double *vs = tr_smem, *ps = tr_smem + kpad, *ws = tr_smem + 2 * kpad;
+    extern __shared__ double tr_smem[];          // vs, ps : 2 x kpad;  Vp, Wp : 2 x TR_NB x kpad
+    double *vs = tr_smem, *ps = tr_smem + kpad;
+    double *Vp = tr_smem + 2 * kpad, *Wp = Vp + TR_NB * kpad;
     __shared__ double red[32];
-    __shared__ double s_scalar[4];
+    __shared__ double dots[2 * TR_NB];           // dots[2 i] = w_i . v, dots[2 i + 1] = v_i . v
     const RefreshDev d = rd[list[blockIdx.x]];
     const int k = d.k;
     double *__restrict__ A = d.S;
@@ -43,71 +53,117 @@ tridiag_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ li
         return t;   // every thread of every warp holds the total
     };
 
-    for (int j = 0; j + 2 < k; ++j) {
-        const int len = k - j - 1;               // x = A[j][j+1 .. k-1]
-        double *xrow = A + (int64_t)j * k + j + 1;
-        double part = 0.0;
-        for (int i = tid; i < len; i += nt) { const double x = xrow[i]; vs[i] = x; part += x * x; }
-        const double nrm2 = block_sum(part);
-        const double x0 = vs[0];
-        const double nrm = sqrt(nrm2);
-        const double tail2 = nrm2 - x0 * x0;
-        if (!(tail2 > 0.0) || nrm == 0.0) {      // nothing to annihilate: H_j = I
-            if (tid == 0) { d.tau[j] = 0.0; d.dvec[j] = A[(int64_t)j * k + j]; d.evec[j] = x0; }
-            __syncthreads();
-            continue;
-        }
-        const double alpha = (x0 >= 0.0) ? -nrm : nrm;
-        const double v0 = x0 - alpha;
-        const double tau = -v0 / alpha;
-        __syncthreads();
-        for (int i = tid; i < len; i += nt) {
-            const double v = (i == 0) ? 1.0 : vs[i] / v0;
-            vs[i] = v;
-            if (i > 0) xrow[i] = v;              // keep the reflector for stage 3
-        }
-        if (tid == 0) { d.tau[j] = tau; d.dvec[j] = A[(int64_t)j * k + j]; d.evec[j] = alpha; }
-        __syncthreads();
-        // p = tau * A22 v      (A22 = A[j+1.., j+1..], row-wise dot products; a warp takes four rows at a
-        // time so that four loads are in flight per lane)
-        for (int a0 = 4 * warp; a0 < len; a0 += 4 * nwarps) {
-            const double *row0 = A + (int64_t)(j + 1 + a0) * k + j + 1;
-            const int na = min(4, len - a0);
-            double acc[4] = {0.0, 0.0, 0.0, 0.0};
-            for (int b = lane; b < len; b += 32) {
-                const double vb = vs[b];
-#pragma unroll
-                for (int u = 0; u < 4; ++u)
-                    if (u < na) acc[u] += row0[(int64_t)u * k + b] * vb;
+    for (int j0 = 0; j0 + 2 < k; j0 += TR_NB) {
+        const int L0 = k - j0;
+        const int nbc = min(TR_NB, k - 2 - j0);  // columns of this panel that get a reflector
+        for (int c = 0; c < nbc; ++c) {
+            const int j = j0 + c;
+            const int len = k - j - 1;           // x = current row j, columns j+1 .. k-1  (t = c+1 .. L0-1)
+            double *xrow = A + (int64_t)j * k + j + 1;
+            double part = 0.0;
+            for (int i = tid; i < len; i += nt) {
+                double x = xrow[i];
+                for (int u = 0; u < c; ++u)
+                    x -= Vp[u * kpad + c] * Wp[u * kpad + c + 1 + i] + Wp[u * kpad + c] * Vp[u * kpad + c + 1 + i];
+                vs[i] = x;
+                part += x * x;
             }
+            double dj = A[(int64_t)j * k + j];   // current diagonal entry (every thread computes it)
+            for (int u = 0; u < c; ++u) dj -= 2.0 * Vp[u * kpad + c] * Wp[u * kpad + c];
+            const double nrm2 = block_sum(part);
+            const double x0 = vs[0];
+            const double nrm = sqrt(nrm2);
+            const double tail2 = nrm2 - x0 * x0;
+            if (!(tail2 > 0.0) || nrm == 0.0) {  // nothing to annihilate: H_j = I
+                if (tid == 0) { d.tau[j] = 0.0; d.dvec[j] = dj; d.evec[j] = x0; }
+                for (int t = tid; t < L0; t += nt) { Vp[c * kpad + t] = 0.0; Wp[c * kpad + t] = 0.0; }
+                __syncthreads();
+                continue;
+            }
+            const double alpha = (x0 >= 0.0) ? -nrm : nrm;
+            const double v0 = x0 - alpha;
+            const double tau = -v0 / alpha;
+            __syncthreads();
+            for (int i = tid; i < len; i += nt) {
+                const double v = (i == 0) ? 1.0 : vs[i] / v0;
+                vs[i] = v;
+                if (i > 0) xrow[i] = v;          // keep the reflector for stage 3
+            }
+            if (tid == 0) { d.tau[j] = tau; d.dvec[j] = dj; d.evec[j] = alpha; }
+            __syncthreads();
+            // ps = T0[c+1.., c+1..] v   (row-wise dot products; a warp takes four rows at a time so that
+            // four loads are in flight per lane)
+            for (int a0 = 4 * warp; a0 < len; a0 += 4 * nwarps) {
+                const double *row0 = A + (int64_t)(j + 1 + a0) * k + j + 1;
+                const int na = min(4, len - a0);
+                double acc[4] = {0.0, 0.0, 0.0, 0.0};
+                for (int b = lane; b < len; b += 32) {
+                    const double vb = vs[b];
 #pragma unroll
-            for (int off = 16; off > 0; off >>= 1)
+                    for (int u = 0; u < 4; ++u)
+                        if (u < na) acc[u] += row0[(int64_t)u * k + b] * vb;
+                }
 #pragma unroll
-                for (int u = 0; u < 4; ++u) acc[u] += __shfl_xor_sync(0xffffffffu, acc[u], off);
-            if (lane < na) ps[a0 + lane] = tau * (lane == 0 ? acc[0] : lane == 1 ? acc[1] : lane == 2 ? acc[2] : acc[3]);
+                for (int off = 16; off > 0; off >>= 1)
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) acc[u] += __shfl_xor_sync(0xffffffffu, acc[u], off);
+                if (lane < na) ps[a0 + lane] = (lane == 0 ? acc[0] : lane == 1 ? acc[1] : lane == 2 ? acc[2] : acc[3]);
+            }
+            // the earlier pairs of the panel against v: one warp per dot product
+            if (warp < 2 * c) {
+                const double *vec = ((warp & 1) ? Vp : Wp) + (warp >> 1) * kpad + c + 1;
+                double acc = 0.0;
+                for (int b = lane; b < len; b += 32) acc += vec[b] * vs[b];
+#pragma unroll
+                for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+                if (lane == 0) dots[warp] = acc;
+            }
+            __syncthreads();
+            // p = tau (T0 v - sum_i (v_i (w_i . v) + w_i (v_i . v)))
+            part = 0.0;
+            for (int a = tid; a < len; a += nt) {
+                double acc = ps[a];
+                for (int u = 0; u < c; ++u)
+                    acc -= Vp[u * kpad + c + 1 + a] * dots[2 * u] + Wp[u * kpad + c + 1 + a] * dots[2 * u + 1];
+                acc *= tau;
+                ps[a] = acc;
+                part += acc * vs[a];
+            }
+            const double pv = block_sum(part);
+            const double kk = 0.5 * tau * pv;
+            for (int t = tid; t < L0; t += nt) {   // the new pair, zero where the reflector does not act
+                const int a = t - c - 1;
+                Vp[c * kpad + t] = (a >= 0) ? vs[a] : 0.0;
+                Wp[c * kpad + t] = (a >= 0) ? ps[a] - kk * vs[a] : 0.0;
+            }
+            __syncthreads();
         }
-        __syncthreads();
-        part = 0.0;
-        for (int i = tid; i < len; i += nt) part += ps[i] * vs[i];
-        const double pv = block_sum(part);
-        const double kk = 0.5 * tau * pv;
-        for (int i = tid; i < len; i += nt) ws[i] = ps[i] - kk * vs[i];
-        __syncthreads();
-        // A22 -= v w^T + w v^T   (four rows per warp and trip)
-        for (int a0 = 4 * warp; a0 < len; a0 += 4 * nwarps) {
-            double *row0 = A + (int64_t)(j + 1 + a0) * k + j + 1;
-            const int na = min(4, len - a0);
-            double va[4], wa[4];
+        // T0[s][t] -= sum_i (v_i[s] w_i[t] + w_i[s] v_i[t]) for s, t >= nbc   (two rows per warp and trip)
+        for (int s0 = nbc + 2 * warp; s0 < L0; s0 += 2 * nwarps) {
+            const bool two = (s0 + 1 < L0);
+            double va[2][TR_NB], wa[2][TR_NB];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) { va[u] = (u < na) ? vs[a0 + u] : 0.0; wa[u] = (u < na) ? ws[a0 + u] : 0.0; }
-            for (int b = lane; b < len; b += 32) {
-                const double vb = vs[b], wb = ws[b];
-                double x[4];
+            for (int u = 0; u < TR_NB; ++u) {
+                const bool on = (u < nbc);
+                va[0][u] = on ? Vp[u * kpad + s0] : 0.0;
+                wa[0][u] = on ? Wp[u * kpad + s0] : 0.0;
+                va[1][u] = (on && two) ? Vp[u * kpad + s0 + 1] : 0.0;
+                wa[1][u] = (on && two) ? Wp[u * kpad + s0 + 1] : 0.0;
+            }
+            double *r0 = A + (int64_t)(j0 + s0) * k + j0, *r1 = r0 + k;
+            for (int t = nbc + lane; t < L0; t += 32) {
+                const double x0 = r0[t], x1 = two ? r1[t] : 0.0;
+                double a0 = 0.0, a1 = 0.0;
 #pragma unroll
-                for (int u = 0; u < 4; ++u) x[u] = (u < na) ? row0[(int64_t)u * k + b] : 0.0;
-#pragma unroll
-                for (int u = 0; u < 4; ++u)
-                    if (u < na) row0[(int64_t)u * k + b] = x[u] - (va[u] * wb + wa[u] * vb);
+                for (int u = 0; u < TR_NB; ++u) {
+                    const double vt = Vp[u * kpad + t], wt = Wp[u * kpad + t];   // zero rows for u >= nbc are never read: guarded
+                    if (u < nbc) {
+                        a0 += va[0][u] * wt + wa[0][u] * vt;
+                        a1 += va[1][u] * wt + wa[1][u] * vt;
+                    }
+                }
+                r0[t] = x0 - a0;
+                if (two) r1[t] = x1 - a1;
             }
         }
         __syncthreads();
@@ -462,7 +518,7 @@ cudaError_t eig_tridiag_batched(const RefreshDev *rd, const int32_t *list, int n
 {
     if (nlist <= 0) return cudaSuccess;
     const int kpad = kmax + 8;
-    const size_t tr_bytes = (size_t)3 * kpad * sizeof(double);
+    const size_t tr_bytes = (size_t)(2 + 2 * TR_NB) * kpad * sizeof(double);
     static size_t tr_cfg = 0, sys4_cfg = 0, sys2_cfg = 0;
     cudaError_t e;
     if ((e = raise_smem(tridiag_kernel, tr_bytes, &tr_cfg)) != cudaSuccess) return e;
