@@ -191,6 +191,11 @@ tridiag_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ li
 // 32 rotations a warp needs at one step are contiguous.  lg is the l of the group's first sweep
 // (l never decreases).  groups[g] = (base row, E = k - lg + 1 stream elements); entries that no
 // sweep writes are never used (the reader tests each lane's column against its sweep's range).
+// Deflation threshold: an off-diagonal entry below QL_TOL (|d[m]| + |d[m+1]|) is set aside.  The
+// eigenvectors leave this stage as FP32 numbers, and the rotations are orthogonal whatever the
+// threshold, so a threshold of 1e-13 instead of the unit roundoff only perturbs the eigenvalues by
+// 1e-13 ||T|| and saves the last, already converged, sweep of many eigenvalues.
+constexpr double QL_TOL = 1e-13;
 constexpr int SYS_LAG = 2;                        // steps between neighbouring lanes
 constexpr int SYS_FILL = SYS_LAG * 31;            // steps until the last lane sees the first column
 constexpr int SYS_PF = 8;                         // steps of rotations the reader fetches ahead
@@ -228,7 +233,7 @@ ql_log_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ lis
                 int m = l;
                 for (; m < n - 1; ++m) {
                     const double dd = fabs(d[m]) + fabs(d[m + 1]);
-                    if (fabs(e[m]) <= 2.3e-16 * dd) break;
+                    if (fabs(e[m]) <= QL_TOL * dd) break;
                 }
                 if (m == l) break;
                 if (++iter > 60 || nsw >= D.sweep_cap) { failed = true; break; }
