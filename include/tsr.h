@@ -201,7 +201,10 @@ TSR_API tsr_status tsr_step_grouped(tsr_ctx *ctx, const tsr_hyper *hyper, uint64
 /* The same step driven from HOST memory: G_host[i] is a host pointer to block i's gradient,
  * dense m x n in the block's g_dtype; each is copied into the bound device G buffer, the step
  * runs, and the cores of all blocks are copied back, packed block after block (r*r floats
- * each), into C_host (may be NULL).  Returns after the stream has been synchronised. */
+ * each), into C_host (may be NULL).  On steps without a refresh the blocks travel in chunks: while
+ * one chunk is stepped, the next one's gradients arrive and the previous one's cores leave on the
+ * context's side streams (pinned host memory is needed for that overlap; pageable memory works but
+ * serialises).  Results are identical to the plain order.  Returns after everything has finished. */
 TSR_API tsr_status tsr_step_grouped_host(tsr_ctx *ctx, const void *const *G_host, float *C_host,
                                          const tsr_hyper *hyper, uint64_t seed, int32_t fuse_adam, void *stream);
 

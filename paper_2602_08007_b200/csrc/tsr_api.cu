@@ -100,6 +100,8 @@ struct tsr_ctx {
     static constexpr int NGROUP = 4;
     cudaStream_t aux[NGROUP] = {};
     cudaEvent_t ev_fork = nullptr, ev_join[NGROUP] = {}, ev_stagger[NGROUP] = {};
+    static constexpr int NPIPE = 8;            // chunks of the pipelined host-buffer step
+    cudaEvent_t ev_pipe_in[NPIPE] = {}, ev_pipe_done[NPIPE] = {};
     bool aux_ready = false;
 };
 
@@ -876,6 +878,7 @@ tsr_status tsr_destroy(tsr_ctx *ctx)
     if (ctx->aux_ready) {
         for (int g = 0; g < tsr_ctx::NGROUP; ++g) { cudaStreamDestroy(ctx->aux[g]); cudaEventDestroy(ctx->ev_join[g]); cudaEventDestroy(ctx->ev_stagger[g]); }
         cudaEventDestroy(ctx->ev_fork);
+        for (int c = 0; c < tsr_ctx::NPIPE; ++c) { cudaEventDestroy(ctx->ev_pipe_in[c]); cudaEventDestroy(ctx->ev_pipe_done[c]); }
     }
     delete ctx;
     return TSR_OK;
@@ -1051,6 +1054,10 @@ tsr_status tsr_bind(tsr_ctx *ctx, const tsr_mat_ptrs *ptrs, int32_t count, void 
             TSR_CUDA(ctx, cudaEventCreateWithFlags(&ctx->ev_stagger[g], cudaEventDisableTiming));
         }
         TSR_CUDA(ctx, cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming));
+        for (int c = 0; c < tsr_ctx::NPIPE; ++c) {
+            TSR_CUDA(ctx, cudaEventCreateWithFlags(&ctx->ev_pipe_in[c], cudaEventDisableTiming));
+            TSR_CUDA(ctx, cudaEventCreateWithFlags(&ctx->ev_pipe_done[c], cudaEventDisableTiming));
+        }
         ctx->aux_ready = true;
     }
     ctx->bound = true;
@@ -1176,25 +1183,75 @@ tsr_status tsr_step_grouped_host(tsr_ctx *ctx, const void *const *G_host, float 
     if ((s = check_hyper(ctx, hyper)) != TSR_OK) return s;
     cudaStream_t st = (cudaStream_t)stream;
     const int nb = (int)ctx->blocks.size();
+    bool refresh_due = false;
     for (int i = 0; i < nb; ++i) {
         const Block &b = ctx->blocks[i];
         if (!G_host[i]) return fail(ctx, TSR_ERR_INVALID_ARG, "G_host[%d] is NULL", i);
-        const size_t es = (size_t)elem_size(b.d.g_dtype);
-        TSR_CUDA(ctx, cudaMemcpy2DAsync(const_cast<void *>(b.p.G), (size_t)b.d.ldg * es, G_host[i], (size_t)b.d.n * es,
-                                        (size_t)b.d.n * es, (size_t)b.d.m, cudaMemcpyHostToDevice, st));
+        if (b.d.K > 0 && hyper->step % b.d.K == 0) refresh_due = true;
     }
-    if ((s = tsr_step_grouped(ctx, hyper, seed, fuse_adam, stream)) != TSR_OK) return s;
-    if (C_host) {
+    auto copy_in = [&](int i, cudaStream_t cs) -> cudaError_t {
+        const Block &b = ctx->blocks[i];
+        const size_t es = (size_t)elem_size(b.d.g_dtype);
+        return cudaMemcpy2DAsync(const_cast<void *>(b.p.G), (size_t)b.d.ldg * es, G_host[i], (size_t)b.d.n * es,
+                                 (size_t)b.d.n * es, (size_t)b.d.m, cudaMemcpyHostToDevice, cs);
+    };
+    std::vector<size_t> c_off(nb, 0);
+    {
         size_t off = 0;
-        for (int i = 0; i < nb; ++i) {
-            const Block &b = ctx->blocks[i];
-            const size_t cnt = (size_t)b.d.r * b.d.r;
-            TSR_CUDA(ctx, cudaMemcpyAsync(C_host + off, b.p.C, cnt * sizeof(float), cudaMemcpyDeviceToHost, st));
-            off += cnt;
+        for (int i = 0; i < nb; ++i) { c_off[i] = off; off += (size_t)ctx->blocks[i].d.r * ctx->blocks[i].d.r; }
+    }
+    auto copy_out = [&](int i, cudaStream_t cs) -> cudaError_t {
+        const Block &b = ctx->blocks[i];
+        return cudaMemcpyAsync(C_host + c_off[i], b.p.C, (size_t)b.d.r * b.d.r * sizeof(float), cudaMemcpyDeviceToHost, cs);
+    };
+    constexpr int NCHUNK = tsr_ctx::NPIPE;
+    if (refresh_due || !ctx->aux_ready || nb < 2 * NCHUNK) {
+        // plain order: all gradients in, the step, all cores out
+        for (int i = 0; i < nb; ++i) TSR_CUDA(ctx, copy_in(i, st));
+        if ((s = tsr_step_grouped(ctx, hyper, seed, fuse_adam, stream)) != TSR_OK) return s;
+        if (C_host)
+            for (int i = 0; i < nb; ++i) TSR_CUDA(ctx, copy_out(i, st));
+        TSR_CUDA(ctx, cudaStreamSynchronize(st));
+        return TSR_OK;
+    }
+    // Pipelined order (no refresh in this step): the blocks go in chunks of about equal gradient bytes;
+    // while chunk c is stepped on the caller's stream, chunk c + 1 arrives on one side stream and the
+    // cores of chunk c - 1 leave on another, so the step hides behind the host link.
+    size_t total_bytes = 0;
+    for (const Block &b : ctx->blocks) total_bytes += (size_t)b.d.m * b.d.n * elem_size(b.d.g_dtype);
+    std::vector<std::vector<int>> chunks(NCHUNK);
+    {
+        size_t acc = 0;
+        for (int bi : ctx->order) {
+            const Block &b = ctx->blocks[bi];
+            const int c = (int)std::min<size_t>(NCHUNK - 1, acc * NCHUNK / std::max<size_t>(1, total_bytes));
+            chunks[c].push_back(bi);
+            acc += (size_t)b.d.m * b.d.n * elem_size(b.d.g_dtype);
         }
     }
+    cudaStream_t s_in = ctx->aux[0], s_out = ctx->aux[1];
+    TSR_CUDA(ctx, cudaEventRecord(ctx->ev_fork, st));
+    TSR_CUDA(ctx, cudaStreamWaitEvent(s_in, ctx->ev_fork, 0));
+    TSR_CUDA(ctx, cudaStreamWaitEvent(s_out, ctx->ev_fork, 0));
+    for (int c = 0; c < NCHUNK; ++c) {
+        for (int bi : chunks[c]) TSR_CUDA(ctx, copy_in(bi, s_in));
+        TSR_CUDA(ctx, cudaEventRecord(ctx->ev_pipe_in[c], s_in));
+    }
+    tsr_status result = TSR_OK;
+    for (int c = 0; c < NCHUNK; ++c) {
+        if (chunks[c].empty()) continue;
+        TSR_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_pipe_in[c], 0));
+        if ((s = do_step(ctx, chunks[c], hyper, seed, fuse_adam != 0, st)) != TSR_OK && result == TSR_OK) result = s;
+        if (C_host) {
+            TSR_CUDA(ctx, cudaEventRecord(ctx->ev_pipe_done[c], st));
+            TSR_CUDA(ctx, cudaStreamWaitEvent(s_out, ctx->ev_pipe_done[c], 0));
+            for (int bi : chunks[c]) TSR_CUDA(ctx, copy_out(bi, s_out));
+        }
+    }
+    TSR_CUDA(ctx, cudaEventRecord(ctx->ev_join[0], s_out));
+    TSR_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_join[0], 0));
     TSR_CUDA(ctx, cudaStreamSynchronize(st));
-    return TSR_OK;
+    return result;
 }
 
 // ---- single-block calls ---------------------------------------------------------------------

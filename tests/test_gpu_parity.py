@@ -343,24 +343,30 @@ def test_unaligned_leading_dimension_takes_cuda_core_path():
     _run_steps(tsr, plan, shapes, torch.bfloat16, 3, True, TOL_F32)
 
 
-def test_step_from_host_buffers():
+@pytest.mark.parametrize("copies", [1, 10])
+def test_step_from_host_buffers(copies):
+    """The host-buffer step gives exactly the device-buffer step; with 20 blocks it takes the
+    chunked, overlapped order (copies in, step, cores out on three streams)."""
     import paper_2602_08007_b200 as tsr
-    shapes = BF16_SHAPES[:2]
+    shapes = BF16_SHAPES[:2] * copies
+    nb = len(shapes)
     plan = tsr.Plan(shapes, g_dtype=torch.bfloat16)
     ref = tsr.Plan(shapes, g_dtype=torch.bfloat16)
     for pl in (plan, ref):
         _given_bases(pl, shapes)
-        for i in range(2):
+        for i in range(nb):
             fill_weights(pl, i, 60 + i)
     gh = [ti.gradient(s["m"], s["n"], 70 + i, dtype=torch.bfloat16).contiguous().pin_memory() for i, s in enumerate(shapes)]
     c_host = torch.empty(sum(s["r"] ** 2 for s in shapes), dtype=torch.float32).pin_memory()
-    plan.step_host(gh, c_host, tsr.make_hyper(1))
-    for i in range(2):
-        ref.G[i].copy_(gh[i].cuda())
-    ref.step(tsr.make_hyper(1))
-    torch.cuda.synchronize()
-    off = 0
-    for i, s in enumerate(shapes):
-        assert torch.equal(plan.W[i], ref.W[i])
-        assert torch.equal(c_host[off:off + s["r"] ** 2].view(s["r"], s["r"]), ref.C[i].cpu())
-        off += s["r"] ** 2
+    for t in (1, 2):
+        plan.step_host(gh, c_host, tsr.make_hyper(t))
+        for i in range(nb):
+            ref.G[i].copy_(gh[i].cuda())
+        ref.step(tsr.make_hyper(t))
+        torch.cuda.synchronize()
+        off = 0
+        for i, s in enumerate(shapes):
+            assert torch.equal(plan.W[i], ref.W[i])
+            assert torch.equal(c_host[off:off + s["r"] ** 2].view(s["r"], s["r"]), ref.C[i].cpu())
+            off += s["r"] ** 2
+    assert plan.poll_status() == [0] * nb
