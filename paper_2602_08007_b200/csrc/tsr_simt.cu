@@ -112,28 +112,65 @@ cudaError_t simt_gemm(int M, int N, int K, const void *A, int a_dtype, int64_t s
 // the fused and the unfused orders agree bit for bit.
 // ---------------------------------------------------------------------------------------
 // mode 0: full update; mode 1: only sum the split-K slabs into Cout.
-__global__ void core_update_kernel(const CoreUpdateArgs *__restrict__ args, const int32_t *__restrict__ list,
-                                   StepScalars sc, int mode)
+// One CTA per 32 x 128 strip of the core (four 32 x 32 tiles): every global access is a full
+// 128-byte (FP32) or 64-byte (BF16) row segment, the loads of a tile are issued before its
+// arithmetic, and the transposed BF16 copy of D goes through shared memory.
+constexpr int CU_TILES = 4;
+
+__global__ void __launch_bounds__(256)
+core_update_kernel(const CoreUpdateArgs *__restrict__ args, const int32_t *__restrict__ list, StepScalars sc, int mode)
 {
-    const CoreUpdateArgs a = args[list[blockIdx.y]];
+    const CoreUpdateArgs a = args[list[blockIdx.z]];
     const int r = a.r;
-    const int64_t total = (int64_t)r * r;
-    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
-        float c = a.C[e];
-        if (a.nsplit > 1) {
-            for (int s = 1; s < a.nsplit; ++s) c = __fadd_rn(c, a.C[e + (int64_t)s * a.split_stride]);
-            a.Cout[e] = c;
+    const int r0 = blockIdx.y * 32;
+    if (r0 >= r || blockIdx.x * 32 * CU_TILES >= r) return;
+    __shared__ float tile[CU_TILES][32][33];
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    const bool sgd = (sc.rule == TSR_RULE_SGD);
+#pragma unroll
+    for (int tt = 0; tt < CU_TILES; ++tt) {
+        const int c0 = (blockIdx.x * CU_TILES + tt) * 32;
+        const int col = c0 + tx;
+        float c[4], m1[4], m2[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int row = r0 + ty + 8 * u;
+            const bool in = (row < r && col < r);
+            const int64_t e = (int64_t)row * r + col;
+            c[u] = in ? a.C[e] : 0.f;
+            if (in && a.nsplit > 1)
+                for (int s = 1; s < a.nsplit; ++s) c[u] = __fadd_rn(c[u], a.C[e + (int64_t)s * a.split_stride]);
+            m1[u] = (in && mode == 0) ? a.mom1[e] : 0.f;
+            m2[u] = (in && mode == 0 && !sgd) ? a.mom2[e] : 0.f;
         }
-        if (mode == 1) continue;
-        float m1 = a.mom1[e];
-        float m2 = (sc.rule == TSR_RULE_SGD) ? 0.f : a.mom2[e];
-        const float d = core_update_elem(c, m1, m2, sc);
-        a.mom1[e] = m1;
-        if (sc.rule != TSR_RULE_SGD) a.mom2[e] = m2;
-        if (a.d_f32) a.d_f32[e] = d;
-        const int row = (int)(e / r), col = (int)(e % r);
-        if (a.d_bf16) a.d_bf16[(int64_t)row * a.ldd + col] = __float2bfloat16_rn(d);
-        if (a.dt_bf16) a.dt_bf16[(int64_t)col * a.ldd + row] = __float2bfloat16_rn(d);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int row = r0 + ty + 8 * u;
+            const bool in = (row < r && col < r);
+            const int64_t e = (int64_t)row * r + col;
+            float d = 0.f;
+            if (in) {
+                if (a.nsplit > 1) a.Cout[e] = c[u];
+                if (mode == 0) {
+                    d = core_update_elem(c[u], m1[u], m2[u], sc);
+                    a.mom1[e] = m1[u];
+                    if (!sgd) a.mom2[e] = m2[u];
+                    if (a.d_f32) a.d_f32[e] = d;
+                    if (a.d_bf16) a.d_bf16[(int64_t)row * a.ldd + col] = __float2bfloat16_rn(d);
+                }
+            }
+            tile[tt][ty + 8 * u][tx] = d;
+        }
+    }
+    if (mode != 0 || a.dt_bf16 == nullptr) return;
+    __syncthreads();
+#pragma unroll
+    for (int tt = 0; tt < CU_TILES; ++tt) {
+        const int c0 = (blockIdx.x * CU_TILES + tt) * 32;
+        for (int i = ty; i < 32; i += 8) {
+            const int col = c0 + i, row = r0 + tx;
+            if (row < r && col < r) a.dt_bf16[(int64_t)col * a.ldd + row] = __float2bfloat16_rn(tile[tt][tx][i]);
+        }
     }
 }
 
@@ -141,10 +178,8 @@ cudaError_t core_update_launch(const CoreUpdateArgs *args_dev, const int32_t *li
                                const StepScalars &sc, int mode, cudaStream_t stream)
 {
     if (nblocks <= 0) return cudaSuccess;
-    int gx = (int)(((int64_t)max_r * max_r + 255) / 256);
-    if (gx > 64) gx = 64;
-    if (gx < 1) gx = 1;
-    core_update_kernel<<<dim3(gx, nblocks), 256, 0, stream>>>(args_dev, list_dev, sc, mode);
+    const int t = (max_r + 31) / 32;
+    core_update_kernel<<<dim3((t + CU_TILES - 1) / CU_TILES, t, nblocks), 256, 0, stream>>>(args_dev, list_dev, sc, mode);
     return cudaGetLastError();
 }
 
