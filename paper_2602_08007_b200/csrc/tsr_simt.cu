@@ -40,20 +40,36 @@ simt_gemm_kernel(int M, int N, int K, const TA *__restrict__ A, int64_t sa_i, in
     const bool a_k_fast = (sa_k == 1);
     const bool b_j_fast = (sb_j == 1);
 
-    for (int k0 = 0; k0 < K; k0 += SG_BK) {
+    // global -> registers -> shared, with the next K slice in flight while the current one is used
+    float ra[4], rb[4];
+    auto fetch = [&](int k0) {
 #pragma unroll
         for (int l = 0; l < 4; ++l) {
             const int e = tid + l * 256;  // 0..1023
             int ai, ak;
             if (a_k_fast) { ak = e % SG_BK; ai = e / SG_BK; } else { ai = e % SG_BM; ak = e / SG_BM; }
             const int gi = m0 + ai, gk = k0 + ak;
-            As[ak][ai] = (gi < M && gk < K) ? load_as_float<TA>(A + (int64_t)gi * sa_i + (int64_t)gk * sa_k) : 0.f;
+            ra[l] = (gi < M && gk < K) ? load_as_float<TA>(A + (int64_t)gi * sa_i + (int64_t)gk * sa_k) : 0.f;
             int bj, bk;
             if (b_j_fast) { bj = e % SG_BN; bk = e / SG_BN; } else { bk = e % SG_BK; bj = e / SG_BK; }
             const int gj = n0 + bj, gk2 = k0 + bk;
-            Bs[bk][bj] = (gj < N && gk2 < K) ? B[(int64_t)gk2 * sb_k + (int64_t)gj * sb_j] : 0.f;
+            rb[l] = (gj < N && gk2 < K) ? B[(int64_t)gk2 * sb_k + (int64_t)gj * sb_j] : 0.f;
+        }
+    };
+    fetch(0);
+    for (int k0 = 0; k0 < K; k0 += SG_BK) {
+#pragma unroll
+        for (int l = 0; l < 4; ++l) {
+            const int e = tid + l * 256;
+            int ai, ak;
+            if (a_k_fast) { ak = e % SG_BK; ai = e / SG_BK; } else { ai = e % SG_BM; ak = e / SG_BM; }
+            As[ak][ai] = ra[l];
+            int bj, bk;
+            if (b_j_fast) { bj = e % SG_BN; bk = e / SG_BN; } else { bk = e % SG_BK; bj = e / SG_BK; }
+            Bs[bk][bj] = rb[l];
         }
         __syncthreads();
+        if (k0 + SG_BK < K) fetch(k0 + SG_BK);
 #pragma unroll
         for (int kk = 0; kk < SG_BK; ++kk) {
             float av[4], bv[4];
