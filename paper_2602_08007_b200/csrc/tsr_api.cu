@@ -328,6 +328,20 @@ tsr_status encode_map_f32(tsr_ctx *ctx, CUtensorMap *out, const void *base, int6
     return TSR_OK;
 }
 
+// BF16 row-major output [rows x cols] (ld elements) -> tensor map with a 32 x 32 box (64-byte rows), 64B swizzle.
+tsr_status encode_map_out_bf16(tsr_ctx *ctx, CUtensorMap *out, const void *base, int64_t rows, int64_t cols, int64_t ld)
+{
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+    cuuint32_t box[2] = {32, 32};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult rc = ctx->encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+                              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (rc != CUDA_SUCCESS) return fail(ctx, TSR_ERR_CUDA, "cuTensorMapEncodeTiled (BF16 output) failed (%d)", (int)rc);
+    return TSR_OK;
+}
+
 // FP32 row-major [rows x cols] (ld elements) -> tensor map with a 32 x 32 box, 128B swizzle.
 tsr_status encode_map_w(tsr_ctx *ctx, CUtensorMap *out, const void *base, int64_t rows, int64_t cols, int64_t ld)
 {
@@ -998,6 +1012,8 @@ tsr_status tsr_bind(tsr_ctx *ctx, const tsr_mat_ptrs *ptrs, int32_t count, void 
             if ((s = encode_map(ctx, &P.tmA, b.Ub, m, r, b.rl, 128)) != TSR_OK) return s;
             if ((s = encode_map(ctx, &P.tmB, b.Dbt, r, r, b.rl, ctx->bn[KP] / 2)) != TSR_OK) return s;
             P.out = b.Pb; P.ld_out = b.rl;
+            if ((s = encode_map_out_bf16(ctx, &P.tmW, b.Pb, m, r, b.rl)) != TSR_OK) return s;
+            P.out_tma = 1;
         }
         {   // W update : A = P [m x r], B = V copy [n x r]
             UmmaProblem &P = probs[KA][i];

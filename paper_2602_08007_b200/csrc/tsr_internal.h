@@ -34,7 +34,8 @@ enum UmmaEpilogue : int {
 struct alignas(64) UmmaProblem {
     CUtensorMap tmA;       // box 64 (K) x 128 (M rows), 128-byte swizzle
     CUtensorMap tmB;       // box 64 (K) x BN (N rows); plane 1 lives plane_rows rows below plane 0
-    CUtensorMap tmW;       // apply only: FP32 W, box 32 columns x 32 rows, 128-byte swizzle
+    CUtensorMap tmW;       // apply: FP32 W, box 32 columns x 32 rows, 128-byte swizzle; EPI_STORE_BF16 with out_tma: the
+                           // BF16 output, box 32 columns x 32 rows, 64-byte swizzle
     int32_t M, N, K;
     int32_t planes;        // 1 or 2
     int32_t plane_rows;    // row offset of the second plane inside the B tensor map
@@ -49,6 +50,7 @@ struct alignas(64) UmmaProblem {
     bf16 *d_bf16;          // D   [r x ldd]
     bf16 *dt_bf16;         // D^T [r x ldd]
     int64_t ldd;
+    int32_t out_tma;       // EPI_STORE_BF16: tmW describes the output, chunks leave through TMA stores
 };
 
 struct UmmaTile {

@@ -180,6 +180,7 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
         const int q = warp & 3;
         const int half = (warp - 4) >> 2;
         float *patch = (float *)(smem + SM::PATCH_OFFSET + (warp - 4) * SM::PATCH_BYTES);   // [32][33]
+        uint32_t nbox = 0;       // EPI_STORE_BF16 through TMA: boxes written so far
         uint32_t tc = 0;
         bool ok = true;
         for (int t = pair; t < num_tiles && ok; t += stride, ++tc) {
@@ -245,6 +246,33 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
                             *(float4 *)(out + j) = make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]),
                                                                __uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
                     }
+                    continue;
+                }
+                if (EPI == EPI_STORE_BF16 && P->out_tma) {
+                    // The chunk goes to a 32 x 32 BF16 box in shared memory (64-byte rows, 64-byte swizzle;
+                    // two boxes per warp inside the patch area) and leaves as one TMA store, which writes
+                    // whole lines and clips at the matrix edge.  Direct stores from the lane = row layout
+                    // cost one 16-byte write request per lane and instruction and were the bound of P = U D.
+                    uint8_t *box = smem + SM::PATCH_OFFSET + (((warp - 4) * 2 + (int)(nbox & 1u)) << 11);
+                    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                    __syncwarp();
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        uint4 pk;
+                        __nv_bfloat162 h0 = __floats2bfloat162_rn(__uint_as_float(v[8 * j]), __uint_as_float(v[8 * j + 1]));
+                        __nv_bfloat162 h1 = __floats2bfloat162_rn(__uint_as_float(v[8 * j + 2]), __uint_as_float(v[8 * j + 3]));
+                        __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(v[8 * j + 4]), __uint_as_float(v[8 * j + 5]));
+                        __nv_bfloat162 h3 = __floats2bfloat162_rn(__uint_as_float(v[8 * j + 6]), __uint_as_float(v[8 * j + 7]));
+                        pk.x = *(uint32_t *)&h0; pk.y = *(uint32_t *)&h1; pk.z = *(uint32_t *)&h2; pk.w = *(uint32_t *)&h3;
+                        *(uint4 *)(box + lane * 64 + ((j ^ ((lane >> 1) & 3)) << 4)) = pk;
+                    }
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
+                    if (lane == 0) {
+                        tma_store_2d(&P->tmW, smem_u32(box), col0, row0);
+                        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                    }
+                    ++nbox;
                     continue;
                 }
                 if (EPI == EPI_STORE_BF16 && ncols == 32 && (P->ld_out & 7) == 0 && (col0 & 7) == 0 &&
@@ -344,6 +372,8 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
                 __syncwarp();
             }
         }
+        // TMA stores read their boxes asynchronously: they must have done so before the CTA goes away
+        if (EPI == EPI_STORE_BF16 && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     }
     if (s_timeout) __nanosleep(2000000);   // let copies in flight land before the CTA goes away
     tc_fence_before();

@@ -44,13 +44,6 @@ struct ApplyCfg {
     static constexpr uint32_t TMEM_COLS = 2 * BN;
 };
 
-__device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, uint32_t src, int x, int y)
-{
-    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
-                 ::"l"((uint64_t)map), "r"(src), "r"(x), "r"(y)
-                 : "memory");
-}
-
 struct ChunkCursor {   // walks the (tile, 32-column chunk) sequence of this CTA
     int tile_idx;      // index into the tile table; >= num_tiles: exhausted
     int c;             // chunk inside the tile
