@@ -240,11 +240,15 @@ def max_over_ranks(values, dist, device):
 
 
 # Measured DRAM traffic of umma_apply_kernel divided by its algorithmic bytes (8 B per weight +
-# BF16 operands), from the ncu capture summarised in profiles/umma_apply_kernel.md.  The
-# 1B workload is too large for a multi-pass capture; traffic grows in proportion to the weights, so
-# the ratio measured on smaller sets (0.98 on the 350M set and on a six-layer slice of the 1B set)
-# is applied to the 1B algorithmic bytes.
-APPLY_TRAFFIC_RATIO = 0.98
+# BF16 operands), from the ncu captures summarised in profiles/umma_apply_kernel.md: 0.98 on the
+# 350M set and on a six-layer slice of the 1B set (full captures), and 11.19 GB against 11.16 GB
+# algorithmic on the full 1B set (a one-pass capture of dram__bytes_read.sum + dram__bytes_write.sum).
+APPLY_TRAFFIC_RATIO = {3: 0.98, 4: 1.00}
+
+
+def apply_traffic_ratio(config_id: int) -> float:
+    return APPLY_TRAFFIC_RATIO.get(config_id, 0.98)
+
 
 def build_plan(w: ti.Workload, device):
     import paper_2602_08007_b200 as tsr
@@ -437,7 +441,7 @@ def run_ours(args, w: ti.Workload):
                          "gemm_UD": st_med[4], "apply": st_med[5]},
             "roofline": {"kernel": "umma_apply_kernel (W <- decay W - lr P V^T)", "bound": "hbm",
                          "achieved": apply_gbs, "peak": hbm, "unit": "GB/s", "frac": apply_gbs / hbm,
-                         "traffic": APPLY_TRAFFIC_RATIO * work["apply_kernel_bytes"],
+                         "traffic": apply_traffic_ratio(w.config_id) * work["apply_kernel_bytes"],
                          "algorithmic_bytes": work["apply_kernel_bytes"],
                          "peak_source": peaks["source"] + " copy bandwidth", "ms": apply_ms, "roof_ms": apply_roof_ms},
             "roofline_projection": {"kernels": "umma_gemm_kernel<EPI_STORE_BF16_T> + <EPI_CORE_UPDATE>",
