@@ -41,6 +41,10 @@ struct Block {
     double *tau = nullptr, *dvec = nullptr, *evec = nullptr;
     double2 *rot = nullptr;
     int2 *sweeps = nullptr, *groups = nullptr;
+    double *dc_z = nullptr, *dc_scal = nullptr;
+    int32_t *dc_nd = nullptr, *dc_info = nullptr;
+    int2 *dc_rot_idx = nullptr;
+    double2 *dc_rot_cs = nullptr;
     float *Xs = nullptr, *Bts = nullptr;   // TF32 operand planes (value truncated to TF32, remainder): rows, small matrix^T
     bool tc_rows = false;                  // tall-times-small products of the refresh run on tensor cores
     int32_t *nsweeps = nullptr, *rank = nullptr;
@@ -215,11 +219,16 @@ void layout(tsr_ctx *ctx, Arena &a, bool assign, size_t *step_end)
         const int rot_cap = (int)std::min<int64_t>(eig_rot_capacity((int)k), 0x7fffffff), sweep_cap = (int)(64 * k);
         void *tau = a.take((size_t)k * 8), *dv = a.take((size_t)k * 8), *ev = a.take((size_t)k * 8);
         void *rot = a.take((size_t)rot_cap * 16), *sw = a.take((size_t)sweep_cap * 8);
-        void *grp = a.take((size_t)(sweep_cap / 32 + 1) * 8);
-        void *nsw = a.take(4), *rk = a.take((size_t)k * 4);
+        void *grp = a.take((size_t)(sweep_cap / 32 + 4) * 8);
+        void *nsw = a.take(16), *rk = a.take((size_t)k * 4);
+        // divide-and-conquer merge: z vector, list of coordinates that take part, deflation rotations, scalars
+        void *dcz = a.take((size_t)k * 8), *dcnd = a.take((size_t)k * 4), *dcri = a.take((size_t)k * 8), *dcrc = a.take((size_t)k * 16);
+        void *dcs = a.take(64), *dci = a.take(64);
         if (assign) {
             b.tau = (double *)tau; b.dvec = (double *)dv; b.evec = (double *)ev; b.rot = (double2 *)rot;
             b.sweeps = (int2 *)sw; b.groups = (int2 *)grp; b.nsweeps = (int32_t *)nsw; b.rank = (int32_t *)rk;
+            b.dc_z = (double *)dcz; b.dc_nd = (int32_t *)dcnd; b.dc_rot_idx = (int2 *)dcri; b.dc_rot_cs = (double2 *)dcrc;
+            b.dc_scal = (double *)dcs; b.dc_info = (int32_t *)dci;
             b.rot_cap = rot_cap; b.sweep_cap = sweep_cap;
         }
         if (b.d.flags & TSR_BLOCK_REEXPRESS_MOMENT) {
@@ -986,6 +995,8 @@ tsr_status tsr_bind(tsr_ctx *ctx, const tsr_mat_ptrs *ptrs, int32_t count, void 
         rd.Rinv = b.Rinv; rd.Wu = b.Wu; rd.Wv = b.Wv; rd.U = b.p.U; rd.V = b.p.V; rd.status = ctx->d_status + i;
         rd.tau = b.tau; rd.dvec = b.dvec; rd.evec = b.evec; rd.rot = b.rot; rd.sweeps = b.sweeps; rd.groups = b.groups; rd.nsweeps = b.nsweeps;
         rd.rank = b.rank; rd.rot_cap = b.rot_cap; rd.sweep_cap = b.sweep_cap;
+        rd.dc_z = b.dc_z; rd.dc_nd = b.dc_nd; rd.dc_rot_idx = b.dc_rot_idx; rd.dc_rot_cs = b.dc_rot_cs;
+        rd.dc_scal = b.dc_scal; rd.dc_info = b.dc_info;
         if (!b.fast) continue;
         auto base = [&](UmmaProblem &P, int M, int N, int K, int epi) {
             P.M = M; P.N = N; P.K = K; P.planes = 1; P.plane_rows = 0; P.block = i; P.epilogue = epi;

@@ -210,95 +210,121 @@ __device__ __forceinline__ double rsqrt_nocheck(double x)
     return fma(y * e, fma(0.375, e, 0.5), y);
 }
 
-__global__ void __launch_bounds__(32)
-ql_log_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ list)
+// One QL problem: d[0..n), e[0..n) (e[n-1] is not used) in shared memory, run by one thread.
+// Returns the number of sweeps logged, or -1 when a budget ran out.
+__device__ int ql_run(double *d, double *e, int n, double2 *__restrict__ rot, int64_t rot_cap, int2 *__restrict__ sweeps,
+                      int sweep_cap, int2 *__restrict__ groups)
+{
+    int nrot = 0, nsw = 0;
+    int64_t next_row = 0;                     // first free row of the skewed log
+    double2 *lane_rot = rot;                  // rot + (base * 32 + t) + 32 * SYS_LAG * t
+    for (int l = 0; l < n; ++l) {
+        int iter = 0;
+        while (true) {
+            int m = l;
+            for (; m < n - 1; ++m) {
+                const double dd = fabs(d[m]) + fabs(d[m + 1]);
+                if (fabs(e[m]) <= QL_TOL * dd) break;
+            }
+            if (m == l) break;
+            if (++iter > 60 || nsw >= sweep_cap) return -1;
+            {
+                const int t = nsw & 31;
+                if (t == 0) {                 // a new group starts with this sweep
+                    const int E = n - l + 1;
+                    if ((next_row + E + SYS_FILL + 2 * SYS_PF) * 32 > rot_cap) return -1;
+                    groups[nsw >> 5] = make_int2((int)next_row, E);
+                    next_row += E + SYS_FILL;
+                }
+                const int2 gr = groups[nsw >> 5];
+                lane_rot = rot + ((int64_t)gr.x + SYS_LAG * t) * 32 + t;
+            }
+            double g = (d[l + 1] - d[l]) / (2.0 * e[l]);
+            double r = sqrt(g * g + 1.0);
+            g = d[m] - d[l] + e[l] / (g + (g >= 0.0 ? r : -r));
+            double s = 1.0, c = 1.0, p = 0.0;
+            const int first = nrot;
+            int i = m - 1;
+            bool early = false;
+            // The loop is one dependent chain g -> r2 -> 1/sqrt(r2) -> g.  Everything that does not need
+            // the reciprocal square root is formed before it: with rinv = 1/sqrt(f^2 + g^2),
+            // s = f rinv, c = g rinv, (d[i] - g1) s + 2 c b = u rinv with u = (d[i] - g1) f + 2 g b,
+            // so p = s (u rinv) = f u rinv^2 and the next g = c (u rinv) - b = g u rinv^2 - b.
+            // d[i+1] and the next d[i], e[i] travel in registers (fetched ahead of the stores).
+            double e_nx = e[i], d_nx = d[i], dprev = d[m];
+            double2 *lr = lane_rot + (int64_t)(n - 1 - i) * 32;
+            for (; i >= l; --i) {
+                const double ei = e_nx, di = d_nx;
+                if (i > l) { e_nx = e[i - 1]; d_nx = d[i - 1]; }
+                const double f = s * ei, b = c * ei;
+                // r = hypot(f, g).  The entries are bounded by the eigenvalues of a Gram matrix of FP32
+                // data, so the squares stay far inside the FP64 range and no rescaling is needed.
+                const double r2 = fma(f, f, g * g);
+                if (r2 == 0.0) { e[i + 1] = 0.0; d[i + 1] = dprev - p; e[m] = 0.0; early = true; break; }
+                const double g1 = dprev - p;
+                const double u = fma(di - g1, f, 2.0 * g * b);
+                const double gu = g * u, fu = f * u;
+                const double rinv = rsqrt_nocheck(r2);
+                const double rinv2 = rinv * rinv;
+                const double gn = fma(gu, rinv2, -b);     // the chain continues here
+                p = fu * rinv2;
+                s = f * rinv;
+                c = g * rinv;
+                g = gn;
+                e[i + 1] = r2 * rinv;
+                d[i + 1] = g1 + p;
+                *lr = make_double2(c, s);
+                lr += 32;
+                ++nrot;
+                dprev = di;
+            }
+            if (nrot > first) sweeps[nsw++] = make_int2(m - 1, nrot - first);
+            if (early) continue;
+            d[l] -= p;
+            e[l] = g;
+            e[m] = 0.0;
+        }
+    }
+    return nsw;
+}
+
+// dc = 0: one problem of size k, run by warp 0.  dc = 1 (divide and conquer, Cuppen): the matrix is
+// torn at s = k / 2, T = diag(T1', T2') + rho u u^T with rho = e[s-1], u = e_{s-1} + e_s and the two
+// diagonal entries next to the tear reduced by rho; warp h runs the QL iteration of half h with its
+// own half of the log buffers, which takes a quarter of the serial chain of the whole problem.
+// The merge is done by dc_secular_kernel.  nsweeps[h] = sweeps of half h.
+__global__ void __launch_bounds__(64)
+ql_log_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ list, int dc)
 {
     extern __shared__ double ql_smem[];           // d[n], e[n]
     const RefreshDev D = rd[list[blockIdx.x]];
     const int n = D.k;
     double *d = ql_smem, *e = ql_smem + n;
-    for (int i = threadIdx.x; i < n; i += 32) { d[i] = D.dvec[i]; e[i] = D.evec[i]; }
-    __syncwarp();
-    if (threadIdx.x == 0) {
-        double2 *__restrict__ rot = D.rot;
-        int2 *__restrict__ sweeps = D.sweeps;
-        int2 *__restrict__ groups = D.groups;
-        int nrot = 0, nsw = 0;
-        int64_t next_row = 0;                     // first free row of the skewed log
-        double2 *lane_rot = rot;                  // rot + (base * 32 + t) + 32 * SYS_LAG * t
-        bool failed = false;
-        for (int l = 0; l < n && !failed; ++l) {
-            int iter = 0;
-            while (true) {
-                int m = l;
-                for (; m < n - 1; ++m) {
-                    const double dd = fabs(d[m]) + fabs(d[m + 1]);
-                    if (fabs(e[m]) <= QL_TOL * dd) break;
-                }
-                if (m == l) break;
-                if (++iter > 60 || nsw >= D.sweep_cap) { failed = true; break; }
-                {
-                    const int t = nsw & 31;
-                    if (t == 0) {                 // a new group starts with this sweep
-                        const int E = n - l + 1;
-                        if ((next_row + E + SYS_FILL + 2 * SYS_PF) * 32 > (int64_t)D.rot_cap) { failed = true; break; }
-                        groups[nsw >> 5] = make_int2((int)next_row, E);
-                        next_row += E + SYS_FILL;
-                    }
-                    const int2 gr = groups[nsw >> 5];
-                    lane_rot = rot + ((int64_t)gr.x + SYS_LAG * t) * 32 + t;
-                }
-                double g = (d[l + 1] - d[l]) / (2.0 * e[l]);
-                double r = sqrt(g * g + 1.0);
-                g = d[m] - d[l] + e[l] / (g + (g >= 0.0 ? r : -r));
-                double s = 1.0, c = 1.0, p = 0.0;
-                const int first = nrot;
-                int i = m - 1;
-                bool early = false;
-                // The loop is one dependent chain g -> r2 -> 1/sqrt(r2) -> g.  Everything that does not need
-                // the reciprocal square root is formed before it: with rinv = 1/sqrt(f^2 + g^2),
-                // s = f rinv, c = g rinv, (d[i] - g1) s + 2 c b = u rinv with u = (d[i] - g1) f + 2 g b,
-                // so p = s (u rinv) = f u rinv^2 and the next g = c (u rinv) - b = g u rinv^2 - b.
-                // d[i+1] and the next d[i], e[i] travel in registers (fetched ahead of the stores).
-                double e_nx = e[i], d_nx = d[i], dprev = d[m];
-                double2 *lr = lane_rot + (int64_t)(n - 1 - i) * 32;
-                for (; i >= l; --i) {
-                    const double ei = e_nx, di = d_nx;
-                    if (i > l) { e_nx = e[i - 1]; d_nx = d[i - 1]; }
-                    const double f = s * ei, b = c * ei;
-                    // r = hypot(f, g).  The entries are bounded by the eigenvalues of a Gram matrix of FP32
-                    // data, so the squares stay far inside the FP64 range and no rescaling is needed.
-                    const double r2 = fma(f, f, g * g);
-                    if (r2 == 0.0) { e[i + 1] = 0.0; d[i + 1] = dprev - p; e[m] = 0.0; early = true; break; }
-                    const double g1 = dprev - p;
-                    const double u = fma(di - g1, f, 2.0 * g * b);
-                    const double gu = g * u, fu = f * u;
-                    const double rinv = rsqrt_nocheck(r2);
-                    const double rinv2 = rinv * rinv;
-                    const double gn = fma(gu, rinv2, -b);     // the chain continues here
-                    p = fu * rinv2;
-                    s = f * rinv;
-                    c = g * rinv;
-                    g = gn;
-                    e[i + 1] = r2 * rinv;
-                    d[i + 1] = g1 + p;
-                    *lr = make_double2(c, s);
-                    lr += 32;
-                    ++nrot;
-                    dprev = di;
-                }
-                if (nrot > first) sweeps[nsw++] = make_int2(m - 1, nrot - first);
-                if (early) continue;
-                d[l] -= p;
-                e[l] = g;
-                e[m] = 0.0;
-            }
-        }
-        *D.nsweeps = nsw;
-        if (failed) atomicMax(D.status, (int)TSR_ERR_NOT_CONVERGED);
+    for (int i = threadIdx.x; i < n; i += 64) { d[i] = D.dvec[i]; e[i] = D.evec[i]; }
+    __syncthreads();
+    const int s = dc ? n / 2 : n;
+    if (dc && threadIdx.x == 0) {
+        const double rho = e[s - 1];
+        D.dc_scal[0] = rho;
+        d[s - 1] -= rho;
+        d[s] -= rho;
+        e[s - 1] = 0.0;
     }
-    __syncwarp();
-    for (int i = threadIdx.x; i < n; i += 32) D.dvec[i] = d[i];
+    __syncthreads();
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (lane == 0 && (warp == 0 || dc)) {
+        const int off = warp ? s : 0, nh = warp ? n - s : s;
+        const int64_t rcap = dc ? (int64_t)(D.rot_cap / 64) * 32 : (int64_t)D.rot_cap;   // entries per half
+        const int scap = dc ? D.sweep_cap / 2 : D.sweep_cap;
+        const int gcap = D.sweep_cap / 64 + 2;                                           // group slots per half
+        const int nsw = ql_run(d + off, e + off, nh, D.rot + (warp ? rcap : 0), rcap, D.sweeps + (warp ? scap : 0), scap,
+                               D.groups + (warp ? gcap : 0));
+        D.nsweeps[warp] = nsw < 0 ? 0 : nsw;
+        if (!dc) D.nsweeps[1] = 0;
+        if (nsw < 0) atomicMax(D.status, (int)TSR_ERR_NOT_CONVERGED);
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < n; i += 64) D.dvec[i] = d[i];
 }
 
 __global__ void eig_rank_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ list)
@@ -325,6 +351,7 @@ __global__ void eig_rank_kernel(const RefreshDev *__restrict__ rd, const int32_t
 // 3a: rows of Q = H_0 H_1 ... in registers.  A warp owns RQ rows (NW warps per CTA); lane holds columns lane + 32 i.
 // The reflectors are staged for the whole CTA, a few at a time, in shared memory.
 constexpr int SYS_KMAX = 1056;
+constexpr int DC_MIN_K = 200;    // the tridiagonal problem is torn in two from this size on
 constexpr int SYS_WARPS = 12;    // warps of the rotation kernel (three per scheduler)
 constexpr int QR_WARPS = 16;     // warps of the Q-rows kernel
 
@@ -402,41 +429,28 @@ eig_qrows_kernel(const RefreshDev *__restrict__ rd, const RowItem *__restrict__ 
 }
 
 // 3b: the logged rotations as a systolic pipeline.  A warp owns R rows of Q in shared memory.
-// Per group of 32 sweeps the columns k-1 ... lg of each row enter at lane 0, one per step; lane t
+// Per group of 32 sweeps the columns kh-1 ... lg of each row enter at lane 0, one per step; lane t
 // applies its sweep's rotation to the incoming column and the value it holds, passes the finished
 // column on to lane t+1 (one shuffle) and keeps the other; lane 31 writes the finished columns
 // back.  All 32 sweeps of a group advance in every step and the R rows are independent chains.
+// z: the warp's rows (row stride zs), already offset to the first of the kh columns the log acts on.
 template <int R>
-__global__ void __launch_bounds__(SYS_WARPS * 32)
-eig_rot_systolic_kernel(const RefreshDev *__restrict__ rd, const RowItem *__restrict__ items)
+__device__ __forceinline__ void systolic_apply(double *z, int zs, int kh, const double2 *__restrict__ rot,
+                                               const int2 *__restrict__ groups, const int2 *__restrict__ sweeps, int nsw,
+                                               int lane)
 {
-    extern __shared__ double zs[];                // [SYS_WARPS][R][k]
-    const RowItem it = items[blockIdx.x];
-    const RefreshDev D = rd[it.block];
-    const int k = D.k, r = D.r;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int row0 = it.row0 + warp * R;
-    if (row0 >= k) return;                        // warps never synchronise with one another
-    double *z = zs + (size_t)warp * R * k;
-#pragma unroll
-    for (int q = 0; q < R; ++q) {
-        const int row = min(row0 + q, k - 1);     // rows past the end shadow the last row, never stored
-        for (int c = lane; c < k; c += 32) z[q * k + c] = D.Wj[(int64_t)row * k + c];
-    }
-    __syncwarp();
-    const int nsw = *D.nsweeps;
     const int ngroups = (nsw + 31) >> 5;
     for (int g = 0; g < ngroups; ++g) {
-        const int2 gr = D.groups[g];
+        const int2 gr = groups[g];
         const int E = gr.y, T = E + SYS_FILL;
         const int sidx = 32 * g + lane;
         int hi = -1, lo = 0;                      // this lane's sweep acts on columns lo .. hi
-        if (sidx < nsw) { const int2 sw = D.sweeps[sidx]; hi = sw.x; lo = sw.x - sw.y + 1; }
-        const double2 *__restrict__ rp = D.rot + (int64_t)gr.x * 32 + lane;
+        if (sidx < nsw) { const int2 sw = sweeps[sidx]; hi = sw.x; lo = sw.x - sw.y + 1; }
+        const double2 *__restrict__ rp = rot + (int64_t)gr.x * 32 + lane;
         double held[R], out[R];
 #pragma unroll
         for (int q = 0; q < R; ++q) { held[q] = 0.0; out[q] = 0.0; }
-        int j = k - 1 + SYS_LAG * lane;           // column this lane consumes at step tau
+        int j = kh - 1 + SYS_LAG * lane;          // column this lane consumes at step tau
         // the rotations of the next SYS_PF steps are fetched while the current ones are applied
         double2 nxt[SYS_PF];
 #pragma unroll
@@ -453,13 +467,13 @@ eig_rot_systolic_kernel(const RefreshDev *__restrict__ rd, const RowItem *__rest
                 if (tau >= T) break;
                 const bool act = (j <= hi) && (j >= lo);
                 const double c = act ? cur[u].x : 1.0, s = act ? cur[u].y : 0.0;
-                const int cin = max(k - 1 - tau, 0);      // column entering lane 0 (all lanes read it: a broadcast)
-                const int cout = k - (tau - SYS_FILL);    // column leaving lane 31
+                const int cin = max(kh - 1 - tau, 0);     // column entering lane 0 (all lanes read it: a broadcast)
+                const int cout = kh - (tau - SYS_FILL);   // column leaving lane 31
                 const bool feed = (lane == 0), real = (tau < E - 1);
                 const bool emit = (lane == 31) && (tau > SYS_FILL);
                 double zin[R];
 #pragma unroll
-                for (int q = 0; q < R; ++q) zin[q] = z[q * k + cin];
+                for (int q = 0; q < R; ++q) zin[q] = z[q * zs + cin];
 #pragma unroll
                 for (int q = 0; q < R; ++q) {
                     const double up = __shfl_up_sync(0xffffffffu, out[q], 1);
@@ -468,8 +482,281 @@ eig_rot_systolic_kernel(const RefreshDev *__restrict__ rd, const RowItem *__rest
                     const double o = fma(s, in, ch);
                     held[q] = fma(c, in, -sh);
                     out[q] = o;
-                    if (emit) z[q * k + cout] = o;
+                    if (emit) z[q * zs + cout] = o;
                 }
+            }
+        }
+        __syncwarp();
+    }
+}
+
+// Offsets of half 1's share of the log buffers (see ql_log_kernel).
+__device__ __forceinline__ int64_t dc_rot_off(const RefreshDev &D) { return (int64_t)(D.rot_cap / 64) * 32; }
+__device__ __forceinline__ int dc_sweep_off(const RefreshDev &D) { return D.sweep_cap / 2; }
+__device__ __forceinline__ int dc_group_off(const RefreshDev &D) { return D.sweep_cap / 64 + 2; }
+
+// Divide and conquer, step 2: z = Z^T u = (last row of Z1, first row of Z2), i.e. the logs of the
+// two halves applied to one unit row vector each (warp h = half h).
+__global__ void __launch_bounds__(64)
+dc_zrows_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ list)
+{
+    extern __shared__ double zr_smem[];          // k
+    const RefreshDev D = rd[list[blockIdx.x]];
+    const int k = D.k, s = k / 2;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int off = warp ? s : 0, kh = warp ? k - s : s;
+    double *z = zr_smem + off;
+    const int one = warp ? 0 : s - 1;            // e_{s-1} of half 0, e_0 of half 1
+    for (int c = lane; c < kh; c += 32) z[c] = (c == one) ? 1.0 : 0.0;
+    __syncwarp();
+    systolic_apply<1>(z, k, kh, D.rot + (warp ? dc_rot_off(D) : 0), D.groups + (warp ? dc_group_off(D) : 0),
+                      D.sweeps + (warp ? dc_sweep_off(D) : 0), D.nsweeps[warp], lane);
+    for (int c = lane; c < kh; c += 32) D.dc_z[off + c] = z[c];
+}
+
+// Divide and conquer, step 3: eigen-decomposition of D + rho z z^T (D = eigenvalues of the halves),
+// one CTA per matrix.  Sort, deflate (negligible z_i; nearly equal d_i, by a plane rotation), solve the
+// secular equation 1 + rho sum_i z_i^2 / (d_i - lambda) = 0 for one root per thread by bisection on
+// the distance tau from the nearer pole (so that all differences d_i - lambda keep full relative
+// accuracy), recompute z from the roots (Gu and Eisenstat's formula, which makes the eigenvectors
+// orthogonal to working precision however close the roots are), and write the eigenvector matrix
+// Uhat (K x K, row pitch k, in Xw), the coordinate list nd, the deflation rotations and the
+// eigenvalues of all k coordinates (dvec).
+constexpr int DC_THREADS = 512;
+
+__global__ void __launch_bounds__(DC_THREADS)
+dc_secular_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ list, int kpad)
+{
+    extern __shared__ double sc_smem[];          // ds, zs, dk, zk, tk, zh : 6 x kpad doubles; perm, org, state : 3 x kpad ints
+    const RefreshDev D = rd[list[blockIdx.x]];
+    const int n = D.k;
+    double *ds = sc_smem, *zs = ds + kpad, *dk = zs + kpad, *zk = dk + kpad, *tk = zk + kpad, *zh = tk + kpad;
+    int *perm = (int *)(zh + kpad), *org = perm + kpad, *state = org + kpad;
+    __shared__ int s_K, s_nr;
+    __shared__ double s_rho, s_flip;
+    const int tid = threadIdx.x, nt = blockDim.x;
+    double rho = D.dc_scal[0];
+    const double flip = (rho < 0.0) ? -1.0 : 1.0;   // solve for -T when rho < 0
+    rho = fabs(rho) * 2.0;                       // ||u||^2 = 2: z is normalised below
+    // sort ascending (rank sort); dk / zk serve as staging for the unsorted values
+    for (int i = tid; i < n; i += nt) { dk[i] = flip * D.dvec[i]; zk[i] = D.dc_z[i] * 0.70710678118654752440; }
+    __syncthreads();
+    for (int i = tid; i < n; i += nt) {
+        const double di = dk[i];
+        int rank = 0;
+        for (int j = 0; j < n; ++j) rank += (dk[j] < di || (dk[j] == di && j < i)) ? 1 : 0;
+        ds[rank] = di; zs[rank] = zk[i]; perm[rank] = i;
+    }
+    __syncthreads();
+    if (tid == 0) {
+        double dmax = 0.0, zmax = 0.0;
+        for (int p = 0; p < n; ++p) { dmax = fmax(dmax, fabs(ds[p])); zmax = fmax(zmax, fabs(zs[p])); }
+        const double tol = 8.0 * 2.220446049250313e-16 * fmax(dmax, zmax);
+        int K = 0, nr = 0, prev = -1;
+        if (!(rho * zmax > tol)) {               // the halves do not interact at working precision
+            for (int p = 0; p < n; ++p) state[p] = 0;
+        } else {
+            for (int p = 0; p < n; ++p) {
+                if (rho * fabs(zs[p]) <= tol) { state[p] = 0; continue; }
+                if (prev < 0) { prev = p; continue; }
+                double sN = zs[prev], cN = zs[p];
+                const double tauN = sqrt(cN * cN + sN * sN);
+                const double t = ds[p] - ds[prev];
+                cN /= tauN; sN = -sN / tauN;
+                if (fabs(t * cN * sN) <= tol) {  // rotate z[prev] into z[p]: prev deflates
+                    zs[p] = tauN; zs[prev] = 0.0;
+                    D.dc_rot_idx[nr] = make_int2(perm[prev], perm[p]);
+                    D.dc_rot_cs[nr] = make_double2(cN, sN);
+                    ++nr;
+                    const double tt = ds[prev] * cN * cN + ds[p] * sN * sN;
+                    ds[p] = ds[prev] * sN * sN + ds[p] * cN * cN;
+                    ds[prev] = tt;
+                    state[prev] = 0;
+                } else {
+                    state[prev] = 1; dk[K] = ds[prev]; zk[K] = zs[prev]; D.dc_nd[K] = perm[prev]; ++K;
+                }
+                prev = p;
+            }
+            if (prev >= 0) { state[prev] = 1; dk[K] = ds[prev]; zk[K] = zs[prev]; D.dc_nd[K] = perm[prev]; ++K; }
+        }
+        // dk is ascending except where a rotation moved a value: restore the order (insertion, rarely needed)
+        for (int a = 1; a < K; ++a) {
+            int bq = a;
+            while (bq > 0 && dk[bq - 1] > dk[bq]) {
+                const double td = dk[bq]; dk[bq] = dk[bq - 1]; dk[bq - 1] = td;
+                const double tz = zk[bq]; zk[bq] = zk[bq - 1]; zk[bq - 1] = tz;
+                const int ti = D.dc_nd[bq]; D.dc_nd[bq] = D.dc_nd[bq - 1]; D.dc_nd[bq - 1] = ti;
+                --bq;
+            }
+        }
+        s_K = K; s_nr = nr; s_rho = rho; s_flip = flip;
+        D.dc_info[0] = K; D.dc_info[1] = nr;
+    }
+    __syncthreads();
+    const int K = s_K;
+    // eigenvalues of the deflated coordinates
+    for (int p = tid; p < n; p += nt)
+        if (state[p] == 0) D.dvec[perm[p]] = flip * ds[p];
+    if (K == 0) return;
+    double z2sum = 0.0;
+    for (int i = 0; i < K; ++i) z2sum += zk[i] * zk[i];
+    // secular roots: lambda_j = dk[org[j]] + tk[j]
+    for (int j = tid; j < K; j += nt) {
+        int o;
+        double hi;        // |tau| lies in (0, hi]
+        double sgn;       // tau = sgn * sigma
+        if (j == K - 1) { o = j; hi = rho * z2sum; sgn = 1.0; }
+        else {
+            const double gap = dk[j + 1] - dk[j];
+            double f = 1.0;                       // f at the midpoint
+            for (int i = 0; i < K; ++i) f += rho * zk[i] * zk[i] / ((dk[i] - dk[j]) - 0.5 * gap);
+            if (f > 0.0) { o = j; sgn = 1.0; } else { o = j + 1; sgn = -1.0; }
+            hi = 0.5 * gap;
+        }
+        const double dorg = dk[o];
+        // g(sigma) = f(dorg + sgn sigma); sgn = +1: g increases from -inf; sgn = -1: g decreases from +inf
+        auto g = [&](double sigma) -> double {
+            double f = 1.0;
+            const double t = sgn * sigma;
+            for (int i = 0; i < K; ++i) f += rho * zk[i] * zk[i] / ((dk[i] - dorg) - t);
+            return f;
+        };
+        // want the sigma where sgn * g changes from negative to positive
+        double lo = 0.0;
+        int it = 0;
+        while (it < 1100) {                       // find the binade of the root
+            const double mid = 0.5 * hi;
+            if (!(mid > 0.0)) break;
+            if (sgn * g(mid) > 0.0) hi = mid; else { lo = mid; break; }
+            ++it;
+        }
+        for (int b = 0; b < 64 && lo > 0.0; ++b) {
+            const double mid = 0.5 * (lo + hi);
+            if (!(mid > lo && mid < hi)) break;
+            if (sgn * g(mid) > 0.0) hi = mid; else lo = mid;
+        }
+        org[j] = o;
+        tk[j] = sgn * 0.5 * (lo + hi);
+    }
+    __syncthreads();
+    // z recomputed from the roots: zh_i^2 = prod_j (lambda_j - d_i) / (rho prod_{j != i} (d_j - d_i))
+    for (int i = tid; i < K; i += nt) {
+        double pr = ((dk[org[i]] - dk[i]) + tk[i]) / rho;
+        for (int j = 0; j < K; ++j) {
+            if (j == i) continue;
+            pr *= ((dk[org[j]] - dk[i]) + tk[j]) / (dk[j] - dk[i]);
+        }
+        const double mag = sqrt(fabs(pr));
+        zh[i] = (zk[i] < 0.0) ? -mag : mag;
+    }
+    __syncthreads();
+    // eigenvectors: column j = zh_i / (d_i - lambda_j), normalised; eigenvalues
+    double *__restrict__ Uh = D.Xw;
+    for (int j = tid; j < K; j += nt) {
+        const double dorg = dk[org[j]], tj = tk[j];
+        double nrm2 = 0.0;
+        for (int i = 0; i < K; ++i) { const double v = zh[i] / ((dk[i] - dorg) - tj); nrm2 += v * v; }
+        const double inv = rsqrt(nrm2);
+        for (int i = 0; i < K; ++i) Uh[(int64_t)i * n + j] = zh[i] / ((dk[i] - dorg) - tj) * inv;
+        D.dvec[D.dc_nd[j]] = flip * (dorg + tj);
+    }
+}
+
+template <int R>
+__global__ void __launch_bounds__(SYS_WARPS * 32)
+eig_rot_systolic_kernel(const RefreshDev *__restrict__ rd, const RowItem *__restrict__ items, int dc)
+{
+    extern __shared__ double zs[];                // [SYS_WARPS][R][k]
+    const RowItem it = items[blockIdx.x];
+    const RefreshDev D = rd[it.block];
+    const int k = D.k, r = D.r;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int row0 = it.row0 + warp * R;
+    if (row0 >= k) return;                        // warps never synchronise with one another
+    double *z = zs + (size_t)warp * R * k;
+#pragma unroll
+    for (int q = 0; q < R; ++q) {
+        const int row = min(row0 + q, k - 1);     // rows past the end shadow the last row, never stored
+        for (int c = lane; c < k; c += 32) z[q * k + c] = D.Wj[(int64_t)row * k + c];
+    }
+    __syncwarp();
+    if (!dc) {
+        systolic_apply<R>(z, k, k, D.rot, D.groups, D.sweeps, D.nsweeps[0], lane);
+    } else {
+        // rows of Q diag(Z1, Z2): each half of the columns through its own log
+        const int s = k / 2;
+        systolic_apply<R>(z, k, s, D.rot, D.groups, D.sweeps, D.nsweeps[0], lane);
+        systolic_apply<R>(z + s, k, k - s, D.rot + dc_rot_off(D), D.groups + dc_group_off(D), D.sweeps + dc_sweep_off(D),
+                          D.nsweeps[1], lane);
+        // deflation rotations (few), one row per lane
+        const int nr = D.dc_info[1];
+        if (lane < R) {
+            double *zr = z + lane * k;
+            for (int t = 0; t < nr; ++t) {
+                const int2 ab = D.dc_rot_idx[t];
+                const double2 cs = D.dc_rot_cs[t];
+                const double xa = zr[ab.x], xb = zr[ab.y];
+                zr[ab.x] = cs.x * xa + cs.y * xb;
+                zr[ab.y] = cs.x * xb - cs.y * xa;
+            }
+        }
+        __syncwarp();
+        // the coordinates of the secular problem: y = x[nd] Uhat, written back over x[nd]
+        const int K = D.dc_info[0];
+        const double *__restrict__ Uh = D.Xw;
+        const int32_t *__restrict__ nd = D.dc_nd;
+        constexpr int NCH = 17;                   // 32-column chunks per pass (544 columns)
+        for (int c0 = 0; c0 < K; c0 += 32 * NCH) {
+            double acc[R][NCH];
+#pragma unroll
+            for (int q = 0; q < R; ++q)
+#pragma unroll
+                for (int u = 0; u < NCH; ++u) acc[q][u] = 0.0;
+            for (int i = 0; i < K; ++i) {
+                const int ci = nd[i];
+                double xv[R];
+#pragma unroll
+                for (int q = 0; q < R; ++q) xv[q] = z[q * k + ci];
+                const double *urow = Uh + (int64_t)i * k + c0 + lane;
+#pragma unroll
+                for (int u = 0; u < NCH; ++u) {
+                    const double uv = (c0 + lane + 32 * u < K) ? urow[32 * u] : 0.0;
+#pragma unroll
+                    for (int q = 0; q < R; ++q) acc[q][u] += xv[q] * uv;
+                }
+            }
+            // results of this pass go to a side buffer first when a second pass still needs the inputs
+            __syncwarp();
+            if (K <= 32 * NCH) {
+#pragma unroll
+                for (int u = 0; u < NCH; ++u) {
+                    const int j = c0 + lane + 32 * u;
+                    if (j < K) {
+                        const int cj = nd[j];
+#pragma unroll
+                        for (int q = 0; q < R; ++q) z[q * k + cj] = acc[q][u];
+                    }
+                }
+            } else {
+                // wide problems: park the results in the (now unused) rows of Wj and copy back at the end
+#pragma unroll
+                for (int u = 0; u < NCH; ++u) {
+                    const int j = c0 + lane + 32 * u;
+                    if (j < K) {
+#pragma unroll
+                        for (int q = 0; q < R; ++q)
+                            if (row0 + q < k) D.Wj[(int64_t)(row0 + q) * k + j] = acc[q][u];
+                    }
+                }
+            }
+        }
+        __syncwarp();
+        if (K > 32 * NCH) {
+            for (int j = lane; j < K; j += 32) {
+                const int cj = nd[j];
+#pragma unroll
+                for (int q = 0; q < R; ++q)
+                    if (row0 + q < k) z[q * k + cj] = D.Wj[(int64_t)(row0 + q) * k + j];
             }
         }
         __syncwarp();
@@ -524,7 +811,7 @@ cudaError_t eig_tridiag_batched(const RefreshDev *rd, const int32_t *list, int n
     if (nlist <= 0) return cudaSuccess;
     const int kpad = kmax + 8;
     const size_t tr_bytes = (size_t)(2 + 2 * TR_NB) * kpad * sizeof(double);
-    static size_t tr_cfg = 0, sys4_cfg = 0, sys2_cfg = 0;
+    static size_t tr_cfg = 0, sys4_cfg = 0, sys2_cfg = 0, sec_cfg = 0;
     cudaError_t e;
     if ((e = raise_smem(tridiag_kernel, tr_bytes, &tr_cfg)) != cudaSuccess) return e;
     tridiag_kernel<<<nlist, TR_THREADS, tr_bytes, stream>>>(rd, list, kpad);
@@ -534,16 +821,23 @@ cudaError_t eig_tridiag_batched(const RefreshDev *rd, const int32_t *list, int n
         if (kmax <= 288) eig_qrows_kernel<9, 2, QR_WARPS><<<nqrows, QR_WARPS * 32, 0, stream>>>(rd, qrows_items);
         else if (kmax <= 544) eig_qrows_kernel<17, 2, QR_WARPS><<<nqrows, QR_WARPS * 32, 0, stream>>>(rd, qrows_items);
         else eig_qrows_kernel<33, 1, QR_WARPS><<<nqrows, QR_WARPS * 32, 0, stream>>>(rd, qrows_items);
-        ql_log_kernel<<<nlist, 32, ql_bytes, stream>>>(rd, list);
+        const int dc = kmax >= DC_MIN_K ? 1 : 0;
+        ql_log_kernel<<<nlist, 64, ql_bytes, stream>>>(rd, list, dc);
+        if (dc) {
+            dc_zrows_kernel<<<nlist, 64, (size_t)kmax * sizeof(double), stream>>>(rd, list);
+            const size_t sec_bytes = (size_t)kpad * (6 * sizeof(double) + 3 * sizeof(int));
+            if ((e = raise_smem(dc_secular_kernel, sec_bytes, &sec_cfg)) != cudaSuccess) return e;
+            dc_secular_kernel<<<nlist, DC_THREADS, sec_bytes, stream>>>(rd, list, kpad);
+        }
         eig_rank_kernel<<<nlist, 256, 0, stream>>>(rd, list);
         const int R = sys_rows_per_warp(kmax);
         const size_t sys_bytes = (size_t)SYS_WARPS * R * kmax * sizeof(double);
         if (R == 4) {
             if ((e = raise_smem(eig_rot_systolic_kernel<4>, sys_bytes, &sys4_cfg)) != cudaSuccess) return e;
-            eig_rot_systolic_kernel<4><<<npanels, threads, sys_bytes, stream>>>(rd, panel_items);
+            eig_rot_systolic_kernel<4><<<npanels, threads, sys_bytes, stream>>>(rd, panel_items, dc);
         } else {
             if ((e = raise_smem(eig_rot_systolic_kernel<2>, sys_bytes, &sys2_cfg)) != cudaSuccess) return e;
-            eig_rot_systolic_kernel<2><<<npanels, threads, sys_bytes, stream>>>(rd, panel_items);
+            eig_rot_systolic_kernel<2><<<npanels, threads, sys_bytes, stream>>>(rd, panel_items, dc);
         }
         return cudaGetLastError();
     }

@@ -140,6 +140,13 @@ struct RefreshDev {
     int32_t *nsweeps;            // number of logged sweeps
     int32_t *rank;               // k: descending rank of each eigenvalue
     int32_t rot_cap, sweep_cap;
+    // divide-and-conquer merge of the two halves of the tridiagonal problem (tsr_eig.cu)
+    double *dc_z;                // k: the rank-one vector in the basis of the halves' eigenvectors
+    int32_t *dc_nd;              // coordinates that take part in the secular problem, ascending eigenvalue
+    int2 *dc_rot_idx;            // deflation rotations: coordinate pair
+    double2 *dc_rot_cs;          //                      (c, s)
+    double *dc_scal;             // [0] rho
+    int32_t *dc_info;            // [0] K (size of the secular problem), [1] number of deflation rotations
 };
 struct RowItem { int32_t block; int32_t row0; };   // a slab of rows of one block
 
