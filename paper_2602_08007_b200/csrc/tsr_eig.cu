@@ -522,7 +522,7 @@ dc_zrows_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ l
 // orthogonal to working precision however close the roots are), and write the eigenvector matrix
 // Uhat (K x K, row pitch k, in Xw), the coordinate list nd, the deflation rotations and the
 // eigenvalues of all k coordinates (dvec).
-constexpr int DC_THREADS = 512;
+constexpr int DC_THREADS = 1024;
 
 __global__ void __launch_bounds__(DC_THREADS)
 dc_secular_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ list, int kpad)
@@ -614,29 +614,42 @@ dc_secular_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__
             hi = 0.5 * gap;
         }
         const double dorg = dk[o];
-        // g(sigma) = f(dorg + sgn sigma); sgn = +1: g increases from -inf; sgn = -1: g decreases from +inf
-        auto g = [&](double sigma) -> double {
-            double f = 1.0;
+        // h(sigma) = sgn f(dorg + sgn sigma) increases from -inf at sigma = 0+ to h(hi) >= 0; its derivative
+        // is rho sum_i z_i^2 / (d_i - lambda)^2 > 0.  Both come out of one pass over the poles.
+        auto h = [&](double sigma, double &dh) -> double {
+            double f = 1.0, df = 0.0;
             const double t = sgn * sigma;
-            for (int i = 0; i < K; ++i) f += rho * zk[i] * zk[i] / ((dk[i] - dorg) - t);
-            return f;
+            for (int i = 0; i < K; ++i) {
+                const double inv = 1.0 / ((dk[i] - dorg) - t);
+                const double w = rho * zk[i] * zk[i] * inv;
+                f += w;
+                df += w * inv;
+            }
+            dh = df;
+            return sgn * f;
         };
-        // want the sigma where sgn * g changes from negative to positive
-        double lo = 0.0;
-        int it = 0;
-        while (it < 1100) {                       // find the binade of the root
+        // 1. the binade of the root: halve hi while h(hi / 2) > 0
+        double lo = 0.0, dh = 0.0;
+        for (int it = 0; it < 1100; ++it) {
             const double mid = 0.5 * hi;
             if (!(mid > 0.0)) break;
-            if (sgn * g(mid) > 0.0) hi = mid; else { lo = mid; break; }
-            ++it;
+            if (h(mid, dh) > 0.0) hi = mid; else { lo = mid; break; }
         }
-        for (int b = 0; b < 64 && lo > 0.0; ++b) {
-            const double mid = 0.5 * (lo + hi);
-            if (!(mid > lo && mid < hi)) break;
-            if (sgn * g(mid) > 0.0) hi = mid; else lo = mid;
+        // 2. Newton's iteration kept inside the bracket [lo, hi] (a step that leaves it is replaced by
+        //    bisection); the bracket shrinks at every step, so the loop ends by itself
+        double x = 0.5 * (lo + hi);
+        for (int it = 0; it < 80 && lo > 0.0; ++it) {
+            const double hx = h(x, dh);
+            if (hx > 0.0) hi = x; else lo = x;
+            double xn = x - hx / dh;
+            if (!(xn > lo && xn < hi)) xn = 0.5 * (lo + hi);
+            if (!(xn > lo && xn < hi)) break;            // the bracket is two neighbouring numbers
+            if (fabs(xn - x) <= 4.0e-16 * xn) { x = xn; break; }
+            x = xn;
         }
+        if (!(lo > 0.0)) x = 0.5 * (lo + hi);
         org[j] = o;
-        tk[j] = sgn * 0.5 * (lo + hi);
+        tk[j] = sgn * x;
     }
     __syncthreads();
     // z recomputed from the roots: zh_i^2 = prod_j (lambda_j - d_i) / (rho prod_{j != i} (d_j - d_i))
