@@ -1,16 +1,20 @@
 // Symmetric eigen-decomposition of the k x k Gram matrix S = B B^T of the refresh (Section 3.5:
 // "compute a small SVD") for ranks too large for a shared-memory Jacobi solver.
 //
-// Classical three-stage scheme, batched over blocks, FP64 throughout:
+// Batched over blocks, FP64 throughout:
 //   1. Householder reduction to tridiagonal form T = Q^T S Q (one CTA per matrix; the
 //      reflectors are kept in the rows of S above the first superdiagonal);
-//   2. implicit-shift QL iteration on (d, e) alone, one thread per matrix, which LOGS every
-//      plane rotation instead of applying it;
-//   3. the eigenvectors W = Q Z, row slab by row slab (rows are independent under
+//   2. divide and conquer on T: it is torn in the middle, T = diag(T1', T2') + rho u u^T, and each
+//      half runs an implicit-shift QL iteration on (d, e) alone, one thread per half, which LOGS
+//      every plane rotation instead of applying it;
+//   3. the merge: eigen-decomposition of D + rho z z^T (D = eigenvalues of the halves, z = Z^T u)
+//      through the secular equation, one root per thread;
+//   4. the eigenvectors W = Q diag(Z1, Z2) G Uhat, row slab by row slab (rows are independent under
 //      right-multiplication): a first kernel forms the rows of Q from the reflectors with the
-//      rows held in registers; a second one streams every row through the logged rotations as
-//      a systolic pipeline over the lanes of a warp (32 sweeps advance per step) and writes the
-//      leading r columns in descending eigenvalue order: Wu = W[:, :r], Wv = W[:, :r] / sqrt(lambda).
+//      rows held in registers; a second one streams every row through the two rotation logs as
+//      a systolic pipeline over the lanes of a warp (32 sweeps advance per step), then through
+//      the deflation rotations G and the merged eigenvector matrix Uhat, and writes the leading r
+//      columns in descending eigenvalue order: Wu = W[:, :r], Wv = W[:, :r] / sqrt(lambda).
 // Failure to converge within the iteration or log budget flags TSR_ERR_NOT_CONVERGED.
 #include "tsr_internal.h"
 
