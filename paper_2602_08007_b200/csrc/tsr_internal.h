@@ -151,7 +151,7 @@ struct RefreshDev {
 struct RowItem { int32_t block; int32_t row0; };   // a slab of rows of one block
 
 constexpr int GRAM_ROWS = 2048;   // rows per Gram work item
-constexpr int RG_ROWS = 64;       // rows per rows_gemm work item
+constexpr int RG_ROWS = 128;      // rows per rows_gemm work item
 __host__ __device__ inline int gram_chunks(int64_t rows) { return (int)((rows + GRAM_ROWS - 1) / GRAM_ROWS); }
 
 // side: 0 = matrices with m rows, 1 = matrices with n rows.

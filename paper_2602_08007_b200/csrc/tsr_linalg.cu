@@ -388,7 +388,8 @@ cudaError_t chol_inverse_batched(const RefreshDev *rd, const int32_t *list, int 
 }
 
 // ---------------------------------------------------------------------------------------
-// dst[rows x N] = src[rows x k] * Mat[k x N]   (FP32, 64 x 64 tiles, one slab of 64 rows per item)
+// dst[rows x N] = src[rows x k] * Mat[k x N]   (FP32; 128 x 64 tiles, one slab of RG_ROWS = 128 rows
+// per item, 8 x 4 outputs per thread)
 // ---------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)
 rows_gemm_kernel(const RefreshDev *__restrict__ rd, const RowItem *__restrict__ items, int side, int src_sel,
@@ -406,23 +407,27 @@ rows_gemm_kernel(const RefreshDev *__restrict__ rd, const RowItem *__restrict__ 
     float *__restrict__ D = (dst_sel < 3) ? d.buf[dst_sel] : (dst_sel == 3 ? d.U : d.V);
     const int m0 = it.row0;
 
-    __shared__ __align__(16) float As[16][64 + 4];
+    __shared__ __align__(16) float As[16][RG_ROWS + 4];
     __shared__ __align__(16) float Bs[16][64 + 4];
     const int tid = threadIdx.x, tx = tid % 16, ty = tid / 16;
-    float acc[4][4];
+    float acc[8][4];
 #pragma unroll
-    for (int a = 0; a < 4; ++a)
+    for (int a = 0; a < 8; ++a)
 #pragma unroll
         for (int b = 0; b < 4; ++b) acc[a][b] = 0.f;
     // global -> registers -> shared, with the next K slice in flight while the current one is used
-    float ra[4], rb[4];
+    float ra[8], rb[4];
     auto fetch = [&](int k0) {
 #pragma unroll
-        for (int l = 0; l < 4; ++l) {
+        for (int l = 0; l < 8; ++l) {
             const int e = tid + l * 256;
             const int ak = e % 16, ai = e / 16;
             const int gi = m0 + ai, gk = k0 + ak;
             ra[l] = (gi < rows && gk < K) ? A[(int64_t)gi * K + gk] : 0.f;
+        }
+#pragma unroll
+        for (int l = 0; l < 4; ++l) {
+            const int e = tid + l * 256;
             const int bj = e % 64, bk = e / 64;
             const int gj = n0 + bj, gk2 = k0 + bk;
             rb[l] = (gj < N && gk2 < K) ? B[(int64_t)gk2 * N + gj] : 0.f;
@@ -433,29 +438,34 @@ rows_gemm_kernel(const RefreshDev *__restrict__ rd, const RowItem *__restrict__ 
     fetch(0);
     for (int k0 = 0; k0 < Kend; k0 += 16) {
 #pragma unroll
-        for (int l = 0; l < 4; ++l) {
+        for (int l = 0; l < 8; ++l) {
             const int e = tid + l * 256;
             As[e % 16][e / 16] = ra[l];
+        }
+#pragma unroll
+        for (int l = 0; l < 4; ++l) {
+            const int e = tid + l * 256;
             Bs[e / 64][e % 64] = rb[l];
         }
         __syncthreads();
         if (k0 + 16 < Kend) fetch(k0 + 16);
 #pragma unroll
         for (int kk = 0; kk < 16; ++kk) {
-            const float4 af = *(const float4 *)&As[kk][ty * 4];
+            const float4 a0 = *(const float4 *)&As[kk][ty * 8];
+            const float4 a1 = *(const float4 *)&As[kk][ty * 8 + 4];
             const float4 bf = *(const float4 *)&Bs[kk][tx * 4];
-            const float av[4] = {af.x, af.y, af.z, af.w};
+            const float av[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
             const float bv[4] = {bf.x, bf.y, bf.z, bf.w};
 #pragma unroll
-            for (int a = 0; a < 4; ++a)
+            for (int a = 0; a < 8; ++a)
 #pragma unroll
                 for (int b = 0; b < 4; ++b) acc[a][b] = fmaf(av[a], bv[b], acc[a][b]);
         }
         __syncthreads();
     }
 #pragma unroll
-    for (int a = 0; a < 4; ++a) {
-        const int gi = m0 + ty * 4 + a;
+    for (int a = 0; a < 8; ++a) {
+        const int gi = m0 + ty * 8 + a;
         if (gi >= rows) continue;
 #pragma unroll
         for (int b = 0; b < 4; ++b) {
