@@ -202,12 +202,21 @@ cudaError_t core_update_launch(const CoreUpdateArgs *args_dev, const int32_t *li
 // ---------------------------------------------------------------------------------------
 // Operand conversion
 // ---------------------------------------------------------------------------------------
+// The transposing kernels below work on tiles of 64 rows x 32 columns: in the transposed copy a lane
+// writes two consecutive rows as one 32-bit word, so a warp stores 128 contiguous bytes.  The row
+// pitches of the transposed copies are multiples of 8 elements, which keeps those words aligned.
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
+{
+    const __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+    return *(const uint32_t *)&h;
+}
+
 __global__ void shadows_kernel(const float *__restrict__ X, int rows, int r, bf16 *__restrict__ Xb, int64_t ldb,
                                bf16 *__restrict__ Xbt, int64_t ldt)
 {
-    __shared__ float tile[32][33];
-    const int r0 = blockIdx.y * 32, c0 = blockIdx.x * 32;
-    for (int i = threadIdx.y; i < 32; i += blockDim.y) {
+    __shared__ float tile[64][33];
+    const int r0 = blockIdx.y * 64, c0 = blockIdx.x * 32;
+    for (int i = threadIdx.y; i < 64; i += blockDim.y) {
         const int row = r0 + i, col = c0 + threadIdx.x;
         float v = 0.f;
         if (row < rows && col < r) {
@@ -219,8 +228,11 @@ __global__ void shadows_kernel(const float *__restrict__ X, int rows, int r, bf1
     __syncthreads();
     if (Xbt) {
         for (int i = threadIdx.y; i < 32; i += blockDim.y) {
-            const int col = c0 + i, row = r0 + threadIdx.x;
-            if (row < rows && col < r) Xbt[(int64_t)col * ldt + row] = __float2bfloat16_rn(tile[threadIdx.x][i]);
+            const int col = c0 + i, row = r0 + 2 * threadIdx.x;
+            if (col >= r || row >= rows) continue;
+            bf16 *dst = Xbt + (int64_t)col * ldt + row;
+            if (row + 1 < rows) *(uint32_t *)dst = pack_bf16x2(tile[2 * threadIdx.x][i], tile[2 * threadIdx.x + 1][i]);
+            else *dst = __float2bfloat16_rn(tile[2 * threadIdx.x][i]);
         }
     }
 }
@@ -228,33 +240,47 @@ __global__ void shadows_kernel(const float *__restrict__ X, int rows, int r, bf1
 cudaError_t make_shadows(const float *X, int rows, int r, bf16 *Xb, int64_t ldb, bf16 *Xbt, int64_t ldt,
                          cudaStream_t stream)
 {
-    dim3 grid((r + 31) / 32, (rows + 31) / 32);
+    dim3 grid((r + 31) / 32, (rows + 63) / 64);
     shadows_kernel<<<grid, dim3(32, 8), 0, stream>>>(X, rows, r, Xb, ldb, Xbt, ldt);
     return cudaGetLastError();
 }
 
+// out[cols x ldo] = in[rows x ldi]^T.  Tiles of 64 x 64, read and written as pairs of BF16.
 __global__ void transpose_bf16_kernel(const bf16 *__restrict__ in, int rows, int cols, int64_t ldi,
-                                      bf16 *__restrict__ out, int64_t ldo)
+                                      bf16 *__restrict__ out, int64_t ldo, int in_pairs)
 {
     __shared__ bf16 tile[64][66];
     const int r0 = blockIdx.y * 64, c0 = blockIdx.x * 64;
-    for (int i = threadIdx.y; i < 64; i += blockDim.y)
-        for (int j = threadIdx.x; j < 64; j += blockDim.x) {
-            const int row = r0 + i, col = c0 + j;
-            tile[i][j] = (row < rows && col < cols) ? in[(int64_t)row * ldi + col] : __float2bfloat16_rn(0.f);
+    for (int i = threadIdx.y; i < 64; i += blockDim.y) {
+        const int row = r0 + i, col = c0 + 2 * threadIdx.x;
+        uint32_t w = 0;
+        if (row < rows && col < cols) {
+            const bf16 *src = in + (int64_t)row * ldi + col;
+            if (in_pairs && col + 1 < cols) w = *(const uint32_t *)src;
+            else {
+                const bf16 a = src[0], bq = (col + 1 < cols) ? src[1] : __float2bfloat16_rn(0.f);
+                w = (uint32_t)(*(const uint16_t *)&a) | ((uint32_t)(*(const uint16_t *)&bq) << 16);
+            }
         }
+        *(uint32_t *)&tile[i][2 * threadIdx.x] = w;
+    }
     __syncthreads();
-    for (int i = threadIdx.y; i < 64; i += blockDim.y)
-        for (int j = threadIdx.x; j < 64; j += blockDim.x) {
-            const int col = c0 + i, row = r0 + j;
-            if (row < rows && col < cols) out[(int64_t)col * ldo + row] = tile[j][i];
-        }
+    for (int i = threadIdx.y; i < 64; i += blockDim.y) {
+        const int col = c0 + i, row = r0 + 2 * threadIdx.x;
+        if (col >= cols || row >= rows) continue;
+        bf16 *dst = out + (int64_t)col * ldo + row;
+        const bf16 a = tile[2 * threadIdx.x][i], bq = tile[2 * threadIdx.x + 1][i];
+        if (row + 1 < rows) *(uint32_t *)dst = (uint32_t)(*(const uint16_t *)&a) | ((uint32_t)(*(const uint16_t *)&bq) << 16);
+        else *dst = a;
+    }
 }
 
 cudaError_t transpose_bf16(const bf16 *in, int rows, int cols, int64_t ldi, bf16 *out, int64_t ldo, cudaStream_t stream)
 {
     dim3 grid((cols + 63) / 64, (rows + 63) / 64);
-    transpose_bf16_kernel<<<grid, dim3(32, 8), 0, stream>>>(in, rows, cols, ldi, out, ldo);
+    // 32-bit loads need an even row pitch and a 4-byte aligned base; the output side always has them
+    const int in_pairs = ((ldi & 1) == 0 && (((uintptr_t)in) & 3) == 0) ? 1 : 0;
+    transpose_bf16_kernel<<<grid, dim3(32, 8), 0, stream>>>(in, rows, cols, ldi, out, ldo, in_pairs);
     return cudaGetLastError();
 }
 
@@ -262,21 +288,26 @@ cudaError_t transpose_bf16(const bf16 *in, int rows, int cols, int64_t ldi, bf16
 __global__ void split_transpose_kernel(const float *__restrict__ X, int rows, int k, bf16 *__restrict__ out,
                                        int64_t ldo, int plane_rows, int planes)
 {
-    __shared__ float tile[32][33];
-    const int r0 = blockIdx.y * 32, c0 = blockIdx.x * 32;
-    for (int i = threadIdx.y; i < 32; i += blockDim.y) {
+    __shared__ float tile[64][33];
+    const int r0 = blockIdx.y * 64, c0 = blockIdx.x * 32;
+    for (int i = threadIdx.y; i < 64; i += blockDim.y) {
         const int row = r0 + i, col = c0 + threadIdx.x;
         tile[i][threadIdx.x] = (row < rows && col < k) ? X[(int64_t)row * k + col] : 0.f;
     }
     __syncthreads();
     for (int i = threadIdx.y; i < 32; i += blockDim.y) {
-        const int col = c0 + i, row = r0 + threadIdx.x;
-        if (row < rows && col < k) {
-            const float v = tile[threadIdx.x][i];
-            const bf16 hi = __float2bfloat16_rn(v);
-            out[(int64_t)col * ldo + row] = hi;
-            if (planes > 1)
-                out[((int64_t)plane_rows + col) * ldo + row] = __float2bfloat16_rn(v - __bfloat162float(hi));
+        const int col = c0 + i, row = r0 + 2 * threadIdx.x;
+        if (col >= k || row >= rows) continue;
+        const float v0 = tile[2 * threadIdx.x][i], v1 = tile[2 * threadIdx.x + 1][i];
+        const bf16 h0 = __float2bfloat16_rn(v0), h1 = __float2bfloat16_rn(v1);
+        bf16 *dhi = out + (int64_t)col * ldo + row;
+        bf16 *dlo = out + ((int64_t)plane_rows + col) * ldo + row;
+        if (row + 1 < rows) {
+            *(uint32_t *)dhi = (uint32_t)(*(const uint16_t *)&h0) | ((uint32_t)(*(const uint16_t *)&h1) << 16);
+            if (planes > 1) *(uint32_t *)dlo = pack_bf16x2(v0 - __bfloat162float(h0), v1 - __bfloat162float(h1));
+        } else {
+            *dhi = h0;
+            if (planes > 1) *dlo = __float2bfloat16_rn(v0 - __bfloat162float(h0));
         }
     }
 }
@@ -284,7 +315,7 @@ __global__ void split_transpose_kernel(const float *__restrict__ X, int rows, in
 cudaError_t split_transpose(const float *X, int rows, int k, bf16 *out, int64_t ldo, int plane_rows, int planes,
                             cudaStream_t stream)
 {
-    dim3 grid((k + 31) / 32, (rows + 31) / 32);
+    dim3 grid((k + 31) / 32, (rows + 63) / 64);
     split_transpose_kernel<<<grid, dim3(32, 8), 0, stream>>>(X, rows, k, out, ldo, plane_rows, planes);
     return cudaGetLastError();
 }
