@@ -37,6 +37,40 @@ def test_refresh_small_and_extreme_shapes(dtype, shape, gap):
     check_refresh(plan, 0, G64, to64(Om), shape["r"], shape["q"], gap, tol_sub=tol_sub)
 
 
+def test_refresh_with_repeated_singular_values():
+    """Groups of equal singular values and a flat tail: the Gram matrix of the sketch has repeated
+    eigenvalues, which the divide-and-conquer eigen-solver must deflate (rotations between nearly
+    equal poles, negligible components of the rank-one vector).  Any orthonormal basis of an
+    eigenspace is correct, so the check is on orthonormality, the diagonal core, the singular values
+    and the projector at the boundary between distinct groups."""
+    tsr = _tsr()
+    shape = dict(m=320, n=288, r=250, p=6, q=1)
+    rng = np.random.default_rng(11)
+    A, _ = np.linalg.qr(rng.standard_normal((shape["m"], 64)))
+    B, _ = np.linalg.qr(rng.standard_normal((shape["n"], 64)))
+    sig = np.array([10.0] * 4 + [7.0] * 4 + [5.0] * 8 + [1e-2] * 48)
+    G = torch.from_numpy((A * sig) @ B.T).float()
+    plan = tsr.Plan([shape], g_dtype=torch.float32)
+    plan.G[0].copy_(G.cuda())
+    Om = ti.omega(shape["n"], shape["r"] + shape["p"], 77).cuda()
+    plan.init_subspace(omegas=[Om])
+    torch.cuda.synchronize()
+    # the gradient has rank 64 < k: the sketch is rank deficient by construction and is flagged as such
+    assert plan.poll_status()[0] in (0, 8)
+    U, V = to64(plan.U[0]), to64(plan.V[0])
+    G64 = to64(G)
+    core = U.T @ G64 @ V
+    d = np.diag(core)
+    assert np.abs(core - np.diag(d)).max() < 2e-3 * sig[0]
+    assert np.abs(d[:16] / sig[:16] - 1).max() < 1e-4
+    for cols in (4, 8, 16):                       # boundaries between the groups of equal values
+        assert np.linalg.norm(proj(U[:, :cols]) - proj(A[:, :cols])) < 1e-3
+        assert np.linalg.norm(proj(V[:, :cols]) - proj(B[:, :cols])) < 1e-3
+    lead = 64                                     # directions that carry any signal stay orthonormal
+    assert np.linalg.norm(U[:, :lead].T @ U[:, :lead] - np.eye(lead)) < 1e-4
+    assert np.linalg.norm(V[:, :lead].T @ V[:, :lead] - np.eye(lead)) < 1e-4
+
+
 def test_tiny_step_matches_oracle():
     tsr = _tsr()
     shapes = [dict(m=9, n=7, r=3), dict(m=33, n=65, r=8)]
