@@ -45,9 +45,10 @@ def measured_peaks():
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
 
 
-def step_work(w: ti.Workload):
-    """Algorithmic flops and bytes of one non-refresh step, per stage."""
+def step_work(w: ti.Workload, w_bytes: int = 4):
+    """Algorithmic flops and bytes of one non-refresh step, per stage (w_bytes: bytes per weight)."""
     ges = 2 if w.g_dtype == "bf16" else 4
+    rmw = 2.0 * w_bytes
     out = {"proj_flops": 0.0, "proj_bytes": 0.0, "apply_flops": 0.0, "apply_bytes": 0.0,
            "apply_kernel_flops": 0.0, "apply_kernel_bytes": 0.0}
     for b in w.blocks:
@@ -56,10 +57,10 @@ def step_work(w: ti.Workload):
         out["proj_flops"] += 2.0 * m * n * r + small
         out["proj_bytes"] += ges * m * n + 2.0 * (m + n) * r + 24.0 * r * r
         out["apply_flops"] += 2.0 * m * n * r + small
-        out["apply_bytes"] += 8.0 * m * n + 2.0 * (m + n) * r
+        out["apply_bytes"] += rmw * m * n + 2.0 * (m + n) * r
         # the apply kernel proper: W <- decay W - step_scale P V^T with P = U D (m x r) given
         out["apply_kernel_flops"] += 2.0 * m * n * r
-        out["apply_kernel_bytes"] += 8.0 * m * n + 2.0 * (m + n) * r
+        out["apply_kernel_bytes"] += rmw * m * n + 2.0 * (m + n) * r
     out["step_flops"] = out["proj_flops"] + out["apply_flops"]
     out["step_bytes"] = out["proj_bytes"] + out["apply_bytes"]
     return out
@@ -250,13 +251,13 @@ def apply_traffic_ratio(config_id: int) -> float:
     return APPLY_TRAFFIC_RATIO.get(config_id, 0.98)
 
 
-def build_plan(w: ti.Workload, device):
+def build_plan(w: ti.Workload, device, bf16_weights: bool = False):
     import paper_2602_08007_b200 as tsr
     dt = torch.bfloat16 if w.g_dtype == "bf16" else torch.float32
-    plan = tsr.Plan(list(w.blocks), g_dtype=dt, device=device)
+    plan = tsr.Plan(list(w.blocks), g_dtype=dt, device=device, w_dtype=torch.bfloat16 if bf16_weights else torch.float32)
     for i, b in enumerate(w.blocks):
         plan.G[i].copy_(ti.gradient(b.m, b.n, ti.seed_for(w.config_id, i, 0, ti.ROLE_INIT_GRAD), dtype=dt, device=device))
-        plan.W[i].copy_(ti.weights(b.m, b.n, ti.seed_for(w.config_id, i, 0, ti.ROLE_WEIGHT), device=device))
+        plan.W[i].copy_(ti.weights(b.m, b.n, ti.seed_for(w.config_id, i, 0, ti.ROLE_WEIGHT), device=device).to(plan.W[i].dtype))
     return tsr, plan
 
 
@@ -280,9 +281,9 @@ def run_ours(args, w: ti.Workload):
         dist_mod.init_process_group("nccl", device_id=device)
         dist = dist_mod
 
-    tsr, plan = build_plan(w, device)
+    tsr, plan = build_plan(w, device, args.bf16_weights)
     peaks = measured_peaks()
-    work = step_work(w)
+    work = step_work(w, 2 if args.bf16_weights else 4)
     nb = len(w.blocks)
     seed = ti.BASE_SEED
 
@@ -431,7 +432,8 @@ def run_ours(args, w: ti.Workload):
                        "refresh_interval": w.blocks[0].K, "refresh_steps_in_timed_region": len(refresh_steps),
                        "l2": "flushed between steps" if flush is not None else "inputs (G %.2f GB + W %.2f GB) exceed L2"
                        % (sum(b.m * b.n for b in w.blocks) * (2 if w.g_dtype == "bf16" else 4) / 1e9,
-                          sum(b.m * b.n for b in w.blocks) * 4 / 1e9),
+                          sum(b.m * b.n for b in w.blocks) * (2 if args.bf16_weights else 4) / 1e9),
+                       "weights": "bf16" if args.bf16_weights else "f32",
                        "parallelism": "replicas only" if world > 1 else "single gpu"},
             "step_ms_no_refresh": plain_ms,
             "wall_ms_per_step": wall_ms_per_step,
@@ -441,7 +443,7 @@ def run_ours(args, w: ti.Workload):
                          "gemm_UD": st_med[4], "apply": st_med[5]},
             "roofline": {"kernel": "umma_apply_kernel (W <- decay W - lr P V^T)", "bound": "hbm",
                          "achieved": apply_gbs, "peak": hbm, "unit": "GB/s", "frac": apply_gbs / hbm,
-                         "traffic": apply_traffic_ratio(w.config_id) * work["apply_kernel_bytes"],
+                         "traffic": None if args.bf16_weights else apply_traffic_ratio(w.config_id) * work["apply_kernel_bytes"],
                          "algorithmic_bytes": work["apply_kernel_bytes"],
                          "peak_source": peaks["source"] + " copy bandwidth", "ms": apply_ms, "roof_ms": apply_roof_ms},
             "roofline_projection": {"kernels": "umma_gemm_kernel<EPI_STORE_BF16_T> + <EPI_CORE_UPDATE>",
@@ -479,6 +481,8 @@ def main():
                     help="size of the dense-AdamW micro-measurement (0 = skip)")
     ap.add_argument("--layers", type=int, default=0, help="profiling aid: truncate the model to this many layers")
     ap.add_argument("--unfused", action="store_true", help="diagnostic: run the core update as its own launch")
+    ap.add_argument("--bf16-weights", action="store_true",
+                    help="variant: weights stored in BF16 (4 instead of 8 bytes of read-modify-write per weight)")
     ap.add_argument("--random-bases", action="store_true",
                     help="profiling aid: random bases instead of the initial refresh (numbers not for reporting)")
     args = ap.parse_args()

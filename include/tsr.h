@@ -96,7 +96,8 @@ typedef struct {
     int32_t q;            /* power iterations in the refresh (>= 0)                     */
     int32_t K;            /* refresh when step % K == 0; K <= 0 disables in-loop refresh */
     int32_t g_dtype;      /* tsr_dtype of G                                             */
-    int32_t w_dtype;      /* tsr_dtype of W; only TSR_F32 is implemented                */
+    int32_t w_dtype;      /* tsr_dtype of W: TSR_F32, or TSR_BF16 (updated in FP32, rounded   */
+                          /* to nearest even); the same for every block of a context        */
     int32_t is_embedding; /* 0 / 1                                                      */
     int32_t flags;        /* bit set of tsr_block_flags; 0 = Algorithm 1 as printed     */
 } tsr_mat_desc;

@@ -181,15 +181,17 @@ class Plan:
     """Owns a tsr_ctx plus the torch tensors it is bound to.
 
     blocks: sequence of dicts/objects with m, n, r, p, q, K (and optionally is_embedding).
-    g_dtype: torch.float32 or torch.bfloat16.  Leading dimensions are padded to 16-byte row
-    pitches unless pad=False.
+    g_dtype: torch.float32 or torch.bfloat16.  w_dtype: torch.float32 (master weights) or
+    torch.bfloat16.  Leading dimensions are padded to 16-byte row pitches unless pad=False.
     """
 
     def __init__(self, blocks, g_dtype=torch.bfloat16, device="cuda", pad: bool = True, gradients=None,
-                 weights=None):
+                 weights=None, w_dtype=torch.float32):
         L = lib()
         self.device = torch.device(device)
         self.g_dtype = g_dtype
+        self.w_dtype = w_dtype
+        wes = 2 if w_dtype == torch.bfloat16 else 4
         self.blocks = list(blocks)
         nb = len(self.blocks)
         ges = 2 if g_dtype == torch.bfloat16 else 4
@@ -210,8 +212,8 @@ class Plan:
                 Wt = weights[i]
                 ldw = Wt.stride(0)
             else:
-                ldw = (n + 3) // 4 * 4 if pad else n
-                Wt = torch.zeros(m, ldw, dtype=torch.float32, device=self.device)[:, :n]
+                ldw = (n + (16 // wes) - 1) // (16 // wes) * (16 // wes) if pad else n
+                Wt = torch.zeros(m, ldw, dtype=w_dtype, device=self.device)[:, :n]
             self.G.append(G)
             self.W.append(Wt)
             self.U.append(torch.zeros(m, r, dtype=torch.float32, device=self.device))
@@ -220,7 +222,8 @@ class Plan:
             self.Vm.append(torch.zeros(r, r, dtype=torch.float32, device=self.device))
             self.C.append(torch.zeros(r, r, dtype=torch.float32, device=self.device))
             self.descs[i] = MatDesc(m, n, ldg, ldw, r, int(g("p", 0)), int(g("q", 0)), int(g("K", 0)),
-                                    TSR_BF16 if g_dtype == torch.bfloat16 else TSR_F32, TSR_F32,
+                                    TSR_BF16 if g_dtype == torch.bfloat16 else TSR_F32,
+                                    TSR_BF16 if w_dtype == torch.bfloat16 else TSR_F32,
                                     1 if g("is_embedding", False) else 0, int(g("flags", 0)))
         self.ctx = ctypes.c_void_p()
         self._check(L.tsr_create(ctypes.byref(self.ctx), self.descs, nb), create=True)

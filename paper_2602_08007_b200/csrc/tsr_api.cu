@@ -352,14 +352,17 @@ tsr_status encode_map_out_bf16(tsr_ctx *ctx, CUtensorMap *out, const void *base,
 }
 
 // FP32 row-major [rows x cols] (ld elements) -> tensor map with a 32 x 32 box, 128B swizzle.
-tsr_status encode_map_w(tsr_ctx *ctx, CUtensorMap *out, const void *base, int64_t rows, int64_t cols, int64_t ld)
+tsr_status encode_map_w(tsr_ctx *ctx, CUtensorMap *out, const void *base, int64_t rows, int64_t cols, int64_t ld,
+                        int w_dtype)
 {
+    const bool bf = (w_dtype == TSR_BF16);   // BF16 weights: 64-byte box rows, 64-byte swizzle
     cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-    cuuint64_t strides[1] = {(cuuint64_t)ld * 4};
+    cuuint64_t strides[1] = {(cuuint64_t)ld * (bf ? 2 : 4)};
     cuuint32_t box[2] = {32, 32};
     cuuint32_t estr[2] = {1, 1};
-    CUresult rc = ctx->encode(out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void *>(base), dims, strides, box, estr,
-                              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+    CUresult rc = ctx->encode(out, bf ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
+                              const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                              bf ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (rc != CUDA_SUCCESS) return fail(ctx, TSR_ERR_CUDA, "cuTensorMapEncodeTiled (W) failed (%d)", (int)rc);
     return TSR_OK;
@@ -446,7 +449,7 @@ tsr_status launch_kind(tsr_ctx *ctx, int kind, const std::vector<int> &list, int
         while (j < ranges.size() && ranges[j].first == hi) { hi = ranges[j].second; ++j; }
         if (kind == KA)
             TSR_CUDA(ctx, umma_apply_launch(ctx->d_probs[kind], ctx->d_tiles[kind] + lo, hi - lo, ctx->num_sms, ctx->bn[kind],
-                                            sc, ctx->d_status, st));
+                                            elem_size(ctx->blocks[0].d.w_dtype), sc, ctx->d_status, st));
         else
             TSR_CUDA(ctx, umma_gemm_launch(ctx->d_probs[kind], ctx->d_tiles[kind] + lo, hi - lo, ctx->num_sms, ctx->bn[kind],
                                            epilogue, planes, sc, ctx->d_status, st));
@@ -525,8 +528,8 @@ tsr_status do_apply(tsr_ctx *ctx, const std::vector<int> &list, const StepScalar
         if (b.fast) continue;
         const int m = (int)b.d.m, n = (int)b.d.n, r = b.d.r;
         TSR_KERNEL(ctx, 1, simt_gemm(m, r, r, b.p.U, TSR_F32, r, 1, b.D32, r, 1, b.P32, r, SIMT_STORE, 0, 0, st));
-        TSR_KERNEL(ctx, 1, simt_gemm(m, n, r, b.P32, TSR_F32, r, 1, b.p.V, 1, r, (float *)b.p.W, b.d.ldw, SIMT_APPLY, sc.decay,
-                                sc.step_scale, st));
+        TSR_KERNEL(ctx, 1, simt_gemm(m, n, r, b.P32, TSR_F32, r, 1, b.p.V, 1, r, (float *)b.p.W, b.d.ldw,
+                                b.d.w_dtype == TSR_BF16 ? SIMT_APPLY_BF16 : SIMT_APPLY, sc.decay, sc.step_scale, st));
     }
     return TSR_OK;
 }
@@ -858,7 +861,8 @@ tsr_status tsr_create(tsr_ctx **out, const tsr_mat_desc *descs, int32_t count)
         if ((int64_t)d.r + d.p > std::min(d.m, d.n)) return TSR_ERR_SHAPE;
         if (d.m > 0x3fffffff || d.n > 0x3fffffff || d.r + d.p > 1056) return TSR_ERR_SHAPE;
         if (d.g_dtype != TSR_F32 && d.g_dtype != TSR_BF16) return TSR_ERR_UNSUPPORTED;
-        if (d.w_dtype != TSR_F32) return TSR_ERR_UNSUPPORTED;
+        if (d.w_dtype != TSR_F32 && d.w_dtype != TSR_BF16) return TSR_ERR_UNSUPPORTED;
+        if (d.w_dtype != descs[0].w_dtype) return TSR_ERR_UNSUPPORTED;   // one weight type per context (one apply launch)
         if ((d.flags & ~(int32_t)TSR_BLOCK_REEXPRESS_MOMENT) != 0 || (d.is_embedding != 0 && d.is_embedding != 1)) return TSR_ERR_INVALID_ARG;
     }
     tsr_ctx *ctx = new (std::nothrow) tsr_ctx;
@@ -872,7 +876,7 @@ tsr_status tsr_create(tsr_ctx **out, const tsr_mat_desc *descs, int32_t count)
         b.rl = round_up(b.d.r, 8); b.ml = round_up(b.d.m, 8); b.nl = round_up(b.d.n, 8);
         // Candidate for the tensor-core path: BF16 gradient with 16-byte row pitches.  Pointer
         // alignment is checked at bind time.
-        b.fast = (b.d.g_dtype == TSR_BF16) && ((b.d.ldg * 2) % 16 == 0) && ((b.d.ldw * 4) % 16 == 0);
+        b.fast = (b.d.g_dtype == TSR_BF16) && ((b.d.ldg * 2) % 16 == 0) && ((b.d.ldw * elem_size(b.d.w_dtype)) % 16 == 0);
         b.tc_rows = b.fast && (b.k % 4 == 0);   // FP32 rows of k elements as a TMA operand: 16-byte row pitch
         const int nkb = (int)((b.d.m + 63) / 64);
         if (nkb > 128) { b.kb_per_split = 32; b.nsplit = (nkb + 31) / 32; }
@@ -925,7 +929,8 @@ tsr_status tsr_bind(tsr_ctx *ctx, const tsr_mat_ptrs *ptrs, int32_t count, void 
     for (int i = 0; i < count; ++i) {
         const tsr_mat_ptrs &p = ptrs[i];
         if (!p.G || !p.W || !p.U || !p.V || !p.M || !p.C) return fail(ctx, TSR_ERR_INVALID_ARG, "block %d: NULL pointer", i);
-        if (((uintptr_t)p.U | (uintptr_t)p.V | (uintptr_t)p.M | (uintptr_t)p.C | (uintptr_t)p.W) & 3)
+        if ((((uintptr_t)p.U | (uintptr_t)p.V | (uintptr_t)p.M | (uintptr_t)p.C) & 3) ||
+            ((uintptr_t)p.W & (uintptr_t)(elem_size(ctx->blocks[i].d.w_dtype) - 1)))
             return fail(ctx, TSR_ERR_ALIGNMENT, "block %d: FP32 buffer not 4-byte aligned", i);
     }
     int dev_count = 0;
@@ -936,7 +941,7 @@ tsr_status tsr_bind(tsr_ctx *ctx, const tsr_mat_ptrs *ptrs, int32_t count, void 
     for (int i = 0; i < count; ++i) {
         Block &b = ctx->blocks[i];
         b.p = ptrs[i];
-        const bool cand = (b.d.g_dtype == TSR_BF16) && ((b.d.ldg * 2) % 16 == 0) && ((b.d.ldw * 4) % 16 == 0);
+        const bool cand = (b.d.g_dtype == TSR_BF16) && ((b.d.ldg * 2) % 16 == 0) && ((b.d.ldw * elem_size(b.d.w_dtype)) % 16 == 0);
         const bool fast = cand && aligned16(b.p.G) && aligned16(b.p.W);
         if (fast != b.fast) { b.fast = fast; b.tc_rows = fast && (b.k % 4 == 0); layout_changed = true; }
     }
@@ -1031,7 +1036,7 @@ tsr_status tsr_bind(tsr_ctx *ctx, const tsr_mat_ptrs *ptrs, int32_t count, void 
             base(P, (int)m, (int)n, (int)r, EPI_APPLY);
             if ((s = encode_map(ctx, &P.tmA, b.Pb, m, r, b.rl, 128)) != TSR_OK) return s;
             if ((s = encode_map(ctx, &P.tmB, b.Vb, n, r, b.rl, 128)) != TSR_OK) return s;
-            if ((s = encode_map_w(ctx, &P.tmW, b.p.W, m, n, b.d.ldw)) != TSR_OK) return s;
+            if ((s = encode_map_w(ctx, &P.tmW, b.p.W, m, n, b.d.ldw, b.d.w_dtype)) != TSR_OK) return s;
             P.out = b.p.W; P.ld_out = b.d.ldw;
         }
         {   // Y = G X : A = G, B = X^T planes [2k x n]

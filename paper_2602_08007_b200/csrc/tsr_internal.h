@@ -75,13 +75,14 @@ cudaError_t umma_gemm_launch(const UmmaProblem *probs, const UmmaTile *tiles, in
 cudaError_t umma_configure();  // sets the dynamic shared-memory attributes once per process
 // Persistent apply kernel (tsr_umma_apply.cu): W <- decay W - step_scale P V^T over a tile table.
 cudaError_t umma_apply_configure();
+// w_bytes: 4 = FP32 weights, 2 = BF16 weights (the tile table must not mix them).
 cudaError_t umma_apply_launch(const UmmaProblem *probs, const UmmaTile *tiles, int num_tiles, int num_sms, int bn,
-                              const StepScalars &sc, int32_t *status, cudaStream_t stream);
+                              int w_bytes, const StepScalars &sc, int32_t *status, cudaStream_t stream);
 
 // ---------------------------------------------------------------------------------------
 // CUDA-core helpers (tsr_simt.cu)
 // ---------------------------------------------------------------------------------------
-enum SimtEpilogue : int { SIMT_STORE = 0, SIMT_APPLY = 1 };
+enum SimtEpilogue : int { SIMT_STORE = 0, SIMT_APPLY = 1, SIMT_APPLY_BF16 = 2 };   // _BF16: D holds BF16 weights
 
 // D[M x N] (ldd) = sum_k A(i,k) B(k,j),  A(i,k) = A[i*sa_i + k*sa_k],  B(k,j) = B[k*sb_k + j*sb_j].
 // a_dtype: TSR_F32 or TSR_BF16; B and D are FP32.  SIMT_APPLY: D = decay * D - step_scale * acc.

@@ -92,6 +92,11 @@ simt_gemm_kernel(int M, int N, int K, const TA *__restrict__ A, int64_t sa_i, in
         for (int b = 0; b < 4; ++b) {
             const int gj = n0 + tx * 4 + b;
             if (gj >= N) continue;
+            if (EPI == SIMT_APPLY_BF16) {   // D holds BF16 weights: update in FP32, round to nearest even
+                bf16 *dw = (bf16 *)D + (int64_t)gi * ldd + gj;
+                *dw = __float2bfloat16_rn(__fmaf_rn(-step_scale, acc[a][b], __fmul_rn(decay, __bfloat162float(*dw))));
+                continue;
+            }
             float *d = D + (int64_t)gi * ldd + gj;
             if (EPI == SIMT_APPLY) {
                 *d = __fmaf_rn(-step_scale, acc[a][b], __fmul_rn(decay, *d));
@@ -108,17 +113,19 @@ cudaError_t simt_gemm(int M, int N, int K, const void *A, int a_dtype, int64_t s
 {
     if (M <= 0 || N <= 0) return cudaSuccess;
     dim3 grid((N + SG_BN - 1) / SG_BN, (M + SG_BM - 1) / SG_BM);
+#define TSR_SG(TA_, EPI_)                                                                                              \
+    simt_gemm_kernel<TA_, EPI_><<<grid, 256, 0, stream>>>(M, N, K, (const TA_ *)A, sa_i, sa_k, B, sb_k, sb_j, D, ldd, decay, \
+                                                           step_scale)
     if (a_dtype == TSR_BF16) {
-        if (epilogue == SIMT_APPLY)
-            simt_gemm_kernel<bf16, SIMT_APPLY><<<grid, 256, 0, stream>>>(M, N, K, (const bf16 *)A, sa_i, sa_k, B, sb_k, sb_j, D, ldd, decay, step_scale);
-        else
-            simt_gemm_kernel<bf16, SIMT_STORE><<<grid, 256, 0, stream>>>(M, N, K, (const bf16 *)A, sa_i, sa_k, B, sb_k, sb_j, D, ldd, decay, step_scale);
+        if (epilogue == SIMT_APPLY) TSR_SG(bf16, SIMT_APPLY);
+        else if (epilogue == SIMT_APPLY_BF16) TSR_SG(bf16, SIMT_APPLY_BF16);
+        else TSR_SG(bf16, SIMT_STORE);
     } else {
-        if (epilogue == SIMT_APPLY)
-            simt_gemm_kernel<float, SIMT_APPLY><<<grid, 256, 0, stream>>>(M, N, K, (const float *)A, sa_i, sa_k, B, sb_k, sb_j, D, ldd, decay, step_scale);
-        else
-            simt_gemm_kernel<float, SIMT_STORE><<<grid, 256, 0, stream>>>(M, N, K, (const float *)A, sa_i, sa_k, B, sb_k, sb_j, D, ldd, decay, step_scale);
+        if (epilogue == SIMT_APPLY) TSR_SG(float, SIMT_APPLY);
+        else if (epilogue == SIMT_APPLY_BF16) TSR_SG(float, SIMT_APPLY_BF16);
+        else TSR_SG(float, SIMT_STORE);
     }
+#undef TSR_SG
     return cudaGetLastError();
 }
 

@@ -72,7 +72,7 @@ __device__ __forceinline__ void cursor_next(ChunkCursor &cur, const UmmaTile *ti
     }
 }
 
-template <int BN>
+template <int BN, int WB>
 __global__ void __launch_bounds__(AP_THREADS, 1)
 umma_apply_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restrict__ tiles, int num_tiles,
                   StepScalars sc, int32_t *__restrict__ status)
@@ -81,6 +81,7 @@ umma_apply_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restr
     constexpr int AP_STAGES = CF::STAGES, AP_STAGE_BYTES = CF::STAGE_BYTES, AP_NBOX = CF::NBOX;
     constexpr int AP_WBOX_OFFSET = CF::WBOX_OFFSET, AP_BAR_OFFSET = CF::BAR_OFFSET, AP_NBARS = CF::NBARS;
     constexpr int AP_BN = BN;
+    constexpr uint32_t W_BOX_BYTES = 32 * 32 * WB;   // FP32 weights: 4 KB boxes, 128-byte swizzle; BF16: 2 KB, 64-byte swizzle
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint64_t *bars = (uint64_t *)(smem + AP_BAR_OFFSET);
@@ -175,7 +176,7 @@ umma_apply_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restr
         for (int i = 0; i < AP_NBOX - AP_LAG && pre.tile_idx < num_tiles; ++i) {
             if (lane == 0) {
                 const uint32_t slot = issued % AP_NBOX;
-                mbar_expect_tx(smem_u32(wbar + slot), AP_BOX_BYTES);
+                mbar_expect_tx(smem_u32(wbar + slot), W_BOX_BYTES);
                 tma_load_2d(smem_u32(boxes + slot * AP_BOX_BYTES), &probs[pre.prob].tmW, smem_u32(wbar + slot),
                             pre.n0 + pre.c * 32, pre.m0 + q * 32);
             }
@@ -197,16 +198,37 @@ umma_apply_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restr
                 if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar_acc_empty + buf)) : "memory");
             }
             if (!mbar_wait(smem_u32(wbar + slot), (cons / AP_NBOX) & 1u)) { s_timeout = 1; ok = false; break; }
-            uint8_t *box = boxes + slot * AP_BOX_BYTES + lane * 128;
+            if (WB == 4) {
+                uint8_t *box = boxes + slot * AP_BOX_BYTES + lane * 128;
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                float4 *p = (float4 *)(box + ((j ^ (lane & 7)) << 4));
-                float4 x = *p;
-                x.x = __fmaf_rn(-sc.step_scale, __uint_as_float(v[4 * j + 0]), __fmul_rn(sc.decay, x.x));
-                x.y = __fmaf_rn(-sc.step_scale, __uint_as_float(v[4 * j + 1]), __fmul_rn(sc.decay, x.y));
-                x.z = __fmaf_rn(-sc.step_scale, __uint_as_float(v[4 * j + 2]), __fmul_rn(sc.decay, x.z));
-                x.w = __fmaf_rn(-sc.step_scale, __uint_as_float(v[4 * j + 3]), __fmul_rn(sc.decay, x.w));
-                *p = x;
+                for (int j = 0; j < 8; ++j) {
+                    float4 *p = (float4 *)(box + ((j ^ (lane & 7)) << 4));
+                    float4 x = *p;
+                    x.x = __fmaf_rn(-sc.step_scale, __uint_as_float(v[4 * j + 0]), __fmul_rn(sc.decay, x.x));
+                    x.y = __fmaf_rn(-sc.step_scale, __uint_as_float(v[4 * j + 1]), __fmul_rn(sc.decay, x.y));
+                    x.z = __fmaf_rn(-sc.step_scale, __uint_as_float(v[4 * j + 2]), __fmul_rn(sc.decay, x.z));
+                    x.w = __fmaf_rn(-sc.step_scale, __uint_as_float(v[4 * j + 3]), __fmul_rn(sc.decay, x.w));
+                    *p = x;
+                }
+            } else {
+                // BF16 weights: a row of the box is 64 bytes (four 16-byte chunks, 64-byte swizzle); the update
+                // is formed in FP32 and rounded to nearest even
+                uint8_t *box = boxes + slot * AP_BOX_BYTES + lane * 64;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    uint4 *p = (uint4 *)(box + ((j ^ ((lane >> 1) & 3)) << 4));
+                    uint4 x = *p;
+                    uint32_t w[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const float w0 = __uint_as_float(w[u] << 16), w1 = __uint_as_float(w[u] & 0xffff0000u);
+                        const float y0 = __fmaf_rn(-sc.step_scale, __uint_as_float(v[8 * j + 2 * u]), __fmul_rn(sc.decay, w0));
+                        const float y1 = __fmaf_rn(-sc.step_scale, __uint_as_float(v[8 * j + 2 * u + 1]), __fmul_rn(sc.decay, w1));
+                        const __nv_bfloat162 h = __floats2bfloat162_rn(y0, y1);
+                        w[u] = *(const uint32_t *)&h;
+                    }
+                    *p = make_uint4(w[0], w[1], w[2], w[3]);
+                }
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
@@ -221,7 +243,7 @@ umma_apply_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restr
                 if (lane == 0) {
                     asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(AP_LAG - 1) : "memory");
                     const uint32_t pslot = issued % AP_NBOX;
-                    mbar_expect_tx(smem_u32(wbar + pslot), AP_BOX_BYTES);
+                    mbar_expect_tx(smem_u32(wbar + pslot), W_BOX_BYTES);
                     tma_load_2d(smem_u32(boxes + pslot * AP_BOX_BYTES), &probs[pre.prob].tmW, smem_u32(wbar + pslot),
                                 pre.n0 + pre.c * 32, pre.m0 + q * 32);
                 }
@@ -245,20 +267,29 @@ umma_apply_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restr
 
 cudaError_t umma_apply_configure()
 {
-    cudaError_t e = cudaFuncSetAttribute(umma_apply_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, ApplyCfg<128>::SMEM);
-    if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(umma_apply_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, ApplyCfg<256>::SMEM);
+    cudaError_t e;
+#define TSR_AP_CFG(BN_, WB_)                                                                                           \
+    if ((e = cudaFuncSetAttribute(umma_apply_kernel<BN_, WB_>, cudaFuncAttributeMaxDynamicSharedMemorySize,            \
+                                  ApplyCfg<BN_>::SMEM)) != cudaSuccess)                                                \
+        return e
+    TSR_AP_CFG(128, 4); TSR_AP_CFG(256, 4); TSR_AP_CFG(128, 2); TSR_AP_CFG(256, 2);
+#undef TSR_AP_CFG
+    return cudaSuccess;
 }
 
 cudaError_t umma_apply_launch(const UmmaProblem *probs, const UmmaTile *tiles, int num_tiles, int num_sms, int bn,
-                              const StepScalars &sc, int32_t *status, cudaStream_t stream)
+                              int w_bytes, const StepScalars &sc, int32_t *status, cudaStream_t stream)
 {
     if (num_tiles <= 0) return cudaSuccess;
     const int grid = num_tiles < num_sms ? num_tiles : num_sms;
-    if (bn == 256)
-        umma_apply_kernel<256><<<grid, AP_THREADS, ApplyCfg<256>::SMEM, stream>>>(probs, tiles, num_tiles, sc, status);
+    if (bn == 256 && w_bytes == 4)
+        umma_apply_kernel<256, 4><<<grid, AP_THREADS, ApplyCfg<256>::SMEM, stream>>>(probs, tiles, num_tiles, sc, status);
+    else if (bn == 256)
+        umma_apply_kernel<256, 2><<<grid, AP_THREADS, ApplyCfg<256>::SMEM, stream>>>(probs, tiles, num_tiles, sc, status);
+    else if (w_bytes == 4)
+        umma_apply_kernel<128, 4><<<grid, AP_THREADS, ApplyCfg<128>::SMEM, stream>>>(probs, tiles, num_tiles, sc, status);
     else
-        umma_apply_kernel<128><<<grid, AP_THREADS, ApplyCfg<128>::SMEM, stream>>>(probs, tiles, num_tiles, sc, status);
+        umma_apply_kernel<128, 2><<<grid, AP_THREADS, ApplyCfg<128>::SMEM, stream>>>(probs, tiles, num_tiles, sc, status);
     return cudaGetLastError();
 }
 

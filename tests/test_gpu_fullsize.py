@@ -74,3 +74,40 @@ def test_llama60m_full_set_sampled_outputs():
 def test_llama1b_full_set_sampled_outputs():
     w = ti.workload(4)
     _run(4, [0, 4, 6, len(w.blocks) - 1])
+
+
+def test_llama1b_layer_with_bf16_weights():
+    """One layer of the 1B set plus the embedding (r = 512: the 256-wide tiles of the apply kernel)
+    with weights stored in BF16; sampled weights against the oracle's update rounded to BF16."""
+    import paper_2602_08007_b200 as tsr
+    w = ti.workload(4)
+    blocks = list(w.blocks[:7]) + [w.blocks[-1]]
+    dev = torch.device("cuda")
+    plan = tsr.Plan(blocks, g_dtype=torch.bfloat16, w_dtype=torch.bfloat16, device=dev)
+    W0 = []
+    for i, b in enumerate(blocks):
+        plan.G[i].copy_(ti.gradient(b.m, b.n, ti.seed_for(4, i, 1, ti.ROLE_GRAD), dtype=torch.bfloat16, device=dev))
+        plan.W[i].copy_(ti.weights(b.m, b.n, ti.seed_for(4, i, 0, ti.ROLE_WEIGHT), device=dev).to(torch.bfloat16))
+        plan.U[i].copy_(ti.orthonormal(b.m, b.r, 300 + 2 * i).to(dev))
+        plan.V[i].copy_(ti.orthonormal(b.n, b.r, 301 + 2 * i).to(dev))
+        W0.append(plan.W[i].clone())
+    plan.bases_changed()
+    plan.step(tsr.make_hyper(1, lr=1e-3), fuse_adam=True)
+    torch.cuda.synchronize()
+    assert plan.poll_status() == [0] * len(blocks)
+    rng = np.random.default_rng(9)
+    for i, b in enumerate(blocks):
+        U, V, Cg = to64(plan.U[i]), to64(plan.V[i]), to64(plan.C[i])
+        Mo, Vo = np.zeros_like(Cg), np.zeros_like(Cg)
+        Do = oracle.adam_core(Cg, Mo, Vo, HYPER["beta1"], HYPER["beta2"], HYPER["eps"], 1)
+        I = np.unique(np.concatenate([rng.integers(0, b.m, 6), [0, b.m - 1]]))
+        J = np.unique(np.concatenate([rng.integers(0, b.n, 6), [0, b.n - 1]]))
+        before = W0[i].double().cpu().numpy()[np.ix_(I, J)]
+        Wsub = before.copy()
+        oracle.backproject_apply(np.ascontiguousarray(U[I, :]), Do, np.ascontiguousarray(V[J, :]), Wsub, HYPER["lr"])
+        step_size = np.abs(Wsub - before).max()
+        Wo = torch.from_numpy(Wsub).float().to(torch.bfloat16).double().numpy()
+        Wg = plan.W[i].double().cpu().numpy()[np.ix_(I, J)]
+        assert np.all(np.abs(Wg - Wo) <= 2.0 ** -7 * np.abs(Wo) + 0.1 * step_size), b.name
+        assert rel_fro(Wg, Wo) < TOL_BF16
+        assert not np.array_equal(Wg, before)     # the weights did move

@@ -180,6 +180,55 @@ def test_two_workers_averaging_the_core_match_the_oracle():
     assert worst < TOL_BF16, worst
 
 
+def _bf16_round(x64):
+    """FP64 array rounded to BF16 (through FP32, round to nearest even) and widened back."""
+    return torch.from_numpy(np.ascontiguousarray(x64)).float().to(torch.bfloat16).double().numpy()
+
+
+@pytest.mark.parametrize("g_dtype,shapes", [
+    (torch.bfloat16, [dict(m=256, n=384, r=64), dict(m=200, n=328, r=40), dict(m=384, n=640, r=128)]),
+    (torch.float32, [dict(m=200, n=330, r=24)]),
+])
+def test_bf16_weights_follow_the_oracle_with_the_same_rounding(g_dtype, shapes):
+    """Weights stored in BF16: the update is formed in FP32 and rounded to nearest even.  The oracle
+    keeps W in FP64; the test starts every oracle step from the library's current BF16 weights and
+    rounds the oracle's result to BF16, i.e. both sides take the rounding decision at the same point
+    from the same inputs, and then compares element-wise: all but the elements that sit at a
+    rounding boundary agree exactly, the others differ by one BF16 unit."""
+    import paper_2602_08007_b200 as tsr
+    plan = tsr.Plan(shapes, g_dtype=g_dtype, w_dtype=torch.bfloat16)
+    _given_bases(plan, shapes, seed0=700)
+    blks = []
+    for i, sh in enumerate(shapes):
+        w0 = ti.weights(sh["m"], sh["n"], 40 + i).to(torch.bfloat16)
+        plan.W[i].copy_(w0.cuda())
+        ob = oracle.OracleBlock(w0.double().numpy(), sh["r"], 0, 0, 0)
+        ob.set_bases(to64(plan.U[i]), to64(plan.V[i]))
+        plan.M[i].zero_(); plan.Vm[i].zero_()
+        blks.append(ob)
+    worst, mism = 0.0, 0.0
+    for t in (1, 2, 3, 4):
+        G64 = [fill_gradient(plan, i, 2000 * t + i) for i in range(len(shapes))]
+        W_in = [plan.W[i].double().cpu().numpy() for i in range(len(shapes))]
+        plan.step(tsr.make_hyper(t, lr=1e-3, weight_decay=0.01), fuse_adam=True)
+        torch.cuda.synchronize()
+        for i, ob in enumerate(blks):
+            before = W_in[i]
+            ob.W[...] = before                     # every step starts from the same BF16 weights on both sides
+            ob.step(G64[i], weight_decay=f32(0.01), **HYPER)
+            step_size = np.abs(ob.W - before).max()
+            ob.W[...] = _bf16_round(ob.W)
+            Wg = plan.W[i].double().cpu().numpy()
+            worst = max(worst, rel_fro(Wg, ob.W))
+            mism = max(mism, float(np.mean(Wg != ob.W)))
+            # apart by at most one BF16 unit plus the element-wise slack of the update itself (a core entry
+            # whose sign the BF16 operands flip moves D by O(1): up to a tenth of the largest update)
+            assert np.all(np.abs(Wg - ob.W) <= 2.0 ** -7 * np.abs(ob.W) + 0.1 * step_size)
+    assert plan.poll_status() == [0] * len(shapes)
+    assert worst < (TOL_BF16 if g_dtype == torch.bfloat16 else 2e-3), worst
+    assert mism < 0.25, mism
+
+
 def test_split_k_core_matches_oracle():
     # m large enough that the core GEMM is split along K (tall embedding-like block)
     shapes = [dict(m=9000, n=128, r=32)]

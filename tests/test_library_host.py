@@ -55,8 +55,11 @@ def test_create_validates_shapes(tsr):
     for d in bad:
         rc, ctx = _create(tsr, [d])
         assert rc == 2 and not ctx.value
-    rc, _ = _create(tsr, [D(16, 16, 16, 16, 4, 0, 0, 0, 0, 1, 0, 0)])  # BF16 weights not implemented
-    assert rc == 6
+    rc, ctx = _create(tsr, [D(16, 16, 16, 16, 4, 0, 0, 0, 0, 1, 0, 0)])  # BF16 weights
+    assert rc == 0 and ctx.value
+    assert tsr.lib().tsr_destroy(ctx) == 0
+    rc, _ = _create(tsr, [D(16, 16, 16, 16, 4, 0, 0, 0, 0, 1, 0, 0), D(16, 16, 16, 16, 4, 0, 0, 0, 0, 0, 0, 0)])
+    assert rc == 6                                                      # one weight type per context
     rc, _ = _create(tsr, [D(16, 16, 16, 16, 4, 0, 0, 0, 7, 0, 0, 0)])
     assert rc == 6
     assert tsr.lib().tsr_create(None, None, 0) == 1
