@@ -281,6 +281,8 @@ void build_tiles(tsr_ctx *ctx)
     // apply: 256-wide tiles halve the P traffic per byte of W, which pays once the operands are as wide
     // as r = 512 (measured 2.28 -> 2.05 ms on the 1B set; at r = 256 the narrow tile is faster)
     ctx->bn[KA] = rmax >= 512 ? 256 : 128;
+    // sketches (N = k columns): wide tiles read the gradient rows fewer times
+    for (int kd : {KY, KZ}) ctx->bn[kd] = rmax >= 256 ? 256 : 128;
     for (int bi : ctx->order) {
         Block &b = ctx->blocks[bi];
         for (int kd = 0; kd < NKIND; ++kd) b.tile_begin[kd] = b.tile_end[kd] = (int)ctx->tiles[kd].size();
@@ -1044,7 +1046,7 @@ tsr_status tsr_bind(tsr_ctx *ctx, const tsr_mat_ptrs *ptrs, int32_t count, void 
             base(P, (int)m, (int)k, (int)n, EPI_STORE_F32);
             P.planes = 2; P.plane_rows = (int)k;
             if ((s = encode_map(ctx, &P.tmA, b.p.G, m, n, b.d.ldg, 128)) != TSR_OK) return s;
-            if ((s = encode_map(ctx, &P.tmB, b.Xt, 2 * k, n, b.nl, 64)) != TSR_OK) return s;
+            if ((s = encode_map(ctx, &P.tmB, b.Xt, 2 * k, n, b.nl, ctx->bn[KY] / 2)) != TSR_OK) return s;
             P.out = b.buf[0]; P.ld_out = k;
         }
         {   // Z = G^T X : A = G^T copy [n x m], B = X^T planes [2k x m]
@@ -1052,7 +1054,7 @@ tsr_status tsr_bind(tsr_ctx *ctx, const tsr_mat_ptrs *ptrs, int32_t count, void 
             base(P, (int)n, (int)k, (int)m, EPI_STORE_F32);
             P.planes = 2; P.plane_rows = (int)k;
             if ((s = encode_map(ctx, &P.tmA, b.Gt, n, m, b.ml, 128)) != TSR_OK) return s;
-            if ((s = encode_map(ctx, &P.tmB, b.Xt, 2 * k, m, b.ml, 64)) != TSR_OK) return s;
+            if ((s = encode_map(ctx, &P.tmB, b.Xt, 2 * k, m, b.ml, ctx->bn[KZ] / 2)) != TSR_OK) return s;
             P.out = b.buf[0]; P.ld_out = k;
         }
         if (b.tc_rows) {   // rows [M x k] (planes Xs) times small matrix^T planes Bts [N x k]

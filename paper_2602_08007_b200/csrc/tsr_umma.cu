@@ -410,6 +410,7 @@ cudaError_t umma_configure()
     if ((e = configure_one<128, EPI_STORE_F32, 1>()) != cudaSuccess) return e;
     if ((e = configure_one<256, EPI_STORE_F32, 1>()) != cudaSuccess) return e;
     if ((e = configure_one<128, EPI_STORE_F32, 2>()) != cudaSuccess) return e;
+    if ((e = configure_one<256, EPI_STORE_F32, 2>()) != cudaSuccess) return e;
     if ((e = configure_one<256, EPI_STORE_F32, 3>()) != cudaSuccess) return e;
     if ((e = configure_one<128, EPI_STORE_BF16, 1>()) != cudaSuccess) return e;
     if ((e = configure_one<256, EPI_STORE_BF16, 1>()) != cudaSuccess) return e;
@@ -427,6 +428,7 @@ cudaError_t umma_gemm_launch(const UmmaProblem *probs, const UmmaTile *tiles, in
 #define TSR_UG(BN_, EPI_, PL_) return launch_one<BN_, EPI_, PL_>(probs, tiles, num_tiles, num_sms, sc, status, stream)
     if (planes == 2) {
         if (bn == 128 && epilogue == EPI_STORE_F32) TSR_UG(128, EPI_STORE_F32, 2);
+        if (bn == 256 && epilogue == EPI_STORE_F32) TSR_UG(256, EPI_STORE_F32, 2);
         return cudaErrorInvalidValue;
     }
     if (planes == 3) {
