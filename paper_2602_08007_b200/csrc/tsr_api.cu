@@ -101,9 +101,9 @@ struct tsr_ctx {
     int stage_next = 0;
     // refresh runs as up to NGROUP independent groups of blocks on side streams, so that the
     // latency-bound small-matrix kernels of one group overlap the GEMM-like kernels of another
-    static constexpr int NGROUP = 4;
+    static constexpr int NGROUP = 8;
     cudaStream_t aux[NGROUP] = {};
-    cudaEvent_t ev_fork = nullptr, ev_join[NGROUP] = {}, ev_stagger[NGROUP] = {};
+    cudaEvent_t ev_fork = nullptr, ev_join[NGROUP] = {};
     static constexpr int NPIPE = 8;            // chunks of the pipelined host-buffer step
     cudaEvent_t ev_pipe_in[NPIPE] = {}, ev_pipe_done[NPIPE] = {};
     bool aux_ready = false;
@@ -633,8 +633,7 @@ tsr_status sketch(tsr_ctx *ctx, const RefreshLists &L, bool transposed, bool fro
 // One group of blocks through the whole refresh on stream st.  list_off / item_off: where this
 // group's slices start inside the context's device list / item tables.
 tsr_status do_refresh_group(tsr_ctx *ctx, const std::vector<int> &list, uint64_t seed, const float *const *omegas,
-                            cudaStream_t st, size_t list_off, const size_t *item_off, bool reexpress,
-                            cudaEvent_t started = nullptr)
+                            cudaStream_t st, size_t list_off, const size_t *item_off, bool reexpress)
 {
     if (list.empty()) return TSR_OK;
     tsr_status s;
@@ -676,7 +675,6 @@ tsr_status do_refresh_group(tsr_ctx *ctx, const std::vector<int> &list, uint64_t
     // Y = G Omega; Q = orth(Y)
     if ((s = sketch(ctx, L, false, true, omegas, st)) != TSR_OK) return s;
     if ((s = orth(ctx, L, 0, qmax == 0, st)) != TSR_OK) return s;
-    if (started) TSR_CUDA(ctx, cudaEventRecord(started, st));   // the next group may start now (see do_refresh)
     for (int it = 0; it < qmax; ++it) {
         // Yrow = G^T Q; Qrow = orth(Yrow); Y = G Qrow; Q = orth(Y)
         if ((s = sketch(ctx, L, true, false, nullptr, st)) != TSR_OK) return s;
@@ -751,12 +749,11 @@ tsr_status do_refresh(tsr_ctx *ctx, const std::vector<int> &list, uint64_t seed,
         std::vector<const float *> om;
         for (size_t i = lo; i < hi; ++i) { grp.push_back(list[perm[i]]); om.push_back(omegas ? omegas[perm[i]] : nullptr); }
         TSR_CUDA(ctx, cudaStreamWaitEvent(ctx->aux[g], ctx->ev_fork, 0));
-        // Groups start one orthonormalisation apart: in lock-step all groups would sit in the same
-        // one-CTA-per-matrix kernel at the same time (more CTAs than SMs, two waves) and leave the
-        // SMs idle that the throughput-bound kernels of another group could use.
-        if (g > 0) TSR_CUDA(ctx, cudaStreamWaitEvent(ctx->aux[g], ctx->ev_stagger[g - 1], 0));
+        // All groups start together: with eight groups of about twenty blocks the one-CTA-per-matrix
+        // kernels of different groups drift apart by themselves, and a forced offset between the
+        // groups only lengthened the critical path when it was measured.
         tsr_status s = do_refresh_group(ctx, grp, seed, omegas ? om.data() : nullptr, ctx->aux[g], list_off, item_off,
-                                        reexpress, ctx->ev_stagger[g]);
+                                        reexpress);
         if (s != TSR_OK && result == TSR_OK) result = s;
         TSR_CUDA(ctx, cudaEventRecord(ctx->ev_join[g], ctx->aux[g]));
         TSR_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_join[g], 0));
@@ -905,7 +902,7 @@ tsr_status tsr_destroy(tsr_ctx *ctx)
     if (ctx->profiling)
         for (cudaEvent_t e : ctx->ev) if (e) cudaEventDestroy(e);
     if (ctx->aux_ready) {
-        for (int g = 0; g < tsr_ctx::NGROUP; ++g) { cudaStreamDestroy(ctx->aux[g]); cudaEventDestroy(ctx->ev_join[g]); cudaEventDestroy(ctx->ev_stagger[g]); }
+        for (int g = 0; g < tsr_ctx::NGROUP; ++g) { cudaStreamDestroy(ctx->aux[g]); cudaEventDestroy(ctx->ev_join[g]); }
         cudaEventDestroy(ctx->ev_fork);
         for (int c = 0; c < tsr_ctx::NPIPE; ++c) { cudaEventDestroy(ctx->ev_pipe_in[c]); cudaEventDestroy(ctx->ev_pipe_done[c]); }
     }
@@ -1085,7 +1082,6 @@ tsr_status tsr_bind(tsr_ctx *ctx, const tsr_mat_ptrs *ptrs, int32_t count, void 
         for (int g = 0; g < tsr_ctx::NGROUP; ++g) {
             TSR_CUDA(ctx, cudaStreamCreateWithFlags(&ctx->aux[g], cudaStreamNonBlocking));
             TSR_CUDA(ctx, cudaEventCreateWithFlags(&ctx->ev_join[g], cudaEventDisableTiming));
-            TSR_CUDA(ctx, cudaEventCreateWithFlags(&ctx->ev_stagger[g], cudaEventDisableTiming));
         }
         TSR_CUDA(ctx, cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming));
         for (int c = 0; c < tsr_ctx::NPIPE; ++c) {
