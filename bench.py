@@ -465,6 +465,95 @@ def run_ours(args, w: ti.Workload):
         dist.destroy_process_group()
 
 
+# --------------------------------------------------------------------------------------------
+# ablation arms (Section 5, "Two-Sidedness, Randomized SVD"): kernel times and bytes
+# --------------------------------------------------------------------------------------------
+def run_ablation(args, w: ti.Workload):
+    """The comparison arms of the paper's ablation on synthetic gradients of the chosen set, one
+    JSON line: optimizer step and synchronized bytes of the two-sided method against the one-sided
+    arm (C = U^T G, r x n), and the randomized refresh against the exact-SVD arm (the same refresh
+    with a sketch as wide as the smaller side of the block and no power iteration, which spans the
+    whole range of G).  Not the headline benchmark: a diagnostic report."""
+    import paper_2602_08007_b200 as tsr
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    device = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(device)
+    dt = torch.bfloat16 if w.g_dtype == "bf16" else torch.float32
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)
+
+    def spec(b, **over):
+        d = dict(m=b.m, n=b.n, r=b.r, p=b.p, q=b.q, K=0, is_embedding=b.is_embedding, flags=0)
+        d.update(over)
+        return d
+
+    def make(specs):
+        plan = tsr.Plan(specs, g_dtype=dt, device=device)
+        for i, b in enumerate(w.blocks):
+            plan.G[i].copy_(ti.gradient(b.m, b.n, ti.seed_for(w.config_id, i, 0, ti.ROLE_INIT_GRAD), dtype=dt, device=device))
+            plan.W[i].copy_(ti.weights(b.m, b.n, ti.seed_for(w.config_id, i, 0, ti.ROLE_WEIGHT), device=device))
+        return plan
+
+    def time_refresh(plan, reps=3):
+        best = float("inf")
+        for rep in range(reps + 1):     # the first call is the warm-up
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            flush.fill_(rep)
+            e0.record()
+            plan.init_subspace(seed=ti.BASE_SEED + rep)
+            e1.record()
+            torch.cuda.synchronize()
+            if rep > 0:
+                best = min(best, e0.elapsed_time(e1))
+        return best
+
+    def time_steps(plan, steps):
+        times = []
+        for t in range(1, steps + args.warmup + 1):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            flush.fill_(t & 0xFF)
+            e0.record()
+            plan.step(tsr.make_hyper(t), seed=ti.BASE_SEED, fuse_adam=True)
+            e1.record()
+            torch.cuda.synchronize()
+            if t > args.warmup:
+                times.append(e0.elapsed_time(e1))
+        return statistics.median(times)
+
+    out = {"mode": "ablation", "config": {"workload": w.name, "blocks": len(w.blocks)}, "data": "synthetic",
+           "steps": args.steps, "warmup": args.warmup, "l2": "256 MB written before every timed call"}
+    arms = {}
+    for name, flags in (("two_sided", 0), ("one_sided", tsr.TSR_BLOCK_ONE_SIDED)):
+        plan = make([spec(b, flags=flags) for b in w.blocks])
+        refresh_ms = time_refresh(plan)
+        step_ms = time_steps(plan, args.steps)
+        core, sketch = plan.comm_bytes(0, 4)
+        arms[name] = {"step_ms": step_ms, "refresh_ms": refresh_ms, "core_bytes_per_step": core,
+                      "sketch_bytes_per_refresh": sketch, "state_elems": plan.state_elems(),
+                      "device_status": sorted(set(plan.poll_status()))}
+        plan.close()
+        del plan
+        torch.cuda.empty_cache()
+    out["arms"] = arms
+    out["one_sided_over_two_sided"] = {
+        "core_bytes": arms["one_sided"]["core_bytes_per_step"] / arms["two_sided"]["core_bytes_per_step"],
+        "step_ms": arms["one_sided"]["step_ms"] / arms["two_sided"]["step_ms"]}
+    if max(min(b.m, b.n) for b in w.blocks) <= 1056:
+        plan = make([spec(b, p=min(b.m, b.n) - b.r, q=0) for b in w.blocks])
+        exact_ms = time_refresh(plan)
+        _, exact_sketch = plan.comm_bytes(0, 4)
+        out["refresh"] = {"rsvd_ms": arms["two_sided"]["refresh_ms"], "exact_svd_ms": exact_ms,
+                          "rsvd_over_exact_ms": arms["two_sided"]["refresh_ms"] / exact_ms,
+                          "rsvd_sketch_bytes": arms["two_sided"]["sketch_bytes_per_refresh"],
+                          "exact_sketch_bytes": exact_sketch,
+                          "device_status": sorted(set(plan.poll_status()))}
+        plan.close()
+    else:
+        out["refresh"] = {"rsvd_ms": arms["two_sided"]["refresh_ms"], "exact_svd_ms": None,
+                          "why": "the exact arm needs a sketch as wide as min(m, n), above the library's limit of 1056"}
+    print(json.dumps(out), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -485,6 +574,8 @@ def main():
                     help="variant: weights stored in BF16 (4 instead of 8 bytes of read-modify-write per weight)")
     ap.add_argument("--random-bases", action="store_true",
                     help="profiling aid: random bases instead of the initial refresh (numbers not for reporting)")
+    ap.add_argument("--ablation", action="store_true",
+                    help="report the one-sided and exact-SVD comparison arms of the chosen set instead of the benchmark")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
@@ -495,7 +586,9 @@ def main():
         w = ti.Workload(w.name + "-first%dlayers" % args.layers, w.config_id, w.g_dtype, w.steps, keep)
     if args.config < 3:
         args.flush_l2 = True
-    if args.impl == "reference":
+    if args.ablation:
+        run_ablation(args, w)
+    elif args.impl == "reference":
         run_reference(args, w)
     else:
         run_ours(args, w)

@@ -83,8 +83,14 @@ typedef enum { TSR_RULE_ADAM = 0, TSR_RULE_SGD = 1 } tsr_rule;
  * whose moments are zero) replace the first moment by M' = Unew^T (Uold M Vold^T) Vnew, i.e. keep
  * the lifted moment, projected onto the refreshed subspaces -- the "refresh alignment" the
  * paper's convergence analysis assumes.  Algorithm 1 as printed leaves M untouched (flag clear).
- * The second moment is never re-expressed.  Costs (m + n) r + 3 r^2 floats of extra scratch. */
-typedef enum { TSR_BLOCK_REEXPRESS_MOMENT = 1 } tsr_block_flags;
+ * The second moment is never re-expressed.  Costs (m + n) r + 3 r^2 floats of extra scratch.
+ * TSR_BLOCK_ONE_SIDED: the one-sided arm of the paper's comparison (Table 1 and the ablation of
+ * Section 5: synchronized object C = U^T G of size r x n): the step of this block is
+ * C = U^T G, moments and D in that r x n space, W <- (1 - lr wd) W - lr scale U D.  M, Vm and C of
+ * the block are then r x n (row-major, dense); V is still bound and still written by every refresh
+ * (the refresh is the same), but no step reads it.  Not combinable with
+ * TSR_BLOCK_REEXPRESS_MOMENT. */
+typedef enum { TSR_BLOCK_REEXPRESS_MOMENT = 1, TSR_BLOCK_ONE_SIDED = 2 } tsr_block_flags;
 
 /* One matrix block.  Embedding blocks are ordinary blocks with their own (r, K)
  * (Section 3.6); is_embedding only labels them for tsr_embed_step. */
@@ -107,7 +113,7 @@ typedef struct {
     void *W;       /* m x n (ldw), FP32, updated in place                               */
     float *U;      /* m x r                                                             */
     float *V;      /* n x r                                                             */
-    float *M;      /* r x r first moment                                                */
+    float *M;      /* r x r first moment (r x n for a TSR_BLOCK_ONE_SIDED block, like Vm and C) */
     float *Vm;     /* r x r second moment (unused by TSR_RULE_SGD, may then be NULL)    */
     float *C;      /* r x r core, written by every projection: the tensor a data-parallel
                       job would all-reduce (Algorithm 1, "C_bar <- AR(C)")              */
@@ -232,12 +238,14 @@ TSR_API tsr_status tsr_dense_adamw(const tsr_dense_tensor *tensors, int32_t coun
 /* ---- reporting -------------------------------------------------------------------------- */
 
 /* Section 3.2: bytes one worker would hand to the all-reduce in one step, summed over blocks:
- * *core = sum r^2 * bytes_per_elem (every step); *sketch = sum (r+p)(m+n) * bytes_per_elem for
- * the blocks that refresh at `step` (0 if none; step <= 0 counts a refresh of every block). */
+ * *core = sum r^2 * bytes_per_elem (every step; r n for a one-sided block, Table 1); *sketch =
+ * sum (r+p)(m+n) * bytes_per_elem for the blocks that refresh at `step` (0 if none; step <= 0
+ * counts a refresh of every block). */
 TSR_API tsr_status tsr_comm_bytes(const tsr_ctx *ctx, int64_t step, int32_t bytes_per_elem, uint64_t *core,
                                   uint64_t *sketch);
 
-/* Optimizer-state elements (U, V, M, Vm) summed over blocks: sum (m+n) r + 2 r^2 (Table 2). */
+/* Optimizer-state elements (U, V, M, Vm) summed over blocks: sum (m+n) r + 2 r^2 (Table 2);
+ * a one-sided block counts U and its r x n moments: m r + 2 r n. */
 TSR_API tsr_status tsr_state_elems(const tsr_ctx *ctx, uint64_t *elems);
 
 /* Copies the per-block device status words (a tsr_status each; TSR_OK if nothing was detected

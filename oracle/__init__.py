@@ -8,6 +8,7 @@ from .tsr_oracle import (  # noqa: F401
     OracleBlock,
     adam_core,
     backproject_apply,
+    backproject_one_sided,
     build,
     core_bytes,
     dense_adamw,

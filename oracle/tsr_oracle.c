@@ -151,6 +151,24 @@ int tsro_backproject_apply(int64_t m, int64_t n, int64_t r, const double *U, con
     return 0;
 }
 
+/* One-sided arm of the comparison (Table 1, "One-sided": the synchronized object is C = U^T G,   */
+/* r x n; Section 5 ablation): the update lives in the left subspace only, dW = U D with D the    */
+/* r x n normalised core, and the weights move as in Algorithm 1:                                 */
+/* W <- W - lr (scale * U D + weight_decay * W).                                                  */
+int tsro_backproject_one_sided(int64_t m, int64_t n, int64_t r, const double *U, const double *D,
+                               double *W, int64_t ldw, double lr, double weight_decay, double scale)
+{
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < m; ++i)
+        for (int64_t j = 0; j < n; ++j) {
+            double dw = 0.0;
+            for (int64_t a = 0; a < r; ++a) dw += U[IDX(i, a, r)] * D[IDX(a, j, n)];
+            const double w = W[IDX(i, j, ldw)];
+            W[IDX(i, j, ldw)] = w - lr * (scale * dw + weight_decay * w);
+        }
+    return 0;
+}
+
 /* ------------------------------------------------------------------------- */
 /* orth(Y): thin QR by Householder reflections (Section 3.5, "implemented by  */
 /* thin QR").  Y is M x k, M >= k.  Q (M x k) = first k columns of            */

@@ -47,6 +47,7 @@ def _load():
             lib.tsro_sgd_core.argtypes = [_i64, _ptr, _ptr, _ptr, _dbl]
             lib.tsro_dense_adamw.argtypes = [_i64, _ptr, _ptr, _ptr, _ptr, _dbl, _dbl, _dbl, _dbl, _dbl, _i64]
             lib.tsro_backproject_apply.argtypes = [_i64, _i64, _i64, _ptr, _ptr, _ptr, _ptr, _i64, _dbl, _dbl, _dbl]
+            lib.tsro_backproject_one_sided.argtypes = [_i64, _i64, _i64, _ptr, _ptr, _ptr, _i64, _dbl, _dbl, _dbl]
             lib.tsro_orth.argtypes = [_i64, _i64, _ptr, _ptr, _ptr]
             lib.tsro_svd_jacobi.argtypes = [_i64, _i64, _ptr, _ptr, _ptr, _ptr, ctypes.c_int]
             lib.tsro_rsvd_refresh.argtypes = [_i64, _i64, _i64, _i64, _i64, _ptr, _i64, _ptr, _ptr, _ptr, _ptr]
@@ -141,6 +142,18 @@ def backproject_apply(U, D, V, W, lr, weight_decay=0.0, scale=1.0) -> None:
     assert U.shape == (m, r) and V.shape == (n, r) and D.shape == (r, r)
     _check(_load().tsro_backproject_apply(m, n, r, _p(U), _p(D), _p(V), _p(W), n, lr, weight_decay, scale),
            "backproject_apply")
+
+
+def backproject_one_sided(U, D, W, lr, weight_decay=0.0, scale=1.0) -> None:
+    """One-sided arm (Table 1): W <- W - lr (scale * U D + weight_decay * W) with D of shape r x n,
+    in place on the float64 array W."""
+    U, D = _f64(U), _f64(D)
+    W = _f64(W, True)
+    m, n = W.shape
+    r = U.shape[1]
+    assert U.shape == (m, r) and D.shape == (r, n)
+    _check(_load().tsro_backproject_one_sided(m, n, r, _p(U), _p(D), _p(W), n, lr, weight_decay, scale),
+           "backproject_one_sided")
 
 
 def orth(Y, return_r: bool = False):

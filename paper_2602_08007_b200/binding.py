@@ -21,6 +21,7 @@ TSR_OK = 0
 TSR_F32, TSR_BF16 = 0, 1
 TSR_RULE_ADAM, TSR_RULE_SGD = 0, 1
 TSR_BLOCK_REEXPRESS_MOMENT = 1
+TSR_BLOCK_ONE_SIDED = 2
 
 STATUS_NAMES = {
     0: "TSR_OK", 1: "TSR_ERR_INVALID_ARG", 2: "TSR_ERR_SHAPE", 3: "TSR_ERR_ALIGNMENT", 4: "TSR_ERR_WORKSPACE",
@@ -180,7 +181,7 @@ def dense_adamw(params, grads, ms, vs, hyper: Hyper, stream=None) -> None:
 class Plan:
     """Owns a tsr_ctx plus the torch tensors it is bound to.
 
-    blocks: sequence of dicts/objects with m, n, r, p, q, K (and optionally is_embedding).
+    blocks: sequence of dicts/objects with m, n, r, p, q, K (and optionally is_embedding, flags).
     g_dtype: torch.float32 or torch.bfloat16.  w_dtype: torch.float32 (master weights) or
     torch.bfloat16.  Leading dimensions are padded to 16-byte row pitches unless pad=False.
     """
@@ -218,9 +219,10 @@ class Plan:
             self.W.append(Wt)
             self.U.append(torch.zeros(m, r, dtype=torch.float32, device=self.device))
             self.V.append(torch.zeros(n, r, dtype=torch.float32, device=self.device))
-            self.M.append(torch.zeros(r, r, dtype=torch.float32, device=self.device))
-            self.Vm.append(torch.zeros(r, r, dtype=torch.float32, device=self.device))
-            self.C.append(torch.zeros(r, r, dtype=torch.float32, device=self.device))
+            cn = n if int(g("flags", 0)) & TSR_BLOCK_ONE_SIDED else r   # one-sided arm: the core is r x n
+            self.M.append(torch.zeros(r, cn, dtype=torch.float32, device=self.device))
+            self.Vm.append(torch.zeros(r, cn, dtype=torch.float32, device=self.device))
+            self.C.append(torch.zeros(r, cn, dtype=torch.float32, device=self.device))
             self.descs[i] = MatDesc(m, n, ldg, ldw, r, int(g("p", 0)), int(g("q", 0)), int(g("K", 0)),
                                     TSR_BF16 if g_dtype == torch.bfloat16 else TSR_F32,
                                     TSR_BF16 if w_dtype == torch.bfloat16 else TSR_F32,

@@ -17,7 +17,7 @@ namespace {
 
 // KR*: tall-times-small products of the refresh on tensor cores (three TF32 products): rows of side
 // 0 (m) or 1 (n) times R^{-1} into buf[1] / buf[2], and the final U = Q Wu, V = B^T Wv.
-enum Kind : int { KT = 0, KC, KCS, KP, KA, KY, KZ, KR01, KR02, KR12, KRU, KRV, NKIND };
+enum Kind : int { KT = 0, KC, KCS, KP, KA, KY, KZ, KR01, KR02, KR12, KRU, KRV, KO, KOA, NKIND };
 constexpr int TSR_NUM_STAGES = 6;  // refresh, G*V, core GEMM, core update, U*D, apply
 
 struct Block {
@@ -29,6 +29,8 @@ struct Block {
     // step scratch
     bf16 *Ub = nullptr, *Ubt = nullptr, *Vb = nullptr, *Vbt = nullptr, *Tt = nullptr, *Pb = nullptr;
     bf16 *Db = nullptr, *Dbt = nullptr;
+    bool one_sided = false;   // C = U^T G (r x n): the comparison arm of Table 1
+    int64_t cn = 0;           // columns of C, M, Vm: r, or n for a one-sided block
     float *partial = nullptr;
     int nsplit = 1, kb_per_split = 0;
     float *T32 = nullptr, *P32 = nullptr, *D32 = nullptr;
@@ -93,7 +95,7 @@ struct tsr_ctx {
     int max_r = 0, max_k = 0;
     uint64_t launches = 0;                     // kernels launched through this context
     int num_sms = 148;
-    int bn[NKIND] = {128, 128, 128, 128, 128, 128, 128, 256, 256, 256, 256, 256};   // tile width of each GEMM kind
+    int bn[NKIND] = {128, 128, 128, 128, 128, 128, 128, 256, 256, 256, 256, 256, 128, 128};   // tile width of each GEMM kind
     bool profiling = false;
     cudaEvent_t ev[TSR_NUM_STAGES + 1] = {};   // stage boundaries of the last step (profiling only)
     bool ev_valid = false;
@@ -181,8 +183,8 @@ void layout(tsr_ctx *ctx, Arena &a, bool assign, size_t *step_end)
             void *ub = a.take((size_t)(m * b.rl) * 2), *ubt = a.take((size_t)(r * b.ml) * 2);
             void *vb = a.take((size_t)(n * b.rl) * 2), *vbt = a.take((size_t)(r * b.nl) * 2);
             void *tt = a.take((size_t)(r * b.ml) * 2), *pb = a.take((size_t)(m * b.rl) * 2);
-            void *db = a.take((size_t)(r * b.rl) * 2), *dbt = a.take((size_t)(r * b.rl) * 2);
-            void *part = b.nsplit > 1 ? a.take((size_t)b.nsplit * r * r * 4) : nullptr;
+            void *db = a.take((size_t)(r * b.rl) * 2), *dbt = a.take((size_t)(b.cn * b.rl) * 2);
+            void *part = (b.nsplit > 1 && !b.one_sided) ? a.take((size_t)b.nsplit * r * r * 4) : nullptr;
             if (assign) {
                 b.Ub = (bf16 *)ub; b.Ubt = (bf16 *)ubt; b.Vb = (bf16 *)vb; b.Vbt = (bf16 *)vbt;
                 b.Tt = (bf16 *)tt; b.Pb = (bf16 *)pb; b.Db = (bf16 *)db; b.Dbt = (bf16 *)dbt;
@@ -192,7 +194,7 @@ void layout(tsr_ctx *ctx, Arena &a, bool assign, size_t *step_end)
             void *t = a.take((size_t)(m * r) * 4), *pp = a.take((size_t)(m * r) * 4);
             if (assign) { b.T32 = (float *)t; b.P32 = (float *)pp; }
         }
-        void *d32 = a.take((size_t)(r * r) * 4);
+        void *d32 = a.take((size_t)(r * b.cn) * 4);
         if (assign) b.D32 = (float *)d32;
     }
     a.off = (a.off + 255) & ~(size_t)255;
@@ -250,7 +252,7 @@ void layout(tsr_ctx *ctx, Arena &a, bool assign, size_t *step_end)
 void add_tiles(tsr_ctx *ctx, int kind, int bi, int M, int N, int K, int kb_per_split, int tri = 0)
 {
     const int bn = ctx->bn[kind];
-    const int bm = (kind == KA) ? 128 : 256;   // the grouped GEMM runs on CTA pairs: 256-row tiles
+    const int bm = (kind == KA || kind == KOA) ? 128 : 256;   // the grouped GEMM runs on CTA pairs: 256-row tiles
     Block &b = ctx->blocks[bi];
     std::vector<UmmaTile> &v = ctx->tiles[kind];
     b.tile_begin[kind] = (int)v.size();
@@ -283,16 +285,23 @@ void build_tiles(tsr_ctx *ctx)
     ctx->bn[KA] = rmax >= 512 ? 256 : 128;
     // sketches (N = k columns): wide tiles read the gradient rows fewer times
     for (int kd : {KY, KZ}) ctx->bn[kd] = rmax >= 256 ? 256 : 128;
+    ctx->bn[KO] = ctx->bn[KT];
+    ctx->bn[KOA] = ctx->bn[KA];
     for (int bi : ctx->order) {
         Block &b = ctx->blocks[bi];
         for (int kd = 0; kd < NKIND; ++kd) b.tile_begin[kd] = b.tile_end[kd] = (int)ctx->tiles[kd].size();
         if (!b.fast) continue;
         const int m = (int)b.d.m, n = (int)b.d.n, r = b.d.r, k = b.k;
-        add_tiles(ctx, KT, bi, m, r, n, 0);
-        if (b.nsplit > 1) add_tiles(ctx, KCS, bi, r, r, m, b.kb_per_split);
-        else add_tiles(ctx, KC, bi, r, r, m, 0);
-        add_tiles(ctx, KP, bi, m, r, r, 0);
-        add_tiles(ctx, KA, bi, m, n, r, 0);
+        if (b.one_sided) {   // C = U^T G with the core update in the epilogue, then W -= U D
+            add_tiles(ctx, KO, bi, r, n, m, 0);
+            add_tiles(ctx, KOA, bi, m, n, r, 0);
+        } else {
+            add_tiles(ctx, KT, bi, m, r, n, 0);
+            if (b.nsplit > 1) add_tiles(ctx, KCS, bi, r, r, m, b.kb_per_split);
+            else add_tiles(ctx, KC, bi, r, r, m, 0);
+            add_tiles(ctx, KP, bi, m, r, r, 0);
+            add_tiles(ctx, KA, bi, m, n, r, 0);
+        }
         add_tiles(ctx, KY, bi, m, k, n, 0);
         add_tiles(ctx, KZ, bi, n, k, m, 0);
         if (b.tc_rows) {   // K blocks of 32 FP32 elements: pass 2 k so that the count comes out as ceil(k / 32)
@@ -449,7 +458,7 @@ tsr_status launch_kind(tsr_ctx *ctx, int kind, const std::vector<int> &list, int
         int lo = ranges[i].first, hi = ranges[i].second;
         size_t j = i + 1;
         while (j < ranges.size() && ranges[j].first == hi) { hi = ranges[j].second; ++j; }
-        if (kind == KA)
+        if (kind == KA || kind == KOA)
             TSR_CUDA(ctx, umma_apply_launch(ctx->d_probs[kind], ctx->d_tiles[kind] + lo, hi - lo, ctx->num_sms, ctx->bn[kind],
                                             elem_size(ctx->blocks[0].d.w_dtype), sc, ctx->d_status, st));
         else
@@ -477,29 +486,42 @@ tsr_status do_project(tsr_ctx *ctx, const std::vector<int> &list, bool fuse, con
         mark_stage(ctx, 2);
         if ((s = launch_kind(ctx, KC, list, fuse ? EPI_CORE_UPDATE : EPI_STORE_F32, 1, sc, st)) != TSR_OK) return s;
         if ((s = launch_kind(ctx, KCS, list, EPI_STORE_F32, 1, sc, st)) != TSR_OK) return s;
+        // one-sided blocks: C = U^T G needs the gradient with m as the contiguous index
+        bool any_one_sided = false;
+        for (int bi : list) {
+            const Block &b = ctx->blocks[bi];
+            if (!b.fast || !b.one_sided) continue;
+            TSR_KERNEL(ctx, 1, transpose_bf16((const bf16 *)b.p.G, (int)b.d.m, (int)b.d.n, b.d.ldg, b.Gt, b.ml, st));
+            any_one_sided = true;
+        }
+        if (any_one_sided && (s = launch_kind(ctx, KO, list, fuse ? EPI_CORE_UPDATE : EPI_STORE_F32, 1, sc, st)) != TSR_OK) return s;
     }
     std::vector<int> split, later;
-    int max_r = 1;
+    int max_r = 1, max_c = 1;
     for (int bi : list) {
         Block &b = ctx->blocks[bi];
         const int m = (int)b.d.m, n = (int)b.d.n, r = b.d.r;
-        if (!b.fast) {
+        if (!b.fast && b.one_sided) {
+            // C = U^T G on CUDA cores
+            TSR_KERNEL(ctx, 1, simt_gemm_bt(r, n, m, b.p.U, 1, r, b.p.G, b.d.g_dtype, b.d.ldg, 1, b.p.C, n, st));
+            if (fuse) { later.push_back(bi); max_r = std::max(max_r, r); max_c = std::max(max_c, n); }
+        } else if (!b.fast) {
             // T = G V, C = U^T T on CUDA cores
             TSR_KERNEL(ctx, 1, simt_gemm(m, r, n, b.p.G, b.d.g_dtype, b.d.ldg, 1, b.p.V, r, 1, b.T32, r, SIMT_STORE, 0, 0, st));
             TSR_KERNEL(ctx, 1, simt_gemm(r, r, m, b.p.U, TSR_F32, 1, r, b.T32, r, 1, b.p.C, r, SIMT_STORE, 0, 0, st));
-            if (fuse) { later.push_back(bi); max_r = std::max(max_r, r); }
+            if (fuse) { later.push_back(bi); max_r = std::max(max_r, r); max_c = std::max(max_c, r); }
         } else if (b.nsplit > 1) {
             split.push_back(bi);
-            max_r = std::max(max_r, r);
+            max_r = std::max(max_r, r); max_c = std::max(max_c, r);
         }
     }
     if (!split.empty()) {   // sum the split-K slabs (and, when fused, run the core update on the sum)
         if ((s = upload_list(ctx, ctx->d_list2, split, st)) != TSR_OK) return s;
-        TSR_KERNEL(ctx, 1, core_update_launch(ctx->d_cu_split, ctx->d_list2, (int)split.size(), max_r, sc, fuse ? 0 : 1, st));
+        TSR_KERNEL(ctx, 1, core_update_launch(ctx->d_cu_split, ctx->d_list2, (int)split.size(), max_r, max_c, sc, fuse ? 0 : 1, st));
     }
     if (!later.empty()) {
         if ((s = upload_list(ctx, ctx->d_list2, later, st)) != TSR_OK) return s;
-        TSR_KERNEL(ctx, 1, core_update_launch(ctx->d_cu_all, ctx->d_list2, (int)later.size(), max_r, sc, 0, st));
+        TSR_KERNEL(ctx, 1, core_update_launch(ctx->d_cu_all, ctx->d_list2, (int)later.size(), max_r, max_c, sc, 0, st));
     }
     mark_stage(ctx, 3);
     return TSR_OK;
@@ -509,10 +531,13 @@ tsr_status do_project(tsr_ctx *ctx, const std::vector<int> &list, bool fuse, con
 tsr_status do_core_update(tsr_ctx *ctx, const std::vector<int> &list, const StepScalars &sc, cudaStream_t st)
 {
     tsr_status s;
-    int max_r = 1;
-    for (int bi : list) max_r = std::max(max_r, (int)ctx->blocks[bi].d.r);
+    int max_r = 1, max_c = 1;
+    for (int bi : list) {
+        max_r = std::max(max_r, (int)ctx->blocks[bi].d.r);
+        max_c = std::max(max_c, (int)ctx->blocks[bi].cn);
+    }
     if ((s = upload_list(ctx, ctx->d_list, list, st)) != TSR_OK) return s;
-    TSR_KERNEL(ctx, 1, core_update_launch(ctx->d_cu_all, ctx->d_list, (int)list.size(), max_r, sc, 0, st));
+    TSR_KERNEL(ctx, 1, core_update_launch(ctx->d_cu_all, ctx->d_list, (int)list.size(), max_r, max_c, sc, 0, st));
     return TSR_OK;
 }
 
@@ -524,11 +549,17 @@ tsr_status do_apply(tsr_ctx *ctx, const std::vector<int> &list, const StepScalar
         if ((s = launch_kind(ctx, KP, list, EPI_STORE_BF16, 1, sc, st)) != TSR_OK) return s;
         mark_stage(ctx, 5);
         if ((s = launch_kind(ctx, KA, list, EPI_APPLY, 1, sc, st)) != TSR_OK) return s;
+        if ((s = launch_kind(ctx, KOA, list, EPI_APPLY, 1, sc, st)) != TSR_OK) return s;
     }
     for (int bi : list) {
         Block &b = ctx->blocks[bi];
         if (b.fast) continue;
         const int m = (int)b.d.m, n = (int)b.d.n, r = b.d.r;
+        if (b.one_sided) {   // W <- decay W - step_scale U D, D being r x n
+            TSR_KERNEL(ctx, 1, simt_gemm(m, n, r, b.p.U, TSR_F32, r, 1, b.D32, n, 1, (float *)b.p.W, b.d.ldw,
+                                    b.d.w_dtype == TSR_BF16 ? SIMT_APPLY_BF16 : SIMT_APPLY, sc.decay, sc.step_scale, st));
+            continue;
+        }
         TSR_KERNEL(ctx, 1, simt_gemm(m, r, r, b.p.U, TSR_F32, r, 1, b.D32, r, 1, b.P32, r, SIMT_STORE, 0, 0, st));
         TSR_KERNEL(ctx, 1, simt_gemm(m, n, r, b.P32, TSR_F32, r, 1, b.p.V, 1, r, (float *)b.p.W, b.d.ldw,
                                 b.d.w_dtype == TSR_BF16 ? SIMT_APPLY_BF16 : SIMT_APPLY, sc.decay, sc.step_scale, st));
@@ -774,7 +805,7 @@ tsr_status zero_moments(tsr_ctx *ctx, const std::vector<int> &list, cudaStream_t
 {
     for (int bi : list) {
         Block &b = ctx->blocks[bi];
-        const int64_t rr = (int64_t)b.d.r * b.d.r;
+        const int64_t rr = (int64_t)b.d.r * b.cn;
         TSR_CUDA(ctx, fill_zero_f32(b.p.M, rr, st));
         if (b.p.Vm) TSR_CUDA(ctx, fill_zero_f32(b.p.Vm, rr, st));
     }
@@ -862,7 +893,8 @@ tsr_status tsr_create(tsr_ctx **out, const tsr_mat_desc *descs, int32_t count)
         if (d.g_dtype != TSR_F32 && d.g_dtype != TSR_BF16) return TSR_ERR_UNSUPPORTED;
         if (d.w_dtype != TSR_F32 && d.w_dtype != TSR_BF16) return TSR_ERR_UNSUPPORTED;
         if (d.w_dtype != descs[0].w_dtype) return TSR_ERR_UNSUPPORTED;   // one weight type per context (one apply launch)
-        if ((d.flags & ~(int32_t)TSR_BLOCK_REEXPRESS_MOMENT) != 0 || (d.is_embedding != 0 && d.is_embedding != 1)) return TSR_ERR_INVALID_ARG;
+        if ((d.flags & ~(int32_t)(TSR_BLOCK_REEXPRESS_MOMENT | TSR_BLOCK_ONE_SIDED)) != 0 || (d.is_embedding != 0 && d.is_embedding != 1)) return TSR_ERR_INVALID_ARG;
+        if ((d.flags & TSR_BLOCK_REEXPRESS_MOMENT) && (d.flags & TSR_BLOCK_ONE_SIDED)) return TSR_ERR_UNSUPPORTED;
     }
     tsr_ctx *ctx = new (std::nothrow) tsr_ctx;
     if (!ctx) return TSR_ERR_INVALID_ARG;
@@ -872,13 +904,15 @@ tsr_status tsr_create(tsr_ctx **out, const tsr_mat_desc *descs, int32_t count)
         b.d = descs[i];
         memset(&b.p, 0, sizeof b.p);
         b.k = b.d.r + b.d.p;
+        b.one_sided = (b.d.flags & TSR_BLOCK_ONE_SIDED) != 0;
+        b.cn = b.one_sided ? b.d.n : b.d.r;
         b.rl = round_up(b.d.r, 8); b.ml = round_up(b.d.m, 8); b.nl = round_up(b.d.n, 8);
         // Candidate for the tensor-core path: BF16 gradient with 16-byte row pitches.  Pointer
         // alignment is checked at bind time.
         b.fast = (b.d.g_dtype == TSR_BF16) && ((b.d.ldg * 2) % 16 == 0) && ((b.d.ldw * elem_size(b.d.w_dtype)) % 16 == 0);
         b.tc_rows = b.fast && (b.k % 4 == 0);   // FP32 rows of k elements as a TMA operand: 16-byte row pitch
         const int nkb = (int)((b.d.m + 63) / 64);
-        if (nkb > 128) { b.kb_per_split = 32; b.nsplit = (nkb + 31) / 32; }
+        if (nkb > 128 && !b.one_sided) { b.kb_per_split = 32; b.nsplit = (nkb + 31) / 32; }
         ctx->max_r = std::max(ctx->max_r, (int)b.d.r);
         ctx->max_k = std::max(ctx->max_k, b.k);
         ctx->order.push_back(i);
@@ -987,7 +1021,7 @@ tsr_status tsr_bind(tsr_ctx *ctx, const tsr_mat_ptrs *ptrs, int32_t count, void 
         memset(&ca, 0, sizeof ca);
         ca.C = b.p.C; ca.Cout = b.p.C; ca.mom1 = b.p.M; ca.mom2 = b.p.Vm; ca.d_f32 = b.D32;
         ca.d_bf16 = nullptr; ca.dt_bf16 = b.fast ? b.Dbt : nullptr; ca.ldd = b.rl;
-        ca.split_stride = 0; ca.r = (int)r; ca.nsplit = 1;
+        ca.split_stride = 0; ca.r = (int)r; ca.nc = (int)b.cn; ca.nsplit = 1;
         cu_split[i] = ca;
         cu_split[i].C = b.partial; cu_split[i].nsplit = b.nsplit; cu_split[i].split_stride = r * r;
         RefreshDev &rd = rdev[i];
@@ -1005,6 +1039,24 @@ tsr_status tsr_bind(tsr_ctx *ctx, const tsr_mat_ptrs *ptrs, int32_t count, void 
         auto base = [&](UmmaProblem &P, int M, int N, int K, int epi) {
             P.M = M; P.N = N; P.K = K; P.planes = 1; P.plane_rows = 0; P.block = i; P.epilogue = epi;
         };
+        if (b.one_sided) {
+            {   // C = U^T G (+ core update) : A = U^T copy [r x m], B = G^T copy [n x m]
+                UmmaProblem &P = probs[KO][i];
+                base(P, (int)r, (int)n, (int)m, EPI_CORE_UPDATE);
+                if ((s = encode_map(ctx, &P.tmA, b.Ubt, r, m, b.ml, 128)) != TSR_OK) return s;
+                if ((s = encode_map(ctx, &P.tmB, b.Gt, n, m, b.ml, ctx->bn[KO] / 2)) != TSR_OK) return s;
+                P.out = b.p.C; P.ld_out = n; P.split_stride = 0;
+                P.mom1 = b.p.M; P.mom2 = b.p.Vm; P.d_bf16 = nullptr; P.dt_bf16 = b.Dbt; P.ldd = b.rl;
+            }
+            {   // W update : A = U copy [m x r], B = D^T copy [n x r]
+                UmmaProblem &P = probs[KOA][i];
+                base(P, (int)m, (int)n, (int)r, EPI_APPLY);
+                if ((s = encode_map(ctx, &P.tmA, b.Ub, m, r, b.rl, 128)) != TSR_OK) return s;
+                if ((s = encode_map(ctx, &P.tmB, b.Dbt, n, r, b.rl, 128)) != TSR_OK) return s;
+                if ((s = encode_map_w(ctx, &P.tmW, b.p.W, m, n, b.d.ldw, b.d.w_dtype)) != TSR_OK) return s;
+                P.out = b.p.W; P.ld_out = b.d.ldw;
+            }
+        }
         {   // T~ = (G V)^T : A = G [m x n], B = V^T copy [r x n]
             UmmaProblem &P = probs[KT][i];
             base(P, (int)m, (int)r, (int)n, EPI_STORE_BF16_T);
@@ -1228,11 +1280,11 @@ tsr_status tsr_step_grouped_host(tsr_ctx *ctx, const void *const *G_host, float 
     std::vector<size_t> c_off(nb, 0);
     {
         size_t off = 0;
-        for (int i = 0; i < nb; ++i) { c_off[i] = off; off += (size_t)ctx->blocks[i].d.r * ctx->blocks[i].d.r; }
+        for (int i = 0; i < nb; ++i) { c_off[i] = off; off += (size_t)ctx->blocks[i].d.r * (size_t)ctx->blocks[i].cn; }
     }
     auto copy_out = [&](int i, cudaStream_t cs) -> cudaError_t {
         const Block &b = ctx->blocks[i];
-        return cudaMemcpyAsync(C_host + c_off[i], b.p.C, (size_t)b.d.r * b.d.r * sizeof(float), cudaMemcpyDeviceToHost, cs);
+        return cudaMemcpyAsync(C_host + c_off[i], b.p.C, (size_t)b.d.r * (size_t)b.cn * sizeof(float), cudaMemcpyDeviceToHost, cs);
     };
     constexpr int NCHUNK = tsr_ctx::NPIPE;
     if (refresh_due || !ctx->aux_ready || nb < 2 * NCHUNK) {
@@ -1315,7 +1367,7 @@ tsr_status tsr_comm_bytes(const tsr_ctx *ctx, int64_t step, int32_t bytes_per_el
     if (!ctx || !core || !sketch || bytes_per_elem <= 0) return TSR_ERR_INVALID_ARG;
     uint64_t c = 0, sk = 0;
     for (const Block &b : ctx->blocks) {
-        c += (uint64_t)b.d.r * (uint64_t)b.d.r * (uint64_t)bytes_per_elem;
+        c += (uint64_t)b.d.r * (uint64_t)b.cn * (uint64_t)bytes_per_elem;
         const bool refresh = step <= 0 || (b.d.K > 0 && step % b.d.K == 0);
         if (refresh) sk += (uint64_t)b.k * (uint64_t)(b.d.m + b.d.n) * (uint64_t)bytes_per_elem;
     }
@@ -1328,7 +1380,8 @@ tsr_status tsr_state_elems(const tsr_ctx *ctx, uint64_t *elems)
 {
     if (!ctx || !elems) return TSR_ERR_INVALID_ARG;
     uint64_t e = 0;
-    for (const Block &b : ctx->blocks) e += (uint64_t)(b.d.m + b.d.n) * b.d.r + 2ull * b.d.r * b.d.r;
+    for (const Block &b : ctx->blocks)
+        e += b.one_sided ? (uint64_t)b.d.m * b.d.r + 2ull * b.d.r * b.d.n : (uint64_t)(b.d.m + b.d.n) * b.d.r + 2ull * b.d.r * b.d.r;
     *elems = e;
     return TSR_OK;
 }

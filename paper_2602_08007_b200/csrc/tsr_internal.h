@@ -89,6 +89,9 @@ enum SimtEpilogue : int { SIMT_STORE = 0, SIMT_APPLY = 1, SIMT_APPLY_BF16 = 2 };
 cudaError_t simt_gemm(int M, int N, int K, const void *A, int a_dtype, int64_t sa_i, int64_t sa_k, const float *B,
                       int64_t sb_k, int64_t sb_j, float *D, int64_t ldd, int epilogue, float decay, float step_scale,
                       cudaStream_t stream);
+// The same product with an FP32 A and a B of either type (b_dtype), plain store.
+cudaError_t simt_gemm_bt(int M, int N, int K, const float *A, int64_t sa_i, int64_t sa_k, const void *B, int b_dtype,
+                         int64_t sb_k, int64_t sb_j, float *D, int64_t ldd, cudaStream_t stream);
 
 struct CoreUpdateArgs {     // one entry per block for the stand-alone core update
     const float *C;         // r x r, or split-K partial slabs
@@ -99,11 +102,12 @@ struct CoreUpdateArgs {     // one entry per block for the stand-alone core upda
     int64_t ldd;
     int64_t split_stride;
     int32_t r, nsplit;
+    int32_t nc;             // columns of C, mom1, mom2 (r; n for a one-sided block)
 };
 // Runs the core update for the blocks args_dev[list_dev[0..nblocks)].  mode 0: full update;
 // mode 1: only sum split-K slabs into Cout.
 cudaError_t core_update_launch(const CoreUpdateArgs *args_dev, const int32_t *list_dev, int nblocks, int max_r,
-                               const StepScalars &sc, int mode, cudaStream_t stream);
+                               int max_cols, const StepScalars &sc, int mode, cudaStream_t stream);
 
 // BF16 operand copies of a basis X (rows x r, FP32): Xb[rows x ldb] and Xbt[r x ldt].
 cudaError_t make_shadows(const float *X, int rows, int r, bf16 *Xb, int64_t ldb, bf16 *Xbt, int64_t ldt,

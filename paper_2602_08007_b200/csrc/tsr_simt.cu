@@ -18,10 +18,10 @@ __device__ __forceinline__ float load_as_float<bf16>(const bf16 *p) { return __b
 
 constexpr int SG_BM = 64, SG_BN = 64, SG_BK = 16;
 
-template <typename TA, int EPI>
+template <typename TA, typename TB, int EPI>
 __global__ void __launch_bounds__(256)
 simt_gemm_kernel(int M, int N, int K, const TA *__restrict__ A, int64_t sa_i, int64_t sa_k,
-                 const float *__restrict__ B, int64_t sb_k, int64_t sb_j, float *__restrict__ D, int64_t ldd,
+                 const TB *__restrict__ B, int64_t sb_k, int64_t sb_j, float *__restrict__ D, int64_t ldd,
                  float decay, float step_scale)
 {
     __shared__ float As[SG_BK][SG_BM + 4];
@@ -53,7 +53,7 @@ simt_gemm_kernel(int M, int N, int K, const TA *__restrict__ A, int64_t sa_i, in
             int bj, bk;
             if (b_j_fast) { bj = e % SG_BN; bk = e / SG_BN; } else { bk = e % SG_BK; bj = e / SG_BK; }
             const int gj = n0 + bj, gk2 = k0 + bk;
-            rb[l] = (gj < N && gk2 < K) ? B[(int64_t)gk2 * sb_k + (int64_t)gj * sb_j] : 0.f;
+            rb[l] = (gj < N && gk2 < K) ? load_as_float<TB>(B + (int64_t)gk2 * sb_k + (int64_t)gj * sb_j) : 0.f;
         }
     };
     fetch(0);
@@ -107,6 +107,21 @@ simt_gemm_kernel(int M, int N, int K, const TA *__restrict__ A, int64_t sa_i, in
     }
 }
 
+// FP32 A (any strides) times a BF16 or FP32 B, plain store: the one-sided projection C = U^T G.
+cudaError_t simt_gemm_bt(int M, int N, int K, const float *A, int64_t sa_i, int64_t sa_k, const void *B, int b_dtype,
+                         int64_t sb_k, int64_t sb_j, float *D, int64_t ldd, cudaStream_t stream)
+{
+    if (M <= 0 || N <= 0) return cudaSuccess;
+    dim3 grid((N + SG_BN - 1) / SG_BN, (M + SG_BM - 1) / SG_BM);
+    if (b_dtype == TSR_BF16)
+        simt_gemm_kernel<float, bf16, SIMT_STORE><<<grid, 256, 0, stream>>>(M, N, K, A, sa_i, sa_k, (const bf16 *)B, sb_k, sb_j,
+                                                                           D, ldd, 0.f, 0.f);
+    else
+        simt_gemm_kernel<float, float, SIMT_STORE><<<grid, 256, 0, stream>>>(M, N, K, A, sa_i, sa_k, (const float *)B, sb_k,
+                                                                            sb_j, D, ldd, 0.f, 0.f);
+    return cudaGetLastError();
+}
+
 cudaError_t simt_gemm(int M, int N, int K, const void *A, int a_dtype, int64_t sa_i, int64_t sa_k, const float *B,
                       int64_t sb_k, int64_t sb_j, float *D, int64_t ldd, int epilogue, float decay, float step_scale,
                       cudaStream_t stream)
@@ -114,8 +129,8 @@ cudaError_t simt_gemm(int M, int N, int K, const void *A, int a_dtype, int64_t s
     if (M <= 0 || N <= 0) return cudaSuccess;
     dim3 grid((N + SG_BN - 1) / SG_BN, (M + SG_BM - 1) / SG_BM);
 #define TSR_SG(TA_, EPI_)                                                                                              \
-    simt_gemm_kernel<TA_, EPI_><<<grid, 256, 0, stream>>>(M, N, K, (const TA_ *)A, sa_i, sa_k, B, sb_k, sb_j, D, ldd, decay, \
-                                                           step_scale)
+    simt_gemm_kernel<TA_, float, EPI_><<<grid, 256, 0, stream>>>(M, N, K, (const TA_ *)A, sa_i, sa_k, B, sb_k, sb_j, D, ldd, \
+                                                                  decay, step_scale)
     if (a_dtype == TSR_BF16) {
         if (epilogue == SIMT_APPLY) TSR_SG(bf16, SIMT_APPLY);
         else if (epilogue == SIMT_APPLY_BF16) TSR_SG(bf16, SIMT_APPLY_BF16);
@@ -144,9 +159,9 @@ __global__ void __launch_bounds__(256)
 core_update_kernel(const CoreUpdateArgs *__restrict__ args, const int32_t *__restrict__ list, StepScalars sc, int mode)
 {
     const CoreUpdateArgs a = args[list[blockIdx.z]];
-    const int r = a.r;
+    const int r = a.r, nc = a.nc;   // rows, columns of the core (square except for a one-sided block)
     const int r0 = blockIdx.y * 32;
-    if (r0 >= r || blockIdx.x * 32 * CU_TILES >= r) return;
+    if (r0 >= r || blockIdx.x * 32 * CU_TILES >= nc) return;
     __shared__ float tile[CU_TILES][32][33];
     const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
     const bool sgd = (sc.rule == TSR_RULE_SGD);
@@ -158,8 +173,8 @@ core_update_kernel(const CoreUpdateArgs *__restrict__ args, const int32_t *__res
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
             const int row = r0 + ty + 8 * u;
-            const bool in = (row < r && col < r);
-            const int64_t e = (int64_t)row * r + col;
+            const bool in = (row < r && col < nc);
+            const int64_t e = (int64_t)row * nc + col;
             c[u] = in ? a.C[e] : 0.f;
             if (in && a.nsplit > 1)
                 for (int s = 1; s < a.nsplit; ++s) c[u] = __fadd_rn(c[u], a.C[e + (int64_t)s * a.split_stride]);
@@ -169,8 +184,8 @@ core_update_kernel(const CoreUpdateArgs *__restrict__ args, const int32_t *__res
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
             const int row = r0 + ty + 8 * u;
-            const bool in = (row < r && col < r);
-            const int64_t e = (int64_t)row * r + col;
+            const bool in = (row < r && col < nc);
+            const int64_t e = (int64_t)row * nc + col;
             float d = 0.f;
             if (in) {
                 if (a.nsplit > 1) a.Cout[e] = c[u];
@@ -192,17 +207,17 @@ core_update_kernel(const CoreUpdateArgs *__restrict__ args, const int32_t *__res
         const int c0 = (blockIdx.x * CU_TILES + tt) * 32;
         for (int i = ty; i < 32; i += 8) {
             const int col = c0 + i, row = r0 + tx;
-            if (row < r && col < r) a.dt_bf16[(int64_t)col * a.ldd + row] = __float2bfloat16_rn(tile[tt][tx][i]);
+            if (row < r && col < nc) a.dt_bf16[(int64_t)col * a.ldd + row] = __float2bfloat16_rn(tile[tt][tx][i]);
         }
     }
 }
 
 cudaError_t core_update_launch(const CoreUpdateArgs *args_dev, const int32_t *list_dev, int nblocks, int max_r,
-                               const StepScalars &sc, int mode, cudaStream_t stream)
+                               int max_cols, const StepScalars &sc, int mode, cudaStream_t stream)
 {
     if (nblocks <= 0) return cudaSuccess;
-    const int t = (max_r + 31) / 32;
-    core_update_kernel<<<dim3((t + CU_TILES - 1) / CU_TILES, t, nblocks), 256, 0, stream>>>(args_dev, list_dev, sc, mode);
+    const int t = (max_r + 31) / 32, tc = (max_cols + 31) / 32;
+    core_update_kernel<<<dim3((tc + CU_TILES - 1) / CU_TILES, t, nblocks), 256, 0, stream>>>(args_dev, list_dev, sc, mode);
     return cudaGetLastError();
 }
 

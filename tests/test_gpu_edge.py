@@ -37,6 +37,36 @@ def test_refresh_small_and_extreme_shapes(dtype, shape, gap):
     check_refresh(plan, 0, G64, to64(Om), shape["r"], shape["q"], gap, tol_sub=tol_sub)
 
 
+@pytest.mark.parametrize("dtype,shape", [
+    (torch.float32, dict(m=200, n=176, r=32)),
+    (torch.bfloat16, dict(m=288, n=320, r=48)),
+])
+def test_exact_svd_arm_matches_the_dense_svd(dtype, shape):
+    """The exact-SVD refresh arm of the ablation (Section 3.5 names it as the costly alternative the
+    randomized refresh replaces) is the same refresh with a sketch as wide as the matrix is small
+    (k = min(m, n), no power iteration): the sketch then spans the whole range of G, B = Q^T G loses
+    nothing, and U, V are the leading singular vectors of G itself.  Checked against the oracle's
+    dense SVD of G: singular values, and the projectors on the signal directions."""
+    tsr = _tsr()
+    r = shape["r"]
+    k = min(shape["m"], shape["n"])
+    full = dict(shape, p=k - r, q=0)
+    plan = tsr.Plan([full], g_dtype=dtype)
+    G64 = fill_gradient(plan, 0, 57, signal_rank=r)
+    Om = ti.omega(shape["n"], k, 58).cuda()
+    plan.init_subspace(omegas=[Om])
+    torch.cuda.synchronize()
+    assert plan.poll_status() == [0]
+    Ue, Ve, Se = oracle.exact_svd_refresh(G64, r)
+    U, V = to64(plan.U[0]), to64(plan.V[0])
+    core = U.T @ G64 @ V
+    assert np.abs(np.diag(core) / Se[:r] - 1).max() < 1e-4
+    assert np.abs(core - np.diag(np.diag(core))).max() < 1e-4 * Se[0]
+    assert np.linalg.norm(proj(U) - proj(Ue)) < 1e-3
+    assert np.linalg.norm(proj(V) - proj(Ve)) < 1e-3
+    assert np.linalg.norm(U.T @ U - np.eye(r)) < 1e-4 and np.linalg.norm(V.T @ V - np.eye(r)) < 1e-4
+
+
 def test_refresh_with_repeated_singular_values():
     """Groups of equal singular values and a flat tail: the Gram matrix of the sketch has repeated
     eigenvalues, which the divide-and-conquer eigen-solver must deflate (rotations between nearly

@@ -419,3 +419,63 @@ def test_step_from_host_buffers(copies):
             assert torch.equal(c_host[off:off + s["r"] ** 2].view(s["r"], s["r"]), ref.C[i].cpu())
             off += s["r"] ** 2
     assert plan.poll_status() == [0] * nb
+
+
+# ---- the one-sided arm of the comparison (Table 1: synchronized object C = U^T G, r x n) ----------
+ONE_SIDED_F32 = [dict(m=200, n=330, r=24, flags=2), dict(m=70, n=65, r=8), dict(m=96, n=40, r=16, flags=2)]
+ONE_SIDED_BF16 = [dict(m=256, n=384, r=64, flags=2), dict(m=200, n=328, r=40), dict(m=640, n=520, r=256, flags=2),
+                  dict(m=1000, n=136, r=16, flags=2)]
+
+
+@pytest.mark.parametrize("dtype,shapes,tol", [(torch.float32, ONE_SIDED_F32, TOL_F32),
+                                              (torch.bfloat16, ONE_SIDED_BF16, TOL_BF16)])
+@pytest.mark.parametrize("fuse", [False, True])
+def test_one_sided_arm_matches_oracle(dtype, shapes, tol, fuse):
+    """Blocks flagged one-sided keep an r x n core: C = U^T G, moments and D in that space,
+    W <- (1 - lr wd) W - lr scale U D.  Two-sided blocks of the same plan are unaffected."""
+    tsr, plan = _plan(shapes, dtype)
+    nb = len(shapes)
+    _given_bases(plan, shapes, seed0=640)
+    wd, scale = 0.05, 0.5
+    W, M, Vm, two = [], [], [], {}
+    for i, s in enumerate(shapes):
+        W0 = fill_weights(plan, i, ti.seed_for(93, i, 0, ti.ROLE_WEIGHT))
+        if s.get("flags", 0) & 2:
+            assert tuple(plan.C[i].shape) == (s["r"], s["n"])
+            W.append(W0.copy()); M.append(np.zeros((s["r"], s["n"]))); Vm.append(np.zeros((s["r"], s["n"])))
+        else:
+            ob = oracle.OracleBlock(W0, s["r"], 0, 0, 0)
+            ob.set_bases(to64(plan.U[i]), to64(plan.V[i]))
+            two[i] = ob
+            W.append(None); M.append(None); Vm.append(None)
+    U64 = [to64(plan.U[i]) for i in range(nb)]
+    worst = {"C": 0.0, "M": 0.0, "Vm": 0.0, "W": 0.0}
+    for t in range(1, 6):
+        G64 = [fill_gradient(plan, i, ti.seed_for(93, i, t, ti.ROLE_GRAD)) for i in range(nb)]
+        h = tsr.make_hyper(t, lr=1e-3, weight_decay=wd, scale=scale)
+        if fuse:
+            plan.step(h, fuse_adam=True)
+        else:
+            plan.project_core()
+            plan.adam_core_step(h)
+            plan.backproject_apply(h)
+        torch.cuda.synchronize()
+        for i in range(nb):
+            if i in two:
+                ob = two[i]
+                ob.step(G64[i], weight_decay=f32(wd), scale=f32(scale), **HYPER)
+                ref = (ob.C, ob.M, ob.Vm, ob.W)
+            else:
+                C = oracle.project_one_sided(G64[i], U64[i])
+                D = oracle.adam_core(C, M[i], Vm[i], HYPER["beta1"], HYPER["beta2"], HYPER["eps"], t)
+                oracle.backproject_one_sided(U64[i], D, W[i], HYPER["lr"], f32(wd), f32(scale))
+                ref = (C, M[i], Vm[i], W[i])
+            got = (plan.C[i], plan.M[i], plan.Vm[i], plan.W[i])
+            for key, g, e in zip(("C", "M", "Vm", "W"), got, ref):
+                worst[key] = max(worst[key], rel_fro(to64(g), e))
+    assert plan.poll_status() == [0] * nb
+    for key, val in worst.items():
+        assert val < tol, (key, val, worst)
+    # bytes a worker would synchronize: r n for the one-sided blocks, r^2 for the others (Table 1)
+    core, _ = plan.comm_bytes(1, 4)
+    assert core == 4 * sum(s["r"] * (s["n"] if s.get("flags", 0) & 2 else s["r"]) for s in shapes)

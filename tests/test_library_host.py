@@ -67,8 +67,10 @@ def test_create_validates_shapes(tsr):
 
 def test_block_flags_are_validated_and_sized(tsr):
     D = tsr.MatDesc
-    rc, ctx = _create(tsr, [D(64, 64, 64, 64, 8, 0, 0, 0, 0, 0, 0, 2)])          # unknown flag bit
+    rc, ctx = _create(tsr, [D(64, 64, 64, 64, 8, 0, 0, 0, 0, 0, 0, 4)])          # unknown flag bit
     assert rc == 1
+    rc, ctx = _create(tsr, [D(64, 64, 64, 64, 8, 0, 0, 0, 0, 0, 0, 3)])          # one-sided with re-expressed moments
+    assert rc == 6
     sizes = []
     for flags in (0, tsr.TSR_BLOCK_REEXPRESS_MOMENT):
         rc, ctx = _create(tsr, [D(256, 320, 320, 320, 32, 8, 1, 0, 0, 0, 0, flags)])
@@ -78,6 +80,22 @@ def test_block_flags_are_validated_and_sized(tsr):
         sizes.append(rb.value)
         tsr.lib().tsr_destroy(ctx)
     assert sizes[1] - sizes[0] >= 4 * ((256 + 320) * 32 + 3 * 32 * 32)             # old bases + three r x r scratch
+
+
+def test_one_sided_block_accounting(tsr):
+    """Table 1: a one-sided block synchronizes C = U^T G, r n elements instead of r^2, and keeps
+    U plus two r x n moments."""
+    D = tsr.MatDesc
+    m, n, r = 256, 320, 32
+    rc, ctx = _create(tsr, [D(m, n, n, n, r, 8, 1, 0, 1, 0, 0, tsr.TSR_BLOCK_ONE_SIDED), D(m, n, n, n, r, 8, 1, 0, 1, 0, 0, 0)])
+    assert rc == 0
+    L = tsr.lib()
+    core, sk, el = ctypes.c_uint64(), ctypes.c_uint64(), ctypes.c_uint64()
+    assert L.tsr_comm_bytes(ctx, 1, 4, ctypes.byref(core), ctypes.byref(sk)) == 0
+    assert core.value == 4 * (r * n + r * r)
+    assert L.tsr_state_elems(ctx, ctypes.byref(el)) == 0
+    assert el.value == (m * r + 2 * r * n) + ((m + n) * r + 2 * r * r)
+    L.tsr_destroy(ctx)
 
 
 def test_compute_before_bind_is_refused(tsr):

@@ -50,6 +50,49 @@ def test_identity_bases_reduce_to_torch_adamw(wd, scale):
     assert blk.t == 11
 
 
+# ---- the one-sided arm (Table 1) with U = I is the same textbook AdamW; rectangular on purpose
+@pytest.mark.parametrize("wd", [0.0, 0.1])
+def test_one_sided_arm_with_identity_basis_reduces_to_torch_adamw(wd):
+    m, n = 7, 12
+    rng = np.random.default_rng(21)
+    W = rng.standard_normal((m, n)) * 0.02
+    M, Vm = np.zeros((m, n)), np.zeros((m, n))
+    w = torch.tensor(W, dtype=torch.float64, requires_grad=True)
+    opt = torch.optim.AdamW([w], lr=1e-2, betas=(0.9, 0.999), eps=1e-8, weight_decay=wd)
+    for t in range(1, 9):
+        G = rng.standard_normal((m, n))
+        C = oracle.project_one_sided(G, np.eye(m))
+        D = oracle.adam_core(C, M, Vm, 0.9, 0.999, 1e-8, t)
+        oracle.backproject_one_sided(np.eye(m), D, W, lr=1e-2, weight_decay=wd)
+        w.grad = torch.tensor(G, dtype=torch.float64)
+        opt.step()
+        assert np.abs(W - w.detach().numpy()).max() < 1e-14
+
+
+def test_one_sided_lift_invariants_and_closed_form():
+    m, n, r = 30, 44, 6
+    U = _rand_orth(m, r, 31)
+    rng = np.random.default_rng(32)
+    D = rng.standard_normal((r, n))
+    W0 = rng.standard_normal((m, n))
+    W = np.zeros((m, n))
+    oracle.backproject_one_sided(U, D, W, lr=1.0)               # W = -U D
+    assert np.abs(U.T @ (-W) - D).max() < 1e-12                  # U^T dW = D
+    assert np.abs(U @ U.T @ W - W).max() < 1e-12                 # dW lives in range(U)
+    W = W0.copy()
+    oracle.backproject_one_sided(U, D, W, lr=0.3, weight_decay=0.2, scale=0.5)
+    assert np.allclose(W, (1 - 0.3 * 0.2) * W0 - 0.3 * 0.5 * (U @ D), atol=1e-13)
+    # a two-sided step whose right basis spans everything is the one-sided step: V = I_n needs the
+    # square core D V^T = D, which the two-sided routine takes when r = n
+    Usq = _rand_orth(n, n, 33)
+    Dsq = rng.standard_normal((n, n))
+    Wa, Wb = rng.standard_normal((n, n)), None
+    Wb = Wa.copy()
+    oracle.backproject_apply(Usq, Dsq, np.eye(n), Wa, lr=0.1, weight_decay=0.05, scale=2.0)
+    oracle.backproject_one_sided(Usq, Dsq, Wb, lr=0.1, weight_decay=0.05, scale=2.0)
+    assert np.abs(Wa - Wb).max() < 1e-12
+
+
 def test_scale_multiplies_lifted_update_only():
     # with U = V = I the step is W - lr*(scale*D + wd*W); check against AdamW run with lr*scale
     # for the update part and decoupled decay lr*wd for the decay part (t = 1, closed form).
