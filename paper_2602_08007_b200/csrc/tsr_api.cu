@@ -17,7 +17,7 @@ namespace {
 
 // KR*: tall-times-small products of the refresh on tensor cores (three TF32 products): rows of side
 // 0 (m) or 1 (n) times R^{-1} into buf[1] / buf[2], and the final U = Q Wu, V = B^T Wv.
-enum Kind : int { KT = 0, KC, KCS, KP, KA, KY, KZ, KR01, KR02, KR12, KRU, KRV, KO, KOA, NKIND };
+enum Kind : int { KT = 0, KC, KP, KA, KY, KZ, KR01, KR02, KR12, KRU, KRV, KO, KOA, NKIND };
 constexpr int TSR_NUM_STAGES = 6;  // refresh, G*V, core GEMM, core update, U*D, apply
 
 struct Block {
@@ -95,7 +95,7 @@ struct tsr_ctx {
     int max_r = 0, max_k = 0;
     uint64_t launches = 0;                     // kernels launched through this context
     int num_sms = 148;
-    int bn[NKIND] = {128, 128, 128, 128, 128, 128, 128, 256, 256, 256, 256, 256, 128, 128};   // tile width of each GEMM kind
+    int bn[NKIND] = {128, 128, 128, 128, 128, 128, 256, 256, 256, 256, 256, 128, 128};   // tile width of each GEMM kind
     bool profiling = false;
     cudaEvent_t ev[TSR_NUM_STAGES + 1] = {};   // stage boundaries of the last step (profiling only)
     bool ev_valid = false;
@@ -279,7 +279,7 @@ void build_tiles(tsr_ctx *ctx)
     for (const Block &b : ctx->blocks) if (b.fast) rmax = std::max(rmax, (int)b.d.r);
     for (int kd : {KT, KP}) ctx->bn[kd] = rmax >= 256 ? 256 : 128;
     // the core GEMM has few, long tiles: 256-wide tiles only pay once r reaches 512 (measured)
-    for (int kd : {KC, KCS}) ctx->bn[kd] = rmax >= 512 ? 256 : 128;
+    ctx->bn[KC] = rmax >= 512 ? 256 : 128;
     // apply: 256-wide tiles halve the P traffic per byte of W, which pays once the operands are as wide
     // as r = 512 (measured 2.28 -> 2.05 ms on the 1B set; at r = 256 the narrow tile is faster)
     ctx->bn[KA] = rmax >= 512 ? 256 : 128;
@@ -297,8 +297,9 @@ void build_tiles(tsr_ctx *ctx)
             add_tiles(ctx, KOA, bi, m, n, r, 0);
         } else {
             add_tiles(ctx, KT, bi, m, r, n, 0);
-            if (b.nsplit > 1) add_tiles(ctx, KCS, bi, r, r, m, b.kb_per_split);
-            else add_tiles(ctx, KC, bi, r, r, m, 0);
+            // a block with a long contraction (an embedding) is cut into split-K slabs; its tiles sit in the same
+            // table, so that one launch covers every block
+            add_tiles(ctx, KC, bi, r, r, m, b.nsplit > 1 ? b.kb_per_split : 0);
             add_tiles(ctx, KP, bi, m, r, r, 0);
             add_tiles(ctx, KA, bi, m, n, r, 0);
         }
@@ -485,7 +486,6 @@ tsr_status do_project(tsr_ctx *ctx, const std::vector<int> &list, bool fuse, con
         if ((s = launch_kind(ctx, KT, list, EPI_STORE_BF16_T, 1, sc, st)) != TSR_OK) return s;
         mark_stage(ctx, 2);
         if ((s = launch_kind(ctx, KC, list, fuse ? EPI_CORE_UPDATE : EPI_STORE_F32, 1, sc, st)) != TSR_OK) return s;
-        if ((s = launch_kind(ctx, KCS, list, EPI_STORE_F32, 1, sc, st)) != TSR_OK) return s;
         // one-sided blocks: C = U^T G needs the gradient with m as the contiguous index
         bool any_one_sided = false;
         for (int bi : list) {
@@ -1064,12 +1064,13 @@ tsr_status tsr_bind(tsr_ctx *ctx, const tsr_mat_ptrs *ptrs, int32_t count, void 
             if ((s = encode_map(ctx, &P.tmB, b.Vbt, r, n, b.nl, ctx->bn[KT] / 2)) != TSR_OK) return s;
             P.out = b.Tt; P.ld_out = b.ml;
         }
-        for (int kd : {KC, KCS}) {   // C = U^T T : A = U^T copy [r x m], B = T~ [r x m]
-            UmmaProblem &P = probs[kd][i];
-            base(P, (int)r, (int)r, (int)m, EPI_CORE_UPDATE);
+        {   // C = U^T T : A = U^T copy [r x m], B = T~ [r x m].  A split-K block only stores its slabs
+            // (the sum and the core update follow in core_update_kernel), whatever epilogue the launch has.
+            UmmaProblem &P = probs[KC][i];
+            base(P, (int)r, (int)r, (int)m, b.nsplit > 1 ? EPI_STORE_F32 : EPI_CORE_UPDATE);
             if ((s = encode_map(ctx, &P.tmA, b.Ubt, r, m, b.ml, 128)) != TSR_OK) return s;
-            if ((s = encode_map(ctx, &P.tmB, b.Tt, r, m, b.ml, ctx->bn[kd] / 2)) != TSR_OK) return s;
-            P.out = (kd == KC) ? (void *)b.p.C : (void *)b.partial;
+            if ((s = encode_map(ctx, &P.tmB, b.Tt, r, m, b.ml, ctx->bn[KC] / 2)) != TSR_OK) return s;
+            P.out = (b.nsplit > 1) ? (void *)b.partial : (void *)b.p.C;
             P.ld_out = r; P.split_stride = r * r;
             P.mom1 = b.p.M; P.mom2 = b.p.Vm; P.d_bf16 = nullptr; P.dt_bf16 = b.Dbt; P.ldd = b.rl;
         }

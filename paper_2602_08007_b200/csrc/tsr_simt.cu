@@ -156,18 +156,21 @@ cudaError_t simt_gemm(int M, int N, int K, const void *A, int a_dtype, int64_t s
 constexpr int CU_TILES = 4;
 
 __global__ void __launch_bounds__(256)
-core_update_kernel(const CoreUpdateArgs *__restrict__ args, const int32_t *__restrict__ list, StepScalars sc, int mode)
+core_update_kernel(const CoreUpdateArgs *__restrict__ args, const int32_t *__restrict__ list, StepScalars sc, int mode,
+                   int ntile)
 {
+    // ntile (1 .. CU_TILES) tiles of 32 x 32 per CTA: small launches take one, so that more CTAs share the work
     const CoreUpdateArgs a = args[list[blockIdx.z]];
     const int r = a.r, nc = a.nc;   // rows, columns of the core (square except for a one-sided block)
     const int r0 = blockIdx.y * 32;
-    if (r0 >= r || blockIdx.x * 32 * CU_TILES >= nc) return;
+    if (r0 >= r || blockIdx.x * 32 * ntile >= nc) return;
     __shared__ float tile[CU_TILES][32][33];
     const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
     const bool sgd = (sc.rule == TSR_RULE_SGD);
 #pragma unroll
     for (int tt = 0; tt < CU_TILES; ++tt) {
-        const int c0 = (blockIdx.x * CU_TILES + tt) * 32;
+        if (tt >= ntile) break;
+        const int c0 = (blockIdx.x * ntile + tt) * 32;
         const int col = c0 + tx;
         float c[4], m1[4], m2[4];
 #pragma unroll
@@ -176,8 +179,17 @@ core_update_kernel(const CoreUpdateArgs *__restrict__ args, const int32_t *__res
             const bool in = (row < r && col < nc);
             const int64_t e = (int64_t)row * nc + col;
             c[u] = in ? a.C[e] : 0.f;
-            if (in && a.nsplit > 1)
-                for (int s = 1; s < a.nsplit; ++s) c[u] = __fadd_rn(c[u], a.C[e + (int64_t)s * a.split_stride]);
+            if (in && a.nsplit > 1) {
+                // slabs are added in slab order; eight loads are in flight at a time
+                for (int s0 = 1; s0 < a.nsplit; s0 += 8) {
+                    float part[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) part[j] = (s0 + j < a.nsplit) ? a.C[e + (int64_t)(s0 + j) * a.split_stride] : 0.f;
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        if (s0 + j < a.nsplit) c[u] = __fadd_rn(c[u], part[j]);
+                }
+            }
             m1[u] = (in && mode == 0) ? a.mom1[e] : 0.f;
             m2[u] = (in && mode == 0 && !sgd) ? a.mom2[e] : 0.f;
         }
@@ -204,7 +216,8 @@ core_update_kernel(const CoreUpdateArgs *__restrict__ args, const int32_t *__res
     __syncthreads();
 #pragma unroll
     for (int tt = 0; tt < CU_TILES; ++tt) {
-        const int c0 = (blockIdx.x * CU_TILES + tt) * 32;
+        if (tt >= ntile) break;
+        const int c0 = (blockIdx.x * ntile + tt) * 32;
         for (int i = ty; i < 32; i += 8) {
             const int col = c0 + i, row = r0 + tx;
             if (row < r && col < nc) a.dt_bf16[(int64_t)col * a.ldd + row] = __float2bfloat16_rn(tile[tt][tx][i]);
@@ -217,7 +230,8 @@ cudaError_t core_update_launch(const CoreUpdateArgs *args_dev, const int32_t *li
 {
     if (nblocks <= 0) return cudaSuccess;
     const int t = (max_r + 31) / 32, tc = (max_cols + 31) / 32;
-    core_update_kernel<<<dim3((tc + CU_TILES - 1) / CU_TILES, t, nblocks), 256, 0, stream>>>(args_dev, list_dev, sc, mode);
+    const int ntile = ((int64_t)t * tc * nblocks >= 4 * 148 * CU_TILES) ? CU_TILES : 1;
+    core_update_kernel<<<dim3((tc + ntile - 1) / ntile, t, nblocks), 256, 0, stream>>>(args_dev, list_dev, sc, mode, ntile);
     return cudaGetLastError();
 }
 

@@ -189,7 +189,9 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
             const uint32_t buf = tc & 1u;
             const int N = P->N, M = P->M;
             const int row0 = tile.m0 + (int)rank * UM_BM + q * 32;   // this CTA holds rows 128 rank .. of the tile
-            if (EPI == EPI_CORE_UPDATE) {
+            // a split-K problem inside a core-update launch only stores its slab
+            const bool store_f32 = (EPI == EPI_STORE_F32) || (EPI == EPI_CORE_UPDATE && P->epilogue == EPI_STORE_F32);
+            if (EPI == EPI_CORE_UPDATE && !store_f32) {
                 // pull this warp's slice of the moments towards L2 while the MMAs of the tile run
                 const int prow = row0 + lane;
                 if (prow < M) {
@@ -236,7 +238,7 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
                 // Fast paths (full 32 x 32 chunk): transpose through the warp's patch so that lane = column;
                 // every global access is then one full row segment (128 bytes of FP32, 64 of BF16).
                 const bool full_chunk = (ncols == 32) && (nrows == 32);
-                if (EPI == EPI_STORE_F32 && ncols == 32 && (P->ld_out & 3) == 0 && (col0 & 3) == 0 &&
+                if (store_f32 && ncols == 32 && (P->ld_out & 3) == 0 && (col0 & 3) == 0 &&
                     (((uintptr_t)P->out) & 15) == 0 && (P->split_stride & 3) == 0) {
                     // lane = row: each lane writes 128 contiguous bytes of its own row
                     if (lane < nrows) {
@@ -338,7 +340,7 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
                 __syncwarp();
                 const int col = col0 + lane;
                 const bool col_ok = lane < ncols;
-                if (EPI == EPI_STORE_F32) {
+                if (store_f32) {
                     float *out = (float *)P->out + (int64_t)tile.split * P->split_stride + (int64_t)row0 * P->ld_out + col;
                     if (col_ok)
                         for (int i = 0; i < nrows; ++i) out[(int64_t)i * P->ld_out] = patch[i * 33 + lane];
