@@ -95,23 +95,44 @@ tridiag_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ li
             }
             if (tid == 0) { d.tau[j] = tau; d.dvec[j] = dj; d.evec[j] = alpha; }
             __syncthreads();
-            // ps = T0[c+1.., c+1..] v   (row-wise dot products; a warp takes four rows at a time so that
-            // four loads are in flight per lane)
+            // ps = T0[c+1.., c+1..] v   (row-wise dot products; a warp takes four rows at a time and four
+            // 32-column segments of each per trip, so that sixteen loads are in flight per lane; the four
+            // sums are then reduced together: two exchange steps leave one sum per group of eight lanes)
             for (int a0 = 4 * warp; a0 < len; a0 += 4 * nwarps) {
                 const double *row0 = A + (int64_t)(j + 1 + a0) * k + j + 1;
                 const int na = min(4, len - a0);
                 double acc[4] = {0.0, 0.0, 0.0, 0.0};
-                for (int b = lane; b < len; b += 32) {
-                    const double vb = vs[b];
+                for (int b0 = 0; b0 < len; b0 += 128) {
+                    double x[4][4], vb[4];
 #pragma unroll
-                    for (int u = 0; u < 4; ++u)
-                        if (u < na) acc[u] += row0[(int64_t)u * k + b] * vb;
+                    for (int q = 0; q < 4; ++q) {
+                        const int b = b0 + 32 * q + lane;
+                        const bool ok = b < len;
+                        vb[q] = ok ? vs[b] : 0.0;
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) x[u][q] = (ok && u < na) ? row0[(int64_t)u * k + b] : 0.0;
+                    }
+#pragma unroll
+                    for (int q = 0; q < 4; ++q)
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) acc[u] += x[u][q] * vb[q];
                 }
+                // lanes with bit 4 set keep sums 2, 3, the others 0, 1; then bit 3 picks one of the two
+                {
+                    const bool hi4 = (lane & 16) != 0;
+                    const double s0 = hi4 ? acc[0] : acc[2], s1 = hi4 ? acc[1] : acc[3];
+                    const double k0 = hi4 ? acc[2] : acc[0], k1 = hi4 ? acc[3] : acc[1];
+                    const double t0 = k0 + __shfl_xor_sync(0xffffffffu, s0, 16);
+                    const double t1 = k1 + __shfl_xor_sync(0xffffffffu, s1, 16);
+                    const bool hi3 = (lane & 8) != 0;
+                    const double snd = hi3 ? t0 : t1, keep = hi3 ? t1 : t0;
+                    double t = keep + __shfl_xor_sync(0xffffffffu, snd, 8);
 #pragma unroll
-                for (int off = 16; off > 0; off >>= 1)
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) acc[u] += __shfl_xor_sync(0xffffffffu, acc[u], off);
-                if (lane < na) ps[a0 + lane] = (lane == 0 ? acc[0] : lane == 1 ? acc[1] : lane == 2 ? acc[2] : acc[3]);
+                    for (int off = 4; off > 0; off >>= 1) t += __shfl_xor_sync(0xffffffffu, t, off);
+                    // lanes 0..7 hold sum 0, 8..15 sum 1, 16..23 sum 2, 24..31 sum 3
+                    const int u = lane >> 3;
+                    if ((lane & 7) == 0 && u < na) ps[a0 + u] = t;
+                }
             }
             // the earlier pairs of the panel against v: one warp per dot product
             if (warp < 2 * c) {
