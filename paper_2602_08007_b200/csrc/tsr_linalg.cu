@@ -158,7 +158,6 @@ cudaError_t gram_batched(const RefreshDev *rd, const RowItem *items, int nitems,
 // ---------------------------------------------------------------------------------------
 constexpr int CH_NB = 16;
 constexpr int CH_THREADS = 512;
-constexpr int CH_U = 2;      // columns per lane and trip in the trailing update
 #ifdef CH_PROFILE
 #define CH_TICK(slot) do { if (threadIdx.x == 0 && blockIdx.x == 0) { const long long t_ = clock64(); ch_prof[slot] += t_ - ch_t0; ch_t0 = t_; } } while (0)
 #else
@@ -168,14 +167,13 @@ constexpr int CH_U = 2;      // columns per lane and trip in the trailing update
 __global__ void __launch_bounds__(CH_THREADS)
 chol_inverse_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ list, int kpad)
 {
-    extern __shared__ __align__(16) double ch_smem[];   // P[CH_NB][kpad]
+    extern __shared__ __align__(16) double ch_smem[];   // P[CH_NB][kpad], then a 16 x 8 patch per warp
     const RefreshDev d = rd[list[blockIdx.x]];
     const int k = d.k;
     double *__restrict__ S = d.S;
     double *__restrict__ X = d.Xw;
     double *P = ch_smem;
     __shared__ double dinv[CH_NB][CH_NB + 1];    // inverse of the current diagonal block (upper triangular)
-    __shared__ double rdiag[CH_NB];              // 1 / R[j][j] of the current diagonal block
     __shared__ double s_floor;
     __shared__ int s_flag;
     const int tid = threadIdx.x, nt = blockDim.x;
@@ -213,51 +211,81 @@ chol_inverse_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict
         }
         __syncthreads();
         CH_TICK(0);
-        if (warp == 0) {                            // the nb x nb diagonal block and its inverse
+        if (warp == 0) {
+            // The nb x nb diagonal block and its inverse, in registers: lane c (< 16) holds column c of the
+            // block; row j of the factor reaches the other lanes by shuffles (all loops unrolled, so every
+            // register index is static).  Lanes 16..31 only take part in the shuffles.
             const double floor_v = s_floor;
-            for (int j = 0; j < nb; ++j) {
-                double v = P[j * kpad + j];
-                if (!(v > floor_v)) {
-                    if (lane == 0 && s_flag == 0) s_flag = TSR_ERR_RANK_DEFICIENT;
-                    v = floor_v;
+            const int c = lane & 15;
+            double col[CH_NB], rinv_d[CH_NB];
+#pragma unroll
+            for (int i = 0; i < CH_NB; ++i) col[i] = (i <= c && c < nb && i < nb) ? P[i * kpad + c] : 0.0;
+            bool floored = false;
+#pragma unroll
+            for (int j = 0; j < CH_NB; ++j) {
+                rinv_d[j] = 0.0;
+                if (j < nb) {                                   // uniform over the warp
+                    double v = __shfl_sync(0xffffffffu, col[j], j);
+                    if (!(v > floor_v)) { floored = true; v = floor_v; }
+                    const double rpiv = rsqrt(v);
+                    const double piv = v * rpiv;
+                    rinv_d[j] = rpiv;
+                    col[j] = (c == j) ? piv : col[j] * rpiv;    // R[j][c] for c >= j (zero for c < j)
+#pragma unroll
+                    for (int i = j + 1; i < CH_NB; ++i) {
+                        const double rji = __shfl_sync(0xffffffffu, col[j], i);   // R[j][i]
+                        col[i] -= rji * col[j];                 // only entries with c >= i are used later
+                    }
                 }
-                const double piv = sqrt(v), rpiv = 1.0 / piv;
-                __syncwarp();
-                if (lane == 0) rdiag[j] = rpiv;
-                if (lane < nb && lane >= j) P[j * kpad + lane] = (lane == j) ? piv : P[j * kpad + lane] * rpiv;
-                __syncwarp();
-                for (int e = lane; e < CH_NB * CH_NB; e += 32) {
-                    const int i = e / CH_NB, c = e % CH_NB;
-                    if (i > j && c >= i && c < nb) P[i * kpad + c] -= P[j * kpad + i] * P[j * kpad + c];
-                }
-                __syncwarp();
             }
-            if (lane < CH_NB) {                     // column `lane` of R11^{-1} by back substitution
-                const int c = lane;
-                for (int i = CH_NB - 1; i >= 0; --i) {
-                    double acc = (i == c) ? 1.0 : 0.0;
-                    for (int l = i + 1; l <= c && l < nb; ++l) acc -= P[i * kpad + l] * dinv[l][c];
-                    const double xi = (i <= c && c < nb) ? acc * rdiag[i] : 0.0;
-                    dinv[i][c] = xi;
+            if (floored && lane == 0 && s_flag == 0) s_flag = TSR_ERR_RANK_DEFICIENT;
+            // column c of R11^{-1} by back substitution; R[i][l] comes from lane l
+            double x[CH_NB];
+#pragma unroll
+            for (int i = CH_NB - 1; i >= 0; --i) {
+                double acc = (i == c) ? 1.0 : 0.0;
+#pragma unroll
+                for (int l = i + 1; l < CH_NB; ++l) {
+                    const double ril = __shfl_sync(0xffffffffu, col[i], l);
+                    if (l <= c) acc -= ril * x[l];
+                }
+                x[i] = (i <= c && c < nb && i < nb) ? acc * rinv_d[i] : 0.0;
+            }
+            if (lane < CH_NB) {
+#pragma unroll
+                for (int i = 0; i < CH_NB; ++i) {
+                    if (i <= c && c < nb) P[i * kpad + c] = col[i];
+                    dinv[i][c] = x[i];
                     if (i < nb && c < nb) {
-                        X[(int64_t)(jb + i) * k + jb + c] = xi;
-                        d.Rinv[(int64_t)(jb + i) * k + jb + c] = (float)xi;
+                        X[(int64_t)(jb + i) * k + jb + c] = x[i];
+                        d.Rinv[(int64_t)(jb + i) * k + jb + c] = (float)x[i];
                     }
                 }
             }
         }
         __syncthreads();
         CH_TICK(1);
-        for (int c = nb + tid; c < w; c += nt) {    // R12 = R11^{-T} S12, one column per thread
-            double sv[CH_NB];
+        {   // R12 = R11^{-T} S12 on the FP64 tensor path: (16 x 16 lower triangular) times 16 x 8 column tiles,
+            // in place (a tile's columns belong to one warp, which reads them before it writes)
+            const int g = lane >> 2, q = lane & 3;
+            for (int c0 = nb + 8 * warp; c0 < w; c0 += 8 * nwarps) {
+                double bfr[4];
 #pragma unroll
-            for (int l = 0; l < CH_NB; ++l) sv[l] = (l < nb) ? P[l * kpad + c] : 0.0;
+                for (int st = 0; st < 4; ++st) bfr[st] = P[(4 * st + q) * kpad + min(c0 + g, w - 1)];
+                double y[2][2] = {{0.0, 0.0}, {0.0, 0.0}};
 #pragma unroll
-            for (int j = 0; j < CH_NB; ++j) {
-                double acc = 0.0;
+                for (int st = 0; st < 4; ++st) {
+                    if (st < 2) dmma_8x8x4(y[0][0], y[0][1], dinv[4 * st + q][g], bfr[st]);   // rows 0..7 end at l = 7
+                    dmma_8x8x4(y[1][0], y[1][1], dinv[4 * st + q][8 + g], bfr[st]);
+                }
+                __syncwarp();
 #pragma unroll
-                for (int l = 0; l <= j; ++l) acc += dinv[l][j] * sv[l];
-                if (j < nb) P[j * kpad + c] = acc;
+                for (int jt = 0; jt < 2; ++jt)
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const int col = c0 + 2 * q + h;
+                        if (col < w) P[(jt * 8 + g) * kpad + col] = y[jt][h];
+                    }
             }
         }
         __syncthreads();
@@ -266,47 +294,65 @@ chol_inverse_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict
             const int j = e / w, c = e - j * w;
             if (c >= j) S[(int64_t)(jb + j) * k + jb + c] = P[j * kpad + c];
         }
-        // rank-nb update of the trailing upper triangle: rows i and i + 1 per warp, CH_U columns per
-        // lane and trip with their loads issued before the arithmetic
-        for (int i = jb + nb + 2 * warp; i < k; i += 2 * nwarps) {
-            const int ci = i - jb;
-            const bool two = (i + 1 < k);
-            double r0[CH_NB], r1[CH_NB];
+        CH_TICK(8);
+        // rank-nb update of the trailing upper triangle on the FP64 tensor path: S22 -= R12^T R12 in
+        // 8 x 8 tiles (mma m8n8k4, four steps over the 16 panel rows).  A warp owns the row tiles
+        // warp, warp + nwarps, ... and takes eight column tiles per trip, all their loads issued
+        // before the first product (the update is bound by the latency of those loads).  Tiles that
+        // straddle the diagonal are updated whole: entries below the diagonal are never read.
+        if (nb == CH_NB) {
+            const int g = lane >> 2, q = lane & 3;
+            const int nt8 = (k + 7) >> 3;
+            const bool k_even = (k & 1) == 0;   // then every pair (l, l + 1) with l even is 16-byte aligned and inside the row
+            for (int ti = ((jb + CH_NB) >> 3) + warp; ti < nt8; ti += nwarps) {
+                const int row = ti * 8 + g;
+                const bool row_ok = row < k;
+                double af[4];
 #pragma unroll
-            for (int j = 0; j < CH_NB; ++j) {
-                r0[j] = (j < nb) ? P[j * kpad + ci] : 0.0;
-                r1[j] = (j < nb && two) ? P[j * kpad + ci + 1] : 0.0;
-            }
-            double *row0 = S + (int64_t)i * k, *row1 = S + (int64_t)(i + 1) * k;
-            for (int lb = i + lane; lb < k; lb += 32 * CH_U) {
-                double s0[CH_U], s1[CH_U], a0[CH_U], a1[CH_U];
+                for (int st = 0; st < 4; ++st) af[st] = P[(4 * st + q) * kpad + min(row, k - 1) - jb];
+                double *srow = S + (int64_t)min(row, k - 1) * k;
+                double cv[8][2], nv[8][2];
+                auto cload = [&](int tj0, double (&v)[8][2]) {
 #pragma unroll
-                for (int u = 0; u < CH_U; ++u) {
-                    const int l = lb + 32 * u;
-                    s0[u] = (l < k) ? row0[l] : 0.0;
-                    s1[u] = (two && l < k && l > i) ? row1[l] : 0.0;
-                    a0[u] = 0.0; a1[u] = 0.0;
-                }
-#pragma unroll
-                for (int j = 0; j < CH_NB; ++j) {
-#pragma unroll
-                    for (int u = 0; u < CH_U; ++u) {
-                        const int cl = min(lb + 32 * u, k - 1) - jb;
-                        const double pj = P[j * kpad + cl];
-                        a0[u] += r0[j] * pj;
-                        a1[u] += r1[j] * pj;
+                    for (int u = 0; u < 8; ++u) {
+                        const int l = (tj0 + u) * 8 + 2 * q;
+                        if (k_even) {   // both entries as one 16-byte access: half as many cache-line visits
+                            const double2 t = (row_ok && l < k) ? *(const double2 *)(srow + l) : make_double2(0.0, 0.0);
+                            v[u][0] = t.x; v[u][1] = t.y;
+                        } else {
+                            v[u][0] = (row_ok && l < k) ? srow[l] : 0.0;
+                            v[u][1] = (row_ok && l + 1 < k) ? srow[l + 1] : 0.0;
+                        }
                     }
-                }
+                };
+                cload(ti, cv);
+                for (int tj0 = ti; tj0 < nt8; tj0 += 8) {
+                    cload(tj0 + 8, nv);              // the next trip's tiles are in flight during this trip's products
 #pragma unroll
-                for (int u = 0; u < CH_U; ++u) {
-                    const int l = lb + 32 * u;
-                    if (l < k) {
-                        row0[l] = s0[u] - a0[u];
-                        if (two && l > i) row1[l] = s1[u] - a1[u];
+                    for (int u = 0; u < 8; ++u) {
+                        if (tj0 + u < nt8) {
+                            double a0 = 0.0, a1 = 0.0, b0 = 0.0, b1 = 0.0;   // two chains of two products each
+#pragma unroll
+                            for (int st = 0; st < 4; ++st) {
+                                const double bfr = P[(4 * st + q) * kpad + min((tj0 + u) * 8 + g, k - 1) - jb];
+                                if (st & 1) dmma_8x8x4(b0, b1, af[st], bfr);
+                                else dmma_8x8x4(a0, a1, af[st], bfr);
+                            }
+                            const int l = (tj0 + u) * 8 + 2 * q;
+                            if (k_even) {
+                                if (row_ok && l < k) *(double2 *)(srow + l) = make_double2(cv[u][0] - (a0 + b0), cv[u][1] - (a1 + b1));
+                            } else {
+                                if (row_ok && l < k) srow[l] = cv[u][0] - (a0 + b0);
+                                if (row_ok && l + 1 < k) srow[l + 1] = cv[u][1] - (a1 + b1);
+                            }
+                        }
                     }
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) { cv[u][0] = nv[u][0]; cv[u][1] = nv[u][1]; }
                 }
             }
         }
+        CH_TICK(9);
         __syncthreads();
         CH_TICK(3);
     }
@@ -326,40 +372,67 @@ chol_inverse_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict
         }
         __syncthreads();
         CH_TICK(4);
-        for (int c = l0 + tid; c < k; c += nt) {
-            double acc[CH_NB];
+        {   // acc = R[I][l0 ..] X[l0 .., c] on the FP64 tensor path: a warp owns 16 x 8 tiles of columns
+            // (two mma row tiles) and runs over l in steps of four; X is zero below its diagonal, so the
+            // sum stops at the last column of the tile.  Eight steps of X values are in flight per lane.
+            const int g = lane >> 2, q = lane & 3;
+            const int nct = (k - l0 + 7) >> 3;
+            double *patch = ch_smem + CH_NB * kpad + warp * 128;    // 16 x 8, private to the warp
+            for (int ct = warp; ct < nct; ct += nwarps) {
+                const int c0 = l0 + ct * 8;
+                const int cg = min(c0 + g, k - 1);                  // columns past k - 1 are computed and dropped
+                const int lend = min(c0 + 8, k);
+                double lo0 = 0.0, lo1 = 0.0, hi0 = 0.0, hi1 = 0.0;
+                auto bload = [&](int l) -> double {
+                    const int row = l + q;
+                    return (row < lend) ? X[(int64_t)row * k + cg] : 0.0;
+                };
+                double bq[8], nq[8];
 #pragma unroll
-            for (int j = 0; j < CH_NB; ++j) acc[j] = 0.0;
-            // rows l0 .. c of X four at a time (X is zero below its diagonal, so a group may reach past
-            // row c); the next group is fetched while the current one is used
-            auto xload = [&](int l) -> double { return (l < k) ? X[(int64_t)l * k + c] : 0.0; };
-            int l = l0;
-            double x0 = xload(l), x1 = xload(l + 1), x2 = xload(l + 2), x3 = xload(l + 3);
-            for (; l <= c; l += 4) {
-                const int ln = l + 4;
-                double n0 = 0.0, n1 = 0.0, n2 = 0.0, n3 = 0.0;
-                if (ln <= c) { n0 = xload(ln); n1 = xload(ln + 1); n2 = xload(ln + 2); n3 = xload(ln + 3); }
+                for (int pp = 0; pp < 8; ++pp) bq[pp] = bload(l0 + 4 * pp);
+                for (int l = l0; l < lend; l += 32) {
 #pragma unroll
-                for (int j = 0; j < CH_NB; ++j) {
-                    const double2 ra = *(const double2 *)&P[j * kpad + l];
-                    const double2 rb = *(const double2 *)&P[j * kpad + l + 2];
-                    acc[j] += (ra.x * x0 + ra.y * x1) + (rb.x * x2 + rb.y * x3);
+                    for (int pp = 0; pp < 8; ++pp) nq[pp] = bload(l + 32 + 4 * pp);
+#pragma unroll
+                    for (int pp = 0; pp < 8; ++pp) {
+                        const int ll = l + 4 * pp;
+                        if (ll < lend) {
+                            const double a_lo = P[g * kpad + ll + q], a_hi = P[(8 + g) * kpad + ll + q];
+                            dmma_8x8x4(lo0, lo1, a_lo, bq[pp]);
+                            dmma_8x8x4(hi0, hi1, a_hi, bq[pp]);
+                        }
+                    }
+#pragma unroll
+                    for (int pp = 0; pp < 8; ++pp) bq[pp] = nq[pp];
                 }
-                x0 = n0; x1 = n1; x2 = n2; x3 = n3;
-            }
-            CH_TICK(5);
-            // X[I][c] = -R11^{-1} acc
+                CH_TICK(5);
+                // X[I][c] = -R11^{-1} acc: the tile goes through the patch to become the B operand
+                patch[g * 8 + 2 * q] = lo0; patch[g * 8 + 2 * q + 1] = lo1;
+                patch[(8 + g) * 8 + 2 * q] = hi0; patch[(8 + g) * 8 + 2 * q + 1] = hi1;
+                __syncwarp();
+                double y[2][2] = {{0.0, 0.0}, {0.0, 0.0}};
 #pragma unroll
-            for (int j = 0; j < CH_NB; ++j) {
-                double y = 0.0;
-#pragma unroll
-                for (int l2 = j; l2 < CH_NB; ++l2) y -= dinv[j][l2] * acc[l2];
-                if (j < nb) {
-                    X[(int64_t)(i0 + j) * k + c] = y;
-                    d.Rinv[(int64_t)(i0 + j) * k + c] = (float)y;
+                for (int st = 0; st < 4; ++st) {
+                    const double bfr = patch[(4 * st + q) * 8 + g];
+                    dmma_8x8x4(y[0][0], y[0][1], dinv[g][4 * st + q], bfr);
+                    if (st >= 2) dmma_8x8x4(y[1][0], y[1][1], dinv[8 + g][4 * st + q], bfr);   // R11^{-1} is upper triangular
                 }
+#pragma unroll
+                for (int jt = 0; jt < 2; ++jt) {
+                    const int j = jt * 8 + g;
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const int col = c0 + 2 * q + h;
+                        if (j < nb && col < k) {
+                            const double v = -y[jt][h];
+                            X[(int64_t)(i0 + j) * k + col] = v;
+                            d.Rinv[(int64_t)(i0 + j) * k + col] = (float)v;
+                        }
+                    }
+                }
+                __syncwarp();
+                CH_TICK(6);
             }
-            CH_TICK(6);
         }
         for (int e = tid; e < nb * i0; e += nt) {    // zeros left of the diagonal block
             const int j = e / i0, c = e - j * i0;
@@ -376,7 +449,7 @@ cudaError_t chol_inverse_batched(const RefreshDev *rd, const int32_t *list, int 
 {
     if (nlist <= 0) return cudaSuccess;
     const int kpad = (kmax + 5) & ~1;   // even row pitch (in doubles): pairs of a row are read as one 16-byte word
-    const size_t bytes = (size_t)CH_NB * kpad * sizeof(double);
+    const size_t bytes = ((size_t)CH_NB * kpad + (CH_THREADS / 32) * 128) * sizeof(double);   // panel + one 16 x 8 patch per warp
     static size_t configured = 0;
     if (bytes > configured) {
         cudaError_t e = cudaFuncSetAttribute(chol_inverse_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
