@@ -144,15 +144,17 @@ cudaError_t gram_batched(const RefreshDev *rd, const RowItem *items, int nitems,
 
 // ---------------------------------------------------------------------------------------
 // Cholesky S = R^T R with R upper triangular (one CTA per matrix, FP64, in place), followed by
-// Rinv = R^{-1} written as FP32.  Both halves are blocked by 16 and synchronise the CTA a few
-// times per block instead of once per row:
-//   factorisation (right-looking): a 16-row panel of S sits in shared memory; one warp factors
-//   its 16 x 16 diagonal block R11 and inverts it (which is also the diagonal block of R^{-1});
-//   every other column of the panel is then one thread's product with R11^{-T}, and the trailing
-//   upper triangle gets one rank-16 update (two rows per warp, four loads in flight per lane);
+// Rinv = R^{-1} written as FP32.  Both halves are blocked by 16, synchronise the CTA a few times per
+// block, and run their products on the FP64 tensor path (mma m8n8k4):
+//   factorisation (right-looking): a 16-row panel of S sits in shared memory; one warp factors its
+//   16 x 16 diagonal block R11 and inverts it in registers (lane = column, rows exchanged by
+//   shuffles); the rest of the panel is R12 = R11^{-T} S12, one 16 x 8 tile of columns per warp
+//   and trip; the trailing upper triangle then gets the rank-16 update S22 -= R12^T R12 in 8 x 8
+//   tiles, a row of tiles per warp, eight tiles of S in flight per lane as 16-byte accesses (the
+//   update is bound by the number of cache lines a warp visits, not by arithmetic);
 //   inverse (X = R^{-1}, block rows from the bottom up): with the 16 rows of R staged in shared
-//   memory, thread c accumulates sum_l R[i][l] X[l][c] over the rows l of X that are already
-//   known (FP64 copy in Xw, coalesced over c) and multiplies by -R11^{-1}.
+//   memory, a warp accumulates the 16 x 8 tile sum_l R[I][l] X[l][c] over the rows l of X that are
+//   already known (FP64 copy in Xw) and multiplies it by -R11^{-1} through a private patch.
 // A pivot that is not safely positive is replaced by a floor relative to the largest diagonal
 // entry and the block is flagged TSR_ERR_RANK_DEFICIENT.
 // ---------------------------------------------------------------------------------------
