@@ -653,12 +653,43 @@ dc_secular_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__
             dh = df;
             return sgn * f;
         };
-        // 1. the binade of the root: halve hi while h(hi / 2) > 0
+        // 1. a bracket [lo, hi] with lo > 0.  Components of z can be tiny (eigenvectors of a graded matrix
+        //    decay towards the ends), and the root then sits many binades below the gap.  Near the pole
+        //    h(sigma) ~ sgn R(0) - rho z_o^2 / sigma, R being the sum over the other poles, so
+        //    sigma ~ rho z_o^2 / (sgn R(0)) is the right binade; a few doublings or halvings from there
+        //    make the bracket.  When the estimate is unusable, halve down from hi instead.
         double lo = 0.0, dh = 0.0;
-        for (int it = 0; it < 1100; ++it) {
-            const double mid = 0.5 * hi;
-            if (!(mid > 0.0)) break;
-            if (h(mid, dh) > 0.0) hi = mid; else { lo = mid; break; }
+        {
+            double R0 = 1.0;
+            for (int i = 0; i < K; ++i)
+                if (i != o) R0 += rho * zk[i] * zk[i] / (dk[i] - dorg);
+            const double est = rho * zk[o] * zk[o] / (sgn * R0);
+            if (est > 0.0 && est < hi) {
+                if (h(est, dh) > 0.0) {
+                    hi = est;
+                    double sg = est;
+                    for (int it = 0; it < 6; ++it) {
+                        sg *= 0.25;
+                        if (!(sg > 0.0)) break;
+                        if (h(sg, dh) > 0.0) hi = sg; else { lo = sg; break; }
+                    }
+                } else {
+                    lo = est;
+                    double sg = est;
+                    for (int it = 0; it < 6; ++it) {
+                        sg *= 4.0;
+                        if (!(sg < hi)) break;
+                        if (h(sg, dh) > 0.0) { hi = sg; break; } else lo = sg;
+                    }
+                }
+            }
+        }
+        if (!(lo > 0.0)) {
+            for (int it = 0; it < 1100; ++it) {
+                const double mid = 0.5 * hi;
+                if (!(mid > 0.0)) break;
+                if (h(mid, dh) > 0.0) hi = mid; else { lo = mid; break; }
+            }
         }
         // 2. Newton's iteration kept inside the bracket [lo, hi] (a step that leaves it is replaced by
         //    bisection); the bracket shrinks at every step, so the loop ends by itself
