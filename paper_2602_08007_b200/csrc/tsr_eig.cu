@@ -22,6 +22,19 @@ namespace tsr {
 
 constexpr int TR_THREADS = 512;
 constexpr int TR_NB = 8;          // columns per panel
+#ifdef TR_PROFILE
+#define TR_TICK(slot) do { if (threadIdx.x == 0 && blockIdx.x == 0) { const long long t_ = clock64(); tr_prof[slot] += t_ - tr_t0; tr_t0 = t_; } } while (0)
+#else
+#define TR_TICK(slot) do { } while (0)
+#endif
+
+// D (8 x 8, two entries per lane) += A (8 x 4) B (4 x 8) on the FP64 tensor path
+__device__ __forceinline__ void dmma_f64(double &c0, double &c1, double a, double b)
+{
+    asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
+                 : "+d"(c0), "+d"(c1)
+                 : "d"(a), "d"(b));
+}
 
 // ---- stage 1: tridiagonalisation -----------------------------------------------------------
 // Panels of TR_NB columns with the rank-2 updates deferred (the scheme of LAPACK's blocked
@@ -57,6 +70,9 @@ tridiag_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ li
         return t;   // every thread of every warp holds the total
     };
 
+#ifdef TR_PROFILE
+    long long tr_t0 = clock64();
+#endif
     for (int j0 = 0; j0 + 2 < k; j0 += TR_NB) {
         const int L0 = k - j0;
         const int nbc = min(TR_NB, k - 2 - j0);  // columns of this panel that get a reflector
@@ -75,6 +91,7 @@ tridiag_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ li
             double dj = A[(int64_t)j * k + j];   // current diagonal entry (every thread computes it)
             for (int u = 0; u < c; ++u) dj -= 2.0 * Vp[u * kpad + c] * Wp[u * kpad + c];
             const double nrm2 = block_sum(part);
+            TR_TICK(0);
             const double x0 = vs[0];
             const double nrm = sqrt(nrm2);
             const double tail2 = nrm2 - x0 * x0;
@@ -95,6 +112,7 @@ tridiag_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ li
             }
             if (tid == 0) { d.tau[j] = tau; d.dvec[j] = dj; d.evec[j] = alpha; }
             __syncthreads();
+            TR_TICK(1);
             // ps = T0[c+1.., c+1..] v   (row-wise dot products; a warp takes four rows at a time and four
             // 32-column segments of each per trip, so that sixteen loads are in flight per lane; the four
             // sums are then reduced together: two exchange steps leave one sum per group of eight lanes)
@@ -144,6 +162,7 @@ tridiag_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ li
                 if (lane == 0) dots[warp] = acc;
             }
             __syncthreads();
+            TR_TICK(2);
             // p = tau (T0 v - sum_i (v_i (w_i . v) + w_i (v_i . v)))
             part = 0.0;
             for (int a = tid; a < len; a += nt) {
@@ -155,6 +174,7 @@ tridiag_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ li
                 part += acc * vs[a];
             }
             const double pv = block_sum(part);
+            TR_TICK(3);
             const double kk = 0.5 * tau * pv;
             for (int t = tid; t < L0; t += nt) {   // the new pair, zero where the reflector does not act
                 const int a = t - c - 1;
@@ -162,36 +182,72 @@ tridiag_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ li
                 Wp[c * kpad + t] = (a >= 0) ? ps[a] - kk * vs[a] : 0.0;
             }
             __syncthreads();
+            TR_TICK(4);
         }
-        // T0[s][t] -= sum_i (v_i[s] w_i[t] + w_i[s] v_i[t]) for s, t >= nbc   (two rows per warp and trip)
-        for (int s0 = nbc + 2 * warp; s0 < L0; s0 += 2 * nwarps) {
-            const bool two = (s0 + 1 < L0);
-            double va[2][TR_NB], wa[2][TR_NB];
+        // T0[s][t] -= sum_i (v_i[s] w_i[t] + w_i[s] v_i[t]) for s, t >= nbc: a rank-16 update [V W] [W V]^T on
+        // the FP64 tensor path (mma m8n8k4, four steps), 8 x 8 tiles, a row of tiles per warp, eight tiles
+        // of T0 in flight per lane as 16-byte accesses and the next eight already requested: the update
+        // is bound by the latency of those loads and by the cache lines a warp visits.
+        if (nbc == TR_NB) {
+            const int g = lane >> 2, q = lane & 3;
+            const bool k_even = (k & 1) == 0;      // then L0 is even and every pair (t, t + 1), t even, is aligned
+            const int ntile = (L0 - TR_NB + 7) >> 3;
+            for (int si = warp; si < ntile; si += nwarps) {
+                const int srow = TR_NB + si * 8 + g;
+                const bool s_ok = srow < L0;
+                const int sc = min(srow, L0 - 1);
+                const double af[4] = {Vp[q * kpad + sc], Vp[(4 + q) * kpad + sc], Wp[q * kpad + sc], Wp[(4 + q) * kpad + sc]};
+                double *trow = A + (int64_t)(j0 + sc) * k + j0;
+                double cv[8][2], nv[8][2];
+                auto cload = [&](int tj0, double (&v)[8][2]) {
 #pragma unroll
-            for (int u = 0; u < TR_NB; ++u) {
-                const bool on = (u < nbc);
-                va[0][u] = on ? Vp[u * kpad + s0] : 0.0;
-                wa[0][u] = on ? Wp[u * kpad + s0] : 0.0;
-                va[1][u] = (on && two) ? Vp[u * kpad + s0 + 1] : 0.0;
-                wa[1][u] = (on && two) ? Wp[u * kpad + s0 + 1] : 0.0;
-            }
-            double *r0 = A + (int64_t)(j0 + s0) * k + j0, *r1 = r0 + k;
-            for (int t = nbc + lane; t < L0; t += 32) {
-                const double x0 = r0[t], x1 = two ? r1[t] : 0.0;
-                double a0 = 0.0, a1 = 0.0;
-#pragma unroll
-                for (int u = 0; u < TR_NB; ++u) {
-                    const double vt = Vp[u * kpad + t], wt = Wp[u * kpad + t];   // zero rows for u >= nbc are never read: guarded
-                    if (u < nbc) {
-                        a0 += va[0][u] * wt + wa[0][u] * vt;
-                        a1 += va[1][u] * wt + wa[1][u] * vt;
+                    for (int u = 0; u < 8; ++u) {
+                        const int t = TR_NB + (tj0 + u) * 8 + 2 * q;
+                        if (k_even) {
+                            const double2 x = (s_ok && t < L0) ? *(const double2 *)(trow + t) : make_double2(0.0, 0.0);
+                            v[u][0] = x.x; v[u][1] = x.y;
+                        } else {
+                            v[u][0] = (s_ok && t < L0) ? trow[t] : 0.0;
+                            v[u][1] = (s_ok && t + 1 < L0) ? trow[t + 1] : 0.0;
+                        }
                     }
+                };
+                cload(0, cv);
+                for (int tj0 = 0; tj0 < ntile; tj0 += 8) {
+                    cload(tj0 + 8, nv);
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        if (tj0 + u < ntile) {
+                            const int tc = min(TR_NB + (tj0 + u) * 8 + g, L0 - 1);
+                            double a0 = 0.0, a1 = 0.0, b0 = 0.0, b1 = 0.0;    // two chains of two products
+                            dmma_f64(a0, a1, af[0], Wp[q * kpad + tc]);
+                            dmma_f64(b0, b1, af[1], Wp[(4 + q) * kpad + tc]);
+                            dmma_f64(a0, a1, af[2], Vp[q * kpad + tc]);
+                            dmma_f64(b0, b1, af[3], Vp[(4 + q) * kpad + tc]);
+                            const int t = TR_NB + (tj0 + u) * 8 + 2 * q;
+                            if (k_even) {
+                                if (s_ok && t < L0) *(double2 *)(trow + t) = make_double2(cv[u][0] - (a0 + b0), cv[u][1] - (a1 + b1));
+                            } else {
+                                if (s_ok && t < L0) trow[t] = cv[u][0] - (a0 + b0);
+                                if (s_ok && t + 1 < L0) trow[t + 1] = cv[u][1] - (a1 + b1);
+                            }
+                        }
+                    }
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) { cv[u][0] = nv[u][0]; cv[u][1] = nv[u][1]; }
                 }
-                r0[t] = x0 - a0;
-                if (two) r1[t] = x1 - a1;
             }
+        } else {
+            // the last, narrower panel: a few entries, straight from shared memory
+            for (int s1 = nbc + warp; s1 < L0; s1 += nwarps)
+                for (int t = nbc + lane; t < L0; t += 32) {
+                    double acc = 0.0;
+                    for (int u = 0; u < nbc; ++u) acc += Vp[u * kpad + s1] * Wp[u * kpad + t] + Wp[u * kpad + s1] * Vp[u * kpad + t];
+                    A[(int64_t)(j0 + s1) * k + j0 + t] -= acc;
+                }
         }
         __syncthreads();
+        TR_TICK(5);
     }
     if (tid == 0) {
         if (k >= 2) {
