@@ -392,12 +392,17 @@ def test_unaligned_leading_dimension_takes_cuda_core_path():
     _run_steps(tsr, plan, shapes, torch.bfloat16, 3, True, TOL_F32)
 
 
-@pytest.mark.parametrize("copies", [1, 10])
-def test_step_from_host_buffers(copies):
+@pytest.mark.parametrize("copies,one_sided", [(1, False), (10, False), (10, True)])
+def test_step_from_host_buffers(copies, one_sided):
     """The host-buffer step gives exactly the device-buffer step; with 20 blocks it takes the
-    chunked, overlapped order (copies in, step, cores out on three streams)."""
+    chunked, overlapped order (copies in, step, cores out on three streams).  With one_sided every
+    second block keeps an r x n core, which the packed host buffer of cores has to account for."""
     import paper_2602_08007_b200 as tsr
-    shapes = BF16_SHAPES[:2] * copies
+    shapes = [dict(s) for s in BF16_SHAPES[:2] * copies]
+    if one_sided:
+        for s in shapes[1::2]:
+            s["flags"] = 2
+    csize = [s["r"] * (s["n"] if s.get("flags", 0) & 2 else s["r"]) for s in shapes]
     nb = len(shapes)
     plan = tsr.Plan(shapes, g_dtype=torch.bfloat16)
     ref = tsr.Plan(shapes, g_dtype=torch.bfloat16)
@@ -406,7 +411,7 @@ def test_step_from_host_buffers(copies):
         for i in range(nb):
             fill_weights(pl, i, 60 + i)
     gh = [ti.gradient(s["m"], s["n"], 70 + i, dtype=torch.bfloat16).contiguous().pin_memory() for i, s in enumerate(shapes)]
-    c_host = torch.empty(sum(s["r"] ** 2 for s in shapes), dtype=torch.float32).pin_memory()
+    c_host = torch.empty(sum(csize), dtype=torch.float32).pin_memory()
     for t in (1, 2):
         plan.step_host(gh, c_host, tsr.make_hyper(t))
         for i in range(nb):
@@ -416,8 +421,8 @@ def test_step_from_host_buffers(copies):
         off = 0
         for i, s in enumerate(shapes):
             assert torch.equal(plan.W[i], ref.W[i])
-            assert torch.equal(c_host[off:off + s["r"] ** 2].view(s["r"], s["r"]), ref.C[i].cpu())
-            off += s["r"] ** 2
+            assert torch.equal(c_host[off:off + csize[i]].view(ref.C[i].shape), ref.C[i].cpu())
+            off += csize[i]
     assert plan.poll_status() == [0] * nb
 
 
