@@ -408,7 +408,11 @@ ql_log_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ lis
     for (int i = threadIdx.x; i < n; i += 64) D.dvec[i] = d[i];
 }
 
-__global__ void eig_rank_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ list)
+// Bit 30 of rank[c] marks a coordinate that takes part in the secular problem (dc only): its column of the
+// eigenvector matrix comes out of the merge product, the other columns are final after the rotations.
+constexpr int RANK_MERGED = 1 << 30;
+
+__global__ void eig_rank_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ list, int dc)
 {
     const RefreshDev D = rd[list[blockIdx.x]];
     const int k = D.k, r = D.r;
@@ -426,6 +430,11 @@ __global__ void eig_rank_kernel(const RefreshDev *__restrict__ rd, const int32_t
         if (rank < r && !(lj > 1e-300) && flag == 0) flag = TSR_ERR_RANK_DEFICIENT;
     }
     if (flag) atomicMax(D.status, flag);
+    if (dc) {
+        __syncthreads();
+        const int K = D.dc_info[0];
+        for (int j = threadIdx.x; j < K; j += blockDim.x) D.rank[D.dc_nd[j]] |= RANK_MERGED;
+    }
 }
 
 // ---- stage 3, systolic form (k <= SYS_KMAX) ---------------------------------------------------
@@ -826,65 +835,33 @@ eig_rot_systolic_kernel(const RefreshDev *__restrict__ rd, const RowItem *__rest
             }
         }
         __syncwarp();
-        // the coordinates of the secular problem: y = x[nd] Uhat, written back over x[nd]
+        // The coordinates of the secular problem still have to be multiplied by Uhat: their values, gathered in
+        // the order of the secular problem, go back to this row of Wj for eig_merge_kernel.  The deflated
+        // coordinates are final: their columns are emitted here.
         const int K = D.dc_info[0];
-        const double *__restrict__ Uh = D.Xw;
         const int32_t *__restrict__ nd = D.dc_nd;
-        constexpr int NCH = 17;                   // 32-column chunks per pass (544 columns)
-        for (int c0 = 0; c0 < K; c0 += 32 * NCH) {
-            double acc[R][NCH];
 #pragma unroll
-            for (int q = 0; q < R; ++q)
+        for (int q = 0; q < R; ++q) {
+            const int row = row0 + q;
+            if (row < k)
+                for (int i = lane; i < K; i += 32) D.Wj[(int64_t)row * k + i] = z[q * k + nd[i]];
+        }
+        for (int jj = lane; jj < k; jj += 32) {
+            const int rk = D.rank[jj];
+            if ((rk & RANK_MERGED) || rk >= r) continue;
+            const double lj = D.dvec[jj];
+            const double inv = (lj > 1e-300) ? 1.0 / sqrt(lj) : 0.0;
 #pragma unroll
-                for (int u = 0; u < NCH; ++u) acc[q][u] = 0.0;
-            for (int i = 0; i < K; ++i) {
-                const int ci = nd[i];
-                double xv[R];
-#pragma unroll
-                for (int q = 0; q < R; ++q) xv[q] = z[q * k + ci];
-                const double *urow = Uh + (int64_t)i * k + c0 + lane;
-#pragma unroll
-                for (int u = 0; u < NCH; ++u) {
-                    const double uv = (c0 + lane + 32 * u < K) ? urow[32 * u] : 0.0;
-#pragma unroll
-                    for (int q = 0; q < R; ++q) acc[q][u] += xv[q] * uv;
-                }
-            }
-            // results of this pass go to a side buffer first when a second pass still needs the inputs
-            __syncwarp();
-            if (K <= 32 * NCH) {
-#pragma unroll
-                for (int u = 0; u < NCH; ++u) {
-                    const int j = c0 + lane + 32 * u;
-                    if (j < K) {
-                        const int cj = nd[j];
-#pragma unroll
-                        for (int q = 0; q < R; ++q) z[q * k + cj] = acc[q][u];
-                    }
-                }
-            } else {
-                // wide problems: park the results in the (now unused) rows of Wj and copy back at the end
-#pragma unroll
-                for (int u = 0; u < NCH; ++u) {
-                    const int j = c0 + lane + 32 * u;
-                    if (j < K) {
-#pragma unroll
-                        for (int q = 0; q < R; ++q)
-                            if (row0 + q < k) D.Wj[(int64_t)(row0 + q) * k + j] = acc[q][u];
-                    }
+            for (int q = 0; q < R; ++q) {
+                const int row = row0 + q;
+                if (row < k) {
+                    const double w = z[q * k + jj];
+                    D.Wu[(int64_t)row * r + rk] = (float)w;
+                    D.Wv[(int64_t)row * r + rk] = (float)(w * inv);
                 }
             }
         }
-        __syncwarp();
-        if (K > 32 * NCH) {
-            for (int j = lane; j < K; j += 32) {
-                const int cj = nd[j];
-#pragma unroll
-                for (int q = 0; q < R; ++q)
-                    if (row0 + q < k) z[q * k + cj] = D.Wj[(int64_t)(row0 + q) * k + j];
-            }
-        }
-        __syncwarp();
+        return;
     }
     // rank the eigenvalues (descending, ties by index) and emit the leading r columns
     const double *__restrict__ lam = D.dvec;
@@ -903,6 +880,95 @@ eig_rot_systolic_kernel(const RefreshDev *__restrict__ rd, const RowItem *__rest
             }
         }
     }
+}
+
+// Divide and conquer, step 4b: the coordinates of the secular problem times the merged eigenvector matrix,
+// Y = Zg Uhat (Zg: k x K, the rows the rotation kernel left in Wj; Uhat: K x K in Xw), on the FP64 tensor
+// path.  A CTA owns a 64 x 64 tile of Y, its eight warps 32 x 16 regions of it as 4 x 2 sub-tiles of 8 x 8
+// (mma m8n8k4); operands are staged 16 columns of Zg / rows of Uhat at a time.  Column j of Y is the
+// eigenvector column of coordinate nd[j]; the leading r columns by eigenvalue are written as Wu and,
+// scaled by 1 / sqrt(lambda), as Wv.
+constexpr int MG_T = 64, MG_K = 16, MG_PITCH = 68;    // 68 = 4 mod 16: the 64-bit fragment loads are conflict-free
+
+__global__ void __launch_bounds__(256)
+eig_merge_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ list)
+{
+    const RefreshDev D = rd[list[blockIdx.z]];
+    const int k = D.k, r = D.r, K = D.dc_info[0];
+    const int r0 = blockIdx.y * MG_T, c0 = blockIdx.x * MG_T;
+    if (r0 >= k || c0 >= K) return;
+    const double *__restrict__ Zg = D.Wj;
+    const double *__restrict__ Uh = D.Xw;
+    __shared__ __align__(16) double As[MG_K][MG_PITCH];     // As[i][row] = Zg[r0 + row][i0 + i]
+    __shared__ __align__(16) double Bs[MG_K][MG_PITCH];     // Bs[i][col] = Uhat[i0 + i][c0 + col]
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int wi = warp >> 2, wj = warp & 3;
+    const int g = lane >> 2, q = lane & 3;
+    double acc[4][2][2];
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+        for (int b = 0; b < 2; ++b) acc[a][b][0] = acc[a][b][1] = 0.0;
+    double ra[4], rb[4];
+    auto fetch = [&](int i0) {
+#pragma unroll
+        for (int l = 0; l < 4; ++l) {
+            const int e = tid + l * 256;
+            {
+                const int row = r0 + (e >> 4), i = i0 + (e & 15);
+                ra[l] = (row < k && i < K) ? Zg[(int64_t)row * k + i] : 0.0;
+            }
+            {
+                const int i = i0 + (e >> 6), col = c0 + (e & 63);
+                rb[l] = (i < K && col < K) ? Uh[(int64_t)i * k + col] : 0.0;
+            }
+        }
+    };
+    fetch(0);
+    for (int i0 = 0; i0 < K; i0 += MG_K) {
+#pragma unroll
+        for (int l = 0; l < 4; ++l) {
+            const int e = tid + l * 256;
+            As[e & 15][e >> 4] = ra[l];
+            Bs[e >> 6][e & 63] = rb[l];
+        }
+        __syncthreads();
+        if (i0 + MG_K < K) fetch(i0 + MG_K);
+#pragma unroll
+        for (int st = 0; st < MG_K / 4; ++st) {
+            double af[4], bf[2];
+#pragma unroll
+            for (int a = 0; a < 4; ++a) af[a] = As[st * 4 + q][wi * 32 + a * 8 + g];
+#pragma unroll
+            for (int b = 0; b < 2; ++b) bf[b] = Bs[st * 4 + q][wj * 16 + b * 8 + g];
+#pragma unroll
+            for (int a = 0; a < 4; ++a)
+#pragma unroll
+                for (int b = 0; b < 2; ++b) dmma_f64(acc[a][b][0], acc[a][b][1], af[a], bf[b]);
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int b = 0; b < 2; ++b)
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int j = c0 + wj * 16 + b * 8 + 2 * q + h;
+            if (j >= K) continue;
+            const int cj = D.dc_nd[j];
+            const int rk = D.rank[cj] & (RANK_MERGED - 1);
+            if (rk >= r) continue;
+            const double lj = D.dvec[cj];
+            const double inv = (lj > 1e-300) ? 1.0 / sqrt(lj) : 0.0;
+#pragma unroll
+            for (int a = 0; a < 4; ++a) {
+                const int row = r0 + wi * 32 + a * 8 + g;
+                if (row < k) {
+                    const double w = acc[a][b][h];
+                    D.Wu[(int64_t)row * r + rk] = (float)w;
+                    D.Wv[(int64_t)row * r + rk] = (float)(w * inv);
+                }
+            }
+        }
 }
 
 static int sys_rows_per_warp(int kmax) { return kmax <= 544 ? 4 : 2; }
@@ -954,7 +1020,7 @@ cudaError_t eig_tridiag_batched(const RefreshDev *rd, const int32_t *list, int n
             if ((e = raise_smem(dc_secular_kernel, sec_bytes, &sec_cfg)) != cudaSuccess) return e;
             dc_secular_kernel<<<nlist, DC_THREADS, sec_bytes, stream>>>(rd, list, kpad);
         }
-        eig_rank_kernel<<<nlist, 256, 0, stream>>>(rd, list);
+        eig_rank_kernel<<<nlist, 256, 0, stream>>>(rd, list, dc);
         const int R = sys_rows_per_warp(kmax);
         const size_t sys_bytes = (size_t)SYS_WARPS * R * kmax * sizeof(double);
         if (R == 4) {
@@ -963,6 +1029,10 @@ cudaError_t eig_tridiag_batched(const RefreshDev *rd, const int32_t *list, int n
         } else {
             if ((e = raise_smem(eig_rot_systolic_kernel<2>, sys_bytes, &sys2_cfg)) != cudaSuccess) return e;
             eig_rot_systolic_kernel<2><<<npanels, threads, sys_bytes, stream>>>(rd, panel_items, dc);
+        }
+        if (dc) {
+            const int t = (kmax + MG_T - 1) / MG_T;
+            eig_merge_kernel<<<dim3(t, t, nlist), 256, 0, stream>>>(rd, list);
         }
         return cudaGetLastError();
     }
