@@ -718,17 +718,12 @@ tsr_status do_refresh_group(tsr_ctx *ctx, const std::vector<int> &list, uint64_t
     const int nl = (int)list.size();
     TSR_KERNEL(ctx, 2, gram_batched(ctx->d_refresh, L.ditems[3], L.nitems[3], L.dlist, nl, 1, 0, L.kmax, st));
     if (L.kmax >= 200) {   // too large for the Jacobi solver: tridiagonal route
-        const int pr = eig_panel_rows(L.kmax), qr = eig_qrows_rows(L.kmax);
+        const int pr = eig_panel_rows(L.kmax);
         std::vector<RowItem> panels;
         for (int bi : list)
             for (int r0 = 0; r0 < ctx->blocks[bi].k; r0 += pr) panels.push_back({bi, r0});
-        const size_t npan = panels.size();
-        if (qr > 0)
-            for (int bi : list)
-                for (int r0 = 0; r0 < ctx->blocks[bi].k; r0 += qr) panels.push_back({bi, r0});
         TSR_CUDA(ctx, cudaMemcpyAsync(L.ditems[4], panels.data(), panels.size() * sizeof(RowItem), cudaMemcpyHostToDevice, st));
-        TSR_KERNEL(ctx, 5, eig_tridiag_batched(ctx->d_refresh, L.dlist, nl, L.ditems[4], (int)npan, L.ditems[4] + npan,
-                                               (int)(panels.size() - npan), L.kmax, st));
+        TSR_KERNEL(ctx, 16, eig_tridiag_batched(ctx->d_refresh, L.dlist, nl, L.ditems[4], (int)panels.size(), L.kmax, st));
     } else {
         TSR_KERNEL(ctx, 1, jacobi_batched(ctx->d_refresh, L.dlist, nl, 40, st));
     }

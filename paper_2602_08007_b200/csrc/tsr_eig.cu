@@ -9,12 +9,13 @@
 //      every plane rotation instead of applying it;
 //   3. the merge: eigen-decomposition of D + rho z z^T (D = eigenvalues of the halves, z = Z^T u)
 //      through the secular equation, one root per thread;
-//   4. the eigenvectors W = Q diag(Z1, Z2) G Uhat, row slab by row slab (rows are independent under
-//      right-multiplication): a first kernel forms the rows of Q from the reflectors with the
-//      rows held in registers; a second one streams every row through the two rotation logs as
-//      a systolic pipeline over the lanes of a warp (32 sweeps advance per step), then through
-//      the deflation rotations G and the merged eigenvector matrix Uhat, and writes the leading r
-//      columns in descending eigenvalue order: Wu = W[:, :r], Wv = W[:, :r] / sqrt(lambda).
+//   4. the eigenvectors W = Q diag(Z1, Z2) G Uhat: Q = I - V T V^T comes out of tiled products on the
+//      FP64 tensor path (compact WY form of all reflectors at once); a second kernel streams every
+//      row of Q through the two rotation logs as a systolic pipeline over the lanes of a warp (32
+//      sweeps advance per step) and through the deflation rotations G (rows are independent under
+//      right-multiplication); a last tiled product multiplies by the merged eigenvector matrix Uhat
+//      and writes the leading r columns in descending eigenvalue order: Wu = W[:, :r],
+//      Wv = W[:, :r] / sqrt(lambda).
 // Failure to converge within the iteration or log budget flags TSR_ERR_NOT_CONVERGED.
 #include "tsr_internal.h"
 
@@ -35,6 +36,10 @@ __device__ __forceinline__ void dmma_f64(double &c0, double &c1, double a, doubl
                  : "+d"(c0), "+d"(c1)
                  : "d"(a), "d"(b));
 }
+
+// Tiled FP64 tensor-path products below: 64 x 64 tiles, operands staged 16 deep, 68 doubles per staged row
+// (68 = 4 mod 16: the 64-bit fragment loads are conflict-free).
+constexpr int MG_T = 64, MG_K = 16, MG_PITCH = 68;
 
 // ---- stage 1: tridiagonalisation -----------------------------------------------------------
 // Panels of TR_NB columns with the rank-2 updates deferred (the scheme of LAPACK's blocked
@@ -437,84 +442,176 @@ __global__ void eig_rank_kernel(const RefreshDev *__restrict__ rd, const int32_t
     }
 }
 
-// ---- stage 3, systolic form (k <= SYS_KMAX) ---------------------------------------------------
-// 3a: rows of Q = H_0 H_1 ... in registers.  A warp owns RQ rows (NW warps per CTA); lane holds columns lane + 32 i.
-// The reflectors are staged for the whole CTA, a few at a time, in shared memory.
+// ---- stage 3: the eigenvectors (k <= SYS_KMAX) -------------------------------------------------
 constexpr int SYS_KMAX = 1056;
 constexpr int DC_MIN_K = 200;    // the tridiagonal problem is torn in two from this size on
 constexpr int SYS_WARPS = 12;    // warps of the rotation kernel (three per scheduler)
-constexpr int QR_WARPS = 16;     // warps of the Q-rows kernel
 
-template <int NCH, int RQ, int NW>
-__global__ void __launch_bounds__(NW * 32)
-eig_qrows_kernel(const RefreshDev *__restrict__ rd, const RowItem *__restrict__ items)
+// 3a: Q = H_0 H_1 ... H_{k-3} = I - V T V^T with V = (v_0 .. v_{k-3}) and T upper
+// triangular (the compact WY representation of all reflectors at once), every step a tiled product on the FP64
+// tensor path (mma m8n8k4; 64 x 64 tiles, eight warps of 32 x 16, operands staged 16 deep):
+//   G  = V^T V (above the diagonal)                                      -> Xw
+//   T  : 64 x 64 diagonal blocks by the column recurrence T[0:i, i] = -tau_i T[0:i, 0:i] G[0:i, i], then
+//        blocks of 64, 128, 256 ... merged pairwise, T_AB = -T_A (G_AB T_B)  -> gpart (X = G_AB T_B in Wj)
+//   M  = T V^T                                                             -> Xw (G is no longer needed)
+//   Q  = I - V M                                                           -> Wj
+// v_j = (0 .. 0, 1 at j + 1, S[j][j + 2 ..]); a reflector with tau_j = 0 has a zero row and column in T and
+// drops out whatever its row of S holds.  About 2.5 k^3 multiply-adds instead of k^3, but as products that
+// run near the rate of the tensor path instead of dependent reduce-and-update rounds.
+enum WyMode : int { WY_G = 0, WY_X, WY_T12, WY_M, WY_Q };
+constexpr int WY_NB = 64;      // base block of T
+
+__device__ __forceinline__ double wy_vt(const double *__restrict__ S, int k, int nr, int j, int c)
 {
-    constexpr int LD = NCH * 32;
-    constexpr int QV_BATCH = NCH > 17 ? 4 : 8;    // reflectors staged per round (static shared memory <= 48 KB)
-    __shared__ double vs[QV_BATCH][LD];
-    __shared__ double taus[QV_BATCH];
-    const RowItem it = items[blockIdx.x];
-    const RefreshDev D = rd[it.block];
-    const int k = D.k;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int row0 = it.row0 + warp * RQ;
-    const double *__restrict__ A = D.S;
-    double x[RQ][NCH];
-#pragma unroll
-    for (int q = 0; q < RQ; ++q)
-#pragma unroll
-        for (int i = 0; i < NCH; ++i) x[q][i] = (lane + 32 * i == row0 + q) ? 1.0 : 0.0;
+    // V^T[j][c]: entry c of reflector j
+    if (j >= nr || c <= j || c >= k) return 0.0;
+    return (c == j + 1) ? 1.0 : S[(int64_t)j * k + c];
+}
 
-    for (int j0 = 0; j0 + 2 < k; j0 += QV_BATCH) {
-        __syncthreads();
-        for (int idx = threadIdx.x; idx < QV_BATCH * LD; idx += NW * 32) {
-            const int b = idx / LD, c = idx - b * LD, j = j0 + b;
-            double v = 0.0;
-            if (j + 2 < k && c < k) v = (c == j + 1) ? 1.0 : (c >= j + 2 ? A[(int64_t)j * k + c] : 0.0);
-            vs[b][c] = v;
-        }
-        if (threadIdx.x < QV_BATCH) taus[threadIdx.x] = (j0 + threadIdx.x + 2 < k) ? D.tau[j0 + threadIdx.x] : 0.0;
-        __syncthreads();
-#pragma unroll 1
-        for (int b = 0; b < QV_BATCH; ++b) {
-            const double tau = taus[b];
-            if (tau == 0.0) continue;
-            const int i0 = (j0 + b + 1) >> 5;     // chunks below hold only zeros of v
-            double dot[RQ];
-#pragma unroll
-            for (int q = 0; q < RQ; ++q) dot[q] = 0.0;
-#pragma unroll
-            for (int i = 0; i < NCH; ++i)
-                if (i >= i0) {
-                    const double v = vs[b][lane + 32 * i];
-#pragma unroll
-                    for (int q = 0; q < RQ; ++q) dot[q] += x[q][i] * v;
-                }
-#pragma unroll
-            for (int off = 16; off > 0; off >>= 1)
-#pragma unroll
-                for (int q = 0; q < RQ; ++q) dot[q] += __shfl_xor_sync(0xffffffffu, dot[q], off);
-#pragma unroll
-            for (int q = 0; q < RQ; ++q) dot[q] *= tau;
-#pragma unroll
-            for (int i = 0; i < NCH; ++i)
-                if (i >= i0) {
-                    const double v = vs[b][lane + 32 * i];
-#pragma unroll
-                    for (int q = 0; q < RQ; ++q) x[q][i] -= dot[q] * v;
-                }
-        }
+template <int MODE>
+__global__ void __launch_bounds__(256)
+eig_wy_gemm_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ list, int s)
+{
+    const RefreshDev D = rd[list[blockIdx.z]];
+    const int k = D.k, nr = k - 2;
+    const int r0 = blockIdx.y * 64, c0 = blockIdx.x * 64;
+    const double *__restrict__ S = D.S;
+    double *__restrict__ G = D.Xw;       // G, later M
+    double *__restrict__ T = D.gpart;
+    double *__restrict__ X = D.Wj;       // X during the merges, Q at the end
+    // extent of this tile's product: rows < Mr, columns < Nc, contraction index in [kb, ke)
+    int Mr, Nc, kb, ke;
+    if (MODE == WY_G) {                  // G[a][b] = sum_c V^T[a][c] V^T[b][c], tiles on or above the diagonal
+        if (c0 < r0) return;
+        Mr = nr; Nc = nr; kb = c0 & ~15; ke = k;      // v_b is zero up to column b >= c0
+    } else if (MODE == WY_X || MODE == WY_T12) {
+        // pair of blocks A = [pa, pa + s), B = [pa + s, pa + 2 s): the tile must lie in rows A, columns B
+        const int pa = (r0 / (2 * s)) * (2 * s), pb = pa + s;
+        if (r0 >= pb || c0 < pb || c0 >= pb + s) return;
+        Mr = min(pb, nr); Nc = min(pb + s, nr);
+        if (MODE == WY_X) { kb = pb; ke = min(c0 + 64, Nc); }        // X[a][j] = sum_{l in B, l <= j} G[a][l] T[l][j]
+        else { kb = r0; ke = Mr; }                                    // T[a][j] = -sum_{l in A, l >= a} T[a][l] X[l][j]
+    } else if (MODE == WY_M) {           // M[i][c] = sum_{l >= i} T[i][l] V^T[l][c]; V^T[l][c] = 0 for l >= c
+        Mr = nr; Nc = k; kb = r0; ke = min(nr, c0 + 64);
+    } else {                             // Q[c][c'] = delta - sum_j V^T[j][c] M[j][c'], j < c
+        Mr = k; Nc = k; kb = 0; ke = min(nr, r0 + 64);
     }
+    if (r0 >= Mr || c0 >= Nc) return;
+    __shared__ __align__(16) double As[MG_K][MG_PITCH];     // As[kk][row]
+    __shared__ __align__(16) double Bs[MG_K][MG_PITCH];     // Bs[kk][col]
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int wi = warp >> 2, wj = warp & 3;
+    const int g = lane >> 2, q = lane & 3;
+    double acc[4][2][2];
 #pragma unroll
-    for (int q = 0; q < RQ; ++q) {
-        const int row = row0 + q;
-        if (row < k) {
+    for (int a = 0; a < 4; ++a)
 #pragma unroll
-            for (int i = 0; i < NCH; ++i) {
-                const int c = lane + 32 * i;
-                if (c < k) D.Wj[(int64_t)row * k + c] = x[q][i];
+        for (int b = 0; b < 2; ++b) acc[a][b][0] = acc[a][b][1] = 0.0;
+    // element maps: the index that is contiguous in memory goes to consecutive threads
+    constexpr bool A_KFAST = (MODE != WY_Q);                 // A(i, kk) contiguous in kk, except V (= V^T transposed)
+    constexpr bool B_KFAST = (MODE == WY_G);                 // B(kk, j) contiguous in j, except V^T[b][c] over c
+    double ra[4], rb[4];
+    auto fetch = [&](int k0) {
+#pragma unroll
+        for (int l = 0; l < 4; ++l) {
+            const int e = tid + l * 256;
+            {
+                const int row = r0 + (A_KFAST ? (e >> 4) : (e & 63)), kk = k0 + (A_KFAST ? (e & 15) : (e >> 6));
+                double v = 0.0;
+                if (row < Mr && kk < ke) {
+                    if (MODE == WY_G) v = wy_vt(S, k, nr, row, kk);
+                    else if (MODE == WY_X) v = G[(int64_t)row * k + kk];
+                    else if (MODE == WY_T12 || MODE == WY_M) v = (kk >= row) ? T[(int64_t)row * k + kk] : 0.0;
+                    else v = wy_vt(S, k, nr, kk, row);
+                }
+                ra[l] = v;
+            }
+            {
+                const int col = c0 + (B_KFAST ? (e >> 4) : (e & 63)), kk = k0 + (B_KFAST ? (e & 15) : (e >> 6));
+                double v = 0.0;
+                if (col < Nc && kk < ke) {
+                    if (MODE == WY_G) v = wy_vt(S, k, nr, col, kk);
+                    else if (MODE == WY_X) v = (kk <= col) ? T[(int64_t)kk * k + col] : 0.0;
+                    else if (MODE == WY_T12) v = X[(int64_t)kk * k + col];
+                    else if (MODE == WY_M) v = wy_vt(S, k, nr, kk, col);
+                    else v = G[(int64_t)kk * k + col];
+                }
+                rb[l] = v;
             }
         }
+    };
+    kb &= ~15;
+    if (kb < ke) fetch(kb);
+    for (int k0 = kb; k0 < ke; k0 += MG_K) {
+#pragma unroll
+        for (int l = 0; l < 4; ++l) {
+            const int e = tid + l * 256;
+            if (A_KFAST) As[e & 15][e >> 4] = ra[l]; else As[e >> 6][e & 63] = ra[l];
+            if (B_KFAST) Bs[e & 15][e >> 4] = rb[l]; else Bs[e >> 6][e & 63] = rb[l];
+        }
+        __syncthreads();
+        if (k0 + MG_K < ke) fetch(k0 + MG_K);
+#pragma unroll
+        for (int st = 0; st < MG_K / 4; ++st) {
+            double af[4], bf[2];
+#pragma unroll
+            for (int a = 0; a < 4; ++a) af[a] = As[st * 4 + q][wi * 32 + a * 8 + g];
+#pragma unroll
+            for (int b = 0; b < 2; ++b) bf[b] = Bs[st * 4 + q][wj * 16 + b * 8 + g];
+#pragma unroll
+            for (int a = 0; a < 4; ++a)
+#pragma unroll
+                for (int b = 0; b < 2; ++b) dmma_f64(acc[a][b][0], acc[a][b][1], af[a], bf[b]);
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+        for (int b = 0; b < 2; ++b)
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int row = r0 + wi * 32 + a * 8 + g, col = c0 + wj * 16 + b * 8 + 2 * q + h;
+                if (row >= Mr || col >= Nc) continue;
+                const double v = acc[a][b][h];
+                if (MODE == WY_G) G[(int64_t)row * k + col] = v;
+                else if (MODE == WY_X) X[(int64_t)row * k + col] = v;
+                else if (MODE == WY_T12) T[(int64_t)row * k + col] = -v;
+                else if (MODE == WY_M) G[(int64_t)row * k + col] = v;
+                else X[(int64_t)row * k + col] = ((row == col) ? 1.0 : 0.0) - v;
+            }
+}
+
+// The 64 x 64 diagonal blocks of T: thread rr owns row rr of a block (T[rr][i] needs T[rr][rr .. i-1] only),
+// with the block of G and the rows of T in shared memory.
+__global__ void __launch_bounds__(WY_NB)
+eig_wy_base_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ list)
+{
+    extern __shared__ double wb_smem[];        // Gs[64][65], Ts[64][65]
+    double *Gs = wb_smem, *Ts = wb_smem + WY_NB * (WY_NB + 1);
+    const RefreshDev D = rd[list[blockIdx.y]];
+    const int k = D.k, nr = k - 2, b0 = blockIdx.x * WY_NB;
+    if (b0 >= nr) return;
+    const double *__restrict__ G = D.Xw;
+    double *__restrict__ T = D.gpart;
+    const int rr = threadIdx.x;
+    const int nb = min(WY_NB, nr - b0);
+    __shared__ double taus[WY_NB];
+    taus[rr] = (rr < nb) ? D.tau[b0 + rr] : 0.0;
+    for (int l = 0; l < nb; ++l) Gs[l * (WY_NB + 1) + rr] = (rr < nb) ? G[(int64_t)(b0 + l) * k + b0 + rr] : 0.0;
+    __syncthreads();
+    if (rr >= nb) return;
+    double *trow = Ts + rr * (WY_NB + 1);
+    for (int i = rr; i < nb; ++i) {
+        double v;
+        if (i == rr) v = taus[i];
+        else {
+            double sacc = 0.0;
+            for (int l = rr; l < i; ++l) sacc += trow[l] * Gs[l * (WY_NB + 1) + i];
+            v = -taus[i] * sacc;
+        }
+        trow[i] = v;
+        T[(int64_t)(b0 + rr) * k + b0 + i] = v;
     }
 }
 
@@ -888,7 +985,6 @@ eig_rot_systolic_kernel(const RefreshDev *__restrict__ rd, const RowItem *__rest
 // (mma m8n8k4); operands are staged 16 columns of Zg / rows of Uhat at a time.  Column j of Y is the
 // eigenvector column of coordinate nd[j]; the leading r columns by eigenvalue are written as Wu and,
 // scaled by 1 / sqrt(lambda), as Wv.
-constexpr int MG_T = 64, MG_K = 16, MG_PITCH = 68;    // 68 = 4 mod 16: the 64-bit fragment loads are conflict-free
 
 __global__ void __launch_bounds__(256)
 eig_merge_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ list)
@@ -973,8 +1069,6 @@ eig_merge_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ 
 
 static int sys_rows_per_warp(int kmax) { return kmax <= 544 ? 4 : 2; }
 
-int eig_qrows_rows(int kmax) { return QR_WARPS * (kmax <= 544 ? 2 : 1); }
-
 int eig_panel_rows(int kmax)
 {
     return SYS_WARPS * sys_rows_per_warp(kmax);
@@ -997,7 +1091,7 @@ static cudaError_t raise_smem(F *fn, size_t bytes, size_t *configured)
 }
 
 cudaError_t eig_tridiag_batched(const RefreshDev *rd, const int32_t *list, int nlist, const RowItem *panel_items,
-                                int npanels, const RowItem *qrows_items, int nqrows, int kmax, cudaStream_t stream)
+                                int npanels, int kmax, cudaStream_t stream)
 {
     if (nlist <= 0) return cudaSuccess;
     const int kpad = kmax + 8;
@@ -1009,9 +1103,21 @@ cudaError_t eig_tridiag_batched(const RefreshDev *rd, const int32_t *list, int n
     const size_t ql_bytes = (size_t)2 * kmax * sizeof(double);
     if (kmax <= SYS_KMAX) {
         const int threads = SYS_WARPS * 32;
-        if (kmax <= 288) eig_qrows_kernel<9, 2, QR_WARPS><<<nqrows, QR_WARPS * 32, 0, stream>>>(rd, qrows_items);
-        else if (kmax <= 544) eig_qrows_kernel<17, 2, QR_WARPS><<<nqrows, QR_WARPS * 32, 0, stream>>>(rd, qrows_items);
-        else eig_qrows_kernel<33, 1, QR_WARPS><<<nqrows, QR_WARPS * 32, 0, stream>>>(rd, qrows_items);
+        {   // Q = I - V T V^T, every step a tiled product (see eig_wy_gemm_kernel)
+            const int t = (kmax + 63) / 64;
+            const dim3 grid(t, t, nlist);
+            const size_t wb_bytes = (size_t)2 * WY_NB * (WY_NB + 1) * sizeof(double);
+            static size_t wb_cfg = 0;
+            if ((e = raise_smem(eig_wy_base_kernel, wb_bytes, &wb_cfg)) != cudaSuccess) return e;
+            eig_wy_gemm_kernel<WY_G><<<grid, 256, 0, stream>>>(rd, list, 0);
+            eig_wy_base_kernel<<<dim3(t, nlist), WY_NB, wb_bytes, stream>>>(rd, list);
+            for (int sz = WY_NB; sz < kmax - 2; sz *= 2) {
+                eig_wy_gemm_kernel<WY_X><<<grid, 256, 0, stream>>>(rd, list, sz);
+                eig_wy_gemm_kernel<WY_T12><<<grid, 256, 0, stream>>>(rd, list, sz);
+            }
+            eig_wy_gemm_kernel<WY_M><<<grid, 256, 0, stream>>>(rd, list, 0);
+            eig_wy_gemm_kernel<WY_Q><<<grid, 256, 0, stream>>>(rd, list, 0);
+        }
         const int dc = kmax >= DC_MIN_K ? 1 : 0;
         ql_log_kernel<<<nlist, 64, ql_bytes, stream>>>(rd, list, dc);
         if (dc) {

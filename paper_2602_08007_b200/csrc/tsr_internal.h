@@ -177,12 +177,10 @@ cudaError_t split_operands_batched(const RefreshDev *rd, const RowItem *items, i
 // The same result through Householder tridiagonalisation + implicit QL with logged rotations
 // (for k too large for the Jacobi solver).  panel_items: (block, row0) slabs of eig_panel_rows(kmax)
 // rows of the k x k eigenvector matrix.  eig_rot_capacity(k): entries of the rotation log to provide.
-// qrows_items: slabs of eig_qrows_rows(kmax) rows for the kernel that forms the rows of Q (0: not used).
 int eig_panel_rows(int kmax);
-int eig_qrows_rows(int kmax);
 int64_t eig_rot_capacity(int k);
 cudaError_t eig_tridiag_batched(const RefreshDev *rd, const int32_t *list, int nlist, const RowItem *panel_items,
-                                int npanels, const RowItem *qrows_items, int nqrows, int kmax, cudaStream_t stream);
+                                int npanels, int kmax, cudaStream_t stream);
 cudaError_t jacobi_batched(const RefreshDev *rd, const int32_t *list, int nlist, int max_sweeps, cudaStream_t stream);
 
 }  // namespace tsr
