@@ -458,7 +458,7 @@ constexpr int SYS_WARPS = 12;    // warps of the rotation kernel (three per sche
 // v_j = (0 .. 0, 1 at j + 1, S[j][j + 2 ..]); a reflector with tau_j = 0 has a zero row and column in T and
 // drops out whatever its row of S holds.  About 2.5 k^3 multiply-adds instead of k^3, but as products that
 // run near the rate of the tensor path instead of dependent reduce-and-update rounds.
-enum WyMode : int { WY_G = 0, WY_X, WY_T12, WY_M, WY_Q };
+enum WyMode : int { WY_G = 0, WY_X, WY_T12, WY_M, WY_Q, WY_W };
 constexpr int WY_NB = 64;      // base block of T
 
 __device__ __forceinline__ double wy_vt(const double *__restrict__ S, int k, int nr, int j, int c)
@@ -493,8 +493,10 @@ eig_wy_gemm_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict_
         else { kb = r0; ke = Mr; }                                    // T[a][j] = -sum_{l in A, l >= a} T[a][l] X[l][j]
     } else if (MODE == WY_M) {           // M[i][c] = sum_{l >= i} T[i][l] V^T[l][c]; V^T[l][c] = 0 for l >= c
         Mr = nr; Nc = k; kb = r0; ke = min(nr, c0 + 64);
-    } else {                             // Q[c][c'] = delta - sum_j V^T[j][c] M[j][c'], j < c
+    } else if (MODE == WY_Q) {           // Q[c][c'] = delta - sum_j V^T[j][c] M[j][c'], j < c
         Mr = k; Nc = k; kb = 0; ke = min(nr, r0 + 64);
+    } else {                             // W = Q Ztot (Q in Wj, Ztot in gpart): the eigenvectors of S
+        Mr = k; Nc = k; kb = 0; ke = k;
     }
     if (r0 >= Mr || c0 >= Nc) return;
     __shared__ __align__(16) double As[MG_K][MG_PITCH];     // As[kk][row]
@@ -509,6 +511,7 @@ eig_wy_gemm_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict_
         for (int b = 0; b < 2; ++b) acc[a][b][0] = acc[a][b][1] = 0.0;
     // element maps: the index that is contiguous in memory goes to consecutive threads
     constexpr bool A_KFAST = (MODE != WY_Q);                 // A(i, kk) contiguous in kk, except V (= V^T transposed)
+    const int r_out = D.r;
     constexpr bool B_KFAST = (MODE == WY_G);                 // B(kk, j) contiguous in j, except V^T[b][c] over c
     double ra[4], rb[4];
     auto fetch = [&](int k0) {
@@ -522,7 +525,8 @@ eig_wy_gemm_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict_
                     if (MODE == WY_G) v = wy_vt(S, k, nr, row, kk);
                     else if (MODE == WY_X) v = G[(int64_t)row * k + kk];
                     else if (MODE == WY_T12 || MODE == WY_M) v = (kk >= row) ? T[(int64_t)row * k + kk] : 0.0;
-                    else v = wy_vt(S, k, nr, kk, row);
+                    else if (MODE == WY_Q) v = wy_vt(S, k, nr, kk, row);
+                    else v = X[(int64_t)row * k + kk];
                 }
                 ra[l] = v;
             }
@@ -534,7 +538,8 @@ eig_wy_gemm_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict_
                     else if (MODE == WY_X) v = (kk <= col) ? T[(int64_t)kk * k + col] : 0.0;
                     else if (MODE == WY_T12) v = X[(int64_t)kk * k + col];
                     else if (MODE == WY_M) v = wy_vt(S, k, nr, kk, col);
-                    else v = G[(int64_t)kk * k + col];
+                    else if (MODE == WY_Q) v = G[(int64_t)kk * k + col];
+                    else v = T[(int64_t)kk * k + col];
                 }
                 rb[l] = v;
             }
@@ -578,7 +583,17 @@ eig_wy_gemm_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict_
                 else if (MODE == WY_X) X[(int64_t)row * k + col] = v;
                 else if (MODE == WY_T12) T[(int64_t)row * k + col] = -v;
                 else if (MODE == WY_M) G[(int64_t)row * k + col] = v;
-                else X[(int64_t)row * k + col] = ((row == col) ? 1.0 : 0.0) - v;
+                else if (MODE == WY_Q) X[(int64_t)row * k + col] = ((row == col) ? 1.0 : 0.0) - v;
+                else {
+                    // the leading r columns in descending eigenvalue order: Wu = W[:, :r], Wv = W[:, :r] / sqrt(lambda)
+                    const int rk = D.rank[col] & (RANK_MERGED - 1);
+                    if (rk < r_out) {
+                        const double lj = D.dvec[col];
+                        const double inv = (lj > 1e-300) ? 1.0 / sqrt(lj) : 0.0;
+                        D.Wu[(int64_t)row * r_out + rk] = (float)v;
+                        D.Wv[(int64_t)row * r_out + rk] = (float)(v * inv);
+                    }
+                }
             }
 }
 
@@ -908,17 +923,20 @@ eig_rot_systolic_kernel(const RefreshDev *__restrict__ rd, const RowItem *__rest
 #pragma unroll
     for (int q = 0; q < R; ++q) {
         const int row = min(row0 + q, k - 1);     // rows past the end shadow the last row, never stored
-        for (int c = lane; c < k; c += 32) z[q * k + c] = D.Wj[(int64_t)row * k + c];
+        // dc: rows of the identity (the kernel forms diag(Z1, Z2) G; Q is multiplied in afterwards); else rows of Q
+        for (int c = lane; c < k; c += 32) z[q * k + c] = dc ? ((c == row) ? 1.0 : 0.0) : D.Wj[(int64_t)row * k + c];
     }
     __syncwarp();
     if (!dc) {
         systolic_apply<R>(z, k, k, D.rot, D.groups, D.sweeps, D.nsweeps[0], lane);
     } else {
-        // rows of Q diag(Z1, Z2): each half of the columns through its own log
+        // rows of diag(Z1, Z2): a unit row lies in one half of the columns and only that half's log changes it
+        // (a group of rows that straddles the middle goes through both: zeros stay zeros)
         const int s = k / 2;
-        systolic_apply<R>(z, k, s, D.rot, D.groups, D.sweeps, D.nsweeps[0], lane);
-        systolic_apply<R>(z + s, k, k - s, D.rot + dc_rot_off(D), D.groups + dc_group_off(D), D.sweeps + dc_sweep_off(D),
-                          D.nsweeps[1], lane);
+        if (row0 < s) systolic_apply<R>(z, k, s, D.rot, D.groups, D.sweeps, D.nsweeps[0], lane);
+        if (row0 + R > s)
+            systolic_apply<R>(z + s, k, k - s, D.rot + dc_rot_off(D), D.groups + dc_group_off(D), D.sweeps + dc_sweep_off(D),
+                              D.nsweeps[1], lane);
         // deflation rotations (few), one row per lane
         const int nr = D.dc_info[1];
         if (lane < R) {
@@ -932,31 +950,18 @@ eig_rot_systolic_kernel(const RefreshDev *__restrict__ rd, const RowItem *__rest
             }
         }
         __syncwarp();
-        // The coordinates of the secular problem still have to be multiplied by Uhat: their values, gathered in
-        // the order of the secular problem, go back to this row of Wj for eig_merge_kernel.  The deflated
-        // coordinates are final: their columns are emitted here.
+        // Z = diag(Z1, Z2) G is done for this row.  The coordinates of the secular problem still have to be
+        // multiplied by Uhat: their values, gathered in the order of the secular problem, go to row `row` of S
+        // (free since Q was formed) for eig_merge_kernel; the other columns are final and go to Ztot (gpart).
         const int K = D.dc_info[0];
         const int32_t *__restrict__ nd = D.dc_nd;
 #pragma unroll
         for (int q = 0; q < R; ++q) {
             const int row = row0 + q;
-            if (row < k)
-                for (int i = lane; i < K; i += 32) D.Wj[(int64_t)row * k + i] = z[q * k + nd[i]];
-        }
-        for (int jj = lane; jj < k; jj += 32) {
-            const int rk = D.rank[jj];
-            if ((rk & RANK_MERGED) || rk >= r) continue;
-            const double lj = D.dvec[jj];
-            const double inv = (lj > 1e-300) ? 1.0 / sqrt(lj) : 0.0;
-#pragma unroll
-            for (int q = 0; q < R; ++q) {
-                const int row = row0 + q;
-                if (row < k) {
-                    const double w = z[q * k + jj];
-                    D.Wu[(int64_t)row * r + rk] = (float)w;
-                    D.Wv[(int64_t)row * r + rk] = (float)(w * inv);
-                }
-            }
+            if (row >= k) continue;
+            for (int i = lane; i < K; i += 32) D.S[(int64_t)row * k + i] = z[q * k + nd[i]];
+            for (int c = lane; c < k; c += 32)
+                if (!(D.rank[c] & RANK_MERGED)) D.gpart[(int64_t)row * k + c] = z[q * k + c];
         }
         return;
     }
@@ -980,11 +985,10 @@ eig_rot_systolic_kernel(const RefreshDev *__restrict__ rd, const RowItem *__rest
 }
 
 // Divide and conquer, step 4b: the coordinates of the secular problem times the merged eigenvector matrix,
-// Y = Zg Uhat (Zg: k x K, the rows the rotation kernel left in Wj; Uhat: K x K in Xw), on the FP64 tensor
+// Y = Zg Uhat (Zg: k x K, the rows the rotation kernel left in S; Uhat: K x K in Xw), on the FP64 tensor
 // path.  A CTA owns a 64 x 64 tile of Y, its eight warps 32 x 16 regions of it as 4 x 2 sub-tiles of 8 x 8
-// (mma m8n8k4); operands are staged 16 columns of Zg / rows of Uhat at a time.  Column j of Y is the
-// eigenvector column of coordinate nd[j]; the leading r columns by eigenvalue are written as Wu and,
-// scaled by 1 / sqrt(lambda), as Wv.
+// (mma m8n8k4); operands are staged 16 columns of Zg / rows of Uhat at a time.  Column j of Y is column
+// nd[j] of Ztot = diag(Z1, Z2) G Uhat (in gpart), whose other columns the rotation kernel wrote.
 
 __global__ void __launch_bounds__(256)
 eig_merge_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ list)
@@ -993,7 +997,7 @@ eig_merge_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ 
     const int k = D.k, r = D.r, K = D.dc_info[0];
     const int r0 = blockIdx.y * MG_T, c0 = blockIdx.x * MG_T;
     if (r0 >= k || c0 >= K) return;
-    const double *__restrict__ Zg = D.Wj;
+    const double *__restrict__ Zg = D.S;
     const double *__restrict__ Uh = D.Xw;
     __shared__ __align__(16) double As[MG_K][MG_PITCH];     // As[i][row] = Zg[r0 + row][i0 + i]
     __shared__ __align__(16) double Bs[MG_K][MG_PITCH];     // Bs[i][col] = Uhat[i0 + i][c0 + col]
@@ -1051,18 +1055,10 @@ eig_merge_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ 
             const int j = c0 + wj * 16 + b * 8 + 2 * q + h;
             if (j >= K) continue;
             const int cj = D.dc_nd[j];
-            const int rk = D.rank[cj] & (RANK_MERGED - 1);
-            if (rk >= r) continue;
-            const double lj = D.dvec[cj];
-            const double inv = (lj > 1e-300) ? 1.0 / sqrt(lj) : 0.0;
 #pragma unroll
             for (int a = 0; a < 4; ++a) {
                 const int row = r0 + wi * 32 + a * 8 + g;
-                if (row < k) {
-                    const double w = acc[a][b][h];
-                    D.Wu[(int64_t)row * r + rk] = (float)w;
-                    D.Wv[(int64_t)row * r + rk] = (float)(w * inv);
-                }
+                if (row < k) D.gpart[(int64_t)row * k + cj] = acc[a][b][h];
             }
         }
 }
@@ -1136,9 +1132,10 @@ cudaError_t eig_tridiag_batched(const RefreshDev *rd, const int32_t *list, int n
             if ((e = raise_smem(eig_rot_systolic_kernel<2>, sys_bytes, &sys2_cfg)) != cudaSuccess) return e;
             eig_rot_systolic_kernel<2><<<npanels, threads, sys_bytes, stream>>>(rd, panel_items, dc);
         }
-        if (dc) {
+        if (dc) {   // Ztot = diag(Z1, Z2) G Uhat, then W = Q Ztot
             const int t = (kmax + MG_T - 1) / MG_T;
             eig_merge_kernel<<<dim3(t, t, nlist), 256, 0, stream>>>(rd, list);
+            eig_wy_gemm_kernel<WY_W><<<dim3(t, t, nlist), 256, 0, stream>>>(rd, list, 0);
         }
         return cudaGetLastError();
     }
