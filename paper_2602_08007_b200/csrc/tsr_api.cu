@@ -252,20 +252,28 @@ void layout(tsr_ctx *ctx, Arena &a, bool assign, size_t *step_end)
 void add_tiles(tsr_ctx *ctx, int kind, int bi, int M, int N, int K, int kb_per_split, int tri = 0)
 {
     const int bn = ctx->bn[kind];
-    const int bm = (kind == KA || kind == KOA) ? 128 : 256;   // the grouped GEMM runs on CTA pairs: 256-row tiles
+    const bool apply = (kind == KA || kind == KOA);
+    const int bm = apply ? 128 : 256;   // the grouped GEMM runs on CTA pairs: 256-row tiles
     Block &b = ctx->blocks[bi];
     std::vector<UmmaTile> &v = ctx->tiles[kind];
     b.tile_begin[kind] = (int)v.size();
     const int nkb = (K + 63) / 64;
     const int nsp = kb_per_split > 0 ? (nkb + kb_per_split - 1) / kb_per_split : 1;
+    // Columns: the grouped GEMM takes tiles of any width that is a multiple of 16, so N is cut into equal parts
+    // (528 columns: three tiles of 176 instead of 256 + 256 + 16, whose narrow tile would cost a whole pass
+    // over the A operand); the apply kernel keeps full-width tiles.
+    const int ntn = (N + bn - 1) / bn;
+    int wn = bn;
+    if (!apply && ntn > 0) wn = std::min(bn, (((N + ntn - 1) / ntn) + 15) & ~15);
     for (int m0 = 0; m0 < M; m0 += bm)
-        for (int n0 = 0; n0 < N; n0 += bn)
+        for (int n0 = 0; n0 < N; n0 += wn)
             for (int s = 0; s < nsp; ++s) {
                 UmmaTile t;
                 t.prob = bi; t.m0 = m0; t.n0 = n0;
                 t.kb0 = kb_per_split > 0 ? s * kb_per_split : 0;
                 t.kb1 = kb_per_split > 0 ? std::min(nkb, (s + 1) * kb_per_split) : nkb;
-                if (tri > 0) t.kb1 = std::min(nkb, (n0 + bn + tri - 1) / tri);
+                t.nw = apply ? 0 : std::min(wn, ((N - n0) + 15) & ~15);
+                if (tri > 0) t.kb1 = std::min(nkb, (n0 + (apply ? bn : t.nw) + tri - 1) / tri);
                 t.split = s;
                 v.push_back(t);
             }

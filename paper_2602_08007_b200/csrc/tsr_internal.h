@@ -58,6 +58,7 @@ struct UmmaTile {
     int32_t m0, n0;        // element offsets of the tile
     int32_t kb0, kb1;      // range of 64-wide K blocks [kb0, kb1)
     int32_t split;         // split-K slab index (0 when not split)
+    int32_t nw;            // width of the tile in columns (a multiple of 16, at most the kernel's tile width); 0: the full width
 };
 
 struct StepScalars {       // per-step scalars shared by all blocks

@@ -108,7 +108,7 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
                 const UmmaTile tile = tiles[t];
                 const UmmaProblem *P = probs + tile.prob;
                 int n_eff = P->N - tile.n0;
-                n_eff = n_eff >= BN ? BN : ((n_eff + 15) & ~15);
+                n_eff = tile.nw > 0 ? tile.nw : (n_eff >= BN ? BN : ((n_eff + 15) & ~15));
                 const int b_row = tile.n0 + (int)rank * (n_eff / 2);   // this CTA's half of the B rows
                 for (int kb = tile.kb0; kb < tile.kb1; ++kb, ++it) {
                     const int s = it % STAGES;
@@ -136,7 +136,7 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
             for (int t = pair; t < num_tiles && ok; t += stride, ++tc) {
                 const UmmaTile tile = tiles[t];
                 int n_eff = probs[tile.prob].N - tile.n0;
-                n_eff = n_eff >= BN ? BN : ((n_eff + 15) & ~15);
+                n_eff = tile.nw > 0 ? tile.nw : (n_eff >= BN ? BN : ((n_eff + 15) & ~15));
                 const uint32_t idesc = PLANES == 3 ? umma_idesc_pair_tf32(n_eff) : umma_idesc_pair(n_eff);
                 const uint32_t buf = tc & 1u;
                 if (!mbar_wait(smem_u32(bar_acc_empty + buf), ((tc >> 1) & 1u) ^ 1u)) { s_timeout = 1; ok = false; break; }
@@ -188,6 +188,7 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
             const UmmaProblem *__restrict__ P = probs + tile.prob;
             const uint32_t buf = tc & 1u;
             const int N = P->N, M = P->M;
+            const int Nt = tile.nw > 0 ? min(N, tile.n0 + tile.nw) : N;   // first column past this tile
             const int row0 = tile.m0 + (int)rank * UM_BM + q * 32;   // this CTA holds rows 128 rank .. of the tile
             // a split-K problem inside a core-update launch only stores its slab
             const bool store_f32 = (EPI == EPI_STORE_F32) || (EPI == EPI_CORE_UPDATE && P->epilogue == EPI_STORE_F32);
@@ -208,7 +209,7 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
             tc_fence_after();
             const int nrows = min(32, M - row0);        // may be <= 0
             const int c_begin = half * (BN / 2), c_end = c_begin + BN / 2;
-            if (tile.n0 + c_begin >= N) {   // this warp's column half lies outside the matrix
+            if (tile.n0 + c_begin >= Nt) {   // this warp's column half lies outside the tile
                 tc_fence_before();
                 if (lane == 0) mbar_arrive_leader(smem_u32(bar_acc_empty + buf));
                 continue;
@@ -216,15 +217,15 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
 #pragma unroll 1
             for (int c0 = c_begin; c0 < c_end; c0 += 32) {
                 const int col0 = tile.n0 + c0;
-                if (col0 >= N) break;
+                if (col0 >= Nt) break;
                 uint32_t v[32];
                 tc_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + buf * BN + (uint32_t)c0, v);
-                if (c0 + 32 >= c_end || col0 + 32 >= N) {   // this warp's last chunk of the tile: release the accumulator
+                if (c0 + 32 >= c_end || col0 + 32 >= Nt) {   // this warp's last chunk of the tile: release the accumulator
                     tc_fence_before();
                     if (lane == 0) mbar_arrive_leader(smem_u32(bar_acc_empty + buf));
                 }
                 if (nrows <= 0) continue;
-                const int ncols = min(32, N - col0);
+                const int ncols = min(32, Nt - col0);
                 if (EPI == EPI_STORE_BF16_T) {
                     // out[col][row]: for a fixed column the 32 lanes hold 32 consecutive rows
                     bf16 *out = (bf16 *)P->out + (int64_t)col0 * P->ld_out + row0 + lane;
