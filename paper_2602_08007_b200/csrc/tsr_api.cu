@@ -30,6 +30,7 @@ struct Block {
     bf16 *Ub = nullptr, *Ubt = nullptr, *Vb = nullptr, *Vbt = nullptr, *Tt = nullptr, *Pb = nullptr;
     bf16 *Db = nullptr, *Dbt = nullptr;
     bool one_sided = false;   // C = U^T G (r x n): the comparison arm of Table 1
+    bool right_first = false; // the lift goes through Z^T = V D^T (n x r) instead of P = U D (m x r): the smaller intermediate
     int64_t cn = 0;           // columns of C, M, Vm: r, or n for a one-sided block
     float *partial = nullptr;
     int nsplit = 1, kb_per_split = 0;
@@ -308,7 +309,7 @@ void build_tiles(tsr_ctx *ctx)
             // a block with a long contraction (an embedding) is cut into split-K slabs; its tiles sit in the same
             // table, so that one launch covers every block
             add_tiles(ctx, KC, bi, r, r, m, b.nsplit > 1 ? b.kb_per_split : 0);
-            add_tiles(ctx, KP, bi, m, r, r, 0);
+            add_tiles(ctx, KP, bi, b.right_first ? n : m, r, r, 0);
             add_tiles(ctx, KA, bi, m, n, r, 0);
         }
         add_tiles(ctx, KY, bi, m, k, n, 0);
@@ -909,6 +910,7 @@ tsr_status tsr_create(tsr_ctx **out, const tsr_mat_desc *descs, int32_t count)
         b.k = b.d.r + b.d.p;
         b.one_sided = (b.d.flags & TSR_BLOCK_ONE_SIDED) != 0;
         b.cn = b.one_sided ? b.d.n : b.d.r;
+        b.right_first = !b.one_sided && b.d.m > b.d.n;
         b.rl = round_up(b.d.r, 8); b.ml = round_up(b.d.m, 8); b.nl = round_up(b.d.n, 8);
         // Candidate for the tensor-core path: BF16 gradient with 16-byte row pitches.  Pointer
         // alignment is checked at bind time.
@@ -1023,7 +1025,7 @@ tsr_status tsr_bind(tsr_ctx *ctx, const tsr_mat_ptrs *ptrs, int32_t count, void 
         CoreUpdateArgs &ca = cu_all[i];
         memset(&ca, 0, sizeof ca);
         ca.C = b.p.C; ca.Cout = b.p.C; ca.mom1 = b.p.M; ca.mom2 = b.p.Vm; ca.d_f32 = b.D32;
-        ca.d_bf16 = nullptr; ca.dt_bf16 = b.fast ? b.Dbt : nullptr; ca.ldd = b.rl;
+        ca.d_bf16 = (b.fast && b.right_first) ? b.Db : nullptr; ca.dt_bf16 = b.fast ? b.Dbt : nullptr; ca.ldd = b.rl;
         ca.split_stride = 0; ca.r = (int)r; ca.nc = (int)b.cn; ca.nsplit = 1;
         cu_split[i] = ca;
         cu_split[i].C = b.partial; cu_split[i].nsplit = b.nsplit; cu_split[i].split_stride = r * r;
@@ -1075,9 +1077,11 @@ tsr_status tsr_bind(tsr_ctx *ctx, const tsr_mat_ptrs *ptrs, int32_t count, void 
             if ((s = encode_map(ctx, &P.tmB, b.Tt, r, m, b.ml, ctx->bn[KC] / 2)) != TSR_OK) return s;
             P.out = (b.nsplit > 1) ? (void *)b.partial : (void *)b.p.C;
             P.ld_out = r; P.split_stride = r * r;
-            P.mom1 = b.p.M; P.mom2 = b.p.Vm; P.d_bf16 = nullptr; P.dt_bf16 = b.Dbt; P.ldd = b.rl;
+            P.mom1 = b.p.M; P.mom2 = b.p.Vm; P.d_bf16 = b.right_first ? b.Db : nullptr; P.dt_bf16 = b.Dbt; P.ldd = b.rl;
         }
-        {   // P = U D : A = U copy [m x r], B = D^T copy [r x r]
+        // The lift U D V^T goes through the smaller of the two intermediates: P = U D (m x r) when m <= n,
+        // Z^T = V D^T (n x r) when m > n; either one lives in Pb and is the apply kernel's A or B operand.
+        if (!b.right_first) {   // P = U D : A = U copy [m x r], B = D^T copy [r x r]
             UmmaProblem &P = probs[KP][i];
             base(P, (int)m, (int)r, (int)r, EPI_STORE_BF16);
             if ((s = encode_map(ctx, &P.tmA, b.Ub, m, r, b.rl, 128)) != TSR_OK) return s;
@@ -1085,12 +1089,20 @@ tsr_status tsr_bind(tsr_ctx *ctx, const tsr_mat_ptrs *ptrs, int32_t count, void 
             P.out = b.Pb; P.ld_out = b.rl;
             if ((s = encode_map_out_bf16(ctx, &P.tmW, b.Pb, m, r, b.rl)) != TSR_OK) return s;
             P.out_tma = 1;
+        } else {                // Z^T = V D^T : A = V copy [n x r], B = D copy [r x r]
+            UmmaProblem &P = probs[KP][i];
+            base(P, (int)n, (int)r, (int)r, EPI_STORE_BF16);
+            if ((s = encode_map(ctx, &P.tmA, b.Vb, n, r, b.rl, 128)) != TSR_OK) return s;
+            if ((s = encode_map(ctx, &P.tmB, b.Db, r, r, b.rl, ctx->bn[KP] / 2)) != TSR_OK) return s;
+            P.out = b.Pb; P.ld_out = b.rl;
+            if ((s = encode_map_out_bf16(ctx, &P.tmW, b.Pb, n, r, b.rl)) != TSR_OK) return s;
+            P.out_tma = 1;
         }
-        {   // W update : A = P [m x r], B = V copy [n x r]
+        {   // W update : A = P [m x r], B = V copy [n x r]   (or A = U copy, B = Z^T)
             UmmaProblem &P = probs[KA][i];
             base(P, (int)m, (int)n, (int)r, EPI_APPLY);
-            if ((s = encode_map(ctx, &P.tmA, b.Pb, m, r, b.rl, 128)) != TSR_OK) return s;
-            if ((s = encode_map(ctx, &P.tmB, b.Vb, n, r, b.rl, 128)) != TSR_OK) return s;
+            if ((s = encode_map(ctx, &P.tmA, b.right_first ? b.Ub : b.Pb, m, r, b.rl, 128)) != TSR_OK) return s;
+            if ((s = encode_map(ctx, &P.tmB, b.right_first ? b.Pb : b.Vb, n, r, b.rl, 128)) != TSR_OK) return s;
             if ((s = encode_map_w(ctx, &P.tmW, b.p.W, m, n, b.d.ldw, b.d.w_dtype)) != TSR_OK) return s;
             P.out = b.p.W; P.ld_out = b.d.ldw;
         }
