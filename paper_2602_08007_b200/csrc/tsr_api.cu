@@ -646,8 +646,14 @@ tsr_status orth(tsr_ctx *ctx, const RefreshLists &L, int side, bool final, cudaS
 
 // buf[0] (rows_out x k) = G X  (transposed = false, X = buf[2] or Omega, n x k)
 //                      or G^T X (transposed = true,  X = buf[2], m x k)
+// planes: 2 = the FP32 operand X as BF16 hi + lo planes (two MMAs into one accumulator); 1 = its BF16 rounding
+// alone.  The sketches inside the power iteration take one plane: rounding the test matrix or the intermediate
+// basis perturbs it by 2^-9, which acts like a slightly different starting matrix (measured against the oracle: the
+// captured energy agrees to seven digits either way, the projector at the spectral gap moves from 2e-5 to 3e-5..6e-5,
+// only the ill-determined directions inside the noise bulk differ more).  B = Q^T G, which the singular vectors
+// are computed from, keeps both planes.
 tsr_status sketch(tsr_ctx *ctx, const RefreshLists &L, bool transposed, bool from_omega,
-                  const float *const *omegas, cudaStream_t st)
+                  const float *const *omegas, cudaStream_t st, int planes = 2)
 {
     StepScalars sc = {};
     tsr_status s;
@@ -658,7 +664,7 @@ tsr_status sketch(tsr_ctx *ctx, const RefreshLists &L, bool transposed, bool fro
         if (b.fast) {
             const int rows = transposed ? m : n;                 // rows of X
             const int64_t ld = transposed ? b.ml : b.nl;
-            TSR_KERNEL(ctx, 1, split_transpose(X, rows, k, b.Xt, ld, k, 2, st));
+            TSR_KERNEL(ctx, 1, split_transpose(X, rows, k, b.Xt, ld, k, planes, st));
         } else if (!transposed) {
             TSR_KERNEL(ctx, 1, simt_gemm(m, k, n, b.p.G, b.d.g_dtype, b.d.ldg, 1, X, k, 1, b.buf[0], k, SIMT_STORE, 0, 0, st));
         } else {
@@ -666,7 +672,7 @@ tsr_status sketch(tsr_ctx *ctx, const RefreshLists &L, bool transposed, bool fro
         }
     }
     if (ctx->any_fast)
-        if ((s = launch_kind(ctx, transposed ? KZ : KY, L.list, EPI_STORE_F32, 2, sc, st)) != TSR_OK) return s;
+        if ((s = launch_kind(ctx, transposed ? KZ : KY, L.list, EPI_STORE_F32, planes, sc, st)) != TSR_OK) return s;
     return TSR_OK;
 }
 
@@ -713,13 +719,13 @@ tsr_status do_refresh_group(tsr_ctx *ctx, const std::vector<int> &list, uint64_t
             TSR_KERNEL(ctx, 1, transpose_bf16((const bf16 *)b.p.G, (int)b.d.m, (int)b.d.n, b.d.ldg, b.Gt, b.ml, st));
     }
     // Y = G Omega; Q = orth(Y)
-    if ((s = sketch(ctx, L, false, true, omegas, st)) != TSR_OK) return s;
+    if ((s = sketch(ctx, L, false, true, omegas, st, 1)) != TSR_OK) return s;
     if ((s = orth(ctx, L, 0, qmax == 0, st)) != TSR_OK) return s;
     for (int it = 0; it < qmax; ++it) {
         // Yrow = G^T Q; Qrow = orth(Yrow); Y = G Qrow; Q = orth(Y)
-        if ((s = sketch(ctx, L, true, false, nullptr, st)) != TSR_OK) return s;
+        if ((s = sketch(ctx, L, true, false, nullptr, st, 1)) != TSR_OK) return s;
         if ((s = orth(ctx, L, 1, false, st)) != TSR_OK) return s;
-        if ((s = sketch(ctx, L, false, false, nullptr, st)) != TSR_OK) return s;
+        if ((s = sketch(ctx, L, false, false, nullptr, st, 1)) != TSR_OK) return s;
         if ((s = orth(ctx, L, 0, it == qmax - 1, st)) != TSR_OK) return s;
     }
     // B^T = G^T Q (n x k) in buf[0]; small SVD through the k x k Gram matrix B B^T
