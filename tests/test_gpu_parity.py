@@ -484,3 +484,31 @@ def test_one_sided_arm_matches_oracle(dtype, shapes, tol, fuse):
     # bytes a worker would synchronize: r n for the one-sided blocks, r^2 for the others (Table 1)
     core, _ = plan.comm_bytes(1, 4)
     assert core == 4 * sum(s["r"] * (s["n"] if s.get("flags", 0) & 2 else s["r"]) for s in shapes)
+
+
+# ---- quality of the refreshed bases, with margins tighter than the gates ------------------------------
+@pytest.mark.parametrize("shape", [dict(m=1376, n=512, r=128, p=8, q=1), dict(m=1024, n=2736, r=256, p=8, q=1)])
+def test_refresh_quality_against_oracle(shape):
+    """The refresh rounds its intermediate bases to BF16 inside the power iteration (one operand plane);
+    what the method needs from it is checked here against the oracle's refresh of the same (G, Omega)
+    bits, with an order of magnitude of margin below the gates: the energy the bases capture, the
+    projectors on the signal directions, orthonormality."""
+    tsr, plan = _plan([shape], torch.bfloat16)
+    G64 = fill_gradient(plan, 0, 31)                     # signal rank 64, noise bulk below
+    r, k, gap = shape["r"], shape["r"] + shape["p"], 64
+    Om = ti.omega(shape["n"], k, 32).cuda()
+    plan.init_subspace(omegas=[Om])
+    torch.cuda.synchronize()
+    assert plan.poll_status() == [0]
+    U, V = to64(plan.U[0]), to64(plan.V[0])
+    Uo, Vo, sig = oracle.rsvd_refresh(G64, to64(Om), r, shape["q"])
+    assert np.linalg.norm(U.T @ U - np.eye(r)) < 1e-5 and np.linalg.norm(V.T @ V - np.eye(r)) < 1e-5
+    proj = lambda X: X @ X.T
+    assert np.linalg.norm(proj(U[:, :gap]) - proj(Uo[:, :gap])) < 2e-4
+    assert np.linalg.norm(proj(V[:, :gap]) - proj(Vo[:, :gap])) < 2e-4
+    # what is left of G outside the two subspaces, relative to G: the same as the oracle's to five digits
+    res = np.linalg.norm(G64 - U @ (U.T @ G64 @ V) @ V.T) / np.linalg.norm(G64)
+    res_o = np.linalg.norm(G64 - Uo @ (Uo.T @ G64 @ Vo) @ Vo.T) / np.linalg.norm(G64)
+    assert abs(res / res_o - 1) < 1e-4
+    core = U.T @ G64 @ V
+    assert np.abs(np.diag(core)[:gap] / sig[:gap] - 1).max() < 1e-5
