@@ -121,7 +121,8 @@ typedef struct {
 
 typedef struct {
     float lr, beta1, beta2, eps, weight_decay;
-    float scale;   /* multiplies the lifted update U D V^T only; 1 = Algorithm 1 as printed */
+    float scale;   /* multiplies the lifted update U D V^T only; 1 = Algorithm 1 as printed.
+                      TSR_RULE_SGD ignores scale and weight_decay (Algorithm 2 has neither). */
     int64_t step;  /* t >= 1: global step counter used for bias correction and refresh schedule */
     int32_t rule;  /* tsr_rule                                                          */
     int32_t reserved;
@@ -269,16 +270,44 @@ TSR_API tsr_status tsr_generate_omega(tsr_ctx *ctx, int32_t i, uint64_t seed, fl
 TSR_API tsr_status tsr_set_profiling(tsr_ctx *ctx, int32_t enable);
 TSR_API tsr_status tsr_get_stage_ms(tsr_ctx *ctx, float *ms, int32_t count);
 
+/* Limits of the device-side loops and waits, and one diagnostic switch.  (No passage of the
+ * paper corresponds to this call; it makes the device-detected conditions of this library
+ * observable.)  Defaults are in force until the first call; a zero field restores its default.
+ *   wait_clocks   bound, in SM clock ticks, of every wait a tensor-core kernel of this context
+ *                 performs on an mbarrier (default 4e9, about two seconds).  When it runs out the
+ *                 CTA gives up on its remaining tiles, releases its tensor memory and returns;
+ *                 every block that owns one of those tiles reads TSR_ERR_TIMEOUT at the next
+ *                 tsr_poll_status and its outputs of that call are undefined.
+ *   max_sweeps    limit of the small eigen-solver of the refresh (Jacobi sweeps for k < 200,
+ *                 QL iterations per eigenvalue above; defaults 40 / 60) for block sweep_block
+ *                 (-1: every block).  A solver that stops at the limit flags
+ *                 TSR_ERR_NOT_CONVERGED on that block; other blocks are not affected.
+ *   starve_block  -1 (off), or a block index: the first projection GEMM (T = G V) issues no
+ *                 loads for the tiles of that block, so that its consumers run into the bounded
+ *                 wait.  Nothing is in flight and no address is touched for those tiles.  It
+ *                 exists to exercise the time-out path and requires 0 < wait_clocks <= 1e8.
+ * Call it between compute calls of the context (it is synchronous).  Host struct. */
+typedef struct {
+    int64_t wait_clocks;
+    int32_t max_sweeps;
+    int32_t sweep_block;
+    int32_t starve_block;
+    int32_t reserved;
+} tsr_limits;
+TSR_API tsr_status tsr_set_limits(tsr_ctx *ctx, const tsr_limits *limits);
+
 /* Number of CUDA kernels this context has launched since tsr_create. */
 TSR_API tsr_status tsr_launch_count(const tsr_ctx *ctx, uint64_t *count);
 
 /* Core projection C = U^T G V of ONE block without any allocation.  (The paper has no
  * counterpart of this call; it exists for callers that cannot allocate device memory.)
  *
- * Who needs it: code that runs where cudaMalloc is off limits -- inside a host callback or a
- * region that must not synchronise the device, in a process whose memory is owned by another
- * framework's pool with nothing left to hand out, or under an allocator that forbids foreign
- * allocations -- and that cannot provide the scratch buffer tsr_bind asks for either.  Here the
+ * Who needs it: code that may neither allocate device memory nor synchronise the device -- a
+ * process whose memory is owned by another framework's pool with nothing left to hand out, an
+ * allocator that forbids foreign allocations, a region where cudaMalloc's implicit
+ * synchronisation is not acceptable -- and that cannot provide the scratch buffer tsr_bind asks
+ * for either.  (It still launches kernels, so it is not for use inside a stream host callback,
+ * where no CUDA call may be made.)  Here the
  * only scratch the computation needs, the m x r intermediate T = G V, sits in a fixed
  * TSR_STATIC_SCRATCH_FLOATS-element FP32 array inside the library image (4 MiB of device
  * memory per GPU that loads the library, held until the process exits).

@@ -53,6 +53,11 @@ class Hyper(ctypes.Structure):
                 ("rule", ctypes.c_int32), ("reserved", ctypes.c_int32)]
 
 
+class Limits(ctypes.Structure):
+    _fields_ = [("wait_clocks", ctypes.c_int64), ("max_sweeps", ctypes.c_int32), ("sweep_block", ctypes.c_int32),
+                ("starve_block", ctypes.c_int32), ("reserved", ctypes.c_int32)]
+
+
 EXPORTS = [
     "tsr_version", "tsr_status_string", "tsr_last_error", "tsr_create", "tsr_destroy", "tsr_workspace_bytes",
     "tsr_bind", "tsr_bases_changed", "tsr_init_subspace", "tsr_project_core", "tsr_adam_core_step",
@@ -61,6 +66,7 @@ EXPORTS = [
     "tsr_rsvd_refresh_grouped", "tsr_embed_step_grouped", "tsr_step_grouped", "tsr_step_grouped_host",
     "tsr_comm_bytes", "tsr_state_elems", "tsr_poll_status", "tsr_generate_omega", "tsr_block_uses_tensor_cores",
     "tsr_set_profiling", "tsr_get_stage_ms", "tsr_launch_count", "tsr_project_core_static", "tsr_dense_adamw",
+    "tsr_set_limits",
 ]
 
 
@@ -119,6 +125,7 @@ def lib():
         L.tsr_launch_count.argtypes = [vp, P(u64)]
         L.tsr_project_core_static.argtypes = [vp, i32, i64, i64, i64, vp, vp, i32, vp, vp]
         L.tsr_dense_adamw.argtypes = [P(DenseTensor), i32, P(Hyper), vp]
+        L.tsr_set_limits.argtypes = [vp, P(Limits)]
         _lib = L
     return _lib
 
@@ -154,8 +161,19 @@ def project_core_static(G: torch.Tensor, U: torch.Tensor, V: torch.Tensor, C: to
     """C = U^T G V through tsr_project_core_static: no context, no workspace, no allocation --
     for callers that are not allowed to allocate device memory.  G is a 2-D (possibly row-padded)
     FP32 or BF16 tensor, U (m x r), V (n x r) and C (r x r) dense FP32, all on the current device."""
+    if G.dim() != 2 or U.dim() != 2 or V.dim() != 2 or C.dim() != 2:
+        raise ValueError("G, U, V and C must be matrices")
     m, n = G.shape
     r = U.shape[1]
+    if G.dtype not in (torch.float32, torch.bfloat16) or G.stride(1) != 1 or G.stride(0) < n:
+        raise ValueError("G must be FP32 or BF16 with unit column stride")
+    if tuple(U.shape) != (m, r) or tuple(V.shape) != (n, r) or tuple(C.shape) != (r, r):
+        raise ValueError("shapes must be U (m, r), V (n, r), C (r, r) for G (m, n)")
+    for t in (U, V, C):
+        if t.dtype != torch.float32 or not t.is_contiguous():
+            raise ValueError("U, V and C must be contiguous FP32 tensors")
+    if not all(t.is_cuda and t.device == G.device for t in (G, U, V, C)):
+        raise ValueError("all tensors must live on the same CUDA device")
     dt = TSR_BF16 if G.dtype == torch.bfloat16 else TSR_F32
     rc = lib().tsr_project_core_static(ctypes.c_void_p(G.data_ptr()), dt, m, n, G.stride(0),
                                        ctypes.c_void_p(U.data_ptr()), ctypes.c_void_p(V.data_ptr()), r,
@@ -245,8 +263,9 @@ class Plan:
         nb = len(self.blocks)
         ptrs = (MatPtrs * nb)()
         for i in range(nb):
+            vm = None if self.Vm[i] is None else self.Vm[i].data_ptr()   # None: a block that only ever runs TSR_RULE_SGD
             ptrs[i] = MatPtrs(self.G[i].data_ptr(), self.W[i].data_ptr(), self.U[i].data_ptr(), self.V[i].data_ptr(),
-                              self.M[i].data_ptr(), self.Vm[i].data_ptr(), self.C[i].data_ptr())
+                              self.M[i].data_ptr(), vm, self.C[i].data_ptr())
         ws = self.workspace.data_ptr()
         ws_al = (ws + 255) // 256 * 256
         self._check(lib().tsr_bind(self.ctx, ptrs, nb, ctypes.c_void_p(ws_al), self.workspace.numel() - (ws_al - ws)))
@@ -327,6 +346,10 @@ class Plan:
         arr = (ctypes.c_int32 * nb)()
         self._check(lib().tsr_poll_status(self.ctx, arr, nb, _stream_ptr(stream)))
         return list(arr)
+
+    def set_limits(self, wait_clocks: int = 0, max_sweeps: int = 0, sweep_block: int = -1, starve_block: int = -1):
+        lim = Limits(wait_clocks, max_sweeps, sweep_block, starve_block, 0)
+        self._check(lib().tsr_set_limits(self.ctx, ctypes.byref(lim)))
 
     def set_profiling(self, enable: bool):
         self._check(lib().tsr_set_profiling(self.ctx, 1 if enable else 0))

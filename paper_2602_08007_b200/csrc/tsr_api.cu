@@ -110,6 +110,10 @@ struct tsr_ctx {
     static constexpr int NPIPE = 8;            // chunks of the pipelined host-buffer step
     cudaEvent_t ev_pipe_in[NPIPE] = {}, ev_pipe_done[NPIPE] = {};
     bool aux_ready = false;
+    // limits (tsr_set_limits)
+    long long wait_clocks = 0;                 // 0: the kernels' default budget
+    std::vector<int32_t> max_sweeps;           // per block; 0: the solvers' defaults
+    int starve_block = -1;                     // diagnostic: block whose first projection GEMM gets no loads
 };
 
 namespace {
@@ -389,9 +393,10 @@ tsr_status encode_map_w(tsr_ctx *ctx, CUtensorMap *out, const void *base, int64_
     return TSR_OK;
 }
 
-StepScalars make_scalars(const tsr_hyper *h)
+StepScalars make_scalars(const tsr_ctx *ctx, const tsr_hyper *h)
 {
     StepScalars sc;
+    sc.wait_clocks = ctx->wait_clocks;
     sc.beta1 = h->beta1; sc.beta2 = h->beta2; sc.eps = h->eps;
     sc.omb1 = (float)(1.0 - (double)h->beta1);
     sc.omb2 = (float)(1.0 - (double)h->beta2);
@@ -416,6 +421,18 @@ tsr_status check_hyper(tsr_ctx *ctx, const tsr_hyper *h)
     if (h->rule != TSR_RULE_ADAM && h->rule != TSR_RULE_SGD) return fail(ctx, TSR_ERR_INVALID_ARG, "unknown rule");
     if (!(h->beta1 >= 0.f && h->beta1 < 1.f) || !(h->beta2 >= 0.f && h->beta2 < 1.f))
         return fail(ctx, TSR_ERR_INVALID_ARG, "betas must lie in [0, 1)");
+    return TSR_OK;
+}
+
+// The Adam rule reads and writes the second moment of every listed block: a block bound with
+// Vm == NULL (allowed for callers that only ever use TSR_RULE_SGD) is an argument error here,
+// found before anything is launched.
+tsr_status check_rule_ptrs(tsr_ctx *ctx, const std::vector<int> &list, int rule)
+{
+    if (rule != TSR_RULE_ADAM) return TSR_OK;
+    for (int bi : list)
+        if (!ctx->blocks[bi].p.Vm)
+            return fail(ctx, TSR_ERR_INVALID_ARG, "block %d: TSR_RULE_ADAM needs a second-moment buffer (Vm is NULL)", bi);
     return TSR_OK;
 }
 
@@ -540,6 +557,7 @@ tsr_status do_project(tsr_ctx *ctx, const std::vector<int> &list, bool fuse, con
 tsr_status do_core_update(tsr_ctx *ctx, const std::vector<int> &list, const StepScalars &sc, cudaStream_t st)
 {
     tsr_status s;
+    if ((s = check_rule_ptrs(ctx, list, sc.rule)) != TSR_OK) return s;
     int max_r = 1, max_c = 1;
     for (int bi : list) {
         max_r = std::max(max_r, (int)ctx->blocks[bi].d.r);
@@ -619,6 +637,7 @@ tsr_status rows_product(tsr_ctx *ctx, const RefreshLists &L, int side, int src, 
                                               mat, L.kmax, st));
     StepScalars sc;
     memset(&sc, 0, sizeof sc);
+    sc.wait_clocks = ctx->wait_clocks;
     return launch_kind(ctx, kind, L.list, EPI_STORE_F32, 3, sc, st);
 }
 
@@ -656,6 +675,7 @@ tsr_status sketch(tsr_ctx *ctx, const RefreshLists &L, bool transposed, bool fro
                   const float *const *omegas, cudaStream_t st, int planes = 2)
 {
     StepScalars sc = {};
+    sc.wait_clocks = ctx->wait_clocks;
     tsr_status s;
     for (size_t j = 0; j < L.list.size(); ++j) {
         Block &b = ctx->blocks[L.list[j]];
@@ -784,20 +804,25 @@ tsr_status do_refresh(tsr_ctx *ctx, const std::vector<int> &list, uint64_t seed,
     TSR_CUDA(ctx, cudaEventRecord(ctx->ev_fork, st));
     size_t list_off = 0, item_off[5] = {0, 0, 0, 0, 0};
     tsr_status result = TSR_OK;
-    for (int g = 0; g < ngroup; ++g) {
+    for (int g = 0; g < ngroup && result == TSR_OK; ++g) {
         const size_t lo = perm.size() * g / ngroup, hi = perm.size() * (g + 1) / ngroup;
         std::vector<int> grp;
         std::vector<const float *> om;
         for (size_t i = lo; i < hi; ++i) { grp.push_back(list[perm[i]]); om.push_back(omegas ? omegas[perm[i]] : nullptr); }
-        TSR_CUDA(ctx, cudaStreamWaitEvent(ctx->aux[g], ctx->ev_fork, 0));
         // All groups start together: with eight groups of about twenty blocks the one-CTA-per-matrix
         // kernels of different groups drift apart by themselves, and a forced offset between the
         // groups only lengthened the critical path when it was measured.
-        tsr_status s = do_refresh_group(ctx, grp, seed, omegas ? om.data() : nullptr, ctx->aux[g], list_off, item_off,
-                                        reexpress);
-        if (s != TSR_OK && result == TSR_OK) result = s;
-        TSR_CUDA(ctx, cudaEventRecord(ctx->ev_join[g], ctx->aux[g]));
-        TSR_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_join[g], 0));
+        if (cudaStreamWaitEvent(ctx->aux[g], ctx->ev_fork, 0) != cudaSuccess)
+            result = fail(ctx, TSR_ERR_CUDA, "cudaStreamWaitEvent failed on a refresh side stream");
+        else
+            result = do_refresh_group(ctx, grp, seed, omegas ? om.data() : nullptr, ctx->aux[g], list_off, item_off, reexpress);
+        // The side stream is joined whether or not its group was issued completely: the caller's
+        // stream must not run ahead of (and the caller must not free buffers under) work in flight.
+        if (cudaEventRecord(ctx->ev_join[g], ctx->aux[g]) != cudaSuccess ||
+            cudaStreamWaitEvent(st, ctx->ev_join[g], 0) != cudaSuccess) {
+            cudaStreamSynchronize(ctx->aux[g]);
+            if (result == TSR_OK) result = fail(ctx, TSR_ERR_CUDA, "joining a refresh side stream failed");
+        }
         list_off += grp.size();
         for (int bi : grp) {
             const Block &b = ctx->blocks[bi];
@@ -826,6 +851,7 @@ tsr_status do_step(tsr_ctx *ctx, const std::vector<int> &list, const tsr_hyper *
                    cudaStream_t st)
 {
     tsr_status s;
+    if ((s = check_rule_ptrs(ctx, list, h->rule)) != TSR_OK) return s;
     if (ctx->profiling) TSR_CUDA(ctx, cudaEventRecord(ctx->ev[0], st));
     std::vector<int> due;
     for (int bi : list) {
@@ -842,7 +868,7 @@ tsr_status do_step(tsr_ctx *ctx, const std::vector<int> &list, const tsr_hyper *
             if ((s = do_refresh(ctx, grp, seed ^ ((uint64_t)h->step * 0x9E3779B97F4A7C15ull), nullptr, st, true)) != TSR_OK) return s;
         }
     }
-    const StepScalars sc = make_scalars(h);
+    const StepScalars sc = make_scalars(ctx, h);
     ctx->stage_stream = st;
     ctx->stage_next = 1;
     if (ctx->profiling) {
@@ -928,6 +954,7 @@ tsr_status tsr_create(tsr_ctx **out, const tsr_mat_desc *descs, int32_t count)
         ctx->max_k = std::max(ctx->max_k, b.k);
         ctx->order.push_back(i);
     }
+    ctx->max_sweeps.assign(count, 0);
     std::stable_sort(ctx->order.begin(), ctx->order.end(), [&](int a, int b) {
         return ctx->blocks[a].d.m * ctx->blocks[a].d.n > ctx->blocks[b].d.m * ctx->blocks[b].d.n;
     });
@@ -1044,6 +1071,7 @@ tsr_status tsr_bind(tsr_ctx *ctx, const tsr_mat_ptrs *ptrs, int32_t count, void 
         rd.Rinv = b.Rinv; rd.Wu = b.Wu; rd.Wv = b.Wv; rd.U = b.p.U; rd.V = b.p.V; rd.status = ctx->d_status + i;
         rd.tau = b.tau; rd.dvec = b.dvec; rd.evec = b.evec; rd.rot = b.rot; rd.sweeps = b.sweeps; rd.groups = b.groups; rd.nsweeps = b.nsweeps;
         rd.rank = b.rank; rd.rot_cap = b.rot_cap; rd.sweep_cap = b.sweep_cap;
+        rd.max_sweeps = ctx->max_sweeps[i];
         rd.dc_z = b.dc_z; rd.dc_nd = b.dc_nd; rd.dc_rot_idx = b.dc_rot_idx; rd.dc_rot_cs = b.dc_rot_cs;
         rd.dc_scal = b.dc_scal; rd.dc_info = b.dc_info;
         if (!b.fast) continue;
@@ -1074,6 +1102,7 @@ tsr_status tsr_bind(tsr_ctx *ctx, const tsr_mat_ptrs *ptrs, int32_t count, void 
             if ((s = encode_map(ctx, &P.tmA, b.p.G, m, n, b.d.ldg, 128)) != TSR_OK) return s;
             if ((s = encode_map(ctx, &P.tmB, b.Vbt, r, n, b.nl, ctx->bn[KT] / 2)) != TSR_OK) return s;
             P.out = b.Tt; P.ld_out = b.ml;
+            P.starve = (ctx->starve_block == i) ? 1 : 0;
         }
         {   // C = U^T T : A = U^T copy [r x m], B = T~ [r x m].  A split-K block only stores its slabs
             // (the sum and the core update follow in core_update_kernel), whatever epilogue the launch has.
@@ -1226,6 +1255,7 @@ tsr_status tsr_project_core_grouped(tsr_ctx *ctx, const int32_t *idx, int32_t co
     std::vector<int> list;
     if ((s = resolve_list(ctx, idx, count, list)) != TSR_OK) return s;
     StepScalars sc = {};
+    sc.wait_clocks = ctx->wait_clocks;
     return do_project(ctx, list, false, sc, (cudaStream_t)stream);
 }
 
@@ -1237,7 +1267,7 @@ tsr_status tsr_adam_core_step_grouped(tsr_ctx *ctx, const int32_t *idx, int32_t 
     if ((s = check_hyper(ctx, hyper)) != TSR_OK) return s;
     std::vector<int> list;
     if ((s = resolve_list(ctx, idx, count, list)) != TSR_OK) return s;
-    return do_core_update(ctx, list, make_scalars(hyper), (cudaStream_t)stream);
+    return do_core_update(ctx, list, make_scalars(ctx, hyper), (cudaStream_t)stream);
 }
 
 tsr_status tsr_backproject_apply_grouped(tsr_ctx *ctx, const int32_t *idx, int32_t count, const tsr_hyper *hyper,
@@ -1248,7 +1278,7 @@ tsr_status tsr_backproject_apply_grouped(tsr_ctx *ctx, const int32_t *idx, int32
     if ((s = check_hyper(ctx, hyper)) != TSR_OK) return s;
     std::vector<int> list;
     if ((s = resolve_list(ctx, idx, count, list)) != TSR_OK) return s;
-    return do_apply(ctx, list, make_scalars(hyper), (cudaStream_t)stream);
+    return do_apply(ctx, list, make_scalars(ctx, hyper), (cudaStream_t)stream);
 }
 
 tsr_status tsr_embed_step_grouped(tsr_ctx *ctx, const int32_t *idx, int32_t count, const tsr_hyper *hyper,
@@ -1287,6 +1317,11 @@ tsr_status tsr_step_grouped_host(tsr_ctx *ctx, const void *const *G_host, float 
     if ((s = check_hyper(ctx, hyper)) != TSR_OK) return s;
     cudaStream_t st = (cudaStream_t)stream;
     const int nb = (int)ctx->blocks.size();
+    {
+        std::vector<int> all;
+        resolve_list(ctx, nullptr, 0, all);
+        if ((s = check_rule_ptrs(ctx, all, hyper->rule)) != TSR_OK) return s;
+    }
     bool refresh_due = false;
     for (int i = 0; i < nb; ++i) {
         const Block &b = ctx->blocks[i];
@@ -1311,11 +1346,15 @@ tsr_status tsr_step_grouped_host(tsr_ctx *ctx, const void *const *G_host, float 
     constexpr int NCHUNK = tsr_ctx::NPIPE;
     if (refresh_due || !ctx->aux_ready || nb < 2 * NCHUNK) {
         // plain order: all gradients in, the step, all cores out
-        for (int i = 0; i < nb; ++i) TSR_CUDA(ctx, copy_in(i, st));
-        if ((s = tsr_step_grouped(ctx, hyper, seed, fuse_adam, stream)) != TSR_OK) return s;
-        if (C_host)
-            for (int i = 0; i < nb; ++i) TSR_CUDA(ctx, copy_out(i, st));
-        TSR_CUDA(ctx, cudaStreamSynchronize(st));
+        cudaError_t e = cudaSuccess;
+        for (int i = 0; i < nb && e == cudaSuccess; ++i) e = copy_in(i, st);
+        s = (e == cudaSuccess) ? tsr_step_grouped(ctx, hyper, seed, fuse_adam, stream) : TSR_OK;
+        if (C_host && s == TSR_OK)
+            for (int i = 0; i < nb && e == cudaSuccess; ++i) e = copy_out(i, st);
+        const cudaError_t es = cudaStreamSynchronize(st);   // also on failure: nothing stays in flight on the host buffers
+        if (s != TSR_OK) return s;
+        if (e != cudaSuccess || es != cudaSuccess)
+            return fail(ctx, TSR_ERR_CUDA, "host-buffer step failed: %s", cudaGetErrorString(e != cudaSuccess ? e : es));
         return TSR_OK;
     }
     // Pipelined order (no refresh in this step): the blocks go in chunks of about equal gradient bytes;
@@ -1334,27 +1373,37 @@ tsr_status tsr_step_grouped_host(tsr_ctx *ctx, const void *const *G_host, float 
         }
     }
     cudaStream_t s_in = ctx->aux[0], s_out = ctx->aux[1];
-    TSR_CUDA(ctx, cudaEventRecord(ctx->ev_fork, st));
-    TSR_CUDA(ctx, cudaStreamWaitEvent(s_in, ctx->ev_fork, 0));
-    TSR_CUDA(ctx, cudaStreamWaitEvent(s_out, ctx->ev_fork, 0));
-    for (int c = 0; c < NCHUNK; ++c) {
-        for (int bi : chunks[c]) TSR_CUDA(ctx, copy_in(bi, s_in));
-        TSR_CUDA(ctx, cudaEventRecord(ctx->ev_pipe_in[c], s_in));
-    }
+    // After the fork every exit, the failing ones included, waits for the side streams and the
+    // caller's stream: copies from G_host or into C_host must not be in flight when the call returns.
     tsr_status result = TSR_OK;
-    for (int c = 0; c < NCHUNK; ++c) {
+    auto cuda_ok = [&](cudaError_t e, const char *what) {
+        if (e != cudaSuccess && result == TSR_OK) result = fail(ctx, TSR_ERR_CUDA, "%s failed: %s", what, cudaGetErrorString(e));
+        return e == cudaSuccess;
+    };
+    bool go = cuda_ok(cudaEventRecord(ctx->ev_fork, st), "cudaEventRecord") &&
+              cuda_ok(cudaStreamWaitEvent(s_in, ctx->ev_fork, 0), "cudaStreamWaitEvent") &&
+              cuda_ok(cudaStreamWaitEvent(s_out, ctx->ev_fork, 0), "cudaStreamWaitEvent");
+    for (int c = 0; c < NCHUNK && go; ++c) {
+        for (int bi : chunks[c]) go = go && cuda_ok(copy_in(bi, s_in), "gradient copy");
+        go = go && cuda_ok(cudaEventRecord(ctx->ev_pipe_in[c], s_in), "cudaEventRecord");
+    }
+    for (int c = 0; c < NCHUNK && go; ++c) {
         if (chunks[c].empty()) continue;
-        TSR_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_pipe_in[c], 0));
-        if ((s = do_step(ctx, chunks[c], hyper, seed, fuse_adam != 0, st)) != TSR_OK && result == TSR_OK) result = s;
+        go = cuda_ok(cudaStreamWaitEvent(st, ctx->ev_pipe_in[c], 0), "cudaStreamWaitEvent");
+        if (!go) break;
+        if ((s = do_step(ctx, chunks[c], hyper, seed, fuse_adam != 0, st)) != TSR_OK) {
+            if (result == TSR_OK) result = s;
+            break;
+        }
         if (C_host) {
-            TSR_CUDA(ctx, cudaEventRecord(ctx->ev_pipe_done[c], st));
-            TSR_CUDA(ctx, cudaStreamWaitEvent(s_out, ctx->ev_pipe_done[c], 0));
-            for (int bi : chunks[c]) TSR_CUDA(ctx, copy_out(bi, s_out));
+            go = cuda_ok(cudaEventRecord(ctx->ev_pipe_done[c], st), "cudaEventRecord") &&
+                 cuda_ok(cudaStreamWaitEvent(s_out, ctx->ev_pipe_done[c], 0), "cudaStreamWaitEvent");
+            for (int bi : chunks[c]) go = go && cuda_ok(copy_out(bi, s_out), "core copy");
         }
     }
-    TSR_CUDA(ctx, cudaEventRecord(ctx->ev_join[0], s_out));
-    TSR_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_join[0], 0));
-    TSR_CUDA(ctx, cudaStreamSynchronize(st));
+    cuda_ok(cudaStreamSynchronize(s_in), "cudaStreamSynchronize");
+    cuda_ok(cudaStreamSynchronize(s_out), "cudaStreamSynchronize");
+    cuda_ok(cudaStreamSynchronize(st), "cudaStreamSynchronize");
     return result;
 }
 
@@ -1428,6 +1477,33 @@ tsr_status tsr_generate_omega(tsr_ctx *ctx, int32_t i, uint64_t seed, float *out
     if (cudaGetDeviceCount(&dev_count) != cudaSuccess || dev_count <= 0) return fail(ctx, TSR_ERR_CUDA, "no CUDA device available");
     const Block &b = ctx->blocks[i];
     TSR_KERNEL(ctx, 1, fill_gaussian(out, (int64_t)b.d.n * b.k, seed, (uint64_t)i, (cudaStream_t)stream));
+    return TSR_OK;
+}
+
+tsr_status tsr_set_limits(tsr_ctx *ctx, const tsr_limits *lim)
+{
+    if (!ctx) return TSR_ERR_INVALID_ARG;
+    if (!lim) return fail(ctx, TSR_ERR_INVALID_ARG, "limits is NULL");
+    const int nb = (int)ctx->blocks.size();
+    if (lim->wait_clocks < 0 || lim->max_sweeps < 0 || lim->sweep_block < -1 || lim->sweep_block >= nb ||
+        lim->starve_block < -1 || lim->starve_block >= nb)
+        return fail(ctx, TSR_ERR_INVALID_ARG, "limit out of range");
+    if (lim->starve_block >= 0 && (lim->wait_clocks <= 0 || lim->wait_clocks > 100000000ll))
+        return fail(ctx, TSR_ERR_INVALID_ARG, "starve_block needs a wait budget of at most 1e8 clock ticks");
+    ctx->wait_clocks = lim->wait_clocks;
+    for (int i = 0; i < nb; ++i)
+        if (lim->sweep_block < 0 || lim->sweep_block == i) ctx->max_sweeps[i] = lim->max_sweeps;
+    ctx->starve_block = lim->starve_block;
+    if (!ctx->bound) return TSR_OK;   // tsr_bind writes the device tables from these values
+    // refresh the two fields inside the device tables (the device is idle with respect to this
+    // context by contract: limits are set between calls, and the copies below are synchronous)
+    for (int i = 0; i < nb; ++i) {
+        TSR_CUDA(ctx, cudaMemcpy(&ctx->d_refresh[i].max_sweeps, &ctx->max_sweeps[i], sizeof(int32_t), cudaMemcpyHostToDevice));
+        if (ctx->blocks[i].fast) {
+            const int32_t sv = (ctx->starve_block == i) ? 1 : 0;
+            TSR_CUDA(ctx, cudaMemcpy(&ctx->d_probs[KT][i].starve, &sv, sizeof(int32_t), cudaMemcpyHostToDevice));
+        }
+    }
     return TSR_OK;
 }
 

@@ -23,11 +23,6 @@ namespace tsr {
 
 constexpr int TR_THREADS = 512;
 constexpr int TR_NB = 8;          // columns per panel
-#ifdef TR_PROFILE
-#define TR_TICK(slot) do { if (threadIdx.x == 0 && blockIdx.x == 0) { const long long t_ = clock64(); tr_prof[slot] += t_ - tr_t0; tr_t0 = t_; } } while (0)
-#else
-#define TR_TICK(slot) do { } while (0)
-#endif
 
 // D (8 x 8, two entries per lane) += A (8 x 4) B (4 x 8) on the FP64 tensor path
 __device__ __forceinline__ void dmma_f64(double &c0, double &c1, double a, double b)
@@ -75,9 +70,6 @@ tridiag_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ li
         return t;   // every thread of every warp holds the total
     };
 
-#ifdef TR_PROFILE
-    long long tr_t0 = clock64();
-#endif
     for (int j0 = 0; j0 + 2 < k; j0 += TR_NB) {
         const int L0 = k - j0;
         const int nbc = min(TR_NB, k - 2 - j0);  // columns of this panel that get a reflector
@@ -96,7 +88,6 @@ tridiag_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ li
             double dj = A[(int64_t)j * k + j];   // current diagonal entry (every thread computes it)
             for (int u = 0; u < c; ++u) dj -= 2.0 * Vp[u * kpad + c] * Wp[u * kpad + c];
             const double nrm2 = block_sum(part);
-            TR_TICK(0);
             const double x0 = vs[0];
             const double nrm = sqrt(nrm2);
             const double tail2 = nrm2 - x0 * x0;
@@ -117,7 +108,6 @@ tridiag_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ li
             }
             if (tid == 0) { d.tau[j] = tau; d.dvec[j] = dj; d.evec[j] = alpha; }
             __syncthreads();
-            TR_TICK(1);
             // ps = T0[c+1.., c+1..] v   (row-wise dot products; a warp takes four rows at a time and four
             // 32-column segments of each per trip, so that sixteen loads are in flight per lane; the four
             // sums are then reduced together: two exchange steps leave one sum per group of eight lanes)
@@ -167,7 +157,6 @@ tridiag_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ li
                 if (lane == 0) dots[warp] = acc;
             }
             __syncthreads();
-            TR_TICK(2);
             // p = tau (T0 v - sum_i (v_i (w_i . v) + w_i (v_i . v)))
             part = 0.0;
             for (int a = tid; a < len; a += nt) {
@@ -179,7 +168,6 @@ tridiag_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ li
                 part += acc * vs[a];
             }
             const double pv = block_sum(part);
-            TR_TICK(3);
             const double kk = 0.5 * tau * pv;
             for (int t = tid; t < L0; t += nt) {   // the new pair, zero where the reflector does not act
                 const int a = t - c - 1;
@@ -187,7 +175,6 @@ tridiag_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ li
                 Wp[c * kpad + t] = (a >= 0) ? ps[a] - kk * vs[a] : 0.0;
             }
             __syncthreads();
-            TR_TICK(4);
         }
         // T0[s][t] -= sum_i (v_i[s] w_i[t] + w_i[s] v_i[t]) for s, t >= nbc: a rank-16 update [V W] [W V]^T on
         // the FP64 tensor path (mma m8n8k4, four steps), 8 x 8 tiles, a row of tiles per warp, eight tiles
@@ -252,7 +239,6 @@ tridiag_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ li
                 }
         }
         __syncthreads();
-        TR_TICK(5);
     }
     if (tid == 0) {
         if (k >= 2) {
@@ -299,7 +285,7 @@ __device__ __forceinline__ double rsqrt_nocheck(double x)
 // One QL problem: d[0..n), e[0..n) (e[n-1] is not used) in shared memory, run by one thread.
 // Returns the number of sweeps logged, or -1 when a budget ran out.
 __device__ int ql_run(double *d, double *e, int n, double2 *__restrict__ rot, int64_t rot_cap, int2 *__restrict__ sweeps,
-                      int sweep_cap, int2 *__restrict__ groups)
+                      int sweep_cap, int2 *__restrict__ groups, int iter_limit)
 {
     int nrot = 0, nsw = 0;
     int64_t next_row = 0;                     // first free row of the skewed log
@@ -313,7 +299,7 @@ __device__ int ql_run(double *d, double *e, int n, double2 *__restrict__ rot, in
                 if (fabs(e[m]) <= QL_TOL * dd) break;
             }
             if (m == l) break;
-            if (++iter > 60 || nsw >= sweep_cap) return -1;
+            if (++iter > iter_limit || nsw >= sweep_cap) return -1;
             {
                 const int t = nsw & 31;
                 if (t == 0) {                 // a new group starts with this sweep
@@ -404,7 +390,7 @@ ql_log_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ lis
         const int scap = dc ? D.sweep_cap / 2 : D.sweep_cap;
         const int gcap = D.sweep_cap / 64 + 2;                                           // group slots per half
         const int nsw = ql_run(d + off, e + off, nh, D.rot + (warp ? rcap : 0), rcap, D.sweeps + (warp ? scap : 0), scap,
-                               D.groups + (warp ? gcap : 0));
+                               D.groups + (warp ? gcap : 0), D.max_sweeps > 0 ? D.max_sweeps : 60);
         D.nsweeps[warp] = nsw < 0 ? 0 : nsw;
         if (!dc) D.nsweeps[1] = 0;
         if (nsw < 0) atomicMax(D.status, (int)TSR_ERR_NOT_CONVERGED);

@@ -51,6 +51,7 @@ struct alignas(64) UmmaProblem {
     bf16 *dt_bf16;         // D^T [r x ldd]
     int64_t ldd;
     int32_t out_tma;       // EPI_STORE_BF16: tmW describes the output, chunks leave through TMA stores
+    int32_t starve;        // diagnostic (tsr_set_limits): the producer issues no loads for this problem's tiles
 };
 
 struct UmmaTile {
@@ -68,6 +69,7 @@ struct StepScalars {       // per-step scalars shared by all blocks
     float decay;            // 1 - lr * weight_decay
     float step_scale;       // lr * scale
     int32_t rule;           // tsr_rule
+    long long wait_clocks;  // bound of every device-side wait in SM clock ticks; <= 0: the default
 };
 
 // Launchers (tsr_umma.cu).  tiles / probs are device pointers.  bn = 128 or 256 (tile width).
@@ -146,6 +148,7 @@ struct RefreshDev {
     int32_t *nsweeps;            // number of logged sweeps
     int32_t *rank;               // k: descending rank of each eigenvalue
     int32_t rot_cap, sweep_cap;
+    int32_t max_sweeps;          // eigen-solver limit (Jacobi sweeps / QL iterations per eigenvalue); <= 0: the default
     // divide-and-conquer merge of the two halves of the tridiagonal problem (tsr_eig.cu)
     double *dc_z;                // k: the rank-one vector in the basis of the halves' eigenvectors
     int32_t *dc_nd;              // coordinates that take part in the secular problem, ascending eigenvalue

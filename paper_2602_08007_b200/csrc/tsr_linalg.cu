@@ -160,11 +160,6 @@ cudaError_t gram_batched(const RefreshDev *rd, const RowItem *items, int nitems,
 // ---------------------------------------------------------------------------------------
 constexpr int CH_NB = 16;
 constexpr int CH_THREADS = 512;
-#ifdef CH_PROFILE
-#define CH_TICK(slot) do { if (threadIdx.x == 0 && blockIdx.x == 0) { const long long t_ = clock64(); ch_prof[slot] += t_ - ch_t0; ch_t0 = t_; } } while (0)
-#else
-#define CH_TICK(slot) do { } while (0)
-#endif
 
 __global__ void __launch_bounds__(CH_THREADS)
 chol_inverse_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ list, int kpad)
@@ -200,9 +195,6 @@ chol_inverse_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict
         }
     }
     __syncthreads();
-#ifdef CH_PROFILE
-    long long ch_t0 = clock64();
-#endif
     // ---- factorisation
     for (int jb = 0; jb < k; jb += CH_NB) {
         const int nb = min(CH_NB, k - jb);
@@ -212,7 +204,6 @@ chol_inverse_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict
             P[j * kpad + c] = (c >= j) ? S[(int64_t)(jb + j) * k + jb + c] : 0.0;
         }
         __syncthreads();
-        CH_TICK(0);
         if (warp == 0) {
             // The nb x nb diagonal block and its inverse, in registers: lane c (< 16) holds column c of the
             // block; row j of the factor reaches the other lanes by shuffles (all loops unrolled, so every
@@ -266,7 +257,6 @@ chol_inverse_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict
             }
         }
         __syncthreads();
-        CH_TICK(1);
         {   // R12 = R11^{-T} S12 on the FP64 tensor path: (16 x 16 lower triangular) times 16 x 8 column tiles,
             // in place (a tile's columns belong to one warp, which reads them before it writes)
             const int g = lane >> 2, q = lane & 3;
@@ -291,12 +281,10 @@ chol_inverse_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict
             }
         }
         __syncthreads();
-        CH_TICK(2);
         for (int e = tid; e < nb * w; e += nt) {    // the finished rows of R
             const int j = e / w, c = e - j * w;
             if (c >= j) S[(int64_t)(jb + j) * k + jb + c] = P[j * kpad + c];
         }
-        CH_TICK(8);
         // rank-nb update of the trailing upper triangle on the FP64 tensor path: S22 -= R12^T R12 in
         // 8 x 8 tiles (mma m8n8k4, four steps over the 16 panel rows).  A warp owns the row tiles
         // warp, warp + nwarps, ... and takes eight column tiles per trip, all their loads issued
@@ -354,9 +342,7 @@ chol_inverse_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict
                 }
             }
         }
-        CH_TICK(9);
         __syncthreads();
-        CH_TICK(3);
     }
     // ---- X = R^{-1}, block rows from the bottom up (the diagonal blocks are already in place)
     const int nblk = (k + CH_NB - 1) / CH_NB;
@@ -373,7 +359,6 @@ chol_inverse_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict
             dinv[i][c] = (i < nb && c < nb && c >= i) ? X[(int64_t)(i0 + i) * k + i0 + c] : 0.0;
         }
         __syncthreads();
-        CH_TICK(4);
         {   // acc = R[I][l0 ..] X[l0 .., c] on the FP64 tensor path: a warp owns 16 x 8 tiles of columns
             // (two mma row tiles) and runs over l in steps of four; X is zero below its diagonal, so the
             // sum stops at the last column of the tile.  Eight steps of X values are in flight per lane.
@@ -407,7 +392,6 @@ chol_inverse_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict
 #pragma unroll
                     for (int pp = 0; pp < 8; ++pp) bq[pp] = nq[pp];
                 }
-                CH_TICK(5);
                 // X[I][c] = -R11^{-1} acc: the tile goes through the patch to become the B operand
                 patch[g * 8 + 2 * q] = lo0; patch[g * 8 + 2 * q + 1] = lo1;
                 patch[(8 + g) * 8 + 2 * q] = hi0; patch[(8 + g) * 8 + 2 * q + 1] = hi1;
@@ -433,7 +417,6 @@ chol_inverse_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict
                     }
                 }
                 __syncwarp();
-                CH_TICK(6);
             }
         }
         for (int e = tid; e < nb * i0; e += nt) {    // zeros left of the diagonal block
@@ -442,7 +425,6 @@ chol_inverse_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict
             d.Rinv[(int64_t)(i0 + j) * k + c] = 0.f;
         }
         __syncthreads();
-        CH_TICK(7);
     }
     if (tid == 0 && s_flag != 0) atomicMax(d.status, s_flag);
 }
@@ -771,7 +753,8 @@ jacobi_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ lis
     __syncthreads();
 
     bool converged = false;
-    for (int sweep = 0; sweep < max_sweeps && !converged; ++sweep) {
+    const int sweep_limit = d.max_sweeps > 0 ? d.max_sweeps : max_sweeps;   // per-block limit, when one was set
+    for (int sweep = 0; sweep < sweep_limit && !converged; ++sweep) {
         if (tid == 0) s_rot = 0;
         __syncthreads();
         for (int round = 0; round < ke - 1; ++round) {

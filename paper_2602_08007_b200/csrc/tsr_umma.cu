@@ -75,9 +75,10 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
     uint64_t *bar_full = bars, *bar_empty = bars + STAGES;
     uint64_t *bar_acc_full = bars + 2 * STAGES, *bar_acc_empty = bar_acc_full + 2;
     uint32_t *tmem_slot = (uint32_t *)(bars + SM::NBARS);
-    __shared__ int s_timeout;
+    __shared__ int s_timeout;   // 0, or 1 + the first tile (table index) this CTA gave up on
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const long long budget = wait_budget(sc);
     const uint32_t rank = cluster_ctarank();          // 0 = leader of the CTA pair
     const int pair = blockIdx.x >> 1;
     const int stride = gridDim.x >> 1;
@@ -107,13 +108,17 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
             for (int t = pair; t < num_tiles && ok; t += stride) {
                 const UmmaTile tile = tiles[t];
                 const UmmaProblem *P = probs + tile.prob;
+                if (P->starve) {   // diagnostic: nothing is loaded for this tile, so every consumer's bounded wait runs out
+                    note_timeout(&s_timeout, t);
+                    break;
+                }
                 int n_eff = P->N - tile.n0;
                 n_eff = tile.nw > 0 ? tile.nw : (n_eff >= BN ? BN : ((n_eff + 15) & ~15));
                 const int b_row = tile.n0 + (int)rank * (n_eff / 2);   // this CTA's half of the B rows
                 for (int kb = tile.kb0; kb < tile.kb1; ++kb, ++it) {
                     const int s = it % STAGES;
                     const uint32_t ph = (it / STAGES) & 1u;
-                    if (!mbar_wait(smem_u32(bar_empty + s), ph ^ 1u)) { s_timeout = 1; ok = false; break; }
+                    if (!mbar_wait(smem_u32(bar_empty + s), ph ^ 1u, budget)) { note_timeout(&s_timeout, t); ok = false; break; }
                     // both CTAs' copies report their bytes to the leader's "full" barrier
                     const uint32_t full = leader_addr(smem_u32(bar_full + s));
                     if (rank == 0) mbar_expect_tx(smem_u32(bar_full + s), 2u * (uint32_t)SM::STAGE_BYTES);
@@ -139,13 +144,13 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
                 n_eff = tile.nw > 0 ? tile.nw : (n_eff >= BN ? BN : ((n_eff + 15) & ~15));
                 const uint32_t idesc = PLANES == 3 ? umma_idesc_pair_tf32(n_eff) : umma_idesc_pair(n_eff);
                 const uint32_t buf = tc & 1u;
-                if (!mbar_wait(smem_u32(bar_acc_empty + buf), ((tc >> 1) & 1u) ^ 1u)) { s_timeout = 1; ok = false; break; }
+                if (!mbar_wait(smem_u32(bar_acc_empty + buf), ((tc >> 1) & 1u) ^ 1u, budget)) { note_timeout(&s_timeout, t); ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + buf * BN;
                 for (int kb = tile.kb0; kb < tile.kb1; ++kb, ++it) {
                     const int s = it % STAGES;
                     const uint32_t ph = (it / STAGES) & 1u;
-                    if (!mbar_wait(smem_u32(bar_full + s), ph)) { s_timeout = 1; ok = false; break; }
+                    if (!mbar_wait(smem_u32(bar_full + s), ph, budget)) { note_timeout(&s_timeout, t); ok = false; break; }
                     tc_fence_after();
                     const uint32_t a_base = smem_u32(smem + s * SM::STAGE_BYTES);
                     if (PLANES == 3) {
@@ -205,7 +210,7 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
                     }
                 }
             }
-            if (!mbar_wait(smem_u32(bar_acc_full + buf), (tc >> 1) & 1u)) { s_timeout = 1; ok = false; break; }
+            if (!mbar_wait(smem_u32(bar_acc_full + buf), (tc >> 1) & 1u, budget)) { note_timeout(&s_timeout, t); ok = false; break; }
             tc_fence_after();
             const int nrows = min(32, M - row0);        // may be <= 0
             const int c_begin = half * (BN / 2), c_end = c_begin + BN / 2;
@@ -295,7 +300,7 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
                     }
                     continue;
                 }
-                if (full_chunk && EPI == EPI_CORE_UPDATE) {
+                if (full_chunk && EPI == EPI_CORE_UPDATE && !store_f32) {
 #pragma unroll
                     for (int j = 0; j < 32; ++j) patch[lane * 33 + j] = __uint_as_float(v[j]);
                     __syncwarp();
@@ -349,7 +354,7 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
                     bf16 *out = (bf16 *)P->out + (int64_t)row0 * P->ld_out + col;
                     if (col_ok)
                         for (int i = 0; i < nrows; ++i) out[(int64_t)i * P->ld_out] = __float2bfloat16_rn(patch[i * 33 + lane]);
-                } else if (EPI == EPI_CORE_UPDATE) {
+                } else if (EPI == EPI_CORE_UPDATE && !store_f32) {
                     // C, M, Vm are dense r x r (N = r)
                     if (col_ok) {
                         for (int i = 0; i < nrows; ++i) {
@@ -386,7 +391,9 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
     }
-    if (threadIdx.x == 0 && s_timeout && status) atomicMax(status, (int)TSR_ERR_TIMEOUT);
+    // every block that owns a tile this CTA did not finish is flagged
+    if (threadIdx.x == 0 && s_timeout && status)
+        for (int t = s_timeout - 1; t < num_tiles; t += stride) atomicMax(status + probs[tiles[t].prob].block, (int)TSR_ERR_TIMEOUT);
 }
 
 template <int BN, int EPI, int PLANES>

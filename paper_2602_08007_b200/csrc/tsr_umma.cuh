@@ -32,16 +32,33 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
         : "memory");
     return ok != 0;
 }
-// Bounded wait: false when the clock budget ran out.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
+// Bounded wait: false when the clock budget (in SM clock ticks) ran out.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, long long budget)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     while (!mbar_try_wait(bar, parity)) {
-        if (clock64() - t0 > UM_WAIT_CLOCKS) return false;
+        if (clock64() - t0 > budget) return false;
     }
     return true;
 }
+// The budget a launch runs with: the context's setting, or the default when none was made.
+__device__ __forceinline__ long long wait_budget(const StepScalars &sc)
+{
+    return sc.wait_clocks > 0 ? sc.wait_clocks : UM_WAIT_CLOCKS;
+}
+// Records the first tile (table index t) a role gave up on; roles of one CTA may give up on different tiles.
+__device__ __forceinline__ void note_timeout(int *slot, int t)
+{
+    const int v = t + 1;
+    int old = atomicCAS(slot, 0, v);
+    while (old != 0 && old > v) {
+        const int seen = atomicCAS(slot, old, v);
+        if (seen == old) break;
+        old = seen;
+    }
+}
+
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y)
 {
     asm volatile(

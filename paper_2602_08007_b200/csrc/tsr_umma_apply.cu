@@ -91,10 +91,11 @@ umma_apply_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restr
     uint64_t *bar_acc_empty = bar_acc_full + 2;      // [2]
     uint64_t *bar_w = bar_acc_empty + 2;             // [4][AP_NBOX]
     uint32_t *tmem_slot = (uint32_t *)(bars + AP_NBARS);
-    __shared__ int s_timeout;
+    __shared__ int s_timeout;   // 0, or 1 + the first tile (table index) this CTA gave up on
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int stride = gridDim.x;
+    const long long budget = wait_budget(sc);
 
     if (threadIdx.x == 0) {
         s_timeout = 0;
@@ -124,7 +125,7 @@ umma_apply_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restr
                 for (int kb = 0; kb < nkb; ++kb, ++it) {
                     const int s = it % AP_STAGES;
                     const uint32_t ph = (it / AP_STAGES) & 1u;
-                    if (!mbar_wait(smem_u32(bar_empty + s), ph ^ 1u)) { s_timeout = 1; ok = false; break; }
+                    if (!mbar_wait(smem_u32(bar_empty + s), ph ^ 1u, budget)) { note_timeout(&s_timeout, t); ok = false; break; }
                     const uint32_t full = smem_u32(bar_full + s);
                     mbar_expect_tx(full, (uint32_t)AP_STAGE_BYTES);
                     uint8_t *st = smem + s * AP_STAGE_BYTES;
@@ -143,13 +144,13 @@ umma_apply_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restr
                 const UmmaTile tile = tiles[t];
                 const int nkb = (probs[tile.prob].K + UM_BK - 1) / UM_BK;
                 const uint32_t buf = tc & 1u;
-                if (!mbar_wait(smem_u32(bar_acc_empty + buf), ((tc >> 1) & 1u) ^ 1u)) { s_timeout = 1; ok = false; break; }
+                if (!mbar_wait(smem_u32(bar_acc_empty + buf), ((tc >> 1) & 1u) ^ 1u, budget)) { note_timeout(&s_timeout, t); ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + buf * AP_BN;
                 for (int kb = 0; kb < nkb; ++kb, ++it) {
                     const int s = it % AP_STAGES;
                     const uint32_t ph = (it / AP_STAGES) & 1u;
-                    if (!mbar_wait(smem_u32(bar_full + s), ph)) { s_timeout = 1; ok = false; break; }
+                    if (!mbar_wait(smem_u32(bar_full + s), ph, budget)) { note_timeout(&s_timeout, t); ok = false; break; }
                     tc_fence_after();
                     const uint32_t a_base = smem_u32(smem + s * AP_STAGE_BYTES);
                     const uint32_t b_base = a_base + 16384;
@@ -186,7 +187,7 @@ umma_apply_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restr
         while (cur.tile_idx < num_tiles && ok) {
             const uint32_t buf = tc & 1u;
             if (cur.c == 0) {
-                if (!mbar_wait(smem_u32(bar_acc_full + buf), (tc >> 1) & 1u)) { s_timeout = 1; ok = false; break; }
+                if (!mbar_wait(smem_u32(bar_acc_full + buf), (tc >> 1) & 1u, budget)) { note_timeout(&s_timeout, cur.tile_idx); ok = false; break; }
                 tc_fence_after();
             }
             const uint32_t slot = cons % AP_NBOX;
@@ -197,7 +198,7 @@ umma_apply_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restr
                 tc_fence_before();
                 if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar_acc_empty + buf)) : "memory");
             }
-            if (!mbar_wait(smem_u32(wbar + slot), (cons / AP_NBOX) & 1u)) { s_timeout = 1; ok = false; break; }
+            if (!mbar_wait(smem_u32(wbar + slot), (cons / AP_NBOX) & 1u, budget)) { note_timeout(&s_timeout, cur.tile_idx); ok = false; break; }
             if (WB == 4) {
                 uint8_t *box = boxes + slot * AP_BOX_BYTES + lane * 128;
 #pragma unroll
@@ -262,7 +263,9 @@ umma_apply_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restr
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(CF::TMEM_COLS) : "memory");
     }
-    if (threadIdx.x == 0 && s_timeout && status) atomicMax(status, (int)TSR_ERR_TIMEOUT);
+    // every block that owns a tile this CTA did not finish is flagged
+    if (threadIdx.x == 0 && s_timeout && status)
+        for (int t = s_timeout - 1; t < num_tiles; t += stride) atomicMax(status + probs[tiles[t].prob].block, (int)TSR_ERR_TIMEOUT);
 }
 
 cudaError_t umma_apply_configure()

@@ -1,91 +1,119 @@
 """The five benchmark configurations, protocol as the task states it: bases initialised by a
 randomized-SVD refresh on a separate seeded gradient, then 10 optimizer steps on freshly drawn
-gradients, the CUDA library and the FP64 oracle in lock-step on the same bits (after every
-refresh the library's bases are handed to the oracle, because singular vectors inside the noise
-bulk are not unique).  Gated on C, M, Vm and W; the error of the accumulated update W_t - W_0 is reported as well.
+gradients with one in-loop refresh (before step 5), the CUDA library and the FP64 oracle in
+lock-step on the same bits.  After every refresh the library's bases are checked against the
+oracle's refresh of the same (G, Omega) -- invariants, captured energy, projectors at the
+spectral gap -- and then handed to the oracle, because singular vectors inside the noise bulk
+are not unique.  Gated on C, M, Vm and W (relative Frobenius error; the FP32 configuration also
+element-wise); the error of the accumulated update W_t - W_0 is reported.
 
-Config 1 runs as it is.  For the LLaMA-shaped sets the FP64 plain-loop oracle cannot afford every
-block (about 3 TFLOP per step at 1B), so a subset fixed in advance is run: one block of every
-distinct shape of the first layer (attention, gate, down) and the embedding -- all ranks, tile
-widths, ragged edges and the split-K core of the full set occur in it.  The whole sets, in the
-benchmark's launch configuration, are covered by test_gpu_fullsize.py on sampled outputs."""
-import json
-import os
-
+Which blocks are gated was fixed before any run:
+  * configurations 1-3 (single matrix, LLaMA-60M and -130M shapes): EVERY block, all 10 steps;
+  * configurations 4-5 (LLaMA-350M and -1B shapes), where ten steps of every block would keep the
+    plain-loop FP64 oracle busy for hours: one block of every distinct shape (attention = q,
+    gate, down) from the FIRST, the MIDDLE and the LAST layer, plus the embedding -- ten blocks,
+    all 10 steps, refreshes included.  Every rank, tile width, ragged edge (5461 = 21 * 256 + 85),
+    the k = 528 eigen-problem and the split-K core of the full set occur in the subset.
+The complete sets, in the benchmark's launch configuration, are covered on sampled outputs of
+every block by test_gpu_fullsize.py."""
 import numpy as np
 import pytest
 import torch
 
+import helpers
 import oracle
 import tsr_inputs as ti
-from helpers import HYPER, TOL_BF16, TOL_F32, check_refresh, rel_fro, to64
+from helpers import HYPER, TOL_BF16, TOL_F32, TOL_F32_MAXABS, check_refresh, max_abs_err, rel_fro, to64
 
 pytestmark = pytest.mark.gpu
 
-SUBSET = {0: [0], 1: [0, 4, 6, -1], 2: [0, 4, 6, -1], 3: [0, 4, 6, -1], 4: [0, 6, -1]}   # 1B: the gate shape is sampled in test_gpu_fullsize.py
-REFRESH_AT = {0: None, 1: 5, 2: 5, 3: 5, 4: None}     # in-loop refresh inside the 10 steps (1B: init only, oracle cost)
+REFRESH_AT = 5          # in-loop refresh before this step (of 10)
+
+
+def gated_blocks(cid):
+    """Indices (into the workload's block list) of the blocks that are gated; see the module text."""
+    w = ti.workload(cid)
+    nb = len(w.blocks)
+    if cid <= 2:
+        return list(range(nb))
+    layers = (nb - 1) // 7
+    picks = []
+    for layer in (0, layers // 2, layers - 1):
+        picks += [7 * layer + 0, 7 * layer + 4, 7 * layer + 6]      # q, gate, down
+    return picks + [nb - 1]                                          # the embedding
 
 
 @pytest.mark.parametrize("cid", [0, 1, 2, 3, 4])
 def test_config_protocol_matches_oracle(cid):
     import paper_2602_08007_b200 as tsr
     w = ti.workload(cid)
-    blocks = [w.blocks[i] for i in SUBSET[cid]]
+    sel = gated_blocks(cid)
+    blocks = [w.blocks[i] for i in sel]
     dt = torch.float32 if w.g_dtype == "f32" else torch.bfloat16
     tol = TOL_F32 if w.g_dtype == "f32" else TOL_BF16
     plan = tsr.Plan([dict(m=b.m, n=b.n, r=b.r, p=b.p, q=b.q, K=0, is_embedding=b.is_embedding) for b in blocks], g_dtype=dt)
     nb = len(blocks)
     assert all(plan.uses_tensor_cores(i) == (w.g_dtype == "bf16") for i in range(nb))
 
-    def draw(step, role):
-        out = []
-        for i, b in enumerate(blocks):
-            g = ti.gradient(b.m, b.n, ti.seed_for(cid, SUBSET[cid][i] % len(w.blocks), step, role), dtype=dt, device="cuda")
-            plan.G[i].copy_(g)
-            out.append(to64(g))
-        return out
+    def draw(i, step, role):
+        b = blocks[i]
+        g = ti.gradient(b.m, b.n, ti.seed_for(cid, sel[i], step, role), dtype=dt, device="cuda")
+        plan.G[i].copy_(g)
+        return g
 
     def omegas(step, role):
-        return [ti.omega(b.n, b.r + b.p, ti.seed_for(cid, SUBSET[cid][i] % len(w.blocks), step, role), device="cuda")
-                for i, b in enumerate(blocks)]
+        return [ti.omega(b.n, b.r + b.p, ti.seed_for(cid, sel[i], step, role), device="cuda") for i, b in enumerate(blocks)]
 
+    helpers.REFRESH_MEASURED.clear()
     gap = min(ti.SIGNAL_RANK, min(min(b.m, b.n) for b in blocks) // 2)
-    G0, Om0 = draw(0, ti.ROLE_INIT_GRAD), omegas(0, ti.ROLE_INIT_OMEGA)
+    G0 = [draw(i, 0, ti.ROLE_INIT_GRAD) for i in range(nb)]
+    Om0 = omegas(0, ti.ROLE_INIT_OMEGA)
     plan.init_subspace(omegas=Om0)
     torch.cuda.synchronize()
     assert plan.poll_status() == [0] * nb
     obs, W0 = [], []
     for i, b in enumerate(blocks):
-        check_refresh(plan, i, G0[i], to64(Om0[i]), b.r, b.q, gap)
-        wt = ti.weights(b.m, b.n, ti.seed_for(cid, i, 0, ti.ROLE_WEIGHT), device="cuda")
+        check_refresh(plan, i, to64(G0[i]), to64(Om0[i]), b.r, b.q, gap)
+        wt = ti.weights(b.m, b.n, ti.seed_for(cid, sel[i], 0, ti.ROLE_WEIGHT), device="cuda")
         plan.W[i].copy_(wt)
         W0.append(to64(wt))
         ob = oracle.OracleBlock(W0[i], b.r, b.p, b.q, 0)
         ob.set_bases(to64(plan.U[i]), to64(plan.V[i]))
         obs.append(ob)
-    worst = {k: 0.0 for k in ("C", "M", "Vm", "W", "dW")}
+    del G0, Om0
+    worst = {k: 0.0 for k in ("C", "M", "Vm", "W", "dW", "maxabs")}
     for t in range(1, 11):
-        G = draw(t, ti.ROLE_GRAD)
-        if REFRESH_AT[cid] == t:
+        G = [draw(i, t, ti.ROLE_GRAD) for i in range(nb)]
+        if t == REFRESH_AT:
             Om = omegas(t, ti.ROLE_OMEGA)
             plan.rsvd_refresh(omegas=Om)
             torch.cuda.synchronize()
+            assert plan.poll_status() == [0] * nb
             for i, b in enumerate(blocks):
-                check_refresh(plan, i, G[i], to64(Om[i]), b.r, b.q, gap)
+                check_refresh(plan, i, to64(G[i]), to64(Om[i]), b.r, b.q, gap)
                 obs[i].set_bases(to64(plan.U[i]), to64(plan.V[i]))
+            del Om
         plan.step(tsr.make_hyper(t), fuse_adam=(t % 2 == 1))
         torch.cuda.synchronize()
         for i, ob in enumerate(obs):
-            ob.step(G[i], skip_refresh=True, **HYPER)
-            worst["C"] = max(worst["C"], rel_fro(to64(plan.C[i]), ob.C))
-            worst["M"] = max(worst["M"], rel_fro(to64(plan.M[i]), ob.M))
-            worst["Vm"] = max(worst["Vm"], rel_fro(to64(plan.Vm[i]), ob.Vm))
-            worst["W"] = max(worst["W"], rel_fro(to64(plan.W[i]), ob.W))
-            worst["dW"] = max(worst["dW"], rel_fro(to64(plan.W[i]) - W0[i], ob.W - W0[i]))
+            ob.step(to64(G[i]), skip_refresh=True, **HYPER)
+            got = dict(C=to64(plan.C[i]), M=to64(plan.M[i]), Vm=to64(plan.Vm[i]), W=to64(plan.W[i]))
+            want = dict(C=ob.C, M=ob.M, Vm=ob.Vm, W=ob.W)
+            for key in ("C", "M", "Vm", "W"):
+                worst[key] = max(worst[key], rel_fro(got[key], want[key]))
+                worst["maxabs"] = max(worst["maxabs"], max_abs_err(got[key], want[key]))
+            worst["dW"] = max(worst["dW"], rel_fro(got["W"] - W0[i], ob.W - W0[i]))
     assert plan.poll_status() == [0] * nb
-    out_dir = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "gpurun_out")
-    if os.path.isdir(out_dir):
-        with open(os.path.join(out_dir, "parity_config%d.json" % cid), "w") as fh:
-            json.dump({"config": w.name, "blocks": [b.name for b in blocks], "tolerance": tol, "worst": worst}, fh)
+    rm = helpers.REFRESH_MEASURED
+    print("\nparity %s: %d of %d blocks, 10 steps, refresh at init and before step %d | worst rel. Frobenius error "
+          "C %.2e  M %.2e  Vm %.2e  W %.2e  (accumulated update %.2e; element-wise / max entry %.2e) | bound %.0e"
+          % (w.name, nb, len(w.blocks), REFRESH_AT, worst["C"], worst["M"], worst["Vm"], worst["W"], worst["dW"],
+             worst["maxabs"], tol))
+    print("refresh vs oracle over %d checks: ||Q^T Q - I|| <= %.1e, off-diagonal of U^T G V <= %.1e sigma_1, leading sigma "
+          "within %.1e, captured energy within %.1e, projector distance at the gap <= %.1e"
+          % (len(rm), max(x["ortho"] for x in rm), max(x["offdiag"] for x in rm), max(x["lead"] for x in rm),
+             max(x["energy"] for x in rm), max(x["proj"] for x in rm)))
     for key in ("C", "M", "Vm", "W"):
         assert worst[key] < tol, (w.name, worst)
+    if w.g_dtype == "f32":
+        assert worst["maxabs"] < TOL_F32_MAXABS, worst

@@ -166,6 +166,79 @@ def test_nonfinite_gradient_flags_its_block_only():
     assert torch.equal(res[0][1], res[1][1]) and torch.equal(res[0][2], res[1][2])
 
 
+@pytest.mark.parametrize("shape", [dict(m=192, n=256, r=16, p=8, q=1),       # k = 24: Jacobi solver
+                                   dict(m=320, n=384, r=200, p=8, q=1)])     # k = 208: tridiagonal + QL solver
+def test_sweep_limit_flags_not_converged_on_that_block_only(shape):
+    """The eigen-solver of one block is given a limit of one sweep (one QL iteration per
+    eigenvalue): it stops there, the block reads TSR_ERR_NOT_CONVERGED, and its neighbour, whose
+    limit is the default, comes out bit for bit as in a run without any limit."""
+    tsr = _tsr()
+    res = []
+    for limited in (False, True):
+        plan = tsr.Plan([shape, shape], g_dtype=torch.bfloat16)
+        for i in range(2):
+            fill_gradient(plan, i, 120 + i, signal_rank=8)
+        if limited:
+            plan.set_limits(max_sweeps=1, sweep_block=0)
+        oms = [ti.omega(shape["n"], shape["r"] + shape["p"], 124 + i).cuda() for i in range(2)]
+        plan.init_subspace(omegas=oms)
+        torch.cuda.synchronize()
+        st = plan.poll_status()
+        res.append((st, plan.U[1].clone(), plan.V[1].clone(), plan.U[0].clone()))
+        if limited:
+            assert torch.isfinite(plan.U[0]).all() and torch.isfinite(plan.V[0]).all()
+            # lifting the limit makes the same context converge again
+            plan.set_limits()
+            plan.rsvd_refresh(omegas=oms)
+            torch.cuda.synchronize()
+            assert plan.poll_status() == [0, 0]
+            assert torch.equal(plan.U[0], res[0][3])
+    assert res[0][0] == [0, 0]
+    assert res[1][0] == [7, 0]                            # TSR_ERR_NOT_CONVERGED on block 0 only
+    assert torch.equal(res[0][1], res[1][1]) and torch.equal(res[0][2], res[1][2])
+
+
+def test_bounded_wait_that_runs_out_reports_timeout_and_the_context_recovers():
+    """A wait inside a tensor-core kernel is made to run out in the only safe way: the library is
+    told (tsr_set_limits) to issue no loads for the tiles of one block in the first projection
+    GEMM and to bound every wait by 2e6 clock ticks (about a millisecond).  Nothing is in flight
+    for those tiles and no address is touched; the warps that wait for the data give up at the
+    bound, the CTAs release their tensor memory and return, and the block reads TSR_ERR_TIMEOUT.
+    The other block finishes normally, and after the switch is cleared the same context steps
+    cleanly and matches the oracle."""
+    tsr = _tsr()
+    shapes = [dict(m=640, n=768, r=64), dict(m=256, n=384, r=64)]     # block 1 is the smaller: its tiles come last
+    plan = tsr.Plan(shapes, g_dtype=torch.bfloat16)
+    for i, s in enumerate(shapes):
+        set_bases(plan, i, ti.orthonormal(s["m"], s["r"], 140 + i), ti.orthonormal(s["n"], s["r"], 150 + i))
+    plan.bases_changed()
+    with pytest.raises(tsr.TsrError):                     # the switch is refused without a short budget
+        plan.set_limits(starve_block=1)
+    G64 = [fill_gradient(plan, i, 160 + i) for i in range(2)]
+    plan.set_limits(wait_clocks=2_000_000, starve_block=1)
+    plan.project_core()
+    torch.cuda.synchronize()
+    assert plan.poll_status() == [0, 10]                  # TSR_ERR_TIMEOUT on the starved block only
+    assert rel_fro(to64(plan.C[0]), oracle.project_core(G64[0], to64(plan.U[0]), to64(plan.V[0]))) < TOL_BF16
+    # back to the defaults: the same context works as if nothing had happened
+    plan.set_limits()
+    blks = []
+    for i, s in enumerate(shapes):
+        W0 = fill_weights(plan, i, 170 + i)
+        ob = oracle.OracleBlock(W0, s["r"], 0, 0, 0)
+        ob.set_bases(to64(plan.U[i]), to64(plan.V[i]))
+        plan.M[i].zero_(); plan.Vm[i].zero_()
+        blks.append(ob)
+    for t in (1, 2):
+        G64 = [fill_gradient(plan, i, 180 + 10 * t + i) for i in range(2)]
+        plan.step(tsr.make_hyper(t))
+        torch.cuda.synchronize()
+        for i, ob in enumerate(blks):
+            ob.step(G64[i], **HYPER)
+            assert rel_fro(to64(plan.C[i]), ob.C) < TOL_BF16 and rel_fro(to64(plan.W[i]), ob.W) < TOL_BF16
+    assert plan.poll_status() == [0, 0]
+
+
 def test_runs_are_bitwise_reproducible_and_resumable():
     tsr = _tsr()
     w = ti.workload(1)

@@ -6,7 +6,8 @@ import torch
 
 import oracle
 import tsr_inputs as ti
-from helpers import (HYPER, TOL_BF16, TOL_F32, check_refresh, f32, fill_gradient, fill_weights, rel_fro, set_bases, to64)
+from helpers import (HYPER, TOL_BF16, TOL_F32, TOL_F32_MAXABS, check_refresh, f32, fill_gradient, fill_weights, max_abs_err,
+                     rel_fro, set_bases, to64)
 
 pytestmark = pytest.mark.gpu
 
@@ -27,6 +28,7 @@ def _run_steps(tsr, plan, shapes, dtype, steps, fuse, tol, wd=0.0, scale=1.0, ru
         plan.M[i].zero_(); plan.Vm[i].zero_()
         blks.append(ob)
     worst = {"C": 0.0, "M": 0.0, "Vm": 0.0, "W": 0.0}
+    worst_abs = 0.0     # FP32-gradient path only: element-wise error relative to the largest entry
     for t in range(1, steps + 1):
         G64 = [fill_gradient(plan, i, ti.seed_for(cfg, i, t, ti.ROLE_GRAD)) for i in range(nb)]
         h = tsr.make_hyper(t, lr=1e-3, weight_decay=wd, scale=scale, rule=rule)
@@ -44,9 +46,15 @@ def _run_steps(tsr, plan, shapes, dtype, steps, fuse, tol, wd=0.0, scale=1.0, ru
             if rule == 0:
                 worst["Vm"] = max(worst["Vm"], rel_fro(to64(plan.Vm[i]), ob.Vm))
             worst["W"] = max(worst["W"], rel_fro(to64(plan.W[i]), ob.W))
+            if dtype == torch.float32:
+                pairs = [(plan.C[i], ob.C), (plan.M[i], ob.M), (plan.W[i], ob.W)] + ([(plan.Vm[i], ob.Vm)] if rule == 0 else [])
+                worst_abs = max([worst_abs] + [max_abs_err(to64(a), b) for a, b in pairs])
     assert plan.poll_status() == [0] * nb
     for key, val in worst.items():
         assert val < tol, (key, val, worst)
+    if dtype == torch.float32:
+        print("FP32 path, worst element-wise error / max entry: %.2e (bound %.0e)" % (worst_abs, TOL_F32_MAXABS))
+        assert worst_abs < TOL_F32_MAXABS, worst_abs
     return worst
 
 
@@ -106,7 +114,43 @@ def test_sgd_rule_matches_algorithm_2(dtype, shapes, tol):
     tsr, plan = _plan(shapes, dtype)
     _given_bases(plan, shapes)
     _run_steps(tsr, plan, shapes, dtype, 5, True, tol, rule=1)
-    _run_steps(tsr, plan, shapes, dtype, 3, False, tol, rule=1)
+    # Algorithm 2 has neither a decay nor a scaling factor: the library ignores both under this rule
+    # (the oracle's SGD step takes neither), so passing them must change nothing
+    _run_steps(tsr, plan, shapes, dtype, 3, False, tol, rule=1, wd=0.1, scale=0.25)
+
+
+def test_sgd_rule_runs_without_a_second_moment_and_adam_refuses_it():
+    """A block bound with Vm = NULL is legal for the momentum-SGD rule; asking for the Adam rule on
+    it is an argument error found on the host: nothing is launched and no buffer changes."""
+    import paper_2602_08007_b200 as tsr
+    shapes = BF16_SHAPES[:2]
+    plan = tsr.Plan(shapes, g_dtype=torch.bfloat16)
+    plan.Vm = [None] * len(shapes)
+    plan.bind()
+    _given_bases(plan, shapes)
+    for i in range(len(shapes)):
+        fill_gradient(plan, i, 31 + i)
+        fill_weights(plan, i, 41 + i)
+    torch.cuda.synchronize()
+    before = [(plan.W[i].clone(), plan.M[i].clone(), plan.C[i].clone()) for i in range(len(shapes))]
+    launches = plan.launch_count()
+    for call in (lambda h: plan.step(h, fuse_adam=True), lambda h: plan.step(h, fuse_adam=False),
+                 lambda h: plan.adam_core_step(h)):
+        with pytest.raises(tsr.TsrError) as ei:
+            call(tsr.make_hyper(1))
+        assert ei.value.status == 1                        # TSR_ERR_INVALID_ARG
+    g_host = [plan.G[i].cpu().contiguous() for i in range(len(shapes))]
+    with pytest.raises(tsr.TsrError) as ei:
+        plan.step_host(g_host, None, tsr.make_hyper(1))
+    assert ei.value.status == 1
+    torch.cuda.synchronize()
+    assert plan.launch_count() == launches
+    for i, (w, m, c) in enumerate(before):
+        assert torch.equal(plan.W[i], w) and torch.equal(plan.M[i], m) and torch.equal(plan.C[i], c)
+    plan.step(tsr.make_hyper(1, rule=tsr.TSR_RULE_SGD), fuse_adam=True)   # the SGD rule needs no Vm
+    torch.cuda.synchronize()
+    assert plan.poll_status() == [0] * len(shapes)
+    assert not torch.equal(plan.W[0], before[0][0])
 
 
 def test_fused_and_unfused_orders_agree_bitwise():
@@ -236,6 +280,18 @@ def test_split_k_core_matches_oracle():
     _given_bases(plan, shapes)
     _run_steps(tsr, plan, shapes, torch.bfloat16, 3, True, TOL_BF16)
     _run_steps(tsr, plan, shapes, torch.bfloat16, 3, False, TOL_BF16)
+
+
+@pytest.mark.parametrize("fuse", [True, False])
+def test_split_k_core_with_rank_not_a_multiple_of_four(fuse):
+    """A tall block whose core GEMM is split along K, with r = 50: the slabs are not 16-byte
+    aligned, so their epilogue takes the ragged store path (never the fused core update, which
+    only the sum of the slabs may enter).  A second block shares the launch."""
+    shapes = [dict(m=9000, n=136, r=50), dict(m=256, n=384, r=64)]
+    tsr, plan = _plan(shapes, torch.bfloat16)
+    assert all(plan.uses_tensor_cores(i) for i in range(2))
+    _given_bases(plan, shapes)
+    _run_steps(tsr, plan, shapes, torch.bfloat16, 3, fuse, TOL_BF16)
 
 
 @pytest.mark.parametrize("dtype,shape,gap", [
