@@ -240,15 +240,21 @@ def max_over_ranks(values, dist, device):
     return [float(x) for x in tens]
 
 
-# Measured DRAM traffic of umma_apply_kernel divided by its algorithmic bytes (8 B per weight +
-# BF16 operands), from the ncu captures summarised in profiles/umma_apply_kernel.md: 0.98 on the
-# 350M set and on a six-layer slice of the 1B set (full captures), and 11.19 GB against 11.16 GB
-# algorithmic on the full 1B set (a one-pass capture of dram__bytes_read.sum + dram__bytes_write.sum).
-APPLY_TRAFFIC_RATIO = {3: 0.98, 4: 1.00}
-
-
-def apply_traffic_ratio(config_id: int) -> float:
-    return APPLY_TRAFFIC_RATIO.get(config_id, 0.98)
+def apply_traffic(w: ti.Workload, algorithmic_bytes: float):
+    """DRAM bytes per launch of the apply kernel as ncu measured them (dram__bytes_read.sum +
+    dram__bytes_write.sum), read from the table profiles/dram_traffic.json keeps per workload together
+    with the commit it was captured at.  A capture of a slice of the workload is scaled to the full
+    launch by the algorithmic bytes (traffic grows in proportion to the weights streamed).  None when
+    the table has no entry for this workload."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    try:
+        with open(path) as fh:
+            table = json.load(fh)
+        e = table["umma_apply_kernel"][w.name]
+        return {"bytes": float(e["dram_bytes"]) * algorithmic_bytes / float(e["algorithmic_bytes"]),
+                "captured_on": e["captured_on"], "commit": e["commit"]}
+    except Exception:
+        return None
 
 
 def build_plan(w: ti.Workload, device, bf16_weights: bool = False):
@@ -265,6 +271,83 @@ def fresh_gradients(plan, w, t, device):
     dt = plan.g_dtype
     for i, b in enumerate(w.blocks):
         plan.G[i].copy_(ti.gradient(b.m, b.n, ti.seed_for(w.config_id, i, t, ti.ROLE_GRAD), dtype=dt, device=device))
+
+
+def quick_config(cid: int, device, peaks, steps: int = 20):
+    """A compact measurement of one of the other benchmark configurations: ms per step with L2 flushed
+    between steps (cold) and not (warm), one refresh, and the roofline fractions of the apply and
+    projection stages.  About two seconds each; the numbers of the headline workload come from the main run."""
+    w = ti.workload(cid)
+    tsr, plan = build_plan(w, device)
+    work = step_work(w)
+    plan.init_subspace(seed=ti.BASE_SEED)
+    fresh_gradients(plan, w, 1, device)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)
+    for _ in range(3):
+        plan.step(tsr.make_hyper(1), seed=ti.BASE_SEED, fuse_adam=True)
+    torch.cuda.synchronize()
+
+    def timed(cold):
+        ev = []
+        for j in range(steps):
+            if cold:
+                flush.fill_(j & 0xFF)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            plan.step(tsr.make_hyper(j + 1), seed=ti.BASE_SEED, fuse_adam=True)
+            b.record()
+            ev.append((a, b))
+        torch.cuda.synchronize()
+        return statistics.median(a.elapsed_time(b) for a, b in ev)
+
+    launches0 = plan.launch_count()
+    cold_ms = timed(True)
+    launches = (plan.launch_count() - launches0) // steps
+    warm_ms = timed(False)
+    plan.set_profiling(True)
+    rows = []
+    for rep in range(7):
+        flush.fill_(rep)
+        plan.step(tsr.make_hyper(1), seed=ti.BASE_SEED, fuse_adam=True)
+        rows.append(plan.stage_ms())
+    st = [statistics.median(r[i] for r in rows) for i in range(6)]
+    plan.set_profiling(False)
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    flush.fill_(1)
+    a.record()
+    plan.rsvd_refresh(seed=ti.BASE_SEED + 1)
+    b.record()
+    torch.cuda.synchronize()
+    refresh_ms = a.elapsed_time(b)
+    status = sorted(set(plan.poll_status()))
+    hbm, tc = peaks["hbm_gbs"], peaks["bf16_tflops"]
+    proj_ms, apply_ms = st[1] + st[2], st[4] + st[5]
+    proj_roof = max(work["proj_flops"] / (tc * 1e12), work["proj_bytes"] / (hbm * 1e9)) * 1e3
+    apply_roof = max(work["apply_flops"] / (tc * 1e12), work["apply_bytes"] / (hbm * 1e9)) * 1e3
+    out = {"workload": w.name, "blocks": len(w.blocks), "dtype": w.g_dtype, "step_ms_cold_l2": cold_ms, "step_ms_warm_l2": warm_ms,
+           "step_roof_ms": proj_roof + apply_roof, "refresh_ms": refresh_ms, "launches_per_step": launches,
+           "projection": {"ms": proj_ms, "roof_ms": proj_roof, "frac": proj_roof / proj_ms if proj_ms > 0 else None},
+           "backprojection": {"ms": apply_ms, "roof_ms": apply_roof, "frac": apply_roof / apply_ms if apply_ms > 0 else None},
+           "device_status": status}
+    plan.close()
+    del plan, flush
+    torch.cuda.empty_cache()
+    return out
+
+
+def oracle_one_thread(cid: int):
+    """The oracle's step time on ONE host thread for a small configuration (a child process, because the
+    OpenMP thread count is fixed when the oracle's library loads): one step of one block per distinct
+    shape, each multiplied by its block count."""
+    import subprocess
+    code = ("import sys; sys.path.insert(0, %r); import bench, tsr_inputs as ti; w = ti.workload(%d); "
+            "print(sum(bench.oracle_step_time(w, blk) * cnt for blk, cnt in bench.distinct_shapes(w)) * 1e3)" % (ROOT, cid))
+    env = dict(os.environ, OMP_NUM_THREADS="1")
+    try:
+        out = subprocess.run([sys.executable, "-c", code], env=env, capture_output=True, text=True, timeout=300)
+        return float(out.stdout.strip().splitlines()[-1])
+    except Exception:
+        return None
 
 
 def run_ours(args, w: ti.Workload):
@@ -424,6 +507,9 @@ def run_ours(args, w: ti.Workload):
         apply_roof_ms = max(work["apply_kernel_flops"] / (tc * 1e12), work["apply_kernel_bytes"] / (hbm * 1e9)) * 1e3
         plain_ms = statistics.median(plain)
         core_b, sketch_b = plan.comm_bytes(0, 4)
+        traffic = apply_traffic(w, work["apply_kernel_bytes"])
+        tc_burst = peaks["bf16_tflops"]
+        proj_roof_burst_ms = max(work["proj_flops"] / (tc_burst * 1e12), work["proj_bytes"] / (hbm * 1e9)) * 1e3
         line = {
             "metric": METRIC, "value": ms_per_step, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak",
@@ -443,13 +529,20 @@ def run_ours(args, w: ti.Workload):
                          "gemm_UD": st_med[4], "apply": st_med[5]},
             "roofline": {"kernel": "umma_apply_kernel (W <- decay W - lr P V^T)", "bound": "hbm",
                          "achieved": apply_gbs, "peak": hbm, "unit": "GB/s", "frac": apply_gbs / hbm,
-                         "traffic": None if args.bf16_weights else apply_traffic_ratio(w.config_id) * work["apply_kernel_bytes"],
+                         "traffic": None if (args.bf16_weights or traffic is None) else traffic["bytes"],
+                         "traffic_source": None if traffic is None else "ncu capture on %s at commit %s (profiles/dram_traffic.json)"
+                         % (traffic["captured_on"], traffic["commit"]),
                          "algorithmic_bytes": work["apply_kernel_bytes"],
                          "peak_source": peaks["source"] + " copy bandwidth", "ms": apply_ms, "roof_ms": apply_roof_ms},
             "roofline_projection": {"kernels": "umma_gemm_kernel<EPI_STORE_BF16_T> + <EPI_CORE_UPDATE>",
                                     "bound": "tensor" if work["proj_flops"] / (tc * 1e12) > work["proj_bytes"] / (hbm * 1e9) else "hbm",
                                     "achieved_tflops": proj_tflops, "ms": proj_ms, "roof_ms": proj_roof_ms,
-                                    "frac": proj_roof_ms / proj_ms},
+                                    "frac": proj_roof_ms / proj_ms, "peak": "sustained BF16 %.0f TFLOP/s" % tc,
+                                    "roof_ms_burst_peak": proj_roof_burst_ms, "frac_of_burst_peak": proj_roof_burst_ms / proj_ms},
+            "peaks": {"hbm_gbs": hbm, "bf16_tflops_burst": tc_burst, "bf16_tflops_sustained": tc, "source": peaks["source"],
+                      "nominal_b200": {"hbm_gbs": 7700.0, "bf16_tflops_dense": 2250.0},
+                      "apply_frac_of_nominal_hbm": apply_gbs / 7700.0,
+                      "projection_frac_of_nominal": (work["proj_flops"] / 2250e12 * 1e3) / proj_ms},
             "comm_bytes": {"core_per_step": core_b, "sketch_per_refresh": sketch_b,
                            "dense_fp32_per_step": 4 * sum(b.m * b.n for b in w.blocks)},
             "dense_adamw": dense,
@@ -460,6 +553,19 @@ def run_ours(args, w: ti.Workload):
         }
         if not args.no_cpu_baseline and world == 1:
             line["cpu_baseline"] = cpu_baseline(w, len(refresh_steps) / float(args.steps))
+        if args.all_configs and world == 1:
+            # the other four benchmark configurations, compactly (the headline workload's numbers are the line's own)
+            plan.close()
+            torch.cuda.empty_cache()
+            others = {}
+            for cid in range(5):
+                if cid == w.config_id:
+                    continue
+                entry = quick_config(cid, device, peaks)
+                if cid <= 1 and not args.no_cpu_baseline:
+                    entry["oracle_step_ms_1_thread"] = oracle_one_thread(cid)
+                others["config%d" % (cid + 1)] = entry
+            line["configs"] = others
         print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()
@@ -568,6 +674,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--dense-params", type=int, default=1 << 26,
                     help="size of the dense-AdamW micro-measurement (0 = skip)")
+    ap.add_argument("--all-configs", dest="all_configs", action="store_true", default=None,
+                    help="add a compact measurement of the other four configurations (default: on for the default workload)")
+    ap.add_argument("--no-all-configs", dest="all_configs", action="store_false")
     ap.add_argument("--layers", type=int, default=0, help="profiling aid: truncate the model to this many layers")
     ap.add_argument("--unfused", action="store_true", help="diagnostic: run the core update as its own launch")
     ap.add_argument("--bf16-weights", action="store_true",
@@ -577,6 +686,16 @@ def main():
     ap.add_argument("--ablation", action="store_true",
                     help="report the one-sided and exact-SVD comparison arms of the chosen set instead of the benchmark")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started without a launcher: start the N replica processes (one per GPU) ourselves
+        import socket
+        import subprocess
+        with socket.socket() as sk:
+            sk.bind(("127.0.0.1", 0))
+            port = sk.getsockname()[1]
+        cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(args.gpus),
+               "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+        raise SystemExit(subprocess.call(cmd))
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
     w = ti.workload(args.config)
@@ -586,6 +705,8 @@ def main():
         w = ti.Workload(w.name + "-first%dlayers" % args.layers, w.config_id, w.g_dtype, w.steps, keep)
     if args.config < 3:
         args.flush_l2 = True
+    if args.all_configs is None:
+        args.all_configs = (args.config == 4 and args.layers == 0 and not args.bf16_weights)
     if args.ablation:
         run_ablation(args, w)
     elif args.impl == "reference":

@@ -17,7 +17,9 @@ namespace {
 
 // KR*: tall-times-small products of the refresh on tensor cores (three TF32 products): rows of side
 // 0 (m) or 1 (n) times R^{-1} into buf[1] / buf[2], and the final U = Q Wu, V = B^T Wv.
-enum Kind : int { KT = 0, KC, KP, KA, KY, KZ, KR01, KR02, KR12, KRU, KRV, KO, KOA, NKIND };
+// KCM: the core problems encoded for the merged projection launch (its B boxes follow the tile width of KT);
+// KM: the merged tile table itself (tiles of KT and KCM problems interleaved; it has no problem table of its own).
+enum Kind : int { KT = 0, KC, KP, KA, KY, KZ, KR01, KR02, KR12, KRU, KRV, KO, KOA, KCM, KM, NKIND };
 constexpr int TSR_NUM_STAGES = 6;  // refresh, G*V, core GEMM, core update, U*D, apply
 
 struct Block {
@@ -90,13 +92,16 @@ struct tsr_ctx {
     int32_t *d_status = nullptr;
     int32_t *d_list = nullptr;                 // scratch: block list of the running call
     int32_t *d_list2 = nullptr;                // scratch: second list (split-K blocks, ...)
+    int32_t *d_rlist = nullptr;                // block lists of the refresh groups
     RowItem *d_items[5] = {};                  // [side*2 + 0]: 64-row slabs, [side*2 + 1]: Gram slabs, [4]: eigenvector panels
     size_t items_cap[5] = {};
     EncodeTiledFn encode = nullptr;
     int max_r = 0, max_k = 0;
     uint64_t launches = 0;                     // kernels launched through this context
     int num_sms = 148;
-    int bn[NKIND] = {128, 128, 128, 128, 128, 128, 256, 256, 256, 256, 256, 128, 128};   // tile width of each GEMM kind
+    int bn[NKIND] = {128, 128, 128, 128, 128, 128, 256, 256, 256, 256, 256, 128, 128, 128, 128};   // tile width of each GEMM kind
+    int32_t *d_counters = nullptr;             // merged projection launch: one dependency counter per block
+    bool merged_ok = true;                     // cleared when the device refuses the cooperative launch
     bool profiling = false;
     cudaEvent_t ev[TSR_NUM_STAGES + 1] = {};   // stage boundaries of the last step (profiling only)
     bool ev_valid = false;
@@ -110,6 +115,11 @@ struct tsr_ctx {
     static constexpr int NPIPE = 8;            // chunks of the pipelined host-buffer step
     cudaEvent_t ev_pipe_in[NPIPE] = {}, ev_pipe_done[NPIPE] = {};
     bool aux_ready = false;
+    // What the device copies of the refresh tables (block lists, row-slab and panel tables) and of the step lists
+    // d_list / d_list2 currently hold, so that a call over the same blocks as the previous one uploads nothing.
+    // Cleared by tsr_bind and by any other writer of those tables.
+    std::vector<int> refresh_sig;              // the refresh (its groups, in order) those tables were last written for
+    std::vector<int> list_cache[2];
     // limits (tsr_set_limits)
     long long wait_clocks = 0;                 // 0: the kernels' default budget
     std::vector<int32_t> max_sweeps;           // per block; 0: the solvers' defaults
@@ -164,7 +174,11 @@ void layout(tsr_ctx *ctx, Arena &a, bool assign, size_t *step_end)
     void *p4 = a.take(sizeof(int32_t) * (size_t)nb);
     void *p5 = a.take(sizeof(int32_t) * (size_t)nb);
     void *p6 = a.take(sizeof(int32_t) * (size_t)nb);
+    void *p7 = a.take(sizeof(int32_t) * (size_t)nb);
+    void *p8 = a.take(sizeof(int32_t) * (size_t)(nb + 1));
     if (assign) {
+        ctx->d_rlist = (int32_t *)p7;
+        ctx->d_counters = (int32_t *)p8;
         ctx->d_cu_all = (CoreUpdateArgs *)p1; ctx->d_cu_split = (CoreUpdateArgs *)p2;
         ctx->d_refresh = (RefreshDev *)p3; ctx->d_status = (int32_t *)p4;
         ctx->d_list = (int32_t *)p5; ctx->d_list2 = (int32_t *)p6;
@@ -254,14 +268,9 @@ void layout(tsr_ctx *ctx, Arena &a, bool assign, size_t *step_end)
 
 // tri > 0: B is the transpose of an upper-triangular matrix, so the columns n0 .. of the product only
 // need the first n0 + bn entries of the contraction (tri = elements per K block).
-void add_tiles(tsr_ctx *ctx, int kind, int bi, int M, int N, int K, int kb_per_split, int tri = 0)
+void gen_tiles(std::vector<UmmaTile> &v, int bi, int M, int N, int K, int kb_per_split, int bn, bool apply, int tri)
 {
-    const int bn = ctx->bn[kind];
-    const bool apply = (kind == KA || kind == KOA);
     const int bm = apply ? 128 : 256;   // the grouped GEMM runs on CTA pairs: 256-row tiles
-    Block &b = ctx->blocks[bi];
-    std::vector<UmmaTile> &v = ctx->tiles[kind];
-    b.tile_begin[kind] = (int)v.size();
     const int nkb = (K + 63) / 64;
     const int nsp = kb_per_split > 0 ? (nkb + kb_per_split - 1) / kb_per_split : 1;
     // Columns: the grouped GEMM takes tiles of any width that is a multiple of 16, so N is cut into equal parts
@@ -274,15 +283,63 @@ void add_tiles(tsr_ctx *ctx, int kind, int bi, int M, int N, int K, int kb_per_s
         for (int n0 = 0; n0 < N; n0 += wn)
             for (int s = 0; s < nsp; ++s) {
                 UmmaTile t;
+                memset(&t, 0, sizeof t);
                 t.prob = bi; t.m0 = m0; t.n0 = n0;
                 t.kb0 = kb_per_split > 0 ? s * kb_per_split : 0;
                 t.kb1 = kb_per_split > 0 ? std::min(nkb, (s + 1) * kb_per_split) : nkb;
                 t.nw = apply ? 0 : std::min(wn, ((N - n0) + 15) & ~15);
                 if (tri > 0) t.kb1 = std::min(nkb, (n0 + (apply ? bn : t.nw) + tri - 1) / tri);
                 t.split = s;
+                t.wait_slot = -1; t.signal_slot = -1;
                 v.push_back(t);
             }
+}
+
+// tri > 0: B is the transpose of an upper-triangular matrix, so the columns n0 .. of the product only
+// need the first n0 + bn entries of the contraction (tri = elements per K block).
+void add_tiles(tsr_ctx *ctx, int kind, int bi, int M, int N, int K, int kb_per_split, int tri = 0)
+{
+    Block &b = ctx->blocks[bi];
+    std::vector<UmmaTile> &v = ctx->tiles[kind];
+    b.tile_begin[kind] = (int)v.size();
+    gen_tiles(v, bi, M, N, K, kb_per_split, ctx->bn[kind], kind == KA || kind == KOA, tri);
     b.tile_end[kind] = (int)v.size();
+}
+
+// The merged projection table: for the two-sided tensor-core blocks in table order, the tiles of T~ = (G V)^T of a
+// block, and -- once at least MERGE_GAP later tiles separate them from the block's last T~ tile -- the tiles of its
+// core C = U^T T.  A core tile therefore always sits behind the tiles it depends on (CTA pairs take tiles in table
+// order, round-robin, so the wait cannot deadlock), close enough that T~ is still in L2 when it is read back, and far
+// enough that its producers have normally finished when a pair reaches it.
+constexpr int MERGE_GAP = 128;
+
+void build_merged(tsr_ctx *ctx)
+{
+    std::vector<UmmaTile> &v = ctx->tiles[KM];
+    v.clear();
+    struct Pending { int bi; size_t t_end; int n_t; };
+    std::vector<Pending> pending;
+    size_t head = 0;
+    auto emit_core = [&](const Pending &pd) {
+        const Block &b = ctx->blocks[pd.bi];
+        const size_t first = v.size();
+        gen_tiles(v, pd.bi, b.d.r, b.d.r, (int)b.d.m, b.nsplit > 1 ? b.kb_per_split : 0, ctx->bn[KCM], false, 0);
+        for (size_t i = first; i < v.size(); ++i) {
+            v[i].kind = 1;
+            v[i].wait_slot = pd.bi;
+            v[i].wait_count = pd.n_t * UMMA_SIGNALS_PER_TILE;
+        }
+    };
+    for (int bi : ctx->order) {
+        const Block &b = ctx->blocks[bi];
+        if (!b.fast || b.one_sided) continue;
+        const size_t first = v.size();
+        gen_tiles(v, bi, (int)b.d.m, b.d.r, (int)b.d.n, 0, ctx->bn[KT], false, 0);
+        for (size_t i = first; i < v.size(); ++i) { v[i].kind = 0; v[i].signal_slot = bi; }
+        pending.push_back({bi, v.size(), (int)(v.size() - first)});
+        while (head < pending.size() && v.size() >= pending[head].t_end + MERGE_GAP) emit_core(pending[head++]);
+    }
+    while (head < pending.size()) emit_core(pending[head++]);
 }
 
 void build_tiles(tsr_ctx *ctx)
@@ -300,6 +357,8 @@ void build_tiles(tsr_ctx *ctx)
     for (int kd : {KY, KZ}) ctx->bn[kd] = rmax >= 256 ? 256 : 128;
     ctx->bn[KO] = ctx->bn[KT];
     ctx->bn[KOA] = ctx->bn[KA];
+    ctx->bn[KCM] = ctx->bn[KT];
+    ctx->bn[KM] = ctx->bn[KT];
     for (int bi : ctx->order) {
         Block &b = ctx->blocks[bi];
         for (int kd = 0; kd < NKIND; ++kd) b.tile_begin[kd] = b.tile_end[kd] = (int)ctx->tiles[kd].size();
@@ -326,6 +385,7 @@ void build_tiles(tsr_ctx *ctx)
             add_tiles(ctx, KRV, bi, n, r, 2 * k, 0);
         }
     }
+    build_merged(ctx);
 }
 
 // BF16 row-major [rows x cols] (ld elements) -> tensor map with a 64 x box_rows box, 128B swizzle.
@@ -497,10 +557,14 @@ tsr_status launch_kind(tsr_ctx *ctx, int kind, const std::vector<int> &list, int
     return TSR_OK;
 }
 
-tsr_status upload_list(tsr_ctx *ctx, int32_t *dst, const std::vector<int> &v, cudaStream_t st)
+// which: 0 = d_list, 1 = d_list2 (their last contents are remembered, so that a step over the same blocks as the
+// previous one uploads nothing), -1 = any other destination, always copied.
+tsr_status upload_list(tsr_ctx *ctx, int32_t *dst, const std::vector<int> &v, cudaStream_t st, int which = -1)
 {
     if (v.empty()) return TSR_OK;
+    if (which >= 0 && ctx->list_cache[which] == v) return TSR_OK;
     TSR_CUDA(ctx, cudaMemcpyAsync(dst, v.data(), v.size() * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    if (which >= 0) ctx->list_cache[which] = v;
     return TSR_OK;
 }
 
@@ -509,9 +573,27 @@ tsr_status do_project(tsr_ctx *ctx, const std::vector<int> &list, bool fuse, con
 {
     tsr_status s;
     if (ctx->any_fast) {
-        if ((s = launch_kind(ctx, KT, list, EPI_STORE_BF16_T, 1, sc, st)) != TSR_OK) return s;
+        // A call that covers every two-sided tensor-core block of the plan runs both contractions as ONE launch
+        // (T~ tiles with the core tiles a few blocks behind them, T~ read back from L2); a partial list, or a
+        // device that cannot take the cooperative launch, runs them as two launches.  The tiles, their
+        // reduction order and therefore the results are the same either way.
+        bool merged = false;
+        if (ctx->merged_ok && !ctx->tiles[KM].empty()) {
+            int have = 0, all = 0;
+            for (const Block &b : ctx->blocks) all += (b.fast && !b.one_sided) ? 1 : 0;
+            for (int bi : list) have += (ctx->blocks[bi].fast && !ctx->blocks[bi].one_sided) ? 1 : 0;
+            if (have == all) {
+                TSR_CUDA(ctx, cudaMemsetAsync(ctx->d_counters, 0, sizeof(int32_t) * (ctx->blocks.size() + 1), st));
+                const cudaError_t e = umma_project_launch(ctx->d_probs[KT], ctx->d_probs[KCM], ctx->d_tiles[KM], (int)ctx->tiles[KM].size(),
+                                                          ctx->num_sms, ctx->bn[KM], fuse ? 1 : 0, ctx->d_counters, sc, ctx->d_status, st,
+                                                          (int)ctx->blocks.size());
+                if (e == cudaSuccess) { merged = true; ctx->launches++; }
+                else { (void)cudaGetLastError(); ctx->merged_ok = false; }   // refused: nothing ran; use two launches from now on
+            }
+        }
+        if (!merged && (s = launch_kind(ctx, KT, list, EPI_STORE_BF16_T, 1, sc, st)) != TSR_OK) return s;
         mark_stage(ctx, 2);
-        if ((s = launch_kind(ctx, KC, list, fuse ? EPI_CORE_UPDATE : EPI_STORE_F32, 1, sc, st)) != TSR_OK) return s;
+        if (!merged && (s = launch_kind(ctx, KC, list, fuse ? EPI_CORE_UPDATE : EPI_STORE_F32, 1, sc, st)) != TSR_OK) return s;
         // one-sided blocks: C = U^T G needs the gradient with m as the contiguous index
         bool any_one_sided = false;
         for (int bi : list) {
@@ -542,11 +624,11 @@ tsr_status do_project(tsr_ctx *ctx, const std::vector<int> &list, bool fuse, con
         }
     }
     if (!split.empty()) {   // sum the split-K slabs (and, when fused, run the core update on the sum)
-        if ((s = upload_list(ctx, ctx->d_list2, split, st)) != TSR_OK) return s;
+        if ((s = upload_list(ctx, ctx->d_list2, split, st, 1)) != TSR_OK) return s;
         TSR_KERNEL(ctx, 1, core_update_launch(ctx->d_cu_split, ctx->d_list2, (int)split.size(), max_r, max_c, sc, fuse ? 0 : 1, st));
     }
     if (!later.empty()) {
-        if ((s = upload_list(ctx, ctx->d_list2, later, st)) != TSR_OK) return s;
+        if ((s = upload_list(ctx, ctx->d_list2, later, st, 1)) != TSR_OK) return s;
         TSR_KERNEL(ctx, 1, core_update_launch(ctx->d_cu_all, ctx->d_list2, (int)later.size(), max_r, max_c, sc, 0, st));
     }
     mark_stage(ctx, 3);
@@ -563,7 +645,7 @@ tsr_status do_core_update(tsr_ctx *ctx, const std::vector<int> &list, const Step
         max_r = std::max(max_r, (int)ctx->blocks[bi].d.r);
         max_c = std::max(max_c, (int)ctx->blocks[bi].cn);
     }
-    if ((s = upload_list(ctx, ctx->d_list, list, st)) != TSR_OK) return s;
+    if ((s = upload_list(ctx, ctx->d_list, list, st, 0)) != TSR_OK) return s;
     TSR_KERNEL(ctx, 1, core_update_launch(ctx->d_cu_all, ctx->d_list, (int)list.size(), max_r, max_c, sc, 0, st));
     return TSR_OK;
 }
@@ -594,14 +676,17 @@ tsr_status do_apply(tsr_ctx *ctx, const std::vector<int> &list, const StepScalar
     return TSR_OK;
 }
 
-tsr_status do_shadows(tsr_ctx *ctx, const std::vector<int> &list, cudaStream_t st)
+// BF16 operand copies of U and V for the listed blocks.  items_m / items_n: device tables of the 128-row
+// slabs of the m and n sides of exactly those blocks.
+tsr_status do_shadows(tsr_ctx *ctx, const std::vector<int> &list, const RowItem *items_m, int n_m, const RowItem *items_n,
+                      int n_n, cudaStream_t st)
 {
-    for (int bi : list) {
-        Block &b = ctx->blocks[bi];
-        if (!b.fast) continue;
-        TSR_KERNEL(ctx, 1, make_shadows(b.p.U, (int)b.d.m, b.d.r, b.Ub, b.rl, b.Ubt, b.ml, st));
-        TSR_KERNEL(ctx, 1, make_shadows(b.p.V, (int)b.d.n, b.d.r, b.Vb, b.rl, b.Vbt, b.nl, st));
-    }
+    int rmax = 0;
+    for (int bi : list)
+        if (ctx->blocks[bi].fast) rmax = std::max(rmax, (int)ctx->blocks[bi].d.r);
+    if (rmax == 0) return TSR_OK;
+    TSR_KERNEL(ctx, 1, shadows_batched(ctx->d_refresh, items_m, n_m, 0, rmax, st));
+    TSR_KERNEL(ctx, 1, shadows_batched(ctx->d_refresh, items_n, n_n, 1, rmax, st));
     return TSR_OK;
 }
 
@@ -677,15 +762,18 @@ tsr_status sketch(tsr_ctx *ctx, const RefreshLists &L, bool transposed, bool fro
     StepScalars sc = {};
     sc.wait_clocks = ctx->wait_clocks;
     tsr_status s;
+    (void)omegas;   // a caller-given Omega has been copied into the block's own buffer by now
+    if (ctx->any_fast) {   // X^T as BF16 plane(s) for every block of the group at once
+        const int side = transposed ? 0 : 1;                     // rows of X: m for G^T X, n for G X
+        TSR_KERNEL(ctx, 1, split_transpose_batched(ctx->d_refresh, L.ditems[side * 2], L.nitems[side * 2], side,
+                                                   from_omega ? -1 : 2, planes, L.kmax, st));
+    }
     for (size_t j = 0; j < L.list.size(); ++j) {
         Block &b = ctx->blocks[L.list[j]];
+        if (b.fast) continue;
         const int m = (int)b.d.m, n = (int)b.d.n, k = b.k;
-        const float *X = from_omega ? ((omegas && omegas[j]) ? omegas[j] : b.Om) : b.buf[2];
-        if (b.fast) {
-            const int rows = transposed ? m : n;                 // rows of X
-            const int64_t ld = transposed ? b.ml : b.nl;
-            TSR_KERNEL(ctx, 1, split_transpose(X, rows, k, b.Xt, ld, k, planes, st));
-        } else if (!transposed) {
+        const float *X = from_omega ? b.Om : b.buf[2];
+        if (!transposed) {
             TSR_KERNEL(ctx, 1, simt_gemm(m, k, n, b.p.G, b.d.g_dtype, b.d.ldg, 1, X, k, 1, b.buf[0], k, SIMT_STORE, 0, 0, st));
         } else {
             TSR_KERNEL(ctx, 1, simt_gemm(n, k, m, b.p.G, b.d.g_dtype, 1, b.d.ldg, X, k, 1, b.buf[0], k, SIMT_STORE, 0, 0, st));
@@ -699,13 +787,13 @@ tsr_status sketch(tsr_ctx *ctx, const RefreshLists &L, bool transposed, bool fro
 // One group of blocks through the whole refresh on stream st.  list_off / item_off: where this
 // group's slices start inside the context's device list / item tables.
 tsr_status do_refresh_group(tsr_ctx *ctx, const std::vector<int> &list, uint64_t seed, const float *const *omegas,
-                            cudaStream_t st, size_t list_off, const size_t *item_off, bool reexpress)
+                            cudaStream_t st, size_t list_off, const size_t *item_off, bool reexpress, bool cached)
 {
     if (list.empty()) return TSR_OK;
     tsr_status s;
     RefreshLists L;
     L.list = list;
-    L.dlist = ctx->d_list + list_off;
+    L.dlist = ctx->d_rlist + list_off;
     for (int i = 0; i < 5; ++i) L.ditems[i] = ctx->d_items[i] + item_off[i];
     L.kmax = 1; L.rmax = 1;
     std::vector<RowItem> items[4];
@@ -724,20 +812,31 @@ tsr_status do_refresh_group(tsr_ctx *ctx, const std::vector<int> &list, uint64_t
     for (int bi : list)
         if (ctx->blocks[bi].d.q != qmax)
             return fail(ctx, TSR_ERR_UNSUPPORTED, "blocks refreshed in one grouped call must share q");
-    if ((s = upload_list(ctx, L.dlist, list, st)) != TSR_OK) return s;
-    for (int i = 0; i < 4; ++i) {
-        L.nitems[i] = (int)items[i].size();
-        TSR_CUDA(ctx, cudaMemcpyAsync(L.ditems[i], items[i].data(), items[i].size() * sizeof(RowItem),
-                                      cudaMemcpyHostToDevice, st));
+    // cached: the device tables still hold exactly this refresh (same groups in the same order) from last time
+    if (!cached) {
+        if ((s = upload_list(ctx, L.dlist, list, st)) != TSR_OK) return s;
+        for (int i = 0; i < 4; ++i)
+            TSR_CUDA(ctx, cudaMemcpyAsync(L.ditems[i], items[i].data(), items[i].size() * sizeof(RowItem),
+                                          cudaMemcpyHostToDevice, st));
     }
-    // Omega and the transposed gradient copies
+    for (int i = 0; i < 4; ++i) L.nitems[i] = (int)items[i].size();
+    // Omega (drawn by the library, or the caller's copied into the block's buffer) and the transposed gradients
+    const int nl_ = (int)list.size();
+    bool all_given = omegas != nullptr;
+    int nmax_fast = 0;
     for (size_t j = 0; j < list.size(); ++j) {
-        Block &b = ctx->blocks[list[j]];
-        if (!(omegas && omegas[j]))
-            TSR_KERNEL(ctx, 1, fill_gaussian(b.Om, (int64_t)b.d.n * b.k, seed, (uint64_t)list[j], st));
-        if (b.fast)
-            TSR_KERNEL(ctx, 1, transpose_bf16((const bf16 *)b.p.G, (int)b.d.m, (int)b.d.n, b.d.ldg, b.Gt, b.ml, st));
+        const Block &b = ctx->blocks[list[j]];
+        if (!(omegas && omegas[j])) all_given = false;
+        if (b.fast) nmax_fast = std::max(nmax_fast, (int)b.d.n);
     }
+    if (!all_given) TSR_KERNEL(ctx, 1, fill_gaussian_batched(ctx->d_refresh, L.dlist, nl_, seed, st));
+    if (omegas)
+        for (size_t j = 0; j < list.size(); ++j) {
+            Block &b = ctx->blocks[list[j]];
+            if (omegas[j])
+                TSR_CUDA(ctx, cudaMemcpyAsync(b.Om, omegas[j], (size_t)b.d.n * b.k * sizeof(float), cudaMemcpyDeviceToDevice, st));
+        }
+    if (nmax_fast > 0) TSR_KERNEL(ctx, 1, transpose_g_batched(ctx->d_refresh, L.ditems[0], L.nitems[0], nmax_fast, st));
     // Y = G Omega; Q = orth(Y)
     if ((s = sketch(ctx, L, false, true, omegas, st, 1)) != TSR_OK) return s;
     if ((s = orth(ctx, L, 0, qmax == 0, st)) != TSR_OK) return s;
@@ -757,7 +856,8 @@ tsr_status do_refresh_group(tsr_ctx *ctx, const std::vector<int> &list, uint64_t
         std::vector<RowItem> panels;
         for (int bi : list)
             for (int r0 = 0; r0 < ctx->blocks[bi].k; r0 += pr) panels.push_back({bi, r0});
-        TSR_CUDA(ctx, cudaMemcpyAsync(L.ditems[4], panels.data(), panels.size() * sizeof(RowItem), cudaMemcpyHostToDevice, st));
+        if (!cached)
+            TSR_CUDA(ctx, cudaMemcpyAsync(L.ditems[4], panels.data(), panels.size() * sizeof(RowItem), cudaMemcpyHostToDevice, st));
         TSR_KERNEL(ctx, 16, eig_tridiag_batched(ctx->d_refresh, L.dlist, nl, L.ditems[4], (int)panels.size(), L.kmax, st));
     } else {
         TSR_KERNEL(ctx, 1, jacobi_batched(ctx->d_refresh, L.dlist, nl, 40, st));
@@ -782,7 +882,7 @@ tsr_status do_refresh_group(tsr_ctx *ctx, const std::vector<int> &list, uint64_t
             TSR_KERNEL(ctx, 1, simt_gemm(r, r, r, b.Ra, TSR_F32, r, 1, b.p.M, r, 1, b.Rt, r, SIMT_STORE, 0, 0, st));
             TSR_KERNEL(ctx, 1, simt_gemm(r, r, r, b.Rt, TSR_F32, r, 1, b.Rb, r, 1, b.p.M, r, SIMT_STORE, 0, 0, st));
         }
-    return do_shadows(ctx, list, st);
+    return do_shadows(ctx, list, L.ditems[0], L.nitems[0], L.ditems[2], L.nitems[2], st);
 }
 
 // Refresh of a list of blocks (all with the same q).  Large lists are cut into up to NGROUP groups
@@ -794,13 +894,29 @@ tsr_status do_refresh(tsr_ctx *ctx, const std::vector<int> &list, uint64_t seed,
     if (list.empty()) return TSR_OK;
     const size_t zero[5] = {0, 0, 0, 0, 0};
     int ngroup = std::min<int>(tsr_ctx::NGROUP, (int)list.size() / 8);
-    if (!ctx->aux_ready || ngroup < 2) return do_refresh_group(ctx, list, seed, omegas, st, 0, zero, reexpress);
+    if (!ctx->aux_ready || ngroup < 2) {
+        std::vector<int> sig = list;
+        sig.push_back(-1);
+        const bool cached = (sig == ctx->refresh_sig);
+        ctx->refresh_sig.clear();
+        const tsr_status s1 = do_refresh_group(ctx, list, seed, omegas, st, 0, zero, reexpress, cached);
+        if (s1 == TSR_OK) ctx->refresh_sig.swap(sig);
+        return s1;
+    }
     // order the listed blocks as the tile tables do, remembering each one's omega
     std::vector<int> pos(ctx->blocks.size(), 0);
     for (size_t i = 0; i < ctx->order.size(); ++i) pos[ctx->order[i]] = (int)i;
     std::vector<size_t> perm(list.size());
     for (size_t i = 0; i < perm.size(); ++i) perm[i] = i;
     std::sort(perm.begin(), perm.end(), [&](size_t x, size_t y) { return pos[list[x]] < pos[list[y]]; });
+    std::vector<int> sig;
+    for (int g = 0; g < ngroup; ++g) {
+        const size_t lo = perm.size() * g / ngroup, hi = perm.size() * (g + 1) / ngroup;
+        for (size_t i = lo; i < hi; ++i) sig.push_back(list[perm[i]]);
+        sig.push_back(-1);
+    }
+    const bool cached = (sig == ctx->refresh_sig);
+    ctx->refresh_sig.clear();
     TSR_CUDA(ctx, cudaEventRecord(ctx->ev_fork, st));
     size_t list_off = 0, item_off[5] = {0, 0, 0, 0, 0};
     tsr_status result = TSR_OK;
@@ -815,7 +931,7 @@ tsr_status do_refresh(tsr_ctx *ctx, const std::vector<int> &list, uint64_t seed,
         if (cudaStreamWaitEvent(ctx->aux[g], ctx->ev_fork, 0) != cudaSuccess)
             result = fail(ctx, TSR_ERR_CUDA, "cudaStreamWaitEvent failed on a refresh side stream");
         else
-            result = do_refresh_group(ctx, grp, seed, omegas ? om.data() : nullptr, ctx->aux[g], list_off, item_off, reexpress);
+            result = do_refresh_group(ctx, grp, seed, omegas ? om.data() : nullptr, ctx->aux[g], list_off, item_off, reexpress, cached);
         // The side stream is joined whether or not its group was issued completely: the caller's
         // stream must not run ahead of (and the caller must not free buffers under) work in flight.
         if (cudaEventRecord(ctx->ev_join[g], ctx->aux[g]) != cudaSuccess ||
@@ -833,6 +949,7 @@ tsr_status do_refresh(tsr_ctx *ctx, const std::vector<int> &list, uint64_t seed,
             item_off[4] += (size_t)((b.k + 7) / 8);
         }
     }
+    if (result == TSR_OK) ctx->refresh_sig.swap(sig);
     return result;
 }
 
@@ -1008,6 +1125,8 @@ tsr_status tsr_bind(tsr_ctx *ctx, const tsr_mat_ptrs *ptrs, int32_t count, void 
     if (cudaGetDeviceCount(&dev_count) != cudaSuccess || dev_count <= 0)
         return fail(ctx, TSR_ERR_CUDA, "no CUDA device available");
     ctx->bound = false;
+    ctx->refresh_sig.clear();
+    ctx->list_cache[0].clear(); ctx->list_cache[1].clear();
     bool layout_changed = false;
     for (int i = 0; i < count; ++i) {
         Block &b = ctx->blocks[i];
@@ -1072,6 +1191,9 @@ tsr_status tsr_bind(tsr_ctx *ctx, const tsr_mat_ptrs *ptrs, int32_t count, void 
         rd.tau = b.tau; rd.dvec = b.dvec; rd.evec = b.evec; rd.rot = b.rot; rd.sweeps = b.sweeps; rd.groups = b.groups; rd.nsweeps = b.nsweeps;
         rd.rank = b.rank; rd.rot_cap = b.rot_cap; rd.sweep_cap = b.sweep_cap;
         rd.max_sweeps = ctx->max_sweeps[i];
+        rd.fast = b.fast ? 1 : 0;
+        rd.G = (const bf16 *)b.p.G; rd.ldg = b.d.ldg; rd.Om = b.Om; rd.Gt = b.Gt; rd.Xt = b.Xt;
+        rd.Ub = b.Ub; rd.Ubt = b.Ubt; rd.Vb = b.Vb; rd.Vbt = b.Vbt; rd.ml = b.ml; rd.nl = b.nl; rd.rl = b.rl;
         rd.dc_z = b.dc_z; rd.dc_nd = b.dc_nd; rd.dc_rot_idx = b.dc_rot_idx; rd.dc_rot_cs = b.dc_rot_cs;
         rd.dc_scal = b.dc_scal; rd.dc_info = b.dc_info;
         if (!b.fast) continue;
@@ -1113,6 +1235,11 @@ tsr_status tsr_bind(tsr_ctx *ctx, const tsr_mat_ptrs *ptrs, int32_t count, void 
             P.out = (b.nsplit > 1) ? (void *)b.partial : (void *)b.p.C;
             P.ld_out = r; P.split_stride = r * r;
             P.mom1 = b.p.M; P.mom2 = b.p.Vm; P.d_bf16 = b.right_first ? b.Db : nullptr; P.dt_bf16 = b.Dbt; P.ldd = b.rl;
+        }
+        {   // the same core problem for the merged projection launch: B boxes as wide as that launch's tiles
+            UmmaProblem &P = probs[KCM][i];
+            P = probs[KC][i];
+            if ((s = encode_map(ctx, &P.tmB, b.Tt, r, m, b.ml, ctx->bn[KCM] / 2)) != TSR_OK) return s;
         }
         // The lift U D V^T goes through the smaller of the two intermediates: P = U D (m x r) when m <= n,
         // Z^T = V D^T (n x r) when m > n; either one lives in Pb and is the apply kernel's A or B operand.
@@ -1204,7 +1331,21 @@ tsr_status tsr_bases_changed(tsr_ctx *ctx, const int32_t *idx, int32_t count, vo
     if (s != TSR_OK) return s;
     std::vector<int> list;
     if ((s = resolve_list(ctx, idx, count, list)) != TSR_OK) return s;
-    return do_shadows(ctx, list, (cudaStream_t)stream);
+    // slab tables of the listed blocks, at the start of the refresh tables (whose cached contents are dropped)
+    std::vector<RowItem> items[2];
+    for (int bi : list) {
+        const Block &b = ctx->blocks[bi];
+        for (int r0 = 0; r0 < b.d.m; r0 += RG_ROWS) items[0].push_back({bi, r0});
+        for (int r0 = 0; r0 < b.d.n; r0 += RG_ROWS) items[1].push_back({bi, r0});
+    }
+    ctx->refresh_sig.clear();
+    cudaStream_t st = (cudaStream_t)stream;
+    for (int side = 0; side < 2; ++side)
+        if (!items[side].empty())
+            TSR_CUDA(ctx, cudaMemcpyAsync(ctx->d_items[side * 2], items[side].data(), items[side].size() * sizeof(RowItem),
+                                          cudaMemcpyHostToDevice, st));
+    // the copy above reads pageable host memory that goes out of scope: the runtime stages it before returning
+    return do_shadows(ctx, list, ctx->d_items[0], (int)items[0].size(), ctx->d_items[2], (int)items[1].size(), st);
 }
 
 static tsr_status refresh_listed(tsr_ctx *ctx, const int32_t *idx, int32_t count, uint64_t seed,

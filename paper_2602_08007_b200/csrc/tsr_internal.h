@@ -28,7 +28,8 @@ enum UmmaEpilogue : int {
     EPI_STORE_BF16 = 1,    // out_bf16[row * ld + col] = bf16(acc)
     EPI_STORE_BF16_T = 2,  // out_bf16[col * ld + row] = bf16(acc)          (transposed)
     EPI_CORE_UPDATE = 3,   // acc is a tile of the core C: write C, update M / Vm, write D, D^T as BF16
-    EPI_APPLY = 4          // W[row * ld + col] = decay * W - step_scale * acc
+    EPI_APPLY = 4,         // W[row * ld + col] = decay * W - step_scale * acc
+    EPI_RUNTIME = 5        // kernel instantiation whose epilogue is chosen per tile (the merged projection launch)
 };
 
 struct alignas(64) UmmaProblem {
@@ -60,6 +61,11 @@ struct UmmaTile {
     int32_t kb0, kb1;      // range of 64-wide K blocks [kb0, kb1)
     int32_t split;         // split-K slab index (0 when not split)
     int32_t nw;            // width of the tile in columns (a multiple of 16, at most the kernel's tile width); 0: the full width
+    // merged projection launch only (zero elsewhere)
+    int32_t kind;          // 0: a tile of T~ = (G V)^T (first problem table); 1: a tile of the core C = U^T T (second table)
+    int32_t wait_slot;     // kind 1: counter that must reach wait_count before the tile's B operand (T~) may be loaded; -1: none
+    int32_t wait_count;
+    int32_t signal_slot;   // kind 0: counter every epilogue warp of the tile increments once its stores are visible; -1: none
 };
 
 struct StepScalars {       // per-step scalars shared by all blocks
@@ -76,6 +82,17 @@ struct StepScalars {       // per-step scalars shared by all blocks
 cudaError_t umma_gemm_launch(const UmmaProblem *probs, const UmmaTile *tiles, int num_tiles, int num_sms, int bn,
                              int epilogue, int planes, const StepScalars &sc, int32_t *status, cudaStream_t stream);
 cudaError_t umma_configure();  // sets the dynamic shared-memory attributes once per process
+// Arrivals one finished tile of kind 0 adds to its counter (every epilogue warp of both CTAs of the pair).
+constexpr int UMMA_SIGNALS_PER_TILE = 16;
+// The merged projection launch (Section 3.3 in one kernel): tiles of T~ = (G V)^T (problems probs_t) and, a few blocks
+// behind them in the same table, the tiles of C = U^T T (problems probs_c) that read T~ back while it is still in L2.
+// A core tile waits (bounded) on a counter in `counters` that the T~ tiles it depends on advance; the launch is
+// cooperative, so that all CTAs are resident while any of them waits.  fuse != 0: core tiles run the fused core update.
+// counters: nslots dependency counters (one per block) followed by the tile counter (nslots + 1 words); they must
+// be zero at launch.  Returns cudaErrorNotSupported when the device cannot hold the whole grid at once.
+cudaError_t umma_project_launch(const UmmaProblem *probs_t, const UmmaProblem *probs_c, const UmmaTile *tiles, int num_tiles,
+                                int num_sms, int bn, int fuse, int32_t *counters, const StepScalars &sc, int32_t *status,
+                                cudaStream_t stream, int nslots);
 // Persistent apply kernel (tsr_umma_apply.cu): W <- decay W - step_scale P V^T over a tile table.
 cudaError_t umma_apply_configure();
 // w_bytes: 4 = FP32 weights, 2 = BF16 weights (the tile table must not mix them).
@@ -121,6 +138,20 @@ cudaError_t transpose_bf16(const bf16 *in, int rows, int cols, int64_t ldi, bf16
 cudaError_t split_transpose(const float *X, int rows, int k, bf16 *out, int64_t ldo, int plane_rows, int planes,
                             cudaStream_t stream);
 cudaError_t fill_gaussian(float *out, int64_t count, uint64_t seed, uint64_t stream_id, cudaStream_t stream);
+// The same conversions for a whole list of blocks in one launch each, driven by the RefreshDev table (blocks
+// that are not on the tensor-core path are skipped, except by the Gaussian fill).  items: 128-row slabs
+// (block, row0) of the side the rows come from; list: the block indices.
+struct RefreshDev;
+struct RowItem;
+// Om of every listed block from (seed, block index); skip[j] != 0 leaves block list[j] alone (caller-given Omega).
+cudaError_t fill_gaussian_batched(const RefreshDev *rd, const int32_t *list, int nlist, uint64_t seed, cudaStream_t stream);
+// Gt = G^T for every listed block; items: slabs of the m rows of G; nmax: largest n in the list.
+cudaError_t transpose_g_batched(const RefreshDev *rd, const RowItem *items, int nitems, int nmax, cudaStream_t stream);
+// Xt planes of X = Om (src_sel = -1) or buf[src_sel]; side: 0 = X has m rows, 1 = n rows.
+cudaError_t split_transpose_batched(const RefreshDev *rd, const RowItem *items, int nitems, int side, int src_sel, int planes,
+                                    int kmax, cudaStream_t stream);
+// BF16 copies of U (side 0) or V (side 1) and of their transposes.
+cudaError_t shadows_batched(const RefreshDev *rd, const RowItem *items, int nitems, int side, int rmax, cudaStream_t stream);
 cudaError_t fill_zero_f32(float *p, int64_t count, cudaStream_t stream);
 
 // ---------------------------------------------------------------------------------------
@@ -140,6 +171,15 @@ struct RefreshDev {
     float *Xs, *Bts;    // TF32 operand planes of the tensor-core row products (may be NULL)
     float *U, *V;       // the block's bases (FP32 masters)
     int32_t *status;    // the block's status word
+    // operand copies of the tensor-core path (fast != 0), written by the batched conversion kernels
+    int32_t fast;
+    const bf16 *G;      // the bound gradient (BF16 on this path), leading dimension ldg
+    int64_t ldg;
+    float *Om;          // n x k test matrix of the sketch
+    bf16 *Gt;           // G^T, n x ml
+    bf16 *Xt;           // sketch operand planes X^T hi / lo, 2k x max(ml, nl)
+    bf16 *Ub, *Ubt, *Vb, *Vbt;   // BF16 copies of the bases: U (m x rl), U^T (r x ml), V (n x rl), V^T (r x nl)
+    int64_t ml, nl, rl; // padded leading dimensions of the copies
     // tridiagonal eigen-solver (tsr_eig.cu)
     double *tau, *dvec, *evec;   // k each: reflector scales, diagonal / eigenvalues, off-diagonal
     double2 *rot;                // logged plane rotations (c, s)

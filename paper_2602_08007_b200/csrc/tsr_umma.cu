@@ -56,15 +56,18 @@ struct UmmaSmem {
     static constexpr int PATCH_OFFSET = STAGES * STAGE_BYTES;
     static constexpr int PATCH_BYTES = 32 * 33 * 4;                  // per epilogue warp
     static constexpr int BAR_OFFSET = PATCH_OFFSET + UG_EPI_WARPS * PATCH_BYTES;
-    static constexpr int NBARS = 2 * STAGES + 4;
+    static constexpr int SCHED_SLOTS = 4;                            // ring of tile indices (dynamic tile order)
+    static constexpr int NBARS = 2 * STAGES + 4 + 2 * SCHED_SLOTS;
     static constexpr int TOTAL = BAR_OFFSET + NBARS * 8 + 64 + 1024;  // + slack for 1024-byte alignment
 };
 
 template <int BN, int EPI, int PLANES>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(UG_THREADS, 1)
 umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restrict__ tiles, int num_tiles,
-                 StepScalars sc, int32_t *__restrict__ status)
+                 StepScalars sc, int32_t *__restrict__ status, const UmmaProblem *__restrict__ probs2, int32_t *counters,
+                 int fuse, int nslots)
 {
+    // counters (merged projection launch): [0, nslots) dependency counters, [nslots] the tile counter
     using SM = UmmaSmem<BN, PLANES>;
     constexpr int STAGES = SM::STAGES;
     constexpr uint32_t TMEM_COLS = 2 * BN;   // 256 or 512
@@ -75,7 +78,18 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
     uint64_t *bar_full = bars, *bar_empty = bars + STAGES;
     uint64_t *bar_acc_full = bars + 2 * STAGES, *bar_acc_empty = bar_acc_full + 2;
     uint32_t *tmem_slot = (uint32_t *)(bars + SM::NBARS);
-    __shared__ int s_timeout;   // 0, or 1 + the first tile (table index) this CTA gave up on
+    __shared__ int s_timeout;   // 0, or 1 + the first tile (table index) this CTA gave up on (INT_MAX: a wait outside any tile)
+    __shared__ int s_fetched, s_done[UG_EPI_WARPS];   // dynamic order: tiles this CTA's producer saw / each epilogue warp finished
+    // Tile order.  Fixed instantiations: static round-robin, pair p takes tiles p, p + pairs, ...  The merged
+    // projection launch (DYN): tiles are handed out in table order by a global counter, so a pair that draws short
+    // tiles simply draws more of them, and a tile is never started before every earlier tile has been (which bounds
+    // how long a core tile waits for the T~ tiles it depends on).  The leader's producer thread draws the index and
+    // publishes it through a ring of SCHED_SLOTS slots (sched_tile, "full" barriers in both CTAs, one "empty" barrier
+    // in the leader) to the other roles of the pair: the peer's producer, the MMA thread, the sixteen epilogue warps.
+    constexpr bool DYN = (EPI == EPI_RUNTIME);
+    constexpr int SR = SM::SCHED_SLOTS;
+    uint64_t *bar_sfull = bar_acc_empty + 2, *bar_sempty = bar_sfull + SR;
+    volatile int *sched_tile = (volatile int *)(tmem_slot + 1);     // [SR]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const long long budget = wait_budget(sc);
@@ -85,29 +99,77 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
 
     if (threadIdx.x == 0) {
         s_timeout = 0;
+        s_fetched = 0;
+        for (int w = 0; w < UG_EPI_WARPS; ++w) s_done[w] = 0;
+        for (int s = 0; s < SR; ++s) sched_tile[s] = -1;
         for (int s = 0; s < STAGES; ++s) { mbar_init(smem_u32(bar_full + s), 1); mbar_init(smem_u32(bar_empty + s), 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(bar_acc_full + b), 1); mbar_init(smem_u32(bar_acc_empty + b), 2 * UG_EPI_WARPS); }
+        // readers of a slot: MMA thread + 8 epilogue warps of the leader, producer + 8 epilogue warps of the peer
+        for (int s = 0; s < SR; ++s) { mbar_init(smem_u32(bar_sfull + s), 1); mbar_init(smem_u32(bar_sempty + s), 2 * UG_EPI_WARPS + 2); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {   // the same warp of both CTAs allocates the pair's tensor memory
         asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
                      "r"(TMEM_COLS)
                      : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
     __syncthreads();
     cluster_sync();      // the peer's barriers are initialised before anything signals them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    // The permit to allocate is given up only now, when BOTH CTAs of the pair hold their tensor memory (the
+    // cluster barrier above): under cta_group::2 the permit belongs to the pair, and a CTA that relinquished it
+    // while its peer had not yet allocated left the peer waiting in tcgen05.alloc for ever (seen when other
+    // kernels on the same SMs delayed one of the two warps).
+    if (warp == 1) asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+
+    // i-th tile of this pair, for a reader of the ring (every role but the leader's producer): false when the wait ran
+    // out; t < 0 when the table is exhausted.  `arrive`: this thread releases the slot (one lane per epilogue warp).
+    // `whole_warp`: all 32 lanes call together (the epilogue warps); the slot is released only after every lane has read it.
+    auto next_tile = [&](uint32_t i, int &t, bool arrive, bool whole_warp = false) -> bool {
+        if (!DYN) {
+            t = pair + (int)i * stride;
+            if (t >= num_tiles) t = -1;
+            return true;
+        }
+        const int s = (int)(i % SR);
+        bool got = mbar_wait_cluster(smem_u32(bar_sfull + s), (i / SR) & 1u, budget);
+        if (whole_warp) got = __all_sync(0xffffffffu, got);   // a warp gives up as a whole
+        if (!got) return false;
+        t = sched_tile[s];
+        if (whole_warp) __syncwarp();
+        if (arrive) mbar_arrive_leader(smem_u32(bar_sempty + s));
+        return true;
+    };
 
     if (warp == 0) {
         if (lane == 0) {
             uint32_t it = 0;
             bool ok = true;
-            for (int t = pair; t < num_tiles && ok; t += stride) {
+            for (uint32_t ti = 0; ok; ++ti) {
+                int t;
+                if (DYN && rank == 0) {
+                    // draw the next tile of the table and publish it to both CTAs
+                    const int s = (int)(ti % SR);
+                    if (!mbar_wait(smem_u32(bar_sempty + s), ((ti / SR) & 1u) ^ 1u, budget)) { note_timeout(&s_timeout, 0x7ffffffe); break; }
+                    t = atomicAdd(counters + nslots, 1);
+                    if (t >= num_tiles) t = -1;
+                    sched_tile[s] = t;
+                    st_shared_peer(smem_u32((const void *)(sched_tile + s)), 1, t);
+                    mbar_arrive_rank(smem_u32(bar_sfull + s), 0);
+                    mbar_arrive_rank(smem_u32(bar_sfull + s), 1);
+                } else if (!next_tile(ti, t, true)) { note_timeout(&s_timeout, 0x7ffffffe); break; }
+                if (t < 0) break;
+                if (DYN) s_fetched = (int)ti + 1;
                 const UmmaTile tile = tiles[t];
-                const UmmaProblem *P = probs + tile.prob;
+                const UmmaProblem *P = ((EPI == EPI_RUNTIME && tile.kind) ? probs2 : probs) + tile.prob;
+                if (EPI == EPI_RUNTIME && tile.kind && tile.wait_slot >= 0) {
+                    // the tile's B operand is T~, written by earlier tiles of this launch (on other SMs): wait until all
+                    // of them have published their stores, then order the TMA (async proxy) reads behind the acquire
+                    if (!counter_wait(counters + tile.wait_slot, tile.wait_count, budget)) { note_timeout(&s_timeout, t); break; }
+                    asm volatile("fence.proxy.async;" ::: "memory");
+                }
                 if (P->starve) {   // diagnostic: nothing is loaded for this tile, so every consumer's bounded wait runs out
                     note_timeout(&s_timeout, t);
                     break;
@@ -138,9 +200,12 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
         if (lane == 0 && rank == 0) {   // the leader issues the pair's MMAs (256 x N x 16 each)
             uint32_t it = 0, tc = 0;
             bool ok = true;
-            for (int t = pair; t < num_tiles && ok; t += stride, ++tc) {
+            for (; ok; ++tc) {
+                int t;
+                if (!next_tile(tc, t, true)) { note_timeout(&s_timeout, 0x7ffffffe); break; }
+                if (t < 0) break;
                 const UmmaTile tile = tiles[t];
-                int n_eff = probs[tile.prob].N - tile.n0;
+                int n_eff = (((EPI == EPI_RUNTIME && tile.kind) ? probs2 : probs) + tile.prob)->N - tile.n0;
                 n_eff = tile.nw > 0 ? tile.nw : (n_eff >= BN ? BN : ((n_eff + 15) & ~15));
                 const uint32_t idesc = PLANES == 3 ? umma_idesc_pair_tf32(n_eff) : umma_idesc_pair(n_eff);
                 const uint32_t buf = tc & 1u;
@@ -188,16 +253,22 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
         uint32_t nbox = 0;       // EPI_STORE_BF16 through TMA: boxes written so far
         uint32_t tc = 0;
         bool ok = true;
-        for (int t = pair; t < num_tiles && ok; t += stride, ++tc) {
+        for (; ok; ++tc) {
+            int t;
+            if (!next_tile(tc, t, lane == 0, true)) { note_timeout(&s_timeout, 0x7ffffffe); break; }
+            if (t < 0) break;
             const UmmaTile tile = tiles[t];
-            const UmmaProblem *__restrict__ P = probs + tile.prob;
+            const UmmaProblem *__restrict__ P = ((EPI == EPI_RUNTIME && tile.kind) ? probs2 : probs) + tile.prob;
+            // the tile's epilogue: fixed by the instantiation, or (merged projection launch) by the tile's kind
+            const int epi = (EPI != EPI_RUNTIME) ? EPI
+                            : (tile.kind == 0 ? (int)EPI_STORE_BF16_T : (fuse ? P->epilogue : (int)EPI_STORE_F32));
             const uint32_t buf = tc & 1u;
             const int N = P->N, M = P->M;
             const int Nt = tile.nw > 0 ? min(N, tile.n0 + tile.nw) : N;   // first column past this tile
             const int row0 = tile.m0 + (int)rank * UM_BM + q * 32;   // this CTA holds rows 128 rank .. of the tile
             // a split-K problem inside a core-update launch only stores its slab
-            const bool store_f32 = (EPI == EPI_STORE_F32) || (EPI == EPI_CORE_UPDATE && P->epilogue == EPI_STORE_F32);
-            if (EPI == EPI_CORE_UPDATE && !store_f32) {
+            const bool store_f32 = (epi == EPI_STORE_F32) || (epi == EPI_CORE_UPDATE && P->epilogue == EPI_STORE_F32);
+            if (epi == EPI_CORE_UPDATE && !store_f32) {
                 // pull this warp's slice of the moments towards L2 while the MMAs of the tile run
                 const int prow = row0 + lane;
                 if (prow < M) {
@@ -210,13 +281,16 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
                     }
                 }
             }
-            if (!mbar_wait(smem_u32(bar_acc_full + buf), (tc >> 1) & 1u, budget)) { note_timeout(&s_timeout, t); ok = false; break; }
+            // (the warp gives up as a whole: the tensor-memory loads below need all 32 lanes)
+            if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(bar_acc_full + buf), (tc >> 1) & 1u, budget))) { note_timeout(&s_timeout, t); ok = false; break; }
             tc_fence_after();
             const int nrows = min(32, M - row0);        // may be <= 0
             const int c_begin = half * (BN / 2), c_end = c_begin + BN / 2;
             if (tile.n0 + c_begin >= Nt) {   // this warp's column half lies outside the tile
                 tc_fence_before();
                 if (lane == 0) mbar_arrive_leader(smem_u32(bar_acc_empty + buf));
+                if (EPI == EPI_RUNTIME && tile.signal_slot >= 0 && lane == 0) counter_signal(counters + tile.signal_slot);
+                if (DYN && lane == 0) s_done[warp - 4] = (int)tc + 1;
                 continue;
             }
 #pragma unroll 1
@@ -231,7 +305,7 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
                 }
                 if (nrows <= 0) continue;
                 const int ncols = min(32, Nt - col0);
-                if (EPI == EPI_STORE_BF16_T) {
+                if (epi == EPI_STORE_BF16_T) {
                     // out[col][row]: for a fixed column the 32 lanes hold 32 consecutive rows
                     bf16 *out = (bf16 *)P->out + (int64_t)col0 * P->ld_out + row0 + lane;
                     if (lane < nrows) {
@@ -256,7 +330,7 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
                     }
                     continue;
                 }
-                if (EPI == EPI_STORE_BF16 && P->out_tma) {
+                if (epi == EPI_STORE_BF16 && P->out_tma) {
                     // The chunk goes to a 32 x 32 BF16 box in shared memory (64-byte rows, 64-byte swizzle;
                     // two boxes per warp inside the patch area) and leaves as one TMA store, which writes
                     // whole lines and clips at the matrix edge.  Direct stores from the lane = row layout
@@ -283,7 +357,7 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
                     ++nbox;
                     continue;
                 }
-                if (EPI == EPI_STORE_BF16 && ncols == 32 && (P->ld_out & 7) == 0 && (col0 & 7) == 0 &&
+                if (epi == EPI_STORE_BF16 && ncols == 32 && (P->ld_out & 7) == 0 && (col0 & 7) == 0 &&
                     (((uintptr_t)P->out) & 15) == 0) {
                     if (lane < nrows) {
                         bf16 *out = (bf16 *)P->out + (int64_t)(row0 + lane) * P->ld_out + col0;
@@ -300,7 +374,7 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
                     }
                     continue;
                 }
-                if (full_chunk && EPI == EPI_CORE_UPDATE && !store_f32) {
+                if (full_chunk && epi == EPI_CORE_UPDATE && !store_f32) {
 #pragma unroll
                     for (int j = 0; j < 32; ++j) patch[lane * 33 + j] = __uint_as_float(v[j]);
                     __syncwarp();
@@ -350,11 +424,11 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
                     float *out = (float *)P->out + (int64_t)tile.split * P->split_stride + (int64_t)row0 * P->ld_out + col;
                     if (col_ok)
                         for (int i = 0; i < nrows; ++i) out[(int64_t)i * P->ld_out] = patch[i * 33 + lane];
-                } else if (EPI == EPI_STORE_BF16) {
+                } else if (epi == EPI_STORE_BF16) {
                     bf16 *out = (bf16 *)P->out + (int64_t)row0 * P->ld_out + col;
                     if (col_ok)
                         for (int i = 0; i < nrows; ++i) out[(int64_t)i * P->ld_out] = __float2bfloat16_rn(patch[i * 33 + lane]);
-                } else if (EPI == EPI_CORE_UPDATE && !store_f32) {
+                } else if (epi == EPI_CORE_UPDATE && !store_f32) {
                     // C, M, Vm are dense r x r (N = r)
                     if (col_ok) {
                         for (int i = 0; i < nrows; ++i) {
@@ -379,9 +453,16 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
                 }
                 __syncwarp();
             }
+            if (EPI == EPI_RUNTIME && tile.signal_slot >= 0) {
+                // this warp's part of the T~ tile is stored: publish it (every lane's stores, then one arrival)
+                __threadfence();
+                __syncwarp();
+                if (lane == 0) counter_signal(counters + tile.signal_slot);
+            }
+            if (DYN && lane == 0) s_done[warp - 4] = (int)tc + 1;
         }
         // TMA stores read their boxes asynchronously: they must have done so before the CTA goes away
-        if (EPI == EPI_STORE_BF16 && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+        if ((EPI == EPI_STORE_BF16 || EPI == EPI_RUNTIME) && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     }
     if (s_timeout) __nanosleep(2000000);   // let copies in flight land before the CTA goes away
     tc_fence_before();
@@ -391,9 +472,22 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
     }
-    // every block that owns a tile this CTA did not finish is flagged
-    if (threadIdx.x == 0 && s_timeout && status)
-        for (int t = s_timeout - 1; t < num_tiles; t += stride) atomicMax(status + probs[tiles[t].prob].block, (int)TSR_ERR_TIMEOUT);
+    // Every block that owns a tile this CTA did not finish is flagged: with the static order, the tile it gave up
+    // on and all its later ones; with the dynamic order (other pairs draw the remaining tiles), the tiles its
+    // producer had drawn that not every epilogue warp has finished (they are still in the ring).
+    if (threadIdx.x == 0 && s_timeout && status) {
+        if (!DYN) {
+            for (int t = s_timeout - 1; t < num_tiles; t += stride) atomicMax(status + probs[tiles[t].prob].block, (int)TSR_ERR_TIMEOUT);
+        } else {
+            if (s_timeout - 1 < num_tiles) atomicMax(status + probs[tiles[s_timeout - 1].prob].block, (int)TSR_ERR_TIMEOUT);
+            int done = s_done[0];
+            for (int w = 1; w < UG_EPI_WARPS; ++w) done = min(done, s_done[w]);
+            for (int i = max(done, s_fetched - SR); i < s_fetched; ++i) {
+                const int t = sched_tile[i % SR];
+                if (t >= 0 && t < num_tiles) atomicMax(status + probs[tiles[t].prob].block, (int)TSR_ERR_TIMEOUT);
+            }
+        }
+    }
 }
 
 template <int BN, int EPI, int PLANES>
@@ -402,7 +496,8 @@ static cudaError_t launch_one(const UmmaProblem *probs, const UmmaTile *tiles, i
 {
     using SM = UmmaSmem<BN, PLANES>;
     const int pairs = num_tiles < num_sms / 2 ? num_tiles : num_sms / 2;
-    umma_gemm_kernel<BN, EPI, PLANES><<<2 * pairs, UG_THREADS, SM::TOTAL, stream>>>(probs, tiles, num_tiles, sc, status);
+    umma_gemm_kernel<BN, EPI, PLANES><<<2 * pairs, UG_THREADS, SM::TOTAL, stream>>>(probs, tiles, num_tiles, sc, status, nullptr,
+                                                                                    nullptr, 0, 0);
     return cudaGetLastError();
 }
 
@@ -428,7 +523,55 @@ cudaError_t umma_configure()
     if ((e = configure_one<256, EPI_STORE_BF16_T, 1>()) != cudaSuccess) return e;
     if ((e = configure_one<128, EPI_CORE_UPDATE, 1>()) != cudaSuccess) return e;
     if ((e = configure_one<256, EPI_CORE_UPDATE, 1>()) != cudaSuccess) return e;
+    if ((e = configure_one<128, EPI_RUNTIME, 1>()) != cudaSuccess) return e;
+    if ((e = configure_one<256, EPI_RUNTIME, 1>()) != cudaSuccess) return e;
     return cudaSuccess;
+}
+
+// The merged projection launch.  Its core tiles wait on counters that other CTAs of the same grid advance, so
+// every CTA has to be resident: the launch is cooperative (the driver refuses it, instead of letting it
+// deadlock, when the grid does not fit), and the grid is one CTA pair per two SMs at most.
+template <int BN>
+static cudaError_t project_launch_one(const UmmaProblem *probs_t, const UmmaProblem *probs_c, const UmmaTile *tiles, int num_tiles,
+                                      int num_sms, int fuse, int32_t *counters, const StepScalars &sc, int32_t *status,
+                                      cudaStream_t stream, int nslots)
+{
+    using SM = UmmaSmem<BN, 1>;
+    static int max_clusters = -1;      // clusters of this kernel the device holds at once (queried once)
+    if (max_clusters < 0) {
+        cudaLaunchConfig_t q = {};
+        q.gridDim = dim3(num_sms & ~1, 1, 1);
+        q.blockDim = dim3(UG_THREADS, 1, 1);
+        q.dynamicSmemBytes = SM::TOTAL;
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, (const void *)umma_gemm_kernel<BN, EPI_RUNTIME, 1>, &q) != cudaSuccess) n = 0;
+        max_clusters = n;
+    }
+    int pairs = num_tiles < num_sms / 2 ? num_tiles : num_sms / 2;
+    if (pairs > max_clusters) pairs = max_clusters;
+    if (pairs <= 0) return cudaErrorNotSupported;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * pairs, 1, 1);
+    cfg.blockDim = dim3(UG_THREADS, 1, 1);
+    cfg.dynamicSmemBytes = SM::TOTAL;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, umma_gemm_kernel<BN, EPI_RUNTIME, 1>, probs_t, tiles, num_tiles, sc, status, probs_c, counters,
+                              fuse, nslots);
+}
+
+cudaError_t umma_project_launch(const UmmaProblem *probs_t, const UmmaProblem *probs_c, const UmmaTile *tiles, int num_tiles,
+                                int num_sms, int bn, int fuse, int32_t *counters, const StepScalars &sc, int32_t *status,
+                                cudaStream_t stream, int nslots)
+{
+    if (num_tiles <= 0) return cudaSuccess;
+    if (bn == 256) return project_launch_one<256>(probs_t, probs_c, tiles, num_tiles, num_sms, fuse, counters, sc, status, stream, nslots);
+    if (bn == 128) return project_launch_one<128>(probs_t, probs_c, tiles, num_tiles, num_sms, fuse, counters, sc, status, stream, nslots);
+    return cudaErrorInvalidValue;
 }
 
 cudaError_t umma_gemm_launch(const UmmaProblem *probs, const UmmaTile *tiles, int num_tiles, int num_sms, int bn,

@@ -42,6 +42,57 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, long lo
     }
     return true;
 }
+// Dependency counters between tiles of one (cooperative) launch.  A producer tile's warps call counter_signal
+// after a __threadfence() that follows their stores; a consumer polls with acquire semantics, bounded by the budget.
+__device__ __forceinline__ void counter_signal(int32_t *c)
+{
+    asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(c) : "memory");
+}
+__device__ __forceinline__ bool counter_wait(const int32_t *c, int32_t target, long long budget)
+{
+    int32_t v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(c) : "memory");
+    if (v >= target) return true;
+    const long long t0 = clock64();
+    while (true) {
+        asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(c) : "memory");
+        if (v >= target) return true;
+        if (clock64() - t0 > budget) return false;
+        __nanosleep(64);
+    }
+}
+// Bounded wait on a barrier that a thread of the OTHER CTA of the cluster may have arrived on after writing
+// shared memory of this CTA: acquire at cluster scope.
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, long long budget)
+{
+    const long long t0 = clock64();
+    while (true) {
+        uint32_t ok;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok)
+            : "r"(bar), "r"(parity)
+            : "memory");
+        if (ok) return true;
+        if (clock64() - t0 > budget) return false;
+    }
+}
+// Arrive (release at cluster scope) on the copy of a barrier that lives in CTA `rank` of the cluster.
+__device__ __forceinline__ void mbar_arrive_rank(uint32_t bar, uint32_t rank)
+{
+    uint32_t remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(bar), "r"(rank));
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote) : "memory");
+}
+// 32-bit store into the shared memory of CTA `rank` of the cluster, at the address that `local` has here.
+__device__ __forceinline__ void st_shared_peer(uint32_t local, uint32_t rank, int value)
+{
+    uint32_t remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"(rank));
+    asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(remote), "r"(value) : "memory");
+}
 // The budget a launch runs with: the context's setting, or the default when none was made.
 __device__ __forceinline__ long long wait_budget(const StepScalars &sc)
 {

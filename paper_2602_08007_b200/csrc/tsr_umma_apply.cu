@@ -187,7 +187,7 @@ umma_apply_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restr
         while (cur.tile_idx < num_tiles && ok) {
             const uint32_t buf = tc & 1u;
             if (cur.c == 0) {
-                if (!mbar_wait(smem_u32(bar_acc_full + buf), (tc >> 1) & 1u, budget)) { note_timeout(&s_timeout, cur.tile_idx); ok = false; break; }
+                if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(bar_acc_full + buf), (tc >> 1) & 1u, budget))) { note_timeout(&s_timeout, cur.tile_idx); ok = false; break; }
                 tc_fence_after();
             }
             const uint32_t slot = cons % AP_NBOX;
@@ -198,7 +198,7 @@ umma_apply_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restr
                 tc_fence_before();
                 if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar_acc_empty + buf)) : "memory");
             }
-            if (!mbar_wait(smem_u32(wbar + slot), (cons / AP_NBOX) & 1u, budget)) { note_timeout(&s_timeout, cur.tile_idx); ok = false; break; }
+            if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(wbar + slot), (cons / AP_NBOX) & 1u, budget))) { note_timeout(&s_timeout, cur.tile_idx); ok = false; break; }
             if (WB == 4) {
                 uint8_t *box = boxes + slot * AP_BOX_BYTES + lane * 128;
 #pragma unroll

@@ -3,6 +3,10 @@ import sys
 
 import pytest
 
+# The oracle's OpenMP teams sleep instead of spinning while they wait: the parity tests run the oracle's refresh
+# of several blocks on concurrent host threads (its small SVD is a serial loop), which oversubscribes the cores.
+os.environ.setdefault("OMP_WAIT_POLICY", "passive")
+
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
