@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libtsr.so")
-SOURCES = ["tsr_api.cu", "tsr_simt.cu", "tsr_linalg.cu", "tsr_umma.cu", "tsr_umma_apply.cu", "tsr_noalloc.cu", "tsr_eig.cu", "tsr_dense.cu"]
+SOURCES = ["tsr_api.cu", "tsr_simt.cu", "tsr_linalg.cu", "tsr_umma.cu", "tsr_umma_apply.cu", "tsr_noalloc.cu", "tsr_eig.cu", "tsr_dense.cu", "tsr_gram_i8.cu"]
 
 
 def _newest_source() -> float:

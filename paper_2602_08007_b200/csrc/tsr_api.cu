@@ -19,7 +19,8 @@ namespace {
 // 0 (m) or 1 (n) times R^{-1} into buf[1] / buf[2], and the final U = Q Wu, V = B^T Wv.
 // KCM: the core problems encoded for the merged projection launch (its B boxes follow the tile width of KT);
 // KM: the merged tile table itself (tiles of KT and KCM problems interleaved; it has no problem table of its own).
-enum Kind : int { KT = 0, KC, KP, KA, KY, KZ, KR01, KR02, KR12, KRU, KRV, KO, KOA, KCM, KM, NKIND };
+// KG0 / KG1: the exact integer Gram matrices of the refresh, of matrices with m / n rows.
+enum Kind : int { KT = 0, KC, KP, KA, KY, KZ, KR01, KR02, KR12, KRU, KRV, KO, KOA, KCM, KM, KG0, KG1, NKIND };
 constexpr int TSR_NUM_STAGES = 6;  // refresh, G*V, core GEMM, core update, U*D, apply
 
 struct Block {
@@ -53,6 +54,9 @@ struct Block {
     float *Xs = nullptr, *Bts = nullptr;   // TF32 operand planes (value truncated to TF32, remainder): rows, small matrix^T
     bool tc_rows = false;                  // tall-times-small products of the refresh run on tensor cores
     int32_t *nsweeps = nullptr, *rank = nullptr;
+    int32_t *col_exp = nullptr;            // exact integer Gram: column exponents, digit planes (k x ldp bytes each, six of them)
+    int8_t *planes = nullptr;
+    int64_t ldp = 0;
     int rot_cap = 0, sweep_cap = 0;
     float *Uold = nullptr, *Vold = nullptr, *Ra = nullptr, *Rb = nullptr, *Rt = nullptr;   // moment re-expression
     int tile_begin[NKIND], tile_end[NKIND];
@@ -99,7 +103,7 @@ struct tsr_ctx {
     int max_r = 0, max_k = 0;
     uint64_t launches = 0;                     // kernels launched through this context
     int num_sms = 148;
-    int bn[NKIND] = {128, 128, 128, 128, 128, 128, 256, 256, 256, 256, 256, 128, 128, 128, 128};   // tile width of each GEMM kind
+    int bn[NKIND] = {128, 128, 128, 128, 128, 128, 256, 256, 256, 256, 256, 128, 128, 128, 128, 64, 64};   // tile width of each GEMM kind
     int32_t *d_counters = nullptr;             // merged projection launch: one dependency counter per block
     bool merged_ok = true;                     // cleared when the device refuses the cooperative launch
     bool profiling = false;
@@ -230,6 +234,11 @@ void layout(tsr_ctx *ctx, Arena &a, bool assign, size_t *step_end)
         if (b.tc_rows) {
             void *xs = a.take((size_t)(2 * mx * k) * 4), *bts = a.take((size_t)(2 * k * k) * 4);
             if (assign) { b.Xs = (float *)xs; b.Bts = (float *)bts; }
+        }
+        if (b.fast) {
+            const int64_t ldp = round_up(mx, 16);
+            void *ce = a.take((size_t)k * 4), *pl = a.take((size_t)(6 * k * ldp));
+            if (assign) { b.col_exp = (int32_t *)ce; b.planes = (int8_t *)pl; b.ldp = ldp; }
         }
         void *om = a.take((size_t)(n * k) * 4);
         void *b0 = a.take((size_t)(mx * k) * 4), *b1 = a.take((size_t)(mx * k) * 4), *b2 = a.take((size_t)(mx * k) * 4);
@@ -384,6 +393,25 @@ void build_tiles(tsr_ctx *ctx)
             add_tiles(ctx, KRU, bi, m, r, 2 * k, 0);
             add_tiles(ctx, KRV, bi, n, r, 2 * k, 0);
         }
+        // exact integer Gram matrices: 256 x 64 tiles on or above the diagonal, one per chunk of GRAM_ROWS rows
+        for (int side = 0; side < 2; ++side) {
+            const int kd = KG0 + side, rows = side ? n : m;
+            std::vector<UmmaTile> &v = ctx->tiles[kd];
+            b.tile_begin[kd] = (int)v.size();
+            for (int c = 0; c < gram_chunks(rows); ++c)
+                for (int i0 = 0; i0 < k; i0 += 256)
+                    for (int j0 = 0; j0 < k; j0 += 64) {
+                        if (j0 + 64 <= i0) continue;
+                        UmmaTile t;
+                        memset(&t, 0, sizeof t);
+                        t.prob = bi; t.m0 = i0; t.n0 = j0; t.split = c;
+                        t.kb0 = c * (GRAM_ROWS / 64);
+                        t.kb1 = (std::min(rows, (c + 1) * GRAM_ROWS) + 63) / 64;
+                        t.wait_slot = -1; t.signal_slot = -1;
+                        v.push_back(t);
+                    }
+            b.tile_end[kd] = (int)v.size();
+        }
     }
     build_merged(ctx);
 }
@@ -402,6 +430,22 @@ tsr_status encode_map(tsr_ctx *ctx, CUtensorMap *out, const void *base, int64_t 
     if (rc != CUDA_SUCCESS)
         return fail(ctx, TSR_ERR_CUDA, "cuTensorMapEncodeTiled failed (%d) rows=%lld cols=%lld ld=%lld", (int)rc,
                     (long long)rows, (long long)cols, (long long)ld);
+    return TSR_OK;
+}
+
+// INT8 row-major [rows x cols] (ld bytes) -> tensor map with a 64-byte x box_rows box, 64B swizzle.
+tsr_status encode_map_i8(tsr_ctx *ctx, CUtensorMap *out, const void *base, int64_t rows, int64_t cols, int64_t ld, int box_rows)
+{
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)ld};
+    cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult rc = ctx->encode(out, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(base), dims, strides, box, estr,
+                              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (rc != CUDA_SUCCESS)
+        return fail(ctx, TSR_ERR_CUDA, "cuTensorMapEncodeTiled (digit planes) failed (%d) rows=%lld cols=%lld", (int)rc,
+                    (long long)rows, (long long)cols);
     return TSR_OK;
 }
 
@@ -676,17 +720,18 @@ tsr_status do_apply(tsr_ctx *ctx, const std::vector<int> &list, const StepScalar
     return TSR_OK;
 }
 
-// BF16 operand copies of U and V for the listed blocks.  items_m / items_n: device tables of the 128-row
-// slabs of the m and n sides of exactly those blocks.
-tsr_status do_shadows(tsr_ctx *ctx, const std::vector<int> &list, const RowItem *items_m, int n_m, const RowItem *items_n,
-                      int n_n, cudaStream_t st)
+// BF16 operand copies of U and V for the listed blocks.  One launch per block and basis: measured against a
+// form that converts all blocks of a refresh group in one launch per stage, the refresh of the 1B set took 141 ms
+// this way and 153 ms batched (with the groups on concurrent streams the small launches interleave with the other
+// groups' kernels; the batched ones kept the groups in step with one another).
+tsr_status do_shadows(tsr_ctx *ctx, const std::vector<int> &list, cudaStream_t st)
 {
-    int rmax = 0;
-    for (int bi : list)
-        if (ctx->blocks[bi].fast) rmax = std::max(rmax, (int)ctx->blocks[bi].d.r);
-    if (rmax == 0) return TSR_OK;
-    TSR_KERNEL(ctx, 1, shadows_batched(ctx->d_refresh, items_m, n_m, 0, rmax, st));
-    TSR_KERNEL(ctx, 1, shadows_batched(ctx->d_refresh, items_n, n_n, 1, rmax, st));
+    for (int bi : list) {
+        Block &b = ctx->blocks[bi];
+        if (!b.fast) continue;
+        TSR_KERNEL(ctx, 1, make_shadows(b.p.U, (int)b.d.m, b.d.r, b.Ub, b.rl, b.Ubt, b.ml, st));
+        TSR_KERNEL(ctx, 1, make_shadows(b.p.V, (int)b.d.n, b.d.r, b.Vb, b.rl, b.Vbt, b.nl, st));
+    }
     return TSR_OK;
 }
 
@@ -726,11 +771,46 @@ tsr_status rows_product(tsr_ctx *ctx, const RefreshLists &L, int side, int src, 
     return launch_kind(ctx, kind, L.list, EPI_STORE_F32, 3, sc, st);
 }
 
+// S = X^T X (X = buf[src], FP64 result) for every block of the group.  Blocks on the tensor-core path whose sketch
+// is a genuine sketch (k <= min(m, n) / 2) take the integer form (digit planes, INT8 MMAs, see tsr_gram_i8.cu): it
+// carries 42 bits below each column's largest entry, i.e. S to about 5e-11 relative to |x_i| |x_j|, against the
+// kappa(X)^2 <= 5e8 of such sketches.  A sketch as wide as the matrix (the exact-SVD arm: kappa(X)^2 up to 1e14)
+// needs everything FP64 has, and goes, like any block off the tensor-core path, through the FP64 tensor path.
+tsr_status gram(tsr_ctx *ctx, const RefreshLists &L, int side, int src, cudaStream_t st)
+{
+    const int nl = (int)L.list.size();
+    bool i8 = true;
+    for (int bi : L.list) {
+        const Block &b = ctx->blocks[bi];
+        i8 = i8 && b.fast && 2 * (int64_t)b.k <= std::min(b.d.m, b.d.n);
+    }
+    if (!i8) {
+        TSR_KERNEL(ctx, 2, gram_batched(ctx->d_refresh, L.ditems[side * 2 + 1], L.nitems[side * 2 + 1], L.dlist, nl, side, src,
+                                        L.kmax, st));
+        return TSR_OK;
+    }
+    TSR_KERNEL(ctx, 2, gram_i8_prepare(ctx->d_refresh, L.ditems[side * 2], L.nitems[side * 2], L.dlist, nl, side, src, L.kmax, st));
+    const int kind = KG0 + side;
+    std::vector<std::pair<int, int>> ranges;
+    for (int bi : L.list) ranges.push_back({ctx->blocks[bi].tile_begin[kind], ctx->blocks[bi].tile_end[kind]});
+    std::sort(ranges.begin(), ranges.end());
+    for (size_t i = 0; i < ranges.size();) {
+        int lo = ranges[i].first, hi = ranges[i].second;
+        size_t j = i + 1;
+        while (j < ranges.size() && ranges[j].first == hi) { hi = ranges[j].second; ++j; }
+        TSR_KERNEL(ctx, 1, gram_i8_launch(ctx->d_probs[kind], ctx->d_tiles[kind] + lo, hi - lo, ctx->num_sms, ctx->wait_clocks,
+                                          ctx->d_status, st));
+        i = j;
+    }
+    TSR_KERNEL(ctx, 1, gram_reduce_batched(ctx->d_refresh, L.dlist, nl, side, L.kmax, st));
+    return TSR_OK;
+}
+
 tsr_status orth_pass(tsr_ctx *ctx, const RefreshLists &L, int side, int src, int dst, bool refined_later, cudaStream_t st)
 {
     const int nl = (int)L.list.size();
-    TSR_KERNEL(ctx, 2, gram_batched(ctx->d_refresh, L.ditems[side * 2 + 1], L.nitems[side * 2 + 1], L.dlist, nl, side,
-                               src, L.kmax, st));
+    tsr_status sg = gram(ctx, L, side, src, st);
+    if (sg != TSR_OK) return sg;
     TSR_KERNEL(ctx, 1, chol_inverse_batched(ctx->d_refresh, L.dlist, nl, L.kmax, st));
     return rows_product(ctx, L, side, src, 0, dst, refined_later, st);
 }
@@ -763,17 +843,13 @@ tsr_status sketch(tsr_ctx *ctx, const RefreshLists &L, bool transposed, bool fro
     sc.wait_clocks = ctx->wait_clocks;
     tsr_status s;
     (void)omegas;   // a caller-given Omega has been copied into the block's own buffer by now
-    if (ctx->any_fast) {   // X^T as BF16 plane(s) for every block of the group at once
-        const int side = transposed ? 0 : 1;                     // rows of X: m for G^T X, n for G X
-        TSR_KERNEL(ctx, 1, split_transpose_batched(ctx->d_refresh, L.ditems[side * 2], L.nitems[side * 2], side,
-                                                   from_omega ? -1 : 2, planes, L.kmax, st));
-    }
     for (size_t j = 0; j < L.list.size(); ++j) {
         Block &b = ctx->blocks[L.list[j]];
-        if (b.fast) continue;
         const int m = (int)b.d.m, n = (int)b.d.n, k = b.k;
         const float *X = from_omega ? b.Om : b.buf[2];
-        if (!transposed) {
+        if (b.fast) {   // X^T as BF16 plane(s): the B operand of the sketch GEMM
+            TSR_KERNEL(ctx, 1, split_transpose(X, transposed ? m : n, k, b.Xt, transposed ? b.ml : b.nl, k, planes, st));
+        } else if (!transposed) {
             TSR_KERNEL(ctx, 1, simt_gemm(m, k, n, b.p.G, b.d.g_dtype, b.d.ldg, 1, X, k, 1, b.buf[0], k, SIMT_STORE, 0, 0, st));
         } else {
             TSR_KERNEL(ctx, 1, simt_gemm(n, k, m, b.p.G, b.d.g_dtype, 1, b.d.ldg, X, k, 1, b.buf[0], k, SIMT_STORE, 0, 0, st));
@@ -821,22 +897,15 @@ tsr_status do_refresh_group(tsr_ctx *ctx, const std::vector<int> &list, uint64_t
     }
     for (int i = 0; i < 4; ++i) L.nitems[i] = (int)items[i].size();
     // Omega (drawn by the library, or the caller's copied into the block's buffer) and the transposed gradients
-    const int nl_ = (int)list.size();
-    bool all_given = omegas != nullptr;
-    int nmax_fast = 0;
     for (size_t j = 0; j < list.size(); ++j) {
-        const Block &b = ctx->blocks[list[j]];
-        if (!(omegas && omegas[j])) all_given = false;
-        if (b.fast) nmax_fast = std::max(nmax_fast, (int)b.d.n);
+        Block &b = ctx->blocks[list[j]];
+        if (omegas && omegas[j])
+            TSR_CUDA(ctx, cudaMemcpyAsync(b.Om, omegas[j], (size_t)b.d.n * b.k * sizeof(float), cudaMemcpyDeviceToDevice, st));
+        else
+            TSR_KERNEL(ctx, 1, fill_gaussian(b.Om, (int64_t)b.d.n * b.k, seed, (uint64_t)list[j], st));
+        if (b.fast)
+            TSR_KERNEL(ctx, 1, transpose_bf16((const bf16 *)b.p.G, (int)b.d.m, (int)b.d.n, b.d.ldg, b.Gt, b.ml, st));
     }
-    if (!all_given) TSR_KERNEL(ctx, 1, fill_gaussian_batched(ctx->d_refresh, L.dlist, nl_, seed, st));
-    if (omegas)
-        for (size_t j = 0; j < list.size(); ++j) {
-            Block &b = ctx->blocks[list[j]];
-            if (omegas[j])
-                TSR_CUDA(ctx, cudaMemcpyAsync(b.Om, omegas[j], (size_t)b.d.n * b.k * sizeof(float), cudaMemcpyDeviceToDevice, st));
-        }
-    if (nmax_fast > 0) TSR_KERNEL(ctx, 1, transpose_g_batched(ctx->d_refresh, L.ditems[0], L.nitems[0], nmax_fast, st));
     // Y = G Omega; Q = orth(Y)
     if ((s = sketch(ctx, L, false, true, omegas, st, 1)) != TSR_OK) return s;
     if ((s = orth(ctx, L, 0, qmax == 0, st)) != TSR_OK) return s;
@@ -850,7 +919,7 @@ tsr_status do_refresh_group(tsr_ctx *ctx, const std::vector<int> &list, uint64_t
     // B^T = G^T Q (n x k) in buf[0]; small SVD through the k x k Gram matrix B B^T
     if ((s = sketch(ctx, L, true, false, nullptr, st)) != TSR_OK) return s;
     const int nl = (int)list.size();
-    TSR_KERNEL(ctx, 2, gram_batched(ctx->d_refresh, L.ditems[3], L.nitems[3], L.dlist, nl, 1, 0, L.kmax, st));
+    if ((s = gram(ctx, L, 1, 0, st)) != TSR_OK) return s;
     if (L.kmax >= 200) {   // too large for the Jacobi solver: tridiagonal route
         const int pr = eig_panel_rows(L.kmax);
         std::vector<RowItem> panels;
@@ -882,7 +951,7 @@ tsr_status do_refresh_group(tsr_ctx *ctx, const std::vector<int> &list, uint64_t
             TSR_KERNEL(ctx, 1, simt_gemm(r, r, r, b.Ra, TSR_F32, r, 1, b.p.M, r, 1, b.Rt, r, SIMT_STORE, 0, 0, st));
             TSR_KERNEL(ctx, 1, simt_gemm(r, r, r, b.Rt, TSR_F32, r, 1, b.Rb, r, 1, b.p.M, r, SIMT_STORE, 0, 0, st));
         }
-    return do_shadows(ctx, list, L.ditems[0], L.nitems[0], L.ditems[2], L.nitems[2], st);
+    return do_shadows(ctx, list, st);
 }
 
 // Refresh of a list of blocks (all with the same q).  Large lists are cut into up to NGROUP groups
@@ -1160,6 +1229,7 @@ tsr_status tsr_bind(tsr_ctx *ctx, const tsr_mat_ptrs *ptrs, int32_t count, void 
         }
         TSR_CUDA(ctx, umma_configure());
         TSR_CUDA(ctx, umma_apply_configure());
+        TSR_CUDA(ctx, gram_i8_configure());
         int dev = 0;
         TSR_CUDA(ctx, cudaGetDevice(&dev));
         TSR_CUDA(ctx, cudaDeviceGetAttribute(&ctx->num_sms, cudaDevAttrMultiProcessorCount, dev));
@@ -1191,9 +1261,7 @@ tsr_status tsr_bind(tsr_ctx *ctx, const tsr_mat_ptrs *ptrs, int32_t count, void 
         rd.tau = b.tau; rd.dvec = b.dvec; rd.evec = b.evec; rd.rot = b.rot; rd.sweeps = b.sweeps; rd.groups = b.groups; rd.nsweeps = b.nsweeps;
         rd.rank = b.rank; rd.rot_cap = b.rot_cap; rd.sweep_cap = b.sweep_cap;
         rd.max_sweeps = ctx->max_sweeps[i];
-        rd.fast = b.fast ? 1 : 0;
-        rd.G = (const bf16 *)b.p.G; rd.ldg = b.d.ldg; rd.Om = b.Om; rd.Gt = b.Gt; rd.Xt = b.Xt;
-        rd.Ub = b.Ub; rd.Ubt = b.Ubt; rd.Vb = b.Vb; rd.Vbt = b.Vbt; rd.ml = b.ml; rd.nl = b.nl; rd.rl = b.rl;
+        rd.col_exp = b.col_exp; rd.planes = b.planes; rd.ldp = b.ldp;
         rd.dc_z = b.dc_z; rd.dc_nd = b.dc_nd; rd.dc_rot_idx = b.dc_rot_idx; rd.dc_rot_cs = b.dc_rot_cs;
         rd.dc_scal = b.dc_scal; rd.dc_info = b.dc_info;
         if (!b.fast) continue;
@@ -1284,6 +1352,14 @@ tsr_status tsr_bind(tsr_ctx *ctx, const tsr_mat_ptrs *ptrs, int32_t count, void 
             if ((s = encode_map(ctx, &P.tmB, b.Xt, 2 * k, m, b.ml, ctx->bn[KZ] / 2)) != TSR_OK) return s;
             P.out = b.buf[0]; P.ld_out = k;
         }
+        for (int side = 0; side < 2; ++side) {   // exact integer Gram: the digit planes as a (6 k) x rows INT8 matrix
+            UmmaProblem &P = probs[KG0 + side][i];
+            const int64_t rows = side ? n : m;
+            base(P, (int)k, (int)k, (int)rows, EPI_STORE_F32);
+            if ((s = encode_map_i8(ctx, &P.tmA, b.planes, 6 * k, rows, b.ldp, 128)) != TSR_OK) return s;
+            if ((s = encode_map_i8(ctx, &P.tmB, b.planes, 6 * k, rows, b.ldp, 32)) != TSR_OK) return s;
+            P.out = b.gpart; P.ld_out = k; P.split_stride = k * k; P.col_exp = b.col_exp;
+        }
         if (b.tc_rows) {   // rows [M x k] (planes Xs) times small matrix^T planes Bts [N x k]
             const int64_t mx = std::max(m, n);
             struct { int kd; int64_t M, N; float *out; } rk[5] = {
@@ -1331,21 +1407,7 @@ tsr_status tsr_bases_changed(tsr_ctx *ctx, const int32_t *idx, int32_t count, vo
     if (s != TSR_OK) return s;
     std::vector<int> list;
     if ((s = resolve_list(ctx, idx, count, list)) != TSR_OK) return s;
-    // slab tables of the listed blocks, at the start of the refresh tables (whose cached contents are dropped)
-    std::vector<RowItem> items[2];
-    for (int bi : list) {
-        const Block &b = ctx->blocks[bi];
-        for (int r0 = 0; r0 < b.d.m; r0 += RG_ROWS) items[0].push_back({bi, r0});
-        for (int r0 = 0; r0 < b.d.n; r0 += RG_ROWS) items[1].push_back({bi, r0});
-    }
-    ctx->refresh_sig.clear();
-    cudaStream_t st = (cudaStream_t)stream;
-    for (int side = 0; side < 2; ++side)
-        if (!items[side].empty())
-            TSR_CUDA(ctx, cudaMemcpyAsync(ctx->d_items[side * 2], items[side].data(), items[side].size() * sizeof(RowItem),
-                                          cudaMemcpyHostToDevice, st));
-    // the copy above reads pageable host memory that goes out of scope: the runtime stages it before returning
-    return do_shadows(ctx, list, ctx->d_items[0], (int)items[0].size(), ctx->d_items[2], (int)items[1].size(), st);
+    return do_shadows(ctx, list, (cudaStream_t)stream);
 }
 
 static tsr_status refresh_listed(tsr_ctx *ctx, const int32_t *idx, int32_t count, uint64_t seed,

@@ -52,6 +52,7 @@ struct alignas(64) UmmaProblem {
     bf16 *dt_bf16;         // D^T [r x ldd]
     int64_t ldd;
     int32_t out_tma;       // EPI_STORE_BF16: tmW describes the output, chunks leave through TMA stores
+    const int32_t *col_exp; // integer Gram kernel: the column exponents of the matrix whose digit planes tmA / tmB describe
     int32_t starve;        // diagnostic (tsr_set_limits): the producer issues no loads for this problem's tiles
 };
 
@@ -138,20 +139,6 @@ cudaError_t transpose_bf16(const bf16 *in, int rows, int cols, int64_t ldi, bf16
 cudaError_t split_transpose(const float *X, int rows, int k, bf16 *out, int64_t ldo, int plane_rows, int planes,
                             cudaStream_t stream);
 cudaError_t fill_gaussian(float *out, int64_t count, uint64_t seed, uint64_t stream_id, cudaStream_t stream);
-// The same conversions for a whole list of blocks in one launch each, driven by the RefreshDev table (blocks
-// that are not on the tensor-core path are skipped, except by the Gaussian fill).  items: 128-row slabs
-// (block, row0) of the side the rows come from; list: the block indices.
-struct RefreshDev;
-struct RowItem;
-// Om of every listed block from (seed, block index); skip[j] != 0 leaves block list[j] alone (caller-given Omega).
-cudaError_t fill_gaussian_batched(const RefreshDev *rd, const int32_t *list, int nlist, uint64_t seed, cudaStream_t stream);
-// Gt = G^T for every listed block; items: slabs of the m rows of G; nmax: largest n in the list.
-cudaError_t transpose_g_batched(const RefreshDev *rd, const RowItem *items, int nitems, int nmax, cudaStream_t stream);
-// Xt planes of X = Om (src_sel = -1) or buf[src_sel]; side: 0 = X has m rows, 1 = n rows.
-cudaError_t split_transpose_batched(const RefreshDev *rd, const RowItem *items, int nitems, int side, int src_sel, int planes,
-                                    int kmax, cudaStream_t stream);
-// BF16 copies of U (side 0) or V (side 1) and of their transposes.
-cudaError_t shadows_batched(const RefreshDev *rd, const RowItem *items, int nitems, int side, int rmax, cudaStream_t stream);
 cudaError_t fill_zero_f32(float *p, int64_t count, cudaStream_t stream);
 
 // ---------------------------------------------------------------------------------------
@@ -171,15 +158,11 @@ struct RefreshDev {
     float *Xs, *Bts;    // TF32 operand planes of the tensor-core row products (may be NULL)
     float *U, *V;       // the block's bases (FP32 masters)
     int32_t *status;    // the block's status word
-    // operand copies of the tensor-core path (fast != 0), written by the batched conversion kernels
-    int32_t fast;
-    const bf16 *G;      // the bound gradient (BF16 on this path), leading dimension ldg
-    int64_t ldg;
-    float *Om;          // n x k test matrix of the sketch
-    bf16 *Gt;           // G^T, n x ml
-    bf16 *Xt;           // sketch operand planes X^T hi / lo, 2k x max(ml, nl)
-    bf16 *Ub, *Ubt, *Vb, *Vbt;   // BF16 copies of the bases: U (m x rl), U^T (r x ml), V (n x rl), V^T (r x nl)
-    int64_t ml, nl, rl; // padded leading dimensions of the copies
+    // exact integer Gram matrices (tsr_gram_i8.cu): power-of-two exponent of every column, and the six INT8 digit
+    // planes of the matrix, transposed: planes[s][col][row], row pitch ldp bytes
+    int32_t *col_exp;
+    int8_t *planes;
+    int64_t ldp;
     // tridiagonal eigen-solver (tsr_eig.cu)
     double *tau, *dvec, *evec;   // k each: reflector scales, diagonal / eigenvalues, off-diagonal
     double2 *rot;                // logged plane rotations (c, s)
@@ -207,6 +190,15 @@ __host__ __device__ inline int gram_chunks(int64_t rows) { return (int)((rows + 
 // S = X^T X with X = buf[src_sel] (FP32), FP64 accumulation, deterministic.
 cudaError_t gram_batched(const RefreshDev *rd, const RowItem *items, int nitems, const int32_t *list, int nlist,
                          int side, int src_sel, int kmax, cudaStream_t stream);
+// The same Gram matrix on the integer tensor cores, exact (tsr_gram_i8.cu): gram_i8_prepare writes the column
+// exponents and digit planes of buf[src_sel] (items128: slabs of RG_ROWS rows), gram_i8_launch runs the products over a
+// tile table (problems: digit-plane tensor maps, out = gpart), gram_reduce_batched adds the chunks into S.
+cudaError_t gram_i8_configure();
+cudaError_t gram_i8_prepare(const RefreshDev *rd, const RowItem *items128, int nitems128, const int32_t *list, int nlist,
+                            int side, int src_sel, int kmax, cudaStream_t stream);
+cudaError_t gram_i8_launch(const UmmaProblem *probs, const UmmaTile *tiles, int num_tiles, int num_sms, long long wait_clocks,
+                           int32_t *status, cudaStream_t stream);
+cudaError_t gram_reduce_batched(const RefreshDev *rd, const int32_t *list, int nlist, int side, int kmax, cudaStream_t stream);
 // Cholesky S = R^T R in place and Rinv = float(R^{-1}).
 cudaError_t chol_inverse_batched(const RefreshDev *rd, const int32_t *list, int nlist, int kmax, cudaStream_t stream);
 // dst = buf[src_sel] * Mat;  mat_sel: 0 Rinv (k x k), 1 Wu (k x r), 2 Wv (k x r);

@@ -136,6 +136,12 @@ cudaError_t gram_batched(const RefreshDev *rd, const RowItem *items, int nitems,
     if (nitems <= 0 || nlist <= 0) return cudaSuccess;
     const int t = (kmax + GR_T - 1) / GR_T;
     gram_partial_kernel<<<dim3(t, t, nitems), 256, 0, stream>>>(rd, items, side, src_sel);
+    return gram_reduce_batched(rd, list, nlist, side, kmax, stream);
+}
+
+cudaError_t gram_reduce_batched(const RefreshDev *rd, const int32_t *list, int nlist, int side, int kmax, cudaStream_t stream)
+{
+    if (nlist <= 0) return cudaSuccess;
     int gx = (int)(((int64_t)kmax * kmax + 255) / 256);
     if (gx > 128) gx = 128;
     gram_reduce_kernel<<<dim3(gx, nlist), 256, 0, stream>>>(rd, list, side);

@@ -389,172 +389,6 @@ cudaError_t fill_gaussian(float *out, int64_t count, uint64_t seed, uint64_t str
     return cudaGetLastError();
 }
 
-// ---------------------------------------------------------------------------------------
-// Batched forms of the conversions above: one launch covers a list of blocks.  A CTA takes one
-// 128-row slab (two 64-row tiles) of one block and one tile of columns; blocks whose matrices are
-// narrower than the widest one of the list leave early.
-// ---------------------------------------------------------------------------------------
-__global__ void gaussian_batched_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ list, uint64_t seed)
-{
-    const int block = list[blockIdx.y];
-    const RefreshDev d = rd[block];
-    float *__restrict__ out = d.Om;
-    const int64_t count = (int64_t)d.n * d.k;
-    const uint64_t base = mix64(seed ^ ((uint64_t)block * 0xD1342543DE82EF95ull));
-    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < count; e += (int64_t)gridDim.x * blockDim.x) {
-        const uint64_t h = mix64(base + (uint64_t)e);
-        const uint32_t a = (uint32_t)h, b = (uint32_t)(h >> 32);
-        const float u1 = ((float)(a >> 8) + 0.5f) * (1.0f / 16777216.0f);  // (0,1)
-        const float u2 = ((float)(b >> 8) + 0.5f) * (1.0f / 16777216.0f);
-        out[e] = sqrtf(-2.0f * logf(u1)) * cospif(2.0f * u2);
-    }
-}
-
-cudaError_t fill_gaussian_batched(const RefreshDev *rd, const int32_t *list, int nlist, uint64_t seed, cudaStream_t stream)
-{
-    if (nlist <= 0) return cudaSuccess;
-    gaussian_batched_kernel<<<dim3(64, nlist), 256, 0, stream>>>(rd, list, seed);
-    return cudaGetLastError();
-}
-
-__global__ void transpose_g_batched_kernel(const RefreshDev *__restrict__ rd, const RowItem *__restrict__ items)
-{
-    const RowItem it = items[blockIdx.x];
-    const RefreshDev d = rd[it.block];
-    const int rows = d.m, cols = d.n;
-    const int c0 = blockIdx.y * 64;
-    if (!d.fast || c0 >= cols) return;
-    const bf16 *__restrict__ in = d.G;
-    bf16 *__restrict__ out = d.Gt;
-    const int64_t ldi = d.ldg, ldo = d.ml;
-    const bool in_pairs = ((ldi & 1) == 0) && ((((uintptr_t)in) & 3) == 0);
-    __shared__ bf16 tile[64][66];
-    for (int h = 0; h < RG_ROWS; h += 64) {
-        const int r0 = it.row0 + h;
-        if (r0 >= rows) break;
-        for (int i = threadIdx.y; i < 64; i += blockDim.y) {
-            const int row = r0 + i, col = c0 + 2 * threadIdx.x;
-            uint32_t w = 0;
-            if (row < rows && col < cols) {
-                const bf16 *src = in + (int64_t)row * ldi + col;
-                if (in_pairs && col + 1 < cols) w = *(const uint32_t *)src;
-                else {
-                    const bf16 a = src[0], bq = (col + 1 < cols) ? src[1] : __float2bfloat16_rn(0.f);
-                    w = (uint32_t)(*(const uint16_t *)&a) | ((uint32_t)(*(const uint16_t *)&bq) << 16);
-                }
-            }
-            *(uint32_t *)&tile[i][2 * threadIdx.x] = w;
-        }
-        __syncthreads();
-        for (int i = threadIdx.y; i < 64; i += blockDim.y) {
-            const int col = c0 + i, row = r0 + 2 * threadIdx.x;
-            if (col >= cols || row >= rows) continue;
-            bf16 *dst = out + (int64_t)col * ldo + row;
-            const bf16 a = tile[2 * threadIdx.x][i], bq = tile[2 * threadIdx.x + 1][i];
-            if (row + 1 < rows) *(uint32_t *)dst = (uint32_t)(*(const uint16_t *)&a) | ((uint32_t)(*(const uint16_t *)&bq) << 16);
-            else *dst = a;
-        }
-        __syncthreads();
-    }
-}
-
-cudaError_t transpose_g_batched(const RefreshDev *rd, const RowItem *items, int nitems, int nmax, cudaStream_t stream)
-{
-    if (nitems <= 0) return cudaSuccess;
-    transpose_g_batched_kernel<<<dim3(nitems, (nmax + 63) / 64), dim3(32, 8), 0, stream>>>(rd, items);
-    return cudaGetLastError();
-}
-
-__global__ void split_transpose_batched_kernel(const RefreshDev *__restrict__ rd, const RowItem *__restrict__ items, int side,
-                                               int src_sel, int planes)
-{
-    const RowItem it = items[blockIdx.x];
-    const RefreshDev d = rd[it.block];
-    const int k = d.k, rows = side ? d.n : d.m;
-    const int c0 = blockIdx.y * 32;
-    if (!d.fast || c0 >= k) return;
-    const float *__restrict__ X = (src_sel < 0) ? d.Om : d.buf[src_sel];
-    bf16 *__restrict__ out = d.Xt;
-    const int64_t ldo = side ? d.nl : d.ml;
-    __shared__ float tile[64][33];
-    for (int h = 0; h < RG_ROWS; h += 64) {
-        const int r0 = it.row0 + h;
-        if (r0 >= rows) break;
-        for (int i = threadIdx.y; i < 64; i += blockDim.y) {
-            const int row = r0 + i, col = c0 + threadIdx.x;
-            tile[i][threadIdx.x] = (row < rows && col < k) ? X[(int64_t)row * k + col] : 0.f;
-        }
-        __syncthreads();
-        for (int i = threadIdx.y; i < 32; i += blockDim.y) {
-            const int col = c0 + i, row = r0 + 2 * threadIdx.x;
-            if (col >= k || row >= rows) continue;
-            const float v0 = tile[2 * threadIdx.x][i], v1 = tile[2 * threadIdx.x + 1][i];
-            const bf16 h0 = __float2bfloat16_rn(v0), h1 = __float2bfloat16_rn(v1);
-            bf16 *dhi = out + (int64_t)col * ldo + row;
-            bf16 *dlo = out + ((int64_t)k + col) * ldo + row;
-            if (row + 1 < rows) {
-                *(uint32_t *)dhi = (uint32_t)(*(const uint16_t *)&h0) | ((uint32_t)(*(const uint16_t *)&h1) << 16);
-                if (planes > 1) *(uint32_t *)dlo = pack_bf16x2(v0 - __bfloat162float(h0), v1 - __bfloat162float(h1));
-            } else {
-                *dhi = h0;
-                if (planes > 1) *dlo = __float2bfloat16_rn(v0 - __bfloat162float(h0));
-            }
-        }
-        __syncthreads();
-    }
-}
-
-cudaError_t split_transpose_batched(const RefreshDev *rd, const RowItem *items, int nitems, int side, int src_sel, int planes,
-                                    int kmax, cudaStream_t stream)
-{
-    if (nitems <= 0) return cudaSuccess;
-    split_transpose_batched_kernel<<<dim3(nitems, (kmax + 31) / 32), dim3(32, 8), 0, stream>>>(rd, items, side, src_sel, planes);
-    return cudaGetLastError();
-}
-
-__global__ void shadows_batched_kernel(const RefreshDev *__restrict__ rd, const RowItem *__restrict__ items, int side)
-{
-    const RowItem it = items[blockIdx.x];
-    const RefreshDev d = rd[it.block];
-    const int r = d.r, rows = side ? d.n : d.m;
-    const int c0 = blockIdx.y * 32;
-    if (!d.fast || c0 >= r) return;
-    const float *__restrict__ X = side ? d.V : d.U;
-    bf16 *__restrict__ Xb = side ? d.Vb : d.Ub;
-    bf16 *__restrict__ Xbt = side ? d.Vbt : d.Ubt;
-    const int64_t ldb = d.rl, ldt = side ? d.nl : d.ml;
-    __shared__ float tile[64][33];
-    for (int h = 0; h < RG_ROWS; h += 64) {
-        const int r0 = it.row0 + h;
-        if (r0 >= rows) break;
-        for (int i = threadIdx.y; i < 64; i += blockDim.y) {
-            const int row = r0 + i, col = c0 + threadIdx.x;
-            float v = 0.f;
-            if (row < rows && col < r) {
-                v = X[(int64_t)row * r + col];
-                Xb[(int64_t)row * ldb + col] = __float2bfloat16_rn(v);
-            }
-            tile[i][threadIdx.x] = v;
-        }
-        __syncthreads();
-        for (int i = threadIdx.y; i < 32; i += blockDim.y) {
-            const int col = c0 + i, row = r0 + 2 * threadIdx.x;
-            if (col >= r || row >= rows) continue;
-            bf16 *dst = Xbt + (int64_t)col * ldt + row;
-            if (row + 1 < rows) *(uint32_t *)dst = pack_bf16x2(tile[2 * threadIdx.x][i], tile[2 * threadIdx.x + 1][i]);
-            else *dst = __float2bfloat16_rn(tile[2 * threadIdx.x][i]);
-        }
-        __syncthreads();
-    }
-}
-
-cudaError_t shadows_batched(const RefreshDev *rd, const RowItem *items, int nitems, int side, int rmax, cudaStream_t stream)
-{
-    if (nitems <= 0) return cudaSuccess;
-    shadows_batched_kernel<<<dim3(nitems, (rmax + 31) / 32), dim3(32, 8), 0, stream>>>(rd, items, side);
-    return cudaGetLastError();
-}
-
 cudaError_t fill_zero_f32(float *p, int64_t count, cudaStream_t stream)
 {
     return cudaMemsetAsync(p, 0, (size_t)count * sizeof(float), stream);
