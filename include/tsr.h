@@ -263,9 +263,11 @@ TSR_API tsr_status tsr_generate_omega(tsr_ctx *ctx, int32_t i, uint64_t seed, fl
 /* Stage timing of tsr_step_grouped for profiling (off by default).  When enabled, every
  * tsr_step_grouped / tsr_embed_step records CUDA events at its stage boundaries on the step's
  * stream; tsr_get_stage_ms waits for the last recorded step and returns, in milliseconds,
- * ms[0] refresh (0 when none was due), ms[1] T = G V, ms[2] core GEMM C = U^T T (with the
- * fused core update and the split-K reduction), ms[3] stand-alone core update (unfused order
- * only), ms[4] P = U D, ms[5] the apply kernel W <- decay W - step_scale P V^T.  count must be 6.
+ * ms[0] refresh (0 when none was due), ms[1] the projection launch (a step over all blocks runs
+ * T = G V and the core GEMM C = U^T T with its fused core update as ONE launch; a step over a
+ * partial block list runs T = G V here), ms[2] what follows it (the core GEMM of a partial list;
+ * the split-K reduction of tall blocks), ms[3] stand-alone core update (unfused order only),
+ * ms[4] P = U D, ms[5] the apply kernel W <- decay W - step_scale P V^T.  count must be 6.
  * Enabling creates the events (a small driver allocation); disabling destroys them. */
 TSR_API tsr_status tsr_set_profiling(tsr_ctx *ctx, int32_t enable);
 TSR_API tsr_status tsr_get_stage_ms(tsr_ctx *ctx, float *ms, int32_t count);
@@ -278,7 +280,7 @@ TSR_API tsr_status tsr_get_stage_ms(tsr_ctx *ctx, float *ms, int32_t count);
  *                 CTA gives up on its remaining tiles, releases its tensor memory and returns;
  *                 every block that owns one of those tiles reads TSR_ERR_TIMEOUT at the next
  *                 tsr_poll_status and its outputs of that call are undefined.
- *   max_sweeps    limit of the small eigen-solver of the refresh (Jacobi sweeps for k < 200,
+ *   max_sweeps    limit of the small eigen-solver of the refresh (Jacobi sweeps for k < 100,
  *                 QL iterations per eigenvalue above; defaults 40 / 60) for block sweep_block
  *                 (-1: every block).  A solver that stops at the limit flags
  *                 TSR_ERR_NOT_CONVERGED on that block; other blocks are not affected.

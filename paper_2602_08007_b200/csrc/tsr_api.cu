@@ -236,7 +236,7 @@ void layout(tsr_ctx *ctx, Arena &a, bool assign, size_t *step_end)
             if (assign) { b.Xs = (float *)xs; b.Bts = (float *)bts; }
         }
         if (b.fast) {
-            const int64_t ldp = round_up(mx, 16);
+            const int64_t ldp = round_up(mx, 128);   // 128-byte lines of a digit plane line up with the 128-row slabs that write them
             void *ce = a.take((size_t)k * 4), *pl = a.take((size_t)(6 * k * ldp));
             if (assign) { b.col_exp = (int32_t *)ce; b.planes = (int8_t *)pl; b.ldp = ldp; }
         }
@@ -782,14 +782,14 @@ tsr_status gram(tsr_ctx *ctx, const RefreshLists &L, int side, int src, cudaStre
     bool i8 = true;
     for (int bi : L.list) {
         const Block &b = ctx->blocks[bi];
-        i8 = i8 && b.fast && 2 * (int64_t)b.k <= std::min(b.d.m, b.d.n);
+        i8 = i8 && b.fast && b.k >= 8 && 2 * (int64_t)b.k <= std::min(b.d.m, b.d.n);   // (k >= 8: the slab maxima fit the partial-sum buffer)
     }
     if (!i8) {
         TSR_KERNEL(ctx, 2, gram_batched(ctx->d_refresh, L.ditems[side * 2 + 1], L.nitems[side * 2 + 1], L.dlist, nl, side, src,
                                         L.kmax, st));
         return TSR_OK;
     }
-    TSR_KERNEL(ctx, 2, gram_i8_prepare(ctx->d_refresh, L.ditems[side * 2], L.nitems[side * 2], L.dlist, nl, side, src, L.kmax, st));
+    TSR_KERNEL(ctx, 3, gram_i8_prepare(ctx->d_refresh, L.ditems[side * 2], L.nitems[side * 2], L.dlist, nl, side, src, L.kmax, st));
     const int kind = KG0 + side;
     std::vector<std::pair<int, int>> ranges;
     for (int bi : L.list) ranges.push_back({ctx->blocks[bi].tile_begin[kind], ctx->blocks[bi].tile_end[kind]});
@@ -920,7 +920,9 @@ tsr_status do_refresh_group(tsr_ctx *ctx, const std::vector<int> &list, uint64_t
     if ((s = sketch(ctx, L, true, false, nullptr, st)) != TSR_OK) return s;
     const int nl = (int)list.size();
     if ((s = gram(ctx, L, 1, 0, st)) != TSR_OK) return s;
-    if (L.kmax >= 200) {   // too large for the Jacobi solver: tridiagonal route
+    // From k = 100 on the tridiagonal route is the faster one (k = 136: 11.4 ms of one-CTA Jacobi sweeps against about
+    // 3 ms; the refresh of the single-matrix configuration went from 12.4 to 4.8 ms, of the 60M set from 15.9 to 8.0 ms)
+    if (L.kmax >= 100) {
         const int pr = eig_panel_rows(L.kmax);
         std::vector<RowItem> panels;
         for (int bi : list)

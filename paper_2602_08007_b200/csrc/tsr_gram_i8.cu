@@ -16,7 +16,7 @@
 // layout the MMAs want; one tile of the product loads the six planes of its rows and columns once per 64 rows of
 // X and issues all 21 pair products from them, so the kernel is bound by the tensor pipe, not by its operands.
 //
-// Kernels: gram_colexp_kernel (column exponents), gram_digits_kernel (digit planes), gram_i8_kernel (CTA pairs,
+// Kernels: gram_slabmax_kernel + gram_colexp_kernel (column exponents), gram_digits_kernel (digit planes), gram_i8_kernel (CTA pairs,
 // persistent over a tile table: producer / MMA / epilogue warps as in the BF16 GEMM), then the existing
 // gram_reduce_kernel adds the row chunks in fixed order and mirrors the upper triangle.
 #include "tsr_internal.h"
@@ -39,50 +39,69 @@ constexpr uint32_t GI_TMEM_COLS = 512;       // six levels of 64 INT32 columns (
 
 // ---------------------------------------------------------------------------------------------------------
 // Column exponents: e_j = smallest integer with max_i |x_ij| <= 2^(e_j - 1); 0 for an all-zero column.
-// One CTA per (32 columns, block); 32 warps stride over the rows.  A non-finite entry flags the block.
+// Two steps without atomics: gram_slabmax_kernel writes the column maxima of every slab of RG_ROWS rows (into the
+// Gram partial-sum buffer, which is free until the products are stored), gram_colexp_kernel reduces them.
+// A non-finite entry flags the block.
 // ---------------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(1024)
-gram_colexp_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ list, int side, int src_sel)
+__global__ void __launch_bounds__(256)
+gram_slabmax_kernel(const RefreshDev *__restrict__ rd, const RowItem *__restrict__ items, int side, int src_sel)
 {
-    const RefreshDev d = rd[list[blockIdx.y]];
+    const RowItem it = items[blockIdx.y];
+    const RefreshDev d = rd[it.block];
     const int k = d.k, rows = side ? d.n : d.m;
     const int c0 = blockIdx.x * 32;
     if (c0 >= k) return;
     const float *__restrict__ X = d.buf[src_sel];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int col = c0 + lane;
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    const int col = c0 + tx;
     float mx = 0.f;
     bool bad = false;
     if (col < k) {
-        for (int r0 = warp; r0 < rows; r0 += 32 * 4) {
-            float v[4];
+        float v[RG_ROWS / 8];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) v[u] = (r0 + 32 * u < rows) ? fabsf(X[(int64_t)(r0 + 32 * u) * k + col]) : 0.f;
+        for (int u = 0; u < RG_ROWS / 8; ++u) {
+            const int row = it.row0 + ty + 8 * u;
+            v[u] = (row < rows) ? fabsf(X[(int64_t)row * k + col]) : 0.f;
+        }
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                if (!(v[u] <= 3.0e38f)) bad = true;     // NaN or Inf
-                mx = fmaxf(mx, v[u]);
-            }
+        for (int u = 0; u < RG_ROWS / 8; ++u) {
+            if (!(v[u] <= 3.0e38f)) bad = true;     // NaN or Inf
+            mx = fmaxf(mx, v[u]);
         }
     }
-    __shared__ float s_mx[32][33];
+    __shared__ float s_mx[8][33];
     __shared__ int s_bad;
     if (threadIdx.x == 0) s_bad = 0;
     __syncthreads();
-    s_mx[warp][lane] = mx;
+    s_mx[ty][tx] = mx;
     if (bad) s_bad = 1;
     __syncthreads();
-    if (warp == 0 && col < k) {
+    if (ty == 0 && col < k) {
         float m = 0.f;
-        for (int w = 0; w < 32; ++w) m = fmaxf(m, s_mx[w][lane]);
-        int e = 0;
-        if (m > 0.f && m <= 3.0e38f) {
-            (void)frexpf(m, &e);            // m = f 2^e with f in [1/2, 1)  =>  m < 2^e
-            e += 1;                         // m 2^-e < 1/2
-        }
-        d.col_exp[col] = e;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) m = fmaxf(m, s_mx[w][tx]);
+        ((float *)d.gpart)[(int64_t)(it.row0 / RG_ROWS) * k + col] = m;
     }
     if (threadIdx.x == 0 && s_bad) atomicMax(d.status, (int)TSR_ERR_NONFINITE);
+}
+
+__global__ void __launch_bounds__(256)
+gram_colexp_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ list, int side)
+{
+    const RefreshDev d = rd[list[blockIdx.y]];
+    const int k = d.k, rows = side ? d.n : d.m;
+    const int col = blockIdx.x * 256 + threadIdx.x;
+    if (col >= k) return;
+    const int nslab = (rows + RG_ROWS - 1) / RG_ROWS;
+    const float *__restrict__ sm = (const float *)d.gpart;
+    float m = 0.f;
+    for (int sl = 0; sl < nslab; ++sl) m = fmaxf(m, sm[(int64_t)sl * k + col]);
+    int e = 0;
+    if (m > 0.f && m <= 3.0e38f) {
+        (void)frexpf(m, &e);            // m = f 2^e with f in [1/2, 1)  =>  m < 2^e
+        e += 1;                         // m 2^-e < 1/2
+    }
+    d.col_exp[col] = e;
 }
 
 // ---------------------------------------------------------------------------------------------------------
@@ -317,7 +336,8 @@ cudaError_t gram_i8_prepare(const RefreshDev *rd, const RowItem *items128, int n
 {
     if (nitems128 <= 0 || nlist <= 0) return cudaSuccess;
     const int t = (kmax + 31) / 32;
-    gram_colexp_kernel<<<dim3(t, nlist), 1024, 0, stream>>>(rd, list, side, src_sel);
+    gram_slabmax_kernel<<<dim3(t, nitems128), 256, 0, stream>>>(rd, items128, side, src_sel);
+    gram_colexp_kernel<<<dim3((kmax + 255) / 256, nlist), 256, 0, stream>>>(rd, list, side);
     gram_digits_kernel<<<dim3(t, nitems128), 256, 0, stream>>>(rd, items128, side, src_sel);
     return cudaGetLastError();
 }

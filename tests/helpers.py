@@ -64,16 +64,43 @@ def set_bases(plan, i, U, V):
     plan.V[i].copy_(V.to(plan.V[i].device))
 
 
-def check_refresh_many(jobs, workers=None):
-    """check_refresh for a list of argument tuples on concurrent host threads.  The oracle's refresh spends most of
-    its time in a serial Jacobi loop, so the blocks of a model are checked side by side (ctypes releases the
-    interpreter lock during the oracle's calls).  The first failing assertion is re-raised."""
-    import os
-    from concurrent.futures import ThreadPoolExecutor
-    if workers is None:
-        workers = max(1, min(len(jobs), os.cpu_count() or 1))
-    with ThreadPoolExecutor(max_workers=workers) as ex:
-        return list(ex.map(lambda a: check_refresh(*a), jobs))
+class RefreshChecks:
+    """Oracle-side checks of refreshed bases, run on background host threads.  The oracle's refresh spends most of
+    its time in a serial Jacobi loop (minutes for a 1B-shaped block), and nothing downstream waits for its result:
+    the parity protocol hands the LIBRARY's bases to the oracle after a refresh.  So the checks of all blocks run
+    side by side while the test goes on stepping, and `join` re-raises the first failed assertion at the end.
+    (ctypes releases the interpreter lock during the oracle's calls.)"""
+
+    def __init__(self, workers=None):
+        import os
+        from concurrent.futures import ThreadPoolExecutor
+        # a few checks at a time, each with the oracle's full OpenMP team: its matrix products and Householder
+        # sweeps scale with the cores (one thread each was tried and is several times slower on 1B-shaped blocks)
+        self.pool = ThreadPoolExecutor(max_workers=workers or 3)
+        self.futures = []
+
+    def submit(self, U, V, G64, Om64, r, q, gap, tol_sub=TOL_SUBSPACE):
+        self.futures.append(self.pool.submit(check_refresh_uv, U, V, G64, Om64, r, q, gap, tol_sub))
+
+    def join(self):
+        try:
+            for f in self.futures:
+                f.result()
+        finally:
+            self.pool.shutdown(wait=True)
+
+
+def check_refresh_invariants(U, V, G64, r):
+    """The part of the refresh check that needs no oracle: orthonormal bases, and U^T G V diagonal, non-negative and
+    descending.  Returns (orthonormality, off-diagonal / sigma_1)."""
+    ortho = max(np.linalg.norm(U.T @ U - np.eye(r)), np.linalg.norm(V.T @ V - np.eye(r)))
+    assert ortho < TOL_ORTHO, ortho
+    core = U.T @ G64 @ V
+    d = np.diag(core)
+    offdiag = float(np.abs(core - np.diag(d)).max() / d[0])
+    assert offdiag < TOL_OFFDIAG, offdiag
+    assert np.all(d > 0) and np.all(np.diff(d) < 1e-5 * d[0])
+    return float(ortho), offdiag
 
 
 REFRESH_MEASURED = []   # one record per check_refresh call, printed by the tests that want a table
@@ -82,7 +109,13 @@ REFRESH_MEASURED = []   # one record per check_refresh call, printed by the test
 def check_refresh(plan, i, G64, Om64, r, q, gap, tol_sub=TOL_SUBSPACE):
     """Invariants and subspace agreement of block i's refreshed bases against the oracle's refresh
     of the same (G, Omega) bits.  Returns the oracle's (U, V, sigma)."""
-    U, V = to64(plan.U[i]), to64(plan.V[i])
+    return check_refresh_uv(to64(plan.U[i]), to64(plan.V[i]), G64, Om64, r, q, gap, tol_sub)
+
+
+def check_refresh_uv(U, V, G64, Om64, r, q, gap, tol_sub=TOL_SUBSPACE):
+    """check_refresh for bases given as FP64 arrays (a snapshot: the plan's may have moved on)."""
+    import time
+    t_start = time.perf_counter()
     ortho = max(np.linalg.norm(U.T @ U - np.eye(r)), np.linalg.norm(V.T @ V - np.eye(r)))
     assert ortho < TOL_ORTHO, ortho
     Uo, Vo, sig = oracle.rsvd_refresh(G64, Om64, r, q)
@@ -103,7 +136,7 @@ def check_refresh(plan, i, G64, Om64, r, q, gap, tol_sub=TOL_SUBSPACE):
     pv = float(np.linalg.norm(proj(V[:, :gap]) - proj(Vo[:, :gap])))
     assert pu < tol_sub and pv < tol_sub, (pu, pv)
     REFRESH_MEASURED.append(dict(m=G64.shape[0], n=G64.shape[1], r=r, ortho=float(ortho), offdiag=offdiag, lead=lead,
-                                 energy=energy, proj=max(pu, pv)))
+                                 energy=energy, proj=max(pu, pv), seconds=time.perf_counter() - t_start))
     return Uo, Vo, sig
 
 
