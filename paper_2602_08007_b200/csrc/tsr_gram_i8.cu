@@ -14,7 +14,13 @@
 //   4. S_ij = 2^(e_i + e_j) sum_level 2^(-7(level + 2)) A_level(i, j), formed in FP64 in the epilogue.
 // The digit planes are stored transposed (k x rows, the row index of X contiguous), which is the K-major operand
 // layout the MMAs want; one tile of the product loads the six planes of its rows and columns once per 64 rows of
-// X and issues all 21 pair products from them, so the kernel is bound by the tensor pipe, not by its operands.
+// X and forms all 21 pair products from them.  An MMA reads its whole A operand from shared memory again, so 21
+// narrow MMAs (N = 64) would keep the tensor pipe waiting for shared memory more than half of the time.  The
+// products of one A plane s with the B planes t = 0 .. 5 - s go to consecutive levels s + t, i.e. to consecutive
+// accumulators: stacked along N they are ONE wide MMA.  In a CTA pair the first half of an MMA's N rows comes from
+// the leader's shared memory and the second half from its peer's, at the same offsets, so the leader keeps the B
+// planes {0, 1, 4} and the peer {2, 3, 5} (each for all 64 columns of the tile): eight MMAs per 32 rows of X do
+// the work of 21 (see the table at the MMA loop); the columns past the sixth level take products nobody reads.
 //
 // Kernels: gram_slabmax_kernel + gram_colexp_kernel (column exponents), gram_digits_kernel (digit planes), gram_i8_kernel (CTA pairs,
 // persistent over a tile table: producer / MMA / epilogue warps as in the BF16 GEMM), then the existing
@@ -29,13 +35,14 @@ constexpr int GI_BN = 64;                    // tile: 256 (pair) x 64 outputs
 constexpr int GI_BK = 64;                    // rows of X per stage (64-byte operand rows, 64-byte swizzle)
 constexpr int GI_STAGES = 3;
 constexpr int GI_A_BYTES = UM_BM * GI_BK;            // one digit plane of this CTA's 128 rows: 8 KB
-constexpr int GI_B_BYTES = (GI_BN / 2) * GI_BK;      // one digit plane of this CTA's half of the 64 columns: 2 KB
-constexpr int GI_STAGE_BYTES = GI_DIGITS * (GI_A_BYTES + GI_B_BYTES);   // 60 KB
+constexpr int GI_B_BYTES = GI_BN * GI_BK;            // one digit plane of the tile's 64 columns: 4 KB
+constexpr int GI_B_SLOTS = 3;                        // B planes a CTA keeps: {0, 1, 4} (leader) or {2, 3, 5} (peer)
+constexpr int GI_STAGE_BYTES = GI_DIGITS * GI_A_BYTES + GI_B_SLOTS * GI_B_BYTES;   // 60 KB
 constexpr int GI_BAR_OFFSET = GI_STAGES * GI_STAGE_BYTES;
 constexpr int GI_NBARS = 2 * GI_STAGES + 2;
 constexpr int GI_SMEM = GI_BAR_OFFSET + GI_NBARS * 8 + 64 + 1024;
 constexpr int GI_THREADS = 384;
-constexpr uint32_t GI_TMEM_COLS = 512;       // six levels of 64 INT32 columns (384), rounded up to a power of two
+constexpr uint32_t GI_TMEM_COLS = 512;       // six levels of 64 INT32 columns (384) + 128 columns of products past the sixth level
 
 // ---------------------------------------------------------------------------------------------------------
 // Column exponents: e_j = smallest integer with max_i |x_ij| <= 2^(e_j - 1); 0 for an all-zero column.
@@ -47,7 +54,7 @@ __global__ void __launch_bounds__(256)
 gram_slabmax_kernel(const RefreshDev *__restrict__ rd, const RowItem *__restrict__ items, int side, int src_sel)
 {
     const RowItem it = items[blockIdx.y];
-    const RefreshDev d = rd[it.block];
+    const RefreshDev &d = rd[it.block];
     const int k = d.k, rows = side ? d.n : d.m;
     const int c0 = blockIdx.x * 32;
     if (c0 >= k) return;
@@ -88,20 +95,29 @@ gram_slabmax_kernel(const RefreshDev *__restrict__ rd, const RowItem *__restrict
 __global__ void __launch_bounds__(256)
 gram_colexp_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ list, int side)
 {
-    const RefreshDev d = rd[list[blockIdx.y]];
+    const RefreshDev &d = rd[list[blockIdx.y]];
     const int k = d.k, rows = side ? d.n : d.m;
-    const int col = blockIdx.x * 256 + threadIdx.x;
-    if (col >= k) return;
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    const int col = blockIdx.x * 32 + tx;
+    if (blockIdx.x * 32 >= k) return;
     const int nslab = (rows + RG_ROWS - 1) / RG_ROWS;
     const float *__restrict__ sm = (const float *)d.gpart;
     float m = 0.f;
-    for (int sl = 0; sl < nslab; ++sl) m = fmaxf(m, sm[(int64_t)sl * k + col]);
-    int e = 0;
-    if (m > 0.f && m <= 3.0e38f) {
-        (void)frexpf(m, &e);            // m = f 2^e with f in [1/2, 1)  =>  m < 2^e
-        e += 1;                         // m 2^-e < 1/2
+    if (col < k)
+        for (int sl = ty; sl < nslab; sl += 8) m = fmaxf(m, sm[(int64_t)sl * k + col]);
+    __shared__ float s_mx[8][33];
+    s_mx[ty][tx] = m;
+    __syncthreads();
+    if (ty == 0 && col < k) {
+#pragma unroll
+        for (int w = 1; w < 8; ++w) m = fmaxf(m, s_mx[w][tx]);
+        int e = 0;
+        if (m > 0.f && m <= 3.0e38f) {
+            (void)frexpf(m, &e);            // m = f 2^e with f in [1/2, 1)  =>  m < 2^e
+            e += 1;                         // m 2^-e < 1/2
+        }
+        d.col_exp[col] = e;
     }
-    d.col_exp[col] = e;
 }
 
 // ---------------------------------------------------------------------------------------------------------
@@ -113,7 +129,7 @@ __global__ void __launch_bounds__(256)
 gram_digits_kernel(const RefreshDev *__restrict__ rd, const RowItem *__restrict__ items, int side, int src_sel)
 {
     const RowItem it = items[blockIdx.y];
-    const RefreshDev d = rd[it.block];
+    const RefreshDev &d = rd[it.block];
     const int k = d.k, rows = side ? d.n : d.m;
     const int c0 = blockIdx.x * 32;
     if (c0 >= k) return;
@@ -142,8 +158,12 @@ gram_digits_kernel(const RefreshDev *__restrict__ rd, const RowItem *__restrict_
         if (!(fabsf(r) <= 64.f)) r = 0.f;                      // a non-finite entry (the block is flagged already)
 #pragma unroll
         for (int s = 0; s < GI_DIGITS; ++s) {
-            const float dgt = rintf(r);                        // in [-64, 64]
-            w[s][i >> 2] |= ((uint32_t)(int)dgt & 0xffu) << (8 * (i & 3));
+            // round to nearest even by adding 1.5 * 2^23: the sum's low mantissa bits are the integer in two's
+            // complement (|r| <= 64), and taking the constant off again gives it back as a float -- the same value
+            // as rintf(r), without the conversion unit
+            const float t = __fadd_rn(r, 12582912.f);
+            const float dgt = __fadd_rn(t, -12582912.f);       // in [-64, 64]
+            w[s][i >> 2] |= (__float_as_uint(t) & 0xffu) << (8 * (i & 3));
             r = (r - dgt) * 128.f;                             // exact: the remainder, |.| <= 1/2, scaled by 2^7
         }
     }
@@ -168,8 +188,8 @@ __device__ __forceinline__ uint64_t umma_desc_sw64(uint32_t saddr)
     d |= (uint64_t)4 << 61;
     return d;
 }
-// Instruction descriptor: signed 8-bit operands, both K-major, INT32 accumulator, M = 256 (CTA pair), N = 64.
-constexpr uint32_t GI_IDESC = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(GI_BN >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+// Instruction descriptor: signed 8-bit operands, both K-major, INT32 accumulator, M = 256 (CTA pair), N columns.
+__host__ __device__ constexpr uint32_t gi_idesc(int n) { return (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(256 >> 4) << 24); }
 
 __device__ __forceinline__ void tc_mma_i8_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
 {
@@ -182,7 +202,7 @@ __device__ __forceinline__ void tc_mma_i8_pair(uint32_t d_tmem, uint64_t adesc, 
 }
 
 // probs[b].tmA / tmB: the digit planes of block b as a (6 k) x rows INT8 matrix (plane s starts at row s k), boxes of
-// 64 bytes x 128 rows and 64 bytes x 32 rows.  A tile: rows m0 .. m0 + 255 and columns n0 .. n0 + 63 of S, the
+// 64 bytes x 128 rows and 64 bytes x 32 rows (two of them per B plane).  A tile: rows m0 .. m0 + 255 and columns n0 .. n0 + 63 of S, the
 // rows [64 kb0, 64 kb1) of X; it writes its part of the chunk's partial sum (FP64, row pitch k).
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GI_THREADS, 1)
 gram_i8_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restrict__ tiles, int num_tiles, long long budget_in,
@@ -235,11 +255,15 @@ gram_i8_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restrict
                     if (rank == 0) mbar_expect_tx(smem_u32(bar_full + s), 2u * (uint32_t)GI_STAGE_BYTES);
                     uint8_t *st = smem + s * GI_STAGE_BYTES;
 #pragma unroll
-                    for (int dg = 0; dg < GI_DIGITS; ++dg) {
+                    for (int dg = 0; dg < GI_DIGITS; ++dg)
                         tma_load_2d_pair(smem_u32(st + dg * GI_A_BYTES), &P->tmA, full, kb * GI_BK,
                                          dg * k + tile.m0 + (int)rank * UM_BM);
-                        tma_load_2d_pair(smem_u32(st + GI_DIGITS * GI_A_BYTES + dg * GI_B_BYTES), &P->tmB, full, kb * GI_BK,
-                                         dg * k + tile.n0 + (int)rank * (GI_BN / 2));
+#pragma unroll
+                    for (int sl = 0; sl < GI_B_SLOTS; ++sl) {
+                        const int dg = sl == 2 ? 4 + (int)rank : 2 * (int)rank + sl;     // leader {0, 1, 4}, peer {2, 3, 5}
+                        uint8_t *dst = st + GI_DIGITS * GI_A_BYTES + sl * GI_B_BYTES;
+                        tma_load_2d_pair(smem_u32(dst), &P->tmB, full, kb * GI_BK, dg * k + tile.n0);
+                        tma_load_2d_pair(smem_u32(dst + GI_B_BYTES / 2), &P->tmB, full, kb * GI_BK, dg * k + tile.n0 + GI_BN / 2);
                     }
                 }
             }
@@ -260,20 +284,28 @@ gram_i8_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restrict
                     const uint32_t a_base = smem_u32(smem + s * GI_STAGE_BYTES);
                     const uint32_t b_base = a_base + GI_DIGITS * GI_A_BYTES;
                     const bool first_kb = (kb == tile.kb0);
-                    // all pairs of digit planes (da, db) with da + db <= 5, into the accumulator of their level
+                    // A plane s against the stacked B planes, accumulator columns from 64 s on (level s + t at 64 (s + t)):
+                    //   N = 256 over slots 0, 1: leader's planes 0, 1 -> levels s, s + 1; peer's planes 2, 3 -> levels s + 2, s + 3
+                    //   N = 128 over slot 2:     leader's plane 4 -> level s + 4; peer's plane 5 -> level s + 5
+                    //   N = 128 over slot 0:     leader's plane 0 -> level s;     peer's plane 2 -> level s + 1 (used for s = 5 only)
+                    // Levels past 5 fall into columns 384 .. 511, which are never read.  The two MMAs of s = 0 cover all six
+                    // levels and start them afresh on the tile's first rows.
 #pragma unroll
-                    for (int da = 0; da < GI_DIGITS; ++da)
+                    for (int k2 = 0; k2 < GI_BK / 32; ++k2) {
+                        const uint32_t fresh = (first_kb && k2 == 0) ? 0u : 1u;
 #pragma unroll
-                        for (int db = 0; db < GI_DIGITS; ++db) {
-                            if (da + db >= GI_DIGITS) continue;
-                            const uint32_t d_tmem = tmem_base + (uint32_t)((da + db) * GI_BN);
-                            // the first pair of a level (da == 0) starts that level's accumulator afresh on the tile's first rows
-#pragma unroll
-                            for (int k2 = 0; k2 < GI_BK / 32; ++k2)
-                                tc_mma_i8_pair(d_tmem, umma_desc_sw64(a_base + da * GI_A_BYTES + k2 * 32),
-                                               umma_desc_sw64(b_base + db * GI_B_BYTES + k2 * 32), GI_IDESC,
-                                               (first_kb && da == 0 && k2 == 0) ? 0u : 1u);
+                        for (int da = 0; da < GI_DIGITS; ++da) {
+                            const uint64_t adesc = umma_desc_sw64(a_base + da * GI_A_BYTES + k2 * 32);
+                            const uint32_t d_tmem = tmem_base + (uint32_t)(da * GI_BN);
+                            if (da < 5)
+                                tc_mma_i8_pair(d_tmem, adesc, umma_desc_sw64(b_base + k2 * 32), gi_idesc(256), da == 0 ? fresh : 1u);
+                            else
+                                tc_mma_i8_pair(d_tmem, adesc, umma_desc_sw64(b_base + k2 * 32), gi_idesc(128), 1u);
+                            if (da < 2)
+                                tc_mma_i8_pair(d_tmem + 4 * GI_BN, adesc, umma_desc_sw64(b_base + 2 * GI_B_BYTES + k2 * 32), gi_idesc(128),
+                                               da == 0 ? fresh : 1u);
                         }
+                    }
                     tc_commit_pair(smem_u32(bar_empty + s));
                 }
                 tc_commit_pair(smem_u32(bar_acc_full));
@@ -337,7 +369,7 @@ cudaError_t gram_i8_prepare(const RefreshDev *rd, const RowItem *items128, int n
     if (nitems128 <= 0 || nlist <= 0) return cudaSuccess;
     const int t = (kmax + 31) / 32;
     gram_slabmax_kernel<<<dim3(t, nitems128), 256, 0, stream>>>(rd, items128, side, src_sel);
-    gram_colexp_kernel<<<dim3((kmax + 255) / 256, nlist), 256, 0, stream>>>(rd, list, side);
+    gram_colexp_kernel<<<dim3(t, nlist), 256, 0, stream>>>(rd, list, side);
     gram_digits_kernel<<<dim3(t, nitems128), 256, 0, stream>>>(rd, items128, side, src_sel);
     return cudaGetLastError();
 }

@@ -33,7 +33,7 @@ __global__ void __launch_bounds__(256)
 gram_partial_kernel(const RefreshDev *__restrict__ rd, const RowItem *__restrict__ items, int side, int src_sel)
 {
     const RowItem it = items[blockIdx.z];
-    const RefreshDev d = rd[it.block];
+    const RefreshDev &d = rd[it.block];
     const int k = d.k;
     const int ti = blockIdx.y, tj = blockIdx.x;
     if (tj < ti || ti * GR_T >= k || tj * GR_T >= k) return;
@@ -114,19 +114,41 @@ gram_partial_kernel(const RefreshDev *__restrict__ rd, const RowItem *__restrict
         }
 }
 
-__global__ void gram_reduce_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ list, int side)
+// S = sum of the chunks' partial sums, in fixed order, for one 32 x 32 tile per CTA.  Only 8 x 8 sub-tiles on or
+// above the diagonal were written: a tile below the diagonal is the transpose of its mirror image, a tile on the
+// diagonal takes its lower sub-tiles from its own transpose (both through shared memory).
+__global__ void __launch_bounds__(256)
+gram_reduce_kernel(const RefreshDev *__restrict__ rd, const int32_t *__restrict__ list, int side)
 {
-    const RefreshDev d = rd[list[blockIdx.y]];
+    const RefreshDev &d = rd[list[blockIdx.z]];
     const int k = d.k;
+    const int ti = blockIdx.y, tj = blockIdx.x;
+    if (ti * 32 >= k || tj * 32 >= k) return;
     const int chunks = gram_chunks(side ? d.n : d.m);
     const int64_t total = (int64_t)k * k;
-    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
-        const int i = (int)(e / k), j = (int)(e % k);
-        const bool upper = (j / GR_S) >= (i / GR_S);  // only sub-tiles on or above the diagonal were written
-        const int64_t src = upper ? e : (int64_t)j * k + i;
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    const int si = ti <= tj ? ti : tj, sj = ti <= tj ? tj : ti;     // the tile that was written
+    __shared__ double t[32][33];
+    const double *__restrict__ gp = d.gpart;
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+        const int i = si * 32 + ty + 8 * u, j = sj * 32 + tx;
         double s = 0.0;
-        for (int c = 0; c < chunks; ++c) s += d.gpart[(int64_t)c * total + src];
-        d.S[e] = s;
+        if (i < k && j < k && (j / GR_S) >= (i / GR_S))
+            for (int c = 0; c < chunks; ++c) s += gp[(int64_t)c * total + (int64_t)i * k + j];
+        t[ty + 8 * u][tx] = s;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+        const int li = ty + 8 * u, lj = tx;
+        const int i = ti * 32 + li, j = tj * 32 + lj;
+        if (i >= k || j >= k) continue;
+        double v;
+        if (ti < tj) v = t[li][lj];
+        else if (ti > tj) v = t[lj][li];
+        else v = (lj / GR_S) >= (li / GR_S) ? t[li][lj] : t[lj][li];
+        d.S[(int64_t)i * k + j] = v;
     }
 }
 
@@ -142,9 +164,8 @@ cudaError_t gram_batched(const RefreshDev *rd, const RowItem *items, int nitems,
 cudaError_t gram_reduce_batched(const RefreshDev *rd, const int32_t *list, int nlist, int side, int kmax, cudaStream_t stream)
 {
     if (nlist <= 0) return cudaSuccess;
-    int gx = (int)(((int64_t)kmax * kmax + 255) / 256);
-    if (gx > 128) gx = 128;
-    gram_reduce_kernel<<<dim3(gx, nlist), 256, 0, stream>>>(rd, list, side);
+    const int t = (kmax + 31) / 32;
+    gram_reduce_kernel<<<dim3(t, t, nlist), 256, 0, stream>>>(rd, list, side);
     return cudaGetLastError();
 }
 
@@ -459,7 +480,7 @@ rows_gemm_kernel(const RefreshDev *__restrict__ rd, const RowItem *__restrict__ 
                  int mat_sel, int dst_sel)
 {
     const RowItem it = items[blockIdx.y];
-    const RefreshDev d = rd[it.block];
+    const RefreshDev &d = rd[it.block];
     const int K = d.k;
     const int N = (mat_sel == 0) ? d.k : d.r;
     const int n0 = blockIdx.x * 64;
@@ -546,7 +567,7 @@ rows_gemm128_kernel(const RefreshDev *__restrict__ rd, const RowItem *__restrict
                     int mat_sel, int dst_sel)
 {
     const RowItem it = items[blockIdx.y];
-    const RefreshDev d = rd[it.block];
+    const RefreshDev &d = rd[it.block];
     const int K = d.k;
     const int N = (mat_sel == 0) ? d.k : d.r;
     const int n0 = blockIdx.x * 128;
@@ -673,7 +694,7 @@ __global__ void __launch_bounds__(256)
 split_rows_kernel(const RefreshDev *__restrict__ rd, const RowItem *__restrict__ items, int side, int src_sel)
 {
     const RowItem it = items[blockIdx.x];
-    const RefreshDev d = rd[it.block];
+    const RefreshDev &d = rd[it.block];
     const int k = d.k;
     const int rows = side ? d.n : d.m;
     const int64_t mx = max(d.m, d.n);

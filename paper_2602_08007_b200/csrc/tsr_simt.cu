@@ -3,11 +3,17 @@
 // operand conversion for the tensor-core path, and the Gaussian generator for Omega.
 #include "tsr_internal.h"
 #include "tsr_device.cuh"
+#include <cooperative_groups.h>
 
 namespace tsr {
 
 // ---------------------------------------------------------------------------------------
 // Generic strided FP32 GEMM, 64 x 64 output tile, 16-deep K slices, 4 x 4 outputs per thread.
+// Products with few output tiles and a long contraction (T = G V of a single matrix: 16 tiles,
+// K = 1376) are split along K over the CTAs of a thread-block cluster (gridDim.z = cluster size
+// <= 8): every CTA sums its slab of K, parks its 64 x 64 partial tile in its own shared memory,
+// and the cluster's first CTA adds the others' tiles through distributed shared memory in rank
+// order -- a fixed order, so the result does not depend on timing -- and runs the epilogue.
 // ---------------------------------------------------------------------------------------
 template <typename TA>
 __device__ __forceinline__ float load_as_float(const TA *p);
@@ -26,9 +32,15 @@ simt_gemm_kernel(int M, int N, int K, const TA *__restrict__ A, int64_t sa_i, in
 {
     __shared__ float As[SG_BK][SG_BM + 4];
     __shared__ float Bs[SG_BK][SG_BN + 4];
+    __shared__ float red[SG_BM * SG_BN];     // this CTA's partial tile, [a][b][thread]: read and written without bank conflicts
     const int tid = threadIdx.x;
     const int tx = tid % 16, ty = tid / 16;
     const int m0 = blockIdx.y * SG_BM, n0 = blockIdx.x * SG_BN;
+    // this CTA's slab of the contraction: whole K slices, the same count for every rank
+    const int nslab = (int)gridDim.z, slab = (int)blockIdx.z;
+    const int slices = (K + SG_BK - 1) / SG_BK;
+    const int per = (slices + nslab - 1) / nslab;
+    const int k_begin = min(K, slab * per * SG_BK), k_end = min(K, (slab + 1) * per * SG_BK);
 
     float acc[4][4];
 #pragma unroll
@@ -49,15 +61,15 @@ simt_gemm_kernel(int M, int N, int K, const TA *__restrict__ A, int64_t sa_i, in
             int ai, ak;
             if (a_k_fast) { ak = e % SG_BK; ai = e / SG_BK; } else { ai = e % SG_BM; ak = e / SG_BM; }
             const int gi = m0 + ai, gk = k0 + ak;
-            ra[l] = (gi < M && gk < K) ? load_as_float<TA>(A + (int64_t)gi * sa_i + (int64_t)gk * sa_k) : 0.f;
+            ra[l] = (gi < M && gk < k_end) ? load_as_float<TA>(A + (int64_t)gi * sa_i + (int64_t)gk * sa_k) : 0.f;
             int bj, bk;
             if (b_j_fast) { bj = e % SG_BN; bk = e / SG_BN; } else { bk = e % SG_BK; bj = e / SG_BK; }
             const int gj = n0 + bj, gk2 = k0 + bk;
-            rb[l] = (gj < N && gk2 < K) ? load_as_float<TB>(B + (int64_t)gk2 * sb_k + (int64_t)gj * sb_j) : 0.f;
+            rb[l] = (gj < N && gk2 < k_end) ? load_as_float<TB>(B + (int64_t)gk2 * sb_k + (int64_t)gj * sb_j) : 0.f;
         }
     };
-    fetch(0);
-    for (int k0 = 0; k0 < K; k0 += SG_BK) {
+    if (k_begin < k_end) fetch(k_begin);
+    for (int k0 = k_begin; k0 < k_end; k0 += SG_BK) {
 #pragma unroll
         for (int l = 0; l < 4; ++l) {
             const int e = tid + l * 256;
@@ -69,7 +81,7 @@ simt_gemm_kernel(int M, int N, int K, const TA *__restrict__ A, int64_t sa_i, in
             Bs[bk][bj] = rb[l];
         }
         __syncthreads();
-        if (k0 + SG_BK < K) fetch(k0 + SG_BK);
+        if (k0 + SG_BK < k_end) fetch(k0 + SG_BK);
 #pragma unroll
         for (int kk = 0; kk < SG_BK; ++kk) {
             float av[4], bv[4];
@@ -83,6 +95,28 @@ simt_gemm_kernel(int M, int N, int K, const TA *__restrict__ A, int64_t sa_i, in
                 for (int b = 0; b < 4; ++b) acc[a][b] = fmaf(av[a], bv[b], acc[a][b]);
         }
         __syncthreads();
+    }
+    if (nslab > 1) {
+        namespace cg = cooperative_groups;
+        cg::cluster_group cluster = cg::this_cluster();
+        if (slab != 0) {
+#pragma unroll
+            for (int a = 0; a < 4; ++a)
+#pragma unroll
+                for (int b = 0; b < 4; ++b) red[(a * 4 + b) * 256 + tid] = acc[a][b];
+        }
+        cluster.sync();                                   // every partial tile is in place
+        if (slab == 0) {
+            for (int sl = 1; sl < nslab; ++sl) {          // rank order: the sum does not depend on timing
+                const float *peer = cluster.map_shared_rank(red, sl);
+#pragma unroll
+                for (int a = 0; a < 4; ++a)
+#pragma unroll
+                    for (int b = 0; b < 4; ++b) acc[a][b] += peer[(a * 4 + b) * 256 + tid];
+            }
+        }
+        cluster.sync();                                   // nobody leaves while its tile may still be read
+        if (slab != 0) return;
     }
 #pragma unroll
     for (int a = 0; a < 4; ++a) {
@@ -108,18 +142,43 @@ simt_gemm_kernel(int M, int N, int K, const TA *__restrict__ A, int64_t sa_i, in
 }
 
 // FP32 A (any strides) times a BF16 or FP32 B, plain store: the one-sided projection C = U^T G.
+// K slabs for a product with `tiles` output tiles: doubled while the grid stays within about one wave of CTAs
+// (148 SMs, several CTAs each) and every slab keeps at least four K slices; a power of two up to the portable
+// cluster size of 8.
+static int simt_slabs(int tiles, int K)
+{
+    int s = 1;
+    while (s < 8 && tiles * s * 2 <= 296 && K / (s * 2) >= 4 * SG_BK) s *= 2;
+    return s;
+}
+
+template <typename Kern, typename... Args>
+static cudaError_t simt_launch(Kern kern, dim3 grid, int slabs, cudaStream_t stream, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid.x, grid.y, (unsigned)slabs);
+    cfg.blockDim = dim3(256);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = (unsigned)slabs;
+    cfg.attrs = attr;
+    cfg.numAttrs = slabs > 1 ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kern, args...);
+}
+
 cudaError_t simt_gemm_bt(int M, int N, int K, const float *A, int64_t sa_i, int64_t sa_k, const void *B, int b_dtype,
                          int64_t sb_k, int64_t sb_j, float *D, int64_t ldd, cudaStream_t stream)
 {
     if (M <= 0 || N <= 0) return cudaSuccess;
     dim3 grid((N + SG_BN - 1) / SG_BN, (M + SG_BM - 1) / SG_BM);
+    const int slabs = simt_slabs((int)(grid.x * grid.y), K);
     if (b_dtype == TSR_BF16)
-        simt_gemm_kernel<float, bf16, SIMT_STORE><<<grid, 256, 0, stream>>>(M, N, K, A, sa_i, sa_k, (const bf16 *)B, sb_k, sb_j,
-                                                                           D, ldd, 0.f, 0.f);
-    else
-        simt_gemm_kernel<float, float, SIMT_STORE><<<grid, 256, 0, stream>>>(M, N, K, A, sa_i, sa_k, (const float *)B, sb_k,
-                                                                            sb_j, D, ldd, 0.f, 0.f);
-    return cudaGetLastError();
+        return simt_launch(simt_gemm_kernel<float, bf16, SIMT_STORE>, grid, slabs, stream, M, N, K, A, sa_i, sa_k, (const bf16 *)B,
+                           sb_k, sb_j, D, ldd, 0.f, 0.f);
+    return simt_launch(simt_gemm_kernel<float, float, SIMT_STORE>, grid, slabs, stream, M, N, K, A, sa_i, sa_k, (const float *)B,
+                       sb_k, sb_j, D, ldd, 0.f, 0.f);
 }
 
 cudaError_t simt_gemm(int M, int N, int K, const void *A, int a_dtype, int64_t sa_i, int64_t sa_k, const float *B,
@@ -128,9 +187,10 @@ cudaError_t simt_gemm(int M, int N, int K, const void *A, int a_dtype, int64_t s
 {
     if (M <= 0 || N <= 0) return cudaSuccess;
     dim3 grid((N + SG_BN - 1) / SG_BN, (M + SG_BM - 1) / SG_BM);
+    const int slabs = simt_slabs((int)(grid.x * grid.y), K);
 #define TSR_SG(TA_, EPI_)                                                                                              \
-    simt_gemm_kernel<TA_, float, EPI_><<<grid, 256, 0, stream>>>(M, N, K, (const TA_ *)A, sa_i, sa_k, B, sb_k, sb_j, D, ldd, \
-                                                                  decay, step_scale)
+    return simt_launch(simt_gemm_kernel<TA_, float, EPI_>, grid, slabs, stream, M, N, K, (const TA_ *)A, sa_i, sa_k, B, sb_k, \
+                       sb_j, D, ldd, decay, step_scale)
     if (a_dtype == TSR_BF16) {
         if (epilogue == SIMT_APPLY) TSR_SG(bf16, SIMT_APPLY);
         else if (epilogue == SIMT_APPLY_BF16) TSR_SG(bf16, SIMT_APPLY_BF16);
@@ -141,7 +201,6 @@ cudaError_t simt_gemm(int M, int N, int K, const void *A, int a_dtype, int64_t s
         else TSR_SG(float, SIMT_STORE);
     }
 #undef TSR_SG
-    return cudaGetLastError();
 }
 
 // ---------------------------------------------------------------------------------------

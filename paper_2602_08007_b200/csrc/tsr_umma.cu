@@ -331,6 +331,18 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
                     continue;
                 }
                 if (epi == EPI_STORE_BF16 && P->out_tma) {
+                    if (ncols < 32 && Nt != N) {
+                        // A box is always 32 columns wide and is clipped only at the matrix edge.  Where the tile ends before
+                        // the matrix does, a box of its last, narrower chunk would also cover the first columns of the
+                        // neighbouring tile (and race with that tile's own store): such a chunk is stored from the registers.
+                        if (lane < nrows) {
+                            bf16 *out = (bf16 *)P->out + (int64_t)(row0 + lane) * P->ld_out + col0;
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                if (j < ncols) out[j] = __float2bfloat16_rn(__uint_as_float(v[j]));
+                        }
+                        continue;
+                    }
                     // The chunk goes to a 32 x 32 BF16 box in shared memory (64-byte rows, 64-byte swizzle;
                     // two boxes per warp inside the patch area) and leaves as one TMA store, which writes
                     // whole lines and clips at the matrix edge.  Direct stores from the lane = row layout

@@ -117,9 +117,10 @@ def test_config_protocol_matches_oracle(cid):
         ob.set_bases(to64(plan.U[i]), to64(plan.V[i]))
         obs.append(ob)
     del G0, Om0
-    worst = {k: 0.0 for k in ("C", "M", "Vm", "W", "dW", "maxabs")}
+    worst = {k: 0.0 for k in ("C", "M", "Vm", "W", "dW", "maxabs", "step1", "step", "after")}
     for t in range(1, 11):
         G = [draw(i, t, ti.ROLE_GRAD) for i in range(nb)]
+        W_gpu_before = [to64(plan.W[i]) for i in range(nb)]
         if t == REFRESH_AT:
             Om = omegas(t, ti.ROLE_OMEGA)
             plan.rsvd_refresh(omegas=Om)
@@ -139,8 +140,12 @@ def test_config_protocol_matches_oracle(cid):
         for i, ob in enumerate(obs):
             if i in short_lockstep and t > 3:
                 continue
+            W_before = ob.W.copy()
             ob.step(to64(G[i]), skip_refresh=True, **HYPER)
             got = dict(C=to64(plan.C[i]), M=to64(plan.M[i]), Vm=to64(plan.Vm[i]), W=to64(plan.W[i]))
+            upd = float(np.linalg.norm((got["W"] - W_gpu_before[i]) - (ob.W - W_before)) / np.linalg.norm(ob.W - W_before))
+            phase = "step1" if t == 1 else ("step" if t < REFRESH_AT else "after")
+            worst[phase] = max(worst[phase], upd)
             want = dict(C=ob.C, M=ob.M, Vm=ob.Vm, W=ob.W)
             for key in ("C", "M", "Vm", "W"):
                 worst[key] = max(worst[key], rel_fro(got[key], want[key]))
@@ -164,5 +169,18 @@ def test_config_protocol_matches_oracle(cid):
              max(x["energy"] for x in rm), max(x["proj"] for x in rm)))
     for key in ("C", "M", "Vm", "W"):
         assert worst[key] < tol, (w.name, worst)
+    # One step's update W_t - W_{t-1} against the oracle's, relative to that update (the weights dwarf it, so the gate
+    # on W would not see a wrong update).  Held to the tolerance of the core from the second step on.  The first
+    # Adam step is sign(c), where every sign the BF16 rounding flips costs 2 (see test_gpu_parity.py); and from the
+    # in-loop refresh on the moments are those of the old basis, so that m / sqrt(v) is large where the new core is
+    # large and the old second moment small, and amplifies the rounding of the core (measured: 0.037 on the
+    # 32000 x 512 embedding block in the step after the refresh, decaying to 0.015 five steps later, everything
+    # else below 0.016): three times the tolerance there.  A factor with a stripe left unwritten gives 0.25 and more.
+    print("one step's update against the oracle's: first step %.2e, steps 2..%d %.2e, from the refresh on %.2e"
+          % (worst["step1"], REFRESH_AT - 1, worst["step"], worst["after"]))
+    bf = w.g_dtype == "bf16"
+    assert worst["step1"] < (0.18 if bf else 100 * tol), (w.name, worst)
+    assert worst["step"] < (tol if bf else 100 * tol), (w.name, worst)
+    assert worst["after"] < (3 * tol if bf else 100 * tol), (w.name, worst)
     if w.g_dtype == "f32":
         assert worst["maxabs"] < TOL_F32_MAXABS, worst
