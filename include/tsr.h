@@ -288,13 +288,20 @@ TSR_API tsr_status tsr_get_stage_ms(tsr_ctx *ctx, float *ms, int32_t count);
  *                 loads for the tiles of that block, so that its consumers run into the bounded
  *                 wait.  Nothing is in flight and no address is touched for those tiles.  It
  *                 exists to exercise the time-out path and requires 0 < wait_clocks <= 1e8.
+ *   projection_launches  how a call that covers every two-sided tensor-core block runs the two
+ *                 contractions of C = U^T G V: 0 = the library decides (ONE launch, with the
+ *                 intermediate T read back from L2, when the T of all blocks together is more than
+ *                 twice the L2 cache; TWO launches otherwise, where T stays in L2 between them
+ *                 anyway and the tiles need not wait for one another), 1 = one launch whenever
+ *                 the device accepts a cooperative launch, 2 = always two.  Tiles, reduction
+ *                 order and results are the same either way.
  * Call it between compute calls of the context (it is synchronous).  Host struct. */
 typedef struct {
     int64_t wait_clocks;
     int32_t max_sweeps;
     int32_t sweep_block;
     int32_t starve_block;
-    int32_t reserved;
+    int32_t projection_launches;
 } tsr_limits;
 TSR_API tsr_status tsr_set_limits(tsr_ctx *ctx, const tsr_limits *limits);
 

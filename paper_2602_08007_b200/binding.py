@@ -55,7 +55,7 @@ class Hyper(ctypes.Structure):
 
 class Limits(ctypes.Structure):
     _fields_ = [("wait_clocks", ctypes.c_int64), ("max_sweeps", ctypes.c_int32), ("sweep_block", ctypes.c_int32),
-                ("starve_block", ctypes.c_int32), ("reserved", ctypes.c_int32)]
+                ("starve_block", ctypes.c_int32), ("projection_launches", ctypes.c_int32)]
 
 
 EXPORTS = [
@@ -347,8 +347,9 @@ class Plan:
         self._check(lib().tsr_poll_status(self.ctx, arr, nb, _stream_ptr(stream)))
         return list(arr)
 
-    def set_limits(self, wait_clocks: int = 0, max_sweeps: int = 0, sweep_block: int = -1, starve_block: int = -1):
-        lim = Limits(wait_clocks, max_sweeps, sweep_block, starve_block, 0)
+    def set_limits(self, wait_clocks: int = 0, max_sweeps: int = 0, sweep_block: int = -1, starve_block: int = -1,
+                   projection_launches: int = 0):
+        lim = Limits(wait_clocks, max_sweeps, sweep_block, starve_block, projection_launches)
         self._check(lib().tsr_set_limits(self.ctx, ctypes.byref(lim)))
 
     def set_profiling(self, enable: bool):

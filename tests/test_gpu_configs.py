@@ -66,6 +66,9 @@ def test_config_protocol_matches_oracle(cid):
     plan = tsr.Plan([dict(m=b.m, n=b.n, r=b.r, p=b.p, q=b.q, K=0, is_embedding=b.is_embedding) for b in blocks], g_dtype=dt)
     nb = len(blocks)
     assert all(plan.uses_tensor_cores(i) == (w.g_dtype == "bf16") for i in range(nb))
+    # the core projection as ONE launch (tiles that wait for one another) on the 60M and 350M sets, as the library
+    # chooses on the others (for sets this small: two plain launches)
+    plan.set_limits(projection_launches=1 if cid in (1, 3) else 0)
 
     def draw(i, step, role):
         b = blocks[i]

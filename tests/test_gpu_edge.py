@@ -198,7 +198,8 @@ def test_sweep_limit_flags_not_converged_on_that_block_only(shape):
     assert torch.equal(res[0][1], res[1][1]) and torch.equal(res[0][2], res[1][2])
 
 
-def test_bounded_wait_that_runs_out_reports_timeout_and_the_context_recovers():
+@pytest.mark.parametrize("launches", [1, 2])
+def test_bounded_wait_that_runs_out_reports_timeout_and_the_context_recovers(launches):
     """A wait inside a tensor-core kernel is made to run out in the only safe way: the library is
     told (tsr_set_limits) to issue no loads for the tiles of one block in the first projection
     GEMM and to bound every wait by 2e6 clock ticks (about a millisecond).  Nothing is in flight
@@ -215,13 +216,14 @@ def test_bounded_wait_that_runs_out_reports_timeout_and_the_context_recovers():
     with pytest.raises(tsr.TsrError):                     # the switch is refused without a short budget
         plan.set_limits(starve_block=1)
     G64 = [fill_gradient(plan, i, 160 + i) for i in range(2)]
-    plan.set_limits(wait_clocks=2_000_000, starve_block=1)
+    # (both forms of the projection: one launch with tiles in dynamic order, two plain launches)
+    plan.set_limits(wait_clocks=2_000_000, starve_block=1, projection_launches=launches)
     plan.project_core()
     torch.cuda.synchronize()
     assert plan.poll_status() == [0, 10]                  # TSR_ERR_TIMEOUT on the starved block only
     assert rel_fro(to64(plan.C[0]), oracle.project_core(G64[0], to64(plan.U[0]), to64(plan.V[0]))) < TOL_BF16
     # back to the defaults: the same context works as if nothing had happened
-    plan.set_limits()
+    plan.set_limits(projection_launches=launches)
     blks = []
     for i, s in enumerate(shapes):
         W0 = fill_weights(plan, i, 170 + i)

@@ -100,9 +100,13 @@ def test_fp32_path_decay_and_scale():
     _run_steps(tsr, plan, F32_SHAPES[1:], torch.float32, 4, True, TOL_F32, wd=0.1, scale=0.25)
 
 
+# projection_launches: 1 = both contractions of the core as ONE launch (tiles in dynamic order that wait for one
+# another through counters), 2 = two plain launches; left to itself the library takes two for sets this small
+@pytest.mark.parametrize("launches", [1, 2])
 @pytest.mark.parametrize("fuse", [False, True])
-def test_bf16_path_steps_match_oracle(fuse):
+def test_bf16_path_steps_match_oracle(fuse, launches):
     tsr, plan = _plan(BF16_SHAPES, torch.bfloat16)
+    plan.set_limits(projection_launches=launches)
     assert all(plan.uses_tensor_cores(i) for i in range(len(BF16_SHAPES)))
     _given_bases(plan, BF16_SHAPES)
     _run_steps(tsr, plan, BF16_SHAPES, torch.bfloat16, 10, fuse, TOL_BF16)
@@ -118,9 +122,11 @@ def test_bf16_path_decay_and_scale():
 WIDE_SHAPES = [dict(m=640, n=768, r=256), dict(m=1100, n=1024, r=512), dict(m=600, n=520, r=264)]
 
 
+@pytest.mark.parametrize("launches", [1, 2])
 @pytest.mark.parametrize("fuse", [False, True])
-def test_bf16_path_wide_tiles_match_oracle(fuse):
+def test_bf16_path_wide_tiles_match_oracle(fuse, launches):
     tsr, plan = _plan(WIDE_SHAPES, torch.bfloat16)
+    plan.set_limits(projection_launches=launches)
     _given_bases(plan, WIDE_SHAPES)
     _run_steps(tsr, plan, WIDE_SHAPES, torch.bfloat16, 3, fuse, TOL_BF16)
 
@@ -142,7 +148,8 @@ def test_update_reaches_every_entry_for_ranks_off_the_tile_grid(m, n, r):
         V = torch.zeros(s["n"], s["r"]); V[:s["r"], :s["r"]] = torch.eye(s["r"])
         set_bases(plan, i, U, V)
     plan.bases_changed()
-    for fuse in (True, False):
+    for fuse, launches in ((True, 1), (False, 1), (True, 2)):
+        plan.set_limits(projection_launches=launches)
         for i, s in enumerate(shapes):
             fill_gradient(plan, i, 700 + i)
             plan.W[i].zero_(); plan.M[i].zero_(); plan.Vm[i].zero_()
