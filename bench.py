@@ -396,7 +396,9 @@ def run_ours(args, w: ti.Workload):
     torch.cuda.synchronize()
     status = plan.poll_status()
 
-    plan.set_profiling(True)
+    # stage events only when they are read inside the loop: an event between two kernels keeps the second one from
+    # setting itself up under the first one's tail (programmatic dependent launch)
+    plan.set_profiling(bool(args.stage_times))
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
     stage = []
     sampler = ClockSampler(physical_gpu_index(local_rank))

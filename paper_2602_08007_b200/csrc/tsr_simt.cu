@@ -3,6 +3,7 @@
 // operand conversion for the tensor-core path, and the Gaussian generator for Omega.
 #include "tsr_internal.h"
 #include "tsr_device.cuh"
+#include "tsr_pdl.cuh"
 #include <cooperative_groups.h>
 
 namespace tsr {
@@ -23,6 +24,7 @@ template <>
 __device__ __forceinline__ float load_as_float<bf16>(const bf16 *p) { return __bfloat162float(*p); }
 
 constexpr int SG_BM = 64, SG_BN = 64, SG_BK = 16;
+constexpr int SG_LD = SG_BM * SG_BK / 256;   // elements of each operand slice a thread moves
 
 template <typename TA, typename TB, int EPI>
 __global__ void __launch_bounds__(256)
@@ -33,6 +35,8 @@ simt_gemm_kernel(int M, int N, int K, const TA *__restrict__ A, int64_t sa_i, in
     __shared__ float As[SG_BK][SG_BM + 4];
     __shared__ float Bs[SG_BK][SG_BN + 4];
     __shared__ float red[SG_BM * SG_BN];     // this CTA's partial tile, [a][b][thread]: read and written without bank conflicts
+    pdl_trigger();
+    pdl_wait();                              // nothing to set up: the operands are the predecessor's results
     const int tid = threadIdx.x;
     const int tx = tid % 16, ty = tid / 16;
     const int m0 = blockIdx.y * SG_BM, n0 = blockIdx.x * SG_BN;
@@ -53,11 +57,11 @@ simt_gemm_kernel(int M, int N, int K, const TA *__restrict__ A, int64_t sa_i, in
     const bool b_j_fast = (sb_j == 1);
 
     // global -> registers -> shared, with the next K slice in flight while the current one is used
-    float ra[4], rb[4];
+    float ra[SG_LD], rb[SG_LD];
     auto fetch = [&](int k0) {
 #pragma unroll
-        for (int l = 0; l < 4; ++l) {
-            const int e = tid + l * 256;  // 0..1023
+        for (int l = 0; l < SG_LD; ++l) {
+            const int e = tid + l * 256;  // 0 .. 64 * SG_BK - 1
             int ai, ak;
             if (a_k_fast) { ak = e % SG_BK; ai = e / SG_BK; } else { ai = e % SG_BM; ak = e / SG_BM; }
             const int gi = m0 + ai, gk = k0 + ak;
@@ -71,7 +75,7 @@ simt_gemm_kernel(int M, int N, int K, const TA *__restrict__ A, int64_t sa_i, in
     if (k_begin < k_end) fetch(k_begin);
     for (int k0 = k_begin; k0 < k_end; k0 += SG_BK) {
 #pragma unroll
-        for (int l = 0; l < 4; ++l) {
+        for (int l = 0; l < SG_LD; ++l) {
             const int e = tid + l * 256;
             int ai, ak;
             if (a_k_fast) { ak = e % SG_BK; ai = e / SG_BK; } else { ai = e % SG_BM; ak = e / SG_BM; }
@@ -155,17 +159,7 @@ static int simt_slabs(int tiles, int K)
 template <typename Kern, typename... Args>
 static cudaError_t simt_launch(Kern kern, dim3 grid, int slabs, cudaStream_t stream, Args... args)
 {
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(grid.x, grid.y, (unsigned)slabs);
-    cfg.blockDim = dim3(256);
-    cfg.dynamicSmemBytes = 0;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = (unsigned)slabs;
-    cfg.attrs = attr;
-    cfg.numAttrs = slabs > 1 ? 1 : 0;
-    return cudaLaunchKernelEx(&cfg, kern, args...);
+    return launch_dependent(kern, dim3(grid.x, grid.y, (unsigned)slabs), dim3(256), 0, stream, slabs, args...);
 }
 
 cudaError_t simt_gemm_bt(int M, int N, int K, const float *A, int64_t sa_i, int64_t sa_k, const void *B, int b_dtype,
@@ -219,6 +213,8 @@ core_update_kernel(const CoreUpdateArgs *__restrict__ args, const int32_t *__res
                    int ntile)
 {
     // ntile (1 .. CU_TILES) tiles of 32 x 32 per CTA: small launches take one, so that more CTAs share the work
+    pdl_trigger();
+    pdl_wait();
     const CoreUpdateArgs a = args[list[blockIdx.z]];
     const int r = a.r, nc = a.nc;   // rows, columns of the core (square except for a one-sided block)
     const int r0 = blockIdx.y * 32;
@@ -290,8 +286,8 @@ cudaError_t core_update_launch(const CoreUpdateArgs *args_dev, const int32_t *li
     if (nblocks <= 0) return cudaSuccess;
     const int t = (max_r + 31) / 32, tc = (max_cols + 31) / 32;
     const int ntile = ((int64_t)t * tc * nblocks >= 4 * 148 * CU_TILES) ? CU_TILES : 1;
-    core_update_kernel<<<dim3((tc + ntile - 1) / ntile, t, nblocks), 256, 0, stream>>>(args_dev, list_dev, sc, mode, ntile);
-    return cudaGetLastError();
+    return launch_dependent(core_update_kernel, dim3((tc + ntile - 1) / ntile, t, nblocks), dim3(256), 0, stream, 1, args_dev, list_dev,
+                            sc, mode, ntile);
 }
 
 // ---------------------------------------------------------------------------------------

@@ -34,6 +34,7 @@
 #include "tsr_device.cuh"
 #include "tsr_internal.h"
 #include "tsr_umma.cuh"
+#include "tsr_pdl.cuh"
 
 namespace tsr {
 
@@ -91,6 +92,7 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
     uint64_t *bar_sfull = bar_acc_empty + 2, *bar_sempty = bar_sfull + SR;
     volatile int *sched_tile = (volatile int *)(tmem_slot + 1);     // [SR]
 
+    pdl_trigger();   // the next kernel of the stream may set itself up on SMs this grid does not (or no longer) use
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const long long budget = wait_budget(sc);
     const uint32_t rank = cluster_ctarank();          // 0 = leader of the CTA pair
@@ -123,6 +125,7 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
     // while its peer had not yet allocated left the peer waiting in tcgen05.alloc for ever (seen when other
     // kernels on the same SMs delayed one of the two warps).
     if (warp == 1) asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    pdl_wait();      // set-up done; from here on the kernel reads what its predecessors wrote
 
     // i-th tile of this pair, for a reader of the ring (every role but the leader's producer): false when the wait ran
     // out; t < 0 when the table is exhausted.  `arrive`: this thread releases the slot (one lane per epilogue warp).
@@ -508,9 +511,8 @@ static cudaError_t launch_one(const UmmaProblem *probs, const UmmaTile *tiles, i
 {
     using SM = UmmaSmem<BN, PLANES>;
     const int pairs = num_tiles < num_sms / 2 ? num_tiles : num_sms / 2;
-    umma_gemm_kernel<BN, EPI, PLANES><<<2 * pairs, UG_THREADS, SM::TOTAL, stream>>>(probs, tiles, num_tiles, sc, status, nullptr,
-                                                                                    nullptr, 0, 0);
-    return cudaGetLastError();
+    return launch_dependent(umma_gemm_kernel<BN, EPI, PLANES>, dim3(2 * pairs), dim3(UG_THREADS), (size_t)SM::TOTAL, stream, 1, probs,
+                            tiles, num_tiles, sc, status, (const UmmaProblem *)nullptr, (int32_t *)nullptr, 0, 0);
 }
 
 template <int BN, int EPI, int PLANES>

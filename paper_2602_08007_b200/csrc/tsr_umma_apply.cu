@@ -20,6 +20,7 @@
 // All waits are bounded (see mbar_wait); on expiry the CTA flags TSR_ERR_TIMEOUT and drains.
 #include "tsr_internal.h"
 #include "tsr_umma.cuh"
+#include "tsr_pdl.cuh"
 
 namespace tsr {
 
@@ -93,6 +94,7 @@ umma_apply_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restr
     uint32_t *tmem_slot = (uint32_t *)(bars + AP_NBARS);
     __shared__ int s_timeout;   // 0, or 1 + the first tile (table index) this CTA gave up on
 
+    pdl_trigger();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int stride = gridDim.x;
     const long long budget = wait_budget(sc);
@@ -113,6 +115,7 @@ umma_apply_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restr
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    pdl_wait();      // set-up done; P = U D of the kernel before this one is read from here on
 
     if (warp == 0) {
         if (lane == 0) {
@@ -286,14 +289,13 @@ cudaError_t umma_apply_launch(const UmmaProblem *probs, const UmmaTile *tiles, i
     if (num_tiles <= 0) return cudaSuccess;
     const int grid = num_tiles < num_sms ? num_tiles : num_sms;
     if (bn == 256 && w_bytes == 4)
-        umma_apply_kernel<256, 4><<<grid, AP_THREADS, ApplyCfg<256>::SMEM, stream>>>(probs, tiles, num_tiles, sc, status);
+        return launch_dependent(umma_apply_kernel<256, 4>, dim3(grid), dim3(AP_THREADS), (size_t)ApplyCfg<256>::SMEM, stream, 1, probs, tiles, num_tiles, sc, status);
     else if (bn == 256)
-        umma_apply_kernel<256, 2><<<grid, AP_THREADS, ApplyCfg<256>::SMEM, stream>>>(probs, tiles, num_tiles, sc, status);
+        return launch_dependent(umma_apply_kernel<256, 2>, dim3(grid), dim3(AP_THREADS), (size_t)ApplyCfg<256>::SMEM, stream, 1, probs, tiles, num_tiles, sc, status);
     else if (w_bytes == 4)
-        umma_apply_kernel<128, 4><<<grid, AP_THREADS, ApplyCfg<128>::SMEM, stream>>>(probs, tiles, num_tiles, sc, status);
+        return launch_dependent(umma_apply_kernel<128, 4>, dim3(grid), dim3(AP_THREADS), (size_t)ApplyCfg<128>::SMEM, stream, 1, probs, tiles, num_tiles, sc, status);
     else
-        umma_apply_kernel<128, 2><<<grid, AP_THREADS, ApplyCfg<128>::SMEM, stream>>>(probs, tiles, num_tiles, sc, status);
-    return cudaGetLastError();
+        return launch_dependent(umma_apply_kernel<128, 2>, dim3(grid), dim3(AP_THREADS), (size_t)ApplyCfg<128>::SMEM, stream, 1, probs, tiles, num_tiles, sc, status);
 }
 
 }  // namespace tsr
