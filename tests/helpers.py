@@ -147,3 +147,22 @@ def f32(x: float) -> float:
 
 
 HYPER = dict(lr=f32(1e-3), beta1=f32(0.9), beta2=f32(0.999), eps=f32(1e-8))
+
+
+def update_err(w_gpu_before, w_gpu_after, w_ref_before, w_ref_after):
+    """Error of one step's update W_t - W_{t-1} of the library against the reference's, relative to the reference's
+    update (FP64 arrays).  The weights dwarf one step's update, so a gate on W alone cannot see a wrong update."""
+    d_ref = w_ref_after - w_ref_before
+    return float(np.linalg.norm((w_gpu_after - w_gpu_before) - d_ref) / np.linalg.norm(d_ref))
+
+
+def update_bound(bf16, first_adam_step=False, after_refresh=False):
+    """Bound on update_err.  BF16 path: the tolerance of the core (2e-2) from the second step on, 0.25 on the first Adam
+    step (D = sign(C): every sign the operand rounding flips costs 2; measured 0.05 .. 0.153, the largest on a 32 x 32 core), three times the tolerance
+    from an in-loop refresh on (moments of the old basis amplify the rounding of the new core; measured up to 0.037).
+    FP32 path: 1e-2 throughout (measured 2e-5 .. 2e-4)."""
+    if not bf16:
+        return 100 * TOL_F32
+    if first_adam_step:
+        return 0.25
+    return 3 * TOL_BF16 if after_refresh else TOL_BF16

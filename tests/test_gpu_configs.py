@@ -182,7 +182,7 @@ def test_config_protocol_matches_oracle(cid):
     print("one step's update against the oracle's: first step %.2e, steps 2..%d %.2e, from the refresh on %.2e"
           % (worst["step1"], REFRESH_AT - 1, worst["step"], worst["after"]))
     bf = w.g_dtype == "bf16"
-    assert worst["step1"] < (0.18 if bf else 100 * tol), (w.name, worst)
+    assert worst["step1"] < (0.25 if bf else 100 * tol), (w.name, worst)
     assert worst["step"] < (tol if bf else 100 * tol), (w.name, worst)
     assert worst["after"] < (3 * tol if bf else 100 * tol), (w.name, worst)
     if w.g_dtype == "f32":

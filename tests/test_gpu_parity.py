@@ -7,7 +7,7 @@ import torch
 import oracle
 import tsr_inputs as ti
 from helpers import (HYPER, TOL_BF16, TOL_F32, TOL_F32_MAXABS, check_refresh, f32, fill_gradient, fill_weights, max_abs_err,
-                     rel_fro, set_bases, to64)
+                     rel_fro, set_bases, to64, update_bound, update_err)
 
 pytestmark = pytest.mark.gpu
 
@@ -62,9 +62,9 @@ def _run_steps(tsr, plan, shapes, dtype, steps, fuse, tol, wd=0.0, scale=1.0, ru
     # second Adam step on, and is held to the tolerance of the core there (measured 4e-3 .. 9e-3 on the BF16 path, where
     # a 16-row stripe of a 264-row factor left unwritten gave 0.25 and more; 2e-5 .. 2e-4 on the FP32 path).  The
     # first Adam step is m / sqrt(v) = sign(c): every core entry whose sign the BF16 rounding of the operands flips
-    # moves by 2 (measured 0.05 .. 0.125), so that step is only held to 0.18 on the BF16 path.
+    # moves by 2 (measured 0.05 .. 0.153, the largest on a 32 x 32 core), so that step is only held to 0.25 on the BF16 path.
     bf = dtype == torch.bfloat16
-    first_tol = (0.18 if rule == 0 else tol) if bf else 100 * tol
+    first_tol = (0.25 if rule == 0 else tol) if bf else 100 * tol
     later_tol = tol if bf else 100 * tol
     print("error of one step's update relative to that update: first step %.2e (bound %.0e), later steps %.2e (bound %.0e)"
           % (worst_upd[0], first_tol, worst_upd[1], later_tol))
@@ -267,6 +267,7 @@ def test_two_workers_averaging_the_core_match_the_oracle():
             avg = sum(pl.C[i] for pl in plans) / nw
             for pl in plans:
                 pl.C[i].copy_(avg)
+        Wg_before = [to64(plans[0].W[i]) for i in range(len(shapes))]
         for pl in plans:
             pl.adam_core_step(h)
             pl.backproject_apply(h)
@@ -274,7 +275,9 @@ def test_two_workers_averaging_the_core_match_the_oracle():
         for i in range(len(shapes)):
             Cbar = sum(oracle.project_core(G64[w][i], Uo[i], Vbo[i]) for w in range(nw)) / nw
             D = oracle.adam_core(Cbar, Mo[i], Vo[i], HYPER["beta1"], HYPER["beta2"], HYPER["eps"], t)
+            Wo_before = Wo[i].copy()
             oracle.backproject_apply(Uo[i], D, Vbo[i], Wo[i], HYPER["lr"])
+            assert update_err(Wg_before[i], to64(plans[0].W[i]), Wo_before, Wo[i]) < update_bound(True, first_adam_step=(t == 1))
             assert torch.equal(plans[0].W[i], plans[1].W[i]) and torch.equal(plans[0].M[i], plans[1].M[i])
             worst = max(worst, rel_fro(to64(plans[0].C[i]), Cbar), rel_fro(to64(plans[0].M[i]), Mo[i]),
                         rel_fro(to64(plans[0].Vm[i]), Vo[i]), rel_fro(to64(plans[0].W[i]), Wo[i]))
@@ -441,6 +444,7 @@ def test_mini_llama_grouped_lockstep_with_refresh():
         ob.set_bases(to64(plan.U[i]), to64(plan.V[i]))
         blks.append(ob)
     worst = 0.0
+    worst_upd = 0.0      # one step's update against the oracle's, as a fraction of its bound
     for t in range(1, 8):
         G64 = [fill_gradient(plan, i, ti.seed_for(cfg, i, t, ti.ROLE_GRAD), signal_rank=8) for i in range(nb)]
         due = [i for i, s in enumerate(shapes) if t % s["K"] == 0]
@@ -453,14 +457,21 @@ def test_mini_llama_grouped_lockstep_with_refresh():
                 check_refresh(plan, i, G64[i], to64(oms[j]), shapes[i]["r"], 1, 8)
                 blks[i].set_bases(to64(plan.U[i]), to64(plan.V[i]))
         h = tsr.make_hyper(t)
+        Wg_before = [to64(plan.W[i]) for i in range(nb)]
         plan.step(h, fuse_adam=(t % 2 == 0))
         torch.cuda.synchronize()
         for i, ob in enumerate(blks):
+            Wo_before = ob.W.copy()
             ob.step(G64[i], skip_refresh=True, **HYPER)
             for a, b in ((plan.C[i], ob.C), (plan.M[i], ob.M), (plan.Vm[i], ob.Vm), (plan.W[i], ob.W)):
                 worst = max(worst, rel_fro(to64(a), b))
+            frac = (update_err(Wg_before[i], to64(plan.W[i]), Wo_before, ob.W)
+                    / update_bound(True, first_adam_step=(t == 1), after_refresh=(t >= shapes[i]["K"])))
+            worst_upd = max(worst_upd, frac)
     assert plan.poll_status() == [0] * nb
     assert worst < TOL_BF16, worst
+    print("mini LLaMA set: worst update error as a fraction of its bound %.2f" % worst_upd)
+    assert worst_upd < 1.0, worst_upd
 
 
 def test_step_grouped_refreshes_on_schedule_and_embed_step():
@@ -571,6 +582,7 @@ def test_one_sided_arm_matches_oracle(dtype, shapes, tol, fuse):
     for t in range(1, 6):
         G64 = [fill_gradient(plan, i, ti.seed_for(93, i, t, ti.ROLE_GRAD)) for i in range(nb)]
         h = tsr.make_hyper(t, lr=1e-3, weight_decay=wd, scale=scale)
+        Wg_before = [to64(plan.W[i]) for i in range(nb)]
         if fuse:
             plan.step(h, fuse_adam=True)
         else:
@@ -581,13 +593,17 @@ def test_one_sided_arm_matches_oracle(dtype, shapes, tol, fuse):
         for i in range(nb):
             if i in two:
                 ob = two[i]
+                Wo_before = ob.W.copy()
                 ob.step(G64[i], weight_decay=f32(wd), scale=f32(scale), **HYPER)
                 ref = (ob.C, ob.M, ob.Vm, ob.W)
             else:
                 C = oracle.project_one_sided(G64[i], U64[i])
                 D = oracle.adam_core(C, M[i], Vm[i], HYPER["beta1"], HYPER["beta2"], HYPER["eps"], t)
+                Wo_before = W[i].copy()
                 oracle.backproject_one_sided(U64[i], D, W[i], HYPER["lr"], f32(wd), f32(scale))
                 ref = (C, M[i], Vm[i], W[i])
+            upd = update_err(Wg_before[i], to64(plan.W[i]), Wo_before, ref[3])
+            assert upd < update_bound(dtype == torch.bfloat16, first_adam_step=(t == 1)), (t, i, upd)
             got = (plan.C[i], plan.M[i], plan.Vm[i], plan.W[i])
             for key, g, e in zip(("C", "M", "Vm", "W"), got, ref):
                 worst[key] = max(worst[key], rel_fro(to64(g), e))
