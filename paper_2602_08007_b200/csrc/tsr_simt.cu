@@ -5,6 +5,7 @@
 #include "tsr_device.cuh"
 #include "tsr_pdl.cuh"
 #include <cooperative_groups.h>
+#include <type_traits>
 
 namespace tsr {
 
@@ -25,6 +26,7 @@ __device__ __forceinline__ float load_as_float<bf16>(const bf16 *p) { return __b
 
 constexpr int SG_BM = 64, SG_BN = 64, SG_BK = 16;
 constexpr int SG_LD = SG_BM * SG_BK / 256;   // elements of each operand slice a thread moves
+constexpr int SG_NST = 3;                      // shared-memory stages of the FP32 operand slices
 
 template <typename TA, typename TB, int EPI>
 __global__ void __launch_bounds__(256)
@@ -32,9 +34,12 @@ simt_gemm_kernel(int M, int N, int K, const TA *__restrict__ A, int64_t sa_i, in
                  const TB *__restrict__ B, int64_t sb_k, int64_t sb_j, float *__restrict__ D, int64_t ldd,
                  float decay, float step_scale)
 {
-    __shared__ float As[SG_BK][SG_BM + 4];
-    __shared__ float Bs[SG_BK][SG_BN + 4];
-    __shared__ float red[SG_BM * SG_BN];     // this CTA's partial tile, [a][b][thread]: read and written without bank conflicts
+    // K slices of both operands, SG_NST stages of [k][row] and [k][column]; after the main loop the same storage holds
+    // this CTA's partial tile for the cluster's reduction
+    __shared__ __align__(16) float smem_ab[SG_NST * 2 * SG_BK * (SG_BM + 4)];
+    float (*As)[SG_BK][SG_BM + 4] = (float (*)[SG_BK][SG_BM + 4])smem_ab;
+    float (*Bs)[SG_BK][SG_BN + 4] = (float (*)[SG_BK][SG_BN + 4])(smem_ab + SG_NST * SG_BK * (SG_BM + 4));
+    float *red = smem_ab;                    // [a][b][thread]: read and written without bank conflicts
     pdl_trigger();
     pdl_wait();                              // nothing to set up: the operands are the predecessor's results
     const int tid = threadIdx.x;
@@ -55,50 +60,91 @@ simt_gemm_kernel(int M, int N, int K, const TA *__restrict__ A, int64_t sa_i, in
     // Loader index maps: put the unit-stride index on consecutive threads.
     const bool a_k_fast = (sa_k == 1);
     const bool b_j_fast = (sb_j == 1);
-
-    // global -> registers -> shared, with the next K slice in flight while the current one is used
-    float ra[SG_LD], rb[SG_LD];
-    auto fetch = [&](int k0) {
-#pragma unroll
-        for (int l = 0; l < SG_LD; ++l) {
-            const int e = tid + l * 256;  // 0 .. 64 * SG_BK - 1
-            int ai, ak;
-            if (a_k_fast) { ak = e % SG_BK; ai = e / SG_BK; } else { ai = e % SG_BM; ak = e / SG_BM; }
-            const int gi = m0 + ai, gk = k0 + ak;
-            ra[l] = (gi < M && gk < k_end) ? load_as_float<TA>(A + (int64_t)gi * sa_i + (int64_t)gk * sa_k) : 0.f;
-            int bj, bk;
-            if (b_j_fast) { bj = e % SG_BN; bk = e / SG_BN; } else { bk = e % SG_BK; bj = e / SG_BK; }
-            const int gj = n0 + bj, gk2 = k0 + bk;
-            rb[l] = (gj < N && gk2 < k_end) ? load_as_float<TB>(B + (int64_t)gk2 * sb_k + (int64_t)gj * sb_j) : 0.f;
-        }
-    };
-    if (k_begin < k_end) fetch(k_begin);
-    for (int k0 = k_begin; k0 < k_end; k0 += SG_BK) {
-#pragma unroll
-        for (int l = 0; l < SG_LD; ++l) {
-            const int e = tid + l * 256;
-            int ai, ak;
-            if (a_k_fast) { ak = e % SG_BK; ai = e / SG_BK; } else { ai = e % SG_BM; ak = e / SG_BM; }
-            As[ak][ai] = ra[l];
-            int bj, bk;
-            if (b_j_fast) { bj = e % SG_BN; bk = e / SG_BN; } else { bk = e % SG_BK; bj = e / SG_BK; }
-            Bs[bk][bj] = rb[l];
-        }
-        __syncthreads();
-        if (k0 + SG_BK < k_end) fetch(k0 + SG_BK);
+    auto a_index = [&](int e, int &ai, int &ak) { if (a_k_fast) { ak = e % SG_BK; ai = e / SG_BK; } else { ai = e % SG_BM; ak = e / SG_BM; } };
+    auto b_index = [&](int e, int &bj, int &bk) { if (b_j_fast) { bj = e % SG_BN; bk = e / SG_BN; } else { bk = e % SG_BK; bj = e / SG_BK; } };
+    auto compute = [&](int stage) {
 #pragma unroll
         for (int kk = 0; kk < SG_BK; ++kk) {
-            float av[4], bv[4];
-#pragma unroll
-            for (int a = 0; a < 4; ++a) av[a] = As[kk][ty * 4 + a];
-#pragma unroll
-            for (int b = 0; b < 4; ++b) bv[b] = Bs[kk][tx * 4 + b];
+            const float4 a4 = *(const float4 *)&As[stage][kk][ty * 4];
+            const float4 b4 = *(const float4 *)&Bs[stage][kk][tx * 4];
+            const float av[4] = {a4.x, a4.y, a4.z, a4.w}, bv[4] = {b4.x, b4.y, b4.z, b4.w};
 #pragma unroll
             for (int a = 0; a < 4; ++a)
 #pragma unroll
                 for (int b = 0; b < 4; ++b) acc[a][b] = fmaf(av[a], bv[b], acc[a][b]);
         }
+    };
+
+    constexpr bool ASYNC = std::is_same<TA, float>::value && std::is_same<TB, float>::value;
+    if (ASYNC) {
+        // FP32 operands go from global to shared memory with 4-byte asynchronous copies (any stride, any alignment;
+        // elements past an edge are zero-filled), SG_NST - 1 slices ahead of the arithmetic: with a handful of slices
+        // per CTA the kernel is a chain of global-memory latencies, and this takes two of every three off it.
+        const float *Af = (const float *)A, *Bf = (const float *)B;
+        auto issue = [&](int stage, int k0) {
+#pragma unroll
+            for (int l = 0; l < SG_LD; ++l) {
+                const int e = tid + l * 256;
+                int ai, ak, bj, bk;
+                a_index(e, ai, ak);
+                b_index(e, bj, bk);
+                const int gi = m0 + ai, gk = k0 + ak, gj = n0 + bj, gk2 = k0 + bk;
+                const bool va = gi < M && gk < k_end, vb = gj < N && gk2 < k_end;
+                const float *pa = va ? Af + (int64_t)gi * sa_i + (int64_t)gk * sa_k : Af;
+                const float *pb = vb ? Bf + (int64_t)gk2 * sb_k + (int64_t)gj * sb_j : Bf;
+                asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"((uint32_t)__cvta_generic_to_shared(&As[stage][ak][ai])),
+                             "l"(pa), "r"(va ? 4 : 0) : "memory");
+                asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"((uint32_t)__cvta_generic_to_shared(&Bs[stage][bk][bj])),
+                             "l"(pb), "r"(vb ? 4 : 0) : "memory");
+            }
+        };
+        const int nsteps = (k_end - k_begin + SG_BK - 1) / SG_BK;
+        for (int st = 0; st < SG_NST - 1; ++st) {
+            if (st < nsteps) issue(st, k_begin + st * SG_BK);
+            asm volatile("cp.async.commit_group;" ::: "memory");
+        }
+        for (int st = 0; st < nsteps; ++st) {
+            asm volatile("cp.async.wait_group %0;" ::"n"(SG_NST - 2) : "memory");
+            __syncthreads();                 // slice st has landed for every thread, and slice st - 1 has been used by all
+            const int nx = st + SG_NST - 1;
+            if (nx < nsteps) issue(nx % SG_NST, k_begin + nx * SG_BK);
+            asm volatile("cp.async.commit_group;" ::: "memory");
+            compute(st % SG_NST);
+        }
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
         __syncthreads();
+    } else {
+        // global -> registers -> shared, with the next K slice in flight while the current one is used
+        float ra[SG_LD], rb[SG_LD];
+        auto fetch = [&](int k0) {
+#pragma unroll
+            for (int l = 0; l < SG_LD; ++l) {
+                const int e = tid + l * 256;  // 0 .. 64 * SG_BK - 1
+                int ai, ak, bj, bk;
+                a_index(e, ai, ak);
+                b_index(e, bj, bk);
+                const int gi = m0 + ai, gk = k0 + ak;
+                ra[l] = (gi < M && gk < k_end) ? load_as_float<TA>(A + (int64_t)gi * sa_i + (int64_t)gk * sa_k) : 0.f;
+                const int gj = n0 + bj, gk2 = k0 + bk;
+                rb[l] = (gj < N && gk2 < k_end) ? load_as_float<TB>(B + (int64_t)gk2 * sb_k + (int64_t)gj * sb_j) : 0.f;
+            }
+        };
+        if (k_begin < k_end) fetch(k_begin);
+        for (int k0 = k_begin; k0 < k_end; k0 += SG_BK) {
+#pragma unroll
+            for (int l = 0; l < SG_LD; ++l) {
+                const int e = tid + l * 256;
+                int ai, ak, bj, bk;
+                a_index(e, ai, ak);
+                b_index(e, bj, bk);
+                As[0][ak][ai] = ra[l];
+                Bs[0][bk][bj] = rb[l];
+            }
+            __syncthreads();
+            if (k0 + SG_BK < k_end) fetch(k0 + SG_BK);
+            compute(0);
+            __syncthreads();
+        }
     }
     if (nslab > 1) {
         namespace cg = cooperative_groups;
