@@ -215,6 +215,9 @@ def test_bounded_wait_that_runs_out_reports_timeout_and_the_context_recovers(lau
     plan.bases_changed()
     with pytest.raises(tsr.TsrError):                     # the switch is refused without a short budget
         plan.set_limits(starve_block=1)
+    with pytest.raises(tsr.TsrError) as ei:               # so is a launch mode that does not exist
+        plan.set_limits(projection_launches=3)
+    assert ei.value.status == 1                           # TSR_ERR_INVALID_ARG
     G64 = [fill_gradient(plan, i, 160 + i) for i in range(2)]
     # (both forms of the projection: one launch with tiles in dynamic order, two plain launches)
     plan.set_limits(wait_clocks=2_000_000, starve_block=1, projection_launches=launches)
