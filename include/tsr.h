@@ -305,6 +305,16 @@ typedef struct {
 } tsr_limits;
 TSR_API tsr_status tsr_set_limits(tsr_ctx *ctx, const tsr_limits *limits);
 
+/* The Gram step of the refresh on its own: S = X^T X for an X of (side == 0 ? m : n) rows and
+ * k = r + p columns, through exactly the kernels the orthonormalisations and the small SVD of
+ * Section 3.5 use for block `block` (the integer tensor-core form for a sketch with
+ * 2k <= min(m, n), k >= 8 on the tensor-core path; the FP64 tensor path otherwise).  (No passage of
+ * the paper defines this call; it exists so that the Gram matrices can be checked against their
+ * definition.)  X: device, FP32, row-major, row pitch k.  S: device, FP64, k x k, row pitch k,
+ * both triangles written.  The block's refresh work buffers are overwritten; U, V, moments and
+ * weights are not touched.  Asynchronous on `stream`; a non-finite X flags TSR_ERR_NONFINITE. */
+TSR_API tsr_status tsr_refresh_gram(tsr_ctx *ctx, int32_t block, int32_t side, const float *X, double *S, void *stream);
+
 /* Number of CUDA kernels this context has launched since tsr_create. */
 TSR_API tsr_status tsr_launch_count(const tsr_ctx *ctx, uint64_t *count);
 

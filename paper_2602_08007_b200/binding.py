@@ -66,7 +66,7 @@ EXPORTS = [
     "tsr_rsvd_refresh_grouped", "tsr_embed_step_grouped", "tsr_step_grouped", "tsr_step_grouped_host",
     "tsr_comm_bytes", "tsr_state_elems", "tsr_poll_status", "tsr_generate_omega", "tsr_block_uses_tensor_cores",
     "tsr_set_profiling", "tsr_get_stage_ms", "tsr_launch_count", "tsr_project_core_static", "tsr_dense_adamw",
-    "tsr_set_limits",
+    "tsr_set_limits", "tsr_refresh_gram",
 ]
 
 
@@ -126,6 +126,7 @@ def lib():
         L.tsr_project_core_static.argtypes = [vp, i32, i64, i64, i64, vp, vp, i32, vp, vp]
         L.tsr_dense_adamw.argtypes = [P(DenseTensor), i32, P(Hyper), vp]
         L.tsr_set_limits.argtypes = [vp, P(Limits)]
+        L.tsr_refresh_gram.argtypes = [vp, i32, i32, vp, vp, vp]
         _lib = L
     return _lib
 
@@ -351,6 +352,17 @@ class Plan:
                    projection_launches: int = 0):
         lim = Limits(wait_clocks, max_sweeps, sweep_block, starve_block, projection_launches)
         self._check(lib().tsr_set_limits(self.ctx, ctypes.byref(lim)))
+
+    def refresh_gram(self, i: int, side: int, X: torch.Tensor, stream=None) -> torch.Tensor:
+        """S = X^T X (FP64, k x k) through the Gram kernels the refresh of block i uses; X is FP32, rows x k with
+        rows = m (side 0) or n (side 1).  Overwrites the block's refresh work buffers."""
+        b = self.blocks[i]
+        rows, k = int(_field(b, "n") if side else _field(b, "m")), int(_field(b, "r")) + int(_field(b, "p", 0))
+        if X.dtype != torch.float32 or tuple(X.shape) != (rows, k) or not X.is_contiguous() or not X.is_cuda:
+            raise ValueError("X must be a contiguous CUDA FP32 tensor of shape (%d, %d)" % (rows, k))
+        S = torch.empty(k, k, dtype=torch.float64, device=X.device)
+        self._check(lib().tsr_refresh_gram(self.ctx, i, side, X.data_ptr(), S.data_ptr(), _stream_ptr(stream)))
+        return S
 
     def set_profiling(self, enable: bool):
         self._check(lib().tsr_set_profiling(self.ctx, 1 if enable else 0))

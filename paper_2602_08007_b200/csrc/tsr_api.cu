@@ -1701,6 +1701,41 @@ tsr_status tsr_generate_omega(tsr_ctx *ctx, int32_t i, uint64_t seed, float *out
     return TSR_OK;
 }
 
+tsr_status tsr_refresh_gram(tsr_ctx *ctx, int32_t block, int32_t side, const float *X, double *S, void *stream)
+{
+    tsr_status s = check_ready(ctx);
+    if (s != TSR_OK) return s;
+    if (block < 0 || block >= (int)ctx->blocks.size() || (side != 0 && side != 1) || !X || !S)
+        return fail(ctx, TSR_ERR_INVALID_ARG, "tsr_refresh_gram: bad argument");
+    cudaStream_t st = (cudaStream_t)stream;
+    Block &b = ctx->blocks[block];
+    const int rows = (int)(side ? b.d.n : b.d.m);
+    // the device tables of the refresh are rewritten for this one block: a cached refresh is no longer valid
+    ctx->refresh_sig.clear();
+    RefreshLists L;
+    L.list = {block};
+    L.dlist = ctx->d_rlist;
+    for (int i = 0; i < 5; ++i) L.ditems[i] = ctx->d_items[i];
+    L.kmax = b.k; L.rmax = (int)b.d.r;
+    std::vector<RowItem> items[4];
+    for (int sd = 0; sd < 2; ++sd) {
+        const int rr = (int)(sd ? b.d.n : b.d.m);
+        for (int r0 = 0; r0 < rr; r0 += RG_ROWS) items[sd * 2].push_back({block, r0});
+        for (int r0 = 0; r0 < rr; r0 += GRAM_ROWS) items[sd * 2 + 1].push_back({block, r0});
+    }
+    if ((s = upload_list(ctx, L.dlist, L.list, st)) != TSR_OK) return s;
+    for (int i = 0; i < 4; ++i) {
+        TSR_CUDA(ctx, cudaMemcpyAsync(L.ditems[i], items[i].data(), items[i].size() * sizeof(RowItem), cudaMemcpyHostToDevice, st));
+        L.nitems[i] = (int)items[i].size();
+    }
+    TSR_CUDA(ctx, cudaMemcpyAsync(b.buf[0], X, (size_t)rows * b.k * sizeof(float), cudaMemcpyDeviceToDevice, st));
+    if ((s = gram(ctx, L, side, 0, st)) != TSR_OK) return s;
+    TSR_CUDA(ctx, cudaMemcpyAsync(S, b.S, (size_t)b.k * b.k * sizeof(double), cudaMemcpyDeviceToDevice, st));
+    // the host vectors above feed asynchronous copies from pageable memory, which the runtime stages before it
+    // returns, so they may go out of scope here
+    return TSR_OK;
+}
+
 tsr_status tsr_set_limits(tsr_ctx *ctx, const tsr_limits *lim)
 {
     if (!ctx) return TSR_ERR_INVALID_ARG;

@@ -357,3 +357,60 @@ def test_optional_moment_reexpression_at_refresh(dtype):
     assert rel_fro(to64(plan.M[0]), Mo[0]) > 1e-2            # it did change
     assert torch.equal(plan.Vm[0], Vm_before)                # the second moment is never re-expressed
     assert np.array_equal(to64(plan.M[1]), Mo[1])            # unflagged block: Algorithm 1 as printed
+
+
+def _gram_reference(X):
+    """X^T X of an FP32 matrix in extended precision (the products of FP32 numbers are exact in it and the sums carry
+    64 bits), returned as FP64."""
+    Xl = X.astype(np.longdouble)
+    return (Xl.T @ Xl).astype(np.float64)
+
+
+@pytest.mark.parametrize("shape,side", [
+    (dict(m=700, n=520, r=64, p=8), 0),        # integer tensor-core form (k = 72 <= min / 2), ragged rows, one 2048-row chunk
+    (dict(m=700, n=520, r=64, p=8), 1),
+    (dict(m=4500, n=600, r=264, p=8), 0),      # k = 272: several 64-column tiles, tiles off the diagonal, three row chunks
+    (dict(m=300, n=260, r=128, p=8), 0),       # k = 136 > min / 2: the FP64 tensor path
+])
+def test_gram_step_of_the_refresh_against_its_definition(shape, side):
+    """S = X^T X as the refresh computes it, against the definition evaluated in extended precision, on columns whose
+    scales span forty binary orders of magnitude, with a zero column, exact powers of two and entries that are tiny
+    next to their column's largest.  The integer form cuts every column, scaled by a power of two to |y| <= 1/2, into
+    six signed 7-bit digits (42 bits below the column's largest entry) and keeps the digit products down to 2^-42:
+    per entry of S the error is bounded by rows * 2^-41 * 2^(e_i + e_j), e_j the exponent of column j's largest
+    entry (what the digits and the digit products below 2^-42 leave out, all with the same sign), and comes to about
+    5e-12 of |x_i| |x_j| for columns without outliers (gated at 2e-11: a level of digit products from the fifth up that
+    went missing or landed in the wrong accumulator would show as 1e-9 and more).  The result must also be symmetric bit for bit
+    and the same on a second call."""
+    tsr = _tsr()
+    plan = tsr.Plan([shape], g_dtype=torch.bfloat16)
+    rows = shape["n"] if side else shape["m"]
+    k = shape["r"] + shape["p"]
+    rng = np.random.default_rng(77 + rows + k)
+    X = rng.standard_normal((rows, k)).astype(np.float32)
+    X *= np.exp2(rng.integers(-20, 21, size=k)).astype(np.float32)[None, :]      # column scales 2^-20 .. 2^20
+    X[:, 3] = 0.0                                                                 # a zero column
+    X[:, 5] = np.exp2(rng.integers(-3, 4, size=rows)).astype(np.float32)          # exact powers of two
+    X[1:, 7] *= np.float32(2.0 ** -30)                                            # one entry dwarfs the rest of its column
+    X[rows // 2, 9] = np.float32(0.5) * np.abs(X[:, 9]).max()                     # a tie in the column maximum's binade
+    Xd = torch.from_numpy(X).cuda()
+    S1 = plan.refresh_gram(0, side, Xd)
+    S2 = plan.refresh_gram(0, side, Xd)
+    torch.cuda.synchronize()
+    assert plan.poll_status() == [0]
+    S = S1.cpu().numpy()
+    assert torch.equal(S1, S2)
+    assert np.array_equal(S, S.T)
+    ref = _gram_reference(X)
+    cmax = np.abs(X).max(axis=0).astype(np.float64)
+    e = np.where(cmax > 0, np.ceil(np.log2(np.maximum(cmax, 1e-300))) + 1, 0.0)   # cmax <= 2^(e - 1)
+    bound = rows * 2.0 ** -41 * np.exp2(e[:, None] + e[None, :])
+    err = np.abs(S - ref)
+    assert np.all(err <= bound), float((err / bound).max())
+    assert np.all(S[3, :] == 0) and np.all(S[:, 3] == 0)
+    norms = np.sqrt(np.diag(ref))
+    rel = err / np.maximum(norms[:, None] * norms[None, :], 1e-300)
+    well = np.ones(k, bool); well[[3, 7]] = False                                 # columns without an outlier entry
+    print("Gram against its definition: worst error %.1e of |x_i||x_j| (columns without outliers), %.2f of the bound"
+          % (rel[np.ix_(well, well)].max(), (err / bound).max()))
+    assert rel[np.ix_(well, well)].max() < 2e-11
