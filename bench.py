@@ -537,7 +537,7 @@ def run_ours(args, w: ti.Workload):
                          % (traffic["captured_on"], traffic["commit"]),
                          "algorithmic_bytes": work["apply_kernel_bytes"],
                          "peak_source": peaks["source"] + " copy bandwidth", "ms": apply_ms, "roof_ms": apply_roof_ms},
-            "roofline_projection": {"kernels": "umma_gemm_kernel<EPI_RUNTIME>: T~ = (G V)^T tiles and core tiles C = U^T T (+ Adam) in one launch"
+            "roofline_projection": {"kernels": "umma_gemm_kernel<EPI_RUNTIME>: tiles of the first contraction (T~ = (G V)^T, or T = U^T G where m > n) and core tiles (+ Adam) in one launch"
                                     if st_med[2] < 0.1 * st_med[1] else "umma_gemm_kernel<EPI_STORE_BF16_T> + <EPI_CORE_UPDATE>",
                                     "bound": "tensor" if work["proj_flops"] / (tc * 1e12) > work["proj_bytes"] / (hbm * 1e9) else "hbm",
                                     "achieved_tflops": proj_tflops, "ms": proj_ms, "roof_ms": proj_roof_ms,

@@ -263,10 +263,11 @@ TSR_API tsr_status tsr_generate_omega(tsr_ctx *ctx, int32_t i, uint64_t seed, fl
 /* Stage timing of tsr_step_grouped for profiling (off by default).  When enabled, every
  * tsr_step_grouped / tsr_embed_step records CUDA events at its stage boundaries on the step's
  * stream; tsr_get_stage_ms waits for the last recorded step and returns, in milliseconds,
- * ms[0] refresh (0 when none was due), ms[1] the projection launch (a step over all blocks runs
- * T = G V and the core GEMM C = U^T T with its fused core update as ONE launch; a step over a
- * partial block list runs T = G V here), ms[2] what follows it (the core GEMM of a partial list;
- * the split-K reduction of tall blocks), ms[3] stand-alone core update (unfused order only),
+ * ms[0] refresh (0 when none was due), ms[1] the projection launch (a step over all blocks may
+ * run the first contraction -- T = G V, or T = U^T G for a block with m > n -- and the core GEMM
+ * with its fused core update as ONE launch; otherwise the first contraction runs here),
+ * ms[2] what follows it (the core GEMM when it is a launch of its own; the split-K reduction of
+ * tall blocks), ms[3] stand-alone core update (unfused order only),
  * ms[4] P = U D, ms[5] the apply kernel W <- decay W - step_scale P V^T.  count must be 6.
  * Enabling creates the events (a small driver allocation); disabling destroys them. */
 TSR_API tsr_status tsr_set_profiling(tsr_ctx *ctx, int32_t enable);
@@ -284,7 +285,7 @@ TSR_API tsr_status tsr_get_stage_ms(tsr_ctx *ctx, float *ms, int32_t count);
  *                 QL iterations per eigenvalue above; defaults 40 / 60) for block sweep_block
  *                 (-1: every block).  A solver that stops at the limit flags
  *                 TSR_ERR_NOT_CONVERGED on that block; other blocks are not affected.
- *   starve_block  -1 (off), or a block index: the first projection GEMM (T = G V) issues no
+ *   starve_block  -1 (off), or a block index: the first projection GEMM (T = G V or U^T G) issues no
  *                 loads for the tiles of that block, so that its consumers run into the bounded
  *                 wait.  Nothing is in flight and no address is touched for those tiles.  It
  *                 exists to exercise the time-out path and requires 0 < wait_clocks <= 1e8.

@@ -34,6 +34,8 @@ struct Block {
     bf16 *Db = nullptr, *Dbt = nullptr;
     bool one_sided = false;   // C = U^T G (r x n): the comparison arm of Table 1
     bool right_first = false; // the lift goes through Z^T = V D^T (n x r) instead of P = U D (m x r): the smaller intermediate
+    bool proj_right = false;  // the projection goes through T = U^T G (r x n) instead of T~ = (G V)^T (r x m): m > n and m short
+                              // enough for one pass over it (Section 3.3: the intermediate whose long side is min(m, n))
     int64_t cn = 0;           // columns of C, M, Vm: r, or n for a one-sided block
     float *partial = nullptr;
     int nsplit = 1, kb_per_split = 0;
@@ -335,7 +337,7 @@ void build_merged(tsr_ctx *ctx)
     auto emit_core = [&](const Pending &pd) {
         const Block &b = ctx->blocks[pd.bi];
         const size_t first = v.size();
-        gen_tiles(v, pd.bi, b.d.r, b.d.r, (int)b.d.m, b.nsplit > 1 ? b.kb_per_split : 0, ctx->bn[KCM], false, 0);
+        gen_tiles(v, pd.bi, b.d.r, b.d.r, (int)(b.proj_right ? b.d.n : b.d.m), b.nsplit > 1 ? b.kb_per_split : 0, ctx->bn[KCM], false, 0);
         for (size_t i = first; i < v.size(); ++i) {
             v[i].kind = 1;
             v[i].wait_slot = pd.bi;
@@ -346,7 +348,8 @@ void build_merged(tsr_ctx *ctx)
         const Block &b = ctx->blocks[bi];
         if (!b.fast || b.one_sided) continue;
         const size_t first = v.size();
-        gen_tiles(v, bi, (int)b.d.m, b.d.r, (int)b.d.n, 0, ctx->bn[KT], false, 0);
+        if (b.proj_right) gen_tiles(v, bi, b.d.r, (int)b.d.n, (int)b.d.m, 0, ctx->bn[KT], false, 0);
+        else gen_tiles(v, bi, (int)b.d.m, b.d.r, (int)b.d.n, 0, ctx->bn[KT], false, 0);
         for (size_t i = first; i < v.size(); ++i) { v[i].kind = 0; v[i].signal_slot = bi; }
         pending.push_back({bi, v.size(), (int)(v.size() - first)});
         while (head < pending.size() && v.size() >= pending[head].t_end + MERGE_GAP) emit_core(pending[head++]);
@@ -380,10 +383,11 @@ void build_tiles(tsr_ctx *ctx)
             add_tiles(ctx, KO, bi, r, n, m, 0);
             add_tiles(ctx, KOA, bi, m, n, r, 0);
         } else {
-            add_tiles(ctx, KT, bi, m, r, n, 0);
+            if (b.proj_right) add_tiles(ctx, KT, bi, r, n, m, 0);      // T = U^T G
+            else add_tiles(ctx, KT, bi, m, r, n, 0);                   // T~ = (G V)^T
             // a block with a long contraction (an embedding) is cut into split-K slabs; its tiles sit in the same
             // table, so that one launch covers every block
-            add_tiles(ctx, KC, bi, r, r, m, b.nsplit > 1 ? b.kb_per_split : 0);
+            add_tiles(ctx, KC, bi, r, r, b.proj_right ? n : m, b.nsplit > 1 ? b.kb_per_split : 0);
             add_tiles(ctx, KP, bi, b.right_first ? n : m, r, r, 0);
             add_tiles(ctx, KA, bi, m, n, r, 0);
         }
@@ -1145,6 +1149,8 @@ tsr_status tsr_create(tsr_ctx **out, const tsr_mat_desc *descs, int32_t count)
         b.tc_rows = b.fast && (b.k % 4 == 0);   // FP32 rows of k elements as a TMA operand: 16-byte row pitch
         const int nkb = (int)((b.d.m + 63) / 64);
         if (nkb > 128 && !b.one_sided) { b.kb_per_split = 32; b.nsplit = (nkb + 31) / 32; }
+        // (an embedding-like block, whose m is a single long contraction for U^T G, keeps T~ = (G V)^T and the split-K core)
+        b.proj_right = b.right_first && nkb <= 128;
         ctx->max_r = std::max(ctx->max_r, (int)b.d.r);
         ctx->max_k = std::max(ctx->max_k, b.k);
         ctx->order.push_back(i);
@@ -1249,7 +1255,7 @@ tsr_status tsr_bind(tsr_ctx *ctx, const tsr_mat_ptrs *ptrs, int32_t count, void 
     {   // bytes of the intermediate T~ (BF16, r x m) over the blocks that go through the merged projection launch
         size_t tt = 0;
         for (const Block &b : ctx->blocks)
-            if (b.fast && !b.one_sided) tt += (size_t)b.d.r * (size_t)b.ml * 2;
+            if (b.fast && !b.one_sided) tt += (size_t)b.d.r * (size_t)(b.proj_right ? b.nl : b.ml) * 2;
         ctx->merge_pays = ctx->l2_bytes > 0 && tt > 2 * ctx->l2_bytes;
     }
 
@@ -1304,7 +1310,15 @@ tsr_status tsr_bind(tsr_ctx *ctx, const tsr_mat_ptrs *ptrs, int32_t count, void 
                 P.out = b.p.W; P.ld_out = b.d.ldw;
             }
         }
-        {   // T~ = (G V)^T : A = G [m x n], B = V^T copy [r x n]
+        if (b.proj_right) {   // T = U^T G : A = U^T copy [r x m], B = G itself, [m x n] contracted over its rows (MN-major)
+            UmmaProblem &P = probs[KT][i];
+            base(P, (int)r, (int)n, (int)m, EPI_STORE_BF16);
+            if ((s = encode_map(ctx, &P.tmA, b.Ubt, r, m, b.ml, 128)) != TSR_OK) return s;
+            if ((s = encode_map(ctx, &P.tmB, b.p.G, m, n, b.d.ldg, 64)) != TSR_OK) return s;
+            P.b_mn = 1;
+            P.out = b.Tt; P.ld_out = b.nl;
+            P.starve = (ctx->starve_block == i) ? 1 : 0;
+        } else {   // T~ = (G V)^T : A = G [m x n], B = V^T copy [r x n]
             UmmaProblem &P = probs[KT][i];
             base(P, (int)m, (int)r, (int)n, EPI_STORE_BF16_T);
             if ((s = encode_map(ctx, &P.tmA, b.p.G, m, n, b.d.ldg, 128)) != TSR_OK) return s;
@@ -1315,9 +1329,15 @@ tsr_status tsr_bind(tsr_ctx *ctx, const tsr_mat_ptrs *ptrs, int32_t count, void 
         {   // C = U^T T : A = U^T copy [r x m], B = T~ [r x m].  A split-K block only stores its slabs
             // (the sum and the core update follow in core_update_kernel), whatever epilogue the launch has.
             UmmaProblem &P = probs[KC][i];
-            base(P, (int)r, (int)r, (int)m, b.nsplit > 1 ? EPI_STORE_F32 : EPI_CORE_UPDATE);
-            if ((s = encode_map(ctx, &P.tmA, b.Ubt, r, m, b.ml, 128)) != TSR_OK) return s;
-            if ((s = encode_map(ctx, &P.tmB, b.Tt, r, m, b.ml, ctx->bn[KC] / 2)) != TSR_OK) return s;
+            if (b.proj_right) {   // C = T V : A = T [r x n], B = V^T copy [r x n]
+                base(P, (int)r, (int)r, (int)n, EPI_CORE_UPDATE);
+                if ((s = encode_map(ctx, &P.tmA, b.Tt, r, n, b.nl, 128)) != TSR_OK) return s;
+                if ((s = encode_map(ctx, &P.tmB, b.Vbt, r, n, b.nl, ctx->bn[KC] / 2)) != TSR_OK) return s;
+            } else {
+                base(P, (int)r, (int)r, (int)m, b.nsplit > 1 ? EPI_STORE_F32 : EPI_CORE_UPDATE);
+                if ((s = encode_map(ctx, &P.tmA, b.Ubt, r, m, b.ml, 128)) != TSR_OK) return s;
+                if ((s = encode_map(ctx, &P.tmB, b.Tt, r, m, b.ml, ctx->bn[KC] / 2)) != TSR_OK) return s;
+            }
             P.out = (b.nsplit > 1) ? (void *)b.partial : (void *)b.p.C;
             P.ld_out = r; P.split_stride = r * r;
             P.mom1 = b.p.M; P.mom2 = b.p.Vm; P.d_bf16 = b.right_first ? b.Db : nullptr; P.dt_bf16 = b.Dbt; P.ldd = b.rl;
@@ -1325,7 +1345,8 @@ tsr_status tsr_bind(tsr_ctx *ctx, const tsr_mat_ptrs *ptrs, int32_t count, void 
         {   // the same core problem for the merged projection launch: B boxes as wide as that launch's tiles
             UmmaProblem &P = probs[KCM][i];
             P = probs[KC][i];
-            if ((s = encode_map(ctx, &P.tmB, b.Tt, r, m, b.ml, ctx->bn[KCM] / 2)) != TSR_OK) return s;
+            if (b.proj_right) { if ((s = encode_map(ctx, &P.tmB, b.Vbt, r, n, b.nl, ctx->bn[KCM] / 2)) != TSR_OK) return s; }
+            else if ((s = encode_map(ctx, &P.tmB, b.Tt, r, m, b.ml, ctx->bn[KCM] / 2)) != TSR_OK) return s;
         }
         // The lift U D V^T goes through the smaller of the two intermediates: P = U D (m x r) when m <= n,
         // Z^T = V D^T (n x r) when m > n; either one lives in Pb and is the apply kernel's A or B operand.

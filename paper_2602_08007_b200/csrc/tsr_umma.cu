@@ -192,10 +192,17 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
                     for (int pl = 0; pl < SM::A_PLANES; ++pl)
                         tma_load_2d_pair(smem_u32(st + pl * SM::A_BYTES), &P->tmA, full, kb * SM::BK_ELEMS,
                                          tile.m0 + (int)rank * UM_BM + pl * P->a_plane_rows);
+                    if (PLANES == 1 && P->b_mn) {
+                        // B = a row-major [K x N] matrix: boxes of 64 columns x 64 rows, this CTA's half of the columns
 #pragma unroll
-                    for (int pl = 0; pl < SM::B_PLANES; ++pl)
-                        tma_load_2d_pair(smem_u32(st + SM::A_PLANES * SM::A_BYTES + pl * SM::B_BYTES), &P->tmB, full,
-                                         kb * SM::BK_ELEMS, b_row + pl * P->plane_rows);
+                        for (int j = 0; j < BN / 128; ++j)
+                            tma_load_2d_pair(smem_u32(st + SM::A_BYTES + j * 8192), &P->tmB, full, b_row + 64 * j, kb * SM::BK_ELEMS);
+                    } else {
+#pragma unroll
+                        for (int pl = 0; pl < SM::B_PLANES; ++pl)
+                            tma_load_2d_pair(smem_u32(st + SM::A_PLANES * SM::A_BYTES + pl * SM::B_BYTES), &P->tmB, full,
+                                             kb * SM::BK_ELEMS, b_row + pl * P->plane_rows);
+                    }
                 }
             }
         }
@@ -208,9 +215,11 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
                 if (!next_tile(tc, t, true)) { note_timeout(&s_timeout, 0x7ffffffe); break; }
                 if (t < 0) break;
                 const UmmaTile tile = tiles[t];
-                int n_eff = (((EPI == EPI_RUNTIME && tile.kind) ? probs2 : probs) + tile.prob)->N - tile.n0;
+                const UmmaProblem *Pm = ((EPI == EPI_RUNTIME && tile.kind) ? probs2 : probs) + tile.prob;
+                int n_eff = Pm->N - tile.n0;
                 n_eff = tile.nw > 0 ? tile.nw : (n_eff >= BN ? BN : ((n_eff + 15) & ~15));
-                const uint32_t idesc = PLANES == 3 ? umma_idesc_pair_tf32(n_eff) : umma_idesc_pair(n_eff);
+                const bool b_mn = PLANES == 1 && Pm->b_mn;
+                const uint32_t idesc = PLANES == 3 ? umma_idesc_pair_tf32(n_eff) : (umma_idesc_pair(n_eff) | (b_mn ? UMMA_IDESC_B_MN_MAJOR : 0u));
                 const uint32_t buf = tc & 1u;
                 if (!mbar_wait(smem_u32(bar_acc_empty + buf), ((tc >> 1) & 1u) ^ 1u, budget)) { note_timeout(&s_timeout, t); ok = false; break; }
                 tc_fence_after();
@@ -238,7 +247,8 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
                             const uint32_t b_base = a_base + SM::A_BYTES + pl * SM::B_BYTES;
 #pragma unroll
                             for (int k4 = 0; k4 < UM_BK / 16; ++k4)
-                                tc_mma_bf16_pair(d_tmem, umma_desc_sw128(a_base + k4 * 32), umma_desc_sw128(b_base + k4 * 32),
+                                tc_mma_bf16_pair(d_tmem, umma_desc_sw128(a_base + k4 * 32),
+                                                 b_mn ? umma_desc_sw128_mn(b_base + k4 * 2048, 8192) : umma_desc_sw128(b_base + k4 * 32),
                                                  idesc, ((kb - tile.kb0) | pl | k4) ? 1u : 0u);
                         }
                     }
@@ -263,8 +273,10 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
             const UmmaTile tile = tiles[t];
             const UmmaProblem *__restrict__ P = ((EPI == EPI_RUNTIME && tile.kind) ? probs2 : probs) + tile.prob;
             // the tile's epilogue: fixed by the instantiation, or (merged projection launch) by the tile's kind
-            const int epi = (EPI != EPI_RUNTIME) ? EPI
-                            : (tile.kind == 0 ? (int)EPI_STORE_BF16_T : (fuse ? P->epilogue : (int)EPI_STORE_F32));
+            // (a problem of the first contraction stores T~ transposed, or -- where it forms T = U^T G -- as it comes)
+            const int epi = (EPI == EPI_STORE_BF16_T) ? P->epilogue
+                            : (EPI != EPI_RUNTIME) ? EPI
+                            : (tile.kind == 0 ? P->epilogue : (fuse ? P->epilogue : (int)EPI_STORE_F32));
             const uint32_t buf = tc & 1u;
             const int N = P->N, M = P->M;
             const int Nt = tile.nw > 0 ? min(N, tile.n0 + tile.nw) : N;   // first column past this tile

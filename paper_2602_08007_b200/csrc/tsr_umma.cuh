@@ -245,6 +245,20 @@ __device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t saddr)
     d |= (uint64_t)2 << 61;
     return d;
 }
+// The same for an MN-major operand: a [K x N] tile with N contiguous, written by TMA as boxes of 64 columns x 64 rows
+// with the 128-byte swizzle.  A swizzle atom is 8 rows (K) of 128 bytes (64 columns); atoms follow one another every
+// 1024 bytes along K (stride byte offset) and every `lbo` bytes -- one box -- along N (leading byte offset).
+__device__ __forceinline__ uint64_t umma_desc_sw128_mn(uint32_t saddr, uint32_t lbo)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr >> 4) & 0x3FFF);
+    d |= (uint64_t)((lbo >> 4) & 0x3FFF) << 16;
+    d |= (uint64_t)(1024 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+constexpr uint32_t UMMA_IDESC_B_MN_MAJOR = 1u << 16;    // instruction descriptor: B operand MN-major
 // Instruction descriptor: FP32 accumulator, BF16 x BF16, both K-major, M = 128, N = BN.
 __host__ __device__ constexpr uint32_t umma_idesc(int bn)
 {
