@@ -41,7 +41,7 @@ struct Block {
     int nsplit = 1, kb_per_split = 0;
     float *T32 = nullptr, *P32 = nullptr, *D32 = nullptr;
     // refresh scratch
-    bf16 *Gt = nullptr, *Xt = nullptr;
+    bf16 *Xt = nullptr;
     float *Om = nullptr;
     float *buf[3] = {nullptr, nullptr, nullptr};
     double *S = nullptr, *Xw = nullptr, *Wj = nullptr, *gpart = nullptr, *lam = nullptr;
@@ -232,9 +232,8 @@ void layout(tsr_ctx *ctx, Arena &a, bool assign, size_t *step_end)
         const int64_t m = b.d.m, n = b.d.n, r = b.d.r, k = b.k;
         const int64_t mx = std::max(m, n);
         if (b.fast) {
-            void *gt = a.take((size_t)(n * b.ml) * 2);
             void *xt = a.take((size_t)(2 * k * std::max(b.ml, b.nl)) * 2);
-            if (assign) { b.Gt = (bf16 *)gt; b.Xt = (bf16 *)xt; }
+            if (assign) b.Xt = (bf16 *)xt;
         }
         if (b.tc_rows) {
             void *xs = a.take((size_t)(2 * mx * k) * 4), *bts = a.take((size_t)(2 * k * k) * 4);
@@ -649,13 +648,11 @@ tsr_status do_project(tsr_ctx *ctx, const std::vector<int> &list, bool fuse, con
         if (!merged && (s = launch_kind(ctx, KT, list, EPI_STORE_BF16_T, 1, sc, st)) != TSR_OK) return s;
         mark_stage(ctx, 2);
         if (!merged && (s = launch_kind(ctx, KC, list, fuse ? EPI_CORE_UPDATE : EPI_STORE_F32, 1, sc, st)) != TSR_OK) return s;
-        // one-sided blocks: C = U^T G needs the gradient with m as the contiguous index
+        // one-sided blocks: C = U^T G contracts the gradient over its rows (read MN-major, no transposed copy)
         bool any_one_sided = false;
         for (int bi : list) {
             const Block &b = ctx->blocks[bi];
-            if (!b.fast || !b.one_sided) continue;
-            TSR_KERNEL(ctx, 1, transpose_bf16((const bf16 *)b.p.G, (int)b.d.m, (int)b.d.n, b.d.ldg, b.Gt, b.ml, st));
-            any_one_sided = true;
+            if (b.fast && b.one_sided) any_one_sided = true;
         }
         if (any_one_sided && (s = launch_kind(ctx, KO, list, fuse ? EPI_CORE_UPDATE : EPI_STORE_F32, 1, sc, st)) != TSR_OK) return s;
     }
@@ -914,8 +911,6 @@ tsr_status do_refresh_group(tsr_ctx *ctx, const std::vector<int> &list, uint64_t
             TSR_CUDA(ctx, cudaMemcpyAsync(b.Om, omegas[j], (size_t)b.d.n * b.k * sizeof(float), cudaMemcpyDeviceToDevice, st));
         else
             TSR_KERNEL(ctx, 1, fill_gaussian(b.Om, (int64_t)b.d.n * b.k, seed, (uint64_t)list[j], st));
-        if (b.fast)
-            TSR_KERNEL(ctx, 1, transpose_bf16((const bf16 *)b.p.G, (int)b.d.m, (int)b.d.n, b.d.ldg, b.Gt, b.ml, st));
     }
     // Y = G Omega; Q = orth(Y)
     if ((s = sketch(ctx, L, false, true, omegas, st, 1)) != TSR_OK) return s;
@@ -1293,11 +1288,12 @@ tsr_status tsr_bind(tsr_ctx *ctx, const tsr_mat_ptrs *ptrs, int32_t count, void 
             P.M = M; P.N = N; P.K = K; P.planes = 1; P.plane_rows = 0; P.block = i; P.epilogue = epi;
         };
         if (b.one_sided) {
-            {   // C = U^T G (+ core update) : A = U^T copy [r x m], B = G^T copy [n x m]
+            {   // C = U^T G (+ core update) : A = U^T copy [r x m], B = G itself, contracted over its rows (MN-major)
                 UmmaProblem &P = probs[KO][i];
                 base(P, (int)r, (int)n, (int)m, EPI_CORE_UPDATE);
                 if ((s = encode_map(ctx, &P.tmA, b.Ubt, r, m, b.ml, 128)) != TSR_OK) return s;
-                if ((s = encode_map(ctx, &P.tmB, b.Gt, n, m, b.ml, ctx->bn[KO] / 2)) != TSR_OK) return s;
+                if ((s = encode_map(ctx, &P.tmB, b.p.G, m, n, b.d.ldg, 64)) != TSR_OK) return s;
+                P.b_mn = 1;
                 P.out = b.p.C; P.ld_out = n; P.split_stride = 0;
                 P.mom1 = b.p.M; P.mom2 = b.p.Vm; P.d_bf16 = nullptr; P.dt_bf16 = b.Dbt; P.ldd = b.rl;
             }
@@ -1383,11 +1379,12 @@ tsr_status tsr_bind(tsr_ctx *ctx, const tsr_mat_ptrs *ptrs, int32_t count, void 
             if ((s = encode_map(ctx, &P.tmB, b.Xt, 2 * k, n, b.nl, ctx->bn[KY] / 2)) != TSR_OK) return s;
             P.out = b.buf[0]; P.ld_out = k;
         }
-        {   // Z = G^T X : A = G^T copy [n x m], B = X^T planes [2k x m]
+        {   // Z = G^T X : A = G itself, contracted over its rows (MN-major), B = X^T planes [2k x m]
             UmmaProblem &P = probs[KZ][i];
             base(P, (int)n, (int)k, (int)m, EPI_STORE_F32);
             P.planes = 2; P.plane_rows = (int)k;
-            if ((s = encode_map(ctx, &P.tmA, b.Gt, n, m, b.ml, 128)) != TSR_OK) return s;
+            if ((s = encode_map(ctx, &P.tmA, b.p.G, m, n, b.d.ldg, 64)) != TSR_OK) return s;
+            P.a_mn = 1;
             if ((s = encode_map(ctx, &P.tmB, b.Xt, 2 * k, m, b.ml, ctx->bn[KZ] / 2)) != TSR_OK) return s;
             P.out = b.buf[0]; P.ld_out = k;
         }

@@ -54,6 +54,7 @@ struct alignas(64) UmmaProblem {
     int32_t out_tma;       // EPI_STORE_BF16: tmW describes the output, chunks leave through TMA stores
     const int32_t *col_exp; // integer Gram kernel: the column exponents of the matrix whose digit planes tmA / tmB describe
     int32_t starve;        // diagnostic (tsr_set_limits): the producer issues no loads for this problem's tiles
+    int32_t a_mn;          // A is given as [K x M] with M contiguous (the same form for the other operand: G^T X reads G itself)
     int32_t b_mn;          // B is given as [K x N] with N contiguous (a row-major matrix contracted over its rows): tmB has
                            // boxes of 64 columns (N) x 64 rows (K), and the MMA reads the operand MN-major
 };

@@ -188,10 +188,17 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
                     const uint32_t full = leader_addr(smem_u32(bar_full + s));
                     if (rank == 0) mbar_expect_tx(smem_u32(bar_full + s), 2u * (uint32_t)SM::STAGE_BYTES);
                     uint8_t *st = smem + s * SM::STAGE_BYTES;
+                    if (PLANES != 3 && P->a_mn) {
+                        // A = a row-major [K x M] matrix: two boxes of 64 columns x 64 rows, this CTA's 128 columns
 #pragma unroll
-                    for (int pl = 0; pl < SM::A_PLANES; ++pl)
-                        tma_load_2d_pair(smem_u32(st + pl * SM::A_BYTES), &P->tmA, full, kb * SM::BK_ELEMS,
-                                         tile.m0 + (int)rank * UM_BM + pl * P->a_plane_rows);
+                        for (int j = 0; j < 2; ++j)
+                            tma_load_2d_pair(smem_u32(st + j * 8192), &P->tmA, full, tile.m0 + (int)rank * UM_BM + 64 * j, kb * SM::BK_ELEMS);
+                    } else {
+#pragma unroll
+                        for (int pl = 0; pl < SM::A_PLANES; ++pl)
+                            tma_load_2d_pair(smem_u32(st + pl * SM::A_BYTES), &P->tmA, full, kb * SM::BK_ELEMS,
+                                             tile.m0 + (int)rank * UM_BM + pl * P->a_plane_rows);
+                    }
                     if (PLANES == 1 && P->b_mn) {
                         // B = a row-major [K x N] matrix: boxes of 64 columns x 64 rows, this CTA's half of the columns
 #pragma unroll
@@ -218,8 +225,9 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
                 const UmmaProblem *Pm = ((EPI == EPI_RUNTIME && tile.kind) ? probs2 : probs) + tile.prob;
                 int n_eff = Pm->N - tile.n0;
                 n_eff = tile.nw > 0 ? tile.nw : (n_eff >= BN ? BN : ((n_eff + 15) & ~15));
-                const bool b_mn = PLANES == 1 && Pm->b_mn;
-                const uint32_t idesc = PLANES == 3 ? umma_idesc_pair_tf32(n_eff) : (umma_idesc_pair(n_eff) | (b_mn ? UMMA_IDESC_B_MN_MAJOR : 0u));
+                const bool b_mn = PLANES == 1 && Pm->b_mn, a_mn = PLANES != 3 && Pm->a_mn;
+                const uint32_t idesc = PLANES == 3 ? umma_idesc_pair_tf32(n_eff)
+                                                   : (umma_idesc_pair(n_eff) | (b_mn ? UMMA_IDESC_B_MN_MAJOR : 0u) | (a_mn ? UMMA_IDESC_A_MN_MAJOR : 0u));
                 const uint32_t buf = tc & 1u;
                 if (!mbar_wait(smem_u32(bar_acc_empty + buf), ((tc >> 1) & 1u) ^ 1u, budget)) { note_timeout(&s_timeout, t); ok = false; break; }
                 tc_fence_after();
@@ -247,7 +255,7 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
                             const uint32_t b_base = a_base + SM::A_BYTES + pl * SM::B_BYTES;
 #pragma unroll
                             for (int k4 = 0; k4 < UM_BK / 16; ++k4)
-                                tc_mma_bf16_pair(d_tmem, umma_desc_sw128(a_base + k4 * 32),
+                                tc_mma_bf16_pair(d_tmem, a_mn ? umma_desc_sw128_mn(a_base + k4 * 2048, 8192) : umma_desc_sw128(a_base + k4 * 32),
                                                  b_mn ? umma_desc_sw128_mn(b_base + k4 * 2048, 8192) : umma_desc_sw128(b_base + k4 * 32),
                                                  idesc, ((kb - tile.kb0) | pl | k4) ? 1u : 0u);
                         }

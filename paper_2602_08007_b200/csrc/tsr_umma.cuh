@@ -258,6 +258,7 @@ __device__ __forceinline__ uint64_t umma_desc_sw128_mn(uint32_t saddr, uint32_t 
     d |= (uint64_t)2 << 61;
     return d;
 }
+constexpr uint32_t UMMA_IDESC_A_MN_MAJOR = 1u << 15;    // instruction descriptor: A operand MN-major
 constexpr uint32_t UMMA_IDESC_B_MN_MAJOR = 1u << 16;    // instruction descriptor: B operand MN-major
 // Instruction descriptor: FP32 accumulator, BF16 x BF16, both K-major, M = 128, N = BN.
 __host__ __device__ constexpr uint32_t umma_idesc(int bn)
