@@ -52,12 +52,16 @@ struct alignas(64) UmmaProblem {
     bf16 *dt_bf16;         // D^T [r x ldd]
     int64_t ldd;
     int32_t out_tma;       // EPI_STORE_BF16: tmW describes the output, chunks leave through TMA stores
+    int32_t a_mn;          // A is given as [K x M] with M contiguous (the same form for the other operand: G^T X reads G itself)
     const int32_t *col_exp; // integer Gram kernel: the column exponents of the matrix whose digit planes tmA / tmB describe
     int32_t starve;        // diagnostic (tsr_set_limits): the producer issues no loads for this problem's tiles
-    int32_t a_mn;          // A is given as [K x M] with M contiguous (the same form for the other operand: G^T X reads G itself)
     int32_t b_mn;          // B is given as [K x N] with N contiguous (a row-major matrix contracted over its rows): tmB has
                            // boxes of 64 columns (N) x 64 rows (K), and the MMA reads the operand MN-major
 };
+
+// 512 bytes: the three tensor maps of every entry of a problem table then start on 128-byte lines (at 576 bytes, with
+// half of the maps straddling two lines, the grouped GEMMs of a step ran a tenth slower)
+static_assert(sizeof(UmmaProblem) == 512, "UmmaProblem must stay a multiple of 128 bytes");
 
 struct UmmaTile {
     int32_t prob;

@@ -35,6 +35,7 @@
 #include "tsr_internal.h"
 #include "tsr_umma.cuh"
 #include "tsr_pdl.cuh"
+#include <type_traits>
 
 namespace tsr {
 
@@ -148,7 +149,8 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
 
     if (warp == 0) {
         if (lane == 0) {
-            uint32_t it = 0;
+            int p_stage = 0;             // stage and phase of the operand ring this thread fills next
+            uint32_t p_phase = 0;
             bool ok = true;
             for (uint32_t ti = 0; ok; ++ti) {
                 int t;
@@ -180,42 +182,53 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
                 int n_eff = P->N - tile.n0;
                 n_eff = tile.nw > 0 ? tile.nw : (n_eff >= BN ? BN : ((n_eff + 15) & ~15));
                 const int b_row = tile.n0 + (int)rank * (n_eff / 2);   // this CTA's half of the B rows
-                for (int kb = tile.kb0; kb < tile.kb1; ++kb, ++it) {
-                    const int s = it % STAGES;
-                    const uint32_t ph = (it / STAGES) & 1u;
-                    if (!mbar_wait(smem_u32(bar_empty + s), ph ^ 1u, budget)) { note_timeout(&s_timeout, t); ok = false; break; }
-                    // both CTAs' copies report their bytes to the leader's "full" barrier
-                    const uint32_t full = leader_addr(smem_u32(bar_full + s));
-                    if (rank == 0) mbar_expect_tx(smem_u32(bar_full + s), 2u * (uint32_t)SM::STAGE_BYTES);
-                    uint8_t *st = smem + s * SM::STAGE_BYTES;
-                    if (PLANES != 3 && P->a_mn) {
-                        // A = a row-major [K x M] matrix: two boxes of 64 columns x 64 rows, this CTA's 128 columns
+                // Everything the K loop needs is fetched once per tile: the loop itself is on the critical path of the
+                // pipeline (a stage is refilled the moment its MMAs retire), and every dependent global access in it --
+                // a flag of the problem record, a plane offset -- showed up as lost operand bandwidth (a tenth of the
+                // kernel's time for two flags read per K block).
+                const bool a_mn = PLANES != 3 && P->a_mn, b_mn = PLANES == 1 && P->b_mn;
+                const int a_row = tile.m0 + (int)rank * UM_BM;
+                const int a_plane_rows = P->a_plane_rows, b_plane_rows = P->plane_rows;
+                const CUtensorMap *tmA = &P->tmA, *tmB = &P->tmB;
+                auto k_loop = [&](auto mn_any) {
+                    constexpr bool MN = decltype(mn_any)::value;   // false: both operands K-major, no branch in the loop
+                    for (int kb = tile.kb0; kb < tile.kb1; ++kb) {
+                        if (!mbar_wait(smem_u32(bar_empty + p_stage), p_phase ^ 1u, budget)) { note_timeout(&s_timeout, t); ok = false; break; }
+                        // both CTAs' copies report their bytes to the leader's "full" barrier
+                        const uint32_t full = leader_addr(smem_u32(bar_full + p_stage));
+                        if (rank == 0) mbar_expect_tx(smem_u32(bar_full + p_stage), 2u * (uint32_t)SM::STAGE_BYTES);
+                        const uint32_t st = smem_u32(smem + p_stage * SM::STAGE_BYTES);
+                        const int kx = kb * SM::BK_ELEMS;
+                        if (MN && a_mn) {
+                            // A = a row-major [K x M] matrix: two boxes of 64 columns x 64 rows, this CTA's 128 columns
 #pragma unroll
-                        for (int j = 0; j < 2; ++j)
-                            tma_load_2d_pair(smem_u32(st + j * 8192), &P->tmA, full, tile.m0 + (int)rank * UM_BM + 64 * j, kb * SM::BK_ELEMS);
-                    } else {
+                            for (int j = 0; j < 2; ++j) tma_load_2d_pair(st + j * 8192, tmA, full, a_row + 64 * j, kx);
+                        } else {
 #pragma unroll
-                        for (int pl = 0; pl < SM::A_PLANES; ++pl)
-                            tma_load_2d_pair(smem_u32(st + pl * SM::A_BYTES), &P->tmA, full, kb * SM::BK_ELEMS,
-                                             tile.m0 + (int)rank * UM_BM + pl * P->a_plane_rows);
+                            for (int pl = 0; pl < SM::A_PLANES; ++pl)
+                                tma_load_2d_pair(st + pl * SM::A_BYTES, tmA, full, kx, a_row + pl * a_plane_rows);
+                        }
+                        if (MN && b_mn) {
+                            // B = a row-major [K x N] matrix: boxes of 64 columns x 64 rows, this CTA's half of the columns
+#pragma unroll
+                            for (int j = 0; j < BN / 128; ++j) tma_load_2d_pair(st + SM::A_BYTES + j * 8192, tmB, full, b_row + 64 * j, kx);
+                        } else {
+#pragma unroll
+                            for (int pl = 0; pl < SM::B_PLANES; ++pl)
+                                tma_load_2d_pair(st + SM::A_PLANES * SM::A_BYTES + pl * SM::B_BYTES, tmB, full, kx, b_row + pl * b_plane_rows);
+                        }
+                        if (++p_stage == STAGES) { p_stage = 0; p_phase ^= 1u; }
                     }
-                    if (PLANES == 1 && P->b_mn) {
-                        // B = a row-major [K x N] matrix: boxes of 64 columns x 64 rows, this CTA's half of the columns
-#pragma unroll
-                        for (int j = 0; j < BN / 128; ++j)
-                            tma_load_2d_pair(smem_u32(st + SM::A_BYTES + j * 8192), &P->tmB, full, b_row + 64 * j, kb * SM::BK_ELEMS);
-                    } else {
-#pragma unroll
-                        for (int pl = 0; pl < SM::B_PLANES; ++pl)
-                            tma_load_2d_pair(smem_u32(st + SM::A_PLANES * SM::A_BYTES + pl * SM::B_BYTES), &P->tmB, full,
-                                             kb * SM::BK_ELEMS, b_row + pl * P->plane_rows);
-                    }
-                }
+                };
+                if (a_mn || b_mn) k_loop(std::true_type{});
+                else k_loop(std::false_type{});
             }
         }
     } else if (warp == 1) {
         if (lane == 0 && rank == 0) {   // the leader issues the pair's MMAs (256 x N x 16 each)
-            uint32_t it = 0, tc = 0;
+            uint32_t tc = 0;
+            int c_stage = 0;             // stage and phase of the operand ring this thread consumes next
+            uint32_t c_phase = 0;
             bool ok = true;
             for (; ok; ++tc) {
                 int t;
@@ -226,16 +239,19 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
                 int n_eff = Pm->N - tile.n0;
                 n_eff = tile.nw > 0 ? tile.nw : (n_eff >= BN ? BN : ((n_eff + 15) & ~15));
                 const bool b_mn = PLANES == 1 && Pm->b_mn, a_mn = PLANES != 3 && Pm->a_mn;
+                // (the operand forms are fixed per tile: the MMA loop below only adds addresses)
+                const uint64_t a_hi = a_mn ? UMMA_DESC_HI_MN : UMMA_DESC_HI_K, b_hi = b_mn ? UMMA_DESC_HI_MN : UMMA_DESC_HI_K;
+                const uint32_t a_step = a_mn ? 2048u : 32u, b_step = b_mn ? 2048u : 32u;
                 const uint32_t idesc = PLANES == 3 ? umma_idesc_pair_tf32(n_eff)
                                                    : (umma_idesc_pair(n_eff) | (b_mn ? UMMA_IDESC_B_MN_MAJOR : 0u) | (a_mn ? UMMA_IDESC_A_MN_MAJOR : 0u));
                 const uint32_t buf = tc & 1u;
                 if (!mbar_wait(smem_u32(bar_acc_empty + buf), ((tc >> 1) & 1u) ^ 1u, budget)) { note_timeout(&s_timeout, t); ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + buf * BN;
-                for (int kb = tile.kb0; kb < tile.kb1; ++kb, ++it) {
-                    const int s = it % STAGES;
-                    const uint32_t ph = (it / STAGES) & 1u;
-                    if (!mbar_wait(smem_u32(bar_full + s), ph, budget)) { note_timeout(&s_timeout, t); ok = false; break; }
+                for (int kb = tile.kb0; kb < tile.kb1; ++kb) {
+                    const int s = c_stage;
+                    if (!mbar_wait(smem_u32(bar_full + s), c_phase, budget)) { note_timeout(&s_timeout, t); ok = false; break; }
+                    if (++c_stage == STAGES) { c_stage = 0; c_phase ^= 1u; }
                     tc_fence_after();
                     const uint32_t a_base = smem_u32(smem + s * SM::STAGE_BYTES);
                     if (PLANES == 3) {
@@ -255,8 +271,7 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
                             const uint32_t b_base = a_base + SM::A_BYTES + pl * SM::B_BYTES;
 #pragma unroll
                             for (int k4 = 0; k4 < UM_BK / 16; ++k4)
-                                tc_mma_bf16_pair(d_tmem, a_mn ? umma_desc_sw128_mn(a_base + k4 * 2048, 8192) : umma_desc_sw128(a_base + k4 * 32),
-                                                 b_mn ? umma_desc_sw128_mn(b_base + k4 * 2048, 8192) : umma_desc_sw128(b_base + k4 * 32),
+                                tc_mma_bf16_pair(d_tmem, umma_desc_at(a_hi, a_base + k4 * a_step), umma_desc_at(b_hi, b_base + k4 * b_step),
                                                  idesc, ((kb - tile.kb0) | pl | k4) ? 1u : 0u);
                         }
                     }

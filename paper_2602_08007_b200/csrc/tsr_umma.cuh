@@ -258,6 +258,11 @@ __device__ __forceinline__ uint64_t umma_desc_sw128_mn(uint32_t saddr, uint32_t 
     d |= (uint64_t)2 << 61;
     return d;
 }
+// The two descriptor forms without their address field (bits 0 .. 13 = address >> 4), and how far one MMA of K = 16 BF16
+// elements moves the address: 32 bytes inside the 128-byte rows of a K-major tile, two 8-row atoms of an MN-major one.
+constexpr uint64_t UMMA_DESC_HI_K = ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) | ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+constexpr uint64_t UMMA_DESC_HI_MN = ((uint64_t)(8192 >> 4) << 16) | ((uint64_t)(1024 >> 4) << 32) | ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+__device__ __forceinline__ uint64_t umma_desc_at(uint64_t hi, uint32_t saddr) { return hi | (uint64_t)((saddr >> 4) & 0x3FFF); }
 constexpr uint32_t UMMA_IDESC_A_MN_MAJOR = 1u << 15;    // instruction descriptor: A operand MN-major
 constexpr uint32_t UMMA_IDESC_B_MN_MAJOR = 1u << 16;    // instruction descriptor: B operand MN-major
 // Instruction descriptor: FP32 accumulator, BF16 x BF16, both K-major, M = 128, N = BN.

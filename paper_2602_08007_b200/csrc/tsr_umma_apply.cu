@@ -119,29 +119,34 @@ umma_apply_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restr
 
     if (warp == 0) {
         if (lane == 0) {
-            uint32_t it = 0;
+            int s = 0;                   // stage and phase of the operand ring this thread fills next
+            uint32_t ph = 0;
             bool ok = true;
             for (int t = blockIdx.x; t < num_tiles && ok; t += stride) {
                 const UmmaTile tile = tiles[t];
                 const UmmaProblem *P = probs + tile.prob;
                 const int nkb = (P->K + UM_BK - 1) / UM_BK;
-                for (int kb = 0; kb < nkb; ++kb, ++it) {
-                    const int s = it % AP_STAGES;
-                    const uint32_t ph = (it / AP_STAGES) & 1u;
+                const CUtensorMap *tmA = &P->tmA, *tmB = &P->tmB;
+                const int m0 = tile.m0, n0 = tile.n0;
+                // (nothing in this loop reads global memory: it is on the critical path of the operand pipeline)
+                for (int kb = 0; kb < nkb; ++kb) {
                     if (!mbar_wait(smem_u32(bar_empty + s), ph ^ 1u, budget)) { note_timeout(&s_timeout, t); ok = false; break; }
                     const uint32_t full = smem_u32(bar_full + s);
                     mbar_expect_tx(full, (uint32_t)AP_STAGE_BYTES);
-                    uint8_t *st = smem + s * AP_STAGE_BYTES;
-                    tma_load_2d(smem_u32(st), &P->tmA, full, kb * UM_BK, tile.m0);
-                    tma_load_2d(smem_u32(st + 16384), &P->tmB, full, kb * UM_BK, tile.n0);
-                    if (BN == 256) tma_load_2d(smem_u32(st + 32768), &P->tmB, full, kb * UM_BK, tile.n0 + 128);
+                    const uint32_t st = smem_u32(smem + s * AP_STAGE_BYTES);
+                    tma_load_2d(st, tmA, full, kb * UM_BK, m0);
+                    tma_load_2d(st + 16384, tmB, full, kb * UM_BK, n0);
+                    if (BN == 256) tma_load_2d(st + 32768, tmB, full, kb * UM_BK, n0 + 128);
+                    if (++s == AP_STAGES) { s = 0; ph ^= 1u; }
                 }
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {
             constexpr uint32_t idesc = umma_idesc(AP_BN);
-            uint32_t it = 0, tc = 0;
+            uint32_t tc = 0;
+            int cs = 0;                  // stage and phase of the operand ring this thread consumes next
+            uint32_t cph = 0;
             bool ok = true;
             for (int t = blockIdx.x; t < num_tiles && ok; t += stride, ++tc) {
                 const UmmaTile tile = tiles[t];
@@ -150,10 +155,10 @@ umma_apply_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restr
                 if (!mbar_wait(smem_u32(bar_acc_empty + buf), ((tc >> 1) & 1u) ^ 1u, budget)) { note_timeout(&s_timeout, t); ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + buf * AP_BN;
-                for (int kb = 0; kb < nkb; ++kb, ++it) {
-                    const int s = it % AP_STAGES;
-                    const uint32_t ph = (it / AP_STAGES) & 1u;
-                    if (!mbar_wait(smem_u32(bar_full + s), ph, budget)) { note_timeout(&s_timeout, t); ok = false; break; }
+                for (int kb = 0; kb < nkb; ++kb) {
+                    const int s = cs;
+                    if (!mbar_wait(smem_u32(bar_full + s), cph, budget)) { note_timeout(&s_timeout, t); ok = false; break; }
+                    if (++cs == AP_STAGES) { cs = 0; cph ^= 1u; }
                     tc_fence_after();
                     const uint32_t a_base = smem_u32(smem + s * AP_STAGE_BYTES);
                     const uint32_t b_base = a_base + 16384;
