@@ -241,15 +241,14 @@ gram_i8_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restrict
 
     if (warp == 0) {
         if (lane == 0) {
-            uint32_t it = 0;
+            int s = 0;                   // stage and phase of the operand ring this thread fills next
+            uint32_t ph = 0;
             bool ok = true;
             for (int t = pair; t < num_tiles && ok; t += stride) {
                 const UmmaTile tile = tiles[t];
                 const UmmaProblem *P = probs + tile.prob;
                 const int k = P->M;
-                for (int kb = tile.kb0; kb < tile.kb1; ++kb, ++it) {
-                    const int s = it % GI_STAGES;
-                    const uint32_t ph = (it / GI_STAGES) & 1u;
+                for (int kb = tile.kb0; kb < tile.kb1; ++kb, s = (s + 1 == GI_STAGES ? 0 : s + 1), ph ^= (s == 0 ? 1u : 0u)) {
                     if (!mbar_wait(smem_u32(bar_empty + s), ph ^ 1u, budget)) { note_timeout(&s_timeout, t); ok = false; break; }
                     const uint32_t full = leader_addr(smem_u32(bar_full + s));
                     if (rank == 0) mbar_expect_tx(smem_u32(bar_full + s), 2u * (uint32_t)GI_STAGE_BYTES);
@@ -270,15 +269,15 @@ gram_i8_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restrict
         }
     } else if (warp == 1) {
         if (lane == 0 && rank == 0) {
-            uint32_t it = 0, tc = 0;
+            uint32_t tc = 0;
+            int s = 0;                   // stage and phase of the operand ring this thread consumes next
+            uint32_t ph = 0;
             bool ok = true;
             for (int t = pair; t < num_tiles && ok; t += stride, ++tc) {
                 const UmmaTile tile = tiles[t];
                 if (!mbar_wait(smem_u32(bar_acc_empty), (tc & 1u) ^ 1u, budget)) { note_timeout(&s_timeout, t); ok = false; break; }
                 tc_fence_after();
-                for (int kb = tile.kb0; kb < tile.kb1; ++kb, ++it) {
-                    const int s = it % GI_STAGES;
-                    const uint32_t ph = (it / GI_STAGES) & 1u;
+                for (int kb = tile.kb0; kb < tile.kb1; ++kb, s = (s + 1 == GI_STAGES ? 0 : s + 1), ph ^= (s == 0 ? 1u : 0u)) {
                     if (!mbar_wait(smem_u32(bar_full + s), ph, budget)) { note_timeout(&s_timeout, t); ok = false; break; }
                     tc_fence_after();
                     const uint32_t a_base = smem_u32(smem + s * GI_STAGE_BYTES);
