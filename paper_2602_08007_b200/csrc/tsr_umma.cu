@@ -107,8 +107,8 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
         for (int s = 0; s < SR; ++s) sched_tile[s] = -1;
         for (int s = 0; s < STAGES; ++s) { mbar_init(smem_u32(bar_full + s), 1); mbar_init(smem_u32(bar_empty + s), 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(bar_acc_full + b), 1); mbar_init(smem_u32(bar_acc_empty + b), 2 * UG_EPI_WARPS); }
-        // readers of a slot: MMA thread + 8 epilogue warps of the leader, producer + 8 epilogue warps of the peer
-        for (int s = 0; s < SR; ++s) { mbar_init(smem_u32(bar_sfull + s), 1); mbar_init(smem_u32(bar_sempty + s), 2 * UG_EPI_WARPS + 2); }
+        // readers of a slot: MMA thread, B loader and 8 epilogue warps of the leader; both loaders and 8 epilogue warps of the peer
+        for (int s = 0; s < SR; ++s) { mbar_init(smem_u32(bar_sfull + s), 1); mbar_init(smem_u32(bar_sempty + s), 2 * UG_EPI_WARPS + 4); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {   // the same warp of both CTAs allocates the pair's tensor memory
@@ -179,17 +179,14 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
                     note_timeout(&s_timeout, t);
                     break;
                 }
-                int n_eff = P->N - tile.n0;
-                n_eff = tile.nw > 0 ? tile.nw : (n_eff >= BN ? BN : ((n_eff + 15) & ~15));
-                const int b_row = tile.n0 + (int)rank * (n_eff / 2);   // this CTA's half of the B rows
                 // Everything the K loop needs is fetched once per tile: the loop itself is on the critical path of the
                 // pipeline (a stage is refilled the moment its MMAs retire), and every dependent global access in it --
                 // a flag of the problem record, a plane offset -- showed up as lost operand bandwidth (a tenth of the
                 // kernel's time for two flags read per K block).
-                const bool a_mn = PLANES != 3 && P->a_mn, b_mn = PLANES == 1 && P->b_mn;
+                const bool a_mn = PLANES != 3 && P->a_mn;
                 const int a_row = tile.m0 + (int)rank * UM_BM;
-                const int a_plane_rows = P->a_plane_rows, b_plane_rows = P->plane_rows;
-                const CUtensorMap *tmA = &P->tmA, *tmB = &P->tmB;
+                const int a_plane_rows = P->a_plane_rows;
+                const CUtensorMap *tmA = &P->tmA;
                 auto k_loop = [&](auto mn_any) {
                     constexpr bool MN = decltype(mn_any)::value;   // false: both operands K-major, no branch in the loop
                     for (int kb = tile.kb0; kb < tile.kb1; ++kb) {
@@ -208,19 +205,58 @@ umma_gemm_kernel(const UmmaProblem *__restrict__ probs, const UmmaTile *__restri
                             for (int pl = 0; pl < SM::A_PLANES; ++pl)
                                 tma_load_2d_pair(st + pl * SM::A_BYTES, tmA, full, kx, a_row + pl * a_plane_rows);
                         }
-                        if (MN && b_mn) {
+                        if (++p_stage == STAGES) { p_stage = 0; p_phase ^= 1u; }
+                    }
+                };
+                if (a_mn) k_loop(std::true_type{});
+                else k_loop(std::false_type{});
+            }
+        }
+    } else if (warp == 2) {
+        // The B operand has a loader of its own: one thread issuing the copies of both operands was what bounded the K loop
+        // (every instruction added to it showed up in the kernel's time), and the two threads issue side by side.  It
+        // follows the tile sequence like the other readers of the ring and waits for the same "empty" barriers.
+        if (lane == 0) {
+            int p_stage = 0;
+            uint32_t p_phase = 0;
+            bool ok = true;
+            for (uint32_t ti = 0; ok; ++ti) {
+                int t;
+                if (!next_tile(ti, t, true)) { note_timeout(&s_timeout, 0x7ffffffe); break; }
+                if (t < 0) break;
+                const UmmaTile tile = tiles[t];
+                const UmmaProblem *P = ((EPI == EPI_RUNTIME && tile.kind) ? probs2 : probs) + tile.prob;
+                if (EPI == EPI_RUNTIME && tile.kind && tile.wait_slot >= 0) {
+                    if (!counter_wait(counters + tile.wait_slot, tile.wait_count, budget)) { note_timeout(&s_timeout, t); break; }
+                    asm volatile("fence.proxy.async;" ::: "memory");
+                }
+                if (P->starve) { note_timeout(&s_timeout, t); break; }
+                int n_eff = P->N - tile.n0;
+                n_eff = tile.nw > 0 ? tile.nw : (n_eff >= BN ? BN : ((n_eff + 15) & ~15));
+                const int b_row = tile.n0 + (int)rank * (n_eff / 2);   // this CTA's half of the B rows
+                const bool b_mn = PLANES == 1 && P->b_mn;
+                const int b_plane_rows = P->plane_rows;
+                const CUtensorMap *tmB = &P->tmB;
+                auto k_loop = [&](auto mn_any) {
+                    constexpr bool MN = decltype(mn_any)::value;
+                    for (int kb = tile.kb0; kb < tile.kb1; ++kb) {
+                        if (!mbar_wait(smem_u32(bar_empty + p_stage), p_phase ^ 1u, budget)) { note_timeout(&s_timeout, t); ok = false; break; }
+                        const uint32_t full = leader_addr(smem_u32(bar_full + p_stage));
+                        const uint32_t st = smem_u32(smem + p_stage * SM::STAGE_BYTES) + SM::A_PLANES * SM::A_BYTES;
+                        const int kx = kb * SM::BK_ELEMS;
+                        if (MN) {
                             // B = a row-major [K x N] matrix: boxes of 64 columns x 64 rows, this CTA's half of the columns
 #pragma unroll
-                            for (int j = 0; j < BN / 128; ++j) tma_load_2d_pair(st + SM::A_BYTES + j * 8192, tmB, full, b_row + 64 * j, kx);
+                            for (int j = 0; j < BN / 128; ++j) tma_load_2d_pair(st + j * 8192, tmB, full, b_row + 64 * j, kx);
                         } else {
 #pragma unroll
                             for (int pl = 0; pl < SM::B_PLANES; ++pl)
-                                tma_load_2d_pair(st + SM::A_PLANES * SM::A_BYTES + pl * SM::B_BYTES, tmB, full, kx, b_row + pl * b_plane_rows);
+                                tma_load_2d_pair(st + pl * SM::B_BYTES, tmB, full, kx, b_row + pl * b_plane_rows);
                         }
                         if (++p_stage == STAGES) { p_stage = 0; p_phase ^= 1u; }
                     }
                 };
-                if (a_mn || b_mn) k_loop(std::true_type{});
+                if (b_mn) k_loop(std::true_type{});
                 else k_loop(std::false_type{});
             }
         }
