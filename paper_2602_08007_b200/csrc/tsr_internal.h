@@ -141,7 +141,6 @@ cudaError_t core_update_launch(const CoreUpdateArgs *args_dev, const int32_t *li
 cudaError_t make_shadows(const float *X, int rows, int r, bf16 *Xb, int64_t ldb, bf16 *Xbt, int64_t ldt,
                          cudaStream_t stream);
 // out[cols x ldo] = in[rows x ldi]^T (BF16)
-cudaError_t transpose_bf16(const bf16 *in, int rows, int cols, int64_t ldi, bf16 *out, int64_t ldo, cudaStream_t stream);
 // X (rows x k FP32) -> planes hi / lo of X^T: out[plane][k x ldo]; plane stride = plane_rows * ldo elements.
 cudaError_t split_transpose(const float *X, int rows, int k, bf16 *out, int64_t ldo, int plane_rows, int planes,
                             cudaStream_t stream);

@@ -382,45 +382,6 @@ cudaError_t make_shadows(const float *X, int rows, int r, bf16 *Xb, int64_t ldb,
     return cudaGetLastError();
 }
 
-// out[cols x ldo] = in[rows x ldi]^T.  Tiles of 64 x 64, read and written as pairs of BF16.
-__global__ void transpose_bf16_kernel(const bf16 *__restrict__ in, int rows, int cols, int64_t ldi,
-                                      bf16 *__restrict__ out, int64_t ldo, int in_pairs)
-{
-    __shared__ bf16 tile[64][66];
-    const int r0 = blockIdx.y * 64, c0 = blockIdx.x * 64;
-    for (int i = threadIdx.y; i < 64; i += blockDim.y) {
-        const int row = r0 + i, col = c0 + 2 * threadIdx.x;
-        uint32_t w = 0;
-        if (row < rows && col < cols) {
-            const bf16 *src = in + (int64_t)row * ldi + col;
-            if (in_pairs && col + 1 < cols) w = *(const uint32_t *)src;
-            else {
-                const bf16 a = src[0], bq = (col + 1 < cols) ? src[1] : __float2bfloat16_rn(0.f);
-                w = (uint32_t)(*(const uint16_t *)&a) | ((uint32_t)(*(const uint16_t *)&bq) << 16);
-            }
-        }
-        *(uint32_t *)&tile[i][2 * threadIdx.x] = w;
-    }
-    __syncthreads();
-    for (int i = threadIdx.y; i < 64; i += blockDim.y) {
-        const int col = c0 + i, row = r0 + 2 * threadIdx.x;
-        if (col >= cols || row >= rows) continue;
-        bf16 *dst = out + (int64_t)col * ldo + row;
-        const bf16 a = tile[2 * threadIdx.x][i], bq = tile[2 * threadIdx.x + 1][i];
-        if (row + 1 < rows) *(uint32_t *)dst = (uint32_t)(*(const uint16_t *)&a) | ((uint32_t)(*(const uint16_t *)&bq) << 16);
-        else *dst = a;
-    }
-}
-
-cudaError_t transpose_bf16(const bf16 *in, int rows, int cols, int64_t ldi, bf16 *out, int64_t ldo, cudaStream_t stream)
-{
-    dim3 grid((cols + 63) / 64, (rows + 63) / 64);
-    // 32-bit loads need an even row pitch and a 4-byte aligned base; the output side always has them
-    const int in_pairs = ((ldi & 1) == 0 && (((uintptr_t)in) & 3) == 0) ? 1 : 0;
-    transpose_bf16_kernel<<<grid, dim3(32, 8), 0, stream>>>(in, rows, cols, ldi, out, ldo, in_pairs);
-    return cudaGetLastError();
-}
-
 // X (rows x k) FP32 -> X^T as BF16 planes: hi = bf16(x), lo = bf16(x - hi).
 __global__ void split_transpose_kernel(const float *__restrict__ X, int rows, int k, bf16 *__restrict__ out,
                                        int64_t ldo, int plane_rows, int planes)
